@@ -1,0 +1,218 @@
+"""CPU oracle for the KV block save/restore path -- TEST INFRASTRUCTURE ONLY.
+
+Thin ctypes wrapper over ``gk_oracle.c`` (plain C, compiled with gcc).  The
+oracle defines what pack / restore must produce, byte for byte; see the header
+of ``gk_oracle.h`` for the passages of the paper it follows (Section 2.2 for
+save, load, check-on-load and the recompute-on-any-failure rule; Table 1 for
+bit-identical restoration).  It imports nothing from the CUDA package and the
+CUDA package imports nothing from here.  Only tests, the smoke check and the
+benchmark's CPU-baseline leg may use it.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libgk_oracle.so")
+_SRC = os.path.join(_HERE, "gk_oracle.c")
+_HDR = os.path.join(_HERE, "gk_oracle.h")
+
+CODE_OK, CODE_CHECKSUM, CODE_PAGE_TABLE, CODE_MISSING = 0, 1, 2, 3
+FLAG_SKIP_VERIFY = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc if the shared object is missing or stale."""
+    stale = (not os.path.exists(_LIB_PATH)
+             or os.path.getmtime(_LIB_PATH) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR)))
+    if force or stale:
+        tmp = _LIB_PATH + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-fPIC", "-shared",
+                               "-o", tmp, _SRC])
+        os.replace(tmp, _LIB_PATH)
+    return _LIB_PATH
+
+
+class _CGeom(ctypes.Structure):
+    _fields_ = [("layers", ctypes.c_uint32), ("kv_heads", ctypes.c_uint32),
+                ("head_dim", ctypes.c_uint32), ("page_tokens", ctypes.c_uint32),
+                ("elem_bytes", ctypes.c_uint32), ("scale_kv", ctypes.c_uint32)]
+
+
+class _CCache(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("num_pages", ctypes.c_uint64),
+                ("layer_stride", ctypes.c_uint64), ("kv_stride", ctypes.c_uint64),
+                ("page_stride", ctypes.c_uint64), ("scales", ctypes.c_void_p),
+                ("s_layer_stride", ctypes.c_uint64), ("s_kv_stride", ctypes.c_uint64),
+                ("s_page_stride", ctypes.c_uint64)]
+
+
+class _CJob(ctypes.Structure):
+    _fields_ = [("blob", ctypes.c_void_p), ("checksums", ctypes.c_void_p),
+                ("page_table", ctypes.c_void_p), ("n_tokens", ctypes.c_uint32)]
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        L.ok_crc64_bitwise.restype = ctypes.c_uint64
+        L.ok_crc64_bitwise.argtypes = [ctypes.c_void_p, ctypes.c_size_t]
+        L.ok_crc64.restype = ctypes.c_uint64
+        L.ok_crc64.argtypes = [ctypes.c_void_p, ctypes.c_size_t]
+        L.ok_crc64_continue.restype = ctypes.c_uint64
+        L.ok_crc64_continue.argtypes = [ctypes.c_uint64, ctypes.c_void_p, ctypes.c_size_t]
+        L.ok_blob_size.restype = ctypes.c_int
+        L.ok_blob_size.argtypes = [ctypes.POINTER(_CGeom), ctypes.c_uint32,
+                                   ctypes.POINTER(ctypes.c_uint64), ctypes.POINTER(ctypes.c_uint32)]
+        L.ok_record_bytes.restype = ctypes.c_uint64
+        L.ok_record_bytes.argtypes = [ctypes.POINTER(_CGeom), ctypes.c_uint32, ctypes.c_uint32]
+        L.ok_record_offset.restype = ctypes.c_uint64
+        L.ok_record_offset.argtypes = [ctypes.POINTER(_CGeom), ctypes.c_uint32]
+        L.ok_pack.restype = ctypes.c_int
+        L.ok_pack.argtypes = [ctypes.POINTER(_CGeom), ctypes.POINTER(_CCache), ctypes.c_void_p,
+                              ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p,
+                              ctypes.POINTER(ctypes.c_int32)]
+        L.ok_restore.restype = None
+        L.ok_restore.argtypes = [ctypes.POINTER(_CGeom), ctypes.POINTER(_CCache),
+                                 ctypes.POINTER(_CJob), ctypes.c_uint32, ctypes.c_uint32,
+                                 ctypes.c_void_p, ctypes.c_void_p]
+        _lib = L
+    return _lib
+
+
+def _as_u8(data) -> np.ndarray:
+    if isinstance(data, (bytes, bytearray, memoryview)):
+        return np.frombuffer(bytes(data), dtype=np.uint8)
+    arr = np.ascontiguousarray(data)
+    return arr.view(np.uint8).reshape(-1)
+
+
+def crc64_bitwise(data) -> int:
+    a = _as_u8(data)
+    return int(lib().ok_crc64_bitwise(a.ctypes.data, a.size))
+
+
+def crc64(data) -> int:
+    a = _as_u8(data)
+    return int(lib().ok_crc64(a.ctypes.data, a.size))
+
+
+def crc64_continue(crc_so_far: int, data) -> int:
+    a = _as_u8(data)
+    return int(lib().ok_crc64_continue(ctypes.c_uint64(crc_so_far), a.ctypes.data, a.size))
+
+
+@dataclass(frozen=True)
+class Geom:
+    """Cache geometry as the oracle sees it (element size in bytes, not a dtype tag)."""
+    layers: int
+    kv_heads: int
+    head_dim: int
+    page_tokens: int
+    elem_bytes: int = 2
+    scale_kv: int = 0
+
+    def c(self) -> _CGeom:
+        return _CGeom(self.layers, self.kv_heads, self.head_dim, self.page_tokens,
+                      self.elem_bytes, self.scale_kv)
+
+
+@dataclass
+class Cache:
+    """A paged cache held in host memory as flat byte arrays plus byte strides."""
+    data: np.ndarray                  # uint8, flat
+    num_pages: int
+    layer_stride: int
+    kv_stride: int
+    page_stride: int
+    scales: Optional[np.ndarray] = None   # uint8, flat (fp32 values as bytes)
+    s_layer_stride: int = 0
+    s_kv_stride: int = 0
+    s_page_stride: int = 0
+
+    def c(self) -> _CCache:
+        assert self.data.dtype == np.uint8 and self.data.flags.c_contiguous
+        sp = 0
+        if self.scales is not None:
+            assert self.scales.dtype == np.uint8 and self.scales.flags.c_contiguous
+            sp = self.scales.ctypes.data
+        return _CCache(self.data.ctypes.data, self.num_pages, self.layer_stride, self.kv_stride,
+                       self.page_stride, sp, self.s_layer_stride, self.s_kv_stride,
+                       self.s_page_stride)
+
+
+def blob_size(g: Geom, n_tokens: int) -> tuple[int, int]:
+    nb, npg = ctypes.c_uint64(0), ctypes.c_uint32(0)
+    cg = g.c()
+    rc = lib().ok_blob_size(ctypes.byref(cg), n_tokens, ctypes.byref(nb), ctypes.byref(npg))
+    if rc != 0:
+        raise ValueError("bad geometry or n_tokens == 0")
+    return int(nb.value), int(npg.value)
+
+
+def record_bytes(g: Geom, n_tokens: int, p: int) -> int:
+    cg = g.c()
+    return int(lib().ok_record_bytes(ctypes.byref(cg), n_tokens, p))
+
+
+def record_offset(g: Geom, p: int) -> int:
+    cg = g.c()
+    return int(lib().ok_record_offset(ctypes.byref(cg), p))
+
+
+def pack(g: Geom, src: Cache, page_table, n_tokens: int):
+    """Returns (blob uint8[blob_bytes], checksums uint64[P], code, bad_index)."""
+    nbytes, npages = blob_size(g, n_tokens)
+    pt = np.ascontiguousarray(page_table, dtype=np.int32)
+    assert pt.size >= npages
+    blob = np.zeros(nbytes, dtype=np.uint8)
+    sums = np.zeros(npages, dtype=np.uint64)
+    bad = ctypes.c_int32(-1)
+    cg, cc = g.c(), src.c()
+    code = lib().ok_pack(ctypes.byref(cg), ctypes.byref(cc), pt.ctypes.data, n_tokens,
+                         blob.ctypes.data, sums.ctypes.data, ctypes.byref(bad))
+    return blob, sums, int(code), int(bad.value)
+
+
+@dataclass
+class Job:
+    blob: Optional[np.ndarray]        # uint8 flat, or None for a missing record
+    checksums: Optional[np.ndarray]   # uint64[P], or None
+    page_table: np.ndarray            # int32[P]
+    n_tokens: int
+
+
+def restore(g: Geom, dst: Cache, jobs: Sequence[Job], flags: int = 0):
+    """Mutates ``dst``; returns (mask uint8[n_jobs], first_bad int32[n_jobs])."""
+    n = len(jobs)
+    arr = (_CJob * max(n, 1))()
+    keep = []
+    for i, jb in enumerate(jobs):
+        pt = np.ascontiguousarray(jb.page_table, dtype=np.int32)
+        keep.append(pt)
+        bp = cp = 0
+        if jb.blob is not None:
+            b = jb.blob
+            assert b.dtype == np.uint8 and b.flags.c_contiguous
+            bp = b.ctypes.data
+        if jb.checksums is not None:
+            c = np.ascontiguousarray(jb.checksums, dtype=np.uint64)
+            keep.append(c)
+            cp = c.ctypes.data
+        arr[i] = _CJob(bp, cp, pt.ctypes.data, jb.n_tokens)
+    mask = np.zeros(n, dtype=np.uint8)
+    first_bad = np.zeros(n, dtype=np.int32)
+    cg, cc = g.c(), dst.c()
+    lib().ok_restore(ctypes.byref(cg), ctypes.byref(cc), arr, n, flags,
+                     mask.ctypes.data, first_bad.ctypes.data)
+    return mask, first_bad

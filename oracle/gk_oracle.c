@@ -1,0 +1,263 @@
+/*
+ * gk_oracle.c -- CPU oracle (test infrastructure only; see gk_oracle.h).
+ *
+ * Written for checking by eye: one loop nest per definition, no blocking, no
+ * threads, no SIMD.  Nothing here is shared with, or derived from, the CUDA
+ * path.
+ */
+#include "gk_oracle.h"
+
+#include <stdlib.h>
+#include <string.h>
+
+/* ------------------------------------------------------------------------
+ * CRC-64/XZ.  Catalogue parameters: width 64, polynomial 0x42F0E1EBA9EA3693,
+ * init all ones, input and output reflected, final xor all ones.  In the
+ * reflected formulation the register shifts right and the polynomial constant
+ * is the bit-reversed one.
+ * ---------------------------------------------------------------------- */
+#define OK_POLY_REFLECTED 0xC96C5795D7870F42ull
+
+static uint64_t crc_step_byte(uint64_t reg, uint8_t byte)
+{
+    reg ^= (uint64_t)byte;
+    for (int bit = 0; bit < 8; ++bit) {
+        if (reg & 1ull)
+            reg = (reg >> 1) ^ OK_POLY_REFLECTED;
+        else
+            reg = reg >> 1;
+    }
+    return reg;
+}
+
+uint64_t ok_crc64_bitwise(const uint8_t *data, size_t len)
+{
+    uint64_t reg = ~0ull;
+    for (size_t i = 0; i < len; ++i)
+        reg = crc_step_byte(reg, data[i]);
+    return ~reg;
+}
+
+static uint64_t g_table[256];
+static int g_table_ready = 0;
+
+static void table_init(void)
+{
+    /* entry b = the register after feeding byte b into an all-zero register */
+    for (int b = 0; b < 256; ++b)
+        g_table[b] = crc_step_byte(0ull, (uint8_t)b);
+    g_table_ready = 1;
+}
+
+uint64_t ok_crc64_continue(uint64_t crc_so_far, const uint8_t *data, size_t len)
+{
+    if (!g_table_ready)
+        table_init();
+    uint64_t reg = ~crc_so_far; /* undo the final xor to get the register back */
+    for (size_t i = 0; i < len; ++i)
+        reg = g_table[(uint8_t)(reg ^ data[i])] ^ (reg >> 8);
+    return ~reg;
+}
+
+uint64_t ok_crc64(const uint8_t *data, size_t len)
+{
+    /* the CRC of the empty string is 0, whose register is all ones = init */
+    return ok_crc64_continue(0ull, data, len);
+}
+
+/* ------------------------------------------------------------------------
+ * Geometry.
+ * ---------------------------------------------------------------------- */
+static uint64_t row_bytes(const ok_geom *g)
+{
+    return (uint64_t)g->kv_heads * g->head_dim * g->elem_bytes;
+}
+
+static uint64_t scale_section_bytes(const ok_geom *g)
+{
+    return (uint64_t)g->layers * g->scale_kv * g->kv_heads * 4u;
+}
+
+static uint32_t page_count(const ok_geom *g, uint32_t n_tokens)
+{
+    return (n_tokens + g->page_tokens - 1u) / g->page_tokens;
+}
+
+/* tokens held by logical page p of a block of n_tokens */
+static uint32_t tokens_in_page(const ok_geom *g, uint32_t n_tokens, uint32_t p)
+{
+    uint32_t P = page_count(g, n_tokens);
+    if (p + 1u < P)
+        return g->page_tokens;
+    return n_tokens - (P - 1u) * g->page_tokens;
+}
+
+uint64_t ok_record_bytes(const ok_geom *g, uint32_t n_tokens, uint32_t p)
+{
+    return scale_section_bytes(g) +
+           (uint64_t)tokens_in_page(g, n_tokens, p) * 2u * g->layers * row_bytes(g);
+}
+
+uint64_t ok_record_offset(const ok_geom *g, uint32_t p)
+{
+    /* every earlier page is full */
+    uint64_t full = scale_section_bytes(g) + (uint64_t)g->page_tokens * 2u * g->layers * row_bytes(g);
+    return (uint64_t)p * full;
+}
+
+int ok_blob_size(const ok_geom *g, uint32_t n_tokens, uint64_t *blob_bytes, uint32_t *n_pages)
+{
+    if (!g || n_tokens == 0 || g->page_tokens == 0)
+        return -1;
+    uint32_t P = page_count(g, n_tokens);
+    uint64_t total = 0;
+    for (uint32_t p = 0; p < P; ++p)
+        total += ok_record_bytes(g, n_tokens, p);
+    if (blob_bytes)
+        *blob_bytes = total;
+    if (n_pages)
+        *n_pages = P;
+    return 0;
+}
+
+static uint8_t *slab_ptr(const ok_cache *c, uint32_t l, uint32_t kv, int32_t page)
+{
+    return c->data + (uint64_t)l * c->layer_stride + (uint64_t)kv * c->kv_stride +
+           (uint64_t)page * c->page_stride;
+}
+
+static uint8_t *scale_ptr(const ok_cache *c, uint32_t l, uint32_t kv, int32_t page, uint32_t h)
+{
+    return c->scales + (uint64_t)l * c->s_layer_stride + (uint64_t)kv * c->s_kv_stride +
+           (uint64_t)page * c->s_page_stride + 4ull * h;
+}
+
+static int32_t lowest_out_of_range(const int32_t *pt, uint32_t P, uint64_t num_pages)
+{
+    for (uint32_t p = 0; p < P; ++p)
+        if (pt[p] < 0 || (uint64_t)pt[p] >= num_pages)
+            return (int32_t)p;
+    return -1;
+}
+
+/* ------------------------------------------------------------------------
+ * Save (pack).
+ * ---------------------------------------------------------------------- */
+int ok_pack(const ok_geom *g, const ok_cache *src, const int32_t *page_table,
+            uint32_t n_tokens, uint8_t *blob, uint64_t *checksums, int32_t *bad_index)
+{
+    uint32_t P = page_count(g, n_tokens);
+    uint64_t row = row_bytes(g);
+    int32_t bad = lowest_out_of_range(page_table, P, src->num_pages);
+    if (bad_index)
+        *bad_index = bad;
+    if (bad >= 0)
+        return OK_CODE_PAGE_TABLE;
+
+    for (uint32_t p = 0; p < P; ++p) {
+        uint8_t *rec = blob + ok_record_offset(g, p);
+        uint8_t *w = rec;
+        int32_t page = page_table[p];
+        uint64_t prefix = (uint64_t)tokens_in_page(g, n_tokens, p) * row;
+
+        for (uint32_t l = 0; l < g->layers; ++l)
+            for (uint32_t kv = 0; kv < g->scale_kv; ++kv)
+                for (uint32_t h = 0; h < g->kv_heads; ++h) {
+                    memcpy(w, scale_ptr(src, l, kv, page, h), 4);
+                    w += 4;
+                }
+        for (uint32_t l = 0; l < g->layers; ++l)
+            for (uint32_t kv = 0; kv < 2; ++kv) {
+                memcpy(w, slab_ptr(src, l, kv, page), prefix);
+                w += prefix;
+            }
+        checksums[p] = ok_crc64(rec, (size_t)(w - rec));
+    }
+    return OK_CODE_OK;
+}
+
+/* ------------------------------------------------------------------------
+ * Load (restore): verify everything, then commit what passed.
+ * ---------------------------------------------------------------------- */
+void ok_restore(const ok_geom *g, const ok_cache *dst, const ok_job *jobs, uint32_t n_jobs,
+                uint32_t flags, uint8_t *mask, int32_t *first_bad)
+{
+    uint64_t row = row_bytes(g);
+    uint32_t *claims = (uint32_t *)calloc(dst->num_pages ? dst->num_pages : 1, sizeof(uint32_t));
+
+    /* ---- phase 1a: missing records, ids out of range ---- */
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        const ok_job *job = &jobs[j];
+        mask[j] = OK_CODE_OK;
+        first_bad[j] = -1;
+        if (job->blob == NULL || job->checksums == NULL) {
+            mask[j] = OK_CODE_MISSING;
+            continue;
+        }
+        int32_t bad = lowest_out_of_range(job->page_table, page_count(g, job->n_tokens), dst->num_pages);
+        if (bad >= 0) {
+            mask[j] = OK_CODE_PAGE_TABLE;
+            first_bad[j] = bad;
+        }
+    }
+    /* ---- phase 1b: a destination page may be claimed once per call ---- */
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        if (mask[j] != OK_CODE_OK)
+            continue;
+        uint32_t P = page_count(g, jobs[j].n_tokens);
+        for (uint32_t p = 0; p < P; ++p)
+            claims[jobs[j].page_table[p]] += 1u;
+    }
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        if (mask[j] != OK_CODE_OK)
+            continue;
+        uint32_t P = page_count(g, jobs[j].n_tokens);
+        for (uint32_t p = 0; p < P; ++p)
+            if (claims[jobs[j].page_table[p]] > 1u) {
+                mask[j] = OK_CODE_PAGE_TABLE;
+                first_bad[j] = (int32_t)p;
+                break;
+            }
+    }
+    /* ---- phase 1c: every page record against its stored checksum ---- */
+    if (!(flags & OK_FLAG_SKIP_VERIFY)) {
+        for (uint32_t j = 0; j < n_jobs; ++j) {
+            if (mask[j] != OK_CODE_OK)
+                continue;
+            uint32_t P = page_count(g, jobs[j].n_tokens);
+            for (uint32_t p = 0; p < P; ++p) {
+                const uint8_t *rec = jobs[j].blob + ok_record_offset(g, p);
+                uint64_t crc = ok_crc64(rec, (size_t)ok_record_bytes(g, jobs[j].n_tokens, p));
+                if (crc != jobs[j].checksums[p]) {
+                    mask[j] = OK_CODE_CHECKSUM;
+                    first_bad[j] = (int32_t)p;
+                    break;
+                }
+            }
+        }
+    }
+    /* ---- phase 2: commit the jobs that passed; nothing else is written ---- */
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        if (mask[j] != OK_CODE_OK)
+            continue;
+        uint32_t P = page_count(g, jobs[j].n_tokens);
+        for (uint32_t p = 0; p < P; ++p) {
+            const uint8_t *r = jobs[j].blob + ok_record_offset(g, p);
+            int32_t page = jobs[j].page_table[p];
+            uint64_t prefix = (uint64_t)tokens_in_page(g, jobs[j].n_tokens, p) * row;
+
+            for (uint32_t l = 0; l < g->layers; ++l)
+                for (uint32_t kv = 0; kv < g->scale_kv; ++kv)
+                    for (uint32_t h = 0; h < g->kv_heads; ++h) {
+                        memcpy(scale_ptr(dst, l, kv, page, h), r, 4);
+                        r += 4;
+                    }
+            for (uint32_t l = 0; l < g->layers; ++l)
+                for (uint32_t kv = 0; kv < 2; ++kv) {
+                    memcpy(slab_ptr(dst, l, kv, page), r, prefix);
+                    r += prefix;
+                }
+        }
+    }
+    free(claims);
+}

@@ -1,0 +1,108 @@
+/*
+ * gk_oracle.h -- CPU oracle for the save/restore path of a block's KV state.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This is the slow, plain definition that the CUDA
+ * library is compared against.  It shares no source, header, table or helper
+ * with the CUDA path; only tests, the smoke check and the benchmark's CPU
+ * baseline may call it.
+ *
+ * What it follows (paper, Section 2.2 "Taliesin: KV memory"): the KV state of a
+ * block of prompt text is written to storage after it is computed, loaded again
+ * when the same block recurs, checked on load, and -- the design rule "serve
+ * without memory, never with wrong memory" -- any record that is missing,
+ * damaged or fails a check is not used: the block is recomputed.  Section 3
+ * (Table 1) demands that what is restored is bit-identical to what was saved;
+ * Section 5 states that reuse is at whole-block granularity and that the design
+ * is fail-closed.  The paper withholds its storage format (end of Section 1),
+ * so the page-record layout, the checksum (CRC-64/XZ per page record) and the
+ * result codes below are this build's own definitions.
+ *
+ * Layout definitions
+ *   cache   : opaque bytes.  The slab of (layer l, kv, page g) starts at
+ *             data + l*layer_stride + kv*kv_stride + g*page_stride and holds
+ *             page_tokens rows of row = kv_heads*head_dim*elem_bytes bytes,
+ *             token-major.  kv = 0 is K, kv = 1 is V.
+ *   scales  : (fp8 caches only) fp32 per (l, kv < scale_kv, page g, head h) at
+ *             scales + l*s_layer_stride + kv*s_kv_stride + g*s_page_stride + 4*h.
+ *   blob    : page records 0..P-1 back to back, no header, no padding.  Record
+ *             p = [scale section: for l, for kv < scale_kv, for h: 4 bytes]
+ *             then for l: K prefix (t_p*row bytes), V prefix (t_p*row bytes),
+ *             where t_p = page_tokens except for a shorter last page.
+ *   checksum: CRC-64/XZ over the bytes of record p, one uint64 per page.
+ *
+ * All pins for these functions are listed in tests/test_oracle_pins.py.
+ */
+#ifndef GK_ORACLE_H
+#define GK_ORACLE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct {
+    uint32_t layers;
+    uint32_t kv_heads;
+    uint32_t head_dim;
+    uint32_t page_tokens;
+    uint32_t elem_bytes; /* 2 for bf16, 1 for fp8 e4m3 */
+    uint32_t scale_kv;   /* 0: no scale section; 1: one scale per (l,page,h); 2: K and V scales */
+} ok_geom;
+
+typedef struct {
+    uint8_t *data;
+    uint64_t num_pages;
+    uint64_t layer_stride, kv_stride, page_stride; /* bytes */
+    uint8_t *scales; /* NULL when scale_kv == 0 */
+    uint64_t s_layer_stride, s_kv_stride, s_page_stride; /* bytes */
+} ok_cache;
+
+typedef struct {
+    const uint8_t *blob;       /* NULL: the record is missing */
+    const uint64_t *checksums; /* NULL: the record is missing */
+    const int32_t *page_table; /* P logical -> physical page ids */
+    uint32_t n_tokens;
+} ok_job;
+
+/* result codes per job */
+enum {
+    OK_CODE_OK = 0,        /* verified and committed */
+    OK_CODE_CHECKSUM = 1,  /* some page record failed its checksum */
+    OK_CODE_PAGE_TABLE = 2,/* id out of range, or a page claimed twice in the call */
+    OK_CODE_MISSING = 3    /* no record */
+};
+
+#define OK_FLAG_SKIP_VERIFY 1u /* sabotage tests: switch the checksum defence off */
+
+/* CRC-64/XZ by its bit-at-a-time definition. */
+uint64_t ok_crc64_bitwise(const uint8_t *data, size_t len);
+/* Same value, one table lookup per byte; the table is generated from the
+ * bit-at-a-time step on first use. */
+uint64_t ok_crc64(const uint8_t *data, size_t len);
+/* Continue a CRC: ok_crc64_continue(ok_crc64(A), B) == ok_crc64(A || B). */
+uint64_t ok_crc64_continue(uint64_t crc_so_far, const uint8_t *data, size_t len);
+
+/* Sizes of a block of n_tokens: pages P = ceil(n/T), blob bytes = P*S + n*tokB. */
+int ok_blob_size(const ok_geom *g, uint32_t n_tokens, uint64_t *blob_bytes, uint32_t *n_pages);
+/* Bytes of page record p of a block of n_tokens, and its offset in the blob. */
+uint64_t ok_record_bytes(const ok_geom *g, uint32_t n_tokens, uint32_t p);
+uint64_t ok_record_offset(const ok_geom *g, uint32_t p);
+
+/* Save: gather the block's pages into blob and checksum each record.
+ * Returns OK_CODE_OK, or OK_CODE_PAGE_TABLE (nothing written) if an id is
+ * outside [0, num_pages); *bad_index then holds the lowest offending index. */
+int ok_pack(const ok_geom *g, const ok_cache *src, const int32_t *page_table,
+            uint32_t n_tokens, uint8_t *blob, uint64_t *checksums, int32_t *bad_index);
+
+/* Load: phase 1 validates and verifies every job without writing; phase 2
+ * commits the jobs whose code is 0.  mask[j] gets the code, first_bad[j] the
+ * lowest failing page index (codes 1, 2) or -1. */
+void ok_restore(const ok_geom *g, const ok_cache *dst, const ok_job *jobs, uint32_t n_jobs,
+                uint32_t flags, uint8_t *mask, int32_t *first_bad);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

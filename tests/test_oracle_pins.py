@@ -1,0 +1,418 @@
+"""Pins for the CPU oracle: everything here checks the oracle against something
+other than itself -- catalogue values, a library routine (stdlib lzma), long
+division of polynomials written independently in Python, closed forms, textbook
+special cases (memcpy), invariants and brute force on tiny inputs."""
+import lzma
+import os
+import struct
+
+import numpy as np
+import pytest
+
+import oracle
+import synth
+from helpers import (cache_bytes, clone_cache, make_cache, n_pages, oracle_geom, random_cache,
+                     slab_bytes)
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+# --------------------------------------------------------------------------
+# CRC-64/XZ
+# --------------------------------------------------------------------------
+def _golden_vectors():
+    out = []
+    with open(os.path.join(GOLDEN, "crc64_xz_vectors.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            msg, crc = line.split()
+            out.append((b"" if msg == "-" else bytes.fromhex(msg), int(crc, 16)))
+    return out
+
+
+def test_crc_catalogue_vectors():
+    vecs = _golden_vectors()
+    assert (b"123456789", 0x995DC9BBDF1939FA) in vecs
+    for msg, crc in vecs:
+        assert oracle.crc64_bitwise(msg) == crc
+        assert oracle.crc64(msg) == crc
+
+
+def _crc_by_long_division(msg: bytes) -> int:
+    """CRC-64/XZ from the polynomial definition: message bits (least significant
+    bit of each byte first) are the coefficients, highest degree first; the
+    register is (M*x^64 + ones*x^n) mod P, xored with ones, bit-reversed."""
+    P = (1 << 64) | 0x42F0E1EBA9EA3693
+    n = 8 * len(msg)
+    M = 0
+    for i, b in enumerate(msg):
+        for k in range(8):
+            if (b >> k) & 1:
+                M |= 1 << (n - 1 - (8 * i + k))
+    ones = (1 << 64) - 1
+    V = (M << 64) ^ (ones << n)
+    for d in range(V.bit_length() - 1, 63, -1):
+        if (V >> d) & 1:
+            V ^= P << (d - 64)
+    V ^= ones
+    return int(format(V, "064b")[::-1], 2)
+
+
+def test_crc_against_polynomial_long_division():
+    rng = np.random.default_rng(1)
+    for n in [0, 1, 2, 7, 8, 9, 63, 64, 65, 200, 1000]:
+        msg = rng.integers(0, 256, size=n, dtype=np.uint8).tobytes()
+        assert oracle.crc64(msg) == _crc_by_long_division(msg)
+    assert _crc_by_long_division(b"\x00") == 0x1FADA17364673F59
+
+
+def _crc_from_xz_container(data: bytes) -> int:
+    """The CRC-64 that liblzma stores for a one-block .xz stream."""
+    x = lzma.compress(data, format=lzma.FORMAT_XZ, check=lzma.CHECK_CRC64)
+    backward = struct.unpack("<I", x[-8:-4])[0]
+    end = len(x) - 12 - 4 * (backward + 1)
+    return int.from_bytes(x[end - 8:end], "little")
+
+
+def test_crc_against_liblzma():
+    rng = np.random.default_rng(2)
+    for n in [1, 3, 16, 255, 256, 257, 4096, 16384, 100003]:
+        msg = rng.integers(0, 256, size=n, dtype=np.uint8).tobytes()
+        want = _crc_from_xz_container(msg)
+        assert oracle.crc64(msg) == want
+        assert oracle.crc64_bitwise(msg) == want
+
+
+def test_crc_table_equals_bitwise_and_streams():
+    rng = np.random.default_rng(3)
+    for n in [0, 1, 5, 64, 1023, 70001]:
+        msg = rng.integers(0, 256, size=n, dtype=np.uint8)
+        full = oracle.crc64_bitwise(msg)
+        assert oracle.crc64(msg) == full
+        for cut in {0, n // 3, n // 2, n}:
+            assert oracle.crc64_continue(oracle.crc64(msg[:cut]), msg[cut:]) == full
+
+
+def test_crc_residue():
+    rng = np.random.default_rng(4)
+    for n in [0, 1, 17, 4096]:
+        msg = rng.integers(0, 256, size=n, dtype=np.uint8).tobytes()
+        tail = oracle.crc64(msg).to_bytes(8, "little")
+        # register residue 0x49958C9ABD7D353F, i.e. CRC value = its complement
+        assert oracle.crc64(msg + tail) == 0x49958C9ABD7D353F ^ 0xFFFFFFFFFFFFFFFF
+
+
+def test_crc_affine_law():
+    """crc(a^b) ^ crc(a) ^ crc(b) == crc(zeros) for equal lengths."""
+    rng = np.random.default_rng(5)
+    for n in [1, 8, 333, 4096]:
+        a = rng.integers(0, 256, size=n, dtype=np.uint8)
+        b = rng.integers(0, 256, size=n, dtype=np.uint8)
+        z = np.zeros(n, dtype=np.uint8)
+        assert oracle.crc64(a ^ b) ^ oracle.crc64(a) ^ oracle.crc64(b) == oracle.crc64(z)
+
+
+def test_crc_detects_every_single_bit_flip_of_a_tiny_record():
+    """Exhaustive over a 16 KiB record (131,072 bits) and over the checksum word."""
+    rng = np.random.default_rng(6)
+    rec = rng.integers(0, 256, size=16384, dtype=np.uint8)
+    good = oracle.crc64(rec)
+    seen = set()
+    for byte in range(rec.size):
+        for bit in range(8):
+            rec[byte] ^= 1 << bit
+            c = oracle.crc64(rec)
+            rec[byte] ^= 1 << bit
+            assert c != good
+            seen.add(c)
+    assert len(seen) == rec.size * 8          # all syndromes distinct as well
+    for bit in range(64):
+        assert (good ^ (1 << bit)) != good
+
+
+def test_crc_detects_every_double_bit_flip_of_a_64_byte_record():
+    rng = np.random.default_rng(7)
+    rec = rng.integers(0, 256, size=64, dtype=np.uint8)
+    good = oracle.crc64(rec)
+    nb = rec.size * 8
+    for i in range(nb):
+        rec[i >> 3] ^= 1 << (i & 7)
+        for j in range(i + 1, nb):
+            rec[j >> 3] ^= 1 << (j & 7)
+            assert oracle.crc64(rec) != good
+            rec[j >> 3] ^= 1 << (j & 7)
+        rec[i >> 3] ^= 1 << (i & 7)
+
+
+# --------------------------------------------------------------------------
+# Sizes: closed form blob_bytes = P*S + n*tokB, and the workloads' figures
+# --------------------------------------------------------------------------
+@pytest.mark.parametrize("w,n,want_bytes,want_pages", [
+    (synth.TINY, 256, 256 * 1024, 16),
+    (synth.GQA7B, 4096, 512 << 20, 256),
+    (synth.CORPUS, 1024, 64 * (3 << 20), 64),
+    (synth.CORPUS, 280, 17 * (3 << 20) + 8 * 192 * 1024, 18),
+    (synth.FP8, 2048, 64 * 7872000, 64),
+    (synth.STRESS, 17, 768 * 1024 + 48 * 1024, 2),
+])
+def test_blob_size_closed_form(w, n, want_bytes, want_pages):
+    g = oracle_geom(w)
+    nbytes, P = oracle.blob_size(g, n)
+    S = g.layers * g.scale_kv * g.kv_heads * 4
+    tokB = 2 * g.layers * g.kv_heads * g.head_dim * g.elem_bytes
+    assert P == -(-n // g.page_tokens) == want_pages
+    assert nbytes == P * S + n * tokB == want_bytes
+    assert sum(oracle.record_bytes(g, n, p) for p in range(P)) == nbytes
+    assert oracle.record_offset(g, P - 1) + oracle.record_bytes(g, n, P - 1) == nbytes
+
+
+def test_corpus_total_bytes():
+    g = oracle_geom(synth.CORPUS)
+    total = sum(oracle.blob_size(g, n)[0] for n in synth.CORPUS_BLOCKS)
+    pages = sum(oracle.blob_size(g, n)[1] for n in synth.CORPUS_BLOCKS)
+    assert total == 19_181_076_480 and pages == 6098
+
+
+# --------------------------------------------------------------------------
+# pack
+# --------------------------------------------------------------------------
+SMALL = oracle.Geom(layers=3, kv_heads=2, head_dim=8, page_tokens=4, elem_bytes=2, scale_kv=0)
+SMALL_FP8 = oracle.Geom(layers=3, kv_heads=4, head_dim=8, page_tokens=4, elem_bytes=1, scale_kv=2)
+
+
+def test_pack_identity_table_page_major_is_memcpy():
+    g, N = SMALL, 7
+    src = random_cache(g, N, seed=10, layout="page_major")
+    blob, sums, code, bad = oracle.pack(g, src, np.arange(N), N * g.page_tokens)
+    assert code == 0 and bad == -1
+    assert np.array_equal(blob, src.data)
+    rec = 2 * g.layers * slab_bytes(g)
+    for p in range(N):
+        assert int(sums[p]) == _crc_from_xz_container(src.data[p * rec:(p + 1) * rec].tobytes())
+
+
+def _pack_by_numpy_indexing(g, src, pt, n_tokens, layer_major_pages):
+    """Independent statement of the record layout with numpy views."""
+    L, H, D, T, E = g.layers, g.kv_heads, g.head_dim, g.page_tokens, g.elem_bytes
+    arr = src.data.reshape(L, 2, layer_major_pages, T, H * D * E)
+    sc = None if src.scales is None else src.scales.reshape(L, g.scale_kv, layer_major_pages, H * 4)
+    out = []
+    for p in range(n_pages(g, n_tokens)):
+        t = min(T, n_tokens - p * T)
+        if sc is not None:
+            out.append(sc[:, :, pt[p], :].reshape(-1))
+        out.append(arr[:, :, pt[p], :t, :].reshape(-1))
+    return np.concatenate(out)
+
+
+@pytest.mark.parametrize("g", [SMALL, SMALL_FP8])
+@pytest.mark.parametrize("n_tokens", [1, 4, 5, 17, 20])
+def test_pack_layout_against_numpy_views(g, n_tokens):
+    N = 11
+    src = random_cache(g, N, seed=11)
+    pt = np.random.default_rng(12).permutation(N).astype(np.int32)
+    blob, sums, code, _ = oracle.pack(g, src, pt, n_tokens)
+    assert code == 0
+    want = _pack_by_numpy_indexing(g, src, pt, n_tokens, N)
+    assert np.array_equal(blob, want)
+    for p in range(n_pages(g, n_tokens)):
+        lo = oracle.record_offset(g, p)
+        hi = lo + oracle.record_bytes(g, n_tokens, p)
+        assert int(sums[p]) == _crc_by_long_division(blob[lo:hi].tobytes())
+
+
+def test_pack_is_a_permutation_of_the_valid_bytes():
+    g, N = SMALL, 9
+    src = random_cache(g, N, seed=13)
+    pt = np.array([8, 0, 3], dtype=np.int32)
+    n = 2 * g.page_tokens + 1
+    blob, _, _, _ = oracle.pack(g, src, pt, n)
+    arr = src.data.reshape(g.layers, 2, N, g.page_tokens, -1)
+    valid = np.concatenate([arr[:, :, 8].reshape(-1), arr[:, :, 0].reshape(-1),
+                            arr[:, :, 3, :1].reshape(-1)])
+    assert np.array_equal(np.sort(blob), np.sort(valid))
+
+
+def test_pack_duplicates_allowed_out_of_range_rejected():
+    g, N = SMALL, 4
+    src = random_cache(g, N, seed=14)
+    blob, sums, code, bad = oracle.pack(g, src, np.array([1, 1], dtype=np.int32), 8)
+    assert code == 0 and np.array_equal(blob[:blob.size // 2], blob[blob.size // 2:])
+    for bad_id in (-1, N):
+        blob, sums, code, bad = oracle.pack(g, src, np.array([0, bad_id, 2], dtype=np.int32), 12)
+        assert code == oracle.CODE_PAGE_TABLE and bad == 1
+        assert not blob.any() and not sums.any()
+
+
+# --------------------------------------------------------------------------
+# restore: round trip, fail-closed, codes
+# --------------------------------------------------------------------------
+def _sentinel_cache(g, N, seed):
+    return random_cache(g, N, seed)
+
+
+@pytest.mark.parametrize("g", [SMALL, SMALL_FP8])
+@pytest.mark.parametrize("n_tokens", [3, 4, 9, 16])
+def test_round_trip_and_untouched_rest(g, n_tokens):
+    Ns, Nd = 6, 10
+    src = random_cache(g, Ns, seed=20)
+    P = n_pages(g, n_tokens)
+    spt = np.random.default_rng(21).permutation(Ns).astype(np.int32)[:P]
+    blob, sums, _, _ = oracle.pack(g, src, spt, n_tokens)
+    dst = _sentinel_cache(g, Nd, seed=22)
+    before = clone_cache(dst)
+    dpt = np.random.default_rng(23).permutation(Nd).astype(np.int32)[:P]
+    mask, fb = oracle.restore(g, dst, [oracle.Job(blob, sums, dpt, n_tokens)])
+    assert mask.tolist() == [0] and fb.tolist() == [-1]
+    L, T = g.layers, g.page_tokens
+    s = src.data.reshape(L, 2, Ns, T, -1)
+    d = dst.data.reshape(L, 2, Nd, T, -1)
+    b = before.data.reshape(L, 2, Nd, T, -1)
+    touched = np.zeros(Nd, dtype=bool)
+    for p in range(P):
+        t = min(T, n_tokens - p * T)
+        assert np.array_equal(d[:, :, dpt[p], :t], s[:, :, spt[p], :t])      # restored == saved
+        assert np.array_equal(d[:, :, dpt[p], t:], b[:, :, dpt[p], t:])      # tail of a partial page
+        touched[dpt[p]] = True
+    assert np.array_equal(d[:, :, ~touched], b[:, :, ~touched])              # unmapped pages
+    if g.scale_kv:
+        ss = src.scales.reshape(L, g.scale_kv, Ns, -1)
+        ds = dst.scales.reshape(L, g.scale_kv, Nd, -1)
+        bs = before.scales.reshape(L, g.scale_kv, Nd, -1)
+        for p in range(P):
+            assert np.array_equal(ds[:, :, dpt[p]], ss[:, :, spt[p]])
+        assert np.array_equal(ds[:, :, ~touched], bs[:, :, ~touched])
+    # a second pack from the destination reproduces the record bytes and checksums
+    blob2, sums2, _, _ = oracle.pack(g, dst, dpt, n_tokens)
+    assert np.array_equal(blob2, blob) and np.array_equal(sums2, sums)
+
+
+@pytest.mark.parametrize("g", [oracle.Geom(1, 1, 8, 2, 2, 0), oracle.Geom(1, 2, 4, 2, 1, 2)])
+def test_every_single_bit_flip_is_rejected_and_nothing_is_written(g):
+    N = 3
+    src = random_cache(g, N, seed=30)
+    n_tokens = 3                                # one full page and one partial page
+    blob, sums, _, _ = oracle.pack(g, src, np.array([2, 0], dtype=np.int32), n_tokens)
+    dpt = np.array([1, 2], dtype=np.int32)
+    clean = _sentinel_cache(g, N, seed=31)
+    rec0 = oracle.record_bytes(g, n_tokens, 0)
+    for bit in range(blob.size * 8):
+        bad = blob.copy()
+        bad[bit >> 3] ^= 1 << (bit & 7)
+        dst = clone_cache(clean)
+        mask, fb = oracle.restore(g, dst, [oracle.Job(bad, sums, dpt, n_tokens)])
+        assert mask[0] == oracle.CODE_CHECKSUM
+        assert fb[0] == (0 if (bit >> 3) < rec0 else 1)
+        assert np.array_equal(dst.data, clean.data)
+        if g.scale_kv:
+            assert np.array_equal(dst.scales, clean.scales)
+    for bit in range(sums.size * 64):           # damage in the checksum array instead
+        bad = sums.copy()
+        bad[bit // 64] ^= np.uint64(1) << np.uint64(bit % 64)
+        dst = clone_cache(clean)
+        mask, fb = oracle.restore(g, dst, [oracle.Job(blob, bad, dpt, n_tokens)])
+        assert mask[0] == oracle.CODE_CHECKSUM and fb[0] == bit // 64
+        assert np.array_equal(dst.data, clean.data)
+
+
+def test_sabotage_triple_defence_on_off_on():
+    """Section 3, sabotage testing: the attack must fail with the defence on,
+    succeed with it off, and fail again with it restored."""
+    g, N = SMALL, 8
+    src = random_cache(g, N, seed=40)
+    n = 10
+    spt = np.array([5, 1, 2], dtype=np.int32)
+    blob, sums, _, _ = oracle.pack(g, src, spt, n)
+    bad = blob.copy()
+    bad[100] ^= 0x40
+    dpt = np.array([0, 7, 3], dtype=np.int32)
+    clean = _sentinel_cache(g, N, seed=41)
+
+    dst = clone_cache(clean)
+    mask, _ = oracle.restore(g, dst, [oracle.Job(bad, sums, dpt, n)])
+    assert mask[0] == oracle.CODE_CHECKSUM and np.array_equal(dst.data, clean.data)
+
+    dst = clone_cache(clean)
+    mask, _ = oracle.restore(g, dst, [oracle.Job(bad, sums, dpt, n)], flags=oracle.FLAG_SKIP_VERIFY)
+    assert mask[0] == 0 and not np.array_equal(dst.data, clean.data)
+    good_dst = clone_cache(clean)
+    oracle.restore(g, good_dst, [oracle.Job(blob, sums, dpt, n)])
+    assert not np.array_equal(dst.data, good_dst.data)      # the wrong bytes really landed
+
+    dst = clone_cache(clean)
+    mask, _ = oracle.restore(g, dst, [oracle.Job(bad, sums, dpt, n)])
+    assert mask[0] == oracle.CODE_CHECKSUM and np.array_equal(dst.data, clean.data)
+
+
+def test_codes_and_first_bad_page():
+    g, N = SMALL, 12
+    src = random_cache(g, N, seed=50)
+    n = 3 * g.page_tokens
+    blob, sums, _, _ = oracle.pack(g, src, np.array([0, 1, 2], dtype=np.int32), n)
+    bad2 = blob.copy()
+    bad2[oracle.record_offset(g, 1) + 5] ^= 1
+    bad2[oracle.record_offset(g, 2) + 5] ^= 1
+    clean = _sentinel_cache(g, N, seed=51)
+    blob1, sums1, _, _ = oracle.pack(g, src, np.array([0], dtype=np.int32), 1)
+    jobs = [
+        oracle.Job(blob, sums, np.array([0, 1, 2], dtype=np.int32), n),       # ok
+        oracle.Job(bad2, sums, np.array([3, 4, 5], dtype=np.int32), n),       # checksum, page 1 first
+        oracle.Job(None, sums, np.array([6, 7, 8], dtype=np.int32), n),       # missing
+        oracle.Job(blob, None, np.array([6, 7, 8], dtype=np.int32), n),       # missing
+        oracle.Job(blob, sums, np.array([9, 12, -1], dtype=np.int32), n),     # out of range at 1
+        oracle.Job(blob, sums, np.array([6, 10, 11], dtype=np.int32), n),     # dup with next at 1
+        oracle.Job(blob, sums, np.array([8, 7, 10], dtype=np.int32), n),      # dup with previous at 2
+        oracle.Job(blob1, sums1, np.array([9], dtype=np.int32), 1),           # page 9: job 4 never claimed it
+    ]
+    dst = clone_cache(clean)
+    mask, fb = oracle.restore(g, dst, jobs)
+    assert mask.tolist() == [0, 1, 3, 3, 2, 2, 2, 0]
+    assert fb.tolist() == [-1, 1, -1, -1, 1, 1, 2, -1]
+    d = dst.data.reshape(g.layers, 2, N, g.page_tokens, -1)
+    c = clean.data.reshape(g.layers, 2, N, g.page_tokens, -1)
+    s = src.data.reshape(g.layers, 2, N, g.page_tokens, -1)
+    assert np.array_equal(d[:, :, [0, 1, 2]], s[:, :, [0, 1, 2]])
+    assert np.array_equal(d[:, :, 9, :1], s[:, :, 0, :1])
+    assert np.array_equal(d[:, :, 9, 1:], c[:, :, 9, 1:])
+    for page in (3, 4, 5, 6, 7, 8, 10, 11):
+        assert np.array_equal(d[:, :, page], c[:, :, page])
+
+
+def test_one_failed_job_does_not_stop_the_others():
+    """Tiny workload: 4 blocks, one flipped bit, 3 ok and 1 rejected."""
+    w = synth.TINY
+    g = oracle_geom(w)
+    src_pages = 64
+    src = make_cache(g, src_pages,
+                     synth.kv_bytes_bf16(cache_bytes(g, src_pages) // 2, w.sigma, w.seed(0)).numpy())
+    perm = synth.page_permutation(synth.TINY_DST_PAGES, w.seed(1))
+    jobs = []
+    for i, n in enumerate(synth.TINY_BLOCKS):
+        blob, sums, code, _ = oracle.pack(g, src, np.arange(16 * i, 16 * i + 16, dtype=np.int32), n)
+        assert code == 0
+        jobs.append(oracle.Job(blob, sums, perm[16 * i:16 * i + 16], n))
+    rng = np.random.default_rng(w.seed(2))
+    victim = int(rng.integers(0, 4))
+    bit = int(synth.bit_flip_positions(jobs[victim].blob.size * 8, 1, w.seed(3))[0])
+    jobs[victim].blob[bit >> 3] ^= 1 << (bit & 7)
+    clean = make_cache(g, synth.TINY_DST_PAGES,
+                       synth.sentinel_bytes(cache_bytes(g, synth.TINY_DST_PAGES), w.seed(4)).numpy().copy())
+    dst = clone_cache(clean)
+    mask, fb = oracle.restore(g, dst, jobs)
+    want = [0, 0, 0, 0]
+    want[victim] = 1
+    assert mask.tolist() == want
+    assert fb[victim] == (bit >> 3) // oracle.record_bytes(g, 256, 0)
+    d = dst.data.reshape(g.layers, 2, synth.TINY_DST_PAGES, g.page_tokens, -1)
+    c = clean.data.reshape(g.layers, 2, synth.TINY_DST_PAGES, g.page_tokens, -1)
+    s = src.data.reshape(g.layers, 2, src_pages, g.page_tokens, -1)
+    for i in range(4):
+        pages = perm[16 * i:16 * i + 16]
+        if i == victim:
+            assert np.array_equal(d[:, :, pages], c[:, :, pages])
+        else:
+            assert np.array_equal(d[:, :, pages], s[:, :, 16 * i:16 * i + 16])
+    rest = perm[64:]
+    assert np.array_equal(d[:, :, rest], c[:, :, rest])
