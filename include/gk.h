@@ -1,0 +1,192 @@
+/*
+ * gk.h -- C ABI of libgk: save and restore of a text block's KV state on one
+ * NVIDIA B200 (sm_100a).
+ *
+ * The operations are those of the paper's KV memory (Section 2.2, "Taliesin: KV
+ * memory"): after the runtime has computed the KV state of a block of prompt
+ * text the state is written out; when the same block recurs it is loaded
+ * instead of recomputed; stored state is checked on load; and by the rule
+ * "serve without memory, never with wrong memory" a record that is missing,
+ * damaged or fails a check is not used at all -- the block is reported for
+ * recompute.  Restored state must be bit-identical to what was saved (Section 3,
+ * Table 1), reuse is per whole block (Section 5, first item) and the design is
+ * fail-closed (Section 5, second item).  The paper does not disclose its record
+ * format (end of Section 1); the format below is this library's own.
+ *
+ * Data model
+ *   paged cache  Opaque bytes.  The slab of (layer l, kv, physical page g)
+ *                starts at data + l*layer_stride + kv*kv_stride + g*page_stride
+ *                and holds page_tokens rows of row = kv_heads*head_dim*elem
+ *                bytes, token-major ([t][h][d]); kv 0 is K, 1 is V.  One page id
+ *                addresses all layers and both K and V.
+ *   scales       fp8 caches only: one fp32 per (l, kv < scale_kv, page, head) at
+ *                scales + l*s_layer_stride + kv*s_kv_stride + g*s_page_stride + 4*h.
+ *   blob         Page records 0..P-1 (P = ceil(n_tokens/page_tokens)) back to
+ *                back, no header, no padding.  Record p = scale section (for l,
+ *                for kv < scale_kv, for h: 4 bytes; absent for bf16), then for
+ *                each layer the K prefix and the V prefix of the page, each
+ *                t_p*row bytes, where t_p = page_tokens except for a shorter
+ *                last page.  blob_bytes = P*S + n_tokens*2*layers*row.
+ *   checksums    uint64 per page: CRC-64/XZ of the bytes of its record.
+ *
+ * Conventions
+ *   Every pointer called "device" must be device memory of the context's GPU;
+ *   "host" means ordinary host memory unless "pinned" is stated.  The caller owns
+ *   every buffer it passes.  A context owns only its internal workspace.
+ *   Functions return GK_OK or a negative GK_ERR_* value; they never abort.  A
+ *   checksum mismatch is NOT an error: the call returns GK_OK and the job's mask
+ *   entry reports it.  Kernels are enqueued on the given stream; outputs are
+ *   valid once that stream has been synchronised.  A context's workspace is
+ *   shared by its calls: calls on one context must be issued in stream order on
+ *   one stream at a time (use one context per concurrent stream).
+ *   Requirements: row % 16 == 0, scale section bytes % 16 == 0, all base
+ *   pointers and strides of data 16-byte aligned (scale pointers 4-byte), blob
+ *   pointers 16-byte aligned, checksum pointers 8-byte aligned; otherwise
+ *   GK_ERR_UNSUPPORTED.
+ */
+#ifndef GK_H
+#define GK_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GK_OK 0
+#define GK_ERR_ARG (-1)         /* null pointer, zero tokens, bad geometry */
+#define GK_ERR_UNSUPPORTED (-2) /* unknown dtype, alignment rules above not met */
+#define GK_ERR_NOT_PINNED (-3)  /* host tier: blob or checksums not in pinned host memory */
+#define GK_ERR_CUDA (-4)        /* a CUDA call failed; see gk_last_error */
+#define GK_ERR_NOMEM (-5)       /* workspace allocation failed */
+#define GK_ERR_DEVICE_WAIT (-6) /* reported by gk_get_stats: a bounded device wait ran out */
+
+#define GK_BF16 0u
+#define GK_FP8_E4M3 1u
+
+/* Per-job result codes (mask entries).  Any non-zero code means that not one
+ * byte of that job was written to the destination. */
+#define GK_JOB_OK 0u          /* every page verified; block committed */
+#define GK_JOB_CHECKSUM 1u    /* a page record failed its checksum */
+#define GK_JOB_PAGE_TABLE 2u  /* page id out of [0,num_pages), or a destination page
+                                 claimed more than once within the call */
+#define GK_JOB_MISSING 3u     /* blob or checksums pointer is null */
+#define GK_JOB_TIMEOUT 4u     /* a bounded wait inside a kernel ran out; nothing of
+                                 the call was committed */
+
+/* Test hook for sabotage tests (Section 3, "Sabotage testing"): switches the
+ * checksum defence off so that a test can show the attack succeeds without it.
+ * Page-table validation stays on. */
+#define GK_FLAG_SKIP_VERIFY 1u
+
+typedef struct gk_ctx gk_ctx;
+
+typedef struct {
+    uint32_t layers;
+    uint32_t kv_heads;
+    uint32_t head_dim;
+    uint32_t page_tokens;
+    uint32_t dtype;    /* GK_BF16 or GK_FP8_E4M3 */
+    uint32_t scale_kv; /* fp8: 2 = a K scale and a V scale per (layer, head, page), 1 = one
+                          shared scale; bf16: 0 */
+    uint32_t flags;    /* 0 or GK_FLAG_SKIP_VERIFY */
+    uint32_t reserved; /* must be 0 */
+} gk_geom;
+
+typedef struct {
+    void *data;         /* device */
+    uint64_t num_pages; /* physical pages addressable through a page table */
+    uint64_t layer_stride, kv_stride, page_stride; /* bytes */
+    void *scales;       /* device; NULL when scale_kv == 0 */
+    uint64_t s_layer_stride, s_kv_stride, s_page_stride; /* bytes */
+} gk_cache;
+
+/* One block.  For gk_pack*, blob and checksums are outputs; for gk_restore* they
+ * are inputs.  page_table always points to DEVICE memory holding
+ * ceil(n_tokens/page_tokens) int32 physical page ids. */
+typedef struct {
+    void *blob;                /* device (pinned host for gk_restore_host); NULL = missing */
+    uint64_t *checksums;       /* device (pinned host for gk_restore_host); NULL = missing */
+    const int32_t *page_table; /* device */
+    uint32_t n_tokens;         /* > 0 */
+    uint32_t request_id;       /* carried for the caller; not interpreted */
+} gk_job;
+
+typedef struct {
+    uint64_t calls_pack, calls_restore, calls_restore_host;
+    uint64_t jobs, pages, bytes_blob; /* submitted so far */
+    uint64_t kernels_launched;        /* kernels enqueued by this context so far */
+    uint32_t device_wait_expired;     /* non-zero once a bounded wait inside a kernel has run out:
+                                         from then on no call of this context commits anything and
+                                         the destination of the call that hit it is undefined */
+    uint32_t reserved;
+} gk_stats;
+
+/* Sizes of a block of n_tokens (Section 2.2: one record per block).  Either output may be NULL. */
+int gk_blob_size(const gk_geom *geom, uint32_t n_tokens, uint64_t *blob_bytes, uint32_t *n_pages);
+
+/* Creates a context for one geometry on one device.  Allocates constant tables
+ * and a small workspace with cudaMalloc / cudaMallocHost; the workspace grows
+ * (with a device synchronisation) when a later call needs more. */
+int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device);
+int gk_ctx_destroy(gk_ctx *ctx);
+/* Text of the last error of this context (never NULL; empty if none). */
+const char *gk_last_error(const gk_ctx *ctx);
+
+/* Save (Section 2.2: "writes it to storage" -- here: gathers it into one
+ * contiguous record with checksums).  jobs is a HOST array of n_jobs entries;
+ * each job's blob (gk_blob_size bytes) and checksums (n_pages entries) are
+ * device outputs.  Duplicate page ids are legal when packing.  A job whose table
+ * holds an id outside [0, src->num_pages) writes neither blob nor checksums and
+ * gets status GK_JOB_PAGE_TABLE; status_dev (device, n_jobs bytes, may be NULL)
+ * receives 0 or that code.  n_jobs == 0 is a no-op. */
+int gk_pack_batch(gk_ctx *ctx, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,
+                  uint8_t *status_dev, void *stream);
+
+/* One block; same as gk_pack_batch with a single job. */
+int gk_pack(gk_ctx *ctx, const gk_cache *src, const int32_t *page_table_dev, uint32_t n_tokens,
+            void *blob_dev, uint64_t *checksums_dev, uint8_t *status_dev, void *stream);
+
+/* Page checksums of an existing device blob (the check that "Stored state is
+ * checked on load" relies on, Section 2.2): checksums_dev[p] = CRC-64/XZ of record p. */
+int gk_page_checksums(gk_ctx *ctx, const void *blob_dev, uint32_t n_tokens,
+                      uint64_t *checksums_dev, void *stream);
+
+/* Load (Section 2.2 and Section 5 "Fail-closed by design").  jobs is a HOST array;
+ * blob, checksums and page_table of each job are device pointers.  Phase 1
+ * validates every page table and verifies every page record of every job and
+ * writes nothing to dst; phase 2 scatters the jobs whose code is GK_JOB_OK into
+ * dst through their page tables (valid token prefix of each page only; fp8 scale
+ * sections to dst->scales).  mask_dev (device, n_jobs bytes) receives the code of
+ * each job, first_bad_page_dev (device, n_jobs int32) the lowest failing logical
+ * page index for codes 1 and 2, else -1.  Destination bytes outside the committed
+ * jobs' valid ranges are never written. */
+int gk_restore(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
+               uint8_t *mask_dev, int32_t *first_bad_page_dev, void *stream);
+
+/* Load from the host tier (Section 4.3, "Long windows at flat GPU memory": saved
+ * blocks are streamed in).  As gk_restore, but each job's blob and checksums lie
+ * in PINNED host memory.  Blobs are copied in batches into an internal device
+ * staging ring on an internal copy stream while the previous batch is verified
+ * and committed on `stream`; the checksum is taken over the bytes as they arrived
+ * in device memory.  All page tables are validated before the first copy.  The
+ * call returns after the last stage has been enqueued; results are valid after
+ * `stream` has been synchronised.  The host buffers must stay valid until then. */
+int gk_restore_host(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
+                    uint8_t *mask_dev, int32_t *first_bad_page_dev, void *stream);
+
+/* Counters of this context.  Reads the device error word with a blocking copy. */
+int gk_get_stats(gk_ctx *ctx, gk_stats *out);
+
+/* Tuning knobs, for tests and measurements; defaults are chosen from the
+ * geometry.  Keys: "seg_granules" (length of a checksum segment in units of
+ * 32 KiB; 0 = one segment per page), "commit_seg_tiles" (length of a commit work
+ * item in 16 KiB tiles), "grid_cap" (upper bound on CTAs per kernel; 0 = fill
+ * the GPU). */
+int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

@@ -1,0 +1,232 @@
+"""ctypes binding of libgk: argument marshalling only.
+
+Every function mirrors the C entry point of the same name in ``include/gk.h``.
+Tensors are torch tensors used purely as device (or pinned host) memory; the
+binding passes their addresses and sizes through and raises ``GkError`` on a
+negative return code.  There is no fallback: if ``libgk.so`` is missing, or no
+sm_100 device is present, calls fail loudly.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional, Sequence
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgk.so")
+
+GK_OK = 0
+GK_BF16, GK_FP8_E4M3 = 0, 1
+GK_FLAG_SKIP_VERIFY = 1
+JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
+
+EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",
+           "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning"]
+
+
+class GkError(RuntimeError):
+    def __init__(self, code: int, where: str, detail: str = ""):
+        super().__init__(f"{where} failed with code {code}" + (f": {detail}" if detail else ""))
+        self.code = code
+
+
+class CGeom(ctypes.Structure):
+    _fields_ = [("layers", ctypes.c_uint32), ("kv_heads", ctypes.c_uint32), ("head_dim", ctypes.c_uint32),
+                ("page_tokens", ctypes.c_uint32), ("dtype", ctypes.c_uint32), ("scale_kv", ctypes.c_uint32),
+                ("flags", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+
+
+class CCache(ctypes.Structure):
+    _fields_ = [("data", ctypes.c_void_p), ("num_pages", ctypes.c_uint64), ("layer_stride", ctypes.c_uint64),
+                ("kv_stride", ctypes.c_uint64), ("page_stride", ctypes.c_uint64), ("scales", ctypes.c_void_p),
+                ("s_layer_stride", ctypes.c_uint64), ("s_kv_stride", ctypes.c_uint64),
+                ("s_page_stride", ctypes.c_uint64)]
+
+
+class CJob(ctypes.Structure):
+    _fields_ = [("blob", ctypes.c_void_p), ("checksums", ctypes.c_void_p), ("page_table", ctypes.c_void_p),
+                ("n_tokens", ctypes.c_uint32), ("request_id", ctypes.c_uint32)]
+
+
+class CStats(ctypes.Structure):
+    _fields_ = [("calls_pack", ctypes.c_uint64), ("calls_restore", ctypes.c_uint64),
+                ("calls_restore_host", ctypes.c_uint64), ("jobs", ctypes.c_uint64), ("pages", ctypes.c_uint64),
+                ("bytes_blob", ctypes.c_uint64), ("kernels_launched", ctypes.c_uint64),
+                ("device_wait_expired", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libgk.so (built in-tree by ``paper_2609_39358_b200.build``)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2609_39358_b200.build` "
+                          "(there is no CPU fallback)")
+    L = ctypes.CDLL(LIB_PATH)
+    vp, u32, u64p = ctypes.c_void_p, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint64)
+    L.gk_blob_size.restype = ctypes.c_int
+    L.gk_blob_size.argtypes = [ctypes.POINTER(CGeom), u32, u64p, ctypes.POINTER(u32)]
+    L.gk_ctx_create.restype = ctypes.c_int
+    L.gk_ctx_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(CGeom), ctypes.c_int]
+    L.gk_ctx_destroy.restype = ctypes.c_int
+    L.gk_ctx_destroy.argtypes = [vp]
+    L.gk_last_error.restype = ctypes.c_char_p
+    L.gk_last_error.argtypes = [vp]
+    L.gk_pack_batch.restype = ctypes.c_int
+    L.gk_pack_batch.argtypes = [vp, ctypes.POINTER(CCache), ctypes.POINTER(CJob), u32, vp, vp]
+    L.gk_pack.restype = ctypes.c_int
+    L.gk_pack.argtypes = [vp, ctypes.POINTER(CCache), vp, u32, vp, vp, vp, vp]
+    L.gk_page_checksums.restype = ctypes.c_int
+    L.gk_page_checksums.argtypes = [vp, vp, u32, vp, vp]
+    L.gk_restore.restype = ctypes.c_int
+    L.gk_restore.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
+    L.gk_restore_host.restype = ctypes.c_int
+    L.gk_restore_host.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
+    L.gk_get_stats.restype = ctypes.c_int
+    L.gk_get_stats.argtypes = [vp, ctypes.POINTER(CStats)]
+    L.gk_ctx_set_tuning.restype = ctypes.c_int
+    L.gk_ctx_set_tuning.argtypes = [vp, ctypes.c_char_p, u32]
+    _lib = L
+    return L
+
+
+@dataclass(frozen=True)
+class Geom:
+    layers: int
+    kv_heads: int
+    head_dim: int
+    page_tokens: int
+    dtype: int = GK_BF16
+    scale_kv: int = 0
+    flags: int = 0
+
+    def c(self) -> CGeom:
+        return CGeom(self.layers, self.kv_heads, self.head_dim, self.page_tokens, self.dtype, self.scale_kv,
+                     self.flags, 0)
+
+
+@dataclass
+class Cache:
+    """A paged cache: a uint8 device tensor plus byte strides (see gk.h)."""
+    data: torch.Tensor
+    num_pages: int
+    layer_stride: int
+    kv_stride: int
+    page_stride: int
+    scales: Optional[torch.Tensor] = None
+    s_layer_stride: int = 0
+    s_kv_stride: int = 0
+    s_page_stride: int = 0
+
+    def c(self) -> CCache:
+        return CCache(self.data.data_ptr(), self.num_pages, self.layer_stride, self.kv_stride, self.page_stride,
+                      0 if self.scales is None else self.scales.data_ptr(), self.s_layer_stride,
+                      self.s_kv_stride, self.s_page_stride)
+
+
+@dataclass
+class Job:
+    blob: Optional[torch.Tensor]        # uint8; device (pinned host for restore_host); None = missing
+    checksums: Optional[torch.Tensor]   # int64/uint64 storage of P entries; None = missing
+    page_table: torch.Tensor            # int32, device
+    n_tokens: int
+    request_id: int = 0
+
+
+def _ptr(t: Optional[torch.Tensor]) -> int:
+    return 0 if t is None else t.data_ptr()
+
+
+def _stream_handle(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def gk_blob_size(geom: Geom, n_tokens: int) -> tuple[int, int]:
+    nb, npg = ctypes.c_uint64(0), ctypes.c_uint32(0)
+    cg = geom.c()
+    rc = load_library().gk_blob_size(ctypes.byref(cg), n_tokens, ctypes.byref(nb), ctypes.byref(npg))
+    if rc != GK_OK:
+        raise GkError(rc, "gk_blob_size")
+    return int(nb.value), int(npg.value)
+
+
+class Context:
+    """Owns a ``gk_ctx``.  One context per concurrently used stream."""
+
+    def __init__(self, geom: Geom, device: int = 0):
+        self._lib = load_library()
+        self.geom = geom
+        self.device = device
+        h = ctypes.c_void_p(0)
+        cg = geom.c()
+        rc = self._lib.gk_ctx_create(ctypes.byref(h), ctypes.byref(cg), device)
+        if rc != GK_OK:
+            raise GkError(rc, "gk_ctx_create")
+        self._h = h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            self._lib.gk_ctx_destroy(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def _check(self, rc: int, where: str):
+        if rc != GK_OK:
+            raise GkError(rc, where, self._lib.gk_last_error(self._h).decode(errors="replace"))
+
+    def _jobs(self, jobs: Sequence[Job]):
+        arr = (CJob * max(len(jobs), 1))()
+        for i, j in enumerate(jobs):
+            arr[i] = CJob(_ptr(j.blob), _ptr(j.checksums), _ptr(j.page_table), j.n_tokens, j.request_id)
+        return arr
+
+    def set_tuning(self, key: str, value: int):
+        self._check(self._lib.gk_ctx_set_tuning(self._h, key.encode(), value), "gk_ctx_set_tuning")
+
+    def gk_pack_batch(self, src: Cache, jobs: Sequence[Job], status: Optional[torch.Tensor] = None, stream=None):
+        cc = src.c()
+        self._check(self._lib.gk_pack_batch(self._h, ctypes.byref(cc), self._jobs(jobs), len(jobs), _ptr(status),
+                                            _stream_handle(stream)), "gk_pack_batch")
+
+    def gk_pack(self, src: Cache, page_table: torch.Tensor, n_tokens: int, blob: torch.Tensor,
+                checksums: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None):
+        cc = src.c()
+        self._check(self._lib.gk_pack(self._h, ctypes.byref(cc), _ptr(page_table), n_tokens, _ptr(blob),
+                                      _ptr(checksums), _ptr(status), _stream_handle(stream)), "gk_pack")
+
+    def gk_page_checksums(self, blob: torch.Tensor, n_tokens: int, checksums: torch.Tensor, stream=None):
+        self._check(self._lib.gk_page_checksums(self._h, _ptr(blob), n_tokens, _ptr(checksums),
+                                                _stream_handle(stream)), "gk_page_checksums")
+
+    def gk_restore(self, jobs: Sequence[Job], dst: Cache, mask: torch.Tensor, first_bad_page: torch.Tensor,
+                   stream=None):
+        cc = dst.c()
+        self._check(self._lib.gk_restore(self._h, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask),
+                                         _ptr(first_bad_page), _stream_handle(stream)), "gk_restore")
+
+    def gk_restore_host(self, jobs: Sequence[Job], dst: Cache, mask: torch.Tensor, first_bad_page: torch.Tensor,
+                        stream=None):
+        cc = dst.c()
+        self._check(self._lib.gk_restore_host(self._h, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask),
+                                              _ptr(first_bad_page), _stream_handle(stream)), "gk_restore_host")
+
+    def gk_get_stats(self) -> dict:
+        st = CStats()
+        self._check(self._lib.gk_get_stats(self._h, ctypes.byref(st)), "gk_get_stats")
+        return {name: int(getattr(st, name)) for name, _ in CStats._fields_ if name != "reserved"}

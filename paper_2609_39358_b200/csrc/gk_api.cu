@@ -1,0 +1,771 @@
+// gk_api.cu -- host side of libgk: the C ABI declared in include/gk.h.
+//
+// Argument checking, per-call job tables, workspace management, kernel
+// launches and the host-tier staging pipeline.  Every step of the data path
+// runs in the kernels of gk_kernels.cuh; there is no CPU fallback.
+#include "../../include/gk.h"
+
+#include <cstdarg>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "gk_kernels.cuh"
+
+#ifndef GK_CRC_NT
+#define GK_CRC_NT 128
+#endif
+#ifndef GK_CRC_STAGE
+#define GK_CRC_STAGE 8192
+#endif
+#ifndef GK_CRC_STAGES
+#define GK_CRC_STAGES 6
+#endif
+#ifndef GK_CRC_MINB
+#define GK_CRC_MINB 2
+#endif
+#ifndef GK_COPY_STAGE
+#define GK_COPY_STAGE 16384
+#endif
+#ifndef GK_COPY_STAGES
+#define GK_COPY_STAGES 4
+#endif
+#ifndef GK_COPY_MINB
+#define GK_COPY_MINB 3
+#endif
+
+using namespace gk;
+
+namespace {
+
+using VerifyCfg = StreamCfg<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES>;
+using PackCfg = StreamCfg<kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES>;
+using CommitCfg = StreamCfg<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES>;
+
+constexpr int kSlots = 2;  // host-tier staging ring
+
+uint64_t gf_xpow(uint64_t n)
+{
+    uint64_t r = 1, base = 2;
+    while (n) {
+        if (n & 1ull) r = gf_mul(r, base);
+        base = gf_mul(base, base);
+        n >>= 1;
+    }
+    return r;
+}
+
+size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+}  // namespace
+
+struct gk_ctx {
+    gk_geom geom{};
+    GeomDev gd{};
+    int device = 0;
+    int sm_count = 0;
+    int occ_verify = 0, occ_pack = 0, occ_commit = 0;
+    uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
+    uint32_t commit_seg_tiles = 0;
+    uint32_t grid_cap = 0;       // 0: SMs * occupancy
+
+    // constant tables + sticky error word
+    uint64_t *d_init_term = nullptr;
+    uint64_t *d_thread_const = nullptr;
+    uint32_t *d_error = nullptr;
+
+    // growing device workspace and pinned staging for job tables
+    uint8_t *d_ws = nullptr;
+    size_t ws_cap = 0;
+    uint8_t *h_stage = nullptr;
+    size_t h_stage_cap = 0;
+    cudaEvent_t ev_stage = nullptr;  // upload of the job table has been consumed
+
+    // host tier
+    cudaStream_t copy_stream = nullptr;
+    uint8_t *d_slot[kSlots] = {nullptr, nullptr};
+    size_t slot_cap = 0;
+    cudaEvent_t ev_slot_free[kSlots] = {nullptr, nullptr};
+    cudaEvent_t ev_copied[kSlots] = {nullptr, nullptr};
+    bool slot_used[kSlots] = {false, false};
+
+    gk_stats stats{};
+    char err[512] = {0};
+};
+
+namespace {
+
+int fail(gk_ctx *c, int code, const char *fmt, ...)
+{
+    if (c) {
+        va_list ap;
+        va_start(ap, fmt);
+        vsnprintf(c->err, sizeof(c->err), fmt, ap);
+        va_end(ap);
+    }
+    return code;
+}
+
+#define GK_CUDA(c, call)                                                                      \
+    do {                                                                                      \
+        cudaError_t e_ = (call);                                                              \
+        if (e_ != cudaSuccess)                                                                \
+            return fail((c), GK_ERR_CUDA, "%s failed: %s", #call, cudaGetErrorString(e_));    \
+    } while (0)
+
+int check_geom(const gk_geom *g, GeomDev *out)
+{
+    if (!g) return GK_ERR_ARG;
+    if (g->layers == 0 || g->kv_heads == 0 || g->head_dim == 0 || g->page_tokens == 0) return GK_ERR_ARG;
+    if (g->reserved != 0 || (g->flags & ~GK_FLAG_SKIP_VERIFY)) return GK_ERR_ARG;
+    uint32_t elem;
+    if (g->dtype == GK_BF16) {
+        elem = 2;
+        if (g->scale_kv != 0) return GK_ERR_ARG;
+    } else if (g->dtype == GK_FP8_E4M3) {
+        elem = 1;
+        if (g->scale_kv != 1 && g->scale_kv != 2) return GK_ERR_ARG;
+    } else {
+        return GK_ERR_UNSUPPORTED;
+    }
+    const uint64_t row = (uint64_t)g->kv_heads * g->head_dim * elem;
+    const uint64_t S = (uint64_t)g->layers * g->scale_kv * g->kv_heads * 4u;
+    if (row % 16 != 0 || S % 16 != 0) return GK_ERR_UNSUPPORTED;
+    if (row * g->page_tokens > (1ull << 30) || S > (1ull << 30)) return GK_ERR_UNSUPPORTED;
+    if (out) {
+        out->layers = g->layers;
+        out->kv_heads = g->kv_heads;
+        out->page_tokens = g->page_tokens;
+        out->scale_kv = g->scale_kv;
+        out->row = (uint32_t)row;
+        out->S = (uint32_t)S;
+        out->h4 = g->kv_heads * 4u;
+        out->flags = g->flags;
+        out->tokB = 2ull * g->layers * row;
+        out->R = S + (uint64_t)g->page_tokens * out->tokB;
+    }
+    return GK_OK;
+}
+
+int check_cache(gk_ctx *c, const gk_cache *k, CacheDev *out)
+{
+    if (!k || !k->data || k->num_pages == 0) return fail(c, GK_ERR_ARG, "cache: null data or zero pages");
+    if (k->num_pages > 0x7fffffffull) return fail(c, GK_ERR_ARG, "cache: too many pages");
+    if (((uintptr_t)k->data | k->layer_stride | k->kv_stride | k->page_stride) & 15u)
+        return fail(c, GK_ERR_UNSUPPORTED, "cache: data pointer and strides must be multiples of 16 bytes");
+    if (c->gd.scale_kv) {
+        if (!k->scales) return fail(c, GK_ERR_ARG, "cache: fp8 geometry needs a scale tensor");
+        if (((uintptr_t)k->scales | k->s_layer_stride | k->s_kv_stride | k->s_page_stride) & 3u)
+            return fail(c, GK_ERR_UNSUPPORTED, "cache: scale pointer and strides must be multiples of 4 bytes");
+    }
+    out->data = (uint8_t *)k->data;
+    out->num_pages = k->num_pages;
+    out->layer_stride = k->layer_stride;
+    out->kv_stride = k->kv_stride;
+    out->page_stride = k->page_stride;
+    out->scales = (uint8_t *)k->scales;
+    out->s_layer_stride = k->s_layer_stride;
+    out->s_kv_stride = k->s_kv_stride;
+    out->s_page_stride = k->s_page_stride;
+    return GK_OK;
+}
+
+Tiling crc_tiling(const gk_ctx *c)
+{
+    Tiling t;
+    t.stage_bytes = GK_CRC_STAGE;
+    t.gran_bytes = VerifyCfg::kGran;
+    const uint32_t gran_full = (uint32_t)((c->gd.R + t.gran_bytes - 1) / t.gran_bytes);
+    uint32_t sg = c->seg_granules ? c->seg_granules : gran_full;
+    if (sg > gran_full) sg = gran_full;
+    t.seg_tiles = sg * VerifyCfg::kTilesPerGran;
+    t.nseg_max = (gran_full + sg - 1) / sg;
+    return t;
+}
+
+Tiling commit_tiling(const gk_ctx *c)
+{
+    Tiling t;
+    t.stage_bytes = GK_COPY_STAGE;
+    t.gran_bytes = GK_COPY_STAGE;
+    const uint32_t tiles_full = (uint32_t)((c->gd.R + t.stage_bytes - 1) / t.stage_bytes);
+    uint32_t st = c->commit_seg_tiles ? c->commit_seg_tiles : 16u;
+    if (st > tiles_full) st = tiles_full;
+    t.seg_tiles = st;
+    t.nseg_max = (tiles_full + st - 1) / st;
+    return t;
+}
+
+// Views into the workspace for one call.
+struct WsLayout {
+    size_t jobs, page_job, seg_res, bad_range, bad_dup, bad_crc, claims, total;
+};
+
+WsLayout ws_layout(uint32_t n_jobs, uint64_t total_pages, uint32_t nseg_max, uint64_t num_pages)
+{
+    WsLayout l;
+    size_t o = 0;
+    l.jobs = o;      o = align_up(o + (size_t)n_jobs * sizeof(JobDev), 256);
+    l.page_job = o;  o = align_up(o + (size_t)total_pages * 4, 256);
+    l.seg_res = o;   o = align_up(o + (size_t)total_pages * nseg_max * 8, 256);
+    l.bad_range = o; o = align_up(o + (size_t)n_jobs * 4, 256);
+    l.bad_dup = o;   o = align_up(o + (size_t)n_jobs * 4, 256);
+    l.bad_crc = o;   o = align_up(o + (size_t)n_jobs * 4, 256);
+    l.claims = o;    o = align_up(o + (size_t)num_pages * 8, 256);
+    l.total = o;
+    return l;
+}
+
+int ensure_workspace(gk_ctx *c, size_t need)
+{
+    if (need <= c->ws_cap) return GK_OK;
+    GK_CUDA(c, cudaDeviceSynchronize());  // earlier calls may still use the old block
+    if (c->d_ws) cudaFree(c->d_ws);
+    c->d_ws = nullptr;
+    c->ws_cap = 0;
+    const size_t cap = align_up(need + need / 2, 1 << 20);
+    if (cudaMalloc(&c->d_ws, cap) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, GK_ERR_NOMEM, "workspace of %zu bytes", cap);
+    }
+    c->ws_cap = cap;
+    return GK_OK;
+}
+
+int ensure_host_stage(gk_ctx *c, size_t need)
+{
+    if (need <= c->h_stage_cap) return GK_OK;
+    GK_CUDA(c, cudaEventSynchronize(c->ev_stage));
+    if (c->h_stage) cudaFreeHost(c->h_stage);
+    c->h_stage = nullptr;
+    c->h_stage_cap = 0;
+    const size_t cap = align_up(need * 2, 1 << 16);
+    if (cudaMallocHost(&c->h_stage, cap) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, GK_ERR_NOMEM, "pinned staging of %zu bytes", cap);
+    }
+    c->h_stage_cap = cap;
+    return GK_OK;
+}
+
+WorkDev make_work(const gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t total_pages, const Tiling &crc)
+{
+    WorkDev w{};
+    w.jobs = (const JobDev *)(c->d_ws + l.jobs);
+    w.n_jobs = n_jobs;
+    w.page_begin = 0;
+    w.total_pages = total_pages;
+    w.page_job = (int32_t *)(c->d_ws + l.page_job);
+    w.seg_res = (uint64_t *)(c->d_ws + l.seg_res);
+    w.bad_range = (int32_t *)(c->d_ws + l.bad_range);
+    w.bad_dup = (int32_t *)(c->d_ws + l.bad_dup);
+    w.bad_crc = (int32_t *)(c->d_ws + l.bad_crc);
+    w.claims = (unsigned long long *)(c->d_ws + l.claims);
+    w.error = c->d_error;
+    w.init_term = c->d_init_term;
+    w.thread_const = c->d_thread_const;
+    w.x_seg = gf_xpow(8ull * crc.seg_tiles * crc.stage_bytes);
+    return w;
+}
+
+// Fills the pinned job table and enqueues its upload.  blob_override /
+// sums_override (may be null) replace the callers' pointers, for the host tier.
+int upload_jobs(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const WsLayout &l, uint8_t *const *blob_override,
+                uint64_t *const *sums_override, bool need_tables, cudaStream_t st, uint64_t *total_pages_out,
+                uint64_t *total_bytes_out)
+{
+    int rc = ensure_host_stage(c, (size_t)n_jobs * sizeof(JobDev));
+    if (rc != GK_OK) return rc;
+    GK_CUDA(c, cudaEventSynchronize(c->ev_stage));
+    JobDev *h = (JobDev *)c->h_stage;
+    uint64_t pages = 0, bytes = 0;
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        const gk_job &jb = jobs[j];
+        if (jb.n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
+        if (need_tables && !jb.page_table) return fail(c, GK_ERR_ARG, "job %u: null page table", j);
+        const uint32_t np = (jb.n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+        h[j].blob = blob_override ? blob_override[j] : (uint8_t *)jb.blob;
+        h[j].checksums = sums_override ? sums_override[j] : jb.checksums;
+        h[j].page_table = jb.page_table;
+        h[j].n_tokens = jb.n_tokens;
+        h[j].n_pages = np;
+        h[j].page_base = (uint32_t)pages;
+        h[j].missing = (jb.blob == nullptr || jb.checksums == nullptr) ? 1u : 0u;
+        if (!h[j].missing) {
+            if (((uintptr_t)h[j].blob & 15u) || ((uintptr_t)h[j].checksums & 7u))
+                return fail(c, GK_ERR_UNSUPPORTED, "job %u: blob must be 16-byte and checksums 8-byte aligned", j);
+        }
+        pages += np;
+        bytes += (uint64_t)np * c->gd.S + (uint64_t)jb.n_tokens * c->gd.tokB;
+        if (pages > 0x7fffffffull) return fail(c, GK_ERR_ARG, "too many pages in one call");
+    }
+    *total_pages_out = pages;
+    if (total_bytes_out) *total_bytes_out = bytes;
+    GK_CUDA(c, cudaMemcpyAsync(c->d_ws + l.jobs, h, (size_t)n_jobs * sizeof(JobDev), cudaMemcpyHostToDevice, st));
+    GK_CUDA(c, cudaEventRecord(c->ev_stage, st));
+    return GK_OK;
+}
+
+uint32_t stream_grid(const gk_ctx *c, int occ, uint32_t n_items)
+{
+    uint32_t g = (uint32_t)(c->sm_count * occ);
+    if (c->grid_cap && g > c->grid_cap) g = c->grid_cap;
+    if (g > n_items) g = n_items;
+    return g ? g : 1u;
+}
+
+template <class Cfg, int MODE, int NT, int SB, int ST, int MINB>
+int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
+{
+    if (P.n_items == 0) return GK_OK;
+    const uint32_t grid = stream_grid(c, occ, P.n_items);
+    stream_kernel<MODE, NT, SB, ST, MINB><<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(P);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched++;
+    return GK_OK;
+}
+
+int launch_verify(gk_ctx *c, const StreamParams &P, cudaStream_t st)
+{
+    return launch_stream<VerifyCfg, kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_CRC_MINB>(c, c->occ_verify, P, st);
+}
+int launch_pack(gk_ctx *c, const StreamParams &P, cudaStream_t st)
+{
+    return launch_stream<PackCfg, kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_CRC_MINB>(c, c->occ_pack, P, st);
+}
+int launch_commit(gk_ctx *c, const StreamParams &P, cudaStream_t st)
+{
+    return launch_stream<CommitCfg, kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES, GK_COPY_MINB>(c, c->occ_commit, P, st);
+}
+
+int launch_validate(gk_ctx *c, const WorkDev &w, uint64_t num_pages, int clear_claims, cudaStream_t st)
+{
+    uint32_t grid = w.n_jobs;
+    if (clear_claims) {
+        uint32_t g2 = (uint32_t)((num_pages + 255) / 256);
+        if (g2 > 2048) g2 = 2048;
+        if (g2 > grid) grid = g2;
+    }
+    validate_kernel<<<grid, 256, 0, st>>>(w, num_pages, clear_claims);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched++;
+    return GK_OK;
+}
+
+int launch_claim(gk_ctx *c, const WorkDev &w, cudaStream_t st)
+{
+    claim_kernel<<<(w.total_pages + 255) / 256, 256, 0, st>>>(w);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched++;
+    return GK_OK;
+}
+
+int launch_finalize(gk_ctx *c, const WorkDev &w, const Tiling &tl, int write_mode, uint8_t *status, cudaStream_t st)
+{
+    finalize_kernel<<<(w.total_pages + 127) / 128, 128, 0, st>>>(c->gd, w, tl, write_mode, status);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched++;
+    return GK_OK;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    explicit DeviceGuard(int dev)
+    {
+        cudaGetDevice(&prev);
+        if (prev != dev) cudaSetDevice(dev);
+        else prev = -1;
+    }
+    ~DeviceGuard()
+    {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+}  // namespace
+
+extern "C" {
+
+int gk_blob_size(const gk_geom *geom, uint32_t n_tokens, uint64_t *blob_bytes, uint32_t *n_pages)
+{
+    GeomDev gd;
+    const int rc = check_geom(geom, &gd);
+    if (rc != GK_OK) return rc;
+    if (n_tokens == 0) return GK_ERR_ARG;
+    const uint32_t np = (n_tokens + gd.page_tokens - 1) / gd.page_tokens;
+    if (blob_bytes) *blob_bytes = (uint64_t)np * gd.S + (uint64_t)n_tokens * gd.tokB;
+    if (n_pages) *n_pages = np;
+    return GK_OK;
+}
+
+int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
+{
+    if (!out) return GK_ERR_ARG;
+    *out = nullptr;
+    GeomDev gd;
+    int rc = check_geom(geom, &gd);
+    if (rc != GK_OK) return rc;
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || device < 0 || device >= ndev) {
+        cudaGetLastError();
+        return GK_ERR_CUDA;
+    }
+    gk_ctx *c = new (std::nothrow) gk_ctx();
+    if (!c) return GK_ERR_NOMEM;
+    c->geom = *geom;
+    c->gd = gd;
+    c->device = device;
+    DeviceGuard guard(device);
+
+    auto bail = [&](int code) {
+        gk_ctx_destroy(c);
+        return code;
+    };
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return bail(GK_ERR_CUDA);
+    if (prop.major != 10) return bail(GK_ERR_UNSUPPORTED);  // built for sm_100a only
+    c->sm_count = prop.multiProcessorCount;
+
+    auto *kv = stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_CRC_MINB>;
+    auto *kp = stream_kernel<kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_CRC_MINB>;
+    auto *kc = stream_kernel<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES, GK_COPY_MINB>;
+    if (cudaFuncSetAttribute(kv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VerifyCfg::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(kp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PackCfg::kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CommitCfg::kSmemBytes) != cudaSuccess)
+        return bail(GK_ERR_CUDA);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_verify, kv, VerifyCfg::kThreads, VerifyCfg::kSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack, kp, PackCfg::kThreads, PackCfg::kSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_commit, kc, CommitCfg::kThreads, CommitCfg::kSmemBytes) != cudaSuccess)
+        return bail(GK_ERR_CUDA);
+    if (c->occ_verify < 1 || c->occ_pack < 1 || c->occ_commit < 1) return bail(GK_ERR_UNSUPPORTED);
+
+    // tables: ones * x^(8*len(t)) for every page fill t, and the per-thread placement constants
+    std::vector<uint64_t> init(gd.page_tokens + 1, 0);
+    for (uint32_t t = 1; t <= gd.page_tokens; ++t)
+        init[t] = gf_mul(~0ull, gf_xpow(8ull * (gd.S + (uint64_t)t * gd.tokB)));
+    std::vector<uint64_t> tc(GK_CRC_NT);
+    for (int t = 0; t < GK_CRC_NT; ++t) tc[t] = gf_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);
+    if (cudaMalloc(&c->d_init_term, init.size() * 8) != cudaSuccess ||
+        cudaMalloc(&c->d_thread_const, tc.size() * 8) != cudaSuccess ||
+        cudaMalloc(&c->d_error, 256) != cudaSuccess)
+        return bail(GK_ERR_NOMEM);
+    if (cudaMemcpy(c->d_init_term, init.data(), init.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(c->d_thread_const, tc.data(), tc.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemset(c->d_error, 0, 256) != cudaSuccess)
+        return bail(GK_ERR_CUDA);
+    if (cudaEventCreateWithFlags(&c->ev_stage, cudaEventDisableTiming) != cudaSuccess) return bail(GK_ERR_CUDA);
+    for (int i = 0; i < kSlots; ++i) {
+        if (cudaEventCreateWithFlags(&c->ev_slot_free[i], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->ev_copied[i], cudaEventDisableTiming) != cudaSuccess)
+            return bail(GK_ERR_CUDA);
+    }
+    if (cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) != cudaSuccess) return bail(GK_ERR_CUDA);
+    *out = c;
+    return GK_OK;
+}
+
+int gk_ctx_destroy(gk_ctx *c)
+{
+    if (!c) return GK_OK;
+    DeviceGuard guard(c->device);
+    cudaDeviceSynchronize();
+    if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    for (int i = 0; i < kSlots; ++i) {
+        if (c->d_slot[i]) cudaFree(c->d_slot[i]);
+        if (c->ev_slot_free[i]) cudaEventDestroy(c->ev_slot_free[i]);
+        if (c->ev_copied[i]) cudaEventDestroy(c->ev_copied[i]);
+    }
+    if (c->ev_stage) cudaEventDestroy(c->ev_stage);
+    if (c->h_stage) cudaFreeHost(c->h_stage);
+    if (c->d_ws) cudaFree(c->d_ws);
+    if (c->d_init_term) cudaFree(c->d_init_term);
+    if (c->d_thread_const) cudaFree(c->d_thread_const);
+    if (c->d_error) cudaFree(c->d_error);
+    cudaGetLastError();
+    delete c;
+    return GK_OK;
+}
+
+const char *gk_last_error(const gk_ctx *c) { return c ? c->err : "null context"; }
+
+int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
+{
+    if (!c || !key) return GK_ERR_ARG;
+    if (!strcmp(key, "seg_granules")) c->seg_granules = value;
+    else if (!strcmp(key, "commit_seg_tiles")) c->commit_seg_tiles = value;
+    else if (!strcmp(key, "grid_cap")) c->grid_cap = value;
+    else return fail(c, GK_ERR_ARG, "unknown tuning key %s", key);
+    return GK_OK;
+}
+
+int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs, uint8_t *status_dev,
+                  void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0) return GK_OK;
+    if (!jobs) return fail(c, GK_ERR_ARG, "null job array");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    CacheDev cd;
+    int rc = check_cache(c, src, &cd);
+    if (rc != GK_OK) return rc;
+    for (uint32_t j = 0; j < n_jobs; ++j)
+        if (!jobs[j].blob || !jobs[j].checksums) return fail(c, GK_ERR_ARG, "job %u: null output", j);
+
+    const Tiling tl = crc_tiling(c);
+    uint64_t pages = 0, bytes = 0;
+    for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
+    if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
+    if ((rc = upload_jobs(c, jobs, n_jobs, l, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
+    WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tl);
+
+    if ((rc = launch_validate(c, w, cd.num_pages, 0, st)) != GK_OK) return rc;
+    StreamParams P{};
+    P.g = c->gd;
+    P.cache = cd;
+    P.w = w;
+    P.tl = tl;
+    P.n_items = (uint32_t)pages * tl.nseg_max;
+    if ((rc = launch_pack(c, P, st)) != GK_OK) return rc;
+    if ((rc = launch_finalize(c, w, tl, 1, status_dev, st)) != GK_OK) return rc;
+    c->stats.calls_pack++;
+    c->stats.jobs += n_jobs;
+    c->stats.pages += pages;
+    c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+int gk_pack(gk_ctx *c, const gk_cache *src, const int32_t *page_table_dev, uint32_t n_tokens, void *blob_dev,
+            uint64_t *checksums_dev, uint8_t *status_dev, void *stream)
+{
+    gk_job jb{};
+    jb.blob = blob_dev;
+    jb.checksums = checksums_dev;
+    jb.page_table = page_table_dev;
+    jb.n_tokens = n_tokens;
+    return gk_pack_batch(c, src, &jb, 1, status_dev, stream);
+}
+
+int gk_page_checksums(gk_ctx *c, const void *blob_dev, uint32_t n_tokens, uint64_t *checksums_dev, void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (!blob_dev || !checksums_dev || n_tokens == 0) return fail(c, GK_ERR_ARG, "null blob/checksums or zero tokens");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    gk_job jb{};
+    jb.blob = const_cast<void *>(blob_dev);
+    jb.checksums = checksums_dev;
+    jb.page_table = nullptr;
+    jb.n_tokens = n_tokens;
+    const Tiling tl = crc_tiling(c);
+    uint64_t pages = (n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens, bytes = 0;
+    const WsLayout l = ws_layout(1, pages, tl.nseg_max, 0);
+    int rc;
+    if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
+    if ((rc = upload_jobs(c, &jb, 1, l, nullptr, nullptr, false, st, &pages, &bytes)) != GK_OK) return rc;
+    WorkDev w = make_work(c, l, 1, (uint32_t)pages, tl);
+    if ((rc = launch_validate(c, w, 0, 0, st)) != GK_OK) return rc;
+    StreamParams P{};
+    P.g = c->gd;
+    P.w = w;
+    P.tl = tl;
+    P.n_items = (uint32_t)pages * tl.nseg_max;
+    if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
+    if ((rc = launch_finalize(c, w, tl, 1, nullptr, st)) != GK_OK) return rc;
+    c->stats.pages += pages;
+    c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+// verify + commit for the pages [page_begin, page_begin + n_pages) of the call
+static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const Tiling &tlv, const Tiling &tlc,
+                                 uint32_t page_begin, uint32_t n_pages, uint8_t *mask_dev, int32_t *first_bad_dev,
+                                 cudaStream_t st)
+{
+    int rc;
+    w.page_begin = page_begin;
+    w.total_pages = n_pages;
+    StreamParams P{};
+    P.g = c->gd;
+    P.cache = cd;
+    P.w = w;
+    P.mask_out = mask_dev;
+    P.first_bad_out = first_bad_dev;
+    if (!(c->gd.flags & GK_FLAG_SKIP_VERIFY)) {
+        P.tl = tlv;
+        P.n_items = n_pages * tlv.nseg_max;
+        if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
+        if ((rc = launch_finalize(c, w, tlv, 0, nullptr, st)) != GK_OK) return rc;
+    }
+    P.tl = tlc;
+    P.n_items = n_pages * tlc.nseg_max;
+    return launch_commit(c, P, st);
+}
+
+int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, uint8_t *mask_dev,
+               int32_t *first_bad_page_dev, void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0) return GK_OK;
+    if (!jobs || !mask_dev || !first_bad_page_dev) return fail(c, GK_ERR_ARG, "null jobs, mask or first_bad_page");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    CacheDev cd;
+    int rc = check_cache(c, dst, &cd);
+    if (rc != GK_OK) return rc;
+
+    const Tiling tlv = crc_tiling(c), tlc = commit_tiling(c);
+    uint64_t pages = 0, bytes = 0;
+    for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
+    if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
+    if ((rc = upload_jobs(c, jobs, n_jobs, l, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
+    WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tlv);
+
+    if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
+    if ((rc = launch_claim(c, w, st)) != GK_OK) return rc;
+    if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, 0, (uint32_t)pages, mask_dev, first_bad_page_dev, st)) != GK_OK)
+        return rc;
+    c->stats.calls_restore++;
+    c->stats.jobs += n_jobs;
+    c->stats.pages += pages;
+    c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, uint8_t *mask_dev,
+                    int32_t *first_bad_page_dev, void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0) return GK_OK;
+    if (!jobs || !mask_dev || !first_bad_page_dev) return fail(c, GK_ERR_ARG, "null jobs, mask or first_bad_page");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    CacheDev cd;
+    int rc = check_cache(c, dst, &cd);
+    if (rc != GK_OK) return rc;
+
+    // sizes, pinned check, batch plan
+    struct Plan { uint64_t blob_bytes, sums_bytes, need; uint32_t pages; };
+    std::vector<Plan> plan(n_jobs);
+    uint64_t max_need = 0, total_need = 0, pages = 0;
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
+        const uint32_t np = (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+        plan[j].pages = np;
+        plan[j].blob_bytes = (uint64_t)np * c->gd.S + (uint64_t)jobs[j].n_tokens * c->gd.tokB;
+        plan[j].sums_bytes = (uint64_t)np * 8;
+        plan[j].need = 0;
+        pages += np;
+        if (jobs[j].blob && jobs[j].checksums) {
+            cudaPointerAttributes a{};
+            for (const void *ptr : {(const void *)jobs[j].blob, (const void *)jobs[j].checksums}) {
+                if (cudaPointerGetAttributes(&a, ptr) != cudaSuccess || a.type != cudaMemoryTypeHost) {
+                    cudaGetLastError();
+                    return fail(c, GK_ERR_NOT_PINNED, "job %u: blob and checksums must be pinned host memory", j);
+                }
+            }
+            plan[j].need = align_up(plan[j].blob_bytes, 256) + align_up(plan[j].sums_bytes, 256);
+        }
+        if (plan[j].need > max_need) max_need = plan[j].need;
+        total_need += plan[j].need;
+    }
+    // staging slots: room for the largest job, and for batches of small jobs up to 256 MiB
+    uint64_t want = max_need;
+    const uint64_t batch_target = 256ull << 20;
+    if (want < batch_target) want = total_need < batch_target ? total_need : batch_target;
+    if (want < 256) want = 256;
+    if (want > c->slot_cap) {
+        GK_CUDA(c, cudaDeviceSynchronize());
+        for (int i = 0; i < kSlots; ++i) {
+            if (c->d_slot[i]) cudaFree(c->d_slot[i]);
+            c->d_slot[i] = nullptr;
+            c->slot_used[i] = false;
+        }
+        c->slot_cap = 0;
+        for (int i = 0; i < kSlots; ++i) {
+            if (cudaMalloc(&c->d_slot[i], want) != cudaSuccess) {
+                cudaGetLastError();
+                return fail(c, GK_ERR_NOMEM, "host-tier staging slot of %llu bytes", (unsigned long long)want);
+            }
+        }
+        c->slot_cap = want;
+    }
+    // assign every job a place in a slot
+    std::vector<uint8_t *> blob_dev(n_jobs, nullptr);
+    std::vector<uint64_t *> sums_dev(n_jobs, nullptr);
+    std::vector<uint32_t> batch_end;  // exclusive job index per batch
+    {
+        uint64_t used = 0;
+        uint32_t b = 0;
+        for (uint32_t j = 0; j < n_jobs; ++j) {
+            if (used + plan[j].need > c->slot_cap && used > 0) {
+                batch_end.push_back(j);
+                ++b;
+                used = 0;
+            }
+            if (plan[j].need) {
+                uint8_t *base = c->d_slot[b % kSlots] + used;
+                blob_dev[j] = base;
+                sums_dev[j] = (uint64_t *)(base + align_up(plan[j].blob_bytes, 256));
+                used += plan[j].need;
+            }
+        }
+        batch_end.push_back(n_jobs);
+    }
+
+    const Tiling tlv = crc_tiling(c), tlc = commit_tiling(c);
+    const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
+    if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
+    uint64_t bytes = 0;
+    if ((rc = upload_jobs(c, jobs, n_jobs, l, blob_dev.data(), sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
+        return rc;
+    WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tlv);
+    if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
+    if ((rc = launch_claim(c, w, st)) != GK_OK) return rc;
+
+    uint32_t j0 = 0, page0 = 0;
+    for (size_t b = 0; b < batch_end.size(); ++b) {
+        const int slot = (int)(b % kSlots);
+        const uint32_t j1 = batch_end[b];
+        if (c->slot_used[slot]) GK_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_slot_free[slot], 0));
+        uint32_t npages = 0;
+        for (uint32_t j = j0; j < j1; ++j) {
+            npages += plan[j].pages;
+            if (!plan[j].need) continue;
+            GK_CUDA(c, cudaMemcpyAsync(blob_dev[j], jobs[j].blob, plan[j].blob_bytes, cudaMemcpyHostToDevice,
+                                       c->copy_stream));
+            GK_CUDA(c, cudaMemcpyAsync(sums_dev[j], jobs[j].checksums, plan[j].sums_bytes, cudaMemcpyHostToDevice,
+                                       c->copy_stream));
+        }
+        GK_CUDA(c, cudaEventRecord(c->ev_copied[slot], c->copy_stream));
+        GK_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied[slot], 0));
+        if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, page0, npages, mask_dev, first_bad_page_dev, st)) != GK_OK)
+            return rc;
+        GK_CUDA(c, cudaEventRecord(c->ev_slot_free[slot], st));
+        c->slot_used[slot] = true;
+        j0 = j1;
+        page0 += npages;
+    }
+    c->stats.calls_restore_host++;
+    c->stats.jobs += n_jobs;
+    c->stats.pages += pages;
+    c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+int gk_get_stats(gk_ctx *c, gk_stats *out)
+{
+    if (!c || !out) return GK_ERR_ARG;
+    DeviceGuard guard(c->device);
+    uint32_t e = 0;
+    GK_CUDA(c, cudaMemcpy(&e, c->d_error, 4, cudaMemcpyDeviceToHost));
+    c->stats.device_wait_expired = e;
+    *out = c->stats;
+    return GK_OK;
+}
+
+}  // extern "C"

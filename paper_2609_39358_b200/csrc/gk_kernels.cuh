@@ -1,0 +1,554 @@
+// gk_kernels.cuh -- the kernels of libgk (sm_100a).
+//
+//   validate_kernel   page ids in range, missing records, page -> job map
+//   claim_kernel      a destination page may be claimed once per call
+//   stream_kernel<>   one warp-specialised streaming kernel in three modes:
+//                       kVerify : blob -> smem -> CRC segment remainders
+//                       kPack   : cache slabs -> smem -> CRC + blob
+//                       kCommit : blob -> smem -> cache slabs (no CRC)
+//   finalize_kernel   segment remainders -> page CRC-64/XZ; compare or write
+//
+// The CRC is computed bit-sliced: a thread reads the words t, t+NT, t+2NT, ...
+// of a segment, and each of the 32 bit positions of those words is treated as
+// an independent bit stream (stride 32*NT bits, a power of two).  64 registers
+// hold the 64 remainder coefficients of the 32 streams, so one step of the
+// shift register costs a handful of 32-wide XORs.  Because squaring is linear
+// over GF(2), a stream M(x^(2^e)) has remainder (M(x) mod P)^(2^e) mod P: the
+// streams are reduced with the plain shift register and the 2^e-th power map,
+// a fixed 64x64 bit matrix, is applied once per thread per segment.  The
+// streams of a thread, the threads of a CTA and the segments of a page are then
+// merged by multiplying each remainder by x^(distance to the end) mod P.
+#pragma once
+
+#include "gk_device.cuh"
+#include "gk_gf2_generated.inc"
+
+namespace gk {
+
+// ---------------------------------------------------------------------------
+// small kernels
+// ---------------------------------------------------------------------------
+// One CTA per job.  Initialises the job's result words, records the lowest
+// out-of-range page id and fills page_job.  All CTAs together clear the claim
+// words of the destination cache.
+__global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims)
+{
+    const uint32_t j = blockIdx.x;
+    if (clear_claims) {
+        for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < num_pages;
+             i += (uint64_t)gridDim.x * blockDim.x)
+            w.claims[i] = 0ull;
+    }
+    if (j >= w.n_jobs) return;
+    const JobDev jb = w.jobs[j];
+    __shared__ int32_t s_bad;
+    if (threadIdx.x == 0) s_bad = kNoPage;
+    __syncthreads();
+    int32_t bad = kNoPage;
+    for (uint32_t p = threadIdx.x; p < jb.n_pages; p += blockDim.x) {
+        w.page_job[jb.page_base + p] = (int32_t)j;
+        if (jb.page_table) {
+            const int32_t id = jb.page_table[p];
+            if ((id < 0 || (uint64_t)id >= num_pages) && (int32_t)p < bad) bad = (int32_t)p;
+        }
+    }
+    if (bad != kNoPage) atomicMin(&s_bad, bad);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        w.bad_range[j] = s_bad;
+        w.bad_dup[j] = kNoPage;
+        w.bad_crc[j] = kNoPage;
+    }
+}
+
+// One thread per page of the call.  The first job to claim a destination page
+// leaves (job+1, index) in its claim word; every later claimant marks itself
+// and that first claimant.  Jobs that are missing or already failed the range
+// check claim nothing.
+__global__ void claim_kernel(WorkDev w)
+{
+    const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
+    if (g >= w.total_pages) return;
+    const uint32_t j = (uint32_t)w.page_job[g];
+    const JobDev jb = w.jobs[j];
+    if (jb.missing || w.bad_range[j] != kNoPage) return;
+    const uint32_t p = g - jb.page_base;
+    const int32_t id = jb.page_table[p];
+    const unsigned long long mine = ((unsigned long long)(j + 1u) << 32) | p;
+    const unsigned long long old = atomicCAS(&w.claims[id], 0ull, mine);
+    if (old != 0ull) {
+        atomicMin(&w.bad_dup[j], (int32_t)p);
+        atomicMin(&w.bad_dup[(uint32_t)(old >> 32) - 1u], (int32_t)(old & 0xffffffffull));
+    }
+}
+
+// Result code of a job from the words the earlier kernels left.
+__device__ __forceinline__ uint32_t job_code(const WorkDev &w, uint32_t j, int32_t *first_bad)
+{
+    *first_bad = -1;
+    if (w.jobs[j].missing) return 3u;
+    int32_t r = w.bad_range[j];
+    if (r == kNoPage) r = w.bad_dup[j];
+    if (r != kNoPage) {
+        *first_bad = r;
+        return 2u;
+    }
+    r = w.bad_crc[j];
+    if (r != kNoPage) {
+        *first_bad = r;
+        return 1u;
+    }
+    if (*w.error != 0u) return 4u;
+    return 0u;
+}
+
+// One thread per page.  Merges the page's segment remainders (Horner with
+// x^(8*segment bytes)), adds the term of the all-ones initial register and
+// the final xor, reflects, and either writes the checksum (write_mode) or
+// compares it with the stored one.
+__global__ void finalize_kernel(GeomDev g, WorkDev w, Tiling tl, int write_mode, uint8_t *status_out)
+{
+    const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= w.total_pages) return;
+    const uint32_t gp = w.page_begin + idx;
+    const uint32_t j = (uint32_t)w.page_job[gp];
+    const JobDev jb = w.jobs[j];
+    const uint32_t p = gp - jb.page_base;
+    const bool bad_table = w.bad_range[j] != kNoPage;
+    if (write_mode && p == 0u && status_out) status_out[j] = bad_table ? 2u : 0u;
+    if (jb.missing || bad_table) return;
+    if (!write_mode && w.bad_dup[j] != kNoPage) return;
+    const PageShape sh = page_shape(g, jb, p, tl);
+    const uint64_t *res = w.seg_res + (uint64_t)gp * tl.nseg_max;
+    uint64_t r = res[0];
+    for (uint32_t q = 1; q < sh.nseg; ++q) r = gf_mul(r, w.x_seg) ^ res[q];
+    const uint64_t crc = __brevll(r ^ w.init_term[sh.t] ^ ~0ull);
+    if (write_mode) {
+        jb.checksums[p] = crc;
+    } else if (crc != jb.checksums[p]) {
+        atomicMin(&w.bad_crc[j], (int32_t)p);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// the streaming kernel
+// ---------------------------------------------------------------------------
+template <int MODE, int NT, int STAGE_BYTES, int STAGES>
+struct StreamCfg {
+    static constexpr bool kCrc = (MODE != kCommit);
+    static constexpr bool kStore = (MODE != kVerify);
+    static constexpr int kConsWarps = kCrc ? NT / 32 : 0;
+    static constexpr int kLoaderWarp = kConsWarps;
+    static constexpr int kStorerWarp = kConsWarps + 1;
+    static constexpr int kThreads = 32 * (kConsWarps + 1 + (kStore ? 1 : 0));
+    static constexpr int kGran = kCrc ? NT * 256 : STAGE_BYTES;  // 8 shift-register steps of 8 words per thread
+    static constexpr int kSps = kCrc ? STAGE_BYTES / (NT * 32) : 1;  // 8-word steps per stage
+    static constexpr int kTilesPerGran = kGran / STAGE_BYTES;
+    static constexpr size_t kSmemBytes = (size_t)STAGES * STAGE_BYTES + 2 * STAGES * 8 + 2 * 8 * 8 + 16 + 128;
+    static_assert(!kCrc || (NT == 32 || NT == 64 || NT == 128 || NT == 256), "NT must be a power of two");
+    static_assert(!kCrc || (STAGE_BYTES % (NT * 32) == 0 && (NT * 256) % STAGE_BYTES == 0), "stage/step mismatch");
+    static_assert(STAGE_BYTES % 128 == 0, "stage alignment");
+};
+
+struct StreamParams {
+    GeomDev g;
+    CacheDev cache;   // kPack: source cache; kCommit: destination cache; kVerify: unused
+    WorkDev w;
+    Tiling tl;
+    uint32_t n_items; // total_pages * nseg_max
+    uint8_t *mask_out;        // kCommit
+    int32_t *first_bad_out;   // kCommit
+};
+
+struct Item {
+    const JobDev *jb;
+    uint32_t j, p, q;
+    uint32_t gp;   // page index within the call
+    uint32_t pad;
+    uint32_t tile_begin, tile_count;
+    int32_t phys;
+    uint32_t t;
+};
+
+template <int MODE>
+__device__ __forceinline__ bool get_item(const StreamParams &P, uint32_t item, Item &it, bool report)
+{
+    const uint32_t local = item / P.tl.nseg_max;
+    it.q = item - local * P.tl.nseg_max;
+    const uint32_t gp = P.w.page_begin + local;
+    it.gp = gp;
+    it.j = (uint32_t)P.w.page_job[gp];
+    it.jb = &P.w.jobs[it.j];
+    const JobDev jb = *it.jb;
+    it.p = gp - jb.page_base;
+    if (MODE == kCommit) {
+        int32_t fb;
+        const uint32_t code = job_code(P.w, it.j, &fb);
+        if (report && it.p == 0u && it.q == 0u) {
+            P.mask_out[it.j] = (uint8_t)code;
+            P.first_bad_out[it.j] = fb;
+        }
+        if (code != 0u) return false;
+    } else {
+        if (jb.missing || P.w.bad_range[it.j] != kNoPage) return false;
+        if (MODE == kVerify && P.w.bad_dup[it.j] != kNoPage) return false;
+    }
+    const PageShape sh = page_shape(P.g, jb, it.p, P.tl);
+    if (it.q >= sh.nseg) return false;
+    it.pad = sh.pad;
+    it.t = sh.t;
+    it.tile_begin = it.q == 0u ? 0u : sh.ntiles0 + (it.q - 1u) * P.tl.seg_tiles;
+    it.tile_count = it.q == 0u ? sh.ntiles0 : P.tl.seg_tiles;
+    it.phys = (MODE != kVerify) ? jb.page_table[it.p] : 0;
+    return true;
+}
+
+// Byte range of a tile inside its record: `lead` zero bytes first (front
+// padding), then `nreal` record bytes starting at record offset r0.
+template <int STAGE_BYTES>
+__device__ __forceinline__ void tile_range(uint32_t tile, uint32_t pad, uint32_t &lead, uint64_t &r0, uint32_t &nreal)
+{
+    const uint64_t v0 = (uint64_t)tile * STAGE_BYTES;
+    lead = 0u;
+    if (v0 < pad) lead = (pad - v0 >= (uint64_t)STAGE_BYTES) ? (uint32_t)STAGE_BYTES : (uint32_t)(pad - v0);
+    r0 = v0 + lead - pad;
+    nreal = (uint32_t)STAGE_BYTES - lead;
+}
+
+__device__ __forceinline__ uint8_t *slab_addr(const CacheDev &c, uint32_t slab, int32_t phys, uint64_t off)
+{
+    return c.data + (uint64_t)(slab >> 1) * c.layer_stride + (uint64_t)(slab & 1u) * c.kv_stride +
+           (uint64_t)phys * c.page_stride + off;
+}
+
+__device__ __forceinline__ uint8_t *scale_addr(const GeomDev &g, const CacheDev &c, uint32_t idx, int32_t phys)
+{
+    // idx counts fp32 values of a scale section: [layer][kv < scale_kv][head]
+    const uint32_t h = idx % g.kv_heads;
+    const uint32_t lk = idx / g.kv_heads;
+    const uint32_t kv = lk % g.scale_kv;
+    const uint32_t l = lk / g.scale_kv;
+    return c.scales + (uint64_t)l * c.s_layer_stride + (uint64_t)kv * c.s_kv_stride +
+           (uint64_t)phys * c.s_page_stride + 4ull * h;
+}
+
+// One 8-bit step of the bit-sliced shift register: state <- state*x^8 + w(x) mod P
+// for 32 streams at once.  U (0..7) is the number of steps taken since the
+// registers were last in natural order; coefficient m lives in R[(m - 8U) & 63],
+// so the shift itself costs nothing.  The eight top coefficients T[j] each add
+// x^(64+j) mod P; their sixteen-by-two partial sums are shared by all outputs.
+template <int U>
+__device__ __forceinline__ void crc_step8(uint32_t (&R)[64], const uint32_t (&w)[8])
+{
+    constexpr uint64_t G[8] = GK_G8_INIT;
+    uint32_t A[16], B[16];
+    A[0] = 0u;
+    B[0] = 0u;
+#pragma unroll
+    for (int pat = 1; pat < 16; ++pat) {
+        const int low = pat & (-pat);
+        const int bit = (low == 1) ? 0 : (low == 2) ? 1 : (low == 4) ? 2 : 3;
+        A[pat] = A[pat ^ low] ^ R[(56 + bit - 8 * U) & 63];
+        B[pat] = B[pat ^ low] ^ R[(60 + bit - 8 * U) & 63];
+    }
+#pragma unroll
+    for (int m = 0; m < 64; ++m) {
+        const int pa = (int)(((G[0] >> m) & 1ull) | (((G[1] >> m) & 1ull) << 1) | (((G[2] >> m) & 1ull) << 2) |
+                             (((G[3] >> m) & 1ull) << 3));
+        const int pb = (int)(((G[4] >> m) & 1ull) | (((G[5] >> m) & 1ull) << 1) | (((G[6] >> m) & 1ull) << 2) |
+                             (((G[7] >> m) & 1ull) << 3));
+        const uint32_t fb = A[pa] ^ B[pb];
+        const int phys = (m - 8 - 8 * U) & 63;
+        if (m < 8)
+            R[phys] = w[7 - m] ^ fb;
+        else
+            R[phys] ^= fb;
+    }
+}
+
+template <int NT>
+struct FrobExp;
+template <> struct FrobExp<32> { static constexpr int e = 10; };
+template <> struct FrobExp<64> { static constexpr int e = 11; };
+template <> struct FrobExp<128> { static constexpr int e = 12; };
+template <> struct FrobExp<256> { static constexpr int e = 13; };
+
+// Remainder of one thread's 32 streams, already placed at the thread's distance
+// from the end of the segment and multiplied by x^64:
+//   x^(32*(NT-1-t)+64) * sum_s x^(31-s) * (R_s)^(32*NT)   mod P
+template <int NT>
+__device__ __forceinline__ uint64_t thread_remainder(const uint32_t (&R)[64], uint64_t kt)
+{
+    uint32_t Q[64];
+    gk_frob<FrobExp<NT>::e>(R, Q);
+    // sum_s x^(31-s) * Q_s: bit s of Q[k] is the coefficient of x^(k+31-s)
+    uint32_t a0 = 0u, a1 = 0u, a2 = 0u;
+#pragma unroll
+    for (int k = 0; k < 64; ++k) {
+        const uint32_t v = __brev(Q[k]);
+        const int sh = k & 31;
+        const uint32_t lo = v << sh;
+        const uint32_t hi = sh ? (v >> (32 - sh)) : 0u;
+        if (k < 32) {
+            a0 ^= lo;
+            a1 ^= hi;
+        } else {
+            a1 ^= lo;
+            a2 ^= hi;
+        }
+    }
+    // fold degrees 64..94 back
+    uint64_t lo64 = ((uint64_t)a1 << 32) | a0;
+    uint32_t hi = a2;
+#pragma unroll
+    for (int b = 30; b >= 0; --b) {
+        if ((hi >> b) & 1u) {
+            lo64 ^= kPoly << b;
+            if (b) hi ^= (uint32_t)(kPoly >> (64 - b));
+        }
+    }
+    return gf_mul(kt, lo64);
+}
+
+// The eight 8-word steps of one granule (after which the registers are back in
+// natural order).  Every kSps steps a new stage is awaited and the finished one
+// is handed back to the loader.
+template <int U, int MODE, int NT, int STAGE_BYTES, int STAGES>
+struct GranuleSteps {
+    using Cfg = StreamCfg<MODE, NT, STAGE_BYTES, STAGES>;
+    static __device__ __forceinline__ void run(uint32_t (&R)[64], const uint8_t *smem, uint32_t full0, uint32_t empty0,
+                                               uint32_t &n, volatile uint32_t *abort_flag, uint32_t *error, int tid,
+                                               int lane)
+    {
+        const uint32_t s = n % STAGES;
+        if (U % Cfg::kSps == 0)
+            mbar_wait(full0 + 8u * s, (n / STAGES) & 1u, abort_flag, error, 0x400u | MODE);
+        const uint32_t *sw = reinterpret_cast<const uint32_t *>(smem + (size_t)s * STAGE_BYTES) + tid;
+        uint32_t w[8];
+#pragma unroll
+        for (int jw = 0; jw < 8; ++jw) w[jw] = sw[((U % Cfg::kSps) * 8 + jw) * NT];
+        crc_step8<U>(R, w);
+        if (U % Cfg::kSps == Cfg::kSps - 1) {
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty0 + 8u * s);
+            ++n;
+        }
+        GranuleSteps<U + 1, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, n, abort_flag, error, tid, lane);
+    }
+};
+template <int MODE, int NT, int STAGE_BYTES, int STAGES>
+struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES> {
+    static __device__ __forceinline__ void run(uint32_t (&)[64], const uint8_t *, uint32_t, uint32_t, uint32_t &,
+                                               volatile uint32_t *, uint32_t *, int, int)
+    {
+    }
+};
+
+template <int MODE, int NT, int STAGE_BYTES, int STAGES, int MINB>
+__global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThreads, MINB)
+    stream_kernel(const __grid_constant__ StreamParams P)
+{
+    using Cfg = StreamCfg<MODE, NT, STAGE_BYTES, STAGES>;
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
+    uint64_t *red = bars + 2 * STAGES;                 // [2][8]
+    volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const uint32_t stage0 = smem_u32(smem);
+    const uint32_t full0 = smem_u32(bars);
+    const uint32_t empty0 = smem_u32(bars + STAGES);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(full0 + 8u * s, 1u);
+            mbar_init(empty0 + 8u * s, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)));
+        }
+        *abort_flag = 0u;
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    if (warp == Cfg::kLoaderWarp) {
+        // ------------------------------ loader ------------------------------
+        uint32_t n = 0;
+        uint64_t policy = 0;
+        if (MODE == kCommit || MODE == kPack) policy = policy_evict_first();
+        for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+            Item it;
+            if (!get_item<MODE>(P, item, it, false)) continue;
+            const uint8_t *rec = (MODE == kPack) ? nullptr : it.jb->blob + (uint64_t)it.p * P.g.R;
+            const uint32_t slab_len = it.t * P.g.row;
+            for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
+                const uint32_t s = n % STAGES;
+                const uint32_t use = n / STAGES;
+                if (use > 0u) mbar_wait(empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE);
+                uint32_t lead, nreal;
+                uint64_t r0;
+                tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
+                const uint32_t sbase = stage0 + s * STAGE_BYTES;
+                uint8_t *sgen = smem + (size_t)s * STAGE_BYTES;
+                if (Cfg::kCrc) {
+                    for (uint32_t o = lane * 16u; o < lead; o += 512u)
+                        *reinterpret_cast<uint4 *>(sgen + o) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                uint32_t scale_bytes = 0u;
+                if (MODE == kPack && r0 < P.g.S && nreal > 0u) {
+                    // scale values of this tile: gathered with ordinary loads
+                    const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
+                    scale_bytes = (uint32_t)(e1 - r0);
+                    for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
+                        const uint32_t v = *reinterpret_cast<const uint32_t *>(scale_addr(P.g, P.cache, i, it.phys));
+                        *reinterpret_cast<uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0)) = v;
+                    }
+                    fence_proxy_async_smem();
+                }
+                __syncwarp();
+                if (lane == 0 && !*abort_flag) {
+                    const uint32_t bar = full0 + 8u * s;
+                    if (MODE == kPack) {
+                        const uint32_t data_bytes = nreal - scale_bytes;
+                        if (data_bytes == 0u) {
+                            mbar_arrive(bar);
+                        } else {
+                            mbar_arrive_expect_tx(bar, data_bytes);
+                            uint64_t d0 = r0 + scale_bytes - P.g.S;  // offset in the record's data part
+                            const uint64_t d1 = d0 + data_bytes;
+                            uint32_t so = sbase + lead + scale_bytes;
+                            uint32_t slab = (uint32_t)(d0 / slab_len);
+                            uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
+                            while (d0 < d1) {
+                                uint32_t nb = slab_len - off;
+                                if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
+                                bulk_g2s_hint(so, slab_addr(P.cache, slab, it.phys, off), nb, bar, policy);
+                                d0 += nb;
+                                so += nb;
+                                ++slab;
+                                off = 0u;
+                            }
+                        }
+                    } else {
+                        if (nreal == 0u) {
+                            mbar_arrive(bar);
+                        } else {
+                            mbar_arrive_expect_tx(bar, nreal);
+                            if (MODE == kCommit)
+                                bulk_g2s_hint(sbase + lead, rec + r0, nreal, bar, policy);
+                            else
+                                bulk_g2s(sbase + lead, rec + r0, nreal, bar);
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        // before leaving: every load this CTA issued must have landed
+        if (lane == 0) {
+            for (uint32_t back = 0; back < (uint32_t)STAGES && back < n; ++back) {
+                const uint32_t m = n - 1u - back;
+                mbar_drain(full0 + 8u * (m % STAGES), (m / STAGES) & 1u);
+            }
+        }
+    } else if (Cfg::kStore && warp == Cfg::kStorerWarp) {
+        // ------------------------------ storer ------------------------------
+        uint32_t n = 0;
+        for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+            Item it;
+            if (!get_item<MODE>(P, item, it, lane == 0)) continue;
+            uint8_t *rec = it.jb->blob + (uint64_t)it.p * P.g.R;
+            const uint32_t slab_len = it.t * P.g.row;
+            for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
+                const uint32_t s = n % STAGES;
+                const bool ok = mbar_wait(full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE);
+                uint32_t lead, nreal;
+                uint64_t r0;
+                tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
+                const uint32_t sbase = stage0 + s * STAGE_BYTES;
+                const uint8_t *sgen = smem + (size_t)s * STAGE_BYTES;
+                uint32_t scale_bytes = 0u;
+                if (MODE == kCommit && r0 < P.g.S && nreal > 0u) {
+                    const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
+                    scale_bytes = (uint32_t)(e1 - r0);
+                    if (ok && !*abort_flag) {
+                        for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
+                            const uint32_t v =
+                                *reinterpret_cast<const uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0));
+                            *reinterpret_cast<uint32_t *>(scale_addr(P.g, P.cache, i, it.phys)) = v;
+                        }
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    if (ok && !*abort_flag && nreal > 0u) {
+                        if (MODE == kPack) {
+                            bulk_s2g(rec + r0, sbase + lead, nreal);
+                        } else {
+                            const uint32_t data_bytes = nreal - scale_bytes;
+                            uint64_t d0 = r0 + scale_bytes - P.g.S;
+                            const uint64_t d1 = d0 + data_bytes;
+                            uint32_t so = sbase + lead + scale_bytes;
+                            uint32_t slab = (uint32_t)(d0 / slab_len);
+                            uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
+                            while (d0 < d1) {
+                                uint32_t nb = slab_len - off;
+                                if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
+                                bulk_s2g(slab_addr(P.cache, slab, it.phys, off), so, nb);
+                                d0 += nb;
+                                so += nb;
+                                ++slab;
+                                off = 0u;
+                            }
+                        }
+                    }
+                    bulk_commit();
+                    // the store of the previous tile has finished reading its stage
+                    if (n > 0u) {
+                        bulk_wait_read<1>();
+                        mbar_arrive(empty0 + 8u * ((n - 1u) % STAGES));
+                    }
+                }
+                __syncwarp();
+            }
+        }
+        if (lane == 0) {
+            bulk_wait_all();
+            if (n > 0u) mbar_arrive(empty0 + 8u * ((n - 1u) % STAGES));
+        }
+    } else if constexpr (Cfg::kCrc) {
+        // ----------------------------- consumers ----------------------------
+        const int tid = threadIdx.x;  // consumer warps come first: 0..NT-1
+        const uint64_t kt = P.w.thread_const[tid];
+        uint32_t n = 0;
+        uint32_t parity_red = 0;
+        for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+            Item it;
+            if (!get_item<MODE>(P, item, it, false)) continue;
+            uint32_t R[64];
+#pragma unroll
+            for (int i = 0; i < 64; ++i) R[i] = 0u;
+            const uint32_t ngran = it.tile_count / Cfg::kTilesPerGran;
+            for (uint32_t gi = 0; gi < ngran; ++gi)
+                GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, n, abort_flag, P.w.error, tid,
+                                                                    lane);
+            // merge streams -> thread -> warp -> CTA
+            uint64_t v = thread_remainder<NT>(R, kt);
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) v ^= __shfl_xor_sync(0xffffffffu, v, d);
+            uint64_t *slot = red + 8 * parity_red;
+            if (lane == 0) slot[warp] = v;
+            asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
+            if (tid == 0) {
+                uint64_t tot = 0;
+#pragma unroll
+                for (int i = 0; i < Cfg::kConsWarps; ++i) tot ^= slot[i];
+                P.w.seg_res[(uint64_t)it.gp * P.tl.nseg_max + it.q] = tot;
+            }
+            parity_red ^= 1u;
+        }
+    }
+    __syncthreads();
+}
+
+}  // namespace gk

@@ -1,0 +1,152 @@
+"""CPU-side checks of the product: the shared library loads and exports every
+entry point the public header declares, size arithmetic agrees with the oracle,
+argument checks answer without a GPU, and the generated GF(2) tables are what
+the kernels' algebra needs (checked with independent big-integer arithmetic)."""
+import ctypes
+import importlib.util
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+import synth
+from helpers import oracle_geom
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def gk():
+    from paper_2609_39358_b200 import build
+    build.build()
+    import paper_2609_39358_b200 as m
+    return m
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "gk.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(gk_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(gk):
+    lib = gk.load_library()
+    names = _declared_functions()
+    assert "gk_pack" in names and "gk_restore" in names and "gk_restore_host" in names
+    for name in names:
+        assert hasattr(lib, name), name
+    from paper_2609_39358_b200 import binding
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_blob_size_matches_oracle_on_all_workloads(gk):
+    from gpu_harness import gk_geom
+    cases = [(synth.TINY, 256), (synth.GQA7B, 4096), (synth.CORPUS, 1024), (synth.CORPUS, 280),
+             (synth.FP8, 2048), (synth.STRESS, 17), (synth.STRESS, 4096), (synth.STRESS, 555)]
+    for w, n in cases:
+        og = oracle_geom(w)
+        assert gk.gk_blob_size(gk_geom(og), n) == oracle.blob_size(og, n)
+
+
+def test_argument_checks_without_gpu(gk):
+    with pytest.raises(gk.GkError) as e:
+        gk.gk_blob_size(gk.Geom(2, 2, 64, 16), 0)
+    assert e.value.code == -1
+    with pytest.raises(gk.GkError) as e:
+        gk.gk_blob_size(gk.Geom(2, 2, 64, 16, dtype=7), 16)
+    assert e.value.code == -2
+    with pytest.raises(gk.GkError) as e:
+        gk.gk_blob_size(gk.Geom(2, 1, 4, 16), 16)          # row = 8 bytes
+    assert e.value.code == -2
+    with pytest.raises(gk.GkError):
+        gk.gk_blob_size(gk.Geom(2, 2, 64, 16, scale_kv=2), 16)   # bf16 has no scales
+    import torch
+    if not torch.cuda.is_available():
+        with pytest.raises(gk.GkError):                    # no device: fails loudly, no fallback
+            gk.Context(gk.Geom(2, 2, 64, 16), 0)
+
+
+# ---------------------------------------------------------------------------
+# generated tables
+# ---------------------------------------------------------------------------
+P_FULL = (1 << 64) | 0x42F0E1EBA9EA3693
+
+
+def _mod(v):
+    while v.bit_length() > 64:
+        v ^= P_FULL << (v.bit_length() - 65)
+    return v
+
+
+def _clmul(a, b):
+    r = 0
+    while b:
+        if b & 1:
+            r ^= a
+        a <<= 1
+        b >>= 1
+    return r
+
+
+def _load_gen():
+    spec = importlib.util.spec_from_file_location(
+        "gen_tables", os.path.join(ROOT, "paper_2609_39358_b200", "csrc", "gen_tables.py"))
+    m = importlib.util.module_from_spec(spec)
+    spec.loader.exec_module(m)
+    return m
+
+
+def test_frobenius_rows_are_repeated_squaring():
+    gen = _load_gen()
+    rng = np.random.default_rng(5)
+    for e in (10, 11, 12, 13):
+        rows = gen.frob_rows(e)
+        for _ in range(20):
+            r = int(rng.integers(0, 1 << 63)) | (int(rng.integers(0, 2)) << 63)
+            want = r
+            for _ in range(e):
+                want = _mod(_clmul(want, want))
+            got = 0
+            for m in range(64):
+                if bin(rows[m] & r).count("1") & 1:
+                    got |= 1 << m
+            assert got == want
+
+
+def test_generated_file_is_current_and_g8_constants():
+    gen = _load_gen()
+    path = os.path.join(ROOT, "paper_2609_39358_b200", "csrc", "gk_gf2_generated.inc")
+    text = open(path).read()
+    assert text == gen.generate()
+    vals = [int(v, 16) for v in re.findall(r"0x([0-9A-F]{16})ull", text.split("GK_G8_INIT")[1].split("\n")[0])]
+    assert len(vals) == 8
+    for j, v in enumerate(vals):
+        assert v == _mod(1 << (64 + j))
+
+
+def test_bit_sliced_scheme_reproduces_crc():
+    """The kernels' algebra, restated with Python integers: 8 threads, streams of
+    stride 32*8 bits reduced by a plain shift register, raised to the 2^8-th power,
+    merged with x^(distance) factors, plus init and final-xor terms."""
+    gen = _load_gen()
+    NT, e = 8, 8
+    rng = np.random.default_rng(6)
+    data = rng.integers(0, 256, size=NT * 4 * 24, dtype=np.uint8).tobytes()
+    words = [int.from_bytes(data[4 * i:4 * i + 4], "little") for i in range(len(data) // 4)]
+    total = 0
+    for t in range(NT):
+        acc = 0
+        for s in range(32):
+            r = 0
+            for w in words[t::NT]:
+                r = _mod((r << 1) | ((w >> s) & 1))
+            for _ in range(e):
+                r = _mod(_clmul(r, r))
+            acc ^= r << (31 - s)
+        total ^= _mod(_clmul(_mod(acc), _mod(1 << (32 * (NT - 1 - t) + 64))))
+    ones = (1 << 64) - 1
+    init = _mod(_clmul(ones, gen.xpow(8 * len(data))))
+    crc = int(format(total ^ init ^ ones, "064b")[::-1], 2)
+    assert crc == oracle.crc64(data)

@@ -1,0 +1,383 @@
+"""GPU parity: libgk (through its C ABI) against the CPU oracle, bit for bit --
+blob bytes, page checksums, result codes, first failing page, and the full
+destination cache image (so that "nothing written" is checked byte by byte).
+Sizes here are small enough for the oracle to finish in seconds yet span
+several 32 KiB granules, several segments and ragged tails."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import synth
+from helpers import (cache_bytes, clone_cache, make_cache, n_pages, oracle_geom, random_cache)
+
+pytestmark = pytest.mark.gpu
+
+G_TINY = oracle.Geom(2, 2, 64, 16, 2, 0)           # record 16 KiB: half a granule
+G_MID = oracle.Geom(5, 4, 64, 16, 2, 0)            # record 80 KiB: 2.5 granules
+G_BIG = oracle.Geom(16, 8, 128, 16, 2, 0)          # record 1 MiB
+G_FP8_S = oracle.Geom(6, 4, 32, 8, 1, 2)           # record 12,480 B, scale section 192 B
+G_FP8_M = oracle.Geom(10, 8, 64, 32, 1, 2)         # record 328,320 B, scale section 640 B
+G_FP8_1 = oracle.Geom(4, 4, 64, 16, 1, 1)          # shared K/V scale
+G_FP8_W = oracle.Geom(40, 64, 16, 8, 1, 2)         # scale section 20,480 B: spans several tiles
+ALL_GEOMS = [G_TINY, G_MID, G_BIG, G_FP8_S, G_FP8_M, G_FP8_1, G_FP8_W]
+
+
+@pytest.fixture(scope="module")
+def gk():
+    import paper_2609_39358_b200 as m
+    assert torch.cuda.is_available()
+    return m
+
+
+def _ctx(gk, og, flags=0, **tuning):
+    from gpu_harness import gk_geom
+    ctx = gk.Context(gk_geom(og, flags), 0)
+    for k, v in tuning.items():
+        ctx.set_tuning(k, v)
+    return ctx
+
+
+# ---------------------------------------------------------------------------
+# checksums of an existing blob
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("og", ALL_GEOMS)
+@pytest.mark.parametrize("seg", [0, 1, 2])
+def test_page_checksums(gk, og, seg):
+    from gpu_harness import sums_to_np
+    ctx = _ctx(gk, og, seg_granules=seg)
+    rng = np.random.default_rng(100 + seg)
+    for n_tokens in [1, og.page_tokens, 3 * og.page_tokens + 1, 5 * og.page_tokens - 1]:
+        nbytes, P = oracle.blob_size(og, n_tokens)
+        blob = rng.integers(0, 256, size=nbytes, dtype=np.uint8)
+        want = np.array([oracle.crc64(blob[oracle.record_offset(og, p):
+                                           oracle.record_offset(og, p) + oracle.record_bytes(og, n_tokens, p)])
+                         for p in range(P)], dtype=np.uint64)
+        d_blob = torch.from_numpy(blob).cuda()
+        d_sums = torch.zeros(P, dtype=torch.int64, device="cuda")
+        ctx.gk_page_checksums(d_blob, n_tokens, d_sums)
+        torch.cuda.synchronize()
+        assert np.array_equal(sums_to_np(d_sums), want)
+    ctx.close()
+
+
+def test_page_checksums_special_contents(gk):
+    """All-zero and all-ones records (the init and final-xor terms must be right
+    even when the data contribute nothing), and the catalogue check string
+    embedded at the very end of a record."""
+    from gpu_harness import sums_to_np
+    og = G_MID
+    ctx = _ctx(gk, og)
+    nbytes, P = oracle.blob_size(og, og.page_tokens)
+    for fill in (0x00, 0xFF):
+        blob = np.full(nbytes, fill, dtype=np.uint8)
+        d_sums = torch.zeros(P, dtype=torch.int64, device="cuda")
+        ctx.gk_page_checksums(torch.from_numpy(blob).cuda(), og.page_tokens, d_sums)
+        torch.cuda.synchronize()
+        assert int(sums_to_np(d_sums)[0]) == oracle.crc64(blob)
+    blob = np.zeros(nbytes, dtype=np.uint8)
+    blob[-9:] = np.frombuffer(b"123456789", dtype=np.uint8)
+    d_sums = torch.zeros(P, dtype=torch.int64, device="cuda")
+    ctx.gk_page_checksums(torch.from_numpy(blob).cuda(), og.page_tokens, d_sums)
+    torch.cuda.synchronize()
+    assert int(sums_to_np(d_sums)[0]) == oracle.crc64(blob)
+    ctx.close()
+
+
+# ---------------------------------------------------------------------------
+# pack
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("og", ALL_GEOMS)
+@pytest.mark.parametrize("layout", ["layer_major", "page_major"])
+def test_pack_parity(gk, og, layout):
+    from gpu_harness import dev_cache, gpu_pack
+    N = 23
+    src = random_cache(og, N, seed=200, layout=layout)
+    dsrc = dev_cache(src)
+    rng = np.random.default_rng(201)
+    T = og.page_tokens
+    lens = [1, T, T + 1, 4 * T, 6 * T - 1, 2 * T]
+    tables = [rng.integers(0, N, size=n_pages(og, n)).astype(np.int32) for n in lens]   # duplicates allowed
+    for seg in (0, 1):
+        ctx = _ctx(gk, og, seg_granules=seg)
+        got, status = gpu_pack(ctx, og, dsrc, tables, lens)
+        assert status.tolist() == [0] * len(lens)
+        for (blob, sums), pt, n in zip(got, tables, lens):
+            wb, ws, code, _ = oracle.pack(og, src, pt, n)
+            assert code == 0
+            assert np.array_equal(blob, wb), f"blob differs at {np.flatnonzero(blob != wb)[:8]}"
+            assert np.array_equal(sums, ws)
+        ctx.close()
+
+
+def test_pack_single_entry_point_and_bad_table(gk):
+    from gpu_harness import dev_cache, dev_i32, sums_to_np
+    og, N = G_MID, 9
+    src = random_cache(og, N, seed=210)
+    dsrc = dev_cache(src)
+    ctx = _ctx(gk, og)
+    n = 2 * og.page_tokens + 3
+    nbytes, P = oracle.blob_size(og, n)
+    pt = np.array([4, 0, 8], dtype=np.int32)
+    blob = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    sums = torch.zeros(P, dtype=torch.int64, device="cuda")
+    status = torch.full((1,), 255, dtype=torch.uint8, device="cuda")
+    ctx.gk_pack(dsrc, dev_i32(pt), n, blob, sums, status)
+    torch.cuda.synchronize()
+    wb, ws, _, _ = oracle.pack(og, src, pt, n)
+    assert status.item() == 0
+    assert np.array_equal(blob.cpu().numpy(), wb) and np.array_equal(sums_to_np(sums), ws)
+    # an id outside the cache: nothing written, status 2
+    for bad_id in (-1, N):
+        blob.fill_(0x5A)
+        sums.fill_(0x5A5A)
+        status.fill_(255)
+        ctx.gk_pack(dsrc, dev_i32(np.array([4, bad_id, 8])), n, blob, sums, status)
+        torch.cuda.synchronize()
+        assert status.item() == 2
+        assert bool((blob == 0x5A).all()) and bool((sums == 0x5A5A).all())
+    ctx.close()
+
+
+# ---------------------------------------------------------------------------
+# restore
+# ---------------------------------------------------------------------------
+def _oracle_jobs(og, src, lens, seed, dst_pages):
+    rng = np.random.default_rng(seed)
+    perm = rng.permutation(dst_pages).astype(np.int32)
+    jobs, used = [], 0
+    for n in lens:
+        P = n_pages(og, n)
+        spt = rng.integers(0, src.num_pages, size=P).astype(np.int32)
+        blob, sums, code, _ = oracle.pack(og, src, spt, n)
+        assert code == 0
+        jobs.append(oracle.Job(blob, sums, perm[used:used + P].copy(), n))
+        used += P
+    assert used <= dst_pages
+    return jobs
+
+
+@pytest.mark.parametrize("og", ALL_GEOMS)
+@pytest.mark.parametrize("host_tier", [False, True])
+def test_restore_parity_with_corruption(gk, og, host_tier):
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
+    T = og.page_tokens
+    src = random_cache(og, 17, seed=300)
+    lens = [3 * T, 1, 2 * T + 1, 5 * T, T, 4 * T - 1]
+    Nd = 40
+    jobs = _oracle_jobs(og, src, lens, 301, Nd)
+    # job 1: one flipped bit in the blob; job 3: one flipped bit in a checksum;
+    # job 5: damage in the last (partial) page only
+    jobs[1].blob[len(jobs[1].blob) // 2] ^= 0x10
+    jobs[3].checksums[2] ^= np.uint64(1 << 40)
+    jobs[5].blob[-1] ^= 0x01
+    clean = random_cache(og, Nd, seed=302)
+    for tuning in ({}, {"seg_granules": 1, "commit_seg_tiles": 1}, {"grid_cap": 3}):
+        ctx = _ctx(gk, og, **tuning)
+        want = clone_cache(clean)
+        wmask, wfb = oracle.restore(og, want, jobs)
+        assert wmask.tolist() == [0, 1, 0, 1, 0, 1]
+        d = dev_cache(clean)
+        mask, fb = gpu_restore(ctx, d, jobs, host_tier=host_tier)
+        assert mask.tolist() == wmask.tolist()
+        assert fb.tolist() == wfb.tolist()
+        assert_cache_equal(d, want)
+        ctx.close()
+
+
+def test_restore_codes_and_first_bad_page(gk):
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
+    og, N = G_MID, 12
+    src = random_cache(og, N, seed=310)
+    T = og.page_tokens
+    n = 3 * T
+    blob, sums, _, _ = oracle.pack(og, src, np.array([0, 1, 2], dtype=np.int32), n)
+    blob1, sums1, _, _ = oracle.pack(og, src, np.array([0], dtype=np.int32), 1)
+    bad2 = blob.copy()
+    bad2[oracle.record_offset(og, 1) + 5] ^= 1
+    bad2[oracle.record_offset(og, 2) + 5] ^= 1
+    clean = random_cache(og, N, seed=311)
+    i32 = lambda *v: np.array(v, dtype=np.int32)
+    jobs = [
+        oracle.Job(blob, sums, i32(0, 1, 2), n),
+        oracle.Job(bad2, sums, i32(3, 4, 5), n),
+        oracle.Job(None, sums, i32(6, 7, 8), n),
+        oracle.Job(blob, None, i32(6, 7, 8), n),
+        oracle.Job(blob, sums, i32(9, 12, -1), n),
+        oracle.Job(blob, sums, i32(6, 10, 11), n),
+        oracle.Job(blob, sums, i32(8, 7, 10), n),
+        oracle.Job(blob1, sums1, i32(9), 1),
+    ]
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs)
+    assert wmask.tolist() == [0, 1, 3, 3, 2, 2, 2, 0]
+    ctx = _ctx(gk, og)
+    for host_tier in (False, True):
+        d = dev_cache(clean)
+        mask, fb = gpu_restore(ctx, d, jobs, host_tier=host_tier)
+        assert mask.tolist() == wmask.tolist()
+        assert fb.tolist() == wfb.tolist()
+        assert_cache_equal(d, want)
+    # a page claimed twice inside one job, and by three jobs
+    jobs2 = [
+        oracle.Job(blob, sums, i32(0, 1, 0), n),
+        oracle.Job(blob, sums, i32(2, 3, 4), n),
+        oracle.Job(blob, sums, i32(5, 4, 6), n),
+        oracle.Job(blob, sums, i32(7, 8, 4), n),
+        oracle.Job(blob, sums, i32(9, 10, 11), n),
+    ]
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs2)
+    assert wmask.tolist() == [2, 2, 2, 2, 0] and wfb.tolist() == [0, 2, 1, 2, -1]
+    d = dev_cache(clean)
+    mask, fb = gpu_restore(ctx, d, jobs2)
+    assert mask.tolist() == wmask.tolist() and fb.tolist() == wfb.tolist()
+    assert_cache_equal(d, want)
+    ctx.close()
+
+
+def test_sabotage_triple_on_gpu(gk):
+    """Defence on: rejected and untouched.  Defence off: the damaged bytes land.
+    Defence on again: rejected and untouched."""
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
+    og = G_MID
+    src = random_cache(og, 8, seed=320)
+    n = 2 * og.page_tokens + 5
+    jobs = _oracle_jobs(og, src, [n], 321, 8)
+    jobs[0].blob[12345] ^= 0x80
+    clean = random_cache(og, 8, seed=322)
+    for flags, want_code in ((0, 1), (oracle.FLAG_SKIP_VERIFY, 0), (0, 1)):
+        ctx = _ctx(gk, og, flags=flags)
+        want = clone_cache(clean)
+        wmask, _ = oracle.restore(og, want, jobs, flags=flags)
+        assert wmask.tolist() == [want_code]
+        d = dev_cache(clean)
+        mask, _ = gpu_restore(ctx, d, jobs)
+        assert mask.tolist() == [want_code]
+        assert_cache_equal(d, want)
+        changed = not np.array_equal(want.data, clean.data)
+        assert changed == (want_code == 0)
+        ctx.close()
+
+
+def test_tiny_workload(gk):
+    """4 blocks of 256 tokens, one flipped bit: 3 ok, 1 rejected with its pages untouched."""
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_pack, gpu_restore
+    w = synth.TINY
+    og = oracle_geom(w)
+    src_pages = 64
+    src = make_cache(og, src_pages,
+                     synth.kv_bytes_bf16(cache_bytes(og, src_pages) // 2, w.sigma, w.seed(0)).numpy())
+    dsrc = dev_cache(src)
+    ctx = _ctx(gk, og)
+    tables = [np.arange(16 * i, 16 * i + 16, dtype=np.int32) for i in range(4)]
+    packed, status = gpu_pack(ctx, og, dsrc, tables, synth.TINY_BLOCKS)
+    assert status.tolist() == [0, 0, 0, 0]
+    perm = synth.page_permutation(synth.TINY_DST_PAGES, w.seed(1))
+    jobs = []
+    for i, ((blob, sums), n) in enumerate(zip(packed, synth.TINY_BLOCKS)):
+        wb, ws, _, _ = oracle.pack(og, src, tables[i], n)
+        assert np.array_equal(blob, wb) and np.array_equal(sums, ws)
+        jobs.append(oracle.Job(blob.copy(), sums.copy(), perm[16 * i:16 * i + 16], n))
+    victim = int(np.random.default_rng(w.seed(2)).integers(0, 4))
+    bit = int(synth.bit_flip_positions(jobs[victim].blob.size * 8, 1, w.seed(3))[0])
+    jobs[victim].blob[bit >> 3] ^= 1 << (bit & 7)
+    clean = make_cache(og, synth.TINY_DST_PAGES,
+                       synth.sentinel_bytes(cache_bytes(og, synth.TINY_DST_PAGES), w.seed(4)).numpy().copy())
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs)
+    assert sorted(wmask.tolist()) == [0, 0, 0, 1]
+    d = dev_cache(clean)
+    mask, fb = gpu_restore(ctx, d, jobs)
+    assert mask.tolist() == wmask.tolist() and fb.tolist() == wfb.tolist()
+    assert_cache_equal(d, want)
+    ctx.close()
+
+
+def test_fp8_scale_and_data_corruption(gk):
+    """A run of damaged bytes inside a scale section of one blob and inside a K
+    slab of another: both rejected, their pages and scale entries untouched."""
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
+    og = G_FP8_M
+    T = og.page_tokens
+    Ns = 12
+    data, scales = synth.kv_bytes_fp8(og.layers, Ns, T, og.kv_heads, og.head_dim, 1.0, synth.FP8.seed(0))
+    src = make_cache(og, Ns, data.numpy().copy(), scales.view(torch.uint8).reshape(-1).numpy().copy())
+    lens = [2 * T] * 5
+    jobs = _oracle_jobs(og, src, lens, 331, 16)
+    S = og.layers * og.scale_kv * og.kv_heads * 4
+    rec = oracle.record_bytes(og, 2 * T, 0)
+    start, xors = synth.byte_run_corruption(rec, rec + S, 8, synth.FP8.seed(1))       # scale section of page 1
+    jobs[1].blob[start:start + 8] ^= xors
+    start, xors = synth.byte_run_corruption(S, S + T * og.kv_heads * og.head_dim, 8, synth.FP8.seed(2))  # K slab, layer 0, page 0
+    jobs[3].blob[start:start + 8] ^= xors
+    clean = random_cache(og, 16, seed=332)
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs)
+    assert wmask.tolist() == [0, 1, 0, 1, 0] and wfb.tolist() == [-1, 1, -1, 0, -1]
+    ctx = _ctx(gk, og)
+    d = dev_cache(clean)
+    mask, fb = gpu_restore(ctx, d, jobs)
+    assert mask.tolist() == wmask.tolist() and fb.tolist() == wfb.tolist()
+    assert_cache_equal(d, want)
+    ctx.close()
+
+
+def test_round_trip_on_gpu_only_path(gk):
+    """restore(pack(x)) == x through libgk alone, then checked against the source bytes."""
+    from gpu_harness import dev_cache, dev_i32
+    og = G_BIG
+    N = 24
+    src = random_cache(og, N, seed=340)
+    dsrc = dev_cache(src)
+    ctx = _ctx(gk, og)
+    n = 10 * og.page_tokens + 7
+    P = n_pages(og, n)
+    nbytes, _ = oracle.blob_size(og, n)
+    spt = np.random.default_rng(341).permutation(N)[:P].astype(np.int32)
+    dpt = np.random.default_rng(342).permutation(N)[:P].astype(np.int32)
+    blob = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+    sums = torch.zeros(P, dtype=torch.int64, device="cuda")
+    ctx.gk_pack(dsrc, dev_i32(spt), n, blob, sums)
+    clean = random_cache(og, N, seed=343)
+    d = dev_cache(clean)
+    mask = torch.full((1,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.gk_restore([gk.Job(blob, sums, dev_i32(dpt), n)], d, mask, fb)
+    torch.cuda.synchronize()
+    assert mask.item() == 0 and fb.item() == -1
+    L, T = og.layers, og.page_tokens
+    got = d.data.cpu().numpy().reshape(L, 2, N, T, -1)
+    s = src.data.reshape(L, 2, N, T, -1)
+    c = clean.data.reshape(L, 2, N, T, -1)
+    touched = np.zeros(N, dtype=bool)
+    for p in range(P):
+        t = min(T, n - p * T)
+        assert np.array_equal(got[:, :, dpt[p], :t], s[:, :, spt[p], :t])
+        assert np.array_equal(got[:, :, dpt[p], t:], c[:, :, dpt[p], t:])
+        touched[dpt[p]] = True
+    assert np.array_equal(got[:, :, ~touched], c[:, :, ~touched])
+    ctx.close()
+
+
+def test_argument_errors(gk):
+    from gpu_harness import dev_cache
+    og = G_MID
+    ctx = _ctx(gk, og)
+    clean = random_cache(og, 4, seed=350)
+    d = dev_cache(clean)
+    mask = torch.zeros(1, dtype=torch.uint8, device="cuda")
+    fb = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ctx.gk_restore([], d, mask, fb)                       # n_jobs == 0: no-op
+    pt = torch.zeros(1, dtype=torch.int32, device="cuda")
+    blob = torch.zeros(oracle.blob_size(og, 1)[0], dtype=torch.uint8)          # pageable host memory
+    sums = torch.zeros(1, dtype=torch.int64)
+    with pytest.raises(gk.GkError) as e:
+        ctx.gk_restore_host([gk.Job(blob, sums, pt, 1)], d, mask, fb)
+    assert e.value.code == -3
+    with pytest.raises(gk.GkError) as e:
+        ctx.gk_restore([gk.Job(blob.cuda(), sums.cuda(), pt, 0)], d, mask, fb)
+    assert e.value.code == -1
+    with pytest.raises(gk.GkError):
+        gk.Context(gk.Geom(2, 1, 4, 16), 0)               # row of 8 bytes: not a multiple of 16
+    ctx.close()
