@@ -232,37 +232,72 @@ __device__ __forceinline__ uint8_t *scale_addr(const GeomDev &g, const CacheDev 
            (uint64_t)phys * c.s_page_stride + 4ull * h;
 }
 
+__device__ __forceinline__ uint32_t xor3(uint32_t a, uint32_t b, uint32_t c)
+{
+    uint32_t d;
+    asm("lop3.b32 %0, %1, %2, %3, 0x96;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+    return d;
+}
+
+__device__ __forceinline__ uint32_t xor2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("xor.b32 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// All non-empty XOR combinations of four words; c[pat] = xor of t[i] for the bits i of pat.
+__device__ __forceinline__ void combos4(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3, uint32_t (&c)[16])
+{
+    c[0] = 0u;
+    c[1] = t0;
+    c[2] = t1;
+    c[4] = t2;
+    c[8] = t3;
+    c[3] = xor2(t0, t1);
+    c[5] = xor2(t0, t2);
+    c[6] = xor2(t1, t2);
+    c[9] = xor2(t0, t3);
+    c[10] = xor2(t1, t3);
+    c[12] = xor2(t2, t3);
+    c[7] = xor3(t0, t1, t2);
+    c[11] = xor3(t0, t1, t3);
+    c[13] = xor3(t0, t2, t3);
+    c[14] = xor3(t1, t2, t3);
+    c[15] = xor3(c[3], t2, t3);
+}
+
 // One 8-bit step of the bit-sliced shift register: state <- state*x^8 + w(x) mod P
 // for 32 streams at once.  U (0..7) is the number of steps taken since the
 // registers were last in natural order; coefficient m lives in R[(m - 8U) & 63],
 // so the shift itself costs nothing.  The eight top coefficients T[j] each add
-// x^(64+j) mod P; their sixteen-by-two partial sums are shared by all outputs.
+// x^(64+j) mod P; their two groups of fifteen partial sums are shared by all
+// outputs, so that every output costs one three-input XOR.  The XORs are spelled
+// as lop3 so that the instruction count is exactly what is written here
+// (64 + 22 per 8 words), whatever the compiler would make of a long ^ chain.
 template <int U>
 __device__ __forceinline__ void crc_step8(uint32_t (&R)[64], const uint32_t (&w)[8])
 {
     constexpr uint64_t G[8] = GK_G8_INIT;
     uint32_t A[16], B[16];
-    A[0] = 0u;
-    B[0] = 0u;
-#pragma unroll
-    for (int pat = 1; pat < 16; ++pat) {
-        const int low = pat & (-pat);
-        const int bit = (low == 1) ? 0 : (low == 2) ? 1 : (low == 4) ? 2 : 3;
-        A[pat] = A[pat ^ low] ^ R[(56 + bit - 8 * U) & 63];
-        B[pat] = B[pat ^ low] ^ R[(60 + bit - 8 * U) & 63];
-    }
+    combos4(R[(56 - 8 * U) & 63], R[(57 - 8 * U) & 63], R[(58 - 8 * U) & 63], R[(59 - 8 * U) & 63], A);
+    combos4(R[(60 - 8 * U) & 63], R[(61 - 8 * U) & 63], R[(62 - 8 * U) & 63], R[(63 - 8 * U) & 63], B);
 #pragma unroll
     for (int m = 0; m < 64; ++m) {
         const int pa = (int)(((G[0] >> m) & 1ull) | (((G[1] >> m) & 1ull) << 1) | (((G[2] >> m) & 1ull) << 2) |
                              (((G[3] >> m) & 1ull) << 3));
         const int pb = (int)(((G[4] >> m) & 1ull) | (((G[5] >> m) & 1ull) << 1) | (((G[6] >> m) & 1ull) << 2) |
                              (((G[7] >> m) & 1ull) << 3));
-        const uint32_t fb = A[pa] ^ B[pb];
         const int phys = (m - 8 - 8 * U) & 63;
-        if (m < 8)
-            R[phys] = w[7 - m] ^ fb;
+        const uint32_t base = (m < 8) ? w[7 - m] : R[phys];
+        if (pa != 0 && pb != 0)
+            R[phys] = xor3(base, A[pa], B[pb]);
+        else if (pa != 0)
+            R[phys] = xor2(base, A[pa]);
+        else if (pb != 0)
+            R[phys] = xor2(base, B[pb]);
         else
-            R[phys] ^= fb;
+            R[phys] = base;
     }
 }
 
@@ -310,6 +345,19 @@ __device__ __forceinline__ uint64_t thread_remainder(const uint32_t (&R)[64], ui
     return gf_mul(kt, lo64);
 }
 
+// Ring position of a pipeline role: stage index and the parity of its use count.
+struct RingPos {
+    uint32_t stage = 0, phase = 0;
+    template <int STAGES>
+    __device__ __forceinline__ void advance()
+    {
+        if (++stage == (uint32_t)STAGES) {
+            stage = 0;
+            phase ^= 1u;
+        }
+    }
+};
+
 // The eight 8-word steps of one granule (after which the registers are back in
 // natural order).  Every kSps steps a new stage is awaited and the finished one
 // is handed back to the loader.
@@ -317,28 +365,27 @@ template <int U, int MODE, int NT, int STAGE_BYTES, int STAGES>
 struct GranuleSteps {
     using Cfg = StreamCfg<MODE, NT, STAGE_BYTES, STAGES>;
     static __device__ __forceinline__ void run(uint32_t (&R)[64], const uint8_t *smem, uint32_t full0, uint32_t empty0,
-                                               uint32_t &n, volatile uint32_t *abort_flag, uint32_t *error, int tid,
+                                               RingPos &pos, volatile uint32_t *abort_flag, uint32_t *error, int tid,
                                                int lane)
     {
-        const uint32_t s = n % STAGES;
-        if (U % Cfg::kSps == 0)
-            mbar_wait(full0 + 8u * s, (n / STAGES) & 1u, abort_flag, error, 0x400u | MODE);
-        const uint32_t *sw = reinterpret_cast<const uint32_t *>(smem + (size_t)s * STAGE_BYTES) + tid;
+        if (U % Cfg::kSps == 0) mbar_wait(full0 + 8u * pos.stage, pos.phase, abort_flag, error, 0x400u | MODE);
+        const uint32_t *sw = reinterpret_cast<const uint32_t *>(smem + (size_t)pos.stage * STAGE_BYTES) + tid;
         uint32_t w[8];
 #pragma unroll
         for (int jw = 0; jw < 8; ++jw) w[jw] = sw[((U % Cfg::kSps) * 8 + jw) * NT];
         crc_step8<U>(R, w);
         if (U % Cfg::kSps == Cfg::kSps - 1) {
             __syncwarp();
-            if (lane == 0) mbar_arrive(empty0 + 8u * s);
-            ++n;
+            if (lane == 0) mbar_arrive(empty0 + 8u * pos.stage);
+            pos.template advance<STAGES>();
         }
-        GranuleSteps<U + 1, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, n, abort_flag, error, tid, lane);
+        GranuleSteps<U + 1, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, pos, abort_flag, error, tid,
+                                                                lane);
     }
 };
 template <int MODE, int NT, int STAGE_BYTES, int STAGES>
 struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES> {
-    static __device__ __forceinline__ void run(uint32_t (&)[64], const uint8_t *, uint32_t, uint32_t, uint32_t &,
+    static __device__ __forceinline__ void run(uint32_t (&)[64], const uint8_t *, uint32_t, uint32_t, RingPos &,
                                                volatile uint32_t *, uint32_t *, int, int)
     {
     }
@@ -520,7 +567,7 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
         // ----------------------------- consumers ----------------------------
         const int tid = threadIdx.x;  // consumer warps come first: 0..NT-1
         const uint64_t kt = P.w.thread_const[tid];
-        uint32_t n = 0;
+        RingPos pos;
         uint32_t parity_red = 0;
         for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
             Item it;
@@ -530,8 +577,8 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
             for (int i = 0; i < 64; ++i) R[i] = 0u;
             const uint32_t ngran = it.tile_count / Cfg::kTilesPerGran;
             for (uint32_t gi = 0; gi < ngran; ++gi)
-                GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, n, abort_flag, P.w.error, tid,
-                                                                    lane);
+                GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, pos, abort_flag, P.w.error,
+                                                                    tid, lane);
             // merge streams -> thread -> warp -> CTA
             uint64_t v = thread_remainder<NT>(R, kt);
 #pragma unroll
