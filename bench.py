@@ -1,0 +1,471 @@
+#!/usr/bin/env python3
+"""Benchmark of the KV block save/restore hot path on B200.
+
+One step = one pass of the whole path over one batch of synthetic input shaped
+like the GQA-7B-like serving workload: gk_pack_batch saves the batch's 16 blocks
+of 4,096 tokens (32 layers, 8 KV heads, head_dim 128, bf16, 16-token pages) from
+a paged source cache into their slots of a 64-block device-resident pool, then
+gk_restore validates the page tables, verifies every page record (CRC-64/XZ),
+and scatters the 16 blocks (8 requests x 2 blocks) into a 16,384-page destination
+cache through seeded random-permutation page tables.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line on rank 0.  `value` counts the KV bytes the step reads plus
+writes (2 x blob bytes for the save, 2 x blob bytes for the restore) per second,
+summed over all GPUs; the restore phase alone, tokens/s and the per-kernel
+roofline are reported beside it.  With N > 1 (launched by torch.distributed.run)
+every rank runs its own batch on its own GPU: the path has no exchange step, so
+this is weak scaling over independent request batches.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "restored KV GB/s (read+write)"
+UNIT = "GB/s"
+
+# DRAM bytes per blob byte of one commit-kernel launch, from the ncu capture
+# summarised in profiles/stream_kernel_commit_gqa7b_2blocks.md (dram read +
+# write of the launch divided by the blob bytes it commits).  Traffic grows in
+# proportion to the blob bytes, so a full launch is this ratio times its bytes.
+COMMIT_DRAM_BYTES_PER_BLOB_BYTE = 1.947
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--blocks", type=int, default=0,
+                    help="restore this many blocks instead of the workload's 16 (small cases for profiling)")
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-baseline-blocks", type=int, default=4)
+    return ap.parse_args()
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+# ---------------------------------------------------------------------------
+# clocks during the timed region
+# ---------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index: int):
+        self.proc = None
+        self.path = None
+        try:
+            import torch
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            if not uuid.startswith("GPU-"):
+                uuid = "GPU-" + uuid
+            fd, self.path = tempfile.mkstemp(prefix="gk_clocks_", suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", uuid, f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "50"], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return None
+        try:
+            self.proc.terminate()
+            self.proc.wait(timeout=5)
+        except Exception:
+            pass
+        self.out.close()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        try:
+            with open(self.path) as f:
+                for line in f:
+                    parts = [p.strip() for p in line.split(",")]
+                    if len(parts) < 7:
+                        continue
+                    try:
+                        sm.append(float(parts[0]))
+                        smax.append(float(parts[1]))
+                    except ValueError:
+                        continue
+                    for name, val in zip(names, parts[3:7]):
+                        if val.lower().startswith("active"):
+                            reasons.add(name)
+            os.unlink(self.path)
+        except Exception:
+            return None
+        if not sm:
+            return None
+        return {"sm_mhz": float(np.median(sm)), "sm_max_mhz": float(max(smax)), "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------
+# workload
+# ---------------------------------------------------------------------------
+def build_workload(args, device, rank):
+    import torch
+    import synth
+    import paper_2609_39358_b200 as gk
+
+    w = synth.GQA7B
+    geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, gk.GK_BF16, 0)
+    n_tok = synth.GQA7B_BLOCK_TOKENS
+    blob_bytes, P = gk.gk_blob_size(geom, n_tok)
+    if args.blocks:
+        n_blocks = args.blocks
+        pool_blocks = n_blocks
+        dst_pages = max(2 * n_blocks * P, 512)
+    else:
+        n_blocks = synth.GQA7B_REQUESTS * synth.GQA7B_BLOCKS_PER_REQUEST
+        pool_blocks = synth.GQA7B_POOL_BLOCKS
+        dst_pages = synth.GQA7B_DST_PAGES
+    slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
+    src_pages = n_blocks * P
+
+    def cache(num_pages, data):
+        return gk.Cache(data, num_pages, 2 * num_pages * slab, num_pages * slab, slab)
+
+    seed0 = w.seed(100 * rank)
+    rng = np.random.default_rng(seed0)
+    pool = [torch.empty(blob_bytes, dtype=torch.uint8, device=device) for _ in range(pool_blocks)]
+    sums = [torch.zeros(P, dtype=torch.int64, device=device) for _ in range(pool_blocks)]
+    ctx = gk.Context(geom, device.index)
+    src_perm = torch.from_numpy(synth.page_permutation(src_pages, seed0 + 1)).to(device)
+    chosen = np.sort(rng.choice(pool_blocks, size=n_blocks, replace=False))
+
+    # fill the pool: the source cache is refilled for every group of n_blocks blocks;
+    # the last fill holds the blocks the timed steps save and restore
+    groups = [list(range(g, min(g + n_blocks, pool_blocks))) for g in range(0, pool_blocks, n_blocks)]
+    src = None
+    for gi, group in enumerate(groups + [list(chosen)]):
+        data = synth.kv_bytes_bf16(2 * w.layers * src_pages * slab // 2, w.sigma, seed0 + 10 + gi, device)
+        src = cache(src_pages, data)
+        jobs = [gk.Job(pool[b], sums[b], src_perm[i * P:(i + 1) * P].contiguous(), n_tok)
+                for i, b in enumerate(group)]
+        ctx.gk_pack_batch(src, jobs)
+        torch.cuda.synchronize(device)
+        if gi < len(groups):
+            del data, src
+    dst_data = synth.sentinel_bytes(2 * w.layers * dst_pages * slab, seed0 + 2, device)
+    dst = cache(dst_pages, dst_data)
+    dst_perm = torch.from_numpy(synth.page_permutation(dst_pages, seed0 + 3)).to(device)
+    pack_jobs, restore_jobs = [], []
+    for i, b in enumerate(chosen):
+        pack_jobs.append(gk.Job(pool[b], sums[b], src_perm[i * P:(i + 1) * P].contiguous(), n_tok, i // 2))
+        restore_jobs.append(gk.Job(pool[b], sums[b], dst_perm[i * P:(i + 1) * P].contiguous(), n_tok, i // 2))
+    return dict(gk=gk, ctx=ctx, geom=geom, w=w, n_tok=n_tok, blob_bytes=blob_bytes, P=P, n_blocks=n_blocks,
+                pool_blocks=pool_blocks, dst_pages=dst_pages, src=src, dst=dst, pack_jobs=pack_jobs,
+                restore_jobs=restore_jobs, chosen=chosen, src_perm=src_perm, dst_perm=dst_perm, slab=slab,
+                src_pages=src_pages)
+
+
+def oracle_sample(wl, n_blocks, steps, warmup):
+    """Times the CPU oracle (as it stands, single-threaded) on the first n_blocks
+    blocks of the batch: pack from a host copy of the source cache, then restore
+    into a host destination cache.  Returns (seconds per step, bytes per step,
+    tokens per step, checksums of the packed blocks)."""
+    import oracle
+    w = wl["w"]
+    og = oracle.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, w.elem_bytes, 0)
+    P, n_tok, slab = wl["P"], wl["n_tok"], wl["slab"]
+    src_pages = wl["src_pages"]
+    src_host = wl["src"].data.cpu().numpy()
+    src = oracle.Cache(src_host, src_pages, 2 * src_pages * slab, src_pages * slab, slab)
+    dpages = n_blocks * P
+    dst = oracle.Cache(np.zeros(2 * w.layers * dpages * slab, dtype=np.uint8), dpages, 2 * dpages * slab,
+                       dpages * slab, slab)
+    src_perm = wl["src_perm"].cpu().numpy()
+    dperm = np.random.default_rng(7).permutation(dpages).astype(np.int32)
+    times, sums_out = [], None
+    for it in range(warmup + steps):
+        t0 = time.perf_counter()
+        jobs = []
+        for i in range(n_blocks):
+            blob, sums, code, _ = oracle.pack(og, src, src_perm[i * P:(i + 1) * P], n_tok)
+            assert code == 0
+            jobs.append(oracle.Job(blob, sums, dperm[i * P:(i + 1) * P], n_tok))
+        mask, _ = oracle.restore(og, dst, jobs)
+        dt = time.perf_counter() - t0
+        assert not mask.any()
+        if it >= warmup:
+            times.append(dt)
+        sums_out = [j.checksums for j in jobs]
+    return float(np.mean(times)), 4 * n_blocks * wl["blob_bytes"], n_blocks * n_tok, sums_out
+
+
+# ---------------------------------------------------------------------------
+# reference arm: the oracle on the host cores
+# ---------------------------------------------------------------------------
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import oracle
+    import synth
+    w = synth.GQA7B
+    og = oracle.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, w.elem_bytes, 0)
+    slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
+    # size the sample so that the whole run stays within about two minutes
+    probe_pages = 8
+    rng = np.random.default_rng(w.seed(900))
+    n_iter = max(1, args.steps + args.warmup)
+    per_page = None
+    pages = probe_pages
+    for _ in range(2):
+        N = pages
+        data = rng.integers(0, 256, size=2 * w.layers * N * slab, dtype=np.uint8)
+        src = oracle.Cache(data, N, 2 * N * slab, N * slab, slab)
+        dst = oracle.Cache(np.zeros_like(data), N, 2 * N * slab, N * slab, slab)
+        spt = rng.permutation(N).astype(np.int32)
+        dpt = rng.permutation(N).astype(np.int32)
+        n_tok = N * w.page_tokens
+        if per_page is None:
+            t0 = time.perf_counter()
+            blob, sums, _, _ = oracle.pack(og, src, spt, n_tok)
+            oracle.restore(og, dst, [oracle.Job(blob, sums, dpt, n_tok)])
+            per_page = (time.perf_counter() - t0) / N
+            pages = int(min(1024, max(8, 100.0 / (per_page * n_iter))))
+    times = []
+    blob_bytes = oracle.blob_size(og, n_tok)[0]
+    for it in range(args.warmup + args.steps):
+        t0 = time.perf_counter()
+        blob, sums, code, _ = oracle.pack(og, src, spt, n_tok)
+        mask, _ = oracle.restore(og, dst, [oracle.Job(blob, sums, dpt, n_tok)])
+        dt = time.perf_counter() - t0
+        assert code == 0 and not mask.any()
+        if it >= args.warmup:
+            times.append(dt)
+    t = float(np.mean(times))
+    value = 4 * blob_bytes / t / 1e9
+    sample = f"one block of {n_tok} tokens ({pages} pages, {blob_bytes / 2**20:.0f} MiB blob) saved and restored per step"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": "gqa7b (32 layers, 8 KV heads, head_dim 128, bf16, 16-token pages), bounded sample",
+                       "sample": sample},
+            "tokens_per_s": n_tok / t,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+# ---------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: libgk has no CPU fallback")
+    device = torch.device("cuda", local_rank)
+    torch.cuda.set_device(device)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=device)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize(device)
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    wl = build_workload(args, device, rank)
+    gk, ctx = wl["gk"], wl["ctx"]
+    n_blocks, blob_bytes, n_tok = wl["n_blocks"], wl["blob_bytes"], wl["n_tok"]
+    batch_bytes = n_blocks * blob_bytes
+    mask = torch.zeros(n_blocks, dtype=torch.uint8, device=device)
+    first_bad = torch.zeros(n_blocks, dtype=torch.int32, device=device)
+    status = torch.zeros(n_blocks, dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream(device)
+
+    def step(events=None):
+        if events:
+            events[0].record(stream)
+        ctx.gk_pack_batch(wl["src"], wl["pack_jobs"], status)
+        if events:
+            events[1].record(stream)
+        ctx.gk_restore(wl["restore_jobs"], wl["dst"], mask, first_bad)
+        if events:
+            events[2].record(stream)
+
+    for _ in range(max(args.warmup, 0)):
+        step()
+    torch.cuda.synchronize(device)
+    ctx.set_tuning("profile", 1)
+    ctx.gk_get_kernel_times()
+    launches0 = ctx.gk_get_stats()["kernels_launched"]
+    phase_events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    barrier()
+    t_begin.record(stream)
+    for k in range(args.steps):
+        step(phase_events[k])
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop() if sampler else None
+    step_ms = max_over_ranks(t_begin.elapsed_time(t_end) / max(args.steps, 1))
+    kt = ctx.gk_get_kernel_times()
+    ctx.set_tuning("profile", 0)
+    stats = ctx.gk_get_stats()
+    launches = stats["kernels_launched"] - launches0
+    assert int(mask.sum().item()) == 0 and int(status.sum().item()) == 0, "a clean block was rejected"
+    assert stats["device_wait_expired"] == 0
+    pack_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in phase_events]))
+    restore_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in phase_events]))
+
+    value = world * 4 * batch_bytes / (step_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peak()
+
+    def kernel_entry(name, alg_bytes_per_launch):
+        ms, n = kt[name]
+        if n == 0:
+            return None
+        per = ms / n
+        ach = alg_bytes_per_launch / (per * 1e-3) / 1e9
+        return {"launches": n, "ms_per_launch": per, "algorithmic_bytes_per_launch": alg_bytes_per_launch,
+                "achieved": ach, "unit": "GB/s", "frac": ach / peak}
+
+    kernels = {"commit": kernel_entry("commit", 2 * batch_bytes),
+               "verify": kernel_entry("verify", batch_bytes),
+               "pack": kernel_entry("pack", 2 * batch_bytes)}
+    dom = kernels["commit"]
+    roofline = {"bound": "hbm", "kernel": "stream_kernel<kCommit> (blob -> paged cache scatter)",
+                "achieved": dom["achieved"], "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
+                "frac": dom["frac"], "traffic": COMMIT_DRAM_BYTES_PER_BLOB_BYTE * batch_bytes,
+                "traffic_note": "ncu dram read+write of a 2-block launch scaled by blob bytes",
+                "algorithmic_bytes_per_launch": 2 * batch_bytes, "ms_per_launch": dom["ms_per_launch"]}
+
+    # ---- end to end: blobs in pinned host memory, through gk_restore_host ----
+    e2e = None
+    if not args.no_e2e:
+        host_jobs, keep = [], []
+        for jb in wl["restore_jobs"]:
+            hb = torch.empty(blob_bytes, dtype=torch.uint8, pin_memory=True)
+            hb.copy_(jb.blob)
+            hs = torch.empty(wl["P"], dtype=torch.int64, pin_memory=True)
+            hs.copy_(jb.checksums)
+            keep.append((hb, hs))
+            host_jobs.append(gk.Job(hb, hs, jb.page_table, n_tok, jb.request_id))
+        mask_h = torch.empty(n_blocks, dtype=torch.uint8, pin_memory=True)
+        fb_h = torch.empty(n_blocks, dtype=torch.int32, pin_memory=True)
+        torch.cuda.synchronize(device)
+
+        def e2e_step():
+            ctx.gk_restore_host(host_jobs, wl["dst"], mask, first_bad)
+            mask_h.copy_(mask, non_blocking=True)
+            fb_h.copy_(first_bad, non_blocking=True)
+
+        e2e_step()
+        torch.cuda.synchronize(device)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        e1.record(stream)
+        barrier()
+        e2e_ms = max_over_ranks(e0.elapsed_time(e1) / max(args.e2e_steps, 1))
+        assert int(mask_h.sum().item()) == 0
+        h2d = batch_bytes + n_blocks * wl["P"] * 8 + n_blocks * 40
+        e2e = {"value": world * 2 * batch_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": n_blocks * 5, "ms_per_step": e2e_ms,
+               "steps": args.e2e_steps, "tokens_per_s": world * n_blocks * n_tok / (e2e_ms * 1e-3),
+               "host_link_gbs": world * h2d / (e2e_ms * 1e-3) / 1e9,
+               "what": "gk_restore_host of the batch from pinned host blobs + D2H read of mask and first_bad_page"}
+        del keep, host_jobs
+
+    cpu_baseline = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        nb = min(args.cpu_baseline_blocks, n_blocks)
+        t, nbytes, ntoks, osums = oracle_sample(wl, nb, steps=1, warmup=0)
+        for i in range(nb):   # the pool blobs the GPU packed carry the same checksums
+            got = wl["pack_jobs"][i].checksums.cpu().numpy().view(np.uint64)
+            assert np.array_equal(got, osums[i]), "GPU checksums differ from the oracle's"
+        cpu_baseline = {"value": nbytes / t / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": f"save + restore of the first {nb} blocks of the batch ({ntoks} tokens, "
+                                  f"{nb * blob_bytes / 2**30:.1f} GiB of blobs), {t:.1f} s",
+                        "tokens_per_s": ntoks / t}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": step_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {
+                "workload": ("gqa7b: 32 layers, 8 KV heads, head_dim 128, bf16 N(0,0.5), 16-token pages; "
+                             f"{n_blocks} blocks of {n_tok} tokens per step per GPU "
+                             f"({synth_requests(n_blocks)}), pool of {wl['pool_blocks']} blocks, "
+                             f"{wl['dst_pages']}-page destination cache, seeded random-permutation page tables"),
+                "step": "gk_pack_batch (save) + gk_restore (validate, verify, commit) of the batch",
+                "value_definition": "(2 x blob bytes saved + 2 x blob bytes restored) / step time, all GPUs",
+                "batch_blob_bytes": batch_bytes, "l2": "inputs larger than L2 (8 GiB per phase vs 126 MB)",
+                "parallelism": f"replicas x{world}, no collective"},
+            "tokens_per_s": world * n_blocks * n_tok / (step_ms * 1e-3),
+            "frac_of_hbm_peak": value / world / peak,
+            "phases": {
+                "pack": {"ms": pack_ms, "gbs": 2 * batch_bytes / (pack_ms * 1e-3) / 1e9},
+                "restore": {"ms": restore_ms, "gbs_useful": 2 * batch_bytes / (restore_ms * 1e-3) / 1e9,
+                            "gbs_dram_model": 3 * batch_bytes / (restore_ms * 1e-3) / 1e9,
+                            "tokens_per_s": n_blocks * n_tok / (restore_ms * 1e-3),
+                            "frac_of_hbm_peak_dram_model": 3 * batch_bytes / (restore_ms * 1e-3) / 1e9 / peak}},
+            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
+            "gpu_launches": launches, "clocks": clocks,
+        }
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def synth_requests(n_blocks):
+    return f"{max(n_blocks // 2, 1)} requests x {min(n_blocks, 2)} blocks"
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -183,8 +183,15 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * geometry.  Keys: "seg_granules" (length of a checksum segment in units of
  * 32 KiB; 0 = one segment per page), "commit_seg_tiles" (length of a commit work
  * item in 16 KiB tiles), "grid_cap" (upper bound on CTAs per kernel; 0 = fill
- * the GPU). */
+ * the GPU), "profile" (1 = time every streaming kernel, see gk_get_kernel_times). */
 int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
+
+/* Per-kernel device time of the three streaming kernels, for measurements.
+ * With the tuning key "profile" set to 1 every launch of a streaming kernel is
+ * bracketed by CUDA events on its stream.  This call waits for the recorded
+ * events, and returns and then clears the totals since the previous call:
+ * index 0 = verify, 1 = pack, 2 = commit; ms = summed duration, launches = count. */
+int gk_get_kernel_times(gk_ctx *ctx, double ms[3], uint64_t launches[3]);
 
 #ifdef __cplusplus
 }

@@ -24,7 +24,7 @@ GK_FLAG_SKIP_VERIFY = 1
 JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
 
 EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",
-           "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning"]
+           "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times"]
 
 
 class GkError(RuntimeError):
@@ -91,6 +91,8 @@ def load_library() -> ctypes.CDLL:
     L.gk_restore_host.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
     L.gk_get_stats.restype = ctypes.c_int
     L.gk_get_stats.argtypes = [vp, ctypes.POINTER(CStats)]
+    L.gk_get_kernel_times.restype = ctypes.c_int
+    L.gk_get_kernel_times.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_uint64)]
     L.gk_ctx_set_tuning.restype = ctypes.c_int
     L.gk_ctx_set_tuning.argtypes = [vp, ctypes.c_char_p, u32]
     _lib = L
@@ -225,6 +227,13 @@ class Context:
         cc = dst.c()
         self._check(self._lib.gk_restore_host(self._h, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask),
                                               _ptr(first_bad_page), _stream_handle(stream)), "gk_restore_host")
+
+    def gk_get_kernel_times(self) -> dict:
+        """{'verify'|'pack'|'commit': (ms, launches)} since the previous call (needs tuning key profile=1)."""
+        ms = (ctypes.c_double * 3)()
+        n = (ctypes.c_uint64 * 3)()
+        self._check(self._lib.gk_get_kernel_times(self._h, ms, n), "gk_get_kernel_times")
+        return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(("verify", "pack", "commit"))}
 
     def gk_get_stats(self) -> dict:
         st = CStats()

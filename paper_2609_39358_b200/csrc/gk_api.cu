@@ -91,6 +91,14 @@ struct gk_ctx {
     cudaEvent_t ev_copied[kSlots] = {nullptr, nullptr};
     bool slot_used[kSlots] = {false, false};
 
+    // optional per-kernel timing (tuning key "profile")
+    bool profile = false;
+    struct ProfSlot { cudaEvent_t a, b; int cls; };
+    std::vector<ProfSlot> prof_pool;
+    size_t prof_used = 0;
+    double prof_ms[3] = {0, 0, 0};
+    uint64_t prof_launches[3] = {0, 0, 0};
+
     gk_stats stats{};
     char err[512] = {0};
 };
@@ -321,8 +329,21 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
 {
     if (P.n_items == 0) return GK_OK;
     const uint32_t grid = stream_grid(c, occ, P.n_items);
+    gk_ctx::ProfSlot *slot = nullptr;
+    if (c->profile) {
+        if (c->prof_used == c->prof_pool.size()) {
+            gk_ctx::ProfSlot ns{};
+            GK_CUDA(c, cudaEventCreate(&ns.a));
+            GK_CUDA(c, cudaEventCreate(&ns.b));
+            c->prof_pool.push_back(ns);
+        }
+        slot = &c->prof_pool[c->prof_used++];
+        slot->cls = MODE;
+        GK_CUDA(c, cudaEventRecord(slot->a, st));
+    }
     stream_kernel<MODE, NT, SB, ST, MINB><<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(P);
     GK_CUDA(c, cudaGetLastError());
+    if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
     return GK_OK;
 }
@@ -472,6 +493,10 @@ int gk_ctx_destroy(gk_ctx *c)
     DeviceGuard guard(c->device);
     cudaDeviceSynchronize();
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+    for (auto &ps : c->prof_pool) {
+        cudaEventDestroy(ps.a);
+        cudaEventDestroy(ps.b);
+    }
     for (int i = 0; i < kSlots; ++i) {
         if (c->d_slot[i]) cudaFree(c->d_slot[i]);
         if (c->ev_slot_free[i]) cudaEventDestroy(c->ev_slot_free[i]);
@@ -496,6 +521,7 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     if (!strcmp(key, "seg_granules")) c->seg_granules = value;
     else if (!strcmp(key, "commit_seg_tiles")) c->commit_seg_tiles = value;
     else if (!strcmp(key, "grid_cap")) c->grid_cap = value;
+    else if (!strcmp(key, "profile")) c->profile = value != 0;
     else return fail(c, GK_ERR_ARG, "unknown tuning key %s", key);
     return GK_OK;
 }
@@ -754,6 +780,28 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
     c->stats.jobs += n_jobs;
     c->stats.pages += pages;
     c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+int gk_get_kernel_times(gk_ctx *c, double ms[3], uint64_t launches[3])
+{
+    if (!c || !ms || !launches) return GK_ERR_ARG;
+    DeviceGuard guard(c->device);
+    for (size_t i = 0; i < c->prof_used; ++i) {
+        gk_ctx::ProfSlot &ps = c->prof_pool[i];
+        GK_CUDA(c, cudaEventSynchronize(ps.b));
+        float t = 0.f;
+        GK_CUDA(c, cudaEventElapsedTime(&t, ps.a, ps.b));
+        c->prof_ms[ps.cls] += t;
+        c->prof_launches[ps.cls]++;
+    }
+    c->prof_used = 0;
+    for (int i = 0; i < 3; ++i) {
+        ms[i] = c->prof_ms[i];
+        launches[i] = c->prof_launches[i];
+        c->prof_ms[i] = 0;
+        c->prof_launches[i] = 0;
+    }
     return GK_OK;
 }
 
