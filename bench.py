@@ -92,6 +92,18 @@ class ClockSampler:
         except Exception:
             self.proc = None
 
+    def wait_first_sample(self, limit_s: float = 8.0):
+        if self.proc is None:
+            return
+        t0 = time.time()
+        while time.time() - t0 < limit_s:
+            try:
+                if os.path.getsize(self.path) > 0:
+                    return
+            except OSError:
+                return
+            time.sleep(0.05)
+
     def stop(self):
         if self.proc is None:
             return None
@@ -326,15 +338,20 @@ def run_ours(args):
         if events:
             events[2].record(stream)
 
-    for _ in range(max(args.warmup, 0)):
+    # warm-up: the per-kernel timing events are created here, not in the timed region
+    ctx.set_tuning("profile", 1)
+    for _ in range(max(args.warmup, 3)):
         step()
     torch.cuda.synchronize(device)
-    ctx.set_tuning("profile", 1)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    if sampler:
+        sampler.wait_first_sample()   # nvidia-smi start-up would otherwise stall CUDA calls of step 0
+    step()
+    torch.cuda.synchronize(device)
     ctx.gk_get_kernel_times()
     launches0 = ctx.gk_get_stats()["kernels_launched"]
     phase_events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
     t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     barrier()
     t_begin.record(stream)
     for k in range(args.steps):

@@ -40,6 +40,8 @@ def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | N
         cmd += ["-Xptxas", "-v"]
     if extra_flags:
         cmd += extra_flags
+    if os.environ.get("GK_NVCC_FLAGS"):
+        cmd += os.environ["GK_NVCC_FLAGS"].split()
     cmd += [os.path.join(_CSRC, s) for s in _SOURCES] + ["-o", tmp, "-lcudart"]
     subprocess.check_call(cmd)
     os.replace(tmp, LIB_PATH)

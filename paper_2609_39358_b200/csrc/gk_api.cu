@@ -23,8 +23,11 @@
 #ifndef GK_CRC_STAGES
 #define GK_CRC_STAGES 6
 #endif
-#ifndef GK_CRC_MINB
-#define GK_CRC_MINB 2
+#ifndef GK_VERIFY_MINB
+#define GK_VERIFY_MINB 3
+#endif
+#ifndef GK_PACK_MINB
+#define GK_PACK_MINB 2
 #endif
 #ifndef GK_COPY_STAGE
 #define GK_COPY_STAGE 16384
@@ -350,11 +353,11 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
 
 int launch_verify(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
-    return launch_stream<VerifyCfg, kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_CRC_MINB>(c, c->occ_verify, P, st);
+    return launch_stream<VerifyCfg, kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB>(c, c->occ_verify, P, st);
 }
 int launch_pack(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
-    return launch_stream<PackCfg, kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_CRC_MINB>(c, c->occ_pack, P, st);
+    return launch_stream<PackCfg, kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_PACK_MINB>(c, c->occ_pack, P, st);
 }
 int launch_commit(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
@@ -449,8 +452,8 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
     if (prop.major != 10) return bail(GK_ERR_UNSUPPORTED);  // built for sm_100a only
     c->sm_count = prop.multiProcessorCount;
 
-    auto *kv = stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_CRC_MINB>;
-    auto *kp = stream_kernel<kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_CRC_MINB>;
+    auto *kv = stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB>;
+    auto *kp = stream_kernel<kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_PACK_MINB>;
     auto *kc = stream_kernel<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES, GK_COPY_MINB>;
     if (cudaFuncSetAttribute(kv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VerifyCfg::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(kp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PackCfg::kSmemBytes) != cudaSuccess ||
