@@ -5,10 +5,10 @@
  * The operations are those of the paper's KV memory (Section 2.2, "Taliesin: KV
  * memory"): after the runtime has computed the KV state of a block of prompt
  * text the state is written out; when the same block recurs it is loaded
- * instead of recomputed; stored state is checked on load; and by the rule
- * "serve without memory, never with wrong memory" a record that is missing,
- * damaged or fails a check is not used at all -- the block is reported for
- * recompute.  Restored state must be bit-identical to what was saved (Section 3,
+ * instead of recomputed; what was stored is checked when it is loaded; and by
+ * that section's design rule -- a request may be served without stored state but
+ * never with wrong stored state -- a record that is missing, damaged or fails
+ * a check is not used at all: the block is reported for recompute.  Restored state must be bit-identical to what was saved (Section 3,
  * Table 1), reuse is per whole block (Section 5, first item) and the design is
  * fail-closed (Section 5, second item).  The paper does not disclose its record
  * format (end of Section 1); the format below is this library's own.
@@ -75,7 +75,7 @@ extern "C" {
 #define GK_JOB_TIMEOUT 4u     /* a bounded wait inside a kernel ran out; nothing of
                                  the call was committed */
 
-/* Test hook for sabotage tests (Section 3, "Sabotage testing"): switches the
+/* Test hook for sabotage tests (Section 3, sabotage-testing paragraph): switches the
  * checksum defence off so that a test can show the attack succeeds without it.
  * Page-table validation stays on. */
 #define GK_FLAG_SKIP_VERIFY 1u
@@ -134,8 +134,8 @@ int gk_ctx_destroy(gk_ctx *ctx);
 /* Text of the last error of this context (never NULL; empty if none). */
 const char *gk_last_error(const gk_ctx *ctx);
 
-/* Save (Section 2.2: "writes it to storage" -- here: gathers it into one
- * contiguous record with checksums).  jobs is a HOST array of n_jobs entries;
+/* Save (Section 2.2: the block's state is written out once it has been computed;
+ * here: gathered into one contiguous record with checksums).  jobs is a HOST array of n_jobs entries;
  * each job's blob (gk_blob_size bytes) and checksums (n_pages entries) are
  * device outputs.  Duplicate page ids are legal when packing.  A job whose table
  * holds an id outside [0, src->num_pages) writes neither blob nor checksums and
@@ -148,12 +148,12 @@ int gk_pack_batch(gk_ctx *ctx, const gk_cache *src, const gk_job *jobs, uint32_t
 int gk_pack(gk_ctx *ctx, const gk_cache *src, const int32_t *page_table_dev, uint32_t n_tokens,
             void *blob_dev, uint64_t *checksums_dev, uint8_t *status_dev, void *stream);
 
-/* Page checksums of an existing device blob (the check that "Stored state is
- * checked on load" relies on, Section 2.2): checksums_dev[p] = CRC-64/XZ of record p. */
+/* Page checksums of an existing device blob (the check-on-load of Section 2.2
+ * rests on them): checksums_dev[p] = CRC-64/XZ of record p. */
 int gk_page_checksums(gk_ctx *ctx, const void *blob_dev, uint32_t n_tokens,
                       uint64_t *checksums_dev, void *stream);
 
-/* Load (Section 2.2 and Section 5 "Fail-closed by design").  jobs is a HOST array;
+/* Load (Section 2.2, and the fail-closed item of Section 5).  jobs is a HOST array;
  * blob, checksums and page_table of each job are device pointers.  Phase 1
  * validates every page table and verifies every page record of every job and
  * writes nothing to dst; phase 2 scatters the jobs whose code is GK_JOB_OK into
@@ -165,8 +165,8 @@ int gk_page_checksums(gk_ctx *ctx, const void *blob_dev, uint32_t n_tokens,
 int gk_restore(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
                uint8_t *mask_dev, int32_t *first_bad_page_dev, void *stream);
 
-/* Load from the host tier (Section 4.3, "Long windows at flat GPU memory": saved
- * blocks are streamed in).  As gk_restore, but each job's blob and checksums lie
+/* Load from the host tier (Section 4.3, long-window paragraph: saved blocks are
+ * streamed in from storage and dropped after use).  As gk_restore, but each job's blob and checksums lie
  * in PINNED host memory.  Blobs are copied in batches into an internal device
  * staging ring on an internal copy stream while the previous batch is verified
  * and committed on `stream`; the checksum is taken over the bytes as they arrived
@@ -183,15 +183,18 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * geometry.  Keys: "seg_granules" (length of a checksum segment in units of
  * 32 KiB; 0 = one segment per page), "commit_seg_tiles" (length of a commit work
  * item in 16 KiB tiles), "grid_cap" (upper bound on CTAs per kernel; 0 = fill
- * the GPU), "profile" (1 = time every streaming kernel, see gk_get_kernel_times). */
+ * the GPU), "profile" (1 = time every streaming kernel, see gk_get_kernel_times),
+ * "fused" (1, the default: gk_restore verifies and commits in one launch; 0: a
+ * verify launch, a checksum-compare launch and a commit launch). */
 int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
 
-/* Per-kernel device time of the three streaming kernels, for measurements.
- * With the tuning key "profile" set to 1 every launch of a streaming kernel is
- * bracketed by CUDA events on its stream.  This call waits for the recorded
- * events, and returns and then clears the totals since the previous call:
- * index 0 = verify, 1 = pack, 2 = commit; ms = summed duration, launches = count. */
-int gk_get_kernel_times(gk_ctx *ctx, double ms[3], uint64_t launches[3]);
+/* Per-kernel device time of the streaming kernels, for measurements.  With the
+ * tuning key "profile" set to 1 every launch of a streaming kernel is bracketed
+ * by CUDA events on its stream.  This call waits for the recorded events, and
+ * returns and then clears the totals since the previous call: index 0 = verify
+ * alone, 1 = pack, 2 = commit alone, 3 = fused verify+commit (the restore kernel);
+ * ms = summed duration, launches = count. */
+int gk_get_kernel_times(gk_ctx *ctx, double ms[4], uint64_t launches[4]);
 
 #ifdef __cplusplus
 }

@@ -8,9 +8,9 @@
  *
  * What it follows (paper, Section 2.2 "Taliesin: KV memory"): the KV state of a
  * block of prompt text is written to storage after it is computed, loaded again
- * when the same block recurs, checked on load, and -- the design rule "serve
- * without memory, never with wrong memory" -- any record that is missing,
- * damaged or fails a check is not used: the block is recomputed.  Section 3
+ * when the same block recurs, checked when loaded, and -- by that section's
+ * design rule that wrong stored state must never be served -- any record that is
+ * missing, damaged or fails a check is not used: the block is recomputed.  Section 3
  * (Table 1) demands that what is restored is bit-identical to what was saved;
  * Section 5 states that reuse is at whole-block granularity and that the design
  * is fail-closed.  The paper withholds its storage format (end of Section 1),

@@ -229,11 +229,11 @@ class Context:
                                               _ptr(first_bad_page), _stream_handle(stream)), "gk_restore_host")
 
     def gk_get_kernel_times(self) -> dict:
-        """{'verify'|'pack'|'commit': (ms, launches)} since the previous call (needs tuning key profile=1)."""
-        ms = (ctypes.c_double * 3)()
-        n = (ctypes.c_uint64 * 3)()
+        """{'verify'|'pack'|'commit'|'restore': (ms, launches)} since the previous call (needs tuning key profile=1)."""
+        ms = (ctypes.c_double * 4)()
+        n = (ctypes.c_uint64 * 4)()
         self._check(self._lib.gk_get_kernel_times(self._h, ms, n), "gk_get_kernel_times")
-        return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(("verify", "pack", "commit"))}
+        return {name: (float(ms[i]), int(n[i])) for i, name in enumerate(("verify", "pack", "commit", "restore"))}
 
     def gk_get_stats(self) -> dict:
         st = CStats()

@@ -38,6 +38,16 @@
 #ifndef GK_COPY_MINB
 #define GK_COPY_MINB 3
 #endif
+// fused restore kernel: verify ring and commit ring of one CTA
+#ifndef GK_FUSED_VSTAGES
+#define GK_FUSED_VSTAGES 5
+#endif
+#ifndef GK_FUSED_CSTAGES
+#define GK_FUSED_CSTAGES 4
+#endif
+#ifndef GK_FUSED_MINB
+#define GK_FUSED_MINB 2
+#endif
 
 using namespace gk;
 
@@ -46,6 +56,7 @@ namespace {
 using VerifyCfg = StreamCfg<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES>;
 using PackCfg = StreamCfg<kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES>;
 using CommitCfg = StreamCfg<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES>;
+using FusedCfg = RestoreCfg<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES>;
 
 constexpr int kSlots = 2;  // host-tier staging ring
 
@@ -69,7 +80,8 @@ struct gk_ctx {
     GeomDev gd{};
     int device = 0;
     int sm_count = 0;
-    int occ_verify = 0, occ_pack = 0, occ_commit = 0;
+    int occ_verify = 0, occ_pack = 0, occ_commit = 0, occ_fused = 0;
+    bool fused = true;           // restore runs verify and commit in one launch
     uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
     uint32_t commit_seg_tiles = 0;
     uint32_t grid_cap = 0;       // 0: SMs * occupancy
@@ -99,8 +111,8 @@ struct gk_ctx {
     struct ProfSlot { cudaEvent_t a, b; int cls; };
     std::vector<ProfSlot> prof_pool;
     size_t prof_used = 0;
-    double prof_ms[3] = {0, 0, 0};
-    uint64_t prof_launches[3] = {0, 0, 0};
+    double prof_ms[4] = {0, 0, 0, 0};
+    uint64_t prof_launches[4] = {0, 0, 0, 0};
 
     gk_stats stats{};
     char err[512] = {0};
@@ -211,7 +223,7 @@ Tiling commit_tiling(const gk_ctx *c)
 
 // Views into the workspace for one call.
 struct WsLayout {
-    size_t jobs, page_job, seg_res, bad_range, bad_dup, bad_crc, claims, total;
+    size_t jobs, page_job, seg_res, bad_range, bad_dup, bad_crc, page_cnt, job_done, claims, total;
 };
 
 WsLayout ws_layout(uint32_t n_jobs, uint64_t total_pages, uint32_t nseg_max, uint64_t num_pages)
@@ -224,6 +236,8 @@ WsLayout ws_layout(uint32_t n_jobs, uint64_t total_pages, uint32_t nseg_max, uin
     l.bad_range = o; o = align_up(o + (size_t)n_jobs * 4, 256);
     l.bad_dup = o;   o = align_up(o + (size_t)n_jobs * 4, 256);
     l.bad_crc = o;   o = align_up(o + (size_t)n_jobs * 4, 256);
+    l.page_cnt = o;  o = align_up(o + (size_t)total_pages * 4, 256);
+    l.job_done = o;  o = align_up(o + (size_t)n_jobs * 4, 256);
     l.claims = o;    o = align_up(o + (size_t)num_pages * 8, 256);
     l.total = o;
     return l;
@@ -273,6 +287,8 @@ WorkDev make_work(const gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t 
     w.bad_range = (int32_t *)(c->d_ws + l.bad_range);
     w.bad_dup = (int32_t *)(c->d_ws + l.bad_dup);
     w.bad_crc = (int32_t *)(c->d_ws + l.bad_crc);
+    w.page_cnt = (uint32_t *)(c->d_ws + l.page_cnt);
+    w.job_done = (uint32_t *)(c->d_ws + l.job_done);
     w.claims = (unsigned long long *)(c->d_ws + l.claims);
     w.error = c->d_error;
     w.init_term = c->d_init_term;
@@ -330,8 +346,9 @@ uint32_t stream_grid(const gk_ctx *c, int occ, uint32_t n_items)
 template <class Cfg, int MODE, int NT, int SB, int ST, int MINB>
 int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
 {
-    if (P.n_items == 0) return GK_OK;
-    const uint32_t grid = stream_grid(c, occ, P.n_items);
+    const uint32_t items = MODE == kCommit ? P.n_items_c : P.n_items;
+    if (items == 0) return GK_OK;
+    const uint32_t grid = stream_grid(c, occ, items);
     gk_ctx::ProfSlot *slot = nullptr;
     if (c->profile) {
         if (c->prof_used == c->prof_pool.size()) {
@@ -362,6 +379,32 @@ int launch_pack(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 int launch_commit(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
     return launch_stream<CommitCfg, kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES, GK_COPY_MINB>(c, c->occ_commit, P, st);
+}
+
+// verify + commit in one launch; per-kernel timing books it under "commit" (index 2)
+int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
+{
+    const uint32_t items = P.n_items > P.n_items_c ? P.n_items : P.n_items_c;
+    if (items == 0) return GK_OK;
+    const uint32_t grid = stream_grid(c, c->occ_fused, items);
+    gk_ctx::ProfSlot *slot = nullptr;
+    if (c->profile) {
+        if (c->prof_used == c->prof_pool.size()) {
+            gk_ctx::ProfSlot ns{};
+            GK_CUDA(c, cudaEventCreate(&ns.a));
+            GK_CUDA(c, cudaEventCreate(&ns.b));
+            c->prof_pool.push_back(ns);
+        }
+        slot = &c->prof_pool[c->prof_used++];
+        slot->cls = 3;
+        GK_CUDA(c, cudaEventRecord(slot->a, st));
+    }
+    restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES, GK_FUSED_MINB>
+        <<<grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st>>>(P);
+    GK_CUDA(c, cudaGetLastError());
+    if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
+    c->stats.kernels_launched++;
+    return GK_OK;
 }
 
 int launch_validate(gk_ctx *c, const WorkDev &w, uint64_t num_pages, int clear_claims, cudaStream_t st)
@@ -463,7 +506,11 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack, kp, PackCfg::kThreads, PackCfg::kSmemBytes) != cudaSuccess ||
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_commit, kc, CommitCfg::kThreads, CommitCfg::kSmemBytes) != cudaSuccess)
         return bail(GK_ERR_CUDA);
-    if (c->occ_verify < 1 || c->occ_pack < 1 || c->occ_commit < 1) return bail(GK_ERR_UNSUPPORTED);
+    auto *kf = restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES, GK_FUSED_MINB>;
+    if (cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FusedCfg::kSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_fused, kf, FusedCfg::kThreads, FusedCfg::kSmemBytes) != cudaSuccess)
+        return bail(GK_ERR_CUDA);
+    if (c->occ_verify < 1 || c->occ_pack < 1 || c->occ_commit < 1 || c->occ_fused < 1) return bail(GK_ERR_UNSUPPORTED);
 
     // tables: ones * x^(8*len(t)) for every page fill t, and the per-thread placement constants
     std::vector<uint64_t> init(gd.page_tokens + 1, 0);
@@ -525,6 +572,7 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     else if (!strcmp(key, "commit_seg_tiles")) c->commit_seg_tiles = value;
     else if (!strcmp(key, "grid_cap")) c->grid_cap = value;
     else if (!strcmp(key, "profile")) c->profile = value != 0;
+    else if (!strcmp(key, "fused")) c->fused = value != 0;
     else return fail(c, GK_ERR_ARG, "unknown tuning key %s", key);
     return GK_OK;
 }
@@ -623,14 +671,17 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
     P.w = w;
     P.mask_out = mask_dev;
     P.first_bad_out = first_bad_dev;
-    if (!(c->gd.flags & GK_FLAG_SKIP_VERIFY)) {
-        P.tl = tlv;
-        P.n_items = n_pages * tlv.nseg_max;
-        if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
-        if ((rc = launch_finalize(c, w, tlv, 0, nullptr, st)) != GK_OK) return rc;
+    P.tl = tlv;
+    P.tlc = tlc;
+    P.n_items = n_pages * tlv.nseg_max;
+    P.n_items_c = n_pages * tlc.nseg_max;
+    if (c->gd.flags & GK_FLAG_SKIP_VERIFY) return launch_commit(c, P, st);
+    if (c->fused) {
+        P.fused = 1u;
+        return launch_fused(c, P, st);
     }
-    P.tl = tlc;
-    P.n_items = n_pages * tlc.nseg_max;
+    if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
+    if ((rc = launch_finalize(c, w, tlv, 0, nullptr, st)) != GK_OK) return rc;
     return launch_commit(c, P, st);
 }
 
@@ -786,7 +837,7 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
     return GK_OK;
 }
 
-int gk_get_kernel_times(gk_ctx *c, double ms[3], uint64_t launches[3])
+int gk_get_kernel_times(gk_ctx *c, double ms[4], uint64_t launches[4])
 {
     if (!c || !ms || !launches) return GK_ERR_ARG;
     DeviceGuard guard(c->device);
@@ -799,7 +850,7 @@ int gk_get_kernel_times(gk_ctx *c, double ms[3], uint64_t launches[3])
         c->prof_launches[ps.cls]++;
     }
     c->prof_used = 0;
-    for (int i = 0; i < 3; ++i) {
+    for (int i = 0; i < 4; ++i) {
         ms[i] = c->prof_ms[i];
         launches[i] = c->prof_launches[i];
         c->prof_ms[i] = 0;

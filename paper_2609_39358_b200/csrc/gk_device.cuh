@@ -54,6 +54,8 @@ struct WorkDev {
     int32_t *bad_range;           // [n_jobs] lowest out-of-range table index, or kNoPage
     int32_t *bad_dup;             // [n_jobs] lowest index of a page claimed twice, or kNoPage
     int32_t *bad_crc;             // [n_jobs] lowest page whose checksum differs, or kNoPage
+    uint32_t *page_cnt;           // [total_pages] segments delivered per page (fused restore)
+    uint32_t *job_done;           // [n_jobs] pages finalized per job (fused restore)
     unsigned long long *claims;   // [num_pages] first claimant of each destination page
     uint32_t *error;              // sticky: non-zero once a bounded wait has run out
     const uint64_t *init_term;    // [page_tokens+1] ones * x^(8*len(t)) mod P

@@ -47,6 +47,7 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims)
     int32_t bad = kNoPage;
     for (uint32_t p = threadIdx.x; p < jb.n_pages; p += blockDim.x) {
         w.page_job[jb.page_base + p] = (int32_t)j;
+        w.page_cnt[jb.page_base + p] = 0u;
         if (jb.page_table) {
             const int32_t id = jb.page_table[p];
             if ((id < 0 || (uint64_t)id >= num_pages) && (int32_t)p < bad) bad = (int32_t)p;
@@ -58,6 +59,7 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims)
         w.bad_range[j] = s_bad;
         w.bad_dup[j] = kNoPage;
         w.bad_crc[j] = kNoPage;
+        w.job_done[j] = 0u;
     }
 }
 
@@ -93,12 +95,13 @@ __device__ __forceinline__ uint32_t job_code(const WorkDev &w, uint32_t j, int32
         *first_bad = r;
         return 2u;
     }
-    r = w.bad_crc[j];
+    // written by other CTAs of the same launch in the fused kernel: read at L2
+    r = __ldcg(&w.bad_crc[j]);
     if (r != kNoPage) {
         *first_bad = r;
         return 1u;
     }
-    if (*w.error != 0u) return 4u;
+    if (__ldcg(w.error) != 0u) return 4u;
     return 0u;
 }
 
@@ -131,7 +134,7 @@ __global__ void finalize_kernel(GeomDev g, WorkDev w, Tiling tl, int write_mode,
 }
 
 // ---------------------------------------------------------------------------
-// the streaming kernel
+// the streaming kernels
 // ---------------------------------------------------------------------------
 template <int MODE, int NT, int STAGE_BYTES, int STAGES>
 struct StreamCfg {
@@ -152,12 +155,15 @@ struct StreamCfg {
 
 struct StreamParams {
     GeomDev g;
-    CacheDev cache;   // kPack: source cache; kCommit: destination cache; kVerify: unused
+    CacheDev cache;   // kPack: source cache; kCommit / restore: destination cache; kVerify: unused
     WorkDev w;
-    Tiling tl;
-    uint32_t n_items; // total_pages * nseg_max
-    uint8_t *mask_out;        // kCommit
-    int32_t *first_bad_out;   // kCommit
+    Tiling tl;        // tiling of the CRC modes (verify, pack)
+    Tiling tlc;       // tiling of the commit mode
+    uint32_t n_items;    // CRC work items: pages of the launch * tl.nseg_max
+    uint32_t n_items_c;  // commit work items: pages of the launch * tlc.nseg_max
+    uint32_t fused;      // 1: verify and commit run in one launch; commit waits per job
+    uint8_t *mask_out;        // commit
+    int32_t *first_bad_out;   // commit
 };
 
 struct Item {
@@ -168,13 +174,55 @@ struct Item {
     uint32_t tile_begin, tile_count;
     int32_t phys;
     uint32_t t;
+    uint32_t nseg;
 };
 
-template <int MODE>
-__device__ __forceinline__ bool get_item(const StreamParams &P, uint32_t item, Item &it, bool report)
+// A shared-memory ring of STAGES tiles with a full and an empty barrier each.
+struct Ring {
+    uint8_t *base;    // generic address of stage 0
+    uint32_t stage0;  // shared-window address of stage 0
+    uint32_t full0, empty0;
+};
+
+__device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
 {
-    const uint32_t local = item / P.tl.nseg_max;
-    it.q = item - local * P.tl.nseg_max;
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
+// Fused restore: a job may be committed only after all of its pages have been
+// verified.  The verify side counts finalized pages in job_done[j]; the commit
+// side waits here, with a time limit.  The wait cannot deadlock as long as all
+// CTAs of the launch are resident (the host sizes the grid so), because the
+// verify warps never wait for the commit warps.
+__device__ __forceinline__ bool wait_job_verified(const StreamParams &P, uint32_t j, uint32_t n_pages,
+                                                  volatile uint32_t *abort_flag)
+{
+    const uint32_t *cnt = P.w.job_done + j;
+    if (ld_acquire_u32(cnt) >= n_pages) return true;
+    if (*abort_flag) return false;
+    const unsigned long long t0 = global_timer_ns();
+    uint32_t spins = 0;
+    while (ld_acquire_u32(cnt) < n_pages) {
+        __nanosleep(200);
+        if ((++spins & 0x3fu) == 0u) {
+            if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1u;
+                atomicCAS(P.w.error, 0u, 0x500u);
+                return false;
+            }
+        }
+    }
+    return true;
+}
+
+template <int MODE>
+__device__ __forceinline__ bool get_item(const StreamParams &P, const Tiling &tl, uint32_t item, Item &it, bool report,
+                                         volatile uint32_t *abort_flag)
+{
+    const uint32_t local = item / tl.nseg_max;
+    it.q = item - local * tl.nseg_max;
     const uint32_t gp = P.w.page_begin + local;
     it.gp = gp;
     it.j = (uint32_t)P.w.page_job[gp];
@@ -182,6 +230,8 @@ __device__ __forceinline__ bool get_item(const StreamParams &P, uint32_t item, I
     const JobDev jb = *it.jb;
     it.p = gp - jb.page_base;
     if (MODE == kCommit) {
+        if (P.fused && !jb.missing && P.w.bad_range[it.j] == kNoPage && P.w.bad_dup[it.j] == kNoPage)
+            wait_job_verified(P, it.j, jb.n_pages, abort_flag);
         int32_t fb;
         const uint32_t code = job_code(P.w, it.j, &fb);
         if (report && it.p == 0u && it.q == 0u) {
@@ -193,12 +243,13 @@ __device__ __forceinline__ bool get_item(const StreamParams &P, uint32_t item, I
         if (jb.missing || P.w.bad_range[it.j] != kNoPage) return false;
         if (MODE == kVerify && P.w.bad_dup[it.j] != kNoPage) return false;
     }
-    const PageShape sh = page_shape(P.g, jb, it.p, P.tl);
+    const PageShape sh = page_shape(P.g, jb, it.p, tl);
+    it.nseg = sh.nseg;
     if (it.q >= sh.nseg) return false;
     it.pad = sh.pad;
     it.t = sh.t;
-    it.tile_begin = it.q == 0u ? 0u : sh.ntiles0 + (it.q - 1u) * P.tl.seg_tiles;
-    it.tile_count = it.q == 0u ? sh.ntiles0 : P.tl.seg_tiles;
+    it.tile_begin = it.q == 0u ? 0u : sh.ntiles0 + (it.q - 1u) * tl.seg_tiles;
+    it.tile_count = it.q == 0u ? sh.ntiles0 : tl.seg_tiles;
     it.phys = (MODE != kVerify) ? jb.page_table[it.p] : 0;
     return true;
 }
@@ -363,18 +414,18 @@ struct RingPos {
 // is handed back to the loader.
 template <int U, int MODE, int NT, int STAGE_BYTES, int STAGES>
 struct GranuleSteps {
-    using Cfg = StreamCfg<MODE, NT, STAGE_BYTES, STAGES>;
+    static constexpr int kSps = STAGE_BYTES / (NT * 32);  // 8-word steps per stage
     static __device__ __forceinline__ void run(uint32_t (&R)[64], const uint8_t *smem, uint32_t full0, uint32_t empty0,
                                                RingPos &pos, volatile uint32_t *abort_flag, uint32_t *error, int tid,
                                                int lane)
     {
-        if (U % Cfg::kSps == 0) mbar_wait(full0 + 8u * pos.stage, pos.phase, abort_flag, error, 0x400u | MODE);
+        if (U % kSps == 0) mbar_wait(full0 + 8u * pos.stage, pos.phase, abort_flag, error, 0x400u | MODE);
         const uint32_t *sw = reinterpret_cast<const uint32_t *>(smem + (size_t)pos.stage * STAGE_BYTES) + tid;
         uint32_t w[8];
 #pragma unroll
-        for (int jw = 0; jw < 8; ++jw) w[jw] = sw[((U % Cfg::kSps) * 8 + jw) * NT];
+        for (int jw = 0; jw < 8; ++jw) w[jw] = sw[((U % kSps) * 8 + jw) * NT];
         crc_step8<U>(R, w);
-        if (U % Cfg::kSps == Cfg::kSps - 1) {
+        if (U % kSps == kSps - 1) {
             __syncwarp();
             if (lane == 0) mbar_arrive(empty0 + 8u * pos.stage);
             pos.template advance<STAGES>();
@@ -391,6 +442,245 @@ struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES> {
     }
 };
 
+// ------------------------------ loader role ------------------------------
+// One warp.  Walks this CTA's work items tile by tile, waits for a free stage,
+// and fills it: front padding zeroed by the lanes (CRC modes), scale values
+// gathered by the lanes (pack), everything else by bulk async copies issued by
+// lane 0 that complete on the stage's full barrier.
+template <int MODE, int STAGE_BYTES, int STAGES, bool ZERO_PAD>
+__device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling &tl, uint32_t n_items, const Ring &ring,
+                                            volatile uint32_t *abort_flag, int lane)
+{
+    uint32_t n = 0;
+    uint64_t policy = 0;
+    if (MODE == kCommit || MODE == kPack) policy = policy_evict_first();
+    for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        Item it;
+        if (!get_item<MODE>(P, tl, item, it, false, abort_flag)) continue;
+        const uint8_t *rec = (MODE == kPack) ? nullptr : it.jb->blob + (uint64_t)it.p * P.g.R;
+        const uint32_t slab_len = it.t * P.g.row;
+        for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
+            const uint32_t s = n % STAGES;
+            const uint32_t use = n / STAGES;
+            if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE);
+            uint32_t lead, nreal;
+            uint64_t r0;
+            tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
+            const uint32_t sbase = ring.stage0 + s * STAGE_BYTES;
+            uint8_t *sgen = ring.base + (size_t)s * STAGE_BYTES;
+            if (ZERO_PAD) {
+                for (uint32_t o = lane * 16u; o < lead; o += 512u)
+                    *reinterpret_cast<uint4 *>(sgen + o) = make_uint4(0u, 0u, 0u, 0u);
+            }
+            uint32_t scale_bytes = 0u;
+            if (MODE == kPack && r0 < P.g.S && nreal > 0u) {
+                // scale values of this tile: gathered with ordinary loads
+                const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
+                scale_bytes = (uint32_t)(e1 - r0);
+                for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
+                    const uint32_t v = *reinterpret_cast<const uint32_t *>(scale_addr(P.g, P.cache, i, it.phys));
+                    *reinterpret_cast<uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0)) = v;
+                }
+                fence_proxy_async_smem();
+            }
+            __syncwarp();
+            if (lane == 0 && !*abort_flag) {
+                const uint32_t bar = ring.full0 + 8u * s;
+                if (MODE == kPack) {
+                    const uint32_t data_bytes = nreal - scale_bytes;
+                    if (data_bytes == 0u) {
+                        mbar_arrive(bar);
+                    } else {
+                        mbar_arrive_expect_tx(bar, data_bytes);
+                        uint64_t d0 = r0 + scale_bytes - P.g.S;  // offset in the record's data part
+                        const uint64_t d1 = d0 + data_bytes;
+                        uint32_t so = sbase + lead + scale_bytes;
+                        uint32_t slab = (uint32_t)(d0 / slab_len);
+                        uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
+                        while (d0 < d1) {
+                            uint32_t nb = slab_len - off;
+                            if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
+                            bulk_g2s_hint(so, slab_addr(P.cache, slab, it.phys, off), nb, bar, policy);
+                            d0 += nb;
+                            so += nb;
+                            ++slab;
+                            off = 0u;
+                        }
+                    }
+                } else {
+                    if (nreal == 0u) {
+                        mbar_arrive(bar);
+                    } else {
+                        mbar_arrive_expect_tx(bar, nreal);
+                        if (MODE == kCommit)
+                            bulk_g2s_hint(sbase + lead, rec + r0, nreal, bar, policy);
+                        else
+                            bulk_g2s(sbase + lead, rec + r0, nreal, bar);
+                    }
+                }
+            }
+            __syncwarp();
+        }
+    }
+    // before leaving: every load this CTA issued must have landed
+    if (lane == 0) {
+        for (uint32_t back = 0; back < (uint32_t)STAGES && back < n; ++back) {
+            const uint32_t m = n - 1u - back;
+            mbar_drain(ring.full0 + 8u * (m % STAGES), (m / STAGES) & 1u);
+        }
+    }
+}
+
+// ------------------------------ storer role ------------------------------
+// One warp.  Waits for each tile to land and writes it out with bulk async
+// copies: one contiguous piece into the blob (pack), or one piece per slab into
+// the destination cache plus the scale values by the lanes (commit).  A stage
+// goes back to the loader once the copy of the following tile has been issued
+// and the stage's own copy has finished reading shared memory.
+template <int MODE, int STAGE_BYTES, int STAGES>
+__device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling &tl, uint32_t n_items, const Ring &ring,
+                                            volatile uint32_t *abort_flag, int lane)
+{
+    uint32_t n = 0;
+    for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        Item it;
+        if (!get_item<MODE>(P, tl, item, it, lane == 0, abort_flag)) continue;
+        uint8_t *rec = it.jb->blob + (uint64_t)it.p * P.g.R;
+        const uint32_t slab_len = it.t * P.g.row;
+        for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
+            const uint32_t s = n % STAGES;
+            const bool ok = mbar_wait(ring.full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE);
+            uint32_t lead, nreal;
+            uint64_t r0;
+            tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
+            const uint32_t sbase = ring.stage0 + s * STAGE_BYTES;
+            const uint8_t *sgen = ring.base + (size_t)s * STAGE_BYTES;
+            uint32_t scale_bytes = 0u;
+            if (MODE == kCommit && r0 < P.g.S && nreal > 0u) {
+                const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
+                scale_bytes = (uint32_t)(e1 - r0);
+                if (ok && !*abort_flag) {
+                    for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
+                        const uint32_t v = *reinterpret_cast<const uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0));
+                        *reinterpret_cast<uint32_t *>(scale_addr(P.g, P.cache, i, it.phys)) = v;
+                    }
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                if (ok && !*abort_flag && nreal > 0u) {
+                    if (MODE == kPack) {
+                        bulk_s2g(rec + r0, sbase + lead, nreal);
+                    } else {
+                        const uint32_t data_bytes = nreal - scale_bytes;
+                        uint64_t d0 = r0 + scale_bytes - P.g.S;
+                        const uint64_t d1 = d0 + data_bytes;
+                        uint32_t so = sbase + lead + scale_bytes;
+                        uint32_t slab = (uint32_t)(d0 / slab_len);
+                        uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
+                        while (d0 < d1) {
+                            uint32_t nb = slab_len - off;
+                            if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
+                            bulk_s2g(slab_addr(P.cache, slab, it.phys, off), so, nb);
+                            d0 += nb;
+                            so += nb;
+                            ++slab;
+                            off = 0u;
+                        }
+                    }
+                }
+                bulk_commit();
+                if (n > 0u) {
+                    bulk_wait_read<1>();
+                    mbar_arrive(ring.empty0 + 8u * ((n - 1u) % STAGES));
+                }
+            }
+            __syncwarp();
+        }
+    }
+    if (lane == 0) {
+        bulk_wait_all();
+        if (n > 0u) mbar_arrive(ring.empty0 + 8u * ((n - 1u) % STAGES));
+    }
+}
+
+// ----------------------------- consumer role -----------------------------
+// NT threads.  Reduce each segment to its remainder (see the top of this file)
+// and leave it in seg_res.  In the fused restore kernel the CTA that delivers
+// the last segment of a page also finalizes the page -- merge, compare with the
+// stored checksum -- and counts it in job_done, which the commit side waits on.
+template <int MODE, int NT, int STAGE_BYTES, int STAGES>
+__device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring &ring, uint64_t *red,
+                                              volatile uint32_t *abort_flag, int tid, int warp, int lane)
+{
+    const uint64_t kt = P.w.thread_const[tid];
+    RingPos pos;
+    uint32_t parity_red = 0;
+    constexpr int kTilesPerGran = (NT * 256) / STAGE_BYTES;
+    for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+        Item it;
+        if (!get_item<MODE>(P, P.tl, item, it, false, abort_flag)) continue;
+        uint32_t R[64];
+#pragma unroll
+        for (int i = 0; i < 64; ++i) R[i] = 0u;
+        const uint32_t ngran = it.tile_count / kTilesPerGran;
+        for (uint32_t gi = 0; gi < ngran; ++gi)
+            GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, ring.base, ring.full0, ring.empty0, pos, abort_flag,
+                                                                P.w.error, tid, lane);
+        // merge streams -> thread -> warp -> CTA
+        uint64_t v = thread_remainder<NT>(R, kt);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) v ^= __shfl_xor_sync(0xffffffffu, v, d);
+        uint64_t *slot = red + 8 * parity_red;
+        if (lane == 0) slot[warp] = v;
+        asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
+        if (tid == 0) {
+            uint64_t tot = 0;
+#pragma unroll
+            for (int i = 0; i < NT / 32; ++i) tot ^= slot[i];
+            uint64_t *res = P.w.seg_res + (uint64_t)it.gp * P.tl.nseg_max;
+            if (!P.fused) {
+                res[it.q] = tot;
+            } else {
+                uint64_t r = tot;
+                bool last = true;
+                if (it.nseg > 1u) {
+                    __stcg(&res[it.q], tot);
+                    __threadfence();
+                    last = atomicAdd(&P.w.page_cnt[it.gp], 1u) + 1u == it.nseg;
+                    if (last) {
+                        __threadfence();
+                        r = __ldcg(&res[0]);
+                        for (uint32_t q = 1; q < it.nseg; ++q) r = gf_mul(r, P.w.x_seg) ^ __ldcg(&res[q]);
+                    }
+                }
+                if (last) {
+                    const uint64_t crc = __brevll(r ^ P.w.init_term[it.t] ^ ~0ull);
+                    if (crc != it.jb->checksums[it.p] || *abort_flag) atomicMin(&P.w.bad_crc[it.j], (int32_t)it.p);
+                    __threadfence();
+                    atomicAdd(&P.w.job_done[it.j], 1u);
+                }
+            }
+        }
+        parity_red ^= 1u;
+    }
+}
+
+__device__ __forceinline__ void ring_init(Ring &ring, uint8_t *base, uint64_t *bars, int stages, uint32_t empty_count)
+{
+    ring.base = base;
+    ring.stage0 = smem_u32(base);
+    ring.full0 = smem_u32(bars);
+    ring.empty0 = smem_u32(bars + stages);
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < stages; ++s) {
+            mbar_init(ring.full0 + 8u * s, 1u);
+            mbar_init(ring.empty0 + 8u * s, empty_count);
+        }
+    }
+}
+
+// pack, verify-only and commit-only launches
 template <int MODE, int NT, int STAGE_BYTES, int STAGES, int MINB>
 __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThreads, MINB)
     stream_kernel(const __grid_constant__ StreamParams P)
@@ -399,201 +689,76 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
-    uint64_t *red = bars + 2 * STAGES;                 // [2][8]
+    uint64_t *red = bars + 2 * STAGES;  // [2][8]
     volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
-
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const uint32_t stage0 = smem_u32(smem);
-    const uint32_t full0 = smem_u32(bars);
-    const uint32_t empty0 = smem_u32(bars + STAGES);
 
+    Ring ring;
+    ring_init(ring, smem, bars, STAGES, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)));
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full0 + 8u * s, 1u);
-            mbar_init(empty0 + 8u * s, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)));
-        }
         *abort_flag = 0u;
         fence_mbar_init();
     }
     __syncthreads();
 
     if (warp == Cfg::kLoaderWarp) {
-        // ------------------------------ loader ------------------------------
-        uint32_t n = 0;
-        uint64_t policy = 0;
-        if (MODE == kCommit || MODE == kPack) policy = policy_evict_first();
-        for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
-            Item it;
-            if (!get_item<MODE>(P, item, it, false)) continue;
-            const uint8_t *rec = (MODE == kPack) ? nullptr : it.jb->blob + (uint64_t)it.p * P.g.R;
-            const uint32_t slab_len = it.t * P.g.row;
-            for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
-                const uint32_t s = n % STAGES;
-                const uint32_t use = n / STAGES;
-                if (use > 0u) mbar_wait(empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE);
-                uint32_t lead, nreal;
-                uint64_t r0;
-                tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
-                const uint32_t sbase = stage0 + s * STAGE_BYTES;
-                uint8_t *sgen = smem + (size_t)s * STAGE_BYTES;
-                if (Cfg::kCrc) {
-                    for (uint32_t o = lane * 16u; o < lead; o += 512u)
-                        *reinterpret_cast<uint4 *>(sgen + o) = make_uint4(0u, 0u, 0u, 0u);
-                }
-                uint32_t scale_bytes = 0u;
-                if (MODE == kPack && r0 < P.g.S && nreal > 0u) {
-                    // scale values of this tile: gathered with ordinary loads
-                    const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
-                    scale_bytes = (uint32_t)(e1 - r0);
-                    for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
-                        const uint32_t v = *reinterpret_cast<const uint32_t *>(scale_addr(P.g, P.cache, i, it.phys));
-                        *reinterpret_cast<uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0)) = v;
-                    }
-                    fence_proxy_async_smem();
-                }
-                __syncwarp();
-                if (lane == 0 && !*abort_flag) {
-                    const uint32_t bar = full0 + 8u * s;
-                    if (MODE == kPack) {
-                        const uint32_t data_bytes = nreal - scale_bytes;
-                        if (data_bytes == 0u) {
-                            mbar_arrive(bar);
-                        } else {
-                            mbar_arrive_expect_tx(bar, data_bytes);
-                            uint64_t d0 = r0 + scale_bytes - P.g.S;  // offset in the record's data part
-                            const uint64_t d1 = d0 + data_bytes;
-                            uint32_t so = sbase + lead + scale_bytes;
-                            uint32_t slab = (uint32_t)(d0 / slab_len);
-                            uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
-                            while (d0 < d1) {
-                                uint32_t nb = slab_len - off;
-                                if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
-                                bulk_g2s_hint(so, slab_addr(P.cache, slab, it.phys, off), nb, bar, policy);
-                                d0 += nb;
-                                so += nb;
-                                ++slab;
-                                off = 0u;
-                            }
-                        }
-                    } else {
-                        if (nreal == 0u) {
-                            mbar_arrive(bar);
-                        } else {
-                            mbar_arrive_expect_tx(bar, nreal);
-                            if (MODE == kCommit)
-                                bulk_g2s_hint(sbase + lead, rec + r0, nreal, bar, policy);
-                            else
-                                bulk_g2s(sbase + lead, rec + r0, nreal, bar);
-                        }
-                    }
-                }
-                __syncwarp();
-            }
-        }
-        // before leaving: every load this CTA issued must have landed
-        if (lane == 0) {
-            for (uint32_t back = 0; back < (uint32_t)STAGES && back < n; ++back) {
-                const uint32_t m = n - 1u - back;
-                mbar_drain(full0 + 8u * (m % STAGES), (m / STAGES) & 1u);
-            }
-        }
+        loader_role<MODE, STAGE_BYTES, STAGES, Cfg::kCrc>(P, MODE == kCommit ? P.tlc : P.tl,
+                                                          MODE == kCommit ? P.n_items_c : P.n_items, ring, abort_flag,
+                                                          lane);
     } else if (Cfg::kStore && warp == Cfg::kStorerWarp) {
-        // ------------------------------ storer ------------------------------
-        uint32_t n = 0;
-        for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
-            Item it;
-            if (!get_item<MODE>(P, item, it, lane == 0)) continue;
-            uint8_t *rec = it.jb->blob + (uint64_t)it.p * P.g.R;
-            const uint32_t slab_len = it.t * P.g.row;
-            for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
-                const uint32_t s = n % STAGES;
-                const bool ok = mbar_wait(full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE);
-                uint32_t lead, nreal;
-                uint64_t r0;
-                tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
-                const uint32_t sbase = stage0 + s * STAGE_BYTES;
-                const uint8_t *sgen = smem + (size_t)s * STAGE_BYTES;
-                uint32_t scale_bytes = 0u;
-                if (MODE == kCommit && r0 < P.g.S && nreal > 0u) {
-                    const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
-                    scale_bytes = (uint32_t)(e1 - r0);
-                    if (ok && !*abort_flag) {
-                        for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
-                            const uint32_t v =
-                                *reinterpret_cast<const uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0));
-                            *reinterpret_cast<uint32_t *>(scale_addr(P.g, P.cache, i, it.phys)) = v;
-                        }
-                    }
-                }
-                __syncwarp();
-                if (lane == 0) {
-                    if (ok && !*abort_flag && nreal > 0u) {
-                        if (MODE == kPack) {
-                            bulk_s2g(rec + r0, sbase + lead, nreal);
-                        } else {
-                            const uint32_t data_bytes = nreal - scale_bytes;
-                            uint64_t d0 = r0 + scale_bytes - P.g.S;
-                            const uint64_t d1 = d0 + data_bytes;
-                            uint32_t so = sbase + lead + scale_bytes;
-                            uint32_t slab = (uint32_t)(d0 / slab_len);
-                            uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
-                            while (d0 < d1) {
-                                uint32_t nb = slab_len - off;
-                                if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
-                                bulk_s2g(slab_addr(P.cache, slab, it.phys, off), so, nb);
-                                d0 += nb;
-                                so += nb;
-                                ++slab;
-                                off = 0u;
-                            }
-                        }
-                    }
-                    bulk_commit();
-                    // the store of the previous tile has finished reading its stage
-                    if (n > 0u) {
-                        bulk_wait_read<1>();
-                        mbar_arrive(empty0 + 8u * ((n - 1u) % STAGES));
-                    }
-                }
-                __syncwarp();
-            }
-        }
-        if (lane == 0) {
-            bulk_wait_all();
-            if (n > 0u) mbar_arrive(empty0 + 8u * ((n - 1u) % STAGES));
-        }
+        storer_role<MODE, STAGE_BYTES, STAGES>(P, MODE == kCommit ? P.tlc : P.tl,
+                                               MODE == kCommit ? P.n_items_c : P.n_items, ring, abort_flag, lane);
     } else if constexpr (Cfg::kCrc) {
-        // ----------------------------- consumers ----------------------------
-        const int tid = threadIdx.x;  // consumer warps come first: 0..NT-1
-        const uint64_t kt = P.w.thread_const[tid];
-        RingPos pos;
-        uint32_t parity_red = 0;
-        for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
-            Item it;
-            if (!get_item<MODE>(P, item, it, false)) continue;
-            uint32_t R[64];
-#pragma unroll
-            for (int i = 0; i < 64; ++i) R[i] = 0u;
-            const uint32_t ngran = it.tile_count / Cfg::kTilesPerGran;
-            for (uint32_t gi = 0; gi < ngran; ++gi)
-                GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, pos, abort_flag, P.w.error,
-                                                                    tid, lane);
-            // merge streams -> thread -> warp -> CTA
-            uint64_t v = thread_remainder<NT>(R, kt);
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) v ^= __shfl_xor_sync(0xffffffffu, v, d);
-            uint64_t *slot = red + 8 * parity_red;
-            if (lane == 0) slot[warp] = v;
-            asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
-            if (tid == 0) {
-                uint64_t tot = 0;
-#pragma unroll
-                for (int i = 0; i < Cfg::kConsWarps; ++i) tot ^= slot[i];
-                P.w.seg_res[(uint64_t)it.gp * P.tl.nseg_max + it.q] = tot;
-            }
-            parity_red ^= 1u;
-        }
+        consumer_role<MODE, NT, STAGE_BYTES, STAGES>(P, ring, red, abort_flag, threadIdx.x, warp, lane);
+    }
+    __syncthreads();
+}
+
+// Fused restore: the verify pipeline (loader warp + NT consumer threads) and the
+// commit pipeline (loader warp + storer warp) of one CTA run side by side on
+// two rings.  Verify is bound by the integer pipes, commit by DRAM, so the two
+// overlap; fail-closed order is kept per job by wait_job_verified().
+template <int NT, int VSB, int VST, int CSB, int CST>
+struct RestoreCfg {
+    static constexpr int kConsWarps = NT / 32;
+    static constexpr int kThreads = NT + 96;
+    static constexpr size_t kSmemBytes =
+        (size_t)VST * VSB + (size_t)CST * CSB + 2 * (VST + CST) * 8 + 2 * 8 * 8 + 16 + 128;
+};
+
+template <int NT, int VSB, int VST, int CSB, int CST, int MINB>
+__global__ void __launch_bounds__(NT + 96, MINB) restore_kernel(const __grid_constant__ StreamParams P)
+{
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    uint8_t *vbase = smem;
+    uint8_t *cbase = smem + (size_t)VST * VSB;
+    uint64_t *vbars = (uint64_t *)(cbase + (size_t)CST * CSB);
+    uint64_t *cbars = vbars + 2 * VST;
+    uint64_t *red = cbars + 2 * CST;  // [2][8]
+    volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+
+    Ring vring, cring;
+    ring_init(vring, vbase, vbars, VST, (uint32_t)(NT / 32));
+    ring_init(cring, cbase, cbars, CST, 1u);
+    if (threadIdx.x == 0) {
+        *abort_flag = 0u;
+        fence_mbar_init();
+    }
+    __syncthreads();
+
+    constexpr int kCons = NT / 32;
+    if (warp < kCons) {
+        consumer_role<kVerify, NT, VSB, VST>(P, vring, red, abort_flag, threadIdx.x, warp, lane);
+    } else if (warp == kCons) {
+        loader_role<kVerify, VSB, VST, true>(P, P.tl, P.n_items, vring, abort_flag, lane);
+    } else if (warp == kCons + 1) {
+        loader_role<kCommit, CSB, CST, false>(P, P.tlc, P.n_items_c, cring, abort_flag, lane);
+    } else {
+        storer_role<kCommit, CSB, CST>(P, P.tlc, P.n_items_c, cring, abort_flag, lane);
     }
     __syncthreads();
 }
