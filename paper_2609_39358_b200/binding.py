@@ -16,7 +16,7 @@ from typing import Optional, Sequence
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libgk.so")
+LIB_PATH = os.environ.get("GK_LIB_PATH") or os.path.join(_HERE, "libgk.so")
 
 GK_OK = 0
 GK_BF16, GK_FP8_E4M3 = 0, 1

@@ -23,6 +23,12 @@
 #ifndef GK_CRC_STAGES
 #define GK_CRC_STAGES 6
 #endif
+#ifndef GK_PACK_STAGE
+#define GK_PACK_STAGE GK_CRC_STAGE
+#endif
+#ifndef GK_PACK_STAGES
+#define GK_PACK_STAGES GK_CRC_STAGES
+#endif
 #ifndef GK_VERIFY_MINB
 #define GK_VERIFY_MINB 3
 #endif
@@ -54,7 +60,7 @@ using namespace gk;
 namespace {
 
 using VerifyCfg = StreamCfg<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES>;
-using PackCfg = StreamCfg<kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES>;
+using PackCfg = StreamCfg<kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES>;
 using CommitCfg = StreamCfg<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES>;
 using FusedCfg = RestoreCfg<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES>;
 
@@ -195,15 +201,15 @@ int check_cache(gk_ctx *c, const gk_cache *k, CacheDev *out)
     return GK_OK;
 }
 
-Tiling crc_tiling(const gk_ctx *c)
+Tiling crc_tiling(const gk_ctx *c, uint32_t stage_bytes = GK_CRC_STAGE)
 {
     Tiling t;
-    t.stage_bytes = GK_CRC_STAGE;
+    t.stage_bytes = stage_bytes;
     t.gran_bytes = VerifyCfg::kGran;
     const uint32_t gran_full = (uint32_t)((c->gd.R + t.gran_bytes - 1) / t.gran_bytes);
     uint32_t sg = c->seg_granules ? c->seg_granules : gran_full;
     if (sg > gran_full) sg = gran_full;
-    t.seg_tiles = sg * VerifyCfg::kTilesPerGran;
+    t.seg_tiles = sg * (t.gran_bytes / stage_bytes);
     t.nseg_max = (gran_full + sg - 1) / sg;
     return t;
 }
@@ -374,7 +380,7 @@ int launch_verify(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 }
 int launch_pack(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
-    return launch_stream<PackCfg, kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_PACK_MINB>(c, c->occ_pack, P, st);
+    return launch_stream<PackCfg, kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>(c, c->occ_pack, P, st);
 }
 int launch_commit(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
@@ -496,7 +502,7 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
     c->sm_count = prop.multiProcessorCount;
 
     auto *kv = stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB>;
-    auto *kp = stream_kernel<kPack, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_PACK_MINB>;
+    auto *kp = stream_kernel<kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>;
     auto *kc = stream_kernel<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES, GK_COPY_MINB>;
     if (cudaFuncSetAttribute(kv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VerifyCfg::kSmemBytes) != cudaSuccess ||
         cudaFuncSetAttribute(kp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PackCfg::kSmemBytes) != cudaSuccess ||
@@ -591,7 +597,7 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
     for (uint32_t j = 0; j < n_jobs; ++j)
         if (!jobs[j].blob || !jobs[j].checksums) return fail(c, GK_ERR_ARG, "job %u: null output", j);
 
-    const Tiling tl = crc_tiling(c);
+    const Tiling tl = crc_tiling(c, GK_PACK_STAGE);
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
     const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
