@@ -61,6 +61,7 @@ extern "C" {
 #define GK_ERR_CUDA (-4)        /* a CUDA call failed; see gk_last_error */
 #define GK_ERR_NOMEM (-5)       /* workspace allocation failed */
 #define GK_ERR_DEVICE_WAIT (-6) /* reported by gk_get_stats: a bounded device wait ran out */
+#define GK_ERR_TOO_LARGE (-7)   /* gk_page_checksums_noalloc: request exceeds its fixed scratch */
 
 #define GK_BF16 0u
 #define GK_FP8_E4M3 1u
@@ -187,6 +188,42 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * "fused" (1, the default: gk_restore verifies and commits in one launch; 0: a
  * verify launch, a checksum-compare launch and a commit launch). */
 int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
+
+/* Page checksums of a device blob for callers that must not allocate.  (The
+ * paper has no counterpart to this entry point; it exists for integration.)
+ *
+ * Everything else in this library works through a gk_ctx, and creating or
+ * growing a context calls cudaMalloc and cudaMallocHost.  Some callers cannot
+ * afford that: a serving engine that has already handed all free HBM to its own
+ * KV-cache pool (a late cudaMalloc can fail there, and it synchronises the whole
+ * device in the middle of serving), or a background scrubber that re-checks
+ * stored blobs beside a running engine and has to stay out of its memory
+ * budget.  For them this call computes checksums_dev[p] = CRC-64/XZ of page record
+ * p of the blob -- the same values gk_page_checksums writes -- and allocates
+ * nothing: no cudaMalloc, cudaFree, cudaMallocHost or any other allocating
+ * routine, no context.  Its scratch is one fixed array of about 133 KiB inside the
+ * library's device image, which every GPU that loads the library holds until the
+ * process exits.
+ *
+ * Limits: at most GK_NOALLOC_MAX_PAGES pages per call (n_tokens <=
+ * GK_NOALLOC_MAX_PAGES * page_tokens) and page_tokens <= GK_NOALLOC_MAX_PAGE_TOKENS;
+ * beyond either the call does nothing and returns GK_ERR_TOO_LARGE.  geom->flags
+ * is ignored.  Other returns: GK_ERR_ARG, GK_ERR_UNSUPPORTED (alignment rules as
+ * above; device not sm_100), GK_ERR_CUDA.
+ *
+ * The first call on a device looks up the scratch array's device address and
+ * sets the kernel's shared-memory attribute, once, with that device current;
+ * make that first call before any stream capture is begun.  All calls on a
+ * device share the one scratch array, which still holds the previous call's
+ * contents when a call starts (the call resets what it needs): two calls that
+ * overlap on the GPU -- different streams, or the same blob checked from two
+ * threads -- race on it and may both return wrong checksums, so serialise them.
+ * Work is enqueued on `stream`; checksums_dev is valid once it has been
+ * synchronised. */
+#define GK_NOALLOC_MAX_PAGES 8192u
+#define GK_NOALLOC_MAX_PAGE_TOKENS 256u
+int gk_page_checksums_noalloc(const gk_geom *geom, const void *blob_dev, uint32_t n_tokens,
+                              uint64_t *checksums_dev, int device, void *stream);
 
 /* Per-kernel device time of the streaming kernels, for measurements.  With the
  * tuning key "profile" set to 1 every launch of a streaming kernel is bracketed

@@ -24,7 +24,8 @@ GK_FLAG_SKIP_VERIFY = 1
 JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
 
 EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",
-           "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times"]
+           "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times",
+           "gk_page_checksums_noalloc"]
 
 
 class GkError(RuntimeError):
@@ -93,6 +94,8 @@ def load_library() -> ctypes.CDLL:
     L.gk_get_stats.argtypes = [vp, ctypes.POINTER(CStats)]
     L.gk_get_kernel_times.restype = ctypes.c_int
     L.gk_get_kernel_times.argtypes = [vp, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_uint64)]
+    L.gk_page_checksums_noalloc.restype = ctypes.c_int
+    L.gk_page_checksums_noalloc.argtypes = [ctypes.POINTER(CGeom), vp, u32, vp, ctypes.c_int, vp]
     L.gk_ctx_set_tuning.restype = ctypes.c_int
     L.gk_ctx_set_tuning.argtypes = [vp, ctypes.c_char_p, u32]
     _lib = L
@@ -161,6 +164,23 @@ def gk_blob_size(geom: Geom, n_tokens: int) -> tuple[int, int]:
     if rc != GK_OK:
         raise GkError(rc, "gk_blob_size")
     return int(nb.value), int(npg.value)
+
+
+GK_NOALLOC_MAX_PAGES = 8192
+GK_NOALLOC_MAX_PAGE_TOKENS = 256
+
+
+def gk_page_checksums_noalloc(geom: Geom, blob: torch.Tensor, n_tokens: int, checksums: torch.Tensor,
+                              device: int = 0, stream=None) -> None:
+    """Page checksums of a device blob through the entry point that allocates
+    nothing and needs no context (see gk.h: fixed scratch, at most
+    GK_NOALLOC_MAX_PAGES pages per call, calls on one device must not overlap)."""
+    cg = geom.c()
+    sh = 0 if stream is None and not torch.cuda.is_available() else _stream_handle(stream)
+    rc = load_library().gk_page_checksums_noalloc(ctypes.byref(cg), _ptr(blob), n_tokens, _ptr(checksums),
+                                                  device, sh)
+    if rc != GK_OK:
+        raise GkError(rc, "gk_page_checksums_noalloc")
 
 
 class Context:

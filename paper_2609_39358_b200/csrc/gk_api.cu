@@ -9,6 +9,7 @@
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -873,6 +874,197 @@ int gk_get_stats(gk_ctx *c, gk_stats *out)
     GK_CUDA(c, cudaMemcpy(&e, c->d_error, 4, cudaMemcpyDeviceToHost));
     c->stats.device_wait_expired = e;
     *out = c->stats;
+    return GK_OK;
+}
+
+// ---------------------------------------------------------------------------
+// gk_page_checksums_noalloc: page checksums without any allocation.
+//
+// Same kernels as gk_page_checksums (verify-mode streaming kernel, then the
+// checksum-writing finalize kernel), but every byte of scratch -- job record,
+// page map, per-page remainders, result words, the GF(2) tables -- lives in
+// the file-scope device array below instead of a context's workspace.
+// ---------------------------------------------------------------------------
+}  // extern "C"
+
+namespace {
+
+constexpr uint32_t kNoallocMaxPages = GK_NOALLOC_MAX_PAGES;
+constexpr uint32_t kNoallocMaxPageTokens = GK_NOALLOC_MAX_PAGE_TOKENS;
+
+// Layout of the static scratch (all offsets multiples of 256 bytes).
+struct NoallocLayout {
+    static constexpr size_t job = 0;                                        // JobDev
+    static constexpr size_t words = 256;                                    // bad_range, bad_dup, bad_crc, job_done, error
+    static constexpr size_t thread_const = 512;                             // [GK_CRC_NT] u64
+    static constexpr size_t init_term = thread_const + 8 * 256;             // [max page tokens + 1] u64
+    static constexpr size_t page_job = init_term + 8 * (kNoallocMaxPageTokens + 1) + 248;  // [max pages] i32
+    static constexpr size_t page_cnt = page_job + 4 * (size_t)kNoallocMaxPages;            // [max pages] u32
+    static constexpr size_t seg_res = page_cnt + 4 * (size_t)kNoallocMaxPages;             // [max pages] u64
+    static constexpr size_t total = seg_res + 8 * (size_t)kNoallocMaxPages;
+};
+static_assert(GK_CRC_NT <= 256, "thread constant table");
+static_assert(NoallocLayout::page_job % 256 == 0 && NoallocLayout::seg_res % 8 == 0, "scratch alignment");
+
+// The scratch itself: about 133 KiB per GPU that loads the library, held until exit.
+// In host code this name is only a stand-in for the symbol; the device address
+// comes from cudaGetSymbolAddress (noalloc_setup below).
+static __device__ __align__(256) unsigned char g_noalloc_scratch[NoallocLayout::total];
+
+__device__ uint64_t dev_xpow(uint64_t n)
+{
+    uint64_t r = 1, base = 2;
+    while (n) {
+        if (n & 1ull) r = gf_mul(r, base);
+        base = gf_mul(base, base);
+        n >>= 1;
+    }
+    return r;
+}
+
+// One CTA.  Writes the job record and the tables into the scratch and resets
+// every word that has to start from a known value; the array keeps whatever the
+// previous call left behind.
+__global__ void noalloc_setup_kernel(unsigned char *scratch, JobDev job, GeomDev g)
+{
+    JobDev *jd = reinterpret_cast<JobDev *>(scratch + NoallocLayout::job);
+    int32_t *words = reinterpret_cast<int32_t *>(scratch + NoallocLayout::words);
+    uint64_t *tc = reinterpret_cast<uint64_t *>(scratch + NoallocLayout::thread_const);
+    uint64_t *it = reinterpret_cast<uint64_t *>(scratch + NoallocLayout::init_term);
+    int32_t *page_job = reinterpret_cast<int32_t *>(scratch + NoallocLayout::page_job);
+    uint32_t *page_cnt = reinterpret_cast<uint32_t *>(scratch + NoallocLayout::page_cnt);
+    if (threadIdx.x == 0) {
+        *jd = job;
+        words[0] = kNoPage;  // bad_range
+        words[1] = kNoPage;  // bad_dup
+        words[2] = kNoPage;  // bad_crc
+        words[3] = 0;        // job_done
+        words[4] = 0;        // error word
+    }
+    for (uint32_t t = threadIdx.x; t < (uint32_t)GK_CRC_NT; t += blockDim.x)
+        tc[t] = dev_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);
+    for (uint32_t t = threadIdx.x; t <= g.page_tokens; t += blockDim.x)
+        it[t] = t ? gf_mul(~0ull, dev_xpow(8ull * (g.S + (uint64_t)t * g.tokB))) : 0ull;
+    for (uint32_t p = threadIdx.x; p < job.n_pages; p += blockDim.x) {
+        page_job[p] = 0;
+        page_cnt[p] = 0u;
+    }
+}
+
+struct NoallocDevice {
+    unsigned char *scratch = nullptr;
+    int sm_count = 0;
+    int occ = 0;
+    bool ready = false;
+};
+NoallocDevice g_noalloc_dev[64];
+std::mutex g_noalloc_mutex;
+
+// Once per device, with that device current: resolve the scratch array's device
+// address and prepare the kernel for its dynamic shared memory size.
+int noalloc_setup(int device, NoallocDevice **out)
+{
+    if (device < 0 || device >= 64) return GK_ERR_ARG;
+    std::lock_guard<std::mutex> lock(g_noalloc_mutex);
+    NoallocDevice &d = g_noalloc_dev[device];
+    if (!d.ready) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_noalloc_scratch) != cudaSuccess || ptr == nullptr) {
+            cudaGetLastError();
+            return GK_ERR_CUDA;
+        }
+        int major = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess ||
+            cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) {
+            cudaGetLastError();
+            return GK_ERR_CUDA;
+        }
+        if (major != 10) return GK_ERR_UNSUPPORTED;
+        auto *kv = stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB>;
+        if (cudaFuncSetAttribute(kv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VerifyCfg::kSmemBytes) != cudaSuccess ||
+            cudaOccupancyMaxActiveBlocksPerMultiprocessor(&d.occ, kv, VerifyCfg::kThreads, VerifyCfg::kSmemBytes) != cudaSuccess ||
+            d.occ < 1) {
+            cudaGetLastError();
+            return GK_ERR_CUDA;
+        }
+        d.scratch = static_cast<unsigned char *>(ptr);
+        d.ready = true;
+    }
+    *out = &d;
+    return GK_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int gk_page_checksums_noalloc(const gk_geom *geom, const void *blob_dev, uint32_t n_tokens, uint64_t *checksums_dev,
+                              int device, void *stream)
+{
+    GeomDev gd;
+    int rc = check_geom(geom, &gd);
+    if (rc != GK_OK) return rc;
+    if (!blob_dev || !checksums_dev || n_tokens == 0) return GK_ERR_ARG;
+    if (((uintptr_t)blob_dev & 15u) || ((uintptr_t)checksums_dev & 7u)) return GK_ERR_UNSUPPORTED;
+    const uint64_t pages = ((uint64_t)n_tokens + gd.page_tokens - 1) / gd.page_tokens;
+    if (pages > kNoallocMaxPages || gd.page_tokens > kNoallocMaxPageTokens) return GK_ERR_TOO_LARGE;
+
+    DeviceGuard guard(device);
+    NoallocDevice *nd = nullptr;
+    if ((rc = noalloc_setup(device, &nd)) != GK_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned char *sc = nd->scratch;
+
+    // one segment per page: the scratch holds one remainder per page
+    Tiling tl;
+    tl.stage_bytes = GK_CRC_STAGE;
+    tl.gran_bytes = VerifyCfg::kGran;
+    const uint32_t gran_full = (uint32_t)((gd.R + tl.gran_bytes - 1) / tl.gran_bytes);
+    tl.seg_tiles = gran_full * VerifyCfg::kTilesPerGran;
+    tl.nseg_max = 1;
+
+    JobDev job{};
+    job.blob = (uint8_t *)const_cast<void *>(blob_dev);
+    job.checksums = checksums_dev;
+    job.page_table = nullptr;
+    job.n_tokens = n_tokens;
+    job.n_pages = (uint32_t)pages;
+    job.page_base = 0;
+    job.missing = 0;
+
+    int32_t *words = reinterpret_cast<int32_t *>(sc + NoallocLayout::words);
+    WorkDev w{};
+    w.jobs = reinterpret_cast<const JobDev *>(sc + NoallocLayout::job);
+    w.n_jobs = 1;
+    w.page_begin = 0;
+    w.total_pages = (uint32_t)pages;
+    w.page_job = reinterpret_cast<int32_t *>(sc + NoallocLayout::page_job);
+    w.seg_res = reinterpret_cast<uint64_t *>(sc + NoallocLayout::seg_res);
+    w.bad_range = words + 0;
+    w.bad_dup = words + 1;
+    w.bad_crc = words + 2;
+    w.page_cnt = reinterpret_cast<uint32_t *>(sc + NoallocLayout::page_cnt);
+    w.job_done = reinterpret_cast<uint32_t *>(words + 3);
+    w.claims = nullptr;
+    w.error = reinterpret_cast<uint32_t *>(words + 4);
+    w.init_term = reinterpret_cast<const uint64_t *>(sc + NoallocLayout::init_term);
+    w.thread_const = reinterpret_cast<const uint64_t *>(sc + NoallocLayout::thread_const);
+    w.x_seg = gf_xpow(8ull * tl.seg_tiles * tl.stage_bytes);
+
+    noalloc_setup_kernel<<<1, 256, 0, st>>>(sc, job, gd);
+    if (cudaGetLastError() != cudaSuccess) return GK_ERR_CUDA;
+    StreamParams P{};
+    P.g = gd;
+    P.w = w;
+    P.tl = tl;
+    P.n_items = (uint32_t)pages;
+    uint32_t grid = (uint32_t)(nd->sm_count * nd->occ);
+    if (grid > P.n_items) grid = P.n_items;
+    stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB>
+        <<<grid, VerifyCfg::kThreads, VerifyCfg::kSmemBytes, st>>>(P);
+    if (cudaGetLastError() != cudaSuccess) return GK_ERR_CUDA;
+    finalize_kernel<<<(uint32_t)((pages + 127) / 128), 128, 0, st>>>(gd, w, tl, 1, nullptr);
+    if (cudaGetLastError() != cudaSuccess) return GK_ERR_CUDA;
     return GK_OK;
 }
 
