@@ -452,8 +452,6 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                                             volatile uint32_t *abort_flag, int lane)
 {
     uint32_t n = 0;
-    uint64_t policy = 0;
-    if (MODE == kCommit || MODE == kPack) policy = policy_evict_first();
     for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
         Item it;
         if (!get_item<MODE>(P, tl, item, it, false, abort_flag)) continue;
@@ -500,7 +498,7 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                         while (d0 < d1) {
                             uint32_t nb = slab_len - off;
                             if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
-                            bulk_g2s_hint(so, slab_addr(P.cache, slab, it.phys, off), nb, bar, policy);
+                            bulk_g2s(so, slab_addr(P.cache, slab, it.phys, off), nb, bar);
                             d0 += nb;
                             so += nb;
                             ++slab;
@@ -512,9 +510,6 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                         mbar_arrive(bar);
                     } else {
                         mbar_arrive_expect_tx(bar, nreal);
-                        if (MODE == kCommit)
-                            bulk_g2s_hint(sbase + lead, rec + r0, nreal, bar, policy);
-                        else
                             bulk_g2s(sbase + lead, rec + r0, nreal, bar);
                     }
                 }
