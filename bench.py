@@ -55,6 +55,8 @@ def parse_args():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline-blocks", type=int, default=4)
+    ap.add_argument("--reference-seconds", type=float, default=100.0,
+                    help="--impl reference: target wall time of all steps together (sizes the sample)")
     return ap.parse_args()
 
 
@@ -139,6 +141,58 @@ class ClockSampler:
 
 
 # ---------------------------------------------------------------------------
+# ranks: one process per GPU, no data-path collective
+# ---------------------------------------------------------------------------
+class RankComm:
+    """Rendezvous, barrier and reductions of scalars over the ranks of a
+    torch.distributed.run launch (env: RANK, LOCAL_RANK, WORLD_SIZE, MASTER_*).
+    The data path itself never communicates; this is only for timing."""
+
+    def __init__(self, backend: str, device=None):
+        import torch
+        import torch.distributed as dist
+        self.torch, self.dist = torch, dist
+        self.world = int(os.environ.get("WORLD_SIZE", "1"))
+        self.rank = int(os.environ.get("RANK", "0"))
+        self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+        self.device = device
+        if self.world > 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29511")
+            kw = {"device_id": device} if (backend == "nccl" and device is not None) else {}
+            dist.init_process_group(backend, rank=self.rank, world_size=self.world, **kw)
+
+    def barrier(self):
+        if self.world > 1:
+            self.dist.barrier()
+        if self.device is not None:
+            self.torch.cuda.synchronize(self.device)
+
+    def _reduce(self, x: float, op) -> float:
+        if self.world == 1:
+            return float(x)
+        t = self.torch.tensor([x], dtype=self.torch.float64,
+                              device=self.device if self.device is not None else "cpu")
+        self.dist.all_reduce(t, op=op)
+        return float(t.item())
+
+    def max(self, x: float) -> float:
+        return self._reduce(x, self.dist.ReduceOp.MAX)
+
+    def sum(self, x: float) -> float:
+        return self._reduce(x, self.dist.ReduceOp.SUM)
+
+    def close(self):
+        if self.world > 1:
+            self.dist.destroy_process_group()
+
+
+def rank_seed(workload, rank: int) -> int:
+    """Every rank works on its own seeded batch (weak scaling over independent batches)."""
+    return workload.seed(100 * rank)
+
+
+# ---------------------------------------------------------------------------
 # workload
 # ---------------------------------------------------------------------------
 def build_workload(args, device, rank):
@@ -164,7 +218,7 @@ def build_workload(args, device, rank):
     def cache(num_pages, data):
         return gk.Cache(data, num_pages, 2 * num_pages * slab, num_pages * slab, slab)
 
-    seed0 = w.seed(100 * rank)
+    seed0 = rank_seed(w, rank)
     rng = np.random.default_rng(seed0)
     pool = [torch.empty(blob_bytes, dtype=torch.uint8, device=device) for _ in range(pool_blocks)]
     sums = [torch.zeros(P, dtype=torch.int64, device=device) for _ in range(pool_blocks)]
@@ -263,7 +317,7 @@ def run_reference(args):
             blob, sums, _, _ = oracle.pack(og, src, spt, n_tok)
             oracle.restore(og, dst, [oracle.Job(blob, sums, dpt, n_tok)])
             per_page = (time.perf_counter() - t0) / N
-            pages = int(min(1024, max(8, 100.0 / (per_page * n_iter))))
+            pages = int(min(1024, max(8, args.reference_seconds / (per_page * n_iter))))
     times = []
     blob_bytes = oracle.blob_size(og, n_tok)[0]
     for it in range(args.warmup + args.steps):
@@ -294,30 +348,15 @@ def run_reference(args):
 # ---------------------------------------------------------------------------
 def run_ours(args):
     import torch
-    import torch.distributed as dist
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device: libgk has no CPU fallback")
     device = torch.device("cuda", local_rank)
     torch.cuda.set_device(device)
-    if world > 1:
-        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
-        dist.init_process_group("nccl", device_id=device)
-
-    def barrier():
-        if world > 1:
-            dist.barrier()
-        torch.cuda.synchronize(device)
-
-    def max_over_ranks(x: float) -> float:
-        if world == 1:
-            return x
-        t = torch.tensor([x], dtype=torch.float64, device=device)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+    comm = RankComm("nccl", device)
+    world, rank = comm.world, comm.rank
+    barrier, max_over_ranks = comm.barrier, comm.max
 
     wl = build_workload(args, device, rank)
     gk, ctx = wl["gk"], wl["ctx"]
@@ -471,8 +510,7 @@ def run_ours(args):
             "gpu_launches": launches, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
-    if world > 1:
-        dist.destroy_process_group()
+    comm.close()
 
 
 def synth_requests(n_blocks):

@@ -1,0 +1,50 @@
+"""The N > 1 launch path on CPU: world_size-2 gloo ranks.  The data path has no
+exchange step, so what is covered is what bench.py does across ranks: rendezvous
+on 127.0.0.1, barrier, max / sum of per-rank timings, distinct per-rank seeds,
+and that the reference arm runs on rank 0 only and prints exactly one line."""
+import json
+import os
+import subprocess
+import sys
+
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _worker(rank, world, port, out_dir):
+    os.environ.update({"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(world),
+                       "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
+    sys.path.insert(0, ROOT)
+    import bench
+    import synth
+    comm = bench.RankComm("gloo")
+    comm.barrier()
+    got = {"max": comm.max(10.0 + rank), "sum": comm.sum(1.0 + rank), "world": comm.world,
+           "seed": bench.rank_seed(synth.GQA7B, rank)}
+    comm.barrier()
+    comm.close()
+    with open(os.path.join(out_dir, f"rank{rank}.json"), "w") as f:
+        json.dump(got, f)
+
+
+def test_rank_comm_over_gloo(tmp_path):
+    world, port = 2, 29533
+    mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
+    res = [json.load(open(tmp_path / f"rank{r}.json")) for r in range(world)]
+    for r in res:
+        assert r["world"] == 2 and r["max"] == 11.0 and r["sum"] == 3.0
+    assert res[0]["seed"] != res[1]["seed"]
+
+
+def test_reference_arm_under_torchrun_prints_one_line_on_rank0():
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
+           "--master-addr", "127.0.0.1", "--master-port", "29534", os.path.join(ROOT, "bench.py"),
+           "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0", "--reference-seconds", "1"]
+    out = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["impl"] == "reference" and d["n_gpus"] == 2 and d["value"] > 0
+    assert d["cpu_baseline"]["kind"] == "oracle" and d["e2e"]["h2d_bytes_per_step"] == 0
