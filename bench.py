@@ -433,44 +433,63 @@ def run_ours(args):
                 "algorithmic_bytes_per_launch": 3 * batch_bytes, "ms_per_launch": dom["ms_per_launch"],
                 "achieved_useful_2x": 2 * batch_bytes / (dom["ms_per_launch"] * 1e-3) / 1e9}
 
-    # ---- end to end: blobs in pinned host memory, through gk_restore_host ----
+    # ---- end to end: the same step with HOST buffers -- gk_pack_host saves the batch into pinned
+    # host memory (D2H inside), gk_restore_host restores it from there (H2D inside), and the
+    # result masks are read back ----
     e2e = None
     if not args.no_e2e:
-        host_jobs, keep = [], []
-        for jb in wl["restore_jobs"]:
+        host_pack, host_restore, keep = [], [], []
+        for pj, rj in zip(wl["pack_jobs"], wl["restore_jobs"]):
             hb = torch.empty(blob_bytes, dtype=torch.uint8, pin_memory=True)
-            hb.copy_(jb.blob)
             hs = torch.empty(wl["P"], dtype=torch.int64, pin_memory=True)
-            hs.copy_(jb.checksums)
             keep.append((hb, hs))
-            host_jobs.append(gk.Job(hb, hs, jb.page_table, n_tok, jb.request_id))
+            host_pack.append(gk.Job(hb, hs, pj.page_table, n_tok, pj.request_id))
+            host_restore.append(gk.Job(hb, hs, rj.page_table, n_tok, rj.request_id))
         mask_h = torch.empty(n_blocks, dtype=torch.uint8, pin_memory=True)
         fb_h = torch.empty(n_blocks, dtype=torch.int32, pin_memory=True)
+        status_h = torch.empty(n_blocks, dtype=torch.uint8, pin_memory=True)
         torch.cuda.synchronize(device)
+        e2e_events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.e2e_steps)]
 
-        def e2e_step():
-            ctx.gk_restore_host(host_jobs, wl["dst"], mask, first_bad)
+        def e2e_step(ev=None):
+            if ev:
+                ev[0].record(stream)
+            ctx.gk_pack_host(wl["src"], host_pack, status)
+            status_h.copy_(status, non_blocking=True)
+            if ev:
+                ev[1].record(stream)
+            ctx.gk_restore_host(host_restore, wl["dst"], mask, first_bad)
             mask_h.copy_(mask, non_blocking=True)
             fb_h.copy_(first_bad, non_blocking=True)
+            if ev:
+                ev[2].record(stream)
 
         e2e_step()
         torch.cuda.synchronize(device)
+        for i in range(min(4, n_blocks)):      # what went over the link is what the device pool holds
+            assert torch.equal(keep[i][1], wl["pack_jobs"][i].checksums.cpu())
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         barrier()
         e0.record(stream)
-        for _ in range(args.e2e_steps):
-            e2e_step()
+        for k in range(args.e2e_steps):
+            e2e_step(e2e_events[k])
         e1.record(stream)
         barrier()
         e2e_ms = max_over_ranks(e0.elapsed_time(e1) / max(args.e2e_steps, 1))
-        assert int(mask_h.sum().item()) == 0
-        h2d = batch_bytes + n_blocks * wl["P"] * 8 + n_blocks * 40
-        e2e = {"value": world * 2 * batch_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": n_blocks * 5, "ms_per_step": e2e_ms,
-               "steps": args.e2e_steps, "tokens_per_s": world * n_blocks * n_tok / (e2e_ms * 1e-3),
-               "host_link_gbs": world * h2d / (e2e_ms * 1e-3) / 1e9,
-               "what": "gk_restore_host of the batch from pinned host blobs + D2H read of mask and first_bad_page"}
-        del keep, host_jobs
+        assert int(mask_h.sum().item()) == 0 and int(status_h.sum().item()) == 0
+        save_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in e2e_events]))
+        load_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in e2e_events]))
+        link = batch_bytes + n_blocks * wl["P"] * 8
+        e2e = {"value": world * 4 * batch_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": link + 2 * n_blocks * 40, "d2h_bytes_per_step": link + n_blocks * 6,
+               "ms_per_step": e2e_ms, "steps": args.e2e_steps,
+               "tokens_per_s": world * n_blocks * n_tok / (e2e_ms * 1e-3),
+               "save": {"ms": save_ms, "host_link_gbs": link / (save_ms * 1e-3) / 1e9},
+               "restore": {"ms": load_ms, "host_link_gbs": link / (load_ms * 1e-3) / 1e9,
+                           "tokens_per_s": n_blocks * n_tok / (load_ms * 1e-3)},
+               "what": "gk_pack_host (save to pinned host) + gk_restore_host (restore from pinned host) + D2H read "
+                       "of status, mask and first_bad_page; value counts 2 x blob bytes for each"}
+        del keep, host_pack, host_restore
 
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:

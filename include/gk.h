@@ -149,6 +149,18 @@ int gk_pack_batch(gk_ctx *ctx, const gk_cache *src, const gk_job *jobs, uint32_t
 int gk_pack(gk_ctx *ctx, const gk_cache *src, const int32_t *page_table_dev, uint32_t n_tokens,
             void *blob_dev, uint64_t *checksums_dev, uint8_t *status_dev, void *stream);
 
+/* Save to the host tier (Section 2.2: stored state goes to storage; Section 4.3,
+ * footprint and long-window paragraphs: the store is bounded by storage, not by
+ * GPU memory).  As gk_pack_batch, but each job's blob and checksums are outputs
+ * in PINNED host memory.  Batches of blocks are packed into the internal device
+ * staging ring on `stream` while the previous batch is copied to the host on an
+ * internal copy stream.  The call returns after enqueuing; `stream` is made to
+ * wait for the last copy, so the host buffers are valid once `stream` has been
+ * synchronised.  For a job with status GK_JOB_PAGE_TABLE the host blob and
+ * checksums are unspecified and must not be used. */
+int gk_pack_host(gk_ctx *ctx, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,
+                 uint8_t *status_dev, void *stream);
+
 /* Page checksums of an existing device blob (the check-on-load of Section 2.2
  * rests on them): checksums_dev[p] = CRC-64/XZ of record p. */
 int gk_page_checksums(gk_ctx *ctx, const void *blob_dev, uint32_t n_tokens,

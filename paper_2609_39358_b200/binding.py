@@ -25,7 +25,7 @@ JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
 
 EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",
            "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times",
-           "gk_page_checksums_noalloc"]
+           "gk_page_checksums_noalloc", "gk_pack_host"]
 
 
 class GkError(RuntimeError):
@@ -82,6 +82,8 @@ def load_library() -> ctypes.CDLL:
     L.gk_last_error.argtypes = [vp]
     L.gk_pack_batch.restype = ctypes.c_int
     L.gk_pack_batch.argtypes = [vp, ctypes.POINTER(CCache), ctypes.POINTER(CJob), u32, vp, vp]
+    L.gk_pack_host.restype = ctypes.c_int
+    L.gk_pack_host.argtypes = [vp, ctypes.POINTER(CCache), ctypes.POINTER(CJob), u32, vp, vp]
     L.gk_pack.restype = ctypes.c_int
     L.gk_pack.argtypes = [vp, ctypes.POINTER(CCache), vp, u32, vp, vp, vp, vp]
     L.gk_page_checksums.restype = ctypes.c_int
@@ -225,6 +227,11 @@ class Context:
         cc = src.c()
         self._check(self._lib.gk_pack_batch(self._h, ctypes.byref(cc), self._jobs(jobs), len(jobs), _ptr(status),
                                             _stream_handle(stream)), "gk_pack_batch")
+
+    def gk_pack_host(self, src: Cache, jobs: Sequence[Job], status: Optional[torch.Tensor] = None, stream=None):
+        cc = src.c()
+        self._check(self._lib.gk_pack_host(self._h, ctypes.byref(cc), self._jobs(jobs), len(jobs), _ptr(status),
+                                           _stream_handle(stream)), "gk_pack_host")
 
     def gk_pack(self, src: Cache, page_table: torch.Tensor, n_tokens: int, blob: torch.Tensor,
                 checksums: torch.Tensor, status: Optional[torch.Tensor] = None, stream=None):

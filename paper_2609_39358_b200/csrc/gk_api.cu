@@ -444,6 +444,89 @@ int launch_finalize(gk_ctx *c, const WorkDev &w, const Tiling &tl, int write_mod
     return GK_OK;
 }
 
+// Host tier (both directions): sizes of every job, the pinned-memory check, the
+// two device staging slots, the place of every job in a slot and the batches.
+struct HostPlan {
+    struct Plan { uint64_t blob_bytes, sums_bytes, need; uint32_t pages; };
+    std::vector<Plan> plan;
+    std::vector<uint8_t *> blob_dev;
+    std::vector<uint64_t *> sums_dev;
+    std::vector<uint32_t> batch_end;  // exclusive job index per batch
+    uint64_t pages = 0;
+};
+
+int make_host_plan(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, bool allow_missing, HostPlan &hp)
+{
+    std::vector<HostPlan::Plan> &plan = hp.plan;
+    plan.resize(n_jobs);
+    uint64_t max_need = 0, total_need = 0, pages = 0;
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
+        const uint32_t np = (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+        plan[j].pages = np;
+        plan[j].blob_bytes = (uint64_t)np * c->gd.S + (uint64_t)jobs[j].n_tokens * c->gd.tokB;
+        plan[j].sums_bytes = (uint64_t)np * 8;
+        plan[j].need = 0;
+        pages += np;
+        if (jobs[j].blob && jobs[j].checksums) {
+            cudaPointerAttributes a{};
+            for (const void *ptr : {(const void *)jobs[j].blob, (const void *)jobs[j].checksums}) {
+                if (cudaPointerGetAttributes(&a, ptr) != cudaSuccess || a.type != cudaMemoryTypeHost) {
+                    cudaGetLastError();
+                    return fail(c, GK_ERR_NOT_PINNED, "job %u: blob and checksums must be pinned host memory", j);
+                }
+            }
+            plan[j].need = align_up(plan[j].blob_bytes, 256) + align_up(plan[j].sums_bytes, 256);
+        } else if (!allow_missing) {
+            return fail(c, GK_ERR_ARG, "job %u: null blob or checksums", j);
+        }
+        if (plan[j].need > max_need) max_need = plan[j].need;
+        total_need += plan[j].need;
+    }
+    hp.pages = pages;
+    // staging slots: room for the largest job, and for batches of small jobs up to 256 MiB
+    uint64_t want = max_need;
+    const uint64_t batch_target = 256ull << 20;
+    if (want < batch_target) want = total_need < batch_target ? total_need : batch_target;
+    if (want < 256) want = 256;
+    if (want > c->slot_cap) {
+        GK_CUDA(c, cudaDeviceSynchronize());
+        for (int i = 0; i < kSlots; ++i) {
+            if (c->d_slot[i]) cudaFree(c->d_slot[i]);
+            c->d_slot[i] = nullptr;
+            c->slot_used[i] = false;
+        }
+        c->slot_cap = 0;
+        for (int i = 0; i < kSlots; ++i) {
+            if (cudaMalloc(&c->d_slot[i], want) != cudaSuccess) {
+                cudaGetLastError();
+                return fail(c, GK_ERR_NOMEM, "host-tier staging slot of %llu bytes", (unsigned long long)want);
+            }
+        }
+        c->slot_cap = want;
+    }
+    // assign every job a place in a slot
+    hp.blob_dev.assign(n_jobs, nullptr);
+    hp.sums_dev.assign(n_jobs, nullptr);
+    uint64_t used = 0;
+    uint32_t b = 0;
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        if (used + plan[j].need > c->slot_cap && used > 0) {
+            hp.batch_end.push_back(j);
+            ++b;
+            used = 0;
+        }
+        if (plan[j].need) {
+            uint8_t *base = c->d_slot[b % kSlots] + used;
+            hp.blob_dev[j] = base;
+            hp.sums_dev[j] = (uint64_t *)(base + align_up(plan[j].blob_bytes, 256));
+            used += plan[j].need;
+        }
+    }
+    hp.batch_end.push_back(n_jobs);
+    return GK_OK;
+}
+
 struct DeviceGuard {
     int prev = -1;
     explicit DeviceGuard(int dev)
@@ -735,74 +818,13 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
     int rc = check_cache(c, dst, &cd);
     if (rc != GK_OK) return rc;
 
-    // sizes, pinned check, batch plan
-    struct Plan { uint64_t blob_bytes, sums_bytes, need; uint32_t pages; };
-    std::vector<Plan> plan(n_jobs);
-    uint64_t max_need = 0, total_need = 0, pages = 0;
-    for (uint32_t j = 0; j < n_jobs; ++j) {
-        if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
-        const uint32_t np = (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
-        plan[j].pages = np;
-        plan[j].blob_bytes = (uint64_t)np * c->gd.S + (uint64_t)jobs[j].n_tokens * c->gd.tokB;
-        plan[j].sums_bytes = (uint64_t)np * 8;
-        plan[j].need = 0;
-        pages += np;
-        if (jobs[j].blob && jobs[j].checksums) {
-            cudaPointerAttributes a{};
-            for (const void *ptr : {(const void *)jobs[j].blob, (const void *)jobs[j].checksums}) {
-                if (cudaPointerGetAttributes(&a, ptr) != cudaSuccess || a.type != cudaMemoryTypeHost) {
-                    cudaGetLastError();
-                    return fail(c, GK_ERR_NOT_PINNED, "job %u: blob and checksums must be pinned host memory", j);
-                }
-            }
-            plan[j].need = align_up(plan[j].blob_bytes, 256) + align_up(plan[j].sums_bytes, 256);
-        }
-        if (plan[j].need > max_need) max_need = plan[j].need;
-        total_need += plan[j].need;
-    }
-    // staging slots: room for the largest job, and for batches of small jobs up to 256 MiB
-    uint64_t want = max_need;
-    const uint64_t batch_target = 256ull << 20;
-    if (want < batch_target) want = total_need < batch_target ? total_need : batch_target;
-    if (want < 256) want = 256;
-    if (want > c->slot_cap) {
-        GK_CUDA(c, cudaDeviceSynchronize());
-        for (int i = 0; i < kSlots; ++i) {
-            if (c->d_slot[i]) cudaFree(c->d_slot[i]);
-            c->d_slot[i] = nullptr;
-            c->slot_used[i] = false;
-        }
-        c->slot_cap = 0;
-        for (int i = 0; i < kSlots; ++i) {
-            if (cudaMalloc(&c->d_slot[i], want) != cudaSuccess) {
-                cudaGetLastError();
-                return fail(c, GK_ERR_NOMEM, "host-tier staging slot of %llu bytes", (unsigned long long)want);
-            }
-        }
-        c->slot_cap = want;
-    }
-    // assign every job a place in a slot
-    std::vector<uint8_t *> blob_dev(n_jobs, nullptr);
-    std::vector<uint64_t *> sums_dev(n_jobs, nullptr);
-    std::vector<uint32_t> batch_end;  // exclusive job index per batch
-    {
-        uint64_t used = 0;
-        uint32_t b = 0;
-        for (uint32_t j = 0; j < n_jobs; ++j) {
-            if (used + plan[j].need > c->slot_cap && used > 0) {
-                batch_end.push_back(j);
-                ++b;
-                used = 0;
-            }
-            if (plan[j].need) {
-                uint8_t *base = c->d_slot[b % kSlots] + used;
-                blob_dev[j] = base;
-                sums_dev[j] = (uint64_t *)(base + align_up(plan[j].blob_bytes, 256));
-                used += plan[j].need;
-            }
-        }
-        batch_end.push_back(n_jobs);
-    }
+    HostPlan hp;
+    if ((rc = make_host_plan(c, jobs, n_jobs, true, hp)) != GK_OK) return rc;
+    std::vector<HostPlan::Plan> &plan = hp.plan;
+    std::vector<uint8_t *> &blob_dev = hp.blob_dev;
+    std::vector<uint64_t *> &sums_dev = hp.sums_dev;
+    std::vector<uint32_t> &batch_end = hp.batch_end;
+    uint64_t pages = hp.pages;
 
     const Tiling tlv = crc_tiling(c), tlc = commit_tiling(c);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
@@ -838,6 +860,73 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
         page0 += npages;
     }
     c->stats.calls_restore_host++;
+    c->stats.jobs += n_jobs;
+    c->stats.pages += pages;
+    c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs, uint8_t *status_dev,
+                 void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0) return GK_OK;
+    if (!jobs) return fail(c, GK_ERR_ARG, "null job array");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    CacheDev cd;
+    int rc = check_cache(c, src, &cd);
+    if (rc != GK_OK) return rc;
+    HostPlan hp;
+    if ((rc = make_host_plan(c, jobs, n_jobs, false, hp)) != GK_OK) return rc;
+
+    const Tiling tl = crc_tiling(c, GK_PACK_STAGE);
+    uint64_t pages = hp.pages, bytes = 0;
+    const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
+    if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
+    if ((rc = upload_jobs(c, jobs, n_jobs, l, hp.blob_dev.data(), hp.sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
+        return rc;
+    WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tl);
+    if ((rc = launch_validate(c, w, cd.num_pages, 0, st)) != GK_OK) return rc;
+
+    uint32_t j0 = 0, page0 = 0;
+    int last_slot[kSlots] = {0, 0};
+    for (size_t b = 0; b < hp.batch_end.size(); ++b) {
+        const int slot = (int)(b % kSlots);
+        const uint32_t j1 = hp.batch_end[b];
+        // the slot's previous contents must have left (earlier D2H, or an earlier restore reading it)
+        if (c->slot_used[slot]) GK_CUDA(c, cudaStreamWaitEvent(st, c->ev_slot_free[slot], 0));
+        uint32_t npages = 0;
+        for (uint32_t j = j0; j < j1; ++j) npages += hp.plan[j].pages;
+        WorkDev wb = w;
+        wb.page_begin = page0;
+        wb.total_pages = npages;
+        StreamParams P{};
+        P.g = c->gd;
+        P.cache = cd;
+        P.w = wb;
+        P.tl = tl;
+        P.n_items = npages * tl.nseg_max;
+        if ((rc = launch_pack(c, P, st)) != GK_OK) return rc;
+        if ((rc = launch_finalize(c, wb, tl, 1, status_dev, st)) != GK_OK) return rc;
+        GK_CUDA(c, cudaEventRecord(c->ev_copied[slot], st));
+        GK_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_copied[slot], 0));
+        for (uint32_t j = j0; j < j1; ++j) {
+            GK_CUDA(c, cudaMemcpyAsync(jobs[j].blob, hp.blob_dev[j], hp.plan[j].blob_bytes, cudaMemcpyDeviceToHost,
+                                       c->copy_stream));
+            GK_CUDA(c, cudaMemcpyAsync(jobs[j].checksums, hp.sums_dev[j], hp.plan[j].sums_bytes,
+                                       cudaMemcpyDeviceToHost, c->copy_stream));
+        }
+        GK_CUDA(c, cudaEventRecord(c->ev_slot_free[slot], c->copy_stream));
+        c->slot_used[slot] = true;
+        last_slot[slot] = 1;
+        j0 = j1;
+        page0 += npages;
+    }
+    // the caller's stream is complete only when the last copies have landed
+    for (int i = 0; i < kSlots; ++i)
+        if (last_slot[i]) GK_CUDA(c, cudaStreamWaitEvent(st, c->ev_slot_free[i], 0));
+    c->stats.calls_pack++;
     c->stats.jobs += n_jobs;
     c->stats.pages += pages;
     c->stats.bytes_blob += bytes;

@@ -198,16 +198,21 @@ def test_corpus_full_device_and_host_tier(gk):
     torch.cuda.synchronize()
     assert mask.cpu().tolist() == [0] * NB
     _check_destination(w, src, dst, sentinel, jobs_meta, [0] * NB)
-    # run B: the same blobs from pinned host memory, one of them damaged on the host
+    # run B: save the corpus to pinned host memory with gk_pack_host (many staging batches),
+    # check it is byte-identical to the device-packed blobs, damage one blob on the host,
+    # restore from the host tier
     dst.data.copy_(sentinel)
     host = []
     for i in range(NB):
         hb = torch.empty(blobs[i].numel(), dtype=torch.uint8, pin_memory=True)
-        hb.copy_(blobs[i])
         hs = torch.empty(pages[i], dtype=torch.int64, pin_memory=True)
-        hs.copy_(sums[i])
         host.append((hb, hs))
+    status.fill_(255)
+    ctx.gk_pack_host(src, [gk.Job(host[i][0], host[i][1], d_spts[i], lens[i]) for i in range(NB)], status)
     torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * NB
+    for i in range(NB):
+        assert torch.equal(host[i][0], blobs[i].cpu()) and torch.equal(host[i][1], sums[i].cpu())
     del blobs
     victim = 37
     host[victim][0][123_456_789] ^= 0x04

@@ -139,6 +139,45 @@ def test_pack_single_entry_point_and_bad_table(gk):
     ctx.close()
 
 
+@pytest.mark.parametrize("og", [G_MID, G_FP8_M])
+def test_pack_host_parity(gk, og):
+    """Save to pinned host memory: same bytes and checksums as the oracle."""
+    from gpu_harness import dev_cache, dev_i32
+    N = 19
+    src = random_cache(og, N, seed=220)
+    dsrc = dev_cache(src)
+    rng = np.random.default_rng(221)
+    T = og.page_tokens
+    lens = [3 * T + 2, 1, 5 * T, T]
+    tables = [rng.integers(0, N, size=n_pages(og, n)).astype(np.int32) for n in lens]
+    tables[2][1] = N + 5                                   # job 2: an id outside the cache
+    ctx = _ctx(gk, og)
+    jobs, keep = [], []
+    for pt, n in zip(tables, lens):
+        nbytes, P = oracle.blob_size(og, n)
+        hb = torch.zeros(nbytes, dtype=torch.uint8).pin_memory()
+        hs = torch.zeros(P, dtype=torch.int64).pin_memory()
+        keep.append((hb, hs))
+        jobs.append(gk.Job(hb, hs, dev_i32(pt), n))
+    status = torch.full((len(jobs),), 255, dtype=torch.uint8, device="cuda")
+    ctx.gk_pack_host(dsrc, jobs, status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, 0, 2, 0]
+    for i, (pt, n) in enumerate(zip(tables, lens)):
+        if i == 2:
+            continue
+        wb, ws, code, _ = oracle.pack(og, src, pt, n)
+        assert code == 0
+        assert np.array_equal(keep[i][0].numpy(), wb)
+        assert np.array_equal(keep[i][1].numpy().view(np.uint64), ws)
+    # pageable outputs are refused
+    with pytest.raises(gk.GkError) as e:
+        ctx.gk_pack_host(dsrc, [gk.Job(torch.zeros(oracle.blob_size(og, 1)[0], dtype=torch.uint8),
+                                       torch.zeros(1, dtype=torch.int64), dev_i32(np.zeros(1)), 1)], None)
+    assert e.value.code == -3
+    ctx.close()
+
+
 # ---------------------------------------------------------------------------
 # restore
 # ---------------------------------------------------------------------------
