@@ -198,7 +198,11 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * item in 16 KiB tiles), "grid_cap" (upper bound on CTAs per kernel; 0 = fill
  * the GPU), "profile" (1 = time every streaming kernel, see gk_get_kernel_times),
  * "fused" (1, the default: gk_restore verifies and commits in one launch; 0: a
- * verify launch, a checksum-compare launch and a commit launch). */
+ * verify launch, a checksum-compare launch and a commit launch), "wait_limit_ms"
+ * (time limit of every wait inside a kernel, default 2000), "test_drop_verify"
+ * (tests only: the fused restore kernel verifies nothing, so that every commit
+ * wait runs into its limit and the time-out handling can be checked without
+ * hanging or faulting the GPU). */
 int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
 
 /* Page checksums of a device blob for callers that must not allocate.  (The

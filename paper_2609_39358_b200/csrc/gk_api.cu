@@ -89,6 +89,8 @@ struct gk_ctx {
     int sm_count = 0;
     int occ_verify = 0, occ_pack = 0, occ_commit = 0, occ_fused = 0;
     bool fused = true;           // restore runs verify and commit in one launch
+    unsigned long long wait_limit_ns = kWaitLimitNs;
+    bool test_drop_verify = false;  // test hook: see gk_ctx_set_tuning
     uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
     uint32_t commit_seg_tiles = 0;
     uint32_t grid_cap = 0;       // 0: SMs * occupancy
@@ -301,6 +303,7 @@ WorkDev make_work(const gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t 
     w.init_term = c->d_init_term;
     w.thread_const = c->d_thread_const;
     w.x_seg = gf_xpow(8ull * crc.seg_tiles * crc.stage_bytes);
+    w.wait_limit_ns = c->wait_limit_ns;
     return w;
 }
 
@@ -663,6 +666,8 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     else if (!strcmp(key, "grid_cap")) c->grid_cap = value;
     else if (!strcmp(key, "profile")) c->profile = value != 0;
     else if (!strcmp(key, "fused")) c->fused = value != 0;
+    else if (!strcmp(key, "wait_limit_ms")) c->wait_limit_ns = (unsigned long long)(value ? value : 1u) * 1000000ull;
+    else if (!strcmp(key, "test_drop_verify")) c->test_drop_verify = value != 0;
     else return fail(c, GK_ERR_ARG, "unknown tuning key %s", key);
     return GK_OK;
 }
@@ -768,6 +773,7 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
     if (c->gd.flags & GK_FLAG_SKIP_VERIFY) return launch_commit(c, P, st);
     if (c->fused) {
         P.fused = 1u;
+        if (c->test_drop_verify) P.n_items = 0;  // nothing gets verified: every commit wait must run out
         return launch_fused(c, P, st);
     }
     if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
@@ -1139,6 +1145,7 @@ int gk_page_checksums_noalloc(const gk_geom *geom, const void *blob_dev, uint32_
     w.init_term = reinterpret_cast<const uint64_t *>(sc + NoallocLayout::init_term);
     w.thread_const = reinterpret_cast<const uint64_t *>(sc + NoallocLayout::thread_const);
     w.x_seg = gf_xpow(8ull * tl.seg_tiles * tl.stage_bytes);
+    w.wait_limit_ns = kWaitLimitNs;
 
     noalloc_setup_kernel<<<1, 256, 0, st>>>(sc, job, gd);
     if (cudaGetLastError() != cudaSuccess) return GK_ERR_CUDA;

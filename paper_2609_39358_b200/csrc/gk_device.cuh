@@ -11,7 +11,7 @@ namespace gk {
 constexpr uint64_t kPoly = 0x42F0E1EBA9EA3693ull;
 constexpr int32_t kNoPage = 0x7fffffff;
 
-// bounded device waits: give up after this many nanoseconds of %globaltimer
+// bounded device waits: by default give up after this many nanoseconds of %globaltimer
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 enum Mode : int { kVerify = 0, kPack = 1, kCommit = 2 };
@@ -61,6 +61,7 @@ struct WorkDev {
     const uint64_t *init_term;    // [page_tokens+1] ones * x^(8*len(t)) mod P
     const uint64_t *thread_const; // [NT] x^(32*(NT-1-t)+64) mod P
     uint64_t x_seg;               // x^(8*segment bytes) mod P
+    unsigned long long wait_limit_ns;  // time limit of every device-side wait
 };
 
 // How a page record is cut into tiles and segments.  A record of `len` bytes is
@@ -155,13 +156,13 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     return t;
 }
 
-// Waits for a barrier phase, but never for ever: after kWaitLimitNs (or at once,
+// Waits for a barrier phase, but never for ever: after limit_ns (or at once,
 // when another thread of the CTA has already given up) it records the failure in
 // *abort_flag (shared) and *error (global) and returns false.  Callers carry on
 // without blocking and without issuing further async copies; the host and the
 // commit kernel treat a set error word as "commit nothing".
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          uint32_t *error, uint32_t where)
+                                          uint32_t *error, uint32_t where, unsigned long long limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
@@ -169,7 +170,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3ffu) == 0u) {
-            if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) {
+            if (*abort_flag || global_timer_ns() - t0 > limit_ns) {
                 *abort_flag = 1u;
                 atomicCAS(error, 0u, where);
                 return false;
@@ -181,13 +182,13 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 
 // Last wait of a loader before its CTA exits: lets copies that are still in
 // flight land, for a bounded time, whether or not the CTA has given up.
-__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity)
+__device__ __forceinline__ void mbar_drain(uint32_t bar, uint32_t parity, unsigned long long limit_ns)
 {
     if (mbar_try_wait(bar, parity)) return;
     const unsigned long long t0 = global_timer_ns();
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
-        if ((++spins & 0x3ffu) == 0u && global_timer_ns() - t0 > kWaitLimitNs / 4) return;
+        if ((++spins & 0x3ffu) == 0u && global_timer_ns() - t0 > limit_ns / 4) return;
     }
 }
 

@@ -207,7 +207,7 @@ __device__ __forceinline__ bool wait_job_verified(const StreamParams &P, uint32_
     while (ld_acquire_u32(cnt) < n_pages) {
         __nanosleep(200);
         if ((++spins & 0x3fu) == 0u) {
-            if (*abort_flag || global_timer_ns() - t0 > kWaitLimitNs) {
+            if (*abort_flag || global_timer_ns() - t0 > P.w.wait_limit_ns) {
                 *abort_flag = 1u;
                 atomicCAS(P.w.error, 0u, 0x500u);
                 return false;
@@ -416,10 +416,10 @@ template <int U, int MODE, int NT, int STAGE_BYTES, int STAGES>
 struct GranuleSteps {
     static constexpr int kSps = STAGE_BYTES / (NT * 32);  // 8-word steps per stage
     static __device__ __forceinline__ void run(uint32_t (&R)[64], const uint8_t *smem, uint32_t full0, uint32_t empty0,
-                                               RingPos &pos, volatile uint32_t *abort_flag, uint32_t *error, int tid,
-                                               int lane)
+                                               RingPos &pos, volatile uint32_t *abort_flag, uint32_t *error,
+                                               unsigned long long limit_ns, int tid, int lane)
     {
-        if (U % kSps == 0) mbar_wait(full0 + 8u * pos.stage, pos.phase, abort_flag, error, 0x400u | MODE);
+        if (U % kSps == 0) mbar_wait(full0 + 8u * pos.stage, pos.phase, abort_flag, error, 0x400u | MODE, limit_ns);
         const uint32_t *sw = reinterpret_cast<const uint32_t *>(smem + (size_t)pos.stage * STAGE_BYTES) + tid;
         uint32_t w[8];
 #pragma unroll
@@ -430,14 +430,14 @@ struct GranuleSteps {
             if (lane == 0) mbar_arrive(empty0 + 8u * pos.stage);
             pos.template advance<STAGES>();
         }
-        GranuleSteps<U + 1, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, pos, abort_flag, error, tid,
-                                                                lane);
+        GranuleSteps<U + 1, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, pos, abort_flag, error, limit_ns,
+                                                                tid, lane);
     }
 };
 template <int MODE, int NT, int STAGE_BYTES, int STAGES>
 struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES> {
     static __device__ __forceinline__ void run(uint32_t (&)[64], const uint8_t *, uint32_t, uint32_t, RingPos &,
-                                               volatile uint32_t *, uint32_t *, int, int)
+                                               volatile uint32_t *, uint32_t *, unsigned long long, int, int)
     {
     }
 };
@@ -460,7 +460,7 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
         for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
             const uint32_t s = n % STAGES;
             const uint32_t use = n / STAGES;
-            if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE);
+            if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE, P.w.wait_limit_ns);
             uint32_t lead, nreal;
             uint64_t r0;
             tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
@@ -521,7 +521,7 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
     if (lane == 0) {
         for (uint32_t back = 0; back < (uint32_t)STAGES && back < n; ++back) {
             const uint32_t m = n - 1u - back;
-            mbar_drain(ring.full0 + 8u * (m % STAGES), (m / STAGES) & 1u);
+            mbar_drain(ring.full0 + 8u * (m % STAGES), (m / STAGES) & 1u, P.w.wait_limit_ns);
         }
     }
 }
@@ -544,7 +544,7 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling 
         const uint32_t slab_len = it.t * P.g.row;
         for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
             const uint32_t s = n % STAGES;
-            const bool ok = mbar_wait(ring.full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE);
+            const bool ok = mbar_wait(ring.full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE, P.w.wait_limit_ns);
             uint32_t lead, nreal;
             uint64_t r0;
             tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
@@ -621,7 +621,7 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
         const uint32_t ngran = it.tile_count / kTilesPerGran;
         for (uint32_t gi = 0; gi < ngran; ++gi)
             GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, ring.base, ring.full0, ring.empty0, pos, abort_flag,
-                                                                P.w.error, tid, lane);
+                                                                P.w.error, P.w.wait_limit_ns, tid, lane);
         // merge streams -> thread -> warp -> CTA
         uint64_t v = thread_remainder<NT>(R, kt);
 #pragma unroll

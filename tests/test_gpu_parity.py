@@ -399,6 +399,81 @@ def test_round_trip_on_gpu_only_path(gk):
     ctx.close()
 
 
+def test_device_wait_time_out_is_fail_closed(gk):
+    """Failure detection without a GPU fault: the commit side's bounded wait for
+    "all pages of the job verified" is made to run out (test hook: nothing gets
+    verified, limit 50 ms).  The kernel must return by itself, report code 4 for
+    every job, write nothing, and leave the context refusing to commit."""
+    from gpu_harness import assert_cache_equal, dev_cache, dev_i32, sums_to_dev
+    og = G_MID
+    src = random_cache(og, 8, seed=360)
+    jobs = _oracle_jobs(og, src, [3 * og.page_tokens, og.page_tokens + 1], 361, 12)
+    clean = random_cache(og, 12, seed=362)
+    ctx = _ctx(gk, og, wait_limit_ms=50, test_drop_verify=1)
+    d = dev_cache(clean)
+    keep = [(torch.from_numpy(j.blob).cuda(), sums_to_dev(j.checksums), dev_i32(j.page_table)) for j in jobs]
+    gjobs = [gk.Job(b, s, t, j.n_tokens) for (b, s, t), j in zip(keep, jobs)]
+    mask = torch.full((2,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.zeros(2, dtype=torch.int32, device="cuda")
+    ctx.gk_restore(gjobs, d, mask, fb)
+    torch.cuda.synchronize()                       # returns: the wait was bounded
+    assert mask.cpu().tolist() == [4, 4] and fb.cpu().tolist() == [-1, -1]
+    assert_cache_equal(d, clean)
+    assert ctx.gk_get_stats()["device_wait_expired"] != 0
+    # the error is sticky: with the hook off the same context still commits nothing
+    ctx.set_tuning("test_drop_verify", 0)
+    mask.fill_(255)
+    ctx.gk_restore(gjobs, d, mask, fb)
+    torch.cuda.synchronize()
+    assert mask.cpu().tolist() == [4, 4]
+    assert_cache_equal(d, clean)
+    ctx.close()
+    # a fresh context on the same device works: nothing was left broken
+    ctx = _ctx(gk, og)
+    want = clone_cache(clean)
+    wmask, _ = oracle.restore(og, want, jobs)
+    mask.fill_(255)
+    ctx.gk_restore(gjobs, d, mask, fb)
+    torch.cuda.synchronize()
+    assert mask.cpu().tolist() == wmask.tolist() == [0, 0]
+    assert_cache_equal(d, want)
+    ctx.close()
+
+
+def test_padded_strides_leave_the_padding_alone(gk):
+    """Caches whose pages, K/V planes and layers are separated by padding: pack reads
+    only slab bytes, restore writes only slab bytes."""
+    from gpu_harness import gpu_pack, gpu_restore
+    import paper_2609_39358_b200 as m
+    og = G_MID
+    T, N = og.page_tokens, 9
+    slab = T * og.kv_heads * og.head_dim * og.elem_bytes
+    ps, ks, ls = slab + 256, N * (slab + 256) + 512, 2 * (N * (slab + 256) + 512) + 1024
+    total = og.layers * ls
+    rng = np.random.default_rng(370)
+    src = oracle.Cache(rng.integers(0, 256, size=total, dtype=np.uint8), N, ls, ks, ps)
+    clean = oracle.Cache(rng.integers(0, 256, size=total, dtype=np.uint8), N, ls, ks, ps)
+    lens = [2 * T + 3, T]
+    tables = [np.array([7, 2, 5], dtype=np.int32), np.array([0], dtype=np.int32)]
+    ctx = _ctx(gk, og)
+    dsrc = m.Cache(torch.from_numpy(src.data).cuda(), N, ls, ks, ps)
+    got, status = gpu_pack(ctx, og, dsrc, tables, lens)
+    assert status.tolist() == [0, 0]
+    jobs = []
+    for (blob, sums), pt, n, dpt in zip(got, tables, lens, [np.array([1, 8, 3], dtype=np.int32),
+                                                              np.array([6], dtype=np.int32)]):
+        wb, ws, _, _ = oracle.pack(og, src, pt, n)
+        assert np.array_equal(blob, wb) and np.array_equal(sums, ws)
+        jobs.append(oracle.Job(blob, sums, dpt, n))
+    want = clone_cache(clean)
+    wmask, _ = oracle.restore(og, want, jobs)
+    d = m.Cache(torch.from_numpy(clean.data).cuda(), N, ls, ks, ps)
+    mask, _ = gpu_restore(ctx, d, jobs)
+    assert mask.tolist() == wmask.tolist() == [0, 0]
+    assert np.array_equal(d.data.cpu().numpy(), want.data)
+    ctx.close()
+
+
 def test_argument_errors(gk):
     from gpu_harness import dev_cache
     og = G_MID
