@@ -464,6 +464,20 @@ def run_ours(args):
             if ev:
                 ev[2].record(stream)
 
+        # the link's own rate on this machine: plain pinned copies of one blob each way, for the host-tier roofline
+        tmp = torch.empty(blob_bytes, dtype=torch.uint8, device=device)
+        link_rate = {}
+        for name, (d, s_) in {"h2d": (tmp, keep[0][0]), "d2h": (keep[0][0], tmp)}.items():
+            d.copy_(s_, non_blocking=True)
+            torch.cuda.synchronize(device)
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            c0.record(stream)
+            for _ in range(3):
+                d.copy_(s_, non_blocking=True)
+            c1.record(stream)
+            torch.cuda.synchronize(device)
+            link_rate[name] = 3 * blob_bytes / (c0.elapsed_time(c1) * 1e-3) / 1e9
+        del tmp
         e2e_step()
         torch.cuda.synchronize(device)
         for i in range(min(4, n_blocks)):      # what went over the link is what the device pool holds
@@ -484,9 +498,12 @@ def run_ours(args):
                "h2d_bytes_per_step": link + 2 * n_blocks * 40, "d2h_bytes_per_step": link + n_blocks * 6,
                "ms_per_step": e2e_ms, "steps": args.e2e_steps,
                "tokens_per_s": world * n_blocks * n_tok / (e2e_ms * 1e-3),
-               "save": {"ms": save_ms, "host_link_gbs": link / (save_ms * 1e-3) / 1e9},
+               "save": {"ms": save_ms, "host_link_gbs": link / (save_ms * 1e-3) / 1e9,
+                        "frac_of_plain_d2h_copy": link / (save_ms * 1e-3) / 1e9 / link_rate["d2h"]},
                "restore": {"ms": load_ms, "host_link_gbs": link / (load_ms * 1e-3) / 1e9,
+                           "frac_of_plain_h2d_copy": link / (load_ms * 1e-3) / 1e9 / link_rate["h2d"],
                            "tokens_per_s": n_blocks * n_tok / (load_ms * 1e-3)},
+               "plain_pinned_copy_gbs": link_rate,
                "what": "gk_pack_host (save to pinned host) + gk_restore_host (restore from pinned host) + D2H read "
                        "of status, mask and first_bad_page; value counts 2 x blob bytes for each"}
         del keep, host_pack, host_restore
