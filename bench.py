@@ -156,20 +156,22 @@ class RankComm:
         self.rank = int(os.environ.get("RANK", "0"))
         self.local_rank = int(os.environ.get("LOCAL_RANK", "0"))
         self.device = device
-        if self.world > 1:
+        # GK_FORCE_DIST=1 brings the process group up even for one rank (to try the NCCL path on one GPU)
+        self.active = self.world > 1 or os.environ.get("GK_FORCE_DIST") == "1"
+        if self.active:
             os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
             os.environ.setdefault("MASTER_PORT", "29511")
             kw = {"device_id": device} if (backend == "nccl" and device is not None) else {}
             dist.init_process_group(backend, rank=self.rank, world_size=self.world, **kw)
 
     def barrier(self):
-        if self.world > 1:
+        if self.active:
             self.dist.barrier()
         if self.device is not None:
             self.torch.cuda.synchronize(self.device)
 
     def _reduce(self, x: float, op) -> float:
-        if self.world == 1:
+        if not self.active:
             return float(x)
         t = self.torch.tensor([x], dtype=self.torch.float64,
                               device=self.device if self.device is not None else "cpu")
@@ -183,7 +185,7 @@ class RankComm:
         return self._reduce(x, self.dist.ReduceOp.SUM)
 
     def close(self):
-        if self.world > 1:
+        if self.active:
             self.dist.destroy_process_group()
 
 
