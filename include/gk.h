@@ -178,6 +178,24 @@ int gk_page_checksums(gk_ctx *ctx, const void *blob_dev, uint32_t n_tokens,
 int gk_restore(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
                uint8_t *mask_dev, int32_t *first_bad_page_dev, void *stream);
 
+/* The two halves of gk_restore as separate calls, for callers that must put a
+ * step of their own between "checked" and "written" -- above all tensor-parallel
+ * serving (Section 3 and Section 4.4 report tensor-parallel runs), where every
+ * rank holds its own shard of a block and a block may be committed only if it
+ * verified on ALL ranks: gk_verify on each rank, a max-reduction of the masks
+ * across ranks, gk_commit with the reduced mask.
+ *
+ * gk_verify validates the page tables against dst (which it does not write) and
+ * verifies every page record; mask_dev / first_bad_page_dev receive what gk_restore
+ * would report, and nothing is committed.  gk_commit validates the tables again
+ * and scatters exactly the jobs whose entry in mask_dev (device, n_jobs bytes,
+ * input) is GK_JOB_OK and whose own table check passes; it verifies no checksum,
+ * so the mask must come from a gk_verify of the same jobs. */
+int gk_verify(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, uint8_t *mask_dev,
+              int32_t *first_bad_page_dev, void *stream);
+int gk_commit(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
+              const uint8_t *mask_dev, void *stream);
+
 /* Load from the host tier (Section 4.3, long-window paragraph: saved blocks are
  * streamed in from storage and dropped after use).  As gk_restore, but each job's blob and checksums lie
  * in PINNED host memory.  Blobs are copied in batches into an internal device

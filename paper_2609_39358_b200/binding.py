@@ -25,7 +25,7 @@ JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
 
 EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",
            "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times",
-           "gk_page_checksums_noalloc", "gk_pack_host"]
+           "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit"]
 
 
 class GkError(RuntimeError):
@@ -90,6 +90,10 @@ def load_library() -> ctypes.CDLL:
     L.gk_page_checksums.argtypes = [vp, vp, u32, vp, vp]
     L.gk_restore.restype = ctypes.c_int
     L.gk_restore.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
+    L.gk_verify.restype = ctypes.c_int
+    L.gk_verify.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
+    L.gk_commit.restype = ctypes.c_int
+    L.gk_commit.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp]
     L.gk_restore_host.restype = ctypes.c_int
     L.gk_restore_host.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
     L.gk_get_stats.restype = ctypes.c_int
@@ -248,6 +252,17 @@ class Context:
         cc = dst.c()
         self._check(self._lib.gk_restore(self._h, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask),
                                          _ptr(first_bad_page), _stream_handle(stream)), "gk_restore")
+
+    def gk_verify(self, jobs: Sequence[Job], dst: Cache, mask: torch.Tensor, first_bad_page: torch.Tensor,
+                  stream=None):
+        cc = dst.c()
+        self._check(self._lib.gk_verify(self._h, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask),
+                                        _ptr(first_bad_page), _stream_handle(stream)), "gk_verify")
+
+    def gk_commit(self, jobs: Sequence[Job], dst: Cache, mask: torch.Tensor, stream=None):
+        cc = dst.c()
+        self._check(self._lib.gk_commit(self._h, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask),
+                                        _stream_handle(stream)), "gk_commit")
 
     def gk_restore_host(self, jobs: Sequence[Job], dst: Cache, mask: torch.Tensor, first_bad_page: torch.Tensor,
                         stream=None):

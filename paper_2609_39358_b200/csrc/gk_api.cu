@@ -812,6 +812,86 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
     return GK_OK;
 }
 
+// shared front part of gk_verify / gk_commit: job table, page tables, claims
+static int prepare_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, cudaStream_t st,
+                           CacheDev *cd, Tiling *tlv, Tiling *tlc, WorkDev *w, uint64_t *pages_out, uint64_t *bytes_out)
+{
+    int rc = check_cache(c, dst, cd);
+    if (rc != GK_OK) return rc;
+    *tlv = crc_tiling(c);
+    *tlc = commit_tiling(c);
+    uint64_t pages = 0, bytes = 0;
+    for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    const WsLayout l = ws_layout(n_jobs, pages, tlv->nseg_max, cd->num_pages);
+    if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
+    if ((rc = upload_jobs(c, jobs, n_jobs, l, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
+    *w = make_work(c, l, n_jobs, (uint32_t)pages, *tlv);
+    if ((rc = launch_validate(c, *w, cd->num_pages, 1, st)) != GK_OK) return rc;
+    if ((rc = launch_claim(c, *w, st)) != GK_OK) return rc;
+    *pages_out = pages;
+    *bytes_out = bytes;
+    return GK_OK;
+}
+
+int gk_verify(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, uint8_t *mask_dev,
+              int32_t *first_bad_page_dev, void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0) return GK_OK;
+    if (!jobs || !mask_dev || !first_bad_page_dev) return fail(c, GK_ERR_ARG, "null jobs, mask or first_bad_page");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    CacheDev cd;
+    Tiling tlv, tlc;
+    WorkDev w;
+    uint64_t pages, bytes;
+    int rc = prepare_restore(c, jobs, n_jobs, dst, st, &cd, &tlv, &tlc, &w, &pages, &bytes);
+    if (rc != GK_OK) return rc;
+    if (!(c->gd.flags & GK_FLAG_SKIP_VERIFY)) {
+        StreamParams P{};
+        P.g = c->gd;
+        P.w = w;
+        P.tl = tlv;
+        P.n_items = (uint32_t)pages * tlv.nseg_max;
+        if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
+        if ((rc = launch_finalize(c, w, tlv, 0, nullptr, st)) != GK_OK) return rc;
+    }
+    report_kernel<<<(n_jobs + 127) / 128, 128, 0, st>>>(w, mask_dev, first_bad_page_dev);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched++;
+    c->stats.jobs += n_jobs;
+    c->stats.pages += pages;
+    c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+int gk_commit(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, const uint8_t *mask_dev,
+              void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0) return GK_OK;
+    if (!jobs || !mask_dev) return fail(c, GK_ERR_ARG, "null jobs or mask");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    CacheDev cd;
+    Tiling tlv, tlc;
+    WorkDev w;
+    uint64_t pages, bytes;
+    int rc = prepare_restore(c, jobs, n_jobs, dst, st, &cd, &tlv, &tlc, &w, &pages, &bytes);
+    if (rc != GK_OK) return rc;
+    w.ext_mask = mask_dev;
+    StreamParams P{};
+    P.g = c->gd;
+    P.cache = cd;
+    P.w = w;
+    P.tl = tlv;
+    P.tlc = tlc;
+    P.n_items_c = (uint32_t)pages * tlc.nseg_max;
+    if ((rc = launch_commit(c, P, st)) != GK_OK) return rc;
+    c->stats.calls_restore++;
+    return GK_OK;
+}
+
 int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, uint8_t *mask_dev,
                     int32_t *first_bad_page_dev, void *stream)
 {

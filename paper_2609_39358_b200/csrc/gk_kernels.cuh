@@ -102,7 +102,19 @@ __device__ __forceinline__ uint32_t job_code(const WorkDev &w, uint32_t j, int32
         return 1u;
     }
     if (__ldcg(w.error) != 0u) return 4u;
+    if (w.ext_mask) return (uint32_t)w.ext_mask[j];  // verified elsewhere (another call, another rank)
     return 0u;
+}
+
+// One thread per job: result code and first failing page (gk_verify, which commits nothing).
+__global__ void report_kernel(WorkDev w, uint8_t *mask_out, int32_t *first_bad_out)
+{
+    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= w.n_jobs) return;
+    int32_t fb;
+    const uint32_t code = job_code(w, j, &fb);
+    mask_out[j] = (uint8_t)code;
+    first_bad_out[j] = fb;
 }
 
 // One thread per page.  Merges the page's segment remainders (Horner with
@@ -234,7 +246,7 @@ __device__ __forceinline__ bool get_item(const StreamParams &P, const Tiling &tl
             wait_job_verified(P, it.j, jb.n_pages, abort_flag);
         int32_t fb;
         const uint32_t code = job_code(P.w, it.j, &fb);
-        if (report && it.p == 0u && it.q == 0u) {
+        if (report && it.p == 0u && it.q == 0u && P.mask_out) {
             P.mask_out[it.j] = (uint8_t)code;
             P.first_bad_out[it.j] = fb;
         }

@@ -399,6 +399,63 @@ def test_round_trip_on_gpu_only_path(gk):
     ctx.close()
 
 
+def test_verify_then_commit_matches_restore(gk):
+    """gk_verify writes nothing and reports what gk_restore would; gk_commit with that
+    mask produces gk_restore's destination; a job failed from outside (another rank's
+    verdict) is not committed."""
+    from gpu_harness import assert_cache_equal, dev_cache, dev_i32, sums_to_dev
+    from paper_2609_39358_b200 import tp
+    og = G_FP8_M
+    T = og.page_tokens
+    src = random_cache(og, 9, seed=380)
+    jobs = _oracle_jobs(og, src, [2 * T, T + 3, 3 * T, 1], 381, 20)
+    jobs[1].blob[77] ^= 0x02
+    used = set(int(x) for j in jobs for x in j.page_table)
+    free_page = next(g for g in range(20) if g not in used)
+    jobs.append(oracle.Job(jobs[0].blob, jobs[0].checksums, np.array([free_page, 25], dtype=np.int32), 2 * T))  # id 25 out of range
+    clean = random_cache(og, 20, seed=382)
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs)
+    assert wmask.tolist() == [0, 1, 0, 0, 2]
+    ctx = _ctx(gk, og)
+    keep = [(torch.from_numpy(j.blob).cuda(), sums_to_dev(j.checksums), dev_i32(j.page_table)) for j in jobs]
+    gjobs = [gk.Job(b, s, t, j.n_tokens) for (b, s, t), j in zip(keep, jobs)]
+    d = dev_cache(clean)
+    mask = torch.full((5,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.zeros(5, dtype=torch.int32, device="cuda")
+    ctx.gk_verify(gjobs, d, mask, fb)
+    torch.cuda.synchronize()
+    assert mask.cpu().tolist() == wmask.tolist() and fb.cpu().tolist() == wfb.tolist()
+    assert_cache_equal(d, clean)                               # verify commits nothing
+    ctx.gk_commit(gjobs, d, mask)
+    torch.cuda.synchronize()
+    assert_cache_equal(d, want)
+    # another rank rejected job 2: with the merged mask it must stay out
+    d = dev_cache(clean)
+    merged = mask.clone()
+    merged[2] = 1
+    ctx.gk_commit(gjobs, d, merged)
+    torch.cuda.synchronize()
+    want2 = clone_cache(clean)
+    oracle.restore(og, want2, [jobs[0], jobs[3]])
+    assert_cache_equal(d, want2)
+    # a mask that claims "ok" for the job with the bad table does not get it written
+    d = dev_cache(clean)
+    ctx.gk_commit(gjobs, d, torch.zeros(5, dtype=torch.uint8, device="cuda"))
+    torch.cuda.synchronize()
+    got = d.data.cpu().numpy().reshape(og.layers, 2, 20, T, -1)
+    c = clean.data.reshape(og.layers, 2, 20, T, -1)
+    assert np.array_equal(got[:, :, free_page], c[:, :, free_page])
+    # single-rank tp_restore is verify + commit
+    d = dev_cache(clean)
+    mask.fill_(255)
+    tp.tp_restore(ctx, gjobs, d, mask, fb)
+    torch.cuda.synchronize()
+    assert mask.cpu().tolist() == wmask.tolist()
+    assert_cache_equal(d, want)
+    ctx.close()
+
+
 def test_device_wait_time_out_is_fail_closed(gk):
     """Failure detection without a GPU fault: the commit side's bounded wait for
     "all pages of the job verified" is made to run out (test hook: nothing gets

@@ -7,6 +7,7 @@ import os
 import subprocess
 import sys
 
+import torch
 import torch.multiprocessing as mp
 
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
@@ -35,6 +36,42 @@ def test_rank_comm_over_gloo(tmp_path):
     for r in res:
         assert r["world"] == 2 and r["max"] == 11.0 and r["sum"] == 3.0
     assert res[0]["seed"] != res[1]["seed"]
+
+
+class _FakeCtx:
+    """Stands in for a gk context on CPU: verify reports this rank's verdicts,
+    commit records which jobs it was allowed to write."""
+
+    def __init__(self, verdicts):
+        self.verdicts, self.committed = verdicts, None
+
+    def gk_verify(self, jobs, dst, mask, first_bad_page, stream=None):
+        mask.copy_(torch.tensor(self.verdicts, dtype=torch.uint8))
+
+    def gk_commit(self, jobs, dst, mask, stream=None):
+        self.committed = [i for i, c in enumerate(mask.tolist()) if c == 0]
+
+
+def _tp_worker(rank, world, port, out_dir):
+    os.environ.update({"RANK": str(rank), "WORLD_SIZE": str(world), "MASTER_ADDR": "127.0.0.1",
+                       "MASTER_PORT": str(port)})
+    sys.path.insert(0, ROOT)
+    import torch.distributed as dist
+    from paper_2609_39358_b200 import tp
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    verdicts = [[0, 1, 0, 0, 3], [0, 0, 0, 2, 0]][rank]     # each rank sees different failures
+    ctx = _FakeCtx(verdicts)
+    mask = torch.zeros(5, dtype=torch.uint8)
+    tp.tp_restore(ctx, [None] * 5, None, mask, torch.zeros(5, dtype=torch.int32))
+    dist.destroy_process_group()
+    with open(os.path.join(out_dir, f"tp{rank}.json"), "w") as f:
+        json.dump({"mask": mask.tolist(), "committed": ctx.committed}, f)
+
+
+def test_tp_restore_commits_a_block_on_all_ranks_or_none(tmp_path):
+    mp.spawn(_tp_worker, args=(2, 29535, str(tmp_path)), nprocs=2, join=True)
+    res = [json.load(open(tmp_path / f"tp{r}.json")) for r in range(2)]
+    assert res[0] == res[1] == {"mask": [0, 1, 0, 2, 3], "committed": [0, 2]}
 
 
 def test_reference_arm_under_torchrun_prints_one_line_on_rank0():
