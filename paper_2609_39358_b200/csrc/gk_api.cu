@@ -5,6 +5,7 @@
 // runs in the kernels of gk_kernels.cuh; there is no CPU fallback.
 #include "../../include/gk.h"
 
+#include <cmath>
 #include <cstdarg>
 #include <cstdio>
 #include <cstdlib>
@@ -204,27 +205,77 @@ int check_cache(gk_ctx *c, const gk_cache *k, CacheDev *out)
     return GK_OK;
 }
 
-Tiling crc_tiling(const gk_ctx *c, uint32_t stage_bytes = GK_CRC_STAGE)
+// Work items wanted per launch: two per resident CTA, so that small calls still fill the GPU
+// (measured: verify of 64 and of 325 GQA pages is fastest with 1-2 and 2-4 items per CTA).
+uint64_t items_wanted(const gk_ctx *c, int occ) { return 2ull * (uint64_t)c->sm_count * (uint64_t)occ; }
+
+// Tiling of the CRC modes for a call of total_pages pages.  Large calls use one
+// segment per page (the per-thread epilogue is paid once per page); small calls
+// cut pages into segments of at least two granules so that every SM gets work.
+Tiling crc_tiling(const gk_ctx *c, uint32_t stage_bytes, uint64_t total_pages, int occ, bool overlap_jobs = false)
 {
     Tiling t;
     t.stage_bytes = stage_bytes;
     t.gran_bytes = VerifyCfg::kGran;
     const uint32_t gran_full = (uint32_t)((c->gd.R + t.gran_bytes - 1) / t.gran_bytes);
-    uint32_t sg = c->seg_granules ? c->seg_granules : gran_full;
+    uint32_t sg = gran_full;
+    if (c->seg_granules) {
+        sg = c->seg_granules;
+    } else if (total_pages > 0 && total_pages < items_wanted(c, occ)) {
+        // Small call: cut pages into k segments each.  Estimated time = rounds * (segment time +
+        // per-item overhead), rounds = ceil(items / resident CTAs); constants fitted to measurements
+        // on B200 (a CTA sharing its SM streams about 15 GB/s through the CRC; ring refill, item
+        // look-up and the per-segment epilogue cost about 20 us per item).
+        const double grid = (double)c->sm_count * occ;
+        const double page_us = (double)c->gd.R / 15e3;
+        const double item_us = 20.0;
+        double best = 1e30;
+        uint32_t best_k = 1;
+        const uint32_t kmax = gran_full > 1 ? gran_full / 2 : 1;  // at least two granules per segment
+        for (uint32_t k = 1; k <= kmax; ++k) {
+            const uint32_t g = (gran_full + k - 1) / k;            // granules per segment
+            const uint32_t nseg = (gran_full + g - 1) / g;
+            const double rounds = std::ceil((double)total_pages * nseg / grid);
+            const double cost = rounds * (page_us / nseg + item_us);
+            if (cost < best * 0.999) {
+                best = cost;
+                best_k = k;
+            }
+        }
+        if (overlap_jobs) {
+            // fused restore of several jobs: finer items let the first jobs finish verifying early,
+            // so that their commit overlaps the verification of the rest (8 jobs x 512 tokens:
+            // 310 us with whole pages, 273 us with three segments per page)
+            const uint64_t per_page = (items_wanted(c, occ) + total_pages - 1) / total_pages;
+            if (per_page > best_k) best_k = (uint32_t)(per_page < kmax ? per_page : kmax);
+        }
+        sg = (gran_full + best_k - 1) / best_k;
+    }
     if (sg > gran_full) sg = gran_full;
+    if (sg < 1) sg = 1;
     t.seg_tiles = sg * (t.gran_bytes / stage_bytes);
     t.nseg_max = (gran_full + sg - 1) / sg;
     return t;
 }
 
-Tiling commit_tiling(const gk_ctx *c)
+Tiling commit_tiling(const gk_ctx *c, uint64_t total_pages, int occ)
 {
     Tiling t;
     t.stage_bytes = GK_COPY_STAGE;
     t.gran_bytes = GK_COPY_STAGE;
     const uint32_t tiles_full = (uint32_t)((c->gd.R + t.stage_bytes - 1) / t.stage_bytes);
-    uint32_t st = c->commit_seg_tiles ? c->commit_seg_tiles : 16u;
+    uint32_t st = 16u;
+    if (c->commit_seg_tiles) {
+        st = c->commit_seg_tiles;
+    } else if (total_pages > 0) {
+        const uint64_t items = total_pages * ((tiles_full + st - 1) / st);
+        if (items < items_wanted(c, occ)) {
+            const uint64_t per_page = (items_wanted(c, occ) + total_pages - 1) / total_pages;
+            st = (uint32_t)((tiles_full + per_page - 1) / per_page);
+        }
+    }
     if (st > tiles_full) st = tiles_full;
+    if (st < 1) st = 1;
     t.seg_tiles = st;
     t.nseg_max = (tiles_full + st - 1) / st;
     return t;
@@ -239,7 +290,7 @@ WsLayout ws_layout(uint32_t n_jobs, uint64_t total_pages, uint32_t nseg_max, uin
 {
     WsLayout l;
     size_t o = 0;
-    l.jobs = o;      o = align_up(o + (size_t)n_jobs * sizeof(JobDev), 256);
+    l.jobs = o;      o = align_up(o + (size_t)n_jobs * sizeof(JobDev) + (size_t)nseg_max * 8, 256);  // + seg_pow
     l.page_job = o;  o = align_up(o + (size_t)total_pages * 4, 256);
     l.seg_res = o;   o = align_up(o + (size_t)total_pages * nseg_max * 8, 256);
     l.bad_range = o; o = align_up(o + (size_t)n_jobs * 4, 256);
@@ -303,20 +354,17 @@ WorkDev make_work(const gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t 
     w.init_term = c->d_init_term;
     w.thread_const = c->d_thread_const;
     w.x_seg = gf_xpow(8ull * crc.seg_tiles * crc.stage_bytes);
+    w.seg_pow = (const uint64_t *)(c->d_ws + l.jobs + (size_t)n_jobs * sizeof(JobDev));
     w.wait_limit_ns = c->wait_limit_ns;
     return w;
 }
 
-// Fills the pinned job table and enqueues its upload.  blob_override /
+// Job records of a call from the caller's gk_job array.  blob_override /
 // sums_override (may be null) replace the callers' pointers, for the host tier.
-int upload_jobs(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const WsLayout &l, uint8_t *const *blob_override,
-                uint64_t *const *sums_override, bool need_tables, cudaStream_t st, uint64_t *total_pages_out,
-                uint64_t *total_bytes_out)
+int fill_job_table(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, JobDev *h, uint8_t *const *blob_override,
+                   uint64_t *const *sums_override, bool need_tables, uint64_t *total_pages_out,
+                   uint64_t *total_bytes_out)
 {
-    int rc = ensure_host_stage(c, (size_t)n_jobs * sizeof(JobDev));
-    if (rc != GK_OK) return rc;
-    GK_CUDA(c, cudaEventSynchronize(c->ev_stage));
-    JobDev *h = (JobDev *)c->h_stage;
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) {
         const gk_job &jb = jobs[j];
@@ -340,8 +388,56 @@ int upload_jobs(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const WsLayout &
     }
     *total_pages_out = pages;
     if (total_bytes_out) *total_bytes_out = bytes;
-    GK_CUDA(c, cudaMemcpyAsync(c->d_ws + l.jobs, h, (size_t)n_jobs * sizeof(JobDev), cudaMemcpyHostToDevice, st));
+    return GK_OK;
+}
+
+// powers of x^(8 * segment bytes), which place segment remainders inside their page
+void fill_seg_pow(const Tiling &crc, uint64_t *pw)
+{
+    const uint64_t xs = gf_xpow(8ull * crc.seg_tiles * crc.stage_bytes);
+    for (uint32_t k = 0; k < crc.nseg_max; ++k) pw[k] = k ? gf_mul(pw[k - 1], xs) : 1ull;
+}
+
+// Fills the pinned job table (and the segment powers behind it) and enqueues the upload.
+int upload_jobs(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const WsLayout &l, const Tiling &crc,
+                uint8_t *const *blob_override, uint64_t *const *sums_override, bool need_tables, cudaStream_t st,
+                uint64_t *total_pages_out, uint64_t *total_bytes_out)
+{
+    const size_t table_bytes = (size_t)n_jobs * sizeof(JobDev) + (size_t)crc.nseg_max * 8;
+    int rc = ensure_host_stage(c, table_bytes);
+    if (rc != GK_OK) return rc;
+    GK_CUDA(c, cudaEventSynchronize(c->ev_stage));
+    JobDev *h = (JobDev *)c->h_stage;
+    if ((rc = fill_job_table(c, jobs, n_jobs, h, blob_override, sums_override, need_tables, total_pages_out,
+                             total_bytes_out)) != GK_OK)
+        return rc;
+    fill_seg_pow(crc, reinterpret_cast<uint64_t *>(c->h_stage + (size_t)n_jobs * sizeof(JobDev)));
+    GK_CUDA(c, cudaMemcpyAsync(c->d_ws + l.jobs, h, table_bytes, cudaMemcpyHostToDevice, st));
     GK_CUDA(c, cudaEventRecord(c->ev_stage, st));
+    return GK_OK;
+}
+
+// Small calls: job table and segment powers travel as kernel arguments of the one
+// preparation launch (no staging copy, no separate validate / claim launches).
+bool is_small_call(uint32_t n_jobs, uint64_t pages, const Tiling &crc)
+{
+    return n_jobs <= kPrepMaxJobs && crc.nseg_max <= kPrepMaxSeg && pages <= 16384;
+}
+
+int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tiling &crc, const WorkDev &w,
+                      uint64_t num_pages, bool need_tables, bool do_claims, cudaStream_t st, uint64_t *pages_out,
+                      uint64_t *bytes_out)
+{
+    PrepSmallParams pp{};
+    int rc = fill_job_table(c, jobs, n_jobs, pp.jobs, nullptr, nullptr, need_tables, pages_out, bytes_out);
+    if (rc != GK_OK) return rc;
+    fill_seg_pow(crc, pp.seg_pow);
+    pp.n_seg_pow = crc.nseg_max;
+    pp.do_claims = do_claims ? 1u : 0u;
+    pp.num_pages = num_pages;
+    prep_small_kernel<<<1, 1024, 0, st>>>(pp, w);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched++;
     return GK_OK;
 }
 
@@ -686,15 +782,19 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
     for (uint32_t j = 0; j < n_jobs; ++j)
         if (!jobs[j].blob || !jobs[j].checksums) return fail(c, GK_ERR_ARG, "job %u: null output", j);
 
-    const Tiling tl = crc_tiling(c, GK_PACK_STAGE);
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    const Tiling tl = crc_tiling(c, GK_PACK_STAGE, pages, c->occ_pack);
     const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
-    if ((rc = upload_jobs(c, jobs, n_jobs, l, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tl);
-
-    if ((rc = launch_validate(c, w, cd.num_pages, 0, st)) != GK_OK) return rc;
+    if (is_small_call(n_jobs, pages, tl)) {
+        if ((rc = launch_prep_small(c, jobs, n_jobs, tl, w, cd.num_pages, true, false, st, &pages, &bytes)) != GK_OK)
+            return rc;
+    } else {
+        if ((rc = upload_jobs(c, jobs, n_jobs, l, tl, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
+        if ((rc = launch_validate(c, w, cd.num_pages, 0, st)) != GK_OK) return rc;
+    }
     StreamParams P{};
     P.g = c->gd;
     P.cache = cd;
@@ -732,12 +832,12 @@ int gk_page_checksums(gk_ctx *c, const void *blob_dev, uint32_t n_tokens, uint64
     jb.checksums = checksums_dev;
     jb.page_table = nullptr;
     jb.n_tokens = n_tokens;
-    const Tiling tl = crc_tiling(c);
     uint64_t pages = (n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens, bytes = 0;
+    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify);
     const WsLayout l = ws_layout(1, pages, tl.nseg_max, 0);
     int rc;
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
-    if ((rc = upload_jobs(c, &jb, 1, l, nullptr, nullptr, false, st, &pages, &bytes)) != GK_OK) return rc;
+    if ((rc = upload_jobs(c, &jb, 1, l, tl, nullptr, nullptr, false, st, &pages, &bytes)) != GK_OK) return rc;
     WorkDev w = make_work(c, l, 1, (uint32_t)pages, tl);
     if ((rc = launch_validate(c, w, 0, 0, st)) != GK_OK) return rc;
     StreamParams P{};
@@ -793,16 +893,22 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
     int rc = check_cache(c, dst, &cd);
     if (rc != GK_OK) return rc;
 
-    const Tiling tlv = crc_tiling(c), tlc = commit_tiling(c);
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    const int occ = c->fused ? c->occ_fused : c->occ_verify;
+    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages, occ, c->fused && n_jobs > 1);
+    const Tiling tlc = commit_tiling(c, pages, c->fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
-    if ((rc = upload_jobs(c, jobs, n_jobs, l, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tlv);
-
-    if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
-    if ((rc = launch_claim(c, w, st)) != GK_OK) return rc;
+    if (is_small_call(n_jobs, pages, tlv)) {
+        if ((rc = launch_prep_small(c, jobs, n_jobs, tlv, w, cd.num_pages, true, true, st, &pages, &bytes)) != GK_OK)
+            return rc;
+    } else {
+        if ((rc = upload_jobs(c, jobs, n_jobs, l, tlv, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
+        if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
+        if ((rc = launch_claim(c, w, st)) != GK_OK) return rc;
+    }
     if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, 0, (uint32_t)pages, mask_dev, first_bad_page_dev, st)) != GK_OK)
         return rc;
     c->stats.calls_restore++;
@@ -818,16 +924,21 @@ static int prepare_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const
 {
     int rc = check_cache(c, dst, cd);
     if (rc != GK_OK) return rc;
-    *tlv = crc_tiling(c);
-    *tlc = commit_tiling(c);
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    *tlv = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify);
+    *tlc = commit_tiling(c, pages, c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv->nseg_max, cd->num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
-    if ((rc = upload_jobs(c, jobs, n_jobs, l, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
     *w = make_work(c, l, n_jobs, (uint32_t)pages, *tlv);
-    if ((rc = launch_validate(c, *w, cd->num_pages, 1, st)) != GK_OK) return rc;
-    if ((rc = launch_claim(c, *w, st)) != GK_OK) return rc;
+    if (is_small_call(n_jobs, pages, *tlv)) {
+        if ((rc = launch_prep_small(c, jobs, n_jobs, *tlv, *w, cd->num_pages, true, true, st, &pages, &bytes)) != GK_OK)
+            return rc;
+    } else {
+        if ((rc = upload_jobs(c, jobs, n_jobs, l, *tlv, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
+        if ((rc = launch_validate(c, *w, cd->num_pages, 1, st)) != GK_OK) return rc;
+        if ((rc = launch_claim(c, *w, st)) != GK_OK) return rc;
+    }
     *pages_out = pages;
     *bytes_out = bytes;
     return GK_OK;
@@ -912,11 +1023,15 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
     std::vector<uint32_t> &batch_end = hp.batch_end;
     uint64_t pages = hp.pages;
 
-    const Tiling tlv = crc_tiling(c), tlc = commit_tiling(c);
+    // batches are what is launched, so size the work items for a batch, not for the call
+    const uint64_t pages_per_launch = (pages + batch_end.size() - 1) / batch_end.size();
+    const int occ = c->fused ? c->occ_fused : c->occ_verify;
+    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages_per_launch, occ, c->fused && n_jobs > batch_end.size());
+    const Tiling tlc = commit_tiling(c, pages_per_launch, c->fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     uint64_t bytes = 0;
-    if ((rc = upload_jobs(c, jobs, n_jobs, l, blob_dev.data(), sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
+    if ((rc = upload_jobs(c, jobs, n_jobs, l, tlv, blob_dev.data(), sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
         return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tlv);
     if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
@@ -966,11 +1081,11 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
     HostPlan hp;
     if ((rc = make_host_plan(c, jobs, n_jobs, false, hp)) != GK_OK) return rc;
 
-    const Tiling tl = crc_tiling(c, GK_PACK_STAGE);
     uint64_t pages = hp.pages, bytes = 0;
+    const Tiling tl = crc_tiling(c, GK_PACK_STAGE, (pages + hp.batch_end.size() - 1) / hp.batch_end.size(), c->occ_pack);
     const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
-    if ((rc = upload_jobs(c, jobs, n_jobs, l, hp.blob_dev.data(), hp.sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
+    if ((rc = upload_jobs(c, jobs, n_jobs, l, tl, hp.blob_dev.data(), hp.sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
         return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tl);
     if ((rc = launch_validate(c, w, cd.num_pages, 0, st)) != GK_OK) return rc;

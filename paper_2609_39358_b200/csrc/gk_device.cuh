@@ -61,6 +61,7 @@ struct WorkDev {
     uint32_t *error;              // sticky: non-zero once a bounded wait has run out
     const uint64_t *init_term;    // [page_tokens+1] ones * x^(8*len(t)) mod P
     const uint64_t *thread_const; // [NT] x^(32*(NT-1-t)+64) mod P
+    const uint64_t *seg_pow;      // [nseg_max] (x^(8*segment bytes))^k mod P: places segment remainders
     uint64_t x_seg;               // x^(8*segment bytes) mod P
     unsigned long long wait_limit_ns;  // time limit of every device-side wait
 };

@@ -84,6 +84,67 @@ __global__ void claim_kernel(WorkDev w)
     }
 }
 
+// Small calls: the whole preparation in ONE single-CTA launch, with the job table
+// and the segment powers passed as kernel arguments instead of a host-to-device
+// copy.  Writes the tables to the workspace, then does what validate_kernel and
+// claim_kernel do, separated by a CTA barrier.  Only the claim words that this
+// call can touch are cleared.
+constexpr uint32_t kPrepMaxJobs = 64;
+constexpr uint32_t kPrepMaxSeg = 96;
+struct PrepSmallParams {
+    JobDev jobs[kPrepMaxJobs];
+    uint64_t seg_pow[kPrepMaxSeg];
+    uint32_t n_seg_pow;
+    uint32_t do_claims;
+    uint64_t num_pages;
+};
+
+__global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant__ PrepSmallParams pp, WorkDev w)
+{
+    JobDev *jobs_out = const_cast<JobDev *>(w.jobs);
+    uint64_t *pow_out = const_cast<uint64_t *>(w.seg_pow);
+    for (uint32_t j = threadIdx.x; j < w.n_jobs; j += blockDim.x) {
+        jobs_out[j] = pp.jobs[j];
+        w.bad_range[j] = kNoPage;
+        w.bad_dup[j] = kNoPage;
+        w.bad_crc[j] = kNoPage;
+        w.job_done[j] = 0u;
+    }
+    for (uint32_t k = threadIdx.x; k < pp.n_seg_pow; k += blockDim.x) pow_out[k] = pp.seg_pow[k];
+    __syncthreads();
+    // pass 1: page -> job map, range check, clear the claim words that will be used
+    for (uint32_t j = 0; j < w.n_jobs; ++j) {
+        const JobDev &jb = pp.jobs[j];
+        for (uint32_t p = threadIdx.x; p < jb.n_pages; p += blockDim.x) {
+            w.page_job[jb.page_base + p] = (int32_t)j;
+            w.page_cnt[jb.page_base + p] = 0u;
+            if (jb.page_table) {
+                const int32_t id = jb.page_table[p];
+                if (id < 0 || (uint64_t)id >= pp.num_pages)
+                    atomicMin(&w.bad_range[j], (int32_t)p);
+                else if (pp.do_claims)
+                    w.claims[id] = 0ull;
+            }
+        }
+    }
+    if (!pp.do_claims) return;
+    __syncthreads();
+    // pass 2: claims, as in claim_kernel
+    for (uint32_t j = 0; j < w.n_jobs; ++j) {
+        const JobDev &jb = pp.jobs[j];
+        if (jb.missing || __ldcg(&w.bad_range[j]) != kNoPage) continue;
+        for (uint32_t p = threadIdx.x; p < jb.n_pages; p += blockDim.x) {
+            const int32_t id = jb.page_table[p];
+            const unsigned long long mine = ((unsigned long long)(j + 1u) << 32) | p;
+            const unsigned long long old = atomicCAS(&w.claims[id], 0ull, mine);
+            if (old != 0ull) {
+                atomicMin(&w.bad_dup[j], (int32_t)p);
+                atomicMin(&w.bad_dup[(uint32_t)(old >> 32) - 1u], (int32_t)(old & 0xffffffffull));
+            }
+        }
+    }
+}
+
 // Result code of a job from the words the earlier kernels left.
 __device__ __forceinline__ uint32_t job_code(const WorkDev &w, uint32_t j, int32_t *first_bad)
 {
@@ -117,9 +178,10 @@ __global__ void report_kernel(WorkDev w, uint8_t *mask_out, int32_t *first_bad_o
     first_bad_out[j] = fb;
 }
 
-// One thread per page.  Merges the page's segment remainders (Horner with
-// x^(8*segment bytes)), adds the term of the all-ones initial register and
-// the final xor, reflects, and either writes the checksum (write_mode) or
+// One thread per page.  Merges the page's segment remainders (each was already
+// multiplied by x^(8 * bytes that follow the segment) by the CTA that produced
+// it, so the merge is an XOR), adds the term of the all-ones initial register
+// and the final xor, reflects, and either writes the checksum (write_mode) or
 // compares it with the stored one.
 __global__ void finalize_kernel(GeomDev g, WorkDev w, Tiling tl, int write_mode, uint8_t *status_out)
 {
@@ -136,7 +198,7 @@ __global__ void finalize_kernel(GeomDev g, WorkDev w, Tiling tl, int write_mode,
     const PageShape sh = page_shape(g, jb, p, tl);
     const uint64_t *res = w.seg_res + (uint64_t)gp * tl.nseg_max;
     uint64_t r = res[0];
-    for (uint32_t q = 1; q < sh.nseg; ++q) r = gf_mul(r, w.x_seg) ^ res[q];
+    for (uint32_t q = 1; q < sh.nseg; ++q) r ^= res[q];  // already placed by their producers
     const uint64_t crc = __brevll(r ^ w.init_term[sh.t] ^ ~0ull);
     if (write_mode) {
         jb.checksums[p] = crc;
@@ -645,6 +707,9 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
             uint64_t tot = 0;
 #pragma unroll
             for (int i = 0; i < NT / 32; ++i) tot ^= slot[i];
+            // place the segment: the short segment comes first and all others are full, so
+            // (nseg - 1 - q) full segments follow this one
+            if (it.nseg > 1u) tot = gf_mul(tot, P.w.seg_pow[it.nseg - 1u - it.q]);
             uint64_t *res = P.w.seg_res + (uint64_t)it.gp * P.tl.nseg_max;
             if (!P.fused) {
                 res[it.q] = tot;
@@ -658,7 +723,7 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
                     if (last) {
                         __threadfence();
                         r = __ldcg(&res[0]);
-                        for (uint32_t q = 1; q < it.nseg; ++q) r = gf_mul(r, P.w.x_seg) ^ __ldcg(&res[q]);
+                        for (uint32_t q = 1; q < it.nseg; ++q) r ^= __ldcg(&res[q]);
                     }
                 }
                 if (last) {
