@@ -40,7 +40,7 @@ UNIT = "GB/s"
 # ncu capture summarised in profiles/restore_kernel_gqa7b_2blocks.md (dram read +
 # write of the launch divided by the blob bytes it restores).  Traffic grows in
 # proportion to the blob bytes, so a full launch is this ratio times its bytes.
-RESTORE_DRAM_BYTES_PER_BLOB_BYTE = 2.95
+RESTORE_DRAM_BYTES_PER_BLOB_BYTE = 2.96
 
 
 def parse_args():
