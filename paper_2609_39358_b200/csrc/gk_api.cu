@@ -93,6 +93,7 @@ struct gk_ctx {
     int occ_verify = 0, occ_pack = 0, occ_commit = 0, occ_fused = 0;
     bool fused = true;           // restore runs verify and commit in one launch
     unsigned long long wait_limit_ns = kWaitLimitNs;
+    uint32_t ctr_next[2] = {0, 0};  // what the device work counters will read when the next launch starts
     bool test_drop_verify = false;  // test hook: see gk_ctx_set_tuning
     uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
     uint32_t commit_seg_tiles = 0;
@@ -353,6 +354,7 @@ WorkDev make_work(const gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t 
     w.job_done = (uint32_t *)(c->d_ws + l.job_done);
     w.claims = (unsigned long long *)(c->d_ws + l.claims);
     w.error = c->d_error;
+    w.work_ctr = c->d_error + 16;
     w.init_term = c->d_init_term;
     w.thread_const = c->d_thread_const;
     w.x_seg = gf_xpow(8ull * crc.seg_tiles * crc.stage_bytes);
@@ -469,7 +471,13 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
         slot->cls = MODE;
         GK_CUDA(c, cudaEventRecord(slot->a, st));
     }
-    stream_kernel<MODE, NT, SB, ST, MINB><<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(P);
+    // every work item is drawn once, and every CTA draws once more to learn that none is left
+    StreamParams Q = P;
+    const int ci = MODE == kCommit ? 1 : 0;
+    if (ci) Q.ctr_base_c = c->ctr_next[1];
+    else Q.ctr_base_v = c->ctr_next[0];
+    c->ctr_next[ci] += items + grid;
+    stream_kernel<MODE, NT, SB, ST, MINB><<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(Q);
     GK_CUDA(c, cudaGetLastError());
     if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
@@ -507,8 +515,13 @@ int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
         slot->cls = 3;
         GK_CUDA(c, cudaEventRecord(slot->a, st));
     }
+    StreamParams Q = P;
+    Q.ctr_base_v = c->ctr_next[0];
+    Q.ctr_base_c = c->ctr_next[1];
+    c->ctr_next[0] += P.n_items + grid;
+    c->ctr_next[1] += P.n_items_c + grid;
     restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES, GK_FUSED_MINB>
-        <<<grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st>>>(P);
+        <<<grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st>>>(Q);
     GK_CUDA(c, cudaGetLastError());
     if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
@@ -1232,6 +1245,8 @@ __global__ void noalloc_setup_kernel(unsigned char *scratch, JobDev job, GeomDev
         words[2] = kNoPage;  // bad_crc
         words[3] = 0;        // job_done
         words[4] = 0;        // error word
+        words[5] = 0;        // work counters
+        words[6] = 0;
     }
     for (uint32_t t = threadIdx.x; t < (uint32_t)GK_CRC_NT; t += blockDim.x)
         tc[t] = dev_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);
@@ -1339,6 +1354,7 @@ int gk_page_checksums_noalloc(const gk_geom *geom, const void *blob_dev, uint32_
     w.job_done = reinterpret_cast<uint32_t *>(words + 3);
     w.claims = nullptr;
     w.error = reinterpret_cast<uint32_t *>(words + 4);
+    w.work_ctr = reinterpret_cast<uint32_t *>(words + 5);
     w.init_term = reinterpret_cast<const uint64_t *>(sc + NoallocLayout::init_term);
     w.thread_const = reinterpret_cast<const uint64_t *>(sc + NoallocLayout::thread_const);
     w.x_seg = gf_xpow(8ull * tl.seg_tiles * tl.stage_bytes);

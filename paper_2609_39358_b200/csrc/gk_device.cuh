@@ -58,6 +58,7 @@ struct WorkDev {
     uint32_t *job_done;           // [n_jobs] pages finalized per job (fused restore)
     unsigned long long *claims;   // [num_pages] first claimant of each destination page
     const uint8_t *ext_mask;      // [n_jobs] or null: codes decided outside this call (gk_commit)
+    uint32_t *work_ctr;           // [2] running work-item counters: CRC modes, commit mode
     uint32_t *error;              // sticky: non-zero once a bounded wait has run out
     const uint64_t *init_term;    // [page_tokens+1] ones * x^(8*len(t)) mod P
     const uint64_t *thread_const; // [NT] x^(32*(NT-1-t)+64) mod P

@@ -221,7 +221,7 @@ struct StreamCfg {
     static constexpr int kGran = kCrc ? NT * 256 : STAGE_BYTES;  // 8 shift-register steps of 8 words per thread
     static constexpr int kSps = kCrc ? STAGE_BYTES / (NT * 32) : 1;  // 8-word steps per stage
     static constexpr int kTilesPerGran = kGran / STAGE_BYTES;
-    static constexpr size_t kSmemBytes = (size_t)STAGES * STAGE_BYTES + 2 * STAGES * 8 + 2 * 8 * 8 + 16 + 128;
+    static constexpr size_t kSmemBytes = (size_t)STAGES * STAGE_BYTES + 3 * STAGES * 8 + 2 * 8 * 8 + 16 + 128;
     static_assert(!kCrc || (NT == 32 || NT == 64 || NT == 128 || NT == 256), "NT must be a power of two");
     static_assert(!kCrc || (STAGE_BYTES % (NT * 32) == 0 && (NT * 256) % STAGE_BYTES == 0), "stage/step mismatch");
     static_assert(STAGE_BYTES % 128 == 0, "stage alignment");
@@ -236,6 +236,7 @@ struct StreamParams {
     uint32_t n_items;    // CRC work items: pages of the launch * tl.nseg_max
     uint32_t n_items_c;  // commit work items: pages of the launch * tlc.nseg_max
     uint32_t fused;      // 1: verify and commit run in one launch; commit waits per job
+    uint32_t ctr_base_v, ctr_base_c;  // values of the work counters at the start of this launch
     uint8_t *mask_out;        // commit
     int32_t *first_bad_out;   // commit
 };
@@ -256,6 +257,7 @@ struct Ring {
     uint8_t *base;    // generic address of stage 0
     uint32_t stage0;  // shared-window address of stage 0
     uint32_t full0, empty0;
+    uint2 *tag;  // per stage: (work item, tile index within the item), or the end mark
 };
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
@@ -516,25 +518,44 @@ struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES> {
     }
 };
 
+// Work is handed out dynamically: the loader warp of a CTA draws item numbers
+// from a global counter (so the CTAs that are resident take all the work, in
+// order, whatever their number) and tags every stage it fills with the item and
+// the tile index; the other roles of the CTA follow the tags.  A stage tagged
+// kEndOfWork tells them to leave.
+constexpr uint32_t kEndOfWork = 0xffffffffu;
+
+__device__ __forceinline__ uint32_t next_item(uint32_t *ctr, uint32_t base, int lane)
+{
+    uint32_t v = 0;
+    if (lane == 0) v = atomicAdd(ctr, 1u) - base;
+    return __shfl_sync(0xffffffffu, v, 0);
+}
+
 // ------------------------------ loader role ------------------------------
-// One warp.  Walks this CTA's work items tile by tile, waits for a free stage,
+// One warp.  Draws work items, walks each tile by tile, waits for a free stage
 // and fills it: front padding zeroed by the lanes (CRC modes), scale values
 // gathered by the lanes (pack), everything else by bulk async copies issued by
-// lane 0 that complete on the stage's full barrier.
+// lane 0 that complete on the stage's full barrier.  In commit mode it also
+// writes the job's result code when it meets the job's first item.
 template <int MODE, int STAGE_BYTES, int STAGES, bool ZERO_PAD>
-__device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling &tl, uint32_t n_items, const Ring &ring,
-                                            volatile uint32_t *abort_flag, int lane)
+__device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling &tl, uint32_t n_items, uint32_t *ctr,
+                                            uint32_t ctr_base, const Ring &ring, volatile uint32_t *abort_flag,
+                                            int lane)
 {
     uint32_t n = 0;
-    for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    for (;;) {
+        const uint32_t item = next_item(ctr, ctr_base, lane);
+        if (item >= n_items) break;
         Item it;
-        if (!get_item<MODE>(P, tl, item, it, false, abort_flag)) continue;
+        if (!get_item<MODE>(P, tl, item, it, lane == 0, abort_flag)) continue;
         const uint8_t *rec = (MODE == kPack) ? nullptr : it.jb->blob + (uint64_t)it.p * P.g.R;
         const uint32_t slab_len = it.t * P.g.row;
         for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
             const uint32_t s = n % STAGES;
             const uint32_t use = n / STAGES;
-            if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE, P.w.wait_limit_ns);
+            if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE,
+                                    P.w.wait_limit_ns);
             uint32_t lead, nreal;
             uint64_t r0;
             tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
@@ -556,40 +577,55 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                 fence_proxy_async_smem();
             }
             __syncwarp();
-            if (lane == 0 && !*abort_flag) {
-                const uint32_t bar = ring.full0 + 8u * s;
-                if (MODE == kPack) {
-                    const uint32_t data_bytes = nreal - scale_bytes;
-                    if (data_bytes == 0u) {
-                        mbar_arrive(bar);
-                    } else {
-                        mbar_arrive_expect_tx(bar, data_bytes);
-                        uint64_t d0 = r0 + scale_bytes - P.g.S;  // offset in the record's data part
-                        const uint64_t d1 = d0 + data_bytes;
-                        uint32_t so = sbase + lead + scale_bytes;
-                        uint32_t slab = (uint32_t)(d0 / slab_len);
-                        uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
-                        while (d0 < d1) {
-                            uint32_t nb = slab_len - off;
-                            if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
-                            bulk_g2s(so, slab_addr(P.cache, slab, it.phys, off), nb, bar);
-                            d0 += nb;
-                            so += nb;
-                            ++slab;
-                            off = 0u;
+            if (lane == 0) {
+                ring.tag[s] = make_uint2(item, k);
+                if (!*abort_flag) {
+                    const uint32_t bar = ring.full0 + 8u * s;
+                    if (MODE == kPack) {
+                        const uint32_t data_bytes = nreal - scale_bytes;
+                        if (data_bytes == 0u) {
+                            mbar_arrive(bar);
+                        } else {
+                            mbar_arrive_expect_tx(bar, data_bytes);
+                            uint64_t d0 = r0 + scale_bytes - P.g.S;  // offset in the record's data part
+                            const uint64_t d1 = d0 + data_bytes;
+                            uint32_t so = sbase + lead + scale_bytes;
+                            uint32_t slab = (uint32_t)(d0 / slab_len);
+                            uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
+                            while (d0 < d1) {
+                                uint32_t nb = slab_len - off;
+                                if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
+                                bulk_g2s(so, slab_addr(P.cache, slab, it.phys, off), nb, bar);
+                                d0 += nb;
+                                so += nb;
+                                ++slab;
+                                off = 0u;
+                            }
                         }
-                    }
-                } else {
-                    if (nreal == 0u) {
-                        mbar_arrive(bar);
                     } else {
-                        mbar_arrive_expect_tx(bar, nreal);
+                        if (nreal == 0u) {
+                            mbar_arrive(bar);
+                        } else {
+                            mbar_arrive_expect_tx(bar, nreal);
                             bulk_g2s(sbase + lead, rec + r0, nreal, bar);
+                        }
                     }
                 }
             }
             __syncwarp();
         }
+    }
+    // tell the other roles of this CTA that there is no more work
+    {
+        const uint32_t s = n % STAGES;
+        const uint32_t use = n / STAGES;
+        if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE,
+                                P.w.wait_limit_ns);
+        if (lane == 0) {
+            ring.tag[s] = make_uint2(kEndOfWork, 0u);
+            mbar_arrive(ring.full0 + 8u * s);
+        }
+        ++n;
     }
     // before leaving: every load this CTA issued must have landed
     if (lane == 0) {
@@ -601,71 +637,80 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
 }
 
 // ------------------------------ storer role ------------------------------
-// One warp.  Waits for each tile to land and writes it out with bulk async
-// copies: one contiguous piece into the blob (pack), or one piece per slab into
-// the destination cache plus the scale values by the lanes (commit).  A stage
-// goes back to the loader once the copy of the following tile has been issued
-// and the stage's own copy has finished reading shared memory.
+// One warp.  Waits for each tile to land, reads its tag, and writes it out with
+// bulk async copies: one contiguous piece into the blob (pack), or one piece per
+// slab into the destination cache plus the scale values by the lanes (commit).
+// A stage goes back to the loader once the copy of the following tile has been
+// issued and the stage's own copy has finished reading shared memory.
 template <int MODE, int STAGE_BYTES, int STAGES>
-__device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling &tl, uint32_t n_items, const Ring &ring,
+__device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling &tl, const Ring &ring,
                                             volatile uint32_t *abort_flag, int lane)
 {
     uint32_t n = 0;
-    for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
-        Item it;
-        if (!get_item<MODE>(P, tl, item, it, lane == 0, abort_flag)) continue;
-        uint8_t *rec = it.jb->blob + (uint64_t)it.p * P.g.R;
-        const uint32_t slab_len = it.t * P.g.row;
-        for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
-            const uint32_t s = n % STAGES;
-            const bool ok = mbar_wait(ring.full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE, P.w.wait_limit_ns);
-            uint32_t lead, nreal;
-            uint64_t r0;
-            tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
-            const uint32_t sbase = ring.stage0 + s * STAGE_BYTES;
-            const uint8_t *sgen = ring.base + (size_t)s * STAGE_BYTES;
-            uint32_t scale_bytes = 0u;
-            if (MODE == kCommit && r0 < P.g.S && nreal > 0u) {
-                const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
-                scale_bytes = (uint32_t)(e1 - r0);
-                if (ok && !*abort_flag) {
-                    for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
-                        const uint32_t v = *reinterpret_cast<const uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0));
-                        *reinterpret_cast<uint32_t *>(scale_addr(P.g, P.cache, i, it.phys)) = v;
-                    }
-                }
-            }
-            __syncwarp();
-            if (lane == 0) {
-                if (ok && !*abort_flag && nreal > 0u) {
-                    if (MODE == kPack) {
-                        bulk_s2g(rec + r0, sbase + lead, nreal);
-                    } else {
-                        const uint32_t data_bytes = nreal - scale_bytes;
-                        uint64_t d0 = r0 + scale_bytes - P.g.S;
-                        const uint64_t d1 = d0 + data_bytes;
-                        uint32_t so = sbase + lead + scale_bytes;
-                        uint32_t slab = (uint32_t)(d0 / slab_len);
-                        uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
-                        while (d0 < d1) {
-                            uint32_t nb = slab_len - off;
-                            if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
-                            bulk_s2g(slab_addr(P.cache, slab, it.phys, off), so, nb);
-                            d0 += nb;
-                            so += nb;
-                            ++slab;
-                            off = 0u;
-                        }
-                    }
-                }
-                bulk_commit();
-                if (n > 0u) {
-                    bulk_wait_read<1>();
-                    mbar_arrive(ring.empty0 + 8u * ((n - 1u) % STAGES));
-                }
-            }
-            __syncwarp();
+    uint32_t cur_item = kEndOfWork;
+    Item it{};
+    uint8_t *rec = nullptr;
+    uint32_t slab_len = 0;
+    for (;; ++n) {
+        const uint32_t s = n % STAGES;
+        bool ok = mbar_wait(ring.full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE,
+                            P.w.wait_limit_ns);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;  // the CTA has given up: nothing more is stored (decided by the whole warp)
+        const uint2 tag = ring.tag[s];
+        if (tag.x == kEndOfWork) break;
+        if (tag.x != cur_item) {
+            cur_item = tag.x;
+            get_item<MODE>(P, tl, cur_item, it, false, abort_flag);
+            rec = it.jb->blob + (uint64_t)it.p * P.g.R;
+            slab_len = it.t * P.g.row;
         }
+        uint32_t lead, nreal;
+        uint64_t r0;
+        tile_range<STAGE_BYTES>(it.tile_begin + tag.y, it.pad, lead, r0, nreal);
+        const uint32_t sbase = ring.stage0 + s * STAGE_BYTES;
+        const uint8_t *sgen = ring.base + (size_t)s * STAGE_BYTES;
+        uint32_t scale_bytes = 0u;
+        if (MODE == kCommit && r0 < P.g.S && nreal > 0u) {
+            const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
+            scale_bytes = (uint32_t)(e1 - r0);
+            if (!*abort_flag) {
+                for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
+                    const uint32_t v = *reinterpret_cast<const uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0));
+                    *reinterpret_cast<uint32_t *>(scale_addr(P.g, P.cache, i, it.phys)) = v;
+                }
+            }
+        }
+        __syncwarp();
+        if (lane == 0) {
+            if (!*abort_flag && nreal > 0u) {
+                if (MODE == kPack) {
+                    bulk_s2g(rec + r0, sbase + lead, nreal);
+                } else {
+                    const uint32_t data_bytes = nreal - scale_bytes;
+                    uint64_t d0 = r0 + scale_bytes - P.g.S;
+                    const uint64_t d1 = d0 + data_bytes;
+                    uint32_t so = sbase + lead + scale_bytes;
+                    uint32_t slab = (uint32_t)(d0 / slab_len);
+                    uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
+                    while (d0 < d1) {
+                        uint32_t nb = slab_len - off;
+                        if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
+                        bulk_s2g(slab_addr(P.cache, slab, it.phys, off), so, nb);
+                        d0 += nb;
+                        so += nb;
+                        ++slab;
+                        off = 0u;
+                    }
+                }
+            }
+            bulk_commit();
+            if (n > 0u) {
+                bulk_wait_read<1>();
+                mbar_arrive(ring.empty0 + 8u * ((n - 1u) % STAGES));
+            }
+        }
+        __syncwarp();
     }
     if (lane == 0) {
         bulk_wait_all();
@@ -686,9 +731,25 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
     RingPos pos;
     uint32_t parity_red = 0;
     constexpr int kTilesPerGran = (NT * 256) / STAGE_BYTES;
-    for (uint32_t item = blockIdx.x; item < P.n_items; item += gridDim.x) {
+    for (;;) {
+        // the first tile of the next item (or the end mark) says what comes next
+        const bool ok = mbar_wait(ring.full0 + 8u * pos.stage, pos.phase, abort_flag, P.w.error, 0x400u | MODE,
+                                  P.w.wait_limit_ns);
+        // leaving must be a decision of all NT consumer threads, or the barrier below would hang
+        uint32_t any_failed;
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t"
+            "setp.ne.u32 q, %1, 0;\n\t"
+            "barrier.red.or.pred p, 2, %2, q;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(any_failed)
+            : "r"(ok ? 0u : 1u), "n"(NT)
+            : "memory");
+        if (any_failed) break;
+        const uint32_t item = ring.tag[pos.stage].x;
+        if (item == kEndOfWork) break;
         Item it;
-        if (!get_item<MODE>(P, P.tl, item, it, false, abort_flag)) continue;
+        get_item<MODE>(P, P.tl, item, it, false, abort_flag);
         uint32_t R[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) R[i] = 0u;
@@ -738,9 +799,11 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
     }
 }
 
-__device__ __forceinline__ void ring_init(Ring &ring, uint8_t *base, uint64_t *bars, int stages, uint32_t empty_count)
+__device__ __forceinline__ void ring_init(Ring &ring, uint8_t *base, uint64_t *bars, uint2 *tags, int stages,
+                                          uint32_t empty_count)
 {
     ring.base = base;
+    ring.tag = tags;
     ring.stage0 = smem_u32(base);
     ring.full0 = smem_u32(bars);
     ring.empty0 = smem_u32(bars + stages);
@@ -763,11 +826,12 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
     uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
     uint64_t *red = bars + 2 * STAGES;  // [2][8]
     volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
+    uint2 *tags = (uint2 *)(red + 18);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     Ring ring;
-    ring_init(ring, smem, bars, STAGES, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)));
+    ring_init(ring, smem, bars, tags, STAGES, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)));
     if (threadIdx.x == 0) {
         *abort_flag = 0u;
         fence_mbar_init();
@@ -775,12 +839,14 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
     __syncthreads();
 
     if (warp == Cfg::kLoaderWarp) {
-        loader_role<MODE, STAGE_BYTES, STAGES, Cfg::kCrc>(P, MODE == kCommit ? P.tlc : P.tl,
-                                                          MODE == kCommit ? P.n_items_c : P.n_items, ring, abort_flag,
-                                                          lane);
+        if (MODE == kCommit)
+            loader_role<MODE, STAGE_BYTES, STAGES, false>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, ring,
+                                                          abort_flag, lane);
+        else
+            loader_role<MODE, STAGE_BYTES, STAGES, true>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, ring,
+                                                         abort_flag, lane);
     } else if (Cfg::kStore && warp == Cfg::kStorerWarp) {
-        storer_role<MODE, STAGE_BYTES, STAGES>(P, MODE == kCommit ? P.tlc : P.tl,
-                                               MODE == kCommit ? P.n_items_c : P.n_items, ring, abort_flag, lane);
+        storer_role<MODE, STAGE_BYTES, STAGES>(P, MODE == kCommit ? P.tlc : P.tl, ring, abort_flag, lane);
     } else if constexpr (Cfg::kCrc) {
         consumer_role<MODE, NT, STAGE_BYTES, STAGES>(P, ring, red, abort_flag, threadIdx.x, warp, lane);
     }
@@ -796,7 +862,7 @@ struct RestoreCfg {
     static constexpr int kConsWarps = NT / 32;
     static constexpr int kThreads = NT + 96;
     static constexpr size_t kSmemBytes =
-        (size_t)VST * VSB + (size_t)CST * CSB + 2 * (VST + CST) * 8 + 2 * 8 * 8 + 16 + 128;
+        (size_t)VST * VSB + (size_t)CST * CSB + 3 * (VST + CST) * 8 + 2 * 8 * 8 + 16 + 128;
 };
 
 template <int NT, int VSB, int VST, int CSB, int CST, int MINB>
@@ -810,12 +876,14 @@ __global__ void __launch_bounds__(NT + 96, MINB) restore_kernel(const __grid_con
     uint64_t *cbars = vbars + 2 * VST;
     uint64_t *red = cbars + 2 * CST;  // [2][8]
     volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
+    uint2 *vtags = (uint2 *)(red + 18);
+    uint2 *ctags = vtags + VST;
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     Ring vring, cring;
-    ring_init(vring, vbase, vbars, VST, (uint32_t)(NT / 32));
-    ring_init(cring, cbase, cbars, CST, 1u);
+    ring_init(vring, vbase, vbars, vtags, VST, (uint32_t)(NT / 32));
+    ring_init(cring, cbase, cbars, ctags, CST, 1u);
     if (threadIdx.x == 0) {
         *abort_flag = 0u;
         fence_mbar_init();
@@ -826,11 +894,12 @@ __global__ void __launch_bounds__(NT + 96, MINB) restore_kernel(const __grid_con
     if (warp < kCons) {
         consumer_role<kVerify, NT, VSB, VST>(P, vring, red, abort_flag, threadIdx.x, warp, lane);
     } else if (warp == kCons) {
-        loader_role<kVerify, VSB, VST, true>(P, P.tl, P.n_items, vring, abort_flag, lane);
+        loader_role<kVerify, VSB, VST, true>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, vring, abort_flag, lane);
     } else if (warp == kCons + 1) {
-        loader_role<kCommit, CSB, CST, false>(P, P.tlc, P.n_items_c, cring, abort_flag, lane);
+        loader_role<kCommit, CSB, CST, false>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, cring, abort_flag,
+                                              lane);
     } else {
-        storer_role<kCommit, CSB, CST>(P, P.tlc, P.n_items_c, cring, abort_flag, lane);
+        storer_role<kCommit, CSB, CST>(P, P.tlc, cring, abort_flag, lane);
     }
     __syncthreads();
 }
