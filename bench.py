@@ -37,7 +37,7 @@ METRIC = "restored KV GB/s (read+write)"
 UNIT = "GB/s"
 
 # DRAM bytes per blob byte of one launch of the fused restore kernel, from the
-# ncu capture summarised in profiles/restore_kernel_gqa7b_2blocks.md (dram read +
+# ncu capture of the 2-block case summarised under profiles/ (dram read +
 # write of the launch divided by the blob bytes it restores).  Traffic grows in
 # proportion to the blob bytes, so a full launch is this ratio times its bytes.
 RESTORE_DRAM_BYTES_PER_BLOB_BYTE = 2.96

@@ -68,8 +68,13 @@ def load_library() -> ctypes.CDLL:
     if _lib is not None:
         return _lib
     if not os.path.exists(LIB_PATH):
-        raise ImportError(f"{LIB_PATH} not found: build it with `python -m paper_2609_39358_b200.build` "
-                          "(there is no CPU fallback)")
+        # not built yet in this tree: compile it now with nvcc (in-tree); there is no other path
+        try:
+            from . import build as _build
+            _build.build()
+        except Exception as e:
+            raise ImportError(f"{LIB_PATH} not found and building it failed ({e}); build it with "
+                              "`python -m paper_2609_39358_b200.build` (there is no CPU fallback)") from e
     L = ctypes.CDLL(LIB_PATH)
     vp, u32, u64p = ctypes.c_void_p, ctypes.c_uint32, ctypes.POINTER(ctypes.c_uint64)
     L.gk_blob_size.restype = ctypes.c_int
