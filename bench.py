@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress"],
+                    help="gqa7b is the headline workload (full JSON line); the others print a shorter line "
+                         "with the save and restore phases of that workload's shape")
     ap.add_argument("--blocks", type=int, default=0,
                     help="restore this many blocks instead of the workload's 16 (small cases for profiling)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -551,6 +554,107 @@ def run_ours(args):
     comm.close()
 
 
+# ---------------------------------------------------------------------------
+# the other workload shapes: save + restore phases only
+# ---------------------------------------------------------------------------
+def run_other_workload(args):
+    import torch
+    import synth
+    import paper_2609_39358_b200 as gk
+
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    w = synth.WORKLOADS[args.workload]
+    if args.workload == "tiny":
+        lens, dst_pages = synth.TINY_BLOCKS, synth.TINY_DST_PAGES
+    elif args.workload == "corpus":
+        lens, dst_pages = synth.CORPUS_BLOCKS, synth.CORPUS_DST_PAGES
+    elif args.workload == "fp8":
+        lens, dst_pages = synth.FP8_BLOCKS, sum(-(-n // w.page_tokens) for n in synth.FP8_BLOCKS) + 100
+    else:   # one wave of the stress mix: the blocks of the first requests that fit a 65,536-page cache
+        all_len = synth.stress_block_lengths(w.seed(0))
+        lens, dst_pages, used = [], 65536, 0
+        for req in synth.stress_requests(w.seed(1)):
+            need = sum(-(-int(all_len[b]) // w.page_tokens) for b in req)
+            if used + need > dst_pages:
+                break
+            lens += [int(all_len[b]) for b in req]
+            used += need
+    dtype = gk.GK_BF16 if w.dtype == "bf16" else gk.GK_FP8_E4M3
+    geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, dtype, w.scale_kv)
+    ctx = gk.Context(geom, device.index)
+    slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
+    pages = [-(-n // w.page_tokens) for n in lens]
+    src_pages = sum(pages)
+
+    def cache(num_pages, seed):
+        if w.dtype == "bf16":
+            data = synth.kv_bytes_bf16(2 * w.layers * num_pages * slab // 2, w.sigma, seed, device)
+            return gk.Cache(data, num_pages, 2 * num_pages * slab, num_pages * slab, slab)
+        data, scales = synth.kv_bytes_fp8(w.layers, num_pages, w.page_tokens, w.kv_heads, w.head_dim, w.sigma,
+                                          seed, device)
+        h4 = w.kv_heads * 4
+        return gk.Cache(data, num_pages, 2 * num_pages * slab, num_pages * slab, slab, scales,
+                        w.scale_kv * num_pages * h4, num_pages * h4, h4)
+
+    src, dst = cache(src_pages, w.seed(10)), cache(dst_pages, w.seed(11))
+    sperm = torch.from_numpy(synth.page_permutation(src_pages, w.seed(12))).to(device)
+    dperm = torch.from_numpy(synth.page_permutation(dst_pages, w.seed(13))).to(device)
+    pack_jobs, restore_jobs, off, total = [], [], 0, 0
+    for n, P in zip(lens, pages):
+        nb, _ = gk.gk_blob_size(geom, n)
+        total += nb
+        blob = torch.empty(nb, dtype=torch.uint8, device=device)
+        sums = torch.zeros(P, dtype=torch.int64, device=device)
+        pack_jobs.append(gk.Job(blob, sums, sperm[off:off + P].contiguous(), n))
+        restore_jobs.append(gk.Job(blob, sums, dperm[off:off + P].contiguous(), n))
+        off += P
+    nj = len(lens)
+    mask = torch.zeros(nj, dtype=torch.uint8, device=device)
+    fb = torch.zeros(nj, dtype=torch.int32, device=device)
+    status = torch.zeros(nj, dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream(device)
+
+    def step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        ctx.gk_pack_batch(src, pack_jobs, status)
+        if ev:
+            ev[1].record(stream)
+        ctx.gk_restore(restore_jobs, dst, mask, fb)
+        if ev:
+            ev[2].record(stream)
+
+    for _ in range(max(args.warmup, 3)):
+        step()
+    torch.cuda.synchronize(device)
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for k in range(args.steps):
+        step(events[k])
+    torch.cuda.synchronize(device)
+    assert int(mask.sum().item()) == 0 and int(status.sum().item()) == 0
+    pack_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in events]))
+    restore_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in events]))
+    step_ms = pack_ms + restore_ms
+    peak, peak_kind = measured_peak()
+    line = {"metric": METRIC, "value": 4 * total / (step_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1,
+            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": f"{args.workload}: {w.layers} layers, {w.kv_heads} KV heads, head_dim {w.head_dim}, "
+                                   f"{w.dtype}, {w.page_tokens}-token pages; {nj} blocks, {sum(lens)} tokens, "
+                                   f"{total / 2**30:.2f} GiB of blobs, {dst_pages}-page destination",
+                       "step": "gk_pack_batch + gk_restore of all blocks in one call each"},
+            "tokens_per_s": sum(lens) / (step_ms * 1e-3),
+            "phases": {"pack": {"ms": pack_ms, "gbs": 2 * total / (pack_ms * 1e-3) / 1e9,
+                                "frac_of_hbm_peak": 2 * total / (pack_ms * 1e-3) / 1e9 / peak},
+                       "restore": {"ms": restore_ms, "gbs_useful": 2 * total / (restore_ms * 1e-3) / 1e9,
+                                   "gbs_dram_model": 3 * total / (restore_ms * 1e-3) / 1e9,
+                                   "frac_of_hbm_peak_dram_model": 3 * total / (restore_ms * 1e-3) / 1e9 / peak,
+                                   "tokens_per_s": sum(lens) / (restore_ms * 1e-3)}},
+            "peak": {"hbm_gbs": peak, "kind": f"of {peak_kind}"}}
+    print(json.dumps(line), flush=True)
+
+
 def synth_requests(n_blocks):
     return f"{max(n_blocks // 2, 1)} requests x {min(n_blocks, 2)} blocks"
 
@@ -559,6 +663,8 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload != "gqa7b":
+        run_other_workload(args)
     else:
         run_ours(args)
 
