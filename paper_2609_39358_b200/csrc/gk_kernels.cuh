@@ -570,9 +570,20 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                 // scale values of this tile: gathered with ordinary loads
                 const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
                 scale_bytes = (uint32_t)(e1 - r0);
-                for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
-                    const uint32_t v = *reinterpret_cast<const uint32_t *>(scale_addr(P.g, P.cache, i, it.phys));
-                    *reinterpret_cast<uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0)) = v;
+                // eight loads in flight per lane: the loader must not sit on one global latency per value
+                const uint32_t i_end = (uint32_t)(e1 >> 2);
+                for (uint32_t i0 = (uint32_t)(r0 >> 2) + lane; i0 < i_end; i0 += 32u * 8u) {
+                    uint32_t v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const uint32_t i = i0 + 32u * u;
+                        v[u] = (i < i_end) ? *reinterpret_cast<const uint32_t *>(scale_addr(P.g, P.cache, i, it.phys)) : 0u;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const uint32_t i = i0 + 32u * u;
+                        if (i < i_end) *reinterpret_cast<uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0)) = v[u];
+                    }
                 }
                 fence_proxy_async_smem();
             }
