@@ -497,6 +497,40 @@ def test_device_wait_time_out_is_fail_closed(gk):
     ctx.close()
 
 
+def test_restore_beside_another_kernel_that_occupies_the_gpu(gk):
+    """The fused restore kernel must not depend on all of its CTAs being resident at once:
+    while a side stream keeps the SMs busy with large matrix products, a multi-job restore
+    still completes, bit-exact, without any wait running out."""
+    from gpu_harness import assert_cache_equal, dev_cache, dev_i32, sums_to_dev
+    og = G_BIG
+    T = og.page_tokens
+    src = random_cache(og, 40, seed=390)
+    jobs = _oracle_jobs(og, src, [12 * T, 9 * T + 1, 15 * T, 3 * T], 391, 48)
+    jobs[2].blob[1 << 20] ^= 0x08
+    clean = random_cache(og, 48, seed=392)
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs)
+    ctx = _ctx(gk, og)
+    keep = [(torch.from_numpy(j.blob).cuda(), sums_to_dev(j.checksums), dev_i32(j.page_table)) for j in jobs]
+    gjobs = [gk.Job(b, s, t, j.n_tokens) for (b, s, t), j in zip(keep, jobs)]
+    mask = torch.full((4,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.zeros(4, dtype=torch.int32, device="cuda")
+    a = torch.randn(8192, 8192, device="cuda", dtype=torch.bfloat16)
+    side = torch.cuda.Stream()
+    for rep in range(3):
+        d = dev_cache(clean)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for _ in range(6):
+                a @ a                                   # a few ms each, all SMs
+        ctx.gk_restore(gjobs, d, mask, fb)
+        torch.cuda.synchronize()
+        assert mask.cpu().tolist() == wmask.tolist() and fb.cpu().tolist() == wfb.tolist()
+        assert_cache_equal(d, want)
+    assert ctx.gk_get_stats()["device_wait_expired"] == 0
+    ctx.close()
+
+
 def test_padded_strides_leave_the_padding_alone(gk):
     """Caches whose pages, K/V planes and layers are separated by padding: pack reads
     only slab bytes, restore writes only slab bytes."""
