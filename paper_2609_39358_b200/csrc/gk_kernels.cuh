@@ -2,11 +2,19 @@
 //
 //   validate_kernel   page ids in range, missing records, page -> job map
 //   claim_kernel      a destination page may be claimed once per call
+//   prep_small_kernel both of the above plus the job table, in one launch (small calls)
 //   stream_kernel<>   one warp-specialised streaming kernel in three modes:
 //                       kVerify : blob -> smem -> CRC segment remainders
 //                       kPack   : cache slabs -> smem -> CRC + blob
 //                       kCommit : blob -> smem -> cache slabs (no CRC)
+//   restore_kernel<>  verify and commit pipelines side by side in one CTA; a job is
+//                     committed only after all of its pages have verified
 //   finalize_kernel   segment remainders -> page CRC-64/XZ; compare or write
+//   report_kernel     result codes of a verify-only call
+//
+// Every role of a streaming CTA is one of: loader warp (draws work items from a
+// global counter, fills ring stages with bulk async copies, tags them), consumer
+// warps (CRC), storer warp (bulk async copies out).  All waits are bounded.
 //
 // The CRC is computed bit-sliced: a thread reads the words t, t+NT, t+2NT, ...
 // of a segment, and each of the 32 bit positions of those words is treated as
