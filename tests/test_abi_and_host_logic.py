@@ -41,6 +41,19 @@ def test_library_exports_every_declared_symbol(gk):
     assert sorted(binding.EXPORTS) == names
 
 
+def test_header_is_plain_c_and_library_links_from_c(gk, tmp_path):
+    import subprocess
+    gk.load_library()
+    libdir = os.path.join(ROOT, "paper_2609_39358_b200")
+    exe = tmp_path / "abi_from_c"
+    build = subprocess.run(["gcc", "-std=c11", "-Wall", "-Wextra", "-Werror", "-pedantic",
+                            os.path.join(ROOT, "tests", "c", "abi_from_c.c"), "-o", str(exe),
+                            "-L" + libdir, "-l:libgk.so", "-Wl,-rpath," + libdir], capture_output=True, text=True)
+    assert build.returncode == 0, build.stderr
+    run = subprocess.run([str(exe)], capture_output=True, text=True, timeout=60)
+    assert run.returncode == 0 and "abi ok" in run.stdout, run.stdout + run.stderr
+
+
 def test_blob_size_matches_oracle_on_all_workloads(gk):
     from gpu_harness import gk_geom
     cases = [(synth.TINY, 256), (synth.GQA7B, 4096), (synth.CORPUS, 1024), (synth.CORPUS, 280),
