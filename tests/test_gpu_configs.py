@@ -293,8 +293,11 @@ def test_fp8_full(gk):
     ctx.close()
 
 
-def test_stress_waves(gk):
-    """20,000-block pool (lengths lognormal, clipped to [17, 4096]), 256 requests of
+@pytest.mark.parametrize("bad_frac", [0.01, 1.0 / 3.0])
+def test_stress_waves(gk, bad_frac):
+    """(bad_frac = 1/3 mirrors the paper's experiment with one in three loads
+    deliberately failed, Section 4.3 / Section 5: every request still completes.)
+    20,000-block pool (lengths lognormal, clipped to [17, 4096]), 256 requests of
     1..40 blocks drawn Zipf(1.1) without replacement, 1% of the blobs with 1..8
     flipped bits.  Only referenced blocks are materialised; requests run in
     waves that fit the destination cache; page tables never reuse a page within
@@ -306,7 +309,7 @@ def test_stress_waves(gk):
     T, s = w.page_tokens, _slab(w)
     lengths = synth.stress_block_lengths(w.seed(0))
     requests = synth.stress_requests(w.seed(1))
-    bad_ids, bad_flips = synth.stress_corrupted_blocks(w.seed(2))
+    bad_ids, bad_flips = synth.stress_corrupted_blocks(w.seed(2), frac=bad_frac)
     bad = dict(zip(bad_ids.tolist(), bad_flips.tolist()))
     unique = sorted({int(b) for r in requests for b in r})
     n_jobs = sum(len(r) for r in requests)
