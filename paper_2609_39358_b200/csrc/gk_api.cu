@@ -430,7 +430,7 @@ bool is_small_call(uint32_t n_jobs, uint64_t pages, const Tiling &crc)
 
 int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tiling &crc, const WorkDev &w,
                       uint64_t num_pages, bool need_tables, bool do_claims, cudaStream_t st, uint64_t *pages_out,
-                      uint64_t *bytes_out)
+                      uint64_t *bytes_out, uint8_t *status_out = nullptr)
 {
     PrepSmallParams pp{};
     int rc = fill_job_table(c, jobs, n_jobs, pp.jobs, nullptr, nullptr, need_tables, pages_out, bytes_out);
@@ -439,6 +439,7 @@ int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tili
     pp.n_seg_pow = crc.nseg_max;
     pp.do_claims = do_claims ? 1u : 0u;
     pp.num_pages = num_pages;
+    pp.status_out = status_out;
     prep_small_kernel<<<1, 1024, 0, st>>>(pp, w);
     GK_CUDA(c, cudaGetLastError());
     c->stats.kernels_launched++;
@@ -528,7 +529,8 @@ int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
     return GK_OK;
 }
 
-int launch_validate(gk_ctx *c, const WorkDev &w, uint64_t num_pages, int clear_claims, cudaStream_t st)
+int launch_validate(gk_ctx *c, const WorkDev &w, uint64_t num_pages, int clear_claims, cudaStream_t st,
+                    uint8_t *status_out = nullptr)
 {
     uint32_t grid = w.n_jobs;
     if (clear_claims) {
@@ -536,7 +538,7 @@ int launch_validate(gk_ctx *c, const WorkDev &w, uint64_t num_pages, int clear_c
         if (g2 > 2048) g2 = 2048;
         if (g2 > grid) grid = g2;
     }
-    validate_kernel<<<grid, 256, 0, st>>>(w, num_pages, clear_claims);
+    validate_kernel<<<grid, 256, 0, st>>>(w, num_pages, clear_claims, status_out);
     GK_CUDA(c, cudaGetLastError());
     c->stats.kernels_launched++;
     return GK_OK;
@@ -804,11 +806,12 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tl);
     if (is_small_call(n_jobs, pages, tl)) {
-        if ((rc = launch_prep_small(c, jobs, n_jobs, tl, w, cd.num_pages, true, false, st, &pages, &bytes)) != GK_OK)
+        if ((rc = launch_prep_small(c, jobs, n_jobs, tl, w, cd.num_pages, true, false, st, &pages, &bytes,
+                                    status_dev)) != GK_OK)
             return rc;
     } else {
         if ((rc = upload_jobs(c, jobs, n_jobs, l, tl, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
-        if ((rc = launch_validate(c, w, cd.num_pages, 0, st)) != GK_OK) return rc;
+        if ((rc = launch_validate(c, w, cd.num_pages, 0, st, status_dev)) != GK_OK) return rc;
     }
     StreamParams P{};
     P.g = c->gd;
@@ -816,8 +819,8 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
     P.w = w;
     P.tl = tl;
     P.n_items = (uint32_t)pages * tl.nseg_max;
+    P.inline_final = 1u;  // checksums are written by the CTA that delivers a page's last segment
     if ((rc = launch_pack(c, P, st)) != GK_OK) return rc;
-    if ((rc = launch_finalize(c, w, tl, 1, status_dev, st)) != GK_OK) return rc;
     c->stats.calls_pack++;
     c->stats.jobs += n_jobs;
     c->stats.pages += pages;
@@ -888,6 +891,7 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
     if (c->gd.flags & GK_FLAG_SKIP_VERIFY) return launch_commit(c, P, st);
     if (c->fused) {
         P.fused = 1u;
+        P.inline_final = 1u;
         if (c->test_drop_verify) P.n_items = 0;  // nothing gets verified: every commit wait must run out
         return launch_fused(c, P, st);
     }
@@ -1103,7 +1107,7 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
     if ((rc = upload_jobs(c, jobs, n_jobs, l, tl, hp.blob_dev.data(), hp.sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
         return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tl);
-    if ((rc = launch_validate(c, w, cd.num_pages, 0, st)) != GK_OK) return rc;
+    if ((rc = launch_validate(c, w, cd.num_pages, 0, st, status_dev)) != GK_OK) return rc;
 
     uint32_t j0 = 0, page0 = 0;
     int last_slot[kSlots] = {0, 0};
@@ -1123,8 +1127,8 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
         P.w = wb;
         P.tl = tl;
         P.n_items = npages * tl.nseg_max;
+        P.inline_final = 1u;
         if ((rc = launch_pack(c, P, st)) != GK_OK) return rc;
-        if ((rc = launch_finalize(c, wb, tl, 1, status_dev, st)) != GK_OK) return rc;
         GK_CUDA(c, cudaEventRecord(c->ev_copied[slot], st));
         GK_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_copied[slot], 0));
         for (uint32_t j = j0; j < j1; ++j) {

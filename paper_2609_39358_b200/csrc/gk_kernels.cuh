@@ -39,7 +39,7 @@ namespace gk {
 // One CTA per job.  Initialises the job's result words, records the lowest
 // out-of-range page id and fills page_job.  All CTAs together clear the claim
 // words of the destination cache.
-__global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims)
+__global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims, uint8_t *status_out)
 {
     const uint32_t j = blockIdx.x;
     if (clear_claims) {
@@ -65,6 +65,7 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims)
     __syncthreads();
     if (threadIdx.x == 0) {
         w.bad_range[j] = s_bad;
+        if (status_out) status_out[j] = s_bad != kNoPage ? 2u : 0u;  // save: the only thing that can fail
         w.bad_dup[j] = kNoPage;
         w.bad_crc[j] = kNoPage;
         w.job_done[j] = 0u;
@@ -105,6 +106,7 @@ struct PrepSmallParams {
     uint32_t n_seg_pow;
     uint32_t do_claims;
     uint64_t num_pages;
+    uint8_t *status_out;  // save calls: 0 or 2 per job; else null
 };
 
 __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant__ PrepSmallParams pp, WorkDev w)
@@ -134,6 +136,11 @@ __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant_
                     w.claims[id] = 0ull;
             }
         }
+    }
+    if (pp.status_out) {
+        __syncthreads();
+        for (uint32_t j = threadIdx.x; j < w.n_jobs; j += blockDim.x)
+            pp.status_out[j] = __ldcg(&w.bad_range[j]) != kNoPage ? 2u : 0u;
     }
     if (!pp.do_claims) return;
     __syncthreads();
@@ -244,6 +251,7 @@ struct StreamParams {
     uint32_t n_items;    // CRC work items: pages of the launch * tl.nseg_max
     uint32_t n_items_c;  // commit work items: pages of the launch * tlc.nseg_max
     uint32_t fused;      // 1: verify and commit run in one launch; commit waits per job
+    uint32_t inline_final;  // 1: the CTA that delivers a page's last segment finalizes the page itself
     uint32_t ctr_base_v, ctr_base_c;  // values of the work counters at the start of this launch
     uint8_t *mask_out;        // commit
     int32_t *first_bad_out;   // commit
@@ -791,7 +799,7 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
             // (nseg - 1 - q) full segments follow this one
             if (it.nseg > 1u) tot = gf_mul(tot, P.w.seg_pow[it.nseg - 1u - it.q]);
             uint64_t *res = P.w.seg_res + (uint64_t)it.gp * P.tl.nseg_max;
-            if (!P.fused) {
+            if (!P.inline_final) {
                 res[it.q] = tot;
             } else {
                 uint64_t r = tot;
@@ -808,9 +816,14 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
                 }
                 if (last) {
                     const uint64_t crc = __brevll(r ^ P.w.init_term[it.t] ^ ~0ull);
-                    if (crc != it.jb->checksums[it.p] || *abort_flag) atomicMin(&P.w.bad_crc[it.j], (int32_t)it.p);
-                    __threadfence();
-                    atomicAdd(&P.w.job_done[it.j], 1u);
+                    if (MODE == kPack) {
+                        it.jb->checksums[it.p] = crc;
+                    } else {
+                        if (crc != it.jb->checksums[it.p] || *abort_flag)
+                            atomicMin(&P.w.bad_crc[it.j], (int32_t)it.p);
+                        __threadfence();
+                        atomicAdd(&P.w.job_done[it.j], 1u);
+                    }
                 }
             }
         }
