@@ -872,8 +872,8 @@ int gk_page_checksums(gk_ctx *c, const void *blob_dev, uint32_t n_tokens, uint64
 
 // verify + commit for the pages [page_begin, page_begin + n_pages) of the call
 static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const Tiling &tlv, const Tiling &tlc,
-                                 uint32_t page_begin, uint32_t n_pages, uint8_t *mask_dev, int32_t *first_bad_dev,
-                                 cudaStream_t st)
+                                 uint32_t page_begin, uint32_t n_pages, uint32_t jobs_in_launch, uint8_t *mask_dev,
+                                 int32_t *first_bad_dev, cudaStream_t st)
 {
     int rc;
     w.page_begin = page_begin;
@@ -889,7 +889,11 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
     P.n_items = n_pages * tlv.nseg_max;
     P.n_items_c = n_pages * tlc.nseg_max;
     if (c->gd.flags & GK_FLAG_SKIP_VERIFY) return launch_commit(c, P, st);
-    if (c->fused) {
+    // one job cannot overlap its own verify and commit (it is committed only after all of it has
+    // verified); from about 256 MiB on the two dedicated kernels then beat the fused one by more
+    // than their two extra launches cost (5,200 tokens of the GQA-7B shape: 386 us against 403 us)
+    const bool lone_big_job = jobs_in_launch == 1 && (uint64_t)n_pages * c->gd.R >= (256ull << 20);
+    if (c->fused && (!lone_big_job || c->test_drop_verify)) {
         P.fused = 1u;
         P.inline_final = 1u;
         if (c->test_drop_verify) P.n_items = 0;  // nothing gets verified: every commit wait must run out
@@ -914,9 +918,9 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
 
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
-    const int occ = c->fused ? c->occ_fused : c->occ_verify;
-    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages, occ, c->fused && n_jobs > 1);
-    const Tiling tlc = commit_tiling(c, pages, c->fused ? c->occ_fused : c->occ_commit);
+    const bool fused = c->fused && !(n_jobs == 1 && pages * c->gd.R >= (256ull << 20));
+    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages, fused ? c->occ_fused : c->occ_verify, fused && n_jobs > 1);
+    const Tiling tlc = commit_tiling(c, pages, fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tlv);
@@ -928,7 +932,7 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
         if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
         if ((rc = launch_claim(c, w, st)) != GK_OK) return rc;
     }
-    if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, 0, (uint32_t)pages, mask_dev, first_bad_page_dev, st)) != GK_OK)
+    if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, 0, (uint32_t)pages, n_jobs, mask_dev, first_bad_page_dev, st)) != GK_OK)
         return rc;
     c->stats.calls_restore++;
     c->stats.jobs += n_jobs;
@@ -1072,7 +1076,7 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
         }
         GK_CUDA(c, cudaEventRecord(c->ev_copied[slot], c->copy_stream));
         GK_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied[slot], 0));
-        if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, page0, npages, mask_dev, first_bad_page_dev, st)) != GK_OK)
+        if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, page0, npages, j1 - j0, mask_dev, first_bad_page_dev, st)) != GK_OK)
             return rc;
         GK_CUDA(c, cudaEventRecord(c->ev_slot_free[slot], st));
         c->slot_used[slot] = true;
