@@ -565,6 +565,38 @@ def test_padded_strides_leave_the_padding_alone(gk):
     ctx.close()
 
 
+@pytest.mark.parametrize("og", [
+    oracle.Geom(3, 2, 16, 1, 1, 2),      # 32-byte slabs (one token per page, fp8): a tile is hundreds of copies
+    oracle.Geom(7, 1, 8, 3, 2, 0),       # 48-byte slabs, odd page size, odd layer count
+    oracle.Geom(1, 1, 8, 1, 2, 0),       # the smallest geometry the library accepts: 32-byte records
+    oracle.Geom(2, 3, 40, 5, 2, 0),      # nothing is a power of two
+])
+def test_extreme_small_geometries(gk, og):
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_pack, gpu_restore
+    T = og.page_tokens
+    N = 37
+    src = random_cache(og, N, seed=400)
+    lens = [1, T, 5 * T + (1 if T > 1 else 0), 11 * T]
+    rng = np.random.default_rng(401)
+    tables = [rng.integers(0, N, size=n_pages(og, n)).astype(np.int32) for n in lens]
+    ctx = _ctx(gk, og)
+    got, status = gpu_pack(ctx, og, dev_cache(src), tables, lens)
+    assert status.tolist() == [0] * len(lens)
+    for (blob, sums), pt, n in zip(got, tables, lens):
+        wb, ws, _, _ = oracle.pack(og, src, pt, n)
+        assert np.array_equal(blob, wb) and np.array_equal(sums, ws)
+    jobs = _oracle_jobs(og, src, lens, 402, 64)
+    jobs[2].blob[len(jobs[2].blob) - 1] ^= 0x40
+    clean = random_cache(og, 64, seed=403)
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs)
+    d = dev_cache(clean)
+    mask, fb = gpu_restore(ctx, d, jobs)
+    assert mask.tolist() == wmask.tolist() == [0, 0, 1, 0] and fb.tolist() == wfb.tolist()
+    assert_cache_equal(d, want)
+    ctx.close()
+
+
 def test_argument_errors(gk):
     from gpu_harness import dev_cache
     og = G_MID
