@@ -13,6 +13,13 @@ import torch.multiprocessing as mp
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 
 
+def _free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as s:
+        s.bind(("127.0.0.1", 0))
+        return s.getsockname()[1]
+
+
 def _worker(rank, world, port, out_dir):
     os.environ.update({"RANK": str(rank), "LOCAL_RANK": str(rank), "WORLD_SIZE": str(world),
                        "MASTER_ADDR": "127.0.0.1", "MASTER_PORT": str(port)})
@@ -30,7 +37,7 @@ def _worker(rank, world, port, out_dir):
 
 
 def test_rank_comm_over_gloo(tmp_path):
-    world, port = 2, 29533
+    world, port = 2, _free_port()
     mp.spawn(_worker, args=(world, port, str(tmp_path)), nprocs=world, join=True)
     res = [json.load(open(tmp_path / f"rank{r}.json")) for r in range(world)]
     for r in res:
@@ -69,14 +76,14 @@ def _tp_worker(rank, world, port, out_dir):
 
 
 def test_tp_restore_commits_a_block_on_all_ranks_or_none(tmp_path):
-    mp.spawn(_tp_worker, args=(2, 29535, str(tmp_path)), nprocs=2, join=True)
+    mp.spawn(_tp_worker, args=(2, _free_port(), str(tmp_path)), nprocs=2, join=True)
     res = [json.load(open(tmp_path / f"tp{r}.json")) for r in range(2)]
     assert res[0] == res[1] == {"mask": [0, 1, 0, 2, 3], "committed": [0, 2]}
 
 
 def test_reference_arm_under_torchrun_prints_one_line_on_rank0():
     cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", "2",
-           "--master-addr", "127.0.0.1", "--master-port", "29534", os.path.join(ROOT, "bench.py"),
+           "--master-addr", "127.0.0.1", "--master-port", str(_free_port()), os.path.join(ROOT, "bench.py"),
            "--impl", "reference", "--gpus", "2", "--steps", "1", "--warmup", "0", "--reference-seconds", "1"]
     out = subprocess.run(cmd, capture_output=True, text=True, timeout=300, cwd=ROOT)
     assert out.returncode == 0, out.stderr[-2000:]
