@@ -80,7 +80,8 @@ static uint64_t scale_section_bytes(const ok_geom *g)
 
 static uint32_t page_count(const ok_geom *g, uint32_t n_tokens)
 {
-    return (n_tokens + g->page_tokens - 1u) / g->page_tokens;
+    /* ceil(n / T), in 64 bits so that n close to 2^32 does not wrap */
+    return (uint32_t)(((uint64_t)n_tokens + g->page_tokens - 1u) / g->page_tokens);
 }
 
 /* tokens held by logical page p of a block of n_tokens */

@@ -83,6 +83,12 @@ uint64_t gf_xpow(uint64_t n)
 
 size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
+// pages of a block; 64-bit so that n_tokens near 2^32 does not wrap
+uint32_t pages_of(uint32_t n_tokens, uint32_t page_tokens)
+{
+    return (uint32_t)(((uint64_t)n_tokens + page_tokens - 1) / page_tokens);
+}
+
 }  // namespace
 
 struct gk_ctx {
@@ -374,7 +380,7 @@ int fill_job_table(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, JobDev *h, ui
         const gk_job &jb = jobs[j];
         if (jb.n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
         if (need_tables && !jb.page_table) return fail(c, GK_ERR_ARG, "job %u: null page table", j);
-        const uint32_t np = (jb.n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+        const uint32_t np = pages_of(jb.n_tokens, c->gd.page_tokens);
         h[j].blob = blob_override ? blob_override[j] : (uint8_t *)jb.blob;
         h[j].checksums = sums_override ? sums_override[j] : jb.checksums;
         h[j].page_table = jb.page_table;
@@ -578,7 +584,7 @@ int make_host_plan(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, bool allow_mi
     uint64_t max_need = 0, total_need = 0, pages = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) {
         if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
-        const uint32_t np = (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+        const uint32_t np = pages_of(jobs[j].n_tokens, c->gd.page_tokens);
         plan[j].pages = np;
         plan[j].blob_bytes = (uint64_t)np * c->gd.S + (uint64_t)jobs[j].n_tokens * c->gd.tokB;
         plan[j].sums_bytes = (uint64_t)np * 8;
@@ -667,7 +673,7 @@ int gk_blob_size(const gk_geom *geom, uint32_t n_tokens, uint64_t *blob_bytes, u
     const int rc = check_geom(geom, &gd);
     if (rc != GK_OK) return rc;
     if (n_tokens == 0) return GK_ERR_ARG;
-    const uint32_t np = (n_tokens + gd.page_tokens - 1) / gd.page_tokens;
+    const uint32_t np = pages_of(n_tokens, gd.page_tokens);
     if (blob_bytes) *blob_bytes = (uint64_t)np * gd.S + (uint64_t)n_tokens * gd.tokB;
     if (n_pages) *n_pages = np;
     return GK_OK;
@@ -800,7 +806,7 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
         if (!jobs[j].blob || !jobs[j].checksums) return fail(c, GK_ERR_ARG, "job %u: null output", j);
 
     uint64_t pages = 0, bytes = 0;
-    for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
     const Tiling tl = crc_tiling(c, GK_PACK_STAGE, pages, c->occ_pack);
     const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
@@ -850,7 +856,7 @@ int gk_page_checksums(gk_ctx *c, const void *blob_dev, uint32_t n_tokens, uint64
     jb.checksums = checksums_dev;
     jb.page_table = nullptr;
     jb.n_tokens = n_tokens;
-    uint64_t pages = (n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens, bytes = 0;
+    uint64_t pages = pages_of(n_tokens, c->gd.page_tokens), bytes = 0;
     const Tiling tl = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify);
     const WsLayout l = ws_layout(1, pages, tl.nseg_max, 0);
     int rc;
@@ -917,7 +923,7 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
     if (rc != GK_OK) return rc;
 
     uint64_t pages = 0, bytes = 0;
-    for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
     const bool fused = c->fused && !(n_jobs == 1 && pages * c->gd.R >= (256ull << 20));
     const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages, fused ? c->occ_fused : c->occ_verify, fused && n_jobs > 1);
     const Tiling tlc = commit_tiling(c, pages, fused ? c->occ_fused : c->occ_commit);
@@ -948,7 +954,7 @@ static int prepare_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const
     int rc = check_cache(c, dst, cd);
     if (rc != GK_OK) return rc;
     uint64_t pages = 0, bytes = 0;
-    for (uint32_t j = 0; j < n_jobs; ++j) pages += (jobs[j].n_tokens + c->gd.page_tokens - 1) / c->gd.page_tokens;
+    for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
     *tlv = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify);
     *tlc = commit_tiling(c, pages, c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv->nseg_max, cd->num_pages);

@@ -63,6 +63,17 @@ def test_blob_size_matches_oracle_on_all_workloads(gk):
         assert gk.gk_blob_size(gk_geom(og), n) == oracle.blob_size(og, n)
 
 
+def test_blob_size_at_the_top_of_the_token_range(gk):
+    """n_tokens = 2^32 - 1: the page count must not wrap (closed form P*S + n*tokB)."""
+    from gpu_harness import gk_geom
+    og = oracle.Geom(1, 1, 8, 16, 2, 0)
+    n = 0xFFFFFFFF
+    want_pages = -(-n // 16)
+    want_bytes = n * 2 * 1 * 16
+    assert gk.gk_blob_size(gk_geom(og), n) == (want_bytes, want_pages)
+    assert oracle.blob_size(og, n) == (want_bytes, want_pages)
+
+
 def test_argument_checks_without_gpu(gk):
     with pytest.raises(gk.GkError) as e:
         gk.gk_blob_size(gk.Geom(2, 2, 64, 16), 0)
