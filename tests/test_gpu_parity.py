@@ -597,6 +597,75 @@ def test_extreme_small_geometries(gk, og):
     ctx.close()
 
 
+def test_guard_bands_around_every_output_buffer(gk):
+    """Every buffer the library writes (blob, checksums, status, destination cache, scales,
+    mask, first_bad_page) sits inside a larger allocation filled with a sentinel: after
+    pack and restore the slack on both sides must be untouched."""
+    from gpu_harness import dev_i32
+    import paper_2609_39358_b200 as m
+    og = G_FP8_M
+    T, N, G = og.page_tokens, 13, 4096                      # G = guard bytes on each side
+    src = random_cache(og, N, seed=410)
+    lens = [2 * T + 1, T, 3 * T]
+    rng = np.random.default_rng(411)
+    tables = [rng.permutation(N)[:n_pages(og, n)].astype(np.int32) for n in lens]
+    ctx = _ctx(gk, og)
+
+    def guarded(nbytes, dtype=torch.uint8):
+        raw = torch.full((nbytes + 2 * G,), 0xA5, dtype=torch.uint8, device="cuda")
+        return raw, raw[G:G + nbytes].view(dtype)
+
+    def slack_ok(raw, nbytes):
+        return bool((raw[:G] == 0xA5).all()) and bool((raw[G + nbytes:] == 0xA5).all())
+
+    dsrc = m.Cache(torch.from_numpy(src.data).cuda(), N, src.layer_stride, src.kv_stride, src.page_stride,
+                   torch.from_numpy(src.scales).cuda(), src.s_layer_stride, src.s_kv_stride, src.s_page_stride)
+    bufs, jobs = [], []
+    for pt, n in zip(tables, lens):
+        nbytes, P = oracle.blob_size(og, n)
+        braw, blob = guarded(nbytes)
+        sraw, sums = guarded(8 * P, torch.int64)
+        bufs.append((braw, nbytes, sraw, 8 * P))
+        jobs.append(m.Job(blob, sums, dev_i32(pt), n))
+    straw, status = guarded(len(jobs))
+    ctx.gk_pack_batch(dsrc, jobs, status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, 0, 0]
+    for (braw, nb, sraw, ns), job, pt, n in zip(bufs, jobs, tables, lens):
+        assert slack_ok(braw, nb) and slack_ok(sraw, ns)
+        wb, ws, _, _ = oracle.pack(og, src, pt, n)
+        assert np.array_equal(job.blob.cpu().numpy(), wb)
+    assert slack_ok(straw, len(jobs))
+    # restore into a guarded destination
+    Nd = 16
+    clean = random_cache(og, Nd, seed=412)
+    draw, ddata = guarded(clean.data.size)
+    ddata.copy_(torch.from_numpy(clean.data))
+    scraw, dscales = guarded(clean.scales.size)
+    dscales.copy_(torch.from_numpy(clean.scales))
+    dst = m.Cache(ddata, Nd, clean.layer_stride, clean.kv_stride, clean.page_stride, dscales,
+                  clean.s_layer_stride, clean.s_kv_stride, clean.s_page_stride)
+    perm = rng.permutation(Nd).astype(np.int32)
+    rjobs, ojobs, off = [], [], 0
+    for job, n in zip(jobs, lens):
+        P = n_pages(og, n)
+        dpt = perm[off:off + P]
+        off += P
+        rjobs.append(m.Job(job.blob, job.checksums, dev_i32(dpt), n))
+        ojobs.append(oracle.Job(job.blob.cpu().numpy(), job.checksums.cpu().numpy().view(np.uint64), dpt, n))
+    mraw, mask = guarded(len(rjobs))
+    fraw, fb = guarded(4 * len(rjobs), torch.int32)
+    ctx.gk_restore(rjobs, dst, mask, fb)
+    torch.cuda.synchronize()
+    want = clone_cache(clean)
+    wmask, _ = oracle.restore(og, want, ojobs)
+    assert mask.cpu().tolist() == wmask.tolist() == [0, 0, 0]
+    assert np.array_equal(ddata.cpu().numpy(), want.data) and np.array_equal(dscales.cpu().numpy(), want.scales)
+    assert slack_ok(draw, clean.data.size) and slack_ok(scraw, clean.scales.size)
+    assert slack_ok(mraw, len(rjobs)) and slack_ok(fraw, 4 * len(rjobs))
+    ctx.close()
+
+
 def test_argument_errors(gk):
     from gpu_harness import dev_cache
     og = G_MID
