@@ -42,7 +42,8 @@ def build(force: bool = False) -> str:
 class _CGeom(ctypes.Structure):
     _fields_ = [("layers", ctypes.c_uint32), ("kv_heads", ctypes.c_uint32),
                 ("head_dim", ctypes.c_uint32), ("page_tokens", ctypes.c_uint32),
-                ("elem_bytes", ctypes.c_uint32), ("scale_kv", ctypes.c_uint32)]
+                ("elem_bytes", ctypes.c_uint32), ("scale_kv", ctypes.c_uint32),
+                ("head_major", ctypes.c_uint32)]
 
 
 class _CCache(ctypes.Structure):
@@ -121,10 +122,11 @@ class Geom:
     page_tokens: int
     elem_bytes: int = 2
     scale_kv: int = 0
+    head_major: int = 0
 
     def c(self) -> _CGeom:
         return _CGeom(self.layers, self.kv_heads, self.head_dim, self.page_tokens,
-                      self.elem_bytes, self.scale_kv)
+                      self.elem_bytes, self.scale_kv, self.head_major)
 
 
 @dataclass

@@ -133,6 +133,30 @@ static uint8_t *scale_ptr(const ok_cache *c, uint32_t l, uint32_t kv, int32_t pa
            (uint64_t)page * c->s_page_stride + 4ull * h;
 }
 
+/* Copies the valid part of one slab (the first t tokens) between a cache slab and
+ * a record: one contiguous prefix for a token-major slab, one prefix per head for
+ * a head-major slab.  to_record != 0: slab -> record, else record -> slab. */
+static uint64_t copy_slab_prefix(const ok_geom *g, uint8_t *slab, uint8_t *rec, uint32_t t, int to_record)
+{
+    uint64_t row = row_bytes(g);
+    if (!g->head_major) {
+        if (to_record)
+            memcpy(rec, slab, (size_t)(t * row));
+        else
+            memcpy(slab, rec, (size_t)(t * row));
+        return t * row;
+    }
+    uint64_t tok = (uint64_t)g->head_dim * g->elem_bytes;       /* one token of one head */
+    uint64_t head_block = (uint64_t)g->page_tokens * tok;       /* one head's part of the slab */
+    for (uint32_t h = 0; h < g->kv_heads; ++h) {
+        if (to_record)
+            memcpy(rec + h * t * tok, slab + h * head_block, (size_t)(t * tok));
+        else
+            memcpy(slab + h * head_block, rec + h * t * tok, (size_t)(t * tok));
+    }
+    return t * row;
+}
+
 static int32_t lowest_out_of_range(const int32_t *pt, uint32_t P, uint64_t num_pages)
 {
     for (uint32_t p = 0; p < P; ++p)
@@ -148,7 +172,6 @@ int ok_pack(const ok_geom *g, const ok_cache *src, const int32_t *page_table,
             uint32_t n_tokens, uint8_t *blob, uint64_t *checksums, int32_t *bad_index)
 {
     uint32_t P = page_count(g, n_tokens);
-    uint64_t row = row_bytes(g);
     int32_t bad = lowest_out_of_range(page_table, P, src->num_pages);
     if (bad_index)
         *bad_index = bad;
@@ -159,7 +182,7 @@ int ok_pack(const ok_geom *g, const ok_cache *src, const int32_t *page_table,
         uint8_t *rec = blob + ok_record_offset(g, p);
         uint8_t *w = rec;
         int32_t page = page_table[p];
-        uint64_t prefix = (uint64_t)tokens_in_page(g, n_tokens, p) * row;
+        uint32_t t = tokens_in_page(g, n_tokens, p);
 
         for (uint32_t l = 0; l < g->layers; ++l)
             for (uint32_t kv = 0; kv < g->scale_kv; ++kv)
@@ -168,10 +191,8 @@ int ok_pack(const ok_geom *g, const ok_cache *src, const int32_t *page_table,
                     w += 4;
                 }
         for (uint32_t l = 0; l < g->layers; ++l)
-            for (uint32_t kv = 0; kv < 2; ++kv) {
-                memcpy(w, slab_ptr(src, l, kv, page), prefix);
-                w += prefix;
-            }
+            for (uint32_t kv = 0; kv < 2; ++kv)
+                w += copy_slab_prefix(g, slab_ptr(src, l, kv, page), w, t, 1);
         checksums[p] = ok_crc64(rec, (size_t)(w - rec));
     }
     return OK_CODE_OK;
@@ -183,7 +204,6 @@ int ok_pack(const ok_geom *g, const ok_cache *src, const int32_t *page_table,
 void ok_restore(const ok_geom *g, const ok_cache *dst, const ok_job *jobs, uint32_t n_jobs,
                 uint32_t flags, uint8_t *mask, int32_t *first_bad)
 {
-    uint64_t row = row_bytes(g);
     uint32_t *claims = (uint32_t *)calloc(dst->num_pages ? dst->num_pages : 1, sizeof(uint32_t));
 
     /* ---- phase 1a: missing records, ids out of range ---- */
@@ -245,7 +265,7 @@ void ok_restore(const ok_geom *g, const ok_cache *dst, const ok_job *jobs, uint3
         for (uint32_t p = 0; p < P; ++p) {
             const uint8_t *r = jobs[j].blob + ok_record_offset(g, p);
             int32_t page = jobs[j].page_table[p];
-            uint64_t prefix = (uint64_t)tokens_in_page(g, jobs[j].n_tokens, p) * row;
+            uint32_t t = tokens_in_page(g, jobs[j].n_tokens, p);
 
             for (uint32_t l = 0; l < g->layers; ++l)
                 for (uint32_t kv = 0; kv < g->scale_kv; ++kv)
@@ -254,10 +274,8 @@ void ok_restore(const ok_geom *g, const ok_cache *dst, const ok_job *jobs, uint3
                         r += 4;
                     }
             for (uint32_t l = 0; l < g->layers; ++l)
-                for (uint32_t kv = 0; kv < 2; ++kv) {
-                    memcpy(slab_ptr(dst, l, kv, page), r, prefix);
-                    r += prefix;
-                }
+                for (uint32_t kv = 0; kv < 2; ++kv)
+                    r += copy_slab_prefix(g, slab_ptr(dst, l, kv, page), (uint8_t *)r, t, 0);
         }
     }
     free(claims);

@@ -21,13 +21,17 @@
  *   cache   : opaque bytes.  The slab of (layer l, kv, page g) starts at
  *             data + l*layer_stride + kv*kv_stride + g*page_stride and holds
  *             page_tokens rows of row = kv_heads*head_dim*elem_bytes bytes,
- *             token-major.  kv = 0 is K, kv = 1 is V.
+ *             token-major ([t][h][d]).  kv = 0 is K, kv = 1 is V.  With
+ *             head_major = 1 the slab is [h][t][d] instead: head h owns
+ *             page_tokens*head_dim*elem_bytes contiguous bytes.
  *   scales  : (fp8 caches only) fp32 per (l, kv < scale_kv, page g, head h) at
  *             scales + l*s_layer_stride + kv*s_kv_stride + g*s_page_stride + 4*h.
  *   blob    : page records 0..P-1 back to back, no header, no padding.  Record
  *             p = [scale section: for l, for kv < scale_kv, for h: 4 bytes]
  *             then for l: K prefix (t_p*row bytes), V prefix (t_p*row bytes),
- *             where t_p = page_tokens except for a shorter last page.
+ *             where t_p = page_tokens except for a shorter last page.  The
+ *             prefix of a head-major slab is, head by head, the first t_p
+ *             tokens of that head (for a full page: the whole slab as it is).
  *   checksum: CRC-64/XZ over the bytes of record p, one uint64 per page.
  *
  * All pins for these functions are listed in tests/test_oracle_pins.py.
@@ -49,6 +53,7 @@ typedef struct {
     uint32_t page_tokens;
     uint32_t elem_bytes; /* 2 for bf16, 1 for fp8 e4m3 */
     uint32_t scale_kv;   /* 0: no scale section; 1: one scale per (l,page,h); 2: K and V scales */
+    uint32_t head_major; /* 0: a slab is [token][head][dim]; 1: a slab is [head][token][dim] */
 } ok_geom;
 
 typedef struct {

@@ -223,6 +223,62 @@ def test_pack_layout_against_numpy_views(g, n_tokens):
         assert int(sums[p]) == _crc_by_long_division(blob[lo:hi].tobytes())
 
 
+# head-major slabs ([head][token][dim]): full pages are the slab as it is, partial pages
+# keep the first t tokens of every head
+SMALL_HM = oracle.Geom(layers=3, kv_heads=4, head_dim=8, page_tokens=4, elem_bytes=2, scale_kv=0, head_major=1)
+SMALL_HM_FP8 = oracle.Geom(layers=2, kv_heads=4, head_dim=16, page_tokens=8, elem_bytes=1, scale_kv=2, head_major=1)
+
+
+@pytest.mark.parametrize("g", [SMALL_HM, SMALL_HM_FP8])
+def test_head_major_full_pages_equal_token_major(g):
+    """A full slab is opaque contiguous bytes in either layout, so on full pages the two
+    layouts must give the same blob and checksums."""
+    N = 9
+    src = random_cache(g, N, seed=60)
+    pt = np.random.default_rng(61).permutation(N)[:5].astype(np.int32)
+    n = 5 * g.page_tokens
+    g_tm = oracle.Geom(g.layers, g.kv_heads, g.head_dim, g.page_tokens, g.elem_bytes, g.scale_kv, 0)
+    b1, s1, c1, _ = oracle.pack(g, src, pt, n)
+    b2, s2, c2, _ = oracle.pack(g_tm, src, pt, n)
+    assert c1 == c2 == 0 and np.array_equal(b1, b2) and np.array_equal(s1, s2)
+
+
+@pytest.mark.parametrize("g", [SMALL_HM, SMALL_HM_FP8])
+@pytest.mark.parametrize("n_tokens", [1, 3, 9, 14])
+def test_head_major_layout_against_numpy_views(g, n_tokens):
+    N = 7
+    src = random_cache(g, N, seed=62)
+    pt = np.random.default_rng(63).permutation(N).astype(np.int32)
+    blob, sums, code, _ = oracle.pack(g, src, pt, n_tokens)
+    assert code == 0
+    L, H, D, T, E = g.layers, g.kv_heads, g.head_dim, g.page_tokens, g.elem_bytes
+    arr = src.data.reshape(L, 2, N, H, T, D * E)
+    sc = None if src.scales is None else src.scales.reshape(L, g.scale_kv, N, H * 4)
+    parts = []
+    for p in range(n_pages(g, n_tokens)):
+        t = min(T, n_tokens - p * T)
+        if sc is not None:
+            parts.append(sc[:, :, pt[p], :].reshape(-1))
+        parts.append(arr[:, :, pt[p], :, :t, :].reshape(-1))
+    assert np.array_equal(blob, np.concatenate(parts))
+    # round trip into a sentinel cache: valid tokens of every head restored, every other byte kept
+    Nd = 9
+    dst = random_cache(g, Nd, seed=64)
+    before = clone_cache(dst)
+    dpt = np.random.default_rng(65).permutation(Nd).astype(np.int32)[:n_pages(g, n_tokens)]
+    mask, _ = oracle.restore(g, dst, [oracle.Job(blob, sums, dpt, n_tokens)])
+    assert mask.tolist() == [0]
+    d = dst.data.reshape(L, 2, Nd, H, T, D * E)
+    b = before.data.reshape(L, 2, Nd, H, T, D * E)
+    touched = np.zeros(Nd, dtype=bool)
+    for p in range(n_pages(g, n_tokens)):
+        t = min(T, n_tokens - p * T)
+        assert np.array_equal(d[:, :, dpt[p], :, :t], arr[:, :, pt[p], :, :t])
+        assert np.array_equal(d[:, :, dpt[p], :, t:], b[:, :, dpt[p], :, t:])
+        touched[dpt[p]] = True
+    assert np.array_equal(d[:, :, ~touched], b[:, :, ~touched])
+
+
 def test_pack_is_a_permutation_of_the_valid_bytes():
     g, N = SMALL, 9
     src = random_cache(g, N, seed=13)
