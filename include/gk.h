@@ -18,7 +18,9 @@
  *                starts at data + l*layer_stride + kv*kv_stride + g*page_stride
  *                and holds page_tokens rows of row = kv_heads*head_dim*elem
  *                bytes, token-major ([t][h][d]); kv 0 is K, 1 is V.  One page id
- *                addresses all layers and both K and V.
+ *                addresses all layers and both K and V.  With GK_FLAG_HEAD_MAJOR
+ *                the slab is head-major instead ([h][t][d]: kv_heads runs of
+ *                page_tokens*head_dim*elem bytes).
  *   scales       fp8 caches only: one fp32 per (l, kv < scale_kv, page, head) at
  *                scales + l*s_layer_stride + kv*s_kv_stride + g*s_page_stride + 4*h.
  *   blob         Page records 0..P-1 (P = ceil(n_tokens/page_tokens)) back to
@@ -26,7 +28,10 @@
  *                for kv < scale_kv, for h: 4 bytes; absent for bf16), then for
  *                each layer the K prefix and the V prefix of the page, each
  *                t_p*row bytes, where t_p = page_tokens except for a shorter
- *                last page.  blob_bytes = P*S + n_tokens*2*layers*row.
+ *                last page.  blob_bytes = P*S + n_tokens*2*layers*row.  A prefix
+ *                of a head-major slab is, head by head, the first t_p tokens of
+ *                that head (t_p*head_dim*elem bytes each): a full page is the
+ *                slab as it lies in either layout, and the sizes do not change.
  *   checksums    uint64 per page: CRC-64/XZ of the bytes of its record.
  *
  * Conventions
@@ -81,6 +86,11 @@ extern "C" {
  * Page-table validation stays on. */
 #define GK_FLAG_SKIP_VERIFY 1u
 
+/* Slabs are head-major ([h][t][d]) instead of token-major.  Needs head_dim*elem to
+ * be a multiple of 16 bytes (else GK_ERR_UNSUPPORTED).  A layout choice of this
+ * library (the paper leaves the cache layout to the runtime it wraps). */
+#define GK_FLAG_HEAD_MAJOR 2u
+
 typedef struct gk_ctx gk_ctx;
 
 typedef struct {
@@ -91,7 +101,7 @@ typedef struct {
     uint32_t dtype;    /* GK_BF16 or GK_FP8_E4M3 */
     uint32_t scale_kv; /* fp8: 2 = a K scale and a V scale per (layer, head, page), 1 = one
                           shared scale; bf16: 0 */
-    uint32_t flags;    /* 0 or GK_FLAG_SKIP_VERIFY */
+    uint32_t flags;    /* 0 or an OR of GK_FLAG_SKIP_VERIFY, GK_FLAG_HEAD_MAJOR */
     uint32_t reserved; /* must be 0 */
 } gk_geom;
 

@@ -161,7 +161,7 @@ int check_geom(const gk_geom *g, GeomDev *out)
 {
     if (!g) return GK_ERR_ARG;
     if (g->layers == 0 || g->kv_heads == 0 || g->head_dim == 0 || g->page_tokens == 0) return GK_ERR_ARG;
-    if (g->reserved != 0 || (g->flags & ~GK_FLAG_SKIP_VERIFY)) return GK_ERR_ARG;
+    if (g->reserved != 0 || (g->flags & ~(GK_FLAG_SKIP_VERIFY | GK_FLAG_HEAD_MAJOR))) return GK_ERR_ARG;
     uint32_t elem;
     if (g->dtype == GK_BF16) {
         elem = 2;
@@ -175,6 +175,8 @@ int check_geom(const gk_geom *g, GeomDev *out)
     const uint64_t row = (uint64_t)g->kv_heads * g->head_dim * elem;
     const uint64_t S = (uint64_t)g->layers * g->scale_kv * g->kv_heads * 4u;
     if (row % 16 != 0 || S % 16 != 0) return GK_ERR_UNSUPPORTED;
+    const bool head_major = (g->flags & GK_FLAG_HEAD_MAJOR) != 0;
+    if (head_major && ((uint64_t)g->head_dim * elem) % 16 != 0) return GK_ERR_UNSUPPORTED;
     if (row * g->page_tokens > (1ull << 30) || S > (1ull << 30)) return GK_ERR_UNSUPPORTED;
     if (out) {
         out->layers = g->layers;
@@ -185,6 +187,8 @@ int check_geom(const gk_geom *g, GeomDev *out)
         out->S = (uint32_t)S;
         out->h4 = g->kv_heads * 4u;
         out->flags = g->flags;
+        out->hrow = g->head_dim * elem;
+        out->head_major = head_major ? 1u : 0u;
         out->tokB = 2ull * g->layers * row;
         out->R = S + (uint64_t)g->page_tokens * out->tokB;
     }

@@ -22,6 +22,8 @@ struct GeomDev {
     uint32_t S;     // scale section bytes of a record: layers*scale_kv*kv_heads*4
     uint32_t h4;    // kv_heads*4
     uint32_t flags;
+    uint32_t hrow;  // bytes of one token of one head: head_dim*elem
+    uint32_t head_major;  // 1: slabs are [head][token][dim]
     uint64_t tokB;  // bytes per token in a record: 2*layers*row
     uint64_t R;     // bytes of a full page record: S + page_tokens*tokB
 };

@@ -364,6 +364,40 @@ __device__ __forceinline__ uint8_t *slab_addr(const CacheDev &c, uint32_t slab, 
            (uint64_t)phys * c.page_stride + off;
 }
 
+// The data part of a record is a sequence of equal chunks, each contiguous in the
+// cache.  Token-major slabs, and full pages in either layout: one chunk per slab
+// (the first t rows).  A partial page of a head-major slab: one chunk per head
+// (that head's first t tokens), kv_heads chunks per slab.
+struct Chunks {
+    uint32_t len;       // bytes of one chunk
+    uint32_t per_slab;  // chunks per slab
+    uint32_t stride;    // distance between the chunks of one slab in the cache
+};
+
+__device__ __forceinline__ Chunks chunks_of(const GeomDev &g, uint32_t t)
+{
+    Chunks c;
+    if (g.head_major && t < g.page_tokens) {
+        c.len = t * g.hrow;
+        c.per_slab = g.kv_heads;
+        c.stride = g.page_tokens * g.hrow;
+    } else {
+        c.len = t * g.row;
+        c.per_slab = 1u;
+        c.stride = 0u;
+    }
+    return c;
+}
+
+__device__ __forceinline__ uint8_t *chunk_addr(const CacheDev &c, const Chunks &ch, uint32_t chunk, int32_t phys,
+                                               uint32_t off)
+{
+    if (ch.per_slab == 1u) return slab_addr(c, chunk, phys, off);  // the common case, without the division
+    const uint32_t slab = chunk / ch.per_slab;
+    const uint32_t sub = chunk - slab * ch.per_slab;
+    return slab_addr(c, slab, phys, (uint64_t)sub * ch.stride + off);
+}
+
 __device__ __forceinline__ uint8_t *scale_addr(const GeomDev &g, const CacheDev &c, uint32_t idx, int32_t phys)
 {
     // idx counts fp32 values of a scale section: [layer][kv < scale_kv][head]
@@ -566,7 +600,7 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
         Item it;
         if (!get_item<MODE>(P, tl, item, it, lane == 0, abort_flag)) continue;
         const uint8_t *rec = (MODE == kPack) ? nullptr : it.jb->blob + (uint64_t)it.p * P.g.R;
-        const uint32_t slab_len = it.t * P.g.row;
+        const Chunks ch = chunks_of(P.g, it.t);
         for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
             const uint32_t s = n % STAGES;
             const uint32_t use = n / STAGES;
@@ -617,15 +651,15 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                             uint64_t d0 = r0 + scale_bytes - P.g.S;  // offset in the record's data part
                             const uint64_t d1 = d0 + data_bytes;
                             uint32_t so = sbase + lead + scale_bytes;
-                            uint32_t slab = (uint32_t)(d0 / slab_len);
-                            uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
+                            uint32_t chunk = (uint32_t)(d0 / ch.len);
+                            uint32_t off = (uint32_t)(d0 - (uint64_t)chunk * ch.len);
                             while (d0 < d1) {
-                                uint32_t nb = slab_len - off;
+                                uint32_t nb = ch.len - off;
                                 if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
-                                bulk_g2s(so, slab_addr(P.cache, slab, it.phys, off), nb, bar);
+                                bulk_g2s(so, chunk_addr(P.cache, ch, chunk, it.phys, off), nb, bar);
                                 d0 += nb;
                                 so += nb;
-                                ++slab;
+                                ++chunk;
                                 off = 0u;
                             }
                         }
@@ -677,7 +711,7 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling 
     uint32_t cur_item = kEndOfWork;
     Item it{};
     uint8_t *rec = nullptr;
-    uint32_t slab_len = 0;
+    Chunks ch{};
     for (;; ++n) {
         const uint32_t s = n % STAGES;
         bool ok = mbar_wait(ring.full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE,
@@ -690,7 +724,7 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling 
             cur_item = tag.x;
             get_item<MODE>(P, tl, cur_item, it, false, abort_flag);
             rec = it.jb->blob + (uint64_t)it.p * P.g.R;
-            slab_len = it.t * P.g.row;
+            ch = chunks_of(P.g, it.t);
         }
         uint32_t lead, nreal;
         uint64_t r0;
@@ -718,15 +752,15 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling 
                     uint64_t d0 = r0 + scale_bytes - P.g.S;
                     const uint64_t d1 = d0 + data_bytes;
                     uint32_t so = sbase + lead + scale_bytes;
-                    uint32_t slab = (uint32_t)(d0 / slab_len);
-                    uint32_t off = (uint32_t)(d0 - (uint64_t)slab * slab_len);
+                    uint32_t chunk = (uint32_t)(d0 / ch.len);
+                    uint32_t off = (uint32_t)(d0 - (uint64_t)chunk * ch.len);
                     while (d0 < d1) {
-                        uint32_t nb = slab_len - off;
+                        uint32_t nb = ch.len - off;
                         if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
-                        bulk_s2g(slab_addr(P.cache, slab, it.phys, off), so, nb);
+                        bulk_s2g(chunk_addr(P.cache, ch, chunk, it.phys, off), so, nb);
                         d0 += nb;
                         so += nb;
-                        ++slab;
+                        ++chunk;
                         off = 0u;
                     }
                 }

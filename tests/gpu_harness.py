@@ -11,6 +11,8 @@ import paper_2609_39358_b200 as gk
 
 def gk_geom(og: oracle.Geom, flags: int = 0) -> gk.Geom:
     dtype = gk.GK_BF16 if og.elem_bytes == 2 else gk.GK_FP8_E4M3
+    if og.head_major:
+        flags |= gk.GK_FLAG_HEAD_MAJOR
     return gk.Geom(og.layers, og.kv_heads, og.head_dim, og.page_tokens, dtype, og.scale_kv, flags)
 
 

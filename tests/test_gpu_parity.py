@@ -179,6 +179,71 @@ def test_pack_host_parity(gk, og):
 
 
 # ---------------------------------------------------------------------------
+# head-major slabs: partial pages are gathered / scattered head by head
+# ---------------------------------------------------------------------------
+HM_MID = oracle.Geom(5, 4, 64, 16, 2, 0, head_major=1)       # 128 B per token and head
+HM_BIG = oracle.Geom(16, 8, 128, 16, 2, 0, head_major=1)     # chunks of t*256 B, 256 chunks per partial page
+HM_FP8 = oracle.Geom(10, 8, 64, 32, 1, 2, head_major=1)      # 64 B per token and head, with scales
+HM_MIN = oracle.Geom(3, 2, 8, 4, 2, 0, head_major=1)         # 16 B per token and head: the smallest allowed
+HM_GEOMS = [HM_MID, HM_BIG, HM_FP8, HM_MIN]
+
+
+@pytest.mark.parametrize("og", HM_GEOMS)
+def test_head_major_pack_parity(gk, og):
+    from gpu_harness import dev_cache, gpu_pack
+    N = 19
+    src = random_cache(og, N, seed=210)
+    dsrc = dev_cache(src)
+    rng = np.random.default_rng(211)
+    T = og.page_tokens
+    lens = [1, T - 1, T, T + 1, 3 * T + T // 2, 2 * T, 5 * T - 1]
+    tables = [rng.integers(0, N, size=n_pages(og, n)).astype(np.int32) for n in lens]
+    for seg in (0, 1):
+        ctx = _ctx(gk, og, seg_granules=seg)
+        got, status = gpu_pack(ctx, og, dsrc, tables, lens)
+        assert status.tolist() == [0] * len(lens)
+        for (blob, sums), pt, n in zip(got, tables, lens):
+            wb, ws, code, _ = oracle.pack(og, src, pt, n)
+            assert code == 0
+            assert np.array_equal(blob, wb), f"blob differs at {np.flatnonzero(blob != wb)[:8]}"
+            assert np.array_equal(sums, ws)
+        ctx.close()
+
+
+@pytest.mark.parametrize("og", HM_GEOMS)
+@pytest.mark.parametrize("host_tier", [False, True])
+def test_head_major_restore_parity(gk, og, host_tier):
+    """Partial pages must land head by head and leave every head's tail as it was;
+    a damaged block leaves everything as it was."""
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
+    T = og.page_tokens
+    src = random_cache(og, 13, seed=310)
+    lens = [2 * T + 1, 1, T - 1, 4 * T, 3 * T + T // 2, T + 2]
+    Nd = 31
+    jobs = _oracle_jobs(og, src, lens, 311, Nd)
+    jobs[4].blob[-3] ^= 0x20                 # damage inside the partial page of job 4
+    clean = random_cache(og, Nd, seed=312)
+    for tuning in ({}, {"seg_granules": 1, "commit_seg_tiles": 1}, {"fused": 0}):
+        ctx = _ctx(gk, og, **tuning)
+        want = clone_cache(clean)
+        wmask, wfb = oracle.restore(og, want, jobs)
+        assert wmask.tolist() == [0, 0, 0, 0, 1, 0]
+        d = dev_cache(clean)
+        mask, fb = gpu_restore(ctx, d, jobs, host_tier=host_tier)
+        assert mask.tolist() == wmask.tolist()
+        assert fb.tolist() == wfb.tolist()
+        assert_cache_equal(d, want)
+        ctx.close()
+
+
+def test_head_major_needs_16_byte_head_rows(gk):
+    with pytest.raises(gk.GkError) as e:
+        gk.gk_blob_size(gk.Geom(2, 4, 4, 16, gk.GK_BF16, 0, gk.GK_FLAG_HEAD_MAJOR), 16)   # 8 B per token and head
+    assert e.value.code == -2
+    assert gk.gk_blob_size(gk.Geom(2, 4, 4, 16, gk.GK_BF16, 0, 0), 16)[1] == 1            # fine token-major
+
+
+# ---------------------------------------------------------------------------
 # restore
 # ---------------------------------------------------------------------------
 def _oracle_jobs(og, src, lens, seed, dst_pages):
