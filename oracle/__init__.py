@@ -59,6 +59,9 @@ class _CJob(ctypes.Structure):
                 ("page_table", ctypes.c_void_p), ("n_tokens", ctypes.c_uint32)]
 
 
+_WINDOW_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32,
+                              ctypes.POINTER(ctypes.c_uint32))
+
 _lib = None
 
 
@@ -87,6 +90,10 @@ def lib() -> ctypes.CDLL:
         L.ok_restore.argtypes = [ctypes.POINTER(_CGeom), ctypes.POINTER(_CCache),
                                  ctypes.POINTER(_CJob), ctypes.c_uint32, ctypes.c_uint32,
                                  ctypes.c_void_p, ctypes.c_void_p]
+        L.ok_restore_stream.restype = ctypes.c_int
+        L.ok_restore_stream.argtypes = [ctypes.POINTER(_CGeom), ctypes.POINTER(_CCache),
+                                        ctypes.POINTER(_CJob), ctypes.c_uint32, ctypes.c_uint32,
+                                        ctypes.c_void_p, ctypes.c_void_p, _WINDOW_FN, ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -194,13 +201,12 @@ class Job:
     n_tokens: int
 
 
-def restore(g: Geom, dst: Cache, jobs: Sequence[Job], flags: int = 0):
-    """Mutates ``dst``; returns (mask uint8[n_jobs], first_bad int32[n_jobs])."""
+def _c_jobs(jobs: Sequence[Job], with_tables: bool = True):
     n = len(jobs)
     arr = (_CJob * max(n, 1))()
     keep = []
     for i, jb in enumerate(jobs):
-        pt = np.ascontiguousarray(jb.page_table, dtype=np.int32)
+        pt = np.ascontiguousarray(jb.page_table if with_tables else np.zeros(1), dtype=np.int32)
         keep.append(pt)
         bp = cp = 0
         if jb.blob is not None:
@@ -212,9 +218,39 @@ def restore(g: Geom, dst: Cache, jobs: Sequence[Job], flags: int = 0):
             keep.append(c)
             cp = c.ctypes.data
         arr[i] = _CJob(bp, cp, pt.ctypes.data, jb.n_tokens)
+    return arr, keep
+
+
+def restore(g: Geom, dst: Cache, jobs: Sequence[Job], flags: int = 0):
+    """Mutates ``dst``; returns (mask uint8[n_jobs], first_bad int32[n_jobs])."""
+    n = len(jobs)
+    arr, keep = _c_jobs(jobs)
     mask = np.zeros(n, dtype=np.uint8)
     first_bad = np.zeros(n, dtype=np.int32)
     cg, cc = g.c(), dst.c()
     lib().ok_restore(ctypes.byref(cg), ctypes.byref(cc), arr, n, flags,
                      mask.ctypes.data, first_bad.ctypes.data)
+    return mask, first_bad
+
+
+def restore_stream(g: Geom, ring: Cache, jobs: Sequence[Job], consume=None, flags: int = 0):
+    """Streams ``jobs`` (their page tables are ignored) through ``ring`` window by window.
+    ``consume(first_job, n_jobs, first_pages)`` runs after each window, while the window's
+    pages are still in ``ring``.  Returns (mask, first_bad), or raises ValueError if one job
+    alone does not fit the ring."""
+    n = len(jobs)
+    arr, keep = _c_jobs(jobs, with_tables=False)
+    mask = np.zeros(n, dtype=np.uint8)
+    first_bad = np.zeros(n, dtype=np.int32)
+
+    def _cb(_user, first_job, count, first_page):
+        if consume is not None:
+            consume(int(first_job), int(count), [int(first_page[i]) for i in range(count)])
+
+    cb = _WINDOW_FN(_cb)
+    cg, cc = g.c(), ring.c()
+    rc = lib().ok_restore_stream(ctypes.byref(cg), ctypes.byref(cc), arr, n, flags,
+                                 mask.ctypes.data, first_bad.ctypes.data, cb, None)
+    if rc != 0:
+        raise ValueError("a job has more pages than the ring")
     return mask, first_bad

@@ -280,3 +280,42 @@ void ok_restore(const ok_geom *g, const ok_cache *dst, const ok_job *jobs, uint3
     }
     free(claims);
 }
+
+/* ------------------------------------------------------------------------
+ * Streaming load: windows of consecutive jobs through one small cache.
+ * ---------------------------------------------------------------------- */
+int ok_restore_stream(const ok_geom *g, const ok_cache *ring, const ok_job *jobs, uint32_t n_jobs,
+                      uint32_t flags, uint8_t *mask, int32_t *first_bad, ok_window_fn consume, void *user)
+{
+    for (uint32_t j = 0; j < n_jobs; ++j)
+        if ((uint64_t)page_count(g, jobs[j].n_tokens) > ring->num_pages)
+            return -1;
+
+    int32_t *ids = (int32_t *)malloc((size_t)(ring->num_pages ? ring->num_pages : 1) * sizeof(int32_t));
+    for (uint64_t i = 0; i < ring->num_pages; ++i)
+        ids[i] = (int32_t)i;
+    ok_job *wjobs = (ok_job *)malloc((size_t)(n_jobs ? n_jobs : 1) * sizeof(ok_job));
+    uint32_t *first_page = (uint32_t *)malloc((size_t)(n_jobs ? n_jobs : 1) * sizeof(uint32_t));
+
+    uint32_t j0 = 0;
+    while (j0 < n_jobs) {
+        /* the longest run of jobs from j0 that fits */
+        uint64_t used = 0;
+        uint32_t j1 = j0;
+        while (j1 < n_jobs && used + page_count(g, jobs[j1].n_tokens) <= ring->num_pages) {
+            first_page[j1 - j0] = (uint32_t)used;
+            wjobs[j1 - j0] = jobs[j1];
+            wjobs[j1 - j0].page_table = ids + used;
+            used += page_count(g, jobs[j1].n_tokens);
+            ++j1;
+        }
+        ok_restore(g, ring, wjobs, j1 - j0, flags, mask + j0, first_bad + j0);
+        if (consume)
+            consume(user, j0, j1 - j0, first_page);
+        j0 = j1;
+    }
+    free(first_page);
+    free(wjobs);
+    free(ids);
+    return 0;
+}

@@ -107,6 +107,22 @@ int ok_pack(const ok_geom *g, const ok_cache *src, const int32_t *page_table,
 void ok_restore(const ok_geom *g, const ok_cache *dst, const ok_job *jobs, uint32_t n_jobs,
                 uint32_t flags, uint8_t *mask, int32_t *first_bad);
 
+/* Streaming load through a cache that is smaller than the corpus (Section 4.3,
+ * the long-window paragraph: saved blocks are streamed in and dropped after
+ * use, so that the size of the corpus is bounded by storage, not GPU memory).
+ * The jobs' own page tables are ignored.  Jobs are taken in order and grouped
+ * into windows: a window is the longest run of consecutive jobs whose pages fit
+ * the cache together; inside a window the jobs get consecutive page ids from 0
+ * (every job takes ceil(n_tokens/page_tokens) pages, whatever its result).  Each
+ * window is one ok_restore; after it `consume` (may be NULL) is called with the
+ * index of the window's first job, its job count, and each job's first page id;
+ * then the pages are reused by the next window.  mask and first_bad cover all
+ * jobs.  Returns 0, or -1 (nothing done) if a single job has more pages than
+ * the cache. */
+typedef void (*ok_window_fn)(void *user, uint32_t first_job, uint32_t n_jobs, const uint32_t *first_page);
+int ok_restore_stream(const ok_geom *g, const ok_cache *ring, const ok_job *jobs, uint32_t n_jobs,
+                      uint32_t flags, uint8_t *mask, int32_t *first_bad, ok_window_fn consume, void *user);
+
 #ifdef __cplusplus
 }
 #endif

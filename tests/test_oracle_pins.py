@@ -472,3 +472,93 @@ def test_one_failed_job_does_not_stop_the_others():
             assert np.array_equal(d[:, :, pages], s[:, :, 16 * i:16 * i + 16])
     rest = perm[64:]
     assert np.array_equal(d[:, :, rest], c[:, :, rest])
+
+
+# --------------------------------------------------------------------------
+# streaming restore through a ring of pages (Section 4.3, long windows at flat memory)
+# --------------------------------------------------------------------------
+def _valid_prefix(g, cache, page, t):
+    """Valid bytes (first t tokens, token-major) of every slab of a page, plus its scales."""
+    L, H, D, T, E = g.layers, g.kv_heads, g.head_dim, g.page_tokens, g.elem_bytes
+    arr = cache.data.reshape(L, 2, cache.num_pages, T, H * D * E)
+    out = [arr[:, :, page, :t].reshape(-1)]
+    if cache.scales is not None:
+        out.append(cache.scales.reshape(L, g.scale_kv, cache.num_pages, H * 4)[:, :, page].reshape(-1))
+    return np.concatenate(out)
+
+
+@pytest.mark.parametrize("g", [oracle.Geom(3, 2, 8, 4, 2, 0), oracle.Geom(2, 4, 16, 8, 1, 2)])
+@pytest.mark.parametrize("ring_pages", [5, 8, 64])
+def test_stream_restore_windows_contents_and_fail_closed(g, ring_pages):
+    T = g.page_tokens
+    src = random_cache(g, 11, seed=70)
+    rng = np.random.default_rng(71)
+    lens = [2 * T, 1, 3 * T + 1, T, 5 * T, 2 * T - 1, T + 1, 4 * T, 1, 3 * T]
+    tables = [rng.integers(0, 11, size=n_pages(g, n)).astype(np.int32) for n in lens]
+    jobs = []
+    for pt, n in zip(tables, lens):
+        blob, sums, code, _ = oracle.pack(g, src, pt, n)
+        assert code == 0
+        jobs.append(oracle.Job(blob, sums, None, n))
+    jobs[3].blob[0] ^= 0x80                       # damaged
+    jobs[6] = oracle.Job(None, None, None, lens[6])  # missing
+    ring = random_cache(g, ring_pages, seed=72)
+    seen = []
+    state = {"before": clone_cache(ring), "next_job": 0}
+
+    def consume(first_job, count, first_pages):
+        # windows arrive in order, are contiguous, and are maximal
+        assert first_job == state["next_job"] and count >= 1
+        pages = [n_pages(g, lens[first_job + k]) for k in range(count)]
+        assert first_pages == [sum(pages[:k]) for k in range(count)]
+        assert sum(pages) <= ring_pages
+        nxt = first_job + count
+        if nxt < len(lens):
+            assert sum(pages) + n_pages(g, lens[nxt]) > ring_pages
+        # contents: a good job's pages hold the saved bytes; every other byte of the ring
+        # (bad jobs' pages, tails of partial pages, pages beyond the window) is as it was
+        expect = clone_cache(state["before"])
+        for k in range(count):
+            j = first_job + k
+            if j in (3, 6):
+                continue
+            for p in range(pages[k]):
+                t = min(T, lens[j] - p * T)
+                assert np.array_equal(_valid_prefix(g, ring, first_pages[k] + p, t),
+                                      _valid_prefix(g, src, tables[j][p], t))
+                # graft the saved bytes into the expectation through numpy views
+                L, H, D, E = g.layers, g.kv_heads, g.head_dim, g.elem_bytes
+                ev = expect.data.reshape(L, 2, ring_pages, T, H * D * E)
+                sv = src.data.reshape(L, 2, 11, T, H * D * E)
+                ev[:, :, first_pages[k] + p, :t] = sv[:, :, tables[j][p], :t]
+                if g.scale_kv:
+                    es = expect.scales.reshape(L, g.scale_kv, ring_pages, H * 4)
+                    ss = src.scales.reshape(L, g.scale_kv, 11, H * 4)
+                    es[:, :, first_pages[k] + p] = ss[:, :, tables[j][p]]
+        assert np.array_equal(ring.data, expect.data)
+        if g.scale_kv:
+            assert np.array_equal(ring.scales, expect.scales)
+        state["before"] = clone_cache(ring)
+        state["next_job"] = nxt
+        seen.append((first_job, count))
+
+    mask, fb = oracle.restore_stream(g, ring, jobs, consume)
+    assert state["next_job"] == len(lens)
+    assert mask.tolist() == [0, 0, 0, 1, 0, 0, 3, 0, 0, 0]
+    assert fb.tolist() == [-1, -1, -1, 0, -1, -1, -1, -1, -1, -1]
+    if ring_pages == 64:
+        assert seen == [(0, len(lens))]            # everything fits: one window
+    if ring_pages == 5:
+        assert (4, 1) in seen                      # the 5-page job fills a window alone
+
+
+def test_stream_restore_refuses_a_job_larger_than_the_ring():
+    g = oracle.Geom(3, 2, 8, 4, 2, 0)
+    src = random_cache(g, 6, seed=73)
+    blob, sums, _, _ = oracle.pack(g, src, np.arange(6, dtype=np.int32), 6 * g.page_tokens)
+    small, _s, _, _ = oracle.pack(g, src, np.arange(1, dtype=np.int32), 1)
+    ring = random_cache(g, 5, seed=74)
+    before = clone_cache(ring)
+    with pytest.raises(ValueError):
+        oracle.restore_stream(g, ring, [oracle.Job(small, _s, None, 1), oracle.Job(blob, sums, None, 6 * g.page_tokens)])
+    assert np.array_equal(ring.data, before.data)   # not even the first job was restored
