@@ -49,9 +49,11 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress"],
+    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress", "longwindow"],
                     help="gqa7b is the headline workload (full JSON line); the others print a shorter line "
                          "with the save and restore phases of that workload's shape")
+    ap.add_argument("--window-blocks", type=int, default=48,
+                    help="longwindow: blocks streamed per step (30,000 tokens each, through a 2-block ring)")
     ap.add_argument("--blocks", type=int, default=0,
                     help="restore this many blocks instead of the workload's 16 (small cases for profiling)")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -655,6 +657,86 @@ def run_other_workload(args):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------
+# long window at flat GPU memory: a corpus far larger than the cache streamed
+# from pinned host memory through a ring of pages (gk_restore_stream)
+# ---------------------------------------------------------------------------
+def run_longwindow(args):
+    import torch
+    import synth
+    import paper_2609_39358_b200 as gk
+
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    w = synth.GQA7B
+    block_tokens, pool_blocks, ring_blocks = 30000, 4, 2
+    geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, gk.GK_BF16, 0)
+    ctx = gk.Context(geom, device.index)
+    slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
+    P = -(-block_tokens // w.page_tokens)
+    nb, _ = gk.gk_blob_size(geom, block_tokens)
+
+    def cache(num_pages, seed):
+        data = synth.kv_bytes_bf16(2 * w.layers * num_pages * slab // 2, w.sigma, seed, device)
+        return gk.Cache(data, num_pages, 2 * num_pages * slab, num_pages * slab, slab)
+
+    # the saved corpus: pool_blocks distinct blobs in pinned host memory, visited round-robin
+    pool = []
+    ident = torch.arange(P, dtype=torch.int32, device=device)
+    for k in range(pool_blocks):
+        src = cache(P, w.seed(700 + k))
+        hb = torch.empty(nb, dtype=torch.uint8, pin_memory=True)
+        hs = torch.zeros(P, dtype=torch.int64, pin_memory=True)
+        ctx.gk_pack_host(src, [gk.Job(hb, hs, ident, block_tokens)])
+        torch.cuda.synchronize(device)
+        pool.append((hb, hs))
+        del src
+    torch.cuda.empty_cache()
+    ring = cache(ring_blocks * P, w.seed(710))
+    n_jobs = args.window_blocks
+    jobs = [gk.Job(pool[j % pool_blocks][0], pool[j % pool_blocks][1], None, block_tokens) for j in range(n_jobs)]
+    mask = torch.zeros(n_jobs, dtype=torch.uint8, device=device)
+    fb = torch.zeros(n_jobs, dtype=torch.int32, device=device)
+    touched = torch.zeros(1, dtype=torch.int64, device=device)
+    windows = []
+
+    def consume(blocks, st):
+        # stand-in for the reader of the window: one cheap stream-ordered pass over part of the ring
+        windows.append(len(blocks))
+        touched.add_(ring.data[:1 << 20].sum())
+
+    stream = torch.cuda.current_stream(device)
+    steps, warmup = max(1, min(args.steps, 3)), 1
+    for _ in range(warmup):
+        ctx.gk_restore_stream(jobs, ring, mask, fb, consume)
+    torch.cuda.synchronize(device)
+    free_before, total_mem = torch.cuda.mem_get_info(device)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    windows.clear()
+    ev[0].record(stream)
+    for _ in range(steps):
+        ctx.gk_restore_stream(jobs, ring, mask, fb, consume)
+    ev[1].record(stream)
+    torch.cuda.synchronize(device)
+    free_after, _ = torch.cuda.mem_get_info(device)
+    assert int(mask.sum().item()) == 0
+    ms = ev[0].elapsed_time(ev[1]) / steps
+    total = n_jobs * nb
+    line = {"metric": "streamed restore from pinned host memory, blob GB/s", "value": total / (ms * 1e-3) / 1e9,
+            "unit": UNIT, "n_gpus": 1, "steps": steps, "warmup": warmup, "ms_per_step": ms, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": f"longwindow: gqa7b geometry, {n_jobs} blocks x {block_tokens} tokens "
+                                   f"({n_jobs * block_tokens / 1e6:.2f} M tokens, {total / 2**30:.1f} GiB of blobs, "
+                                   f"{pool_blocks} distinct blobs visited round-robin) through a ring of "
+                                   f"{ring_blocks} blocks ({ring_blocks * P} pages)",
+                       "step": "one gk_restore_stream call; the consumer touches the ring after every window"},
+            "tokens_per_s": n_jobs * block_tokens / (ms * 1e-3),
+            "windows_per_step": len(windows) // steps,
+            "device_memory": {"used_bytes": total_mem - free_after, "growth_during_timed_steps": free_before - free_after,
+                              "ring_bytes": ring.data.numel(), "total_bytes": total_mem}}
+    print(json.dumps(line), flush=True)
+
+
 def synth_requests(n_blocks):
     return f"{max(n_blocks // 2, 1)} requests x {min(n_blocks, 2)} blocks"
 
@@ -663,6 +745,8 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.workload == "longwindow":
+        run_longwindow(args)
     elif args.workload != "gqa7b":
         run_other_workload(args)
     else:

@@ -132,6 +132,7 @@ typedef struct {
                                          from then on no call of this context commits anything and
                                          the destination of the call that hit it is undefined */
     uint32_t reserved;
+    uint64_t calls_restore_stream;    /* its windows are counted in calls_restore_host as well */
 } gk_stats;
 
 /* Sizes of a block of n_tokens (Section 2.2: one record per block).  Either output may be NULL. */
@@ -216,6 +217,38 @@ int gk_commit(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *
  * `stream` has been synchronised.  The host buffers must stay valid until then. */
 int gk_restore_host(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
                     uint8_t *mask_dev, int32_t *first_bad_page_dev, void *stream);
+
+/* Streaming load of a corpus that is larger than the cache (Section 4.3,
+ * long-window paragraph: blocks are streamed in, used and dropped, so that GPU
+ * memory stays flat while the corpus grows).  `ring` is a small cache whose pages
+ * are handed out by this call; the jobs' own page_table fields are ignored.  Jobs
+ * are taken in order and grouped into windows: a window is the longest run of
+ * consecutive jobs whose pages fit `ring` together, and inside a window the jobs
+ * get consecutive page ids from 0 (every job takes ceil(n_tokens/page_tokens)
+ * pages, whatever its result).  Each window is loaded as by gk_restore_host
+ * (blobs and checksums in PINNED host memory; verify, then commit, fail-closed per
+ * job); then `consume` (may be NULL) is called ON THE HOST with the window's
+ * blocks, and the next window reuses the pages.  Everything is ordered on
+ * `stream`: the callback must only enqueue its work on `stream` (it may also
+ * synchronise it); it must not call into this context.  While the consumer's
+ * work runs, the copies of the next window are already in flight.
+ * `blocks[i].page_table` is device memory owned by the context, valid until the
+ * next call on the context; mask_dev / first_bad_page_dev (device, n_jobs
+ * entries) cover the whole call and are indexed by blocks[i].job.
+ * Returns GK_ERR_TOO_LARGE, having done nothing, if one job alone has more pages
+ * than `ring`.  Device memory held: the ring, two staging slots (each the size of
+ * the largest blob, or up to 256 MiB of smaller ones) and a workspace of a few
+ * bytes per page of a window. */
+typedef struct {
+    uint32_t job;              /* index into the call's job array */
+    uint32_t n_tokens;
+    const int32_t *page_table; /* device: ids of the ring pages that hold the block */
+} gk_window_block;
+typedef void (*gk_window_fn)(void *user, const gk_window_block *blocks, uint32_t n_blocks,
+                             const uint8_t *mask_dev, void *stream);
+int gk_restore_stream(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *ring,
+                      uint8_t *mask_dev, int32_t *first_bad_page_dev, gk_window_fn consume, void *user,
+                      void *stream);
 
 /* Counters of this context.  Reads the device error word with a blocking copy. */
 int gk_get_stats(gk_ctx *ctx, gk_stats *out);

@@ -11,7 +11,7 @@ from __future__ import annotations
 import ctypes
 import os
 from dataclasses import dataclass
-from typing import Optional, Sequence
+from typing import Callable, Optional, Sequence
 
 import torch
 
@@ -26,7 +26,7 @@ JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
 
 EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",
            "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times",
-           "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit"]
+           "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit", "gk_restore_stream"]
 
 
 class GkError(RuntimeError):
@@ -57,7 +57,24 @@ class CStats(ctypes.Structure):
     _fields_ = [("calls_pack", ctypes.c_uint64), ("calls_restore", ctypes.c_uint64),
                 ("calls_restore_host", ctypes.c_uint64), ("jobs", ctypes.c_uint64), ("pages", ctypes.c_uint64),
                 ("bytes_blob", ctypes.c_uint64), ("kernels_launched", ctypes.c_uint64),
-                ("device_wait_expired", ctypes.c_uint32), ("reserved", ctypes.c_uint32)]
+                ("device_wait_expired", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("calls_restore_stream", ctypes.c_uint64)]
+
+
+class CWindowBlock(ctypes.Structure):
+    _fields_ = [("job", ctypes.c_uint32), ("n_tokens", ctypes.c_uint32), ("page_table", ctypes.c_void_p)]
+
+
+WINDOW_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.POINTER(CWindowBlock), ctypes.c_uint32, ctypes.c_void_p,
+                             ctypes.c_void_p)
+
+
+@dataclass(frozen=True)
+class WindowBlock:
+    """One block of a streaming-restore window, as handed to the consumer."""
+    job: int          # index into the call's job list
+    n_tokens: int
+    page_table: int   # device address of the block's int32 ring page ids
 
 
 _lib = None
@@ -102,6 +119,8 @@ def load_library() -> ctypes.CDLL:
     L.gk_commit.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp]
     L.gk_restore_host.restype = ctypes.c_int
     L.gk_restore_host.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
+    L.gk_restore_stream.restype = ctypes.c_int
+    L.gk_restore_stream.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, WINDOW_FN, vp, vp]
     L.gk_get_stats.restype = ctypes.c_int
     L.gk_get_stats.argtypes = [vp, ctypes.POINTER(CStats)]
     L.gk_get_kernel_times.restype = ctypes.c_int
@@ -157,8 +176,11 @@ class Job:
     request_id: int = 0
 
 
-def _ptr(t: Optional[torch.Tensor]) -> int:
-    return 0 if t is None else t.data_ptr()
+def _ptr(t) -> int:
+    """Address of a tensor's storage; an int is taken as a raw address, None as NULL."""
+    if t is None:
+        return 0
+    return t if isinstance(t, int) else t.data_ptr()
 
 
 def _stream_handle(stream) -> int:
@@ -275,6 +297,30 @@ class Context:
         cc = dst.c()
         self._check(self._lib.gk_restore_host(self._h, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask),
                                               _ptr(first_bad_page), _stream_handle(stream)), "gk_restore_host")
+
+    def gk_restore_stream(self, jobs: Sequence[Job], ring: Cache, mask: torch.Tensor, first_bad_page: torch.Tensor,
+                          consume: Optional[Callable] = None, stream=None):
+        """``consume(blocks: list[WindowBlock], stream_handle: int)`` runs on the host after each window has
+        been enqueued; it may only enqueue work on that stream.  An exception it raises is re-raised here
+        after the call has returned (the remaining windows still run)."""
+        cc = ring.c()
+        raised = []
+
+        def _cb(_user, blocks, n, _mask, st):
+            if consume is None:
+                return
+            try:
+                consume([WindowBlock(blocks[i].job, blocks[i].n_tokens, blocks[i].page_table or 0) for i in range(n)],
+                        st or 0)
+            except BaseException as e:  # must not unwind through the C frames
+                raised.append(e)
+
+        cb = WINDOW_FN(_cb)
+        rc = self._lib.gk_restore_stream(self._h, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask),
+                                         _ptr(first_bad_page), cb, None, _stream_handle(stream))
+        if raised:
+            raise raised[0]
+        self._check(rc, "gk_restore_stream")
 
     def gk_get_kernel_times(self) -> dict:
         """{'verify'|'pack'|'commit'|'restore': (ms, launches)} since the previous call (needs tuning key profile=1)."""

@@ -124,6 +124,11 @@ struct gk_ctx {
     cudaEvent_t ev_slot_free[kSlots] = {nullptr, nullptr};
     cudaEvent_t ev_copied[kSlots] = {nullptr, nullptr};
     bool slot_used[kSlots] = {false, false};
+    uint32_t slot_next = 0;  // the slot the next batch goes to (carried across calls)
+
+    // streaming restore: the ids 0..iota_cap-1, from which window page tables are cut
+    int32_t *d_iota = nullptr;
+    uint64_t iota_cap = 0;
 
     // optional per-kernel timing (tuning key "profile")
     bool profile = false;
@@ -623,6 +628,7 @@ int make_host_plan(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, bool allow_mi
             c->slot_used[i] = false;
         }
         c->slot_cap = 0;
+        c->slot_next = 0;
         for (int i = 0; i < kSlots; ++i) {
             if (cudaMalloc(&c->d_slot[i], want) != cudaSuccess) {
                 cudaGetLastError();
@@ -643,7 +649,7 @@ int make_host_plan(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, bool allow_mi
             used = 0;
         }
         if (plan[j].need) {
-            uint8_t *base = c->d_slot[b % kSlots] + used;
+            uint8_t *base = c->d_slot[(c->slot_next + b) % kSlots] + used;
             hp.blob_dev[j] = base;
             hp.sums_dev[j] = (uint64_t *)(base + align_up(plan[j].blob_bytes, 256));
             used += plan[j].need;
@@ -771,6 +777,7 @@ int gk_ctx_destroy(gk_ctx *c)
     if (c->ev_stage) cudaEventDestroy(c->ev_stage);
     if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->d_ws) cudaFree(c->d_ws);
+    if (c->d_iota) cudaFree(c->d_iota);
     if (c->d_init_term) cudaFree(c->d_init_term);
     if (c->d_thread_const) cudaFree(c->d_thread_const);
     if (c->d_error) cudaFree(c->d_error);
@@ -1072,7 +1079,7 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
 
     uint32_t j0 = 0, page0 = 0;
     for (size_t b = 0; b < batch_end.size(); ++b) {
-        const int slot = (int)(b % kSlots);
+        const int slot = (int)((c->slot_next + b) % kSlots);
         const uint32_t j1 = batch_end[b];
         if (c->slot_used[slot]) GK_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_slot_free[slot], 0));
         uint32_t npages = 0;
@@ -1093,10 +1100,70 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
         j0 = j1;
         page0 += npages;
     }
+    c->slot_next = (uint32_t)((c->slot_next + batch_end.size()) % kSlots);
     c->stats.calls_restore_host++;
     c->stats.jobs += n_jobs;
     c->stats.pages += pages;
     c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+int gk_restore_stream(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *ring, uint8_t *mask_dev,
+                      int32_t *first_bad_page_dev, gk_window_fn consume, void *user, void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0) return GK_OK;
+    if (!jobs || !mask_dev || !first_bad_page_dev) return fail(c, GK_ERR_ARG, "null jobs, mask or first_bad_page");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    CacheDev cd;
+    int rc = check_cache(c, ring, &cd);
+    if (rc != GK_OK) return rc;
+    std::vector<uint32_t> np(n_jobs);
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
+        np[j] = pages_of(jobs[j].n_tokens, c->gd.page_tokens);
+        if ((uint64_t)np[j] > cd.num_pages)
+            return fail(c, GK_ERR_TOO_LARGE, "job %u: %u pages do not fit a ring of %llu", j, np[j],
+                        (unsigned long long)cd.num_pages);
+    }
+    // the page ids 0..num_pages-1 on the device; a window's tables are slices of them
+    if (c->iota_cap < cd.num_pages) {
+        GK_CUDA(c, cudaDeviceSynchronize());  // an earlier call's consumer may still read the old array
+        if (c->d_iota) cudaFree(c->d_iota);
+        c->d_iota = nullptr;
+        c->iota_cap = 0;
+        if (cudaMalloc(&c->d_iota, cd.num_pages * sizeof(int32_t)) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(c, GK_ERR_NOMEM, "page id array of %llu entries", (unsigned long long)cd.num_pages);
+        }
+        c->iota_cap = cd.num_pages;
+        iota_kernel<<<(unsigned)((cd.num_pages + 255) / 256), 256, 0, st>>>(c->d_iota, (uint32_t)cd.num_pages);
+        GK_CUDA(c, cudaGetLastError());
+        c->stats.kernels_launched++;
+    }
+    std::vector<gk_job> wjobs;
+    std::vector<gk_window_block> blocks;
+    uint32_t j0 = 0;
+    while (j0 < n_jobs) {
+        uint64_t used = 0;
+        uint32_t j1 = j0;
+        wjobs.clear();
+        blocks.clear();
+        while (j1 < n_jobs && used + np[j1] <= cd.num_pages) {
+            gk_job w = jobs[j1];
+            w.page_table = c->d_iota + used;
+            wjobs.push_back(w);
+            blocks.push_back(gk_window_block{j1, jobs[j1].n_tokens, c->d_iota + used});
+            used += np[j1];
+            ++j1;
+        }
+        rc = gk_restore_host(c, wjobs.data(), j1 - j0, ring, mask_dev + j0, first_bad_page_dev + j0, stream);
+        if (rc != GK_OK) return rc;
+        if (consume) consume(user, blocks.data(), j1 - j0, mask_dev, stream);
+        j0 = j1;
+    }
+    c->stats.calls_restore_stream++;
     return GK_OK;
 }
 
@@ -1126,7 +1193,7 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
     uint32_t j0 = 0, page0 = 0;
     int last_slot[kSlots] = {0, 0};
     for (size_t b = 0; b < hp.batch_end.size(); ++b) {
-        const int slot = (int)(b % kSlots);
+        const int slot = (int)((c->slot_next + b) % kSlots);
         const uint32_t j1 = hp.batch_end[b];
         // the slot's previous contents must have left (earlier D2H, or an earlier restore reading it)
         if (c->slot_used[slot]) GK_CUDA(c, cudaStreamWaitEvent(st, c->ev_slot_free[slot], 0));
@@ -1160,6 +1227,7 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
     // the caller's stream is complete only when the last copies have landed
     for (int i = 0; i < kSlots; ++i)
         if (last_slot[i]) GK_CUDA(c, cudaStreamWaitEvent(st, c->ev_slot_free[i], 0));
+    c->slot_next = (uint32_t)((c->slot_next + hp.batch_end.size()) % kSlots);
     c->stats.calls_pack++;
     c->stats.jobs += n_jobs;
     c->stats.pages += pages;

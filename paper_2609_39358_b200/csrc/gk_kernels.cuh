@@ -36,6 +36,13 @@ namespace gk {
 // ---------------------------------------------------------------------------
 // small kernels
 // ---------------------------------------------------------------------------
+// ids[i] = i: the page ids from which the streaming restore cuts its window page tables
+__global__ void iota_kernel(int32_t *ids, uint32_t n)
+{
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) ids[i] = (int32_t)i;
+}
+
 // One CTA per job.  Initialises the job's result words, records the lowest
 // out-of-range page id and fills page_job.  All CTAs together clear the claim
 // words of the destination cache.

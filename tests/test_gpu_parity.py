@@ -289,6 +289,140 @@ def test_restore_parity_with_corruption(gk, og, host_tier):
         ctx.close()
 
 
+# ---------------------------------------------------------------------------
+# streaming restore through a ring of pages
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("og", [G_MID, G_FP8_M, HM_MID])
+@pytest.mark.parametrize("ring_pages", [6, 9, 64])
+def test_stream_restore_parity(gk, og, ring_pages):
+    """Window by window: same windows, same ring image after every window, same codes.
+    The consumer also packs every block back out of the ring through the page table it
+    was handed, which must give the saved blob again."""
+    from gpu_harness import dev_cache, sums_to_np
+    T = og.page_tokens
+    src = random_cache(og, 17, seed=320)
+    rng = np.random.default_rng(321)
+    lens = [2 * T, 1, 3 * T + 1, T, 6 * T, 2 * T - 1, T + 1, 4 * T, 1, 3 * T, 5 * T + 2]
+    ojobs = []
+    for n in lens:
+        spt = rng.integers(0, src.num_pages, size=n_pages(og, n)).astype(np.int32)
+        blob, sums, code, _ = oracle.pack(og, src, spt, n)
+        assert code == 0
+        ojobs.append(oracle.Job(blob, sums, None, n))
+    pristine = [jb.blob.copy() for jb in ojobs]
+    ojobs[3].blob[7] ^= 0x04
+    ojobs[7].checksums[1] ^= np.uint64(2)
+    ojobs[8] = oracle.Job(None, None, None, lens[8])
+    bad = {3, 7, 8}
+    clean = random_cache(og, ring_pages, seed=322)
+
+    want_ring = clone_cache(clean)
+    owin = []
+
+    def oconsume(first, count, first_pages):
+        owin.append((first, count, first_pages, want_ring.data.copy(),
+                     None if want_ring.scales is None else want_ring.scales.copy()))
+
+    wmask, wfb = oracle.restore_stream(og, want_ring, ojobs, oconsume)
+    assert [int(m) for m in wmask] == [1 if j in (3, 7) else 3 if j == 8 else 0 for j in range(len(lens))]
+
+    ctx, ctx2 = _ctx(gk, og), _ctx(gk, og)
+    d = dev_cache(clean)
+    jobs, keep = [], []
+    for jb in ojobs:
+        hb = None if jb.blob is None else torch.from_numpy(jb.blob).pin_memory()
+        hs = None if jb.checksums is None else torch.from_numpy(jb.checksums.view(np.int64).copy()).pin_memory()
+        keep.append((hb, hs))
+        jobs.append(gk.Job(hb, hs, None, jb.n_tokens))
+    mask = torch.full((len(jobs),), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.full((len(jobs),), -7, dtype=torch.int32, device="cuda")
+    gwin = []
+
+    def consume(blocks, st):
+        assert st == torch.cuda.current_stream().cuda_stream
+        packed = []
+        for b in blocks:
+            nbytes, P = oracle.blob_size(og, b.n_tokens)
+            ob = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+            os_ = torch.zeros(P, dtype=torch.int64, device="cuda")
+            ctx2.gk_pack_batch(d, [gk.Job(ob, os_, b.page_table, b.n_tokens)])
+            packed.append((b.job, ob, os_))
+        gwin.append(([b.job for b in blocks], [b.page_table for b in blocks], d.data.clone(),
+                     None if d.scales is None else d.scales.clone(), packed))
+
+    ctx.gk_restore_stream(jobs, d, mask, fb, consume)
+    torch.cuda.synchronize()
+    assert ctx.gk_get_stats()["device_wait_expired"] == 0
+    assert mask.cpu().tolist() == wmask.tolist()
+    assert fb.cpu().tolist() == wfb.tolist()
+    assert len(gwin) == len(owin)
+    for (first, count, first_pages, odata, oscales), (gjobs, gtables, gdata, gscales, packed) in zip(owin, gwin):
+        assert gjobs == list(range(first, first + count))
+        assert [(a - gtables[0]) // 4 for a in gtables] == first_pages
+        assert np.array_equal(gdata.cpu().numpy(), odata)
+        if oscales is not None:
+            assert np.array_equal(gscales.cpu().numpy(), oscales)
+        for j, ob, os_ in packed:
+            if j in bad:
+                continue
+            assert np.array_equal(ob.cpu().numpy(), pristine[j])
+            assert np.array_equal(sums_to_np(os_), ojobs[j].checksums)
+    if ring_pages == 64:
+        assert len(gwin) == 1
+    ctx.close()
+    ctx2.close()
+
+
+def test_stream_restore_on_a_side_stream_and_refusals(gk):
+    from gpu_harness import assert_cache_equal, dev_cache
+    og = G_MID
+    T = og.page_tokens
+    src = random_cache(og, 9, seed=330)
+    lens = [3 * T, 2 * T + 1, 4 * T, T]
+    ojobs = []
+    for i, n in enumerate(lens):
+        blob, sums, code, _ = oracle.pack(og, src, np.arange(n_pages(og, n), dtype=np.int32) + i, n)
+        ojobs.append(oracle.Job(blob, sums, None, n))
+    clean = random_cache(og, 5, seed=331)
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore_stream(og, want, ojobs)
+    ctx = _ctx(gk, og)
+    d = dev_cache(clean)
+    keep = [(torch.from_numpy(j.blob).pin_memory(), torch.from_numpy(j.checksums.view(np.int64).copy()).pin_memory())
+            for j in ojobs]
+    jobs = [gk.Job(b, s, None, j.n_tokens) for (b, s), j in zip(keep, ojobs)]
+    mask = torch.full((4,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.full((4,), -7, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    seen = []
+    with torch.cuda.stream(side):
+        ctx.gk_restore_stream(jobs, d, mask, fb, lambda blocks, st: seen.append((len(blocks), st)))
+    side.synchronize()
+    h = side.cuda_stream
+    assert seen == [(1, h), (1, h), (2, h)]            # pages 3 | 3 | 4 + 1 through a 5-page ring
+    assert mask.cpu().tolist() == wmask.tolist() == [0, 0, 0, 0]
+    assert_cache_equal(d, want)                        # the final image: what the last window left
+    assert ctx.gk_get_stats()["calls_restore_stream"] == 1
+
+    # a job that alone does not fit: refused before anything runs
+    d2 = dev_cache(clean)
+    big, bs, _, _ = oracle.pack(og, src, np.arange(6, dtype=np.int32), 6 * T)
+    hb, hs = torch.from_numpy(big).pin_memory(), torch.from_numpy(bs.view(np.int64).copy()).pin_memory()
+    with pytest.raises(gk.GkError) as e:
+        ctx.gk_restore_stream([jobs[0], gk.Job(hb, hs, None, 6 * T)], d2, mask, fb)
+    assert e.value.code == -7
+    torch.cuda.synchronize()
+    assert_cache_equal(d2, clean)
+    # an exception in the consumer surfaces after the call
+    def boom(blocks, st):
+        raise KeyError("consumer failed")
+    with pytest.raises(KeyError):
+        ctx.gk_restore_stream(jobs[:1], d2, mask, fb, boom)
+    torch.cuda.synchronize()
+    ctx.close()
+
+
 def test_restore_codes_and_first_bad_page(gk):
     from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
     og, N = G_MID, 12
