@@ -20,8 +20,8 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libgk_oracle.so")
-_SRC = os.path.join(_HERE, "gk_oracle.c")
-_HDR = os.path.join(_HERE, "gk_oracle.h")
+_SRCS = [os.path.join(_HERE, "gk_oracle.c"), os.path.join(_HERE, "gk_sha256_oracle.c")]
+_HDRS = [os.path.join(_HERE, "gk_oracle.h"), os.path.join(_HERE, "gk_sha256_oracle.h")]
 
 CODE_OK, CODE_CHECKSUM, CODE_PAGE_TABLE, CODE_MISSING = 0, 1, 2, 3
 FLAG_SKIP_VERIFY = 1
@@ -30,11 +30,11 @@ FLAG_SKIP_VERIFY = 1
 def build(force: bool = False) -> str:
     """Compile the oracle with gcc if the shared object is missing or stale."""
     stale = (not os.path.exists(_LIB_PATH)
-             or os.path.getmtime(_LIB_PATH) < max(os.path.getmtime(_SRC), os.path.getmtime(_HDR)))
+             or os.path.getmtime(_LIB_PATH) < max(os.path.getmtime(f) for f in _SRCS + _HDRS))
     if force or stale:
         tmp = _LIB_PATH + f".tmp{os.getpid()}"
         subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-fPIC", "-shared",
-                               "-o", tmp, _SRC])
+                               "-o", tmp] + _SRCS)
         os.replace(tmp, _LIB_PATH)
     return _LIB_PATH
 
@@ -94,6 +94,16 @@ def lib() -> ctypes.CDLL:
         L.ok_restore_stream.argtypes = [ctypes.POINTER(_CGeom), ctypes.POINTER(_CCache),
                                         ctypes.POINTER(_CJob), ctypes.c_uint32, ctypes.c_uint32,
                                         ctypes.c_void_p, ctypes.c_void_p, _WINDOW_FN, ctypes.c_void_p]
+        L.ok_sha256.restype = None
+        L.ok_sha256.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
+        L.ok_sha256_constants.restype = None
+        L.ok_sha256_constants.argtypes = [ctypes.c_void_p, ctypes.c_void_p]
+        L.ok_fingerprints.restype = ctypes.c_int
+        L.ok_fingerprints.argtypes = [ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p,
+                                      ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        L.ok_blob_digest.restype = None
+        L.ok_blob_digest.argtypes = [ctypes.POINTER(_CGeom), ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p,
+                                     ctypes.c_void_p, ctypes.c_void_p]
         _lib = L
     return _lib
 
@@ -254,3 +264,55 @@ def restore_stream(g: Geom, ring: Cache, jobs: Sequence[Job], consume=None, flag
     if rc != 0:
         raise ValueError("a job has more pages than the ring")
     return mask, first_bad
+
+
+# ---------------------------------------------------------------------------
+# fingerprints and blob digests (gk_sha256_oracle.c)
+# ---------------------------------------------------------------------------
+DIGEST_CHUNK = 4096
+
+
+def sha256(data) -> bytes:
+    a = _as_u8(data)
+    out = np.zeros(32, dtype=np.uint8)
+    lib().ok_sha256(a.ctypes.data if a.size else None, a.size, out.ctypes.data)
+    return out.tobytes()
+
+
+def sha256_constants():
+    k = np.zeros(64, dtype=np.uint32)
+    h0 = np.zeros(8, dtype=np.uint32)
+    lib().ok_sha256_constants(k.ctypes.data, h0.ctypes.data)
+    return k, h0
+
+
+def fingerprints(data, offsets, parent, model: bytes, tenant: bytes) -> np.ndarray:
+    """Keys (uint8[n, 32]) of the messages data[offsets[i]:offsets[i+1]]; parent may be None."""
+    d = _as_u8(data)
+    off = np.ascontiguousarray(offsets, dtype=np.uint64)
+    n = off.size - 1
+    par = None if parent is None else np.ascontiguousarray(parent, dtype=np.int32)
+    m, t = _as_u8(model), _as_u8(tenant)
+    assert m.size == 32 and t.size == 32 and (par is None or par.size == n)
+    keys = np.zeros((max(n, 1), 32), dtype=np.uint8)
+    rc = lib().ok_fingerprints(n, d.ctypes.data if d.size else None, off.ctypes.data,
+                               None if par is None else par.ctypes.data, m.ctypes.data, t.ctypes.data,
+                               keys.ctypes.data)
+    if rc != 0:
+        raise ValueError("parent[i] must be < i")
+    return keys[:n]
+
+
+def blob_digest(g: Geom, blob: np.ndarray, n_tokens: int, key: bytes):
+    """Returns (digest bytes[32], page digests uint8[P, 32])."""
+    nbytes, npages = blob_size(g, n_tokens)
+    b = _as_u8(blob)
+    assert b.size == nbytes
+    k = _as_u8(key)
+    assert k.size == 32
+    pages = np.zeros((npages, 32), dtype=np.uint8)
+    out = np.zeros(32, dtype=np.uint8)
+    cg = g.c()
+    lib().ok_blob_digest(ctypes.byref(cg), b.ctypes.data, n_tokens, k.ctypes.data, pages.ctypes.data,
+                         out.ctypes.data)
+    return out.tobytes(), pages

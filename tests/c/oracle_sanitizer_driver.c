@@ -9,6 +9,7 @@
 #include <string.h>
 
 #include "../../oracle/gk_oracle.h"
+#include "../../oracle/gk_sha256_oracle.h"
 
 static uint64_t rng_state = 0x9E3779B97F4A7C15ull;
 static uint8_t rnd(void)
@@ -83,6 +84,38 @@ static int run(const ok_geom *g, uint32_t n_src, uint32_t n_dst, uint32_t n_toke
     return 0;
 }
 
+/* fingerprints and digests on exact-size heap buffers */
+static int run_sha(const ok_geom *g, uint32_t n_tokens)
+{
+    uint8_t out[32];
+    for (size_t len = 0; len < 130; ++len) {
+        uint8_t *m = malloc(len ? len : 1);
+        for (size_t i = 0; i < len; ++i) m[i] = (uint8_t)(i * 7u + len);
+        ok_sha256(len ? m : NULL, len, out);
+        free(m);
+    }
+    uint64_t offsets[5] = {0, 0, 7, 64, 200};
+    int32_t parent[4] = {-1, 0, 1, -1};
+    uint8_t *data = malloc(200);
+    for (int i = 0; i < 200; ++i) data[i] = (uint8_t)(i * 3);
+    uint8_t model[32] = {1}, tenant[32] = {2};
+    uint8_t *keys = malloc(4 * 32);
+    if (ok_fingerprints(4, data, offsets, parent, model, tenant, keys) != 0) return 20;
+    parent[2] = 2;
+    if (ok_fingerprints(4, data, offsets, parent, model, tenant, keys) != -1) return 21;
+
+    uint64_t nbytes = 0;
+    uint32_t P = 0;
+    ok_blob_size(g, n_tokens, &nbytes, &P);
+    uint8_t *blob = malloc((size_t)nbytes);
+    for (uint64_t i = 0; i < nbytes; ++i) blob[i] = (uint8_t)(i ^ (i >> 8));
+    uint8_t *pages = malloc((size_t)P * 32);
+    ok_blob_digest(g, blob, n_tokens, keys, pages, out);
+    ok_blob_digest(g, blob, n_tokens, keys + 32, NULL, out);
+    free(pages); free(blob); free(keys); free(data);
+    return 0;
+}
+
 int main(void)
 {
     ok_geom bf16 = {3, 2, 8, 4, 2, 0};
@@ -95,6 +128,8 @@ int main(void)
         if ((rc = run(&fp8, 5, 11, lens[i])) != 0) { printf("fp8 len %u: %d\n", lens[i], rc); return 1; }
         if ((rc = run(&fp8_shared, 5, 11, lens[i])) != 0) { printf("fp8/1 len %u: %d\n", lens[i], rc); return 1; }
     }
+    ok_geom wide = {6, 4, 32, 8, 1, 2};   /* records of 12,480 bytes: three full digest chunks and a short one */
+    if (run_sha(&bf16, 9) != 0 || run_sha(&wide, 17) != 0) { printf("sha\n"); return 1; }
     printf("clean\n");
     return 0;
 }

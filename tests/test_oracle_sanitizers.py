@@ -12,6 +12,7 @@ def test_oracle_is_clean_under_asan_and_ubsan(tmp_path):
     exe = tmp_path / "oracle_san"
     cmd = ["gcc", "-std=c11", "-O1", "-g", "-fsanitize=address,undefined", "-fno-sanitize-recover=all",
            os.path.join(ROOT, "tests", "c", "oracle_sanitizer_driver.c"), os.path.join(ROOT, "oracle", "gk_oracle.c"),
+           os.path.join(ROOT, "oracle", "gk_sha256_oracle.c"),
            "-o", str(exe)]
     build = subprocess.run(cmd, capture_output=True, text=True)
     if build.returncode != 0 and "sanitize" in build.stderr:
