@@ -49,7 +49,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress", "longwindow"],
+    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress", "longwindow", "digest"],
                     help="gqa7b is the headline workload (full JSON line); the others print a shorter line "
                          "with the save and restore phases of that workload's shape")
     ap.add_argument("--window-blocks", type=int, default=48,
@@ -737,6 +737,87 @@ def run_longwindow(args):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------
+# second tier: block fingerprints and blob digests (SHA-256) on the headline batch
+# ---------------------------------------------------------------------------
+# Integer instructions per 64-byte SHA-256 block in the kernels (14 per round, 10 per
+# message-schedule word, 16 byte swaps, 8 final adds, loads and loop overhead), all of
+# which issue on the 64-lane integer pipe of an SM.
+SHA_INSTR_PER_BLOCK = 64 * 14 + 48 * 10 + 16 + 8 + 10
+INT_LANES_PER_SM_CLK = 64
+SM_COUNT = 148
+
+
+def run_digest(args):
+    import torch
+    import synth
+    import paper_2609_39358_b200 as gk
+
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    w = synth.GQA7B
+    n_blocks = args.blocks or synth.GQA7B_REQUESTS * synth.GQA7B_BLOCKS_PER_REQUEST
+    n_tok = synth.GQA7B_BLOCK_TOKENS
+    geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, gk.GK_BF16, 0)
+    ctx = gk.Context(geom, device.index)
+    nb, P = gk.gk_blob_size(geom, n_tok)
+    # blob bytes: any bytes do for a hash; bf16 N(0, sigma) patterns like the cache contents
+    blobs = [synth.kv_bytes_bf16(nb // 2, w.sigma, w.seed(800 + j), device) for j in range(n_blocks)]
+    jobs = [gk.Job(b, None, None, n_tok) for b in blobs]
+    # token ids of the blocks (int32), two-block chains per request
+    g = torch.Generator(device=device)
+    g.manual_seed(w.seed(820))
+    ids = torch.randint(0, 128000, (n_blocks * n_tok,), generator=g, device=device, dtype=torch.int32)
+    offsets = torch.arange(n_blocks + 1, dtype=torch.int64, device=device) * (4 * n_tok)
+    parent = [(-1 if j % synth.GQA7B_BLOCKS_PER_REQUEST == 0 else j - 1) for j in range(n_blocks)]
+    model, tenant = bytes(range(32)), bytes(range(32, 64))
+    keys = torch.zeros(n_blocks, 32, dtype=torch.uint8, device=device)
+    digests = torch.zeros(n_blocks, 32, dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream(device)
+    steps, warmup = min(args.steps, 20), max(args.warmup, 3)
+
+    def step(ev=None):
+        if ev:
+            ev[0].record(stream)
+        ctx.gk_fingerprints(ids.view(torch.uint8), offsets, parent, model, tenant, keys)
+        if ev:
+            ev[1].record(stream)
+        ctx.gk_blob_digests(jobs, keys, digests)
+        if ev:
+            ev[2].record(stream)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize(device)
+    sampler = ClockSampler(device.index)
+    sampler.wait_first_sample()
+    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(steps)]
+    for k in range(steps):
+        step(events[k])
+    torch.cuda.synchronize(device)
+    clocks = sampler.stop() or {}
+    fp_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in events]))
+    dg_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in events]))
+    total = n_blocks * nb
+    sm_mhz = clocks.get("sm_mhz") or clocks.get("sm_max_mhz") or 1965
+    peak = SM_COUNT * INT_LANES_PER_SM_CLK * sm_mhz * 1e6 / (SHA_INSTR_PER_BLOCK / 64.0) / 1e9
+    achieved = total / (dg_ms * 1e-3) / 1e9
+    line = {"metric": "blob digest GB/s (SHA-256 tree)", "value": achieved, "unit": UNIT, "n_gpus": 1, "steps": steps,
+            "warmup": warmup, "ms_per_step": fp_ms + dg_ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u32", "data": "synthetic",
+            "config": {"workload": f"digest: gqa7b geometry, {n_blocks} blocks x {n_tok} tokens, {total / 2**30:.2f} GiB of "
+                                   f"blobs, {n_blocks} keys over {4 * n_tok}-byte token-id blocks in chains of "
+                                   f"{synth.GQA7B_BLOCKS_PER_REQUEST}",
+                       "step": "gk_fingerprints + gk_blob_digests; inputs (8 GiB) larger than L2"},
+            "phases": {"fingerprints": {"ms": fp_ms}, "blob_digests": {"ms": dg_ms, "gbs": achieved}},
+            "roofline": {"bound": "alu", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                         "traffic": None,
+                         "peak_kind": f"derived: {SM_COUNT} SMs x {INT_LANES_PER_SM_CLK} integer lanes per clock x "
+                                      f"{sm_mhz} MHz (sampled) / {SHA_INSTR_PER_BLOCK / 64.0:.1f} instructions per byte"},
+            "clocks": clocks}
+    print(json.dumps(line), flush=True)
+
+
 def synth_requests(n_blocks):
     return f"{max(n_blocks // 2, 1)} requests x {min(n_blocks, 2)} blocks"
 
@@ -747,6 +828,8 @@ def main():
         run_reference(args)
     elif args.workload == "longwindow":
         run_longwindow(args)
+    elif args.workload == "digest":
+        run_digest(args)
     elif args.workload != "gqa7b":
         run_other_workload(args)
     else:

@@ -250,6 +250,41 @@ int gk_restore_stream(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk
                       uint8_t *mask_dev, int32_t *first_bad_page_dev, gk_window_fn consume, void *user,
                       void *stream);
 
+/* Block fingerprints (Section 2.2: a block's state is filed under a fingerprint of
+ * the exact input bytes, the model and the tenant; Section 2.1: state of one model
+ * or tenant must not load under another; Section 2.2 and Section 5: a block is
+ * reused only where its token positions match).  The paper gives no format; this
+ * library's keys are, with SHA-256 (FIPS 180-4), || for concatenation and
+ * little-endian integers,
+ *     inner_i = SHA-256( bytes_i || model[32] || tenant[32] || u64(len_i) || "GKF1" )
+ *     key_i   = SHA-256( parent_key || inner_i || "GKF2" )
+ * where bytes_i = data_dev[offsets_dev[i] .. offsets_dev[i+1]) (device; any
+ * alignment, 16-byte aligned starts are fastest) and parent_key is key_{parent[i]},
+ * or 32 zero bytes if parent[i] == -1: the key of a block depends on every block
+ * before it in its prompt.  parent is a HOST array of n entries with
+ * -1 <= parent[i] < i (else GK_ERR_ARG), or NULL for no chains; model and tenant
+ * are HOST arrays of 32 bytes.  keys_dev: device, n*32 bytes, 16-byte aligned.
+ * One thread hashes one message, so a call takes as long as its longest message
+ * (about 40 ns per 64 bytes) however many messages it has. */
+int gk_fingerprints(gk_ctx *ctx, const void *data_dev, const uint64_t *offsets_dev, const int32_t *parent,
+                    uint32_t n, const uint8_t *model, const uint8_t *tenant, uint8_t *keys_dev, void *stream);
+
+/* Confirmation hash of stored blocks (Section 3, sabotage-testing paragraph, lists
+ * a confirmation hash among the safety mechanisms; Section 7: loaded state is
+ * judged by byte comparison and cryptographic hashes).  A three-level SHA-256 tree
+ * over each blob, bound to the key the block is filed under:
+ *     leaf   = SHA-256( chunk || "GKL0" )      chunk = 4096 record bytes, the last may be shorter
+ *     page_p = SHA-256( leaf_0 || ... || leaf_{m-1} || u64(record bytes) || "GKP0" )
+ *     digest = SHA-256( page_0 || ... || page_{P-1} || key[32] || u32(n_tokens) || u32(P) || "GKB0" )
+ * jobs[j].blob: device, not NULL (else GK_ERR_ARG); checksums and page_table are
+ * ignored.  keys_dev: device, n_jobs*32 bytes.  digests_dev: device, n_jobs*32
+ * bytes, 16-byte aligned.  page_digests_dev: NULL, or device, 32 bytes per page of
+ * the call in job order, 16-byte aligned (tells which page of a blob changed).
+ * This is integer arithmetic, about 22 instructions per byte: an order of
+ * magnitude slower than the CRC path, meant as a second tier. */
+int gk_blob_digests(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const uint8_t *keys_dev,
+                    uint8_t *digests_dev, uint8_t *page_digests_dev, void *stream);
+
 /* Counters of this context.  Reads the device error word with a blocking copy. */
 int gk_get_stats(gk_ctx *ctx, gk_stats *out);
 

@@ -26,7 +26,8 @@ JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
 
 EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",
            "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times",
-           "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit", "gk_restore_stream"]
+           "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit", "gk_restore_stream",
+           "gk_fingerprints", "gk_blob_digests"]
 
 
 class GkError(RuntimeError):
@@ -121,6 +122,10 @@ def load_library() -> ctypes.CDLL:
     L.gk_restore_host.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
     L.gk_restore_stream.restype = ctypes.c_int
     L.gk_restore_stream.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, WINDOW_FN, vp, vp]
+    L.gk_fingerprints.restype = ctypes.c_int
+    L.gk_fingerprints.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_int32), u32, ctypes.c_char_p, ctypes.c_char_p, vp, vp]
+    L.gk_blob_digests.restype = ctypes.c_int
+    L.gk_blob_digests.argtypes = [vp, ctypes.POINTER(CJob), u32, vp, vp, vp, vp]
     L.gk_get_stats.restype = ctypes.c_int
     L.gk_get_stats.argtypes = [vp, ctypes.POINTER(CStats)]
     L.gk_get_kernel_times.restype = ctypes.c_int
@@ -321,6 +326,23 @@ class Context:
         if raised:
             raise raised[0]
         self._check(rc, "gk_restore_stream")
+
+    def gk_fingerprints(self, data: torch.Tensor, offsets: torch.Tensor, parent: Optional[Sequence[int]],
+                        model: bytes, tenant: bytes, keys: torch.Tensor, stream=None):
+        """data: device bytes; offsets: device int64/uint64 [n+1]; parent: host ints or None; keys: device uint8 [n, 32]."""
+        n = offsets.numel() - 1
+        assert len(model) == 32 and len(tenant) == 32 and keys.numel() >= 32 * n
+        par = None
+        if parent is not None:
+            assert len(parent) == n
+            par = (ctypes.c_int32 * max(n, 1))(*[int(x) for x in parent])
+        self._check(self._lib.gk_fingerprints(self._h, _ptr(data), _ptr(offsets), par, n, bytes(model), bytes(tenant),
+                                              _ptr(keys), _stream_handle(stream)), "gk_fingerprints")
+
+    def gk_blob_digests(self, jobs: Sequence[Job], keys: torch.Tensor, digests: torch.Tensor,
+                        page_digests: Optional[torch.Tensor] = None, stream=None):
+        self._check(self._lib.gk_blob_digests(self._h, self._jobs(jobs), len(jobs), _ptr(keys), _ptr(digests),
+                                              _ptr(page_digests), _stream_handle(stream)), "gk_blob_digests")
 
     def gk_get_kernel_times(self) -> dict:
         """{'verify'|'pack'|'commit'|'restore': (ms, launches)} since the previous call (needs tuning key profile=1)."""

@@ -15,6 +15,7 @@
 #include <vector>
 
 #include "gk_kernels.cuh"
+#include "gk_sha256.cuh"
 
 #ifndef GK_CRC_NT
 #define GK_CRC_NT 128
@@ -1232,6 +1233,104 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
     c->stats.jobs += n_jobs;
     c->stats.pages += pages;
     c->stats.bytes_blob += bytes;
+    return GK_OK;
+}
+
+int gk_fingerprints(gk_ctx *c, const void *data_dev, const uint64_t *offsets_dev, const int32_t *parent, uint32_t n,
+                    const uint8_t *model, const uint8_t *tenant, uint8_t *keys_dev, void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n == 0) return GK_OK;
+    if (!offsets_dev || !model || !tenant || !keys_dev) return fail(c, GK_ERR_ARG, "null offsets, model, tenant or keys");
+    if ((uintptr_t)keys_dev & 15u) return fail(c, GK_ERR_UNSUPPORTED, "keys must be 16-byte aligned");
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    // workspace: [parent n][depth n] | inner n*32
+    const size_t meta = align_up((size_t)n * 8, 256);
+    int rc = ensure_workspace(c, meta + (size_t)n * 32);
+    if (rc != GK_OK) return rc;
+    FingerprintParams P{};
+    P.data = (const uint8_t *)data_dev;
+    P.offsets = offsets_dev;
+    P.n = n;
+    std::memcpy(P.model, model, 32);
+    std::memcpy(P.tenant, tenant, 32);
+    P.inner = c->d_ws + meta;
+    P.keys = keys_dev;
+    if (parent) {
+        if ((rc = ensure_host_stage(c, (size_t)n * 8)) != GK_OK) return rc;
+        GK_CUDA(c, cudaEventSynchronize(c->ev_stage));
+        int32_t *hp = (int32_t *)c->h_stage;
+        uint32_t *hd = (uint32_t *)(c->h_stage + (size_t)n * 4);
+        uint32_t max_depth = 0;
+        for (uint32_t i = 0; i < n; ++i) {
+            if (parent[i] < -1 || (parent[i] >= 0 && (uint32_t)parent[i] >= i))
+                return fail(c, GK_ERR_ARG, "parent[%u] = %d: need -1 <= parent[i] < i", i, parent[i]);
+            hp[i] = parent[i];
+            hd[i] = parent[i] < 0 ? 0u : hd[parent[i]] + 1u;
+            if (hd[i] > max_depth) max_depth = hd[i];
+        }
+        GK_CUDA(c, cudaMemcpyAsync(c->d_ws, c->h_stage, (size_t)n * 8, cudaMemcpyHostToDevice, st));
+        GK_CUDA(c, cudaEventRecord(c->ev_stage, st));
+        P.parent = (const int32_t *)c->d_ws;
+        P.depth = (const uint32_t *)(c->d_ws + (size_t)n * 4);
+        P.max_depth = max_depth;
+    }
+    fingerprint_inner_kernel<<<(n + 63u) / 64u, 64, 0, st>>>(P);
+    GK_CUDA(c, cudaGetLastError());
+    fingerprint_chain_kernel<<<1, 1024, 0, st>>>(P);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched += 2;
+    return GK_OK;
+}
+
+int gk_blob_digests(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const uint8_t *keys_dev, uint8_t *digests_dev,
+                    uint8_t *page_digests_dev, void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0) return GK_OK;
+    if (!jobs || !keys_dev || !digests_dev) return fail(c, GK_ERR_ARG, "null jobs, keys or digests");
+    if (((uintptr_t)digests_dev | (uintptr_t)page_digests_dev) & 15u)
+        return fail(c, GK_ERR_UNSUPPORTED, "digest arrays must be 16-byte aligned");
+    for (uint32_t j = 0; j < n_jobs; ++j)
+        if (!jobs[j].blob) return fail(c, GK_ERR_ARG, "job %u: null blob", j);
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    uint64_t pages = 0;
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
+        pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
+    }
+    if (pages > 0x7fffffffull) return fail(c, GK_ERR_ARG, "too many pages in one call");
+    const uint32_t m_max = (uint32_t)((c->gd.R + kDigestChunk - 1) / kDigestChunk);
+    // workspace: job table | leaves | page digests (unless the caller wants them)
+    WsLayout l{};
+    l.jobs = 0;
+    const size_t o_leaves = align_up((size_t)n_jobs * sizeof(JobDev), 256);
+    const size_t o_pages = align_up(o_leaves + (size_t)pages * m_max * 32, 256);
+    int rc = ensure_workspace(c, o_pages + (size_t)pages * 32);
+    if (rc != GK_OK) return rc;
+    Tiling none{};
+    uint64_t bytes = 0;
+    if ((rc = upload_jobs(c, jobs, n_jobs, l, none, nullptr, nullptr, false, st, &pages, &bytes)) != GK_OK) return rc;
+    DigestParams P{};
+    P.g = c->gd;
+    P.jobs = (const JobDev *)c->d_ws;
+    P.n_jobs = n_jobs;
+    P.total_pages = (uint32_t)pages;
+    P.m_max = m_max;
+    P.leaves = c->d_ws + o_leaves;
+    P.page_digests = page_digests_dev ? page_digests_dev : c->d_ws + o_pages;
+    P.keys = keys_dev;
+    P.digests = digests_dev;
+    const uint64_t leaf_threads = pages * m_max;
+    sha_leaf_kernel<<<(unsigned)((leaf_threads + 127) / 128), 128, 0, st>>>(P);
+    GK_CUDA(c, cudaGetLastError());
+    sha_page_kernel<<<(unsigned)((pages + 63) / 64), 64, 0, st>>>(P);
+    GK_CUDA(c, cudaGetLastError());
+    sha_blob_kernel<<<(n_jobs + 63u) / 64u, 64, 0, st>>>(P);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched += 3;
     return GK_OK;
 }
 

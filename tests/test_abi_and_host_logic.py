@@ -174,3 +174,16 @@ def test_bit_sliced_scheme_reproduces_crc():
     init = _mod(_clmul(ones, gen.xpow(8 * len(data))))
     crc = int(format(total ^ init ^ ones, "064b")[::-1], 2)
     assert crc == oracle.crc64(data)
+
+
+def test_sha256_round_constants_in_the_kernel_source_match_the_derived_ones():
+    """The kernels carry the SHA-256 round constants and initial state as typed literals;
+    the oracle derives them from the primes.  Neither reads the other: compare them here."""
+    text = open(os.path.join(ROOT, "paper_2609_39358_b200", "csrc", "gk_sha256.cuh")).read()
+    table = text.split("kShaK[64] = {")[1].split("}")[0]
+    typed_k = [int(v, 16) for v in re.findall(r"0x([0-9a-f]{8})u", table)]
+    init = text.split("void sha_init(uint32_t h[8])")[1].split("}")[0]
+    typed_h = [int(v, 16) for v in re.findall(r"0x([0-9a-f]{8})u", init)]
+    k, h0 = oracle.sha256_constants()
+    assert typed_k == [int(v) for v in k]
+    assert typed_h == [int(v) for v in h0]
