@@ -121,3 +121,56 @@ def test_blob_digests_parity(gk, og):
     with pytest.raises(gk.GkError):
         ctx.gk_blob_digests([gk.Job(None, None, None, T)], dkeys, one)
     ctx.close()
+
+
+def test_confirmation_hash_sabotage_triple(gk):
+    """Section 3, sabotage testing: the attack -- an intact record of one block filed under
+    another block's key -- must succeed with the defence off and fail with it on.  The page
+    checksums cannot see this attack (every record byte is intact); the digest, which is
+    bound to the key, can."""
+    from gpu_harness import dev_cache, gpu_restore
+    og = oracle.Geom(5, 4, 64, 16, 2, 0)
+    T = og.page_tokens
+    n = 2 * T + 3
+    src = random_cache(og, 9, seed=520)
+    blob_a, sums_a, _, _ = oracle.pack(og, src, np.array([0, 1, 2], dtype=np.int32), n)
+    blob_b, sums_b, _, _ = oracle.pack(og, src, np.array([3, 4, 5], dtype=np.int32), n)
+    ctx = _ctx(gk, og)
+    # keys of two different texts, and the digests stored with each record at save time
+    text = np.frombuffer(b"first block of text " * 8 + b"another block, other text " * 8, dtype=np.uint8).copy()
+    off = np.array([0, 160, text.size], dtype=np.uint64)
+    keys = torch.from_numpy(_gpu_keys(ctx, text, off, None)).cuda()
+    assert not torch.equal(keys[0], keys[1])
+    stored = torch.zeros(2, 32, dtype=torch.uint8, device="cuda")
+    da, db = torch.from_numpy(blob_a).cuda(), torch.from_numpy(blob_b).cuda()
+    ctx.gk_blob_digests([gk.Job(da, None, None, n), gk.Job(db, None, None, n)], keys, stored)
+
+    def load_under_key_a(record_blob, record_sums, record_digest, defence_on):
+        """What a loader does with the record it found under key A."""
+        if defence_on:
+            got = torch.zeros(1, 32, dtype=torch.uint8, device="cuda")
+            ctx.gk_blob_digests([gk.Job(torch.from_numpy(record_blob).cuda(), None, None, n)], keys[0:1].contiguous(), got)
+            torch.cuda.synchronize()
+            if not torch.equal(got[0], record_digest):
+                return None                       # reported for recompute; nothing restored
+        dst = random_cache(og, 6, seed=521)
+        d = dev_cache(dst)
+        mask, _ = gpu_restore(ctx, d, [oracle.Job(record_blob, record_sums, np.array([1, 3, 5], dtype=np.int32), n)])
+        assert mask.tolist() == [0]               # the checksums see nothing wrong
+        return d
+
+    def holds(d, blob):
+        back = torch.zeros(blob.size, dtype=torch.uint8, device="cuda")
+        sums = torch.zeros(3, dtype=torch.int64, device="cuda")
+        ctx.gk_pack_batch(d, [gk.Job(back, sums, torch.tensor([1, 3, 5], dtype=torch.int32, device="cuda"), n)])
+        torch.cuda.synchronize()
+        return np.array_equal(back.cpu().numpy(), blob)
+
+    # attack: B's record (blob, checksums, digest) is filed under key A
+    assert load_under_key_a(blob_b, sums_b, stored[1], defence_on=True) is None        # defence on: refused
+    served = load_under_key_a(blob_b, sums_b, stored[1], defence_on=False)             # defence off: B's state is served for A
+    assert served is not None and holds(served, blob_b)
+    assert load_under_key_a(blob_b, sums_b, stored[1], defence_on=True) is None        # defence restored: refused again
+    ok = load_under_key_a(blob_a, sums_a, stored[0], defence_on=True)                  # the honest record loads
+    assert ok is not None and holds(ok, blob_a)
+    ctx.close()
