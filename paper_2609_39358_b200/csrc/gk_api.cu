@@ -126,6 +126,7 @@ struct gk_ctx {
     cudaEvent_t ev_copied[kSlots] = {nullptr, nullptr};
     bool slot_used[kSlots] = {false, false};
     uint32_t slot_next = 0;  // the slot the next batch goes to (carried across calls)
+    bool pdl_next = false;   // the kernel just enqueued lets the next one start early (small calls)
 
     // streaming restore: the ids 0..iota_cap-1, from which window page tables are cut
     int32_t *d_iota = nullptr;
@@ -459,6 +460,7 @@ int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tili
     prep_small_kernel<<<1, 1024, 0, st>>>(pp, w);
     GK_CUDA(c, cudaGetLastError());
     c->stats.kernels_launched++;
+    c->pdl_next = !c->profile;  // timing events between the two launches would break the pairing
     return GK_OK;
 }
 
@@ -470,11 +472,35 @@ uint32_t stream_grid(const gk_ctx *c, int occ, uint32_t n_items)
     return g ? g : 1u;
 }
 
+// Launches a streaming kernel; right behind the small-call preparation kernel it is
+// launched as a programmatic dependent, so that its CTAs are resident and their
+// rings set up by the time the preparation kernel ends.
+template <class Kernel>
+cudaError_t launch_streaming(gk_ctx *c, Kernel kernel, uint32_t grid, int threads, size_t smem, cudaStream_t st,
+                             const StreamParams &Q)
+{
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3((unsigned)threads);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr{};
+    attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr.val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = &attr;
+    cfg.numAttrs = c->pdl_next ? 1u : 0u;
+    c->pdl_next = false;
+    return cudaLaunchKernelEx(&cfg, kernel, Q);
+}
+
 template <class Cfg, int MODE, int NT, int SB, int ST, int MINB>
 int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
 {
     const uint32_t items = MODE == kCommit ? P.n_items_c : P.n_items;
-    if (items == 0) return GK_OK;
+    if (items == 0) {
+        c->pdl_next = false;
+        return GK_OK;
+    }
     const uint32_t grid = stream_grid(c, occ, items);
     gk_ctx::ProfSlot *slot = nullptr;
     if (c->profile) {
@@ -494,8 +520,7 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
     if (ci) Q.ctr_base_c = c->ctr_next[1];
     else Q.ctr_base_v = c->ctr_next[0];
     c->ctr_next[ci] += items + grid;
-    stream_kernel<MODE, NT, SB, ST, MINB><<<grid, Cfg::kThreads, Cfg::kSmemBytes, st>>>(Q);
-    GK_CUDA(c, cudaGetLastError());
+    GK_CUDA(c, launch_streaming(c, stream_kernel<MODE, NT, SB, ST, MINB>, grid, Cfg::kThreads, Cfg::kSmemBytes, st, Q));
     if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
     return GK_OK;
@@ -518,7 +543,10 @@ int launch_commit(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
     const uint32_t items = P.n_items > P.n_items_c ? P.n_items : P.n_items_c;
-    if (items == 0) return GK_OK;
+    if (items == 0) {
+        c->pdl_next = false;
+        return GK_OK;
+    }
     const uint32_t grid = stream_grid(c, c->occ_fused, items);
     gk_ctx::ProfSlot *slot = nullptr;
     if (c->profile) {
@@ -537,9 +565,9 @@ int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
     Q.ctr_base_c = c->ctr_next[1];
     c->ctr_next[0] += P.n_items + grid;
     c->ctr_next[1] += P.n_items_c + grid;
-    restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES, GK_FUSED_MINB>
-        <<<grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st>>>(Q);
-    GK_CUDA(c, cudaGetLastError());
+    GK_CUDA(c, launch_streaming(c, restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE,
+                                                  GK_FUSED_CSTAGES, GK_FUSED_MINB>,
+                                grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st, Q));
     if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
     return GK_OK;

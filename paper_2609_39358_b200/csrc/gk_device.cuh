@@ -251,6 +251,21 @@ __device__ __forceinline__ void fence_mbar_init()
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
 
+// Programmatic dependent launch.  A kernel launched with the programmatic stream
+// serialization attribute may start while the kernel before it in the stream is
+// still running; grid_dependency_wait() then blocks until that kernel has finished
+// and its writes are visible (without the attribute it returns at once).  The
+// earlier kernel calls allow_dependent_launch() to let the next one start early.
+__device__ __forceinline__ void grid_dependency_wait()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+__device__ __forceinline__ void allow_dependent_launch()
+{
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ uint64_t policy_evict_first()
 {
     uint64_t p;

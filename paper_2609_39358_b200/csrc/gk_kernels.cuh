@@ -118,6 +118,7 @@ struct PrepSmallParams {
 
 __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant__ PrepSmallParams pp, WorkDev w)
 {
+    allow_dependent_launch();  // the streaming kernel behind this one may set up its rings meanwhile
     JobDev *jobs_out = const_cast<JobDev *>(w.jobs);
     uint64_t *pow_out = const_cast<uint64_t *>(w.seg_pow);
     for (uint32_t j = threadIdx.x; j < w.n_jobs; j += blockDim.x) {
@@ -909,6 +910,7 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
         *abort_flag = 0u;
         fence_mbar_init();
     }
+    grid_dependency_wait();  // everything above is CTA-local; the tables of the call are read below
     __syncthreads();
 
     if (warp == Cfg::kLoaderWarp) {
@@ -961,6 +963,7 @@ __global__ void __launch_bounds__(NT + 96, MINB) restore_kernel(const __grid_con
         *abort_flag = 0u;
         fence_mbar_init();
     }
+    grid_dependency_wait();  // everything above is CTA-local; the tables of the call are read below
     __syncthreads();
 
     constexpr int kCons = NT / 32;
