@@ -78,6 +78,28 @@ class WindowBlock:
     page_table: int   # device address of the block's int32 ring page ids
 
 
+def _marshal_jobs(jobs: Sequence["Job"]):
+    arr = (CJob * max(len(jobs), 1))()
+    for i, j in enumerate(jobs):
+        arr[i] = CJob(_ptr(j.blob), _ptr(j.checksums), _ptr(j.page_table), j.n_tokens, j.request_id)
+    return arr
+
+
+class JobArray:
+    """A job list marshalled once, for callers that submit the same jobs repeatedly: every
+    method that takes a job list also takes a JobArray.  Keeps the jobs' tensors alive."""
+
+    def __init__(self, jobs: Sequence["Job"]):
+        self.jobs = list(jobs)
+        self.arr = _marshal_jobs(self.jobs)
+
+    def __len__(self):
+        return len(self.jobs)
+
+    def __getitem__(self, i):
+        return self.jobs[i]
+
+
 _lib = None
 
 
@@ -251,11 +273,8 @@ class Context:
         if rc != GK_OK:
             raise GkError(rc, where, self._lib.gk_last_error(self._h).decode(errors="replace"))
 
-    def _jobs(self, jobs: Sequence[Job]):
-        arr = (CJob * max(len(jobs), 1))()
-        for i, j in enumerate(jobs):
-            arr[i] = CJob(_ptr(j.blob), _ptr(j.checksums), _ptr(j.page_table), j.n_tokens, j.request_id)
-        return arr
+    def _jobs(self, jobs):
+        return jobs.arr if isinstance(jobs, JobArray) else _marshal_jobs(jobs)
 
     def set_tuning(self, key: str, value: int):
         self._check(self._lib.gk_ctx_set_tuning(self._h, key.encode(), value), "gk_ctx_set_tuning")

@@ -140,6 +140,12 @@ struct gk_ctx {
     double prof_ms[4] = {0, 0, 0, 0};
     uint64_t prof_launches[4] = {0, 0, 0, 0};
 
+    // powers of x^(8 * segment bytes) for the segment lengths used recently (host arithmetic
+    // of a few microseconds per length, which small calls would otherwise pay every time)
+    struct SegPowers { uint64_t seg_bytes = 0; uint64_t x_seg = 0; std::vector<uint64_t> pw; uint64_t used = 0; };
+    SegPowers seg_cache[4];
+    uint64_t seg_cache_clock = 0;
+
     gk_stats stats{};
     char err[512] = {0};
 };
@@ -355,7 +361,26 @@ int ensure_host_stage(gk_ctx *c, size_t need)
     return GK_OK;
 }
 
-WorkDev make_work(const gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t total_pages, const Tiling &crc)
+// x^(8*seg_bytes) and its powers 0..n-1 mod P, from the context's cache
+const gk_ctx::SegPowers &seg_powers(gk_ctx *c, uint64_t seg_bytes, uint32_t n)
+{
+    gk_ctx::SegPowers *e = nullptr, *oldest = &c->seg_cache[0];
+    for (auto &s : c->seg_cache) {
+        if (s.seg_bytes == seg_bytes && s.x_seg != 0) e = &s;
+        if (s.used < oldest->used) oldest = &s;
+    }
+    if (!e) {
+        e = oldest;
+        e->seg_bytes = seg_bytes;
+        e->x_seg = gf_xpow(8ull * seg_bytes);
+        e->pw.assign(1, 1ull);
+    }
+    while (e->pw.size() < n) e->pw.push_back(gf_mul(e->pw.back(), e->x_seg));
+    e->used = ++c->seg_cache_clock;
+    return *e;
+}
+
+WorkDev make_work(gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t total_pages, const Tiling &crc)
 {
     WorkDev w{};
     w.jobs = (const JobDev *)(c->d_ws + l.jobs);
@@ -374,7 +399,7 @@ WorkDev make_work(const gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t 
     w.work_ctr = c->d_error + 16;
     w.init_term = c->d_init_term;
     w.thread_const = c->d_thread_const;
-    w.x_seg = gf_xpow(8ull * crc.seg_tiles * crc.stage_bytes);
+    w.x_seg = seg_powers(c, (uint64_t)crc.seg_tiles * crc.stage_bytes, 1).x_seg;
     w.seg_pow = (const uint64_t *)(c->d_ws + l.jobs + (size_t)n_jobs * sizeof(JobDev));
     w.wait_limit_ns = c->wait_limit_ns;
     return w;
@@ -413,10 +438,11 @@ int fill_job_table(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, JobDev *h, ui
 }
 
 // powers of x^(8 * segment bytes), which place segment remainders inside their page
-void fill_seg_pow(const Tiling &crc, uint64_t *pw)
+void fill_seg_pow(gk_ctx *c, const Tiling &crc, uint64_t *pw)
 {
-    const uint64_t xs = gf_xpow(8ull * crc.seg_tiles * crc.stage_bytes);
-    for (uint32_t k = 0; k < crc.nseg_max; ++k) pw[k] = k ? gf_mul(pw[k - 1], xs) : 1ull;
+    if (crc.nseg_max == 0) return;
+    const gk_ctx::SegPowers &sp = seg_powers(c, (uint64_t)crc.seg_tiles * crc.stage_bytes, crc.nseg_max);
+    std::memcpy(pw, sp.pw.data(), (size_t)crc.nseg_max * 8);
 }
 
 // Fills the pinned job table (and the segment powers behind it) and enqueues the upload.
@@ -432,7 +458,7 @@ int upload_jobs(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const WsLayout &
     if ((rc = fill_job_table(c, jobs, n_jobs, h, blob_override, sums_override, need_tables, total_pages_out,
                              total_bytes_out)) != GK_OK)
         return rc;
-    fill_seg_pow(crc, reinterpret_cast<uint64_t *>(c->h_stage + (size_t)n_jobs * sizeof(JobDev)));
+    fill_seg_pow(c, crc, reinterpret_cast<uint64_t *>(c->h_stage + (size_t)n_jobs * sizeof(JobDev)));
     GK_CUDA(c, cudaMemcpyAsync(c->d_ws + l.jobs, h, table_bytes, cudaMemcpyHostToDevice, st));
     GK_CUDA(c, cudaEventRecord(c->ev_stage, st));
     return GK_OK;
@@ -452,7 +478,7 @@ int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tili
     PrepSmallParams pp{};
     int rc = fill_job_table(c, jobs, n_jobs, pp.jobs, nullptr, nullptr, need_tables, pages_out, bytes_out);
     if (rc != GK_OK) return rc;
-    fill_seg_pow(crc, pp.seg_pow);
+    fill_seg_pow(c, crc, pp.seg_pow);
     pp.n_seg_pow = crc.nseg_max;
     pp.do_claims = do_claims ? 1u : 0u;
     pp.num_pages = num_pages;

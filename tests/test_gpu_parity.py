@@ -423,6 +423,30 @@ def test_stream_restore_on_a_side_stream_and_refusals(gk):
     ctx.close()
 
 
+def test_job_array_marshalled_once_gives_the_same_result(gk):
+    from gpu_harness import assert_cache_equal, dev_cache, dev_i32, sums_to_dev
+    og = G_MID
+    T = og.page_tokens
+    src = random_cache(og, 9, seed=340)
+    ojobs = _oracle_jobs(og, src, [2 * T, T + 3, 1], 341, 12)
+    clean = random_cache(og, 12, seed=342)
+    want = clone_cache(clean)
+    wmask, _ = oracle.restore(og, want, ojobs)
+    ctx = _ctx(gk, og)
+    jobs = gk.JobArray([gk.Job(torch.from_numpy(j.blob).cuda(), sums_to_dev(j.checksums), dev_i32(j.page_table), j.n_tokens)
+                        for j in ojobs])
+    assert len(jobs) == 3 and jobs[1].n_tokens == T + 3
+    for _ in range(3):                                   # the same marshalled array, call after call
+        d = dev_cache(clean)
+        mask = torch.full((3,), 255, dtype=torch.uint8, device="cuda")
+        fb = torch.full((3,), -7, dtype=torch.int32, device="cuda")
+        ctx.gk_restore(jobs, d, mask, fb)
+        torch.cuda.synchronize()
+        assert mask.cpu().tolist() == wmask.tolist()
+        assert_cache_equal(d, want)
+    ctx.close()
+
+
 def test_restore_codes_and_first_bad_page(gk):
     from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
     og, N = G_MID, 12
