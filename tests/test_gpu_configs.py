@@ -408,3 +408,122 @@ def test_stress_waves(gk, bad_frac):
     assert total_rejected > 0
     assert ctx.gk_get_stats()["device_wait_expired"] == 0
     ctx.close()
+
+
+def test_long_window_stream_restore(gk):
+    """Blocks of 30,000 tokens (the block size of the paper's flat-memory experiment,
+    Section 4.3) in the GQA-7B geometry, streamed from pinned host memory through a ring of
+    two blocks: sampled records against the oracle, and, inside the consumer of every
+    window, every page of the ring against the source caches on the device."""
+    w = synth.GQA7B
+    T = w.page_tokens
+    geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens)
+    ctx = gk.Context(geom, 0)
+    s = _slab(w)
+    lens3 = [30000, 29999, 30000]                       # A, B (partial last page), C (will be damaged)
+    P = 1875
+    srcs, host, tables = [], [], []
+    rng = np.random.default_rng(w.seed(40))
+    for k, n in enumerate(lens3):
+        src = _dev_cache(gk, w, P, synth.kv_bytes_bf16(w.layers * P * s, w.sigma, w.seed(41 + k), "cuda"))
+        spt = synth.page_permutation(P, w.seed(45 + k))
+        hb = torch.empty(gk.gk_blob_size(geom, n)[0], dtype=torch.uint8, pin_memory=True)
+        hs = torch.empty(P, dtype=torch.int64, pin_memory=True)
+        status = torch.full((1,), 255, dtype=torch.uint8, device="cuda")
+        ctx.gk_pack_host(src, [gk.Job(hb, hs, torch.from_numpy(spt.copy()).cuda(), n)], status)
+        torch.cuda.synchronize()
+        assert status.item() == 0
+        _check_sampled_records(w, src, [(hb, hs, spt, n)], rng, 6)
+        srcs.append(src)
+        host.append((hb, hs))
+        tables.append(spt)
+    host[2][0][2_000_000_001] ^= 0x40                   # C: one flipped bit, in page 953
+    order = [0, 1, 2, 0, 1, 2, 1]                       # windows: {A,B} {C,A} {B,C} {B}
+    jobs = [gk.Job(host[k][0], host[k][1], None, lens3[k]) for k in order]
+    ring_pages = 2 * P + 10
+    sentinel = synth.sentinel_bytes(2 * w.layers * ring_pages * s, w.seed(49), "cuda")
+    ring = _dev_cache(gk, w, ring_pages, sentinel.clone())
+    rv = _view(w, ring)
+    mask = torch.full((len(order),), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.full((len(order),), -7, dtype=torch.int32, device="cuda")
+    checks, windows = [], []
+    prev = {"img": sentinel.clone()}
+
+    def consume(blocks, st):
+        windows.append([b.job for b in blocks])
+        pv = prev["img"].view(w.layers, 2, ring_pages, T, -1)
+        first = 0
+        for b in blocks:
+            assert (b.page_table - blocks[0].page_table) // 4 == first
+            k = order[b.job]
+            n = lens3[k]
+            if k == 2:      # damaged: its pages keep what the previous window left there
+                checks.append(torch.equal(rv[:, :, first:first + P], pv[:, :, first:first + P]))
+            else:
+                full = n // T
+                idx = torch.from_numpy(tables[k][:full].astype(np.int64)).cuda()
+                checks.append(torch.equal(rv[:, :, first:first + full], _view(w, srcs[k])[:, :, idx]))
+                if full < P:
+                    t, sp = n - full * T, int(tables[k][full])
+                    checks.append(torch.equal(rv[:, :, first + full, :t], _view(w, srcs[k])[:, :, sp, :t]))
+                    checks.append(torch.equal(rv[:, :, first + full, t:], pv[:, :, first + full, t:]))
+            first += P
+        checks.append(torch.equal(rv[:, :, first:], pv[:, :, first:]))      # pages beyond the window
+        prev["img"] = ring.data.clone()
+
+    ctx.gk_restore_stream(jobs, ring, mask, fb, consume)
+    torch.cuda.synchronize()
+    assert windows == [[0, 1], [2, 3], [4, 5], [6]]
+    assert mask.cpu().tolist() == [1 if k == 2 else 0 for k in order]
+    og = oracle_geom(w)
+    bad_page = 2_000_000_001 // oracle.record_bytes(og, 30000, 0)
+    assert [fb.cpu().tolist()[i] for i, k in enumerate(order) if k == 2] == [bad_page] * 2
+    assert all(checks) and len(checks) >= 12
+    assert ctx.gk_get_stats()["device_wait_expired"] == 0
+    ctx.close()
+
+
+def test_gqa7b_full_digests_and_keys(gk):
+    """The second tier at the headline batch size: 16 blocks of 4,096 tokens (8 GiB).  Sampled
+    page digests against the oracle; every root recomputed with hashlib from the page
+    digests the GPU reports; keys of the 16 token-id blocks against the oracle."""
+    import hashlib
+    import struct
+    w = synth.GQA7B
+    og = oracle_geom(w)
+    geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens)
+    ctx = gk.Context(geom, 0)
+    n_tok, NB = synth.GQA7B_BLOCK_TOKENS, synth.GQA7B_REQUESTS * synth.GQA7B_BLOCKS_PER_REQUEST
+    nbytes, P = gk.gk_blob_size(geom, n_tok)
+    blobs = [synth.kv_bytes_bf16(nbytes // 2, w.sigma, w.seed(60 + j), "cuda") for j in range(NB)]
+    # keys
+    g = torch.Generator(device="cuda")
+    g.manual_seed(w.seed(80))
+    ids = torch.randint(0, 128000, (NB * n_tok,), generator=g, device="cuda", dtype=torch.int32)
+    offsets = torch.arange(NB + 1, dtype=torch.int64, device="cuda") * (4 * n_tok)
+    parent = [(-1 if j % 2 == 0 else j - 1) for j in range(NB)]
+    model, tenant = bytes(range(32)), bytes(range(64, 96))
+    keys = torch.zeros(NB, 32, dtype=torch.uint8, device="cuda")
+    ctx.gk_fingerprints(ids.view(torch.uint8), offsets, parent, model, tenant, keys)
+    torch.cuda.synchronize()
+    want_keys = oracle.fingerprints(ids.cpu().numpy().view(np.uint8), offsets.cpu().numpy().astype(np.uint64), parent,
+                                    model, tenant)
+    assert np.array_equal(keys.cpu().numpy(), want_keys)
+    # digests
+    digests = torch.zeros(NB, 32, dtype=torch.uint8, device="cuda")
+    pages = torch.zeros(NB * P, 32, dtype=torch.uint8, device="cuda")
+    ctx.gk_blob_digests([gk.Job(b, None, None, n_tok) for b in blobs], keys, digests, pages)
+    torch.cuda.synchronize()
+    hp, hd, hk = pages.cpu().numpy(), digests.cpu().numpy(), keys.cpu().numpy()
+    rng = np.random.default_rng(w.seed(81))
+    R = oracle.record_bytes(og, n_tok, 0)
+    for _ in range(12):
+        j, p = int(rng.integers(0, NB)), int(rng.integers(0, P))
+        rec = blobs[j][p * R:(p + 1) * R].cpu().numpy()
+        _, one = oracle.blob_digest(og, rec, w.page_tokens, bytes(32))        # a one-page blob: its page node
+        assert np.array_equal(hp[j * P + p], one[0]), (j, p)
+    for j in range(NB):
+        root = hashlib.sha256(hp[j * P:(j + 1) * P].tobytes() + hk[j].tobytes() + struct.pack("<II", n_tok, P)
+                              + b"GKB0").digest()
+        assert hd[j].tobytes() == root
+    ctx.close()
