@@ -25,6 +25,7 @@ _HDRS = [os.path.join(_HERE, "gk_oracle.h"), os.path.join(_HERE, "gk_sha256_orac
 
 CODE_OK, CODE_CHECKSUM, CODE_PAGE_TABLE, CODE_MISSING = 0, 1, 2, 3
 FLAG_SKIP_VERIFY = 1
+FLAG_SINGLE_PASS = 4
 
 
 def build(force: bool = False) -> str:

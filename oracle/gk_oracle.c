@@ -257,9 +257,12 @@ void ok_restore(const ok_geom *g, const ok_cache *dst, const ok_job *jobs, uint3
             }
         }
     }
-    /* ---- phase 2: commit the jobs that passed; nothing else is written ---- */
+    /* ---- phase 2: commit the jobs that passed; nothing else is written ----
+     * (single-pass reading: a job whose only fault is a checksum mismatch is written too) */
     for (uint32_t j = 0; j < n_jobs; ++j) {
-        if (mask[j] != OK_CODE_OK)
+        int write_it = mask[j] == OK_CODE_OK ||
+                       ((flags & OK_FLAG_SINGLE_PASS) && mask[j] == OK_CODE_CHECKSUM);
+        if (!write_it)
             continue;
         uint32_t P = page_count(g, jobs[j].n_tokens);
         for (uint32_t p = 0; p < P; ++p) {

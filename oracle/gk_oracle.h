@@ -80,6 +80,13 @@ enum {
 };
 
 #define OK_FLAG_SKIP_VERIFY 1u /* sabotage tests: switch the checksum defence off */
+/* Single-pass load.  Section 2.2 has the runtime recompute a block whose record
+ * fails a check, which overwrites the block's pages anyway; under this optional
+ * reading a block whose only fault is a checksum mismatch is still reported with
+ * code 1, but its destination pages receive the record bytes as they are
+ * (unverified).  Blocks with code 2 or 3 still write nothing, and nothing
+ * outside the reported block's own pages changes.  Off by default. */
+#define OK_FLAG_SINGLE_PASS 4u
 
 /* CRC-64/XZ by its bit-at-a-time definition. */
 uint64_t ok_crc64_bitwise(const uint8_t *data, size_t len);

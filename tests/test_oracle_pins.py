@@ -402,6 +402,58 @@ def test_sabotage_triple_defence_on_off_on():
     assert mask[0] == oracle.CODE_CHECKSUM and np.array_equal(dst.data, clean.data)
 
 
+@pytest.mark.parametrize("g", [SMALL, SMALL_FP8])
+def test_single_pass_reading(g):
+    """Optional reading: a block whose only fault is a checksum mismatch is reported but its
+    own pages receive the unverified bytes; every other rule stands."""
+    N = 14
+    T = g.page_tokens
+    src = random_cache(g, 9, seed=55)
+    lens = [2 * T + 1, T, 3 * T, 1, 2 * T]
+    rng = np.random.default_rng(56)
+    perm = rng.permutation(N).astype(np.int32)
+    jobs, used = [], 0
+    for n in lens:
+        P = n_pages(g, n)
+        blob, sums, _, _ = oracle.pack(g, src, rng.integers(0, 9, size=P).astype(np.int32), n)
+        jobs.append(oracle.Job(blob, sums, perm[used:used + P].copy(), n))
+        used += P
+    clean = _sentinel_cache(g, N, seed=57)
+    # all good: the flag changes nothing
+    a, b = clone_cache(clean), clone_cache(clean)
+    ma, fa = oracle.restore(g, a, jobs)
+    mb, fb_ = oracle.restore(g, b, jobs, flags=oracle.FLAG_SINGLE_PASS)
+    assert ma.tolist() == mb.tolist() == [0] * 5 and fa.tolist() == fb_.tolist()
+    assert np.array_equal(a.data, b.data)
+    # job 0 damaged in its partial page, job 2 with an out-of-range id, job 3 missing, job 4 damaged
+    jobs[0].blob[-1] ^= 0x01
+    jobs[2].page_table[1] = N + 3
+    jobs[3] = oracle.Job(None, None, jobs[3].page_table, 1)
+    jobs[4].checksums[0] ^= np.uint64(1)
+    strict, single, forced = clone_cache(clean), clone_cache(clean), clone_cache(clean)
+    ms, fs = oracle.restore(g, strict, jobs)
+    m1, f1 = oracle.restore(g, single, jobs, flags=oracle.FLAG_SINGLE_PASS)
+    assert ms.tolist() == m1.tolist() == [1, 0, 2, 3, 1]             # same report either way
+    assert fs.tolist() == f1.tolist() == [2, -1, 1, -1, 0]
+    # what differs are exactly the pages of the two checksum failures, which hold what a
+    # restore without any check would have put there
+    oracle.restore(g, forced, [jobs[0], jobs[4]], flags=oracle.FLAG_SKIP_VERIFY)
+    expect = clone_cache(strict)
+    L = g.layers
+    for jb in (jobs[0], jobs[4]):
+        for page in jb.page_table[:n_pages(g, jb.n_tokens)]:
+            for arr_e, arr_f, per_page in ((expect.data, forced.data, slab_bytes(g)),) + (
+                    ((expect.scales, forced.scales, g.kv_heads * 4),) if g.scale_kv else ()):
+                kvn = 2 if per_page == slab_bytes(g) else g.scale_kv
+                ve = arr_e.reshape(L, kvn, N, per_page)
+                vf = arr_f.reshape(L, kvn, N, per_page)
+                ve[:, :, page] = vf[:, :, page]
+    assert np.array_equal(single.data, expect.data)
+    if g.scale_kv:
+        assert np.array_equal(single.scales, expect.scales)
+    assert not np.array_equal(single.data, strict.data)
+
+
 def test_codes_and_first_bad_page():
     g, N = SMALL, 12
     src = random_cache(g, N, seed=50)
