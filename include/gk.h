@@ -91,6 +91,18 @@ extern "C" {
  * library (the paper leaves the cache layout to the runtime it wraps). */
 #define GK_FLAG_HEAD_MAJOR 2u
 
+/* Single-pass restore.  Section 2.2 has the runtime recompute every block whose
+ * record fails a check, which rewrites that block's pages; a caller that does so
+ * may set this flag: gk_restore* then checks and scatters each record in ONE pass
+ * over the blob (2 bytes of memory traffic per blob byte instead of 3).  A block
+ * whose only fault is a checksum mismatch is reported exactly as without the flag
+ * (GK_JOB_CHECKSUM, same first bad page), but its OWN destination pages have
+ * received the unverified record bytes and must not be used.  Blocks with
+ * GK_JOB_PAGE_TABLE or GK_JOB_MISSING still write nothing, and no byte outside a
+ * reported block's own pages (valid token range) changes.  Off by default: without
+ * it nothing of a failing block is written.  gk_verify and gk_commit ignore it. */
+#define GK_FLAG_SINGLE_PASS 4u
+
 typedef struct gk_ctx gk_ctx;
 
 typedef struct {
@@ -101,7 +113,7 @@ typedef struct {
     uint32_t dtype;    /* GK_BF16 or GK_FP8_E4M3 */
     uint32_t scale_kv; /* fp8: 2 = a K scale and a V scale per (layer, head, page), 1 = one
                           shared scale; bf16: 0 */
-    uint32_t flags;    /* 0 or an OR of GK_FLAG_SKIP_VERIFY, GK_FLAG_HEAD_MAJOR */
+    uint32_t flags;    /* 0 or an OR of GK_FLAG_SKIP_VERIFY, GK_FLAG_HEAD_MAJOR, GK_FLAG_SINGLE_PASS */
     uint32_t reserved; /* must be 0 */
 } gk_geom;
 

@@ -22,6 +22,7 @@ GK_OK = 0
 GK_BF16, GK_FP8_E4M3 = 0, 1
 GK_FLAG_SKIP_VERIFY = 1
 GK_FLAG_HEAD_MAJOR = 2
+GK_FLAG_SINGLE_PASS = 4
 JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
 
 EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",

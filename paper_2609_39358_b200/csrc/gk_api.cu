@@ -67,6 +67,7 @@ namespace {
 using VerifyCfg = StreamCfg<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES>;
 using PackCfg = StreamCfg<kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES>;
 using CommitCfg = StreamCfg<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES>;
+using SingleCfg = StreamCfg<kSingle, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES>;
 using FusedCfg = RestoreCfg<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES>;
 
 constexpr int kSlots = 2;  // host-tier staging ring
@@ -97,7 +98,7 @@ struct gk_ctx {
     GeomDev gd{};
     int device = 0;
     int sm_count = 0;
-    int occ_verify = 0, occ_pack = 0, occ_commit = 0, occ_fused = 0;
+    int occ_verify = 0, occ_pack = 0, occ_commit = 0, occ_fused = 0, occ_single = 0;
     bool fused = true;           // restore runs verify and commit in one launch
     unsigned long long wait_limit_ns = kWaitLimitNs;
     uint32_t ctr_next[2] = {0, 0};  // what the device work counters will read when the next launch starts
@@ -174,7 +175,8 @@ int check_geom(const gk_geom *g, GeomDev *out)
 {
     if (!g) return GK_ERR_ARG;
     if (g->layers == 0 || g->kv_heads == 0 || g->head_dim == 0 || g->page_tokens == 0) return GK_ERR_ARG;
-    if (g->reserved != 0 || (g->flags & ~(GK_FLAG_SKIP_VERIFY | GK_FLAG_HEAD_MAJOR))) return GK_ERR_ARG;
+    if (g->reserved != 0 || (g->flags & ~(GK_FLAG_SKIP_VERIFY | GK_FLAG_HEAD_MAJOR | GK_FLAG_SINGLE_PASS)))
+        return GK_ERR_ARG;
     uint32_t elem;
     if (g->dtype == GK_BF16) {
         elem = 2;
@@ -537,7 +539,7 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
             c->prof_pool.push_back(ns);
         }
         slot = &c->prof_pool[c->prof_used++];
-        slot->cls = MODE;
+        slot->cls = MODE;  // kSingle == 3: booked with the fused restore kernel
         GK_CUDA(c, cudaEventRecord(slot->a, st));
     }
     // every work item is drawn once, and every CTA draws once more to learn that none is left
@@ -559,6 +561,11 @@ int launch_verify(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 int launch_pack(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
     return launch_stream<PackCfg, kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>(c, c->occ_pack, P, st);
+}
+// single-pass restore; per-kernel timing books it under "restore" (index 3)
+int launch_single(gk_ctx *c, const StreamParams &P, cudaStream_t st)
+{
+    return launch_stream<SingleCfg, kSingle, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>(c, c->occ_single, P, st);
 }
 int launch_commit(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
@@ -787,7 +794,12 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
     if (cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FusedCfg::kSmemBytes) != cudaSuccess ||
         cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_fused, kf, FusedCfg::kThreads, FusedCfg::kSmemBytes) != cudaSuccess)
         return bail(GK_ERR_CUDA);
-    if (c->occ_verify < 1 || c->occ_pack < 1 || c->occ_commit < 1 || c->occ_fused < 1) return bail(GK_ERR_UNSUPPORTED);
+    auto *ks = stream_kernel<kSingle, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>;
+    if (cudaFuncSetAttribute(ks, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SingleCfg::kSmemBytes) != cudaSuccess ||
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_single, ks, SingleCfg::kThreads, SingleCfg::kSmemBytes) != cudaSuccess)
+        return bail(GK_ERR_CUDA);
+    if (c->occ_verify < 1 || c->occ_pack < 1 || c->occ_commit < 1 || c->occ_fused < 1 || c->occ_single < 1)
+        return bail(GK_ERR_UNSUPPORTED);
 
     // tables: ones * x^(8*len(t)) for every page fill t, and the per-thread placement constants
     std::vector<uint64_t> init(gd.page_tokens + 1, 0);
@@ -961,6 +973,16 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
     P.n_items = n_pages * tlv.nseg_max;
     P.n_items_c = n_pages * tlc.nseg_max;
     if (c->gd.flags & GK_FLAG_SKIP_VERIFY) return launch_commit(c, P, st);
+    if (c->gd.flags & GK_FLAG_SINGLE_PASS) {
+        // one pass: every tile is checksummed and scattered from the same shared-memory stage;
+        // the codes are known only when the launch has ended, so a small kernel reports them
+        P.inline_final = 1u;
+        if ((rc = launch_single(c, P, st)) != GK_OK) return rc;
+        report_kernel<<<(w.n_jobs + 127) / 128, 128, 0, st>>>(w, mask_dev, first_bad_dev);
+        GK_CUDA(c, cudaGetLastError());
+        c->stats.kernels_launched++;
+        return GK_OK;
+    }
     // one job cannot overlap its own verify and commit (it is committed only after all of it has
     // verified); from about 256 MiB on the two dedicated kernels then beat the fused one by more
     // than their two extra launches cost (5,200 tokens of the GQA-7B shape: 386 us against 403 us)
@@ -990,8 +1012,10 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
 
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
-    const bool fused = c->fused && !(n_jobs == 1 && pages * c->gd.R >= (256ull << 20));
-    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages, fused ? c->occ_fused : c->occ_verify, fused && n_jobs > 1);
+    const bool single = (c->gd.flags & GK_FLAG_SINGLE_PASS) && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
+    const bool fused = !single && c->fused && !(n_jobs == 1 && pages * c->gd.R >= (256ull << 20));
+    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages, single ? c->occ_single : fused ? c->occ_fused : c->occ_verify,
+                                  fused && n_jobs > 1);
     const Tiling tlc = commit_tiling(c, pages, fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;

@@ -14,7 +14,7 @@ constexpr int32_t kNoPage = 0x7fffffff;
 // bounded device waits: by default give up after this many nanoseconds of %globaltimer
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
-enum Mode : int { kVerify = 0, kPack = 1, kCommit = 2 };
+enum Mode : int { kVerify = 0, kPack = 1, kCommit = 2, kSingle = 3 };
 
 struct GeomDev {
     uint32_t layers, kv_heads, page_tokens, scale_kv;

@@ -7,6 +7,9 @@
 //                       kVerify : blob -> smem -> CRC segment remainders
 //                       kPack   : cache slabs -> smem -> CRC + blob
 //                       kCommit : blob -> smem -> cache slabs (no CRC)
+//                       kSingle : blob -> smem -> CRC + cache slabs (single-pass restore:
+//                                 a block that fails only its checksum is reported, but
+//                                 its own pages have received the unverified bytes)
 //   restore_kernel<>  verify and commit pipelines side by side in one CTA; a job is
 //                     committed only after all of its pages have verified
 //   finalize_kernel   segment remainders -> page CRC-64/XZ; compare or write
@@ -341,7 +344,7 @@ __device__ __forceinline__ bool get_item(const StreamParams &P, const Tiling &tl
         if (code != 0u) return false;
     } else {
         if (jb.missing || P.w.bad_range[it.j] != kNoPage) return false;
-        if (MODE == kVerify && P.w.bad_dup[it.j] != kNoPage) return false;
+        if ((MODE == kVerify || MODE == kSingle) && P.w.bad_dup[it.j] != kNoPage) return false;
     }
     const PageShape sh = page_shape(P.g, jb, it.p, tl);
     it.nseg = sh.nseg;
@@ -740,7 +743,7 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling 
         const uint32_t sbase = ring.stage0 + s * STAGE_BYTES;
         const uint8_t *sgen = ring.base + (size_t)s * STAGE_BYTES;
         uint32_t scale_bytes = 0u;
-        if (MODE == kCommit && r0 < P.g.S && nreal > 0u) {
+        if ((MODE == kCommit || MODE == kSingle) && r0 < P.g.S && nreal > 0u) {
             const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
             scale_bytes = (uint32_t)(e1 - r0);
             if (!*abort_flag) {

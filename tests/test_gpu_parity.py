@@ -447,6 +447,42 @@ def test_job_array_marshalled_once_gives_the_same_result(gk):
     ctx.close()
 
 
+# ---------------------------------------------------------------------------
+# single-pass restore (GK_FLAG_SINGLE_PASS)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("og", ALL_GEOMS + [HM_MID, HM_FP8])
+@pytest.mark.parametrize("host_tier", [False, True])
+def test_single_pass_restore_parity(gk, og, host_tier):
+    """Same report as the two-phase restore; the pages of a block that fails only its checksum
+    hold the unverified bytes, everything else is byte-identical to the strict result."""
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
+    T = og.page_tokens
+    src = random_cache(og, 17, seed=350)
+    lens = [3 * T, 1, 2 * T + 1, 5 * T, T, 4 * T - 1, 2 * T]
+    Nd = 44
+    jobs = _oracle_jobs(og, src, lens, 351, Nd)
+    jobs[1].blob[len(jobs[1].blob) // 2] ^= 0x10           # checksum failure
+    jobs[3].checksums[2] ^= np.uint64(1 << 40)             # checksum failure (damaged checksum)
+    jobs[4] = oracle.Job(None, None, jobs[4].page_table, T)  # missing
+    jobs[5].page_table[1] = jobs[0].page_table[0]          # page claimed twice: jobs 0 and 5 write nothing
+    clean = random_cache(og, Nd, seed=352)
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs, flags=oracle.FLAG_SINGLE_PASS)
+    assert wmask.tolist() == [2, 1, 0, 1, 3, 2, 0]
+    strict = clone_cache(clean)
+    smask, sfb = oracle.restore(og, strict, jobs)
+    assert smask.tolist() == wmask.tolist() and sfb.tolist() == wfb.tolist()
+    assert not np.array_equal(strict.data, want.data)
+    for tuning in ({}, {"seg_granules": 1}, {"grid_cap": 3}):
+        ctx = _ctx(gk, og, flags=gk.GK_FLAG_SINGLE_PASS, **tuning)
+        d = dev_cache(clean)
+        mask, fb = gpu_restore(ctx, d, jobs, host_tier=host_tier)
+        assert mask.tolist() == wmask.tolist()
+        assert fb.tolist() == wfb.tolist()
+        assert_cache_equal(d, want)
+        ctx.close()
+
+
 def test_restore_codes_and_first_bad_page(gk):
     from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
     og, N = G_MID, 12
