@@ -59,7 +59,9 @@ def parse_args():
                          "its checksum receive the unverified bytes); prints the short line, never the headline")
     ap.add_argument("--blocks", type=int, default=0,
                     help="restore this many blocks instead of the workload's 16 (small cases for profiling)")
-    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the one-step-at-a-time end-to-end leg")
+    ap.add_argument("--e2e-pipelined-steps", type=int, default=10,
+                    help="steps of the pipelined end-to-end leg (save of step k+1 overlaps restore of step k)")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline-blocks", type=int, default=4)
@@ -504,10 +506,68 @@ def run_ours(args):
         save_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in e2e_events]))
         load_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in e2e_events]))
         link = batch_bytes + n_blocks * wl["P"] * 8
-        e2e = {"value": world * 4 * batch_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT,
+
+        # ---- the same steps pipelined: a second context restores step k on its own stream while the
+        # first saves step k+1 (two sets of pinned buffers), so that both directions of the host link
+        # are busy at once.  Every step still copies its whole batch out and in and reads its results.
+        keep2, host_pack2, host_restore2 = [], [], []
+        for pj, rj in zip(wl["pack_jobs"], wl["restore_jobs"]):
+            hb = torch.empty(blob_bytes, dtype=torch.uint8, pin_memory=True)
+            hs = torch.empty(wl["P"], dtype=torch.int64, pin_memory=True)
+            keep2.append((hb, hs))
+            host_pack2.append(gk.Job(hb, hs, pj.page_table, n_tok, pj.request_id))
+            host_restore2.append(gk.Job(hb, hs, rj.page_table, n_tok, rj.request_id))
+        sets = [(host_pack, host_restore), (host_pack2, host_restore2)]
+        ctx_r = gk.Context(wl["geom"], device.index)
+        s_save, s_rest = torch.cuda.Stream(device), torch.cuda.Stream(device)
+        status2 = torch.zeros_like(status)
+
+        def pipelined(n_steps):
+            saved = [torch.cuda.Event() for _ in range(n_steps)]
+            restored = [torch.cuda.Event() for _ in range(n_steps)]
+            b0, b1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            b0.record(stream)
+            s_save.wait_event(b0)
+            s_rest.wait_event(b0)
+            for k in range(n_steps):
+                hp, hr = sets[k % 2]
+                with torch.cuda.stream(s_save):
+                    if k >= 2:
+                        s_save.wait_event(restored[k - 2])      # this buffer set has been read back in
+                    ctx.gk_pack_host(wl["src"], hp, status2, stream=s_save)
+                    status_h.copy_(status2, non_blocking=True)
+                    saved[k].record(s_save)
+                with torch.cuda.stream(s_rest):
+                    s_rest.wait_event(saved[k])
+                    ctx_r.gk_restore_host(hr, wl["dst"], mask, first_bad, stream=s_rest)
+                    mask_h.copy_(mask, non_blocking=True)
+                    fb_h.copy_(first_bad, non_blocking=True)
+                    restored[k].record(s_rest)
+            stream.wait_stream(s_save)
+            stream.wait_stream(s_rest)
+            b1.record(stream)
+            return b0, b1
+
+        pipelined(2)
+        torch.cuda.synchronize(device)
+        barrier()
+        b0, b1 = pipelined(args.e2e_pipelined_steps)
+        barrier()
+        pipe_ms = max_over_ranks(b0.elapsed_time(b1) / max(args.e2e_pipelined_steps, 1))
+        assert int(mask_h.sum().item()) == 0 and int(status_h.sum().item()) == 0
+        for i in range(min(4, n_blocks)):
+            assert torch.equal(keep2[i][1], wl["pack_jobs"][i].checksums.cpu())
+        assert ctx_r.gk_get_stats()["device_wait_expired"] == 0
+        ctx_r.close()
+        del keep2, host_pack2, host_restore2, sets
+        e2e = {"value": world * 4 * batch_bytes / (pipe_ms * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": link + 2 * n_blocks * 40, "d2h_bytes_per_step": link + n_blocks * 6,
-               "ms_per_step": e2e_ms, "steps": args.e2e_steps,
-               "tokens_per_s": world * n_blocks * n_tok / (e2e_ms * 1e-3),
+               "ms_per_step": pipe_ms, "steps": args.e2e_pipelined_steps,
+               "tokens_per_s": world * n_blocks * n_tok / (pipe_ms * 1e-3),
+               "pipelining": "save of step k+1 (context 1, stream 1) overlaps restore of step k (context 2, stream 2); "
+                             "two sets of pinned buffers; both directions of the host link in use at once",
+               "one_step_at_a_time": {"value": world * 4 * batch_bytes / (e2e_ms * 1e-3) / 1e9,
+                                      "ms_per_step": e2e_ms, "steps": args.e2e_steps},
                "save": {"ms": save_ms, "host_link_gbs": link / (save_ms * 1e-3) / 1e9,
                         "frac_of_plain_d2h_copy": link / (save_ms * 1e-3) / 1e9 / link_rate["d2h"]},
                "restore": {"ms": load_ms, "host_link_gbs": link / (load_ms * 1e-3) / 1e9,

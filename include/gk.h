@@ -226,7 +226,9 @@ int gk_commit(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *
  * and committed on `stream`; the checksum is taken over the bytes as they arrived
  * in device memory.  All page tables are validated before the first copy.  The
  * call returns after the last stage has been enqueued; results are valid after
- * `stream` has been synchronised.  The host buffers must stay valid until then. */
+ * `stream` has been synchronised.  The host buffers must stay valid until then.
+ * The first copy starts only when the work already enqueued on `stream` has
+ * finished, so the host buffers may be filled by earlier work on that stream. */
 int gk_restore_host(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
                     uint8_t *mask_dev, int32_t *first_bad_page_dev, void *stream);
 

@@ -118,6 +118,7 @@ struct gk_ctx {
     uint8_t *h_stage = nullptr;
     size_t h_stage_cap = 0;
     cudaEvent_t ev_stage = nullptr;  // upload of the job table has been consumed
+    cudaEvent_t ev_entry = nullptr;  // host tier: where the caller's stream stood when the call came in
 
     // host tier
     cudaStream_t copy_stream = nullptr;
@@ -816,6 +817,7 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
         cudaMemset(c->d_error, 0, 256) != cudaSuccess)
         return bail(GK_ERR_CUDA);
     if (cudaEventCreateWithFlags(&c->ev_stage, cudaEventDisableTiming) != cudaSuccess) return bail(GK_ERR_CUDA);
+    if (cudaEventCreateWithFlags(&c->ev_entry, cudaEventDisableTiming) != cudaSuccess) return bail(GK_ERR_CUDA);
     for (int i = 0; i < kSlots; ++i) {
         if (cudaEventCreateWithFlags(&c->ev_slot_free[i], cudaEventDisableTiming) != cudaSuccess ||
             cudaEventCreateWithFlags(&c->ev_copied[i], cudaEventDisableTiming) != cudaSuccess)
@@ -842,6 +844,7 @@ int gk_ctx_destroy(gk_ctx *c)
         if (c->ev_copied[i]) cudaEventDestroy(c->ev_copied[i]);
     }
     if (c->ev_stage) cudaEventDestroy(c->ev_stage);
+    if (c->ev_entry) cudaEventDestroy(c->ev_entry);
     if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->d_ws) cudaFree(c->d_ws);
     if (c->d_iota) cudaFree(c->d_iota);
@@ -1122,8 +1125,12 @@ int gk_commit(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *ds
     return GK_OK;
 }
 
-int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, uint8_t *mask_dev,
-                    int32_t *first_bad_page_dev, void *stream)
+// order_after_stream: the host buffers may still be being written by earlier work on the
+// caller's stream, so the first copy must wait for that work.  The streaming restore passes
+// false for every window but the first: its buffers were ready when the call came in, and the
+// copies of a window are meant to run under the consumer of the window before it.
+static int restore_host_impl(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, uint8_t *mask_dev,
+                             int32_t *first_bad_page_dev, void *stream, bool order_after_stream)
 {
     if (!c) return GK_ERR_ARG;
     if (n_jobs == 0) return GK_OK;
@@ -1133,6 +1140,10 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
     CacheDev cd;
     int rc = check_cache(c, dst, &cd);
     if (rc != GK_OK) return rc;
+    if (order_after_stream) {
+        GK_CUDA(c, cudaEventRecord(c->ev_entry, st));
+        GK_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_entry, 0));
+    }
 
     HostPlan hp;
     if ((rc = make_host_plan(c, jobs, n_jobs, true, hp)) != GK_OK) return rc;
@@ -1187,6 +1198,12 @@ int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cac
     return GK_OK;
 }
 
+int gk_restore_host(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst, uint8_t *mask_dev,
+                    int32_t *first_bad_page_dev, void *stream)
+{
+    return restore_host_impl(c, jobs, n_jobs, dst, mask_dev, first_bad_page_dev, stream, true);
+}
+
 int gk_restore_stream(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *ring, uint8_t *mask_dev,
                       int32_t *first_bad_page_dev, gk_window_fn consume, void *user, void *stream)
 {
@@ -1237,7 +1254,7 @@ int gk_restore_stream(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_c
             used += np[j1];
             ++j1;
         }
-        rc = gk_restore_host(c, wjobs.data(), j1 - j0, ring, mask_dev + j0, first_bad_page_dev + j0, stream);
+        rc = restore_host_impl(c, wjobs.data(), j1 - j0, ring, mask_dev + j0, first_bad_page_dev + j0, stream, j0 == 0);
         if (rc != GK_OK) return rc;
         if (consume) consume(user, blocks.data(), j1 - j0, mask_dev, stream);
         j0 = j1;

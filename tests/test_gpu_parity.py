@@ -483,6 +483,40 @@ def test_single_pass_restore_parity(gk, og, host_tier):
         ctx.close()
 
 
+def test_restore_host_is_ordered_after_earlier_work_on_the_stream(gk):
+    """The pinned blob is still being filled by an asynchronous copy on the caller's stream
+    when gk_restore_host is called: its copies must wait for that work."""
+    from gpu_harness import assert_cache_equal, dev_cache, dev_i32
+    og = G_BIG                                             # 1 MiB records
+    T = og.page_tokens
+    n = 96 * T                                             # a 96 MiB blob: the fill takes milliseconds
+    src = random_cache(og, 96, seed=360)
+    spt = np.random.default_rng(361).permutation(96).astype(np.int32)
+    blob, sums, code, _ = oracle.pack(og, src, spt, n)
+    assert code == 0
+    dpt = np.random.default_rng(362).permutation(100).astype(np.int32)[:96]
+    clean = random_cache(og, 100, seed=363)
+    want = clone_cache(clean)
+    wmask, _ = oracle.restore(og, want, [oracle.Job(blob, sums, dpt, n)])
+    assert wmask.tolist() == [0]
+    ctx = _ctx(gk, og)
+    d = dev_cache(clean)
+    d_blob = torch.from_numpy(blob).cuda()
+    d_sums = torch.from_numpy(sums.view(np.int64).copy()).cuda()
+    h_blob = torch.zeros(blob.size, dtype=torch.uint8).pin_memory()        # zeros: a premature copy fails its checksums
+    h_sums = torch.zeros(sums.size, dtype=torch.int64).pin_memory()
+    mask = torch.full((1,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.full((1,), -7, dtype=torch.int32, device="cuda")
+    torch.cuda.synchronize()
+    h_blob.copy_(d_blob, non_blocking=True)                # device -> pinned host, on the current stream
+    h_sums.copy_(d_sums, non_blocking=True)
+    ctx.gk_restore_host([gk.Job(h_blob, h_sums, dev_i32(dpt), n)], d, mask, fb)
+    torch.cuda.synchronize()
+    assert mask.cpu().tolist() == [0]
+    assert_cache_equal(d, want)
+    ctx.close()
+
+
 def test_restore_codes_and_first_bad_page(gk):
     from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
     og, N = G_MID, 12
