@@ -1,0 +1,97 @@
+"""Seeded random cases on the GPU against the oracle: random geometries (both dtypes, both
+slab layouts), block lengths, page tables, kinds of damage, flags, tunings and tiers.  Every
+case compares the blob, the checksums, the codes, the first bad pages and the full
+destination image."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from helpers import clone_cache, n_pages, random_cache
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def gk():
+    import paper_2609_39358_b200 as m
+    assert torch.cuda.is_available()
+    return m
+
+
+def _random_geom(rng):
+    fp8 = bool(rng.integers(0, 2))
+    head_major = int(rng.integers(0, 2))
+    elem = 1 if fp8 else 2
+    while True:
+        layers = int(rng.integers(1, 7))
+        heads = int(rng.choice([1, 2, 3, 4, 8]))
+        dim = int(rng.choice([16, 32, 64, 128]))
+        T = int(rng.choice([1, 2, 4, 8, 16, 32]))
+        scale_kv = int(rng.integers(1, 3)) if fp8 else 0
+        row = heads * dim * elem
+        S = layers * scale_kv * heads * 4
+        if row % 16 or S % 16:
+            continue
+        return oracle.Geom(layers, heads, dim, T, elem, scale_kv, head_major)
+
+
+@pytest.mark.parametrize("case", range(128))
+def test_random_case(gk, case):
+    from gpu_harness import assert_cache_equal, dev_cache, gk_geom, gpu_pack, gpu_restore
+    rng = np.random.default_rng(9000 + case)
+    og = _random_geom(rng)
+    T = og.page_tokens
+    n_jobs = int(rng.integers(1, 9))
+    lens = [int(rng.integers(1, 6 * T + 1)) for _ in range(n_jobs)]
+    Ns = int(rng.integers(4, 24))
+    src = random_cache(og, Ns, seed=9100 + case, layout=str(rng.choice(["layer_major", "page_major"])))
+    tables = [rng.integers(0, Ns, size=n_pages(og, n)).astype(np.int32) for n in lens]
+    single = bool(rng.integers(0, 2))
+    flags = gk.GK_FLAG_SINGLE_PASS if single else 0
+    tuning = [{}, {"seg_granules": 1}, {"seg_granules": 2, "commit_seg_tiles": 1}, {"grid_cap": int(rng.integers(1, 9))},
+              {"fused": 0}][int(rng.integers(0, 5))]
+    ctx = gk.Context(gk_geom(og, flags), 0)
+    for k, v in tuning.items():
+        ctx.set_tuning(k, v)
+
+    # save: every blob and checksum against the oracle
+    got, status = gpu_pack(ctx, og, dev_cache(src), tables, lens)
+    assert status.tolist() == [0] * n_jobs
+    ojobs = []
+    total = sum(n_pages(og, n) for n in lens)
+    Nd = total + int(rng.integers(0, 6))
+    perm = rng.permutation(Nd).astype(np.int32)
+    used = 0
+    for (blob, sums), pt, n in zip(got, tables, lens):
+        wb, ws, code, _ = oracle.pack(og, src, pt, n)
+        assert code == 0 and np.array_equal(blob, wb) and np.array_equal(sums, ws)
+        P = n_pages(og, n)
+        ojobs.append(oracle.Job(wb.copy(), ws.copy(), perm[used:used + P].copy(), n))
+        used += P
+
+    # damage: each job independently gets nothing, bit flips, a damaged checksum, a missing record,
+    # an out-of-range id, or a page shared with another job
+    for j, jb in enumerate(ojobs):
+        kind = int(rng.integers(0, 8))
+        if kind == 1:
+            for _ in range(int(rng.integers(1, 5))):
+                jb.blob[int(rng.integers(0, jb.blob.size))] ^= np.uint8(1 << int(rng.integers(0, 8)))
+        elif kind == 2:
+            jb.checksums[int(rng.integers(0, jb.checksums.size))] ^= np.uint64(1) << np.uint64(int(rng.integers(0, 64)))
+        elif kind == 3:
+            ojobs[j] = oracle.Job(None, None, jb.page_table, jb.n_tokens)
+        elif kind == 4:
+            jb.page_table[int(rng.integers(0, jb.page_table.size))] = Nd + int(rng.integers(0, 3)) if rng.random() < 0.5 else -1
+        elif kind == 5 and n_jobs > 1:
+            other = ojobs[(j + 1) % n_jobs]
+            jb.page_table[0] = other.page_table[0]
+    clean = random_cache(og, Nd, seed=9200 + case, layout=str(rng.choice(["layer_major", "page_major"])))
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, ojobs, flags=oracle.FLAG_SINGLE_PASS if single else 0)
+    d = dev_cache(clean)
+    mask, fb = gpu_restore(ctx, d, ojobs, host_tier=bool(rng.integers(0, 2)))
+    assert mask.tolist() == wmask.tolist(), (og, lens, tuning, single)
+    assert fb.tolist() == wfb.tolist()
+    assert_cache_equal(d, want)
+    ctx.close()
