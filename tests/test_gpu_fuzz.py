@@ -95,3 +95,52 @@ def test_random_case(gk, case):
     assert fb.tolist() == wfb.tolist()
     assert_cache_equal(d, want)
     ctx.close()
+
+
+@pytest.mark.parametrize("case", range(32))
+def test_random_stream_restore_case(gk, case):
+    """Random corpora through random rings: windows, ring image after every window, codes."""
+    from gpu_harness import dev_cache, gk_geom
+    rng = np.random.default_rng(9500 + case)
+    og = _random_geom(rng)
+    T = og.page_tokens
+    n_jobs = int(rng.integers(1, 12))
+    lens = [int(rng.integers(1, 5 * T + 1)) for _ in range(n_jobs)]
+    src = random_cache(og, 9, seed=9600 + case)
+    ojobs = []
+    for n in lens:
+        blob, sums, code, _ = oracle.pack(og, src, rng.integers(0, 9, size=n_pages(og, n)).astype(np.int32), n)
+        assert code == 0
+        kind = int(rng.integers(0, 6))
+        if kind == 1:
+            blob[int(rng.integers(0, blob.size))] ^= np.uint8(1 << int(rng.integers(0, 8)))
+        if kind == 2:
+            ojobs.append(oracle.Job(None, None, None, n))
+        else:
+            ojobs.append(oracle.Job(blob, sums, None, n))
+    ring_pages = max(n_pages(og, n) for n in lens) + int(rng.integers(0, 8))
+    single = bool(rng.integers(0, 2))
+    clean = random_cache(og, ring_pages, seed=9700 + case)
+    want = clone_cache(clean)
+    owin = []
+    wmask, wfb = oracle.restore_stream(og, want, ojobs,
+                                       lambda first, count, pages: owin.append((first, count, want.data.copy())),
+                                       flags=oracle.FLAG_SINGLE_PASS if single else 0)
+    ctx = gk.Context(gk_geom(og, gk.GK_FLAG_SINGLE_PASS if single else 0), 0)
+    d = dev_cache(clean)
+    jobs, keep = [], []
+    for jb in ojobs:
+        hb = None if jb.blob is None else torch.from_numpy(jb.blob).pin_memory()
+        hs = None if jb.checksums is None else torch.from_numpy(jb.checksums.view(np.int64).copy()).pin_memory()
+        keep.append((hb, hs))
+        jobs.append(gk.Job(hb, hs, None, jb.n_tokens))
+    mask = torch.full((n_jobs,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.full((n_jobs,), -7, dtype=torch.int32, device="cuda")
+    gwin = []
+    ctx.gk_restore_stream(jobs, d, mask, fb, lambda blocks, st: gwin.append((blocks[0].job, len(blocks), d.data.clone())))
+    torch.cuda.synchronize()
+    assert mask.cpu().tolist() == wmask.tolist() and fb.cpu().tolist() == wfb.tolist()
+    assert [(a, b) for a, b, _ in gwin] == [(a, b) for a, b, _ in owin]
+    for (_, _, gimg), (_, _, oimg) in zip(gwin, owin):
+        assert np.array_equal(gimg.cpu().numpy(), oimg)
+    ctx.close()
