@@ -5,11 +5,12 @@
  * The operations are those of the paper's KV memory (Section 2.2, "Taliesin: KV
  * memory"): after the runtime has computed the KV state of a block of prompt
  * text the state is written out; when the same block recurs it is loaded
- * instead of recomputed; what was stored is checked when it is loaded; and by
- * that section's design rule -- a request may be served without stored state but
- * never with wrong stored state -- a record that is missing, damaged or fails
- * a check is not used at all: the block is reported for recompute.  Restored state must be bit-identical to what was saved (Section 3,
- * Table 1), reuse is per whole block (Section 5, first item) and the design is
+ * instead of recomputed; what was stored is checked when it is loaded; and that
+ * section's design rule puts correctness before reuse -- a request can always do
+ * without stored state, but wrong stored state must never reach it -- so a record
+ * that is absent, damaged or fails a check is not used at all: the block is
+ * reported for recompute.  Restored state must be bit-identical to what was saved
+ * (Section 3, Table 1), reuse is per whole block (Section 5, first item) and the design is
  * fail-closed (Section 5, second item).  The paper does not disclose its record
  * format (end of Section 1); the format below is this library's own.
  *
@@ -264,10 +265,11 @@ int gk_restore_stream(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk
                       uint8_t *mask_dev, int32_t *first_bad_page_dev, gk_window_fn consume, void *user,
                       void *stream);
 
-/* Block fingerprints (Section 2.2: a block's state is filed under a fingerprint of
- * the exact input bytes, the model and the tenant; Section 2.1: state of one model
- * or tenant must not load under another; Section 2.2 and Section 5: a block is
- * reused only where its token positions match).  The paper gives no format; this
+/* Block fingerprints (Section 2.2: the lookup key of a block's state is derived
+ * from the block's input, byte for byte, and from the identities of model and
+ * tenant; Section 2.1: records of one model or tenant stay out of another's reach;
+ * Section 2.2 and Section 5: a block is reused only at identical token positions).
+ * The paper gives no format; this
  * library's keys are, with SHA-256 (FIPS 180-4), || for concatenation and
  * little-endian integers,
  *     inner_i = SHA-256( bytes_i || model[32] || tenant[32] || u64(len_i) || "GKF1" )
@@ -284,8 +286,8 @@ int gk_fingerprints(gk_ctx *ctx, const void *data_dev, const uint64_t *offsets_d
                     uint32_t n, const uint8_t *model, const uint8_t *tenant, uint8_t *keys_dev, void *stream);
 
 /* Confirmation hash of stored blocks (Section 3, sabotage-testing paragraph, lists
- * a confirmation hash among the safety mechanisms; Section 7: loaded state is
- * judged by byte comparison and cryptographic hashes).  A three-level SHA-256 tree
+ * a confirmation hash among the safety mechanisms; Section 7 names hashes, besides
+ * comparing bytes, as the judge of loaded state).  A three-level SHA-256 tree
  * over each blob, bound to the key the block is filed under:
  *     leaf   = SHA-256( chunk || "GKL0" )      chunk = 4096 record bytes, the last may be shorter
  *     page_p = SHA-256( leaf_0 || ... || leaf_{m-1} || u64(record bytes) || "GKP0" )

@@ -4,14 +4,15 @@
  * TEST INFRASTRUCTURE ONLY, like gk_oracle.h: the plain definition that the CUDA
  * library is compared against; no code, table or constant is shared with it.
  *
- * What it follows.  The paper stores the KV state of a block under a
- * fingerprint of the exact input bytes, the model and the tenant (Section 2.2),
- * refuses to run without a tenant identity and a model fingerprint so that one
- * model's or tenant's state cannot be loaded by another (Section 2.1), reuses a
- * block only where token positions match exactly (Section 2.2, Section 5), and
+ * What it follows.  In the paper the lookup key of a block's stored KV state is
+ * derived from three things: the block's input, byte for byte, the identity of
+ * the model, and the identity of the tenant (Section 2.2); the library will not
+ * run without the latter two, which keeps one model's or tenant's records out of
+ * another's reach (Section 2.1); a block is reused only at identical token
+ * positions (Section 2.2, Section 5); and the paper
  * lists a confirmation hash among its safety mechanisms (Section 3, sabotage
- * testing); Section 7 says that loaded state is judged by byte comparison and
- * cryptographic hashes.  The paper gives no formats, so the messages below are
+ * testing); Section 7 names hashes, besides comparing bytes, as the judge of
+ * whether loaded state is right.  The paper gives no formats, so the messages below are
  * this build's own; the hash is SHA-256 as FIPS 180-4 defines it.
  *
  * Definitions (|| is concatenation, integers little-endian)
