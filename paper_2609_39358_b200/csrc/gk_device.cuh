@@ -119,7 +119,7 @@ __host__ __device__ inline uint64_t gf_mul(uint64_t a, uint64_t b)
     return r;
 }
 
-// ---- PTX wrappers: mbarrier, bulk async copies (no multicast anywhere) ----
+// ---- PTX wrappers: mbarrier, bulk async copies (every copy has one destination CTA) ----
 __device__ __forceinline__ uint32_t smem_u32(const void *p)
 {
     return (uint32_t)__cvta_generic_to_shared(p);
