@@ -10,7 +10,7 @@ _CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libgk.so")
 
 _SOURCES = ["gk_api.cu"]
-_DEPS = ["gk_api.cu", "gk_kernels.cuh", "gk_device.cuh", "gk_gf2_generated.inc", "gen_tables.py",
+_DEPS = ["gk_api.cu", "gk_kernels.cuh", "gk_device.cuh", "gk_sha256.cuh", "gk_gf2_generated.inc", "gen_tables.py",
          os.path.join("..", "..", "include", "gk.h")]
 
 
