@@ -133,19 +133,30 @@ __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant_
     }
     for (uint32_t k = threadIdx.x; k < pp.n_seg_pow; k += blockDim.x) pow_out[k] = pp.seg_pow[k];
     __syncthreads();
+    // Both passes run over the pages of the whole call at once (a thread finds the job of its
+    // page by bisection), so that the loads of all page tables are in flight together.
+    const uint32_t total_pages = pp.jobs[w.n_jobs - 1u].page_base + pp.jobs[w.n_jobs - 1u].n_pages;
+    auto job_of = [&](uint32_t gp) {
+        uint32_t lo = 0, hi = w.n_jobs - 1u;
+        while (lo < hi) {
+            const uint32_t mid = (lo + hi + 1u) >> 1;
+            if (pp.jobs[mid].page_base <= gp) lo = mid; else hi = mid - 1u;
+        }
+        return lo;
+    };
     // pass 1: page -> job map, range check, clear the claim words that will be used
-    for (uint32_t j = 0; j < w.n_jobs; ++j) {
+    for (uint32_t gp = threadIdx.x; gp < total_pages; gp += blockDim.x) {
+        const uint32_t j = job_of(gp);
         const JobDev &jb = pp.jobs[j];
-        for (uint32_t p = threadIdx.x; p < jb.n_pages; p += blockDim.x) {
-            w.page_job[jb.page_base + p] = (int32_t)j;
-            w.page_cnt[jb.page_base + p] = 0u;
-            if (jb.page_table) {
-                const int32_t id = jb.page_table[p];
-                if (id < 0 || (uint64_t)id >= pp.num_pages)
-                    atomicMin(&w.bad_range[j], (int32_t)p);
-                else if (pp.do_claims)
-                    w.claims[id] = 0ull;
-            }
+        const uint32_t p = gp - jb.page_base;
+        w.page_job[gp] = (int32_t)j;
+        w.page_cnt[gp] = 0u;
+        if (jb.page_table) {
+            const int32_t id = jb.page_table[p];
+            if (id < 0 || (uint64_t)id >= pp.num_pages)
+                atomicMin(&w.bad_range[j], (int32_t)p);
+            else if (pp.do_claims)
+                w.claims[id] = 0ull;
         }
     }
     if (pp.status_out) {
@@ -156,17 +167,17 @@ __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant_
     if (!pp.do_claims) return;
     __syncthreads();
     // pass 2: claims, as in claim_kernel
-    for (uint32_t j = 0; j < w.n_jobs; ++j) {
+    for (uint32_t gp = threadIdx.x; gp < total_pages; gp += blockDim.x) {
+        const uint32_t j = job_of(gp);
         const JobDev &jb = pp.jobs[j];
         if (jb.missing || __ldcg(&w.bad_range[j]) != kNoPage) continue;
-        for (uint32_t p = threadIdx.x; p < jb.n_pages; p += blockDim.x) {
-            const int32_t id = jb.page_table[p];
-            const unsigned long long mine = ((unsigned long long)(j + 1u) << 32) | p;
-            const unsigned long long old = atomicCAS(&w.claims[id], 0ull, mine);
-            if (old != 0ull) {
-                atomicMin(&w.bad_dup[j], (int32_t)p);
-                atomicMin(&w.bad_dup[(uint32_t)(old >> 32) - 1u], (int32_t)(old & 0xffffffffull));
-            }
+        const uint32_t p = gp - jb.page_base;
+        const int32_t id = jb.page_table[p];
+        const unsigned long long mine = ((unsigned long long)(j + 1u) << 32) | p;
+        const unsigned long long old = atomicCAS(&w.claims[id], 0ull, mine);
+        if (old != 0ull) {
+            atomicMin(&w.bad_dup[j], (int32_t)p);
+            atomicMin(&w.bad_dup[(uint32_t)(old >> 32) - 1u], (int32_t)(old & 0xffffffffull));
         }
     }
 }
