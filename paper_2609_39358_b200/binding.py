@@ -259,6 +259,13 @@ class Context:
             raise GkError(rc, "gk_ctx_create")
         self._h = h
 
+    def __enter__(self):
+        return self
+
+    def __exit__(self, *exc):
+        self.close()
+        return False
+
     def close(self):
         if getattr(self, "_h", None):
             self._lib.gk_ctx_destroy(self._h)
