@@ -9,7 +9,12 @@ import torch
 import oracle
 from helpers import clone_cache, n_pages, random_cache
 
+import os
+
 pytestmark = pytest.mark.gpu
+
+# more cases for a soak run: GK_FUZZ_CASES=3000 python -m pytest tests/test_gpu_fuzz.py -m gpu
+N_CASES = int(os.environ.get("GK_FUZZ_CASES", "128"))
 
 
 @pytest.fixture(scope="module")
@@ -36,7 +41,7 @@ def _random_geom(rng):
         return oracle.Geom(layers, heads, dim, T, elem, scale_kv, head_major)
 
 
-@pytest.mark.parametrize("case", range(128))
+@pytest.mark.parametrize("case", range(N_CASES))
 def test_random_case(gk, case):
     from gpu_harness import assert_cache_equal, dev_cache, gk_geom, gpu_pack, gpu_restore
     rng = np.random.default_rng(9000 + case)
@@ -97,7 +102,7 @@ def test_random_case(gk, case):
     ctx.close()
 
 
-@pytest.mark.parametrize("case", range(32))
+@pytest.mark.parametrize("case", range(max(N_CASES // 4, 1)))
 def test_random_stream_restore_case(gk, case):
     """Random corpora through random rings: windows, ring image after every window, codes."""
     from gpu_harness import dev_cache, gk_geom
