@@ -149,3 +149,49 @@ def test_random_stream_restore_case(gk, case):
     for (_, _, gimg), (_, _, oimg) in zip(gwin, owin):
         assert np.array_equal(gimg.cpu().numpy(), oimg)
     ctx.close()
+
+
+@pytest.mark.parametrize("case", range(12))
+def test_random_medium_case(gk, case):
+    """Records of 0.25 to 3 MiB and up to a few hundred pages per call: adaptive segment
+    tiling, many CTAs drawing items at once, jobs finishing out of order."""
+    from gpu_harness import assert_cache_equal, dev_cache, gk_geom, gpu_pack, gpu_restore
+    rng = np.random.default_rng(9800 + case)
+    fp8 = bool(rng.integers(0, 2))
+    og = oracle.Geom(int(rng.choice([8, 16, 24, 48])), int(rng.choice([4, 8])), 128, int(rng.choice([16, 32])),
+                     1 if fp8 else 2, 2 if fp8 else 0, int(rng.integers(0, 2)))
+    T = og.page_tokens
+    rec = oracle.record_bytes(og, T, 0)
+    budget_pages = max(int(160e6 // rec), 8)
+    n_jobs = int(rng.integers(1, 10))
+    lens = []
+    for _ in range(n_jobs):
+        lens.append(int(rng.integers(1, max(2, budget_pages // n_jobs) * T + 1)))
+    Ns = 12
+    src = random_cache(og, Ns, seed=9900 + case)
+    tables = [rng.integers(0, Ns, size=n_pages(og, n)).astype(np.int32) for n in lens]
+    single = bool(rng.integers(0, 2))
+    ctx = gk.Context(gk_geom(og, gk.GK_FLAG_SINGLE_PASS if single else 0), 0)
+    got, status = gpu_pack(ctx, og, dev_cache(src), tables, lens)
+    assert status.tolist() == [0] * n_jobs
+    total = sum(n_pages(og, n) for n in lens)
+    Nd = total + 3
+    perm = rng.permutation(Nd).astype(np.int32)
+    ojobs, used = [], 0
+    for (blob, sums), pt, n in zip(got, tables, lens):
+        wb, ws, code, _ = oracle.pack(og, src, pt, n)
+        assert code == 0 and np.array_equal(blob, wb) and np.array_equal(sums, ws)
+        P = n_pages(og, n)
+        ojobs.append(oracle.Job(wb.copy(), ws.copy(), perm[used:used + P].copy(), n))
+        used += P
+    for jb in ojobs:
+        if rng.random() < 0.3:
+            jb.blob[int(rng.integers(0, jb.blob.size))] ^= np.uint8(1 << int(rng.integers(0, 8)))
+    clean = random_cache(og, Nd, seed=9950 + case)
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, ojobs, flags=oracle.FLAG_SINGLE_PASS if single else 0)
+    d = dev_cache(clean)
+    mask, fb = gpu_restore(ctx, d, ojobs, host_tier=bool(rng.integers(0, 2)))
+    assert mask.tolist() == wmask.tolist() and fb.tolist() == wfb.tolist()
+    assert_cache_equal(d, want)
+    ctx.close()
