@@ -101,7 +101,8 @@ struct gk_ctx {
     int occ_verify = 0, occ_pack = 0, occ_commit = 0, occ_fused = 0, occ_single = 0;
     bool fused = true;           // restore runs verify and commit in one launch
     unsigned long long wait_limit_ns = kWaitLimitNs;
-    uint32_t ctr_next[2] = {0, 0};  // what the device work counters will read when the next launch starts
+    uint32_t ctr_next[2] = {0, 0};  // what the device work counters will read when the next launch of
+                                    // the current call starts (the first kernel of a call zeroes them)
     bool test_drop_verify = false;  // test hook: see gk_ctx_set_tuning
     uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
     uint32_t commit_seg_tiles = 0;
@@ -486,6 +487,7 @@ int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tili
     pp.do_claims = do_claims ? 1u : 0u;
     pp.num_pages = num_pages;
     pp.status_out = status_out;
+    c->ctr_next[0] = c->ctr_next[1] = 0;  // the kernel zeroes the device counters
     prep_small_kernel<<<1, 1024, 0, st>>>(pp, w);
     GK_CUDA(c, cudaGetLastError());
     c->stats.kernels_launched++;
@@ -616,6 +618,7 @@ int launch_validate(gk_ctx *c, const WorkDev &w, uint64_t num_pages, int clear_c
         if (g2 > 2048) g2 = 2048;
         if (g2 > grid) grid = g2;
     }
+    c->ctr_next[0] = c->ctr_next[1] = 0;  // the kernel zeroes the device counters
     validate_kernel<<<grid, 256, 0, st>>>(w, num_pages, clear_claims, status_out);
     GK_CUDA(c, cudaGetLastError());
     c->stats.kernels_launched++;

@@ -52,6 +52,11 @@ __global__ void iota_kernel(int32_t *ids, uint32_t n)
 __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims, uint8_t *status_out)
 {
     const uint32_t j = blockIdx.x;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        // every call draws its work items from zero (the host counts the draws of its launches)
+        w.work_ctr[0] = 0u;
+        w.work_ctr[1] = 0u;
+    }
     if (clear_claims) {
         for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < num_pages;
              i += (uint64_t)gridDim.x * blockDim.x)
@@ -132,6 +137,10 @@ __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant_
         w.job_done[j] = 0u;
     }
     for (uint32_t k = threadIdx.x; k < pp.n_seg_pow; k += blockDim.x) pow_out[k] = pp.seg_pow[k];
+    if (threadIdx.x == 0) {
+        w.work_ctr[0] = 0u;  // every call draws its work items from zero
+        w.work_ctr[1] = 0u;
+    }
     __syncthreads();
     // Both passes run over the pages of the whole call at once (a thread finds the job of its
     // page by bisection), so that the loads of all page tables are in flight together.

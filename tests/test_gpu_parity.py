@@ -517,6 +517,74 @@ def test_restore_host_is_ordered_after_earlier_work_on_the_stream(gk):
     ctx.close()
 
 
+def test_small_calls_replay_from_a_cuda_graph(gk):
+    """A small save + restore captured once and replayed: every replay does the real work
+    (the work-item counters start from zero in every call), so damage done to the source
+    cache or to a blob between replays shows up exactly as in a direct call."""
+    from gpu_harness import dev_cache, dev_i32
+    og = G_MID
+    T = og.page_tokens
+    lens = [2 * T + 3, T, 3 * T]
+    src = random_cache(og, 9, seed=370)
+    rng = np.random.default_rng(371)
+    tables = [rng.integers(0, 9, size=n_pages(og, n)).astype(np.int32) for n in lens]
+    Nd = 12
+    dperm = rng.permutation(Nd).astype(np.int32)
+    clean = random_cache(og, Nd, seed=372)
+    ctx = _ctx(gk, og)
+    dsrc, ddst = dev_cache(src), dev_cache(clean)
+    pack_jobs, restore_jobs, used = [], [], 0
+    for pt, n in zip(tables, lens):
+        nbytes, P = oracle.blob_size(og, n)
+        blob = torch.zeros(nbytes, dtype=torch.uint8, device="cuda")
+        sums = torch.zeros(P, dtype=torch.int64, device="cuda")
+        pack_jobs.append(gk.Job(blob, sums, dev_i32(pt), n))
+        restore_jobs.append(gk.Job(blob, sums, dev_i32(dperm[used:used + P]), n))
+        used += P
+    pack_jobs, restore_jobs = gk.JobArray(pack_jobs), gk.JobArray(restore_jobs)
+    status = torch.full((3,), 255, dtype=torch.uint8, device="cuda")
+    mask = torch.full((3,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.full((3,), -7, dtype=torch.int32, device="cuda")
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):                       # warm-up outside the capture: workspace allocation
+        ctx.gk_pack_batch(dsrc, pack_jobs, status)
+        ctx.gk_restore(restore_jobs, ddst, mask, fb)
+    side.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        ctx.gk_pack_batch(dsrc, pack_jobs, status)
+        ctx.gk_restore(restore_jobs, ddst, mask, fb)
+
+    def expect(src_cache):
+        ojobs, used = [], 0
+        for pt, n in zip(tables, lens):
+            b, s_, code, _ = oracle.pack(og, src_cache, pt, n)
+            assert code == 0
+            P = n_pages(og, n)
+            ojobs.append(oracle.Job(b, s_, dperm[used:used + P].copy(), n))
+            used += P
+        want = clone_cache(clean)
+        wmask, _ = oracle.restore(og, want, ojobs)
+        return ojobs, want, wmask
+
+    for round_ in range(4):
+        if round_ % 2 == 1:                             # new cache contents: the replay must save and restore them
+            src = random_cache(og, 9, seed=373 + round_)
+            dsrc.data.copy_(torch.from_numpy(src.data))
+        ddst.data.copy_(torch.from_numpy(clean.data))
+        mask.fill_(255)
+        graph.replay()
+        torch.cuda.synchronize()
+        ojobs, want, wmask = expect(src)
+        assert status.cpu().tolist() == [0, 0, 0] and mask.cpu().tolist() == wmask.tolist() == [0, 0, 0]
+        for jb, oj in zip(pack_jobs.jobs, ojobs):
+            assert np.array_equal(jb.blob.cpu().numpy(), oj.blob)
+            assert np.array_equal(jb.checksums.cpu().numpy().view(np.uint64), oj.checksums)
+        assert np.array_equal(ddst.data.cpu().numpy(), want.data)
+    assert ctx.gk_get_stats()["device_wait_expired"] == 0
+    ctx.close()
+
+
 def test_restore_codes_and_first_bad_page(gk):
     from gpu_harness import assert_cache_equal, dev_cache, gpu_restore
     og, N = G_MID, 12
