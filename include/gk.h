@@ -44,10 +44,11 @@
  *   entry reports it.  Kernels are enqueued on the given stream; outputs are
  *   valid once that stream has been synchronised.  A context's workspace is
  *   shared by its calls: calls on one context must be issued in stream order on
- *   one stream at a time (use one context per concurrent stream).  Device-tier
- *   calls of at most 64 jobs and 16,384 pages make no host-device copy and no
- *   synchronisation once the workspace has its size, and may be captured in a
- *   CUDA graph and replayed; host-tier calls and larger calls may not.
+ *   one stream at a time (use one context per concurrent stream).  gk_pack,
+ *   gk_pack_batch, gk_restore, gk_verify and gk_commit calls of at most 64 jobs
+ *   and 16,384 pages make no host-device copy and no synchronisation once the
+ *   workspace has its size, and may be captured in a CUDA graph and replayed;
+ *   the other entry points and larger calls may not.
  *   Requirements: row % 16 == 0, scale section bytes % 16 == 0, all base
  *   pointers and strides of data 16-byte aligned (scale pointers 4-byte), blob
  *   pointers 16-byte aligned, checksum pointers 8-byte aligned; otherwise
