@@ -36,11 +36,12 @@ sys.path.insert(0, ROOT)
 METRIC = "restored KV GB/s (read+write)"
 UNIT = "GB/s"
 
-# DRAM bytes per blob byte of one launch of the fused restore kernel, from the
-# ncu capture of the 2-block case summarised under profiles/ (dram read +
-# write of the launch divided by the blob bytes it restores).  Traffic grows in
-# proportion to the blob bytes, so a full launch is this ratio times its bytes.
-RESTORE_DRAM_BYTES_PER_BLOB_BYTE = 2.96
+# DRAM bytes per blob byte of one launch of the fused restore kernel: ncu's
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the full-size
+# (16-block) workload, a one-pass capture summarised under profiles/
+# (17.18 GB read + 8.56 GB written for 8.59 GB of blobs); the full --set full
+# capture of a 2-block launch gives 2.96.
+RESTORE_DRAM_BYTES_PER_BLOB_BYTE = 25.74 / 8.59
 
 
 def parse_args():
@@ -445,7 +446,8 @@ def run_ours(args):
         roofline = {"bound": "hbm", "kernel": "restore_kernel (fused verify + commit: blob -> CRC check -> paged cache)",
                     "achieved": dom["achieved"], "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                     "frac": dom["frac"], "traffic": RESTORE_DRAM_BYTES_PER_BLOB_BYTE * batch_bytes,
-                    "traffic_note": "ncu dram read+write of a 2-block launch scaled by blob bytes",
+                    "traffic_note": "ncu dram read+write per blob byte of a launch of this workload (one-pass capture), "
+                                    "times the blob bytes of the launch",
                     "algorithmic_bytes_per_launch": 3 * batch_bytes, "ms_per_launch": dom["ms_per_launch"],
                     "achieved_useful_2x": 2 * batch_bytes / (dom["ms_per_launch"] * 1e-3) / 1e9}
     else:
