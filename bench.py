@@ -259,6 +259,7 @@ def build_workload(args, device, rank):
     for i, b in enumerate(chosen):
         pack_jobs.append(gk.Job(pool[b], sums[b], src_perm[i * P:(i + 1) * P].contiguous(), n_tok, i // 2))
         restore_jobs.append(gk.Job(pool[b], sums[b], dst_perm[i * P:(i + 1) * P].contiguous(), n_tok, i // 2))
+    pack_jobs, restore_jobs = gk.JobArray(pack_jobs), gk.JobArray(restore_jobs)   # marshalled once
     return dict(gk=gk, ctx=ctx, geom=geom, w=w, n_tok=n_tok, blob_bytes=blob_bytes, P=P, n_blocks=n_blocks,
                 pool_blocks=pool_blocks, dst_pages=dst_pages, src=src, dst=dst, pack_jobs=pack_jobs,
                 restore_jobs=restore_jobs, chosen=chosen, src_perm=src_perm, dst_perm=dst_perm, slab=slab,
@@ -713,6 +714,7 @@ def run_other_workload(args):
         restore_jobs.append(gk.Job(blob, sums, dperm[off:off + P].contiguous(), n))
         off += P
     nj = len(lens)
+    pack_jobs, restore_jobs = gk.JobArray(pack_jobs), gk.JobArray(restore_jobs)   # marshalled once
     mask = torch.zeros(nj, dtype=torch.uint8, device=device)
     fb = torch.zeros(nj, dtype=torch.int32, device=device)
     status = torch.zeros(nj, dtype=torch.uint8, device=device)
