@@ -63,6 +63,8 @@ class _CJob(ctypes.Structure):
 _WINDOW_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32,
                               ctypes.POINTER(ctypes.c_uint32))
 
+_GROUP_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32)
+
 _lib = None
 
 
@@ -95,6 +97,15 @@ def lib() -> ctypes.CDLL:
         L.ok_restore_stream.argtypes = [ctypes.POINTER(_CGeom), ctypes.POINTER(_CCache),
                                         ctypes.POINTER(_CJob), ctypes.c_uint32, ctypes.c_uint32,
                                         ctypes.c_void_p, ctypes.c_void_p, _WINDOW_FN, ctypes.c_void_p]
+        L.ok_pack_layerwise.restype = ctypes.c_int
+        L.ok_pack_layerwise.argtypes = [ctypes.POINTER(_CGeom), ctypes.c_uint32, ctypes.POINTER(_CCache),
+                                        ctypes.c_void_p, ctypes.c_uint32, ctypes.c_void_p, ctypes.c_void_p,
+                                        ctypes.POINTER(ctypes.c_int32)]
+        L.ok_restore_layerwise.restype = None
+        L.ok_restore_layerwise.argtypes = [ctypes.POINTER(_CGeom), ctypes.c_uint32, ctypes.POINTER(_CCache),
+                                           ctypes.POINTER(_CJob), ctypes.c_uint32, ctypes.c_uint32,
+                                           ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, _GROUP_FN,
+                                           ctypes.c_void_p]
         L.ok_sha256.restype = None
         L.ok_sha256.argtypes = [ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p]
         L.ok_sha256_constants.restype = None
@@ -265,6 +276,40 @@ def restore_stream(g: Geom, ring: Cache, jobs: Sequence[Job], consume=None, flag
     if rc != 0:
         raise ValueError("a job has more pages than the ring")
     return mask, first_bad
+
+
+def pack_layerwise(g: Geom, n_groups: int, src: Cache, page_table, n_tokens: int):
+    """``g`` describes one layer group; ``src`` holds n_groups * g.layers layers.
+    Returns (blob, checksums uint64[n_groups * P], code, bad_index)."""
+    group_bytes, npages = blob_size(g, n_tokens)
+    pt = np.ascontiguousarray(page_table, dtype=np.int32)
+    blob = np.zeros(n_groups * group_bytes, dtype=np.uint8)
+    sums = np.zeros(n_groups * npages, dtype=np.uint64)
+    bad = ctypes.c_int32(-1)
+    cg, cc = g.c(), src.c()
+    code = lib().ok_pack_layerwise(ctypes.byref(cg), n_groups, ctypes.byref(cc), pt.ctypes.data, n_tokens,
+                                   blob.ctypes.data, sums.ctypes.data, ctypes.byref(bad))
+    return blob, sums, int(code), int(bad.value)
+
+
+def restore_layerwise(g: Geom, n_groups: int, dst: Cache, jobs: Sequence[Job], consume=None, flags: int = 0):
+    """Mutates ``dst``; ``consume(group, first_layer, n_layers)`` runs after each group.
+    Returns (mask, first_bad, group_mask uint8[n_groups, n_jobs])."""
+    n = len(jobs)
+    arr, keep = _c_jobs(jobs)
+    mask = np.zeros(n, dtype=np.uint8)
+    first_bad = np.zeros(n, dtype=np.int32)
+    group_mask = np.zeros((n_groups, max(n, 1)), dtype=np.uint8)
+
+    def _cb(_user, group, first_layer, n_layers):
+        if consume is not None:
+            consume(int(group), int(first_layer), int(n_layers))
+
+    cb = _GROUP_FN(_cb)
+    cg, cc = g.c(), dst.c()
+    lib().ok_restore_layerwise(ctypes.byref(cg), n_groups, ctypes.byref(cc), arr, n, flags, mask.ctypes.data,
+                               first_bad.ctypes.data, group_mask.ctypes.data, cb, None)
+    return mask, first_bad, group_mask[:, :n]
 
 
 # ---------------------------------------------------------------------------

@@ -322,3 +322,71 @@ int ok_restore_stream(const ok_geom *g, const ok_cache *ring, const ok_job *jobs
     free(ids);
     return 0;
 }
+
+/* ------------------------------------------------------------------------
+ * Layer-wise save and load: the ordinary format, once per group of layers.
+ * ---------------------------------------------------------------------- */
+static ok_cache layer_view(const ok_geom *g, const ok_cache *c, uint32_t group)
+{
+    ok_cache v = *c;
+    v.data = c->data + (uint64_t)group * g->layers * c->layer_stride;
+    if (c->scales)
+        v.scales = c->scales + (uint64_t)group * g->layers * c->s_layer_stride;
+    return v;
+}
+
+int ok_pack_layerwise(const ok_geom *g, uint32_t n_groups, const ok_cache *src, const int32_t *page_table,
+                      uint32_t n_tokens, uint8_t *blob, uint64_t *checksums, int32_t *bad_index)
+{
+    uint64_t group_bytes = 0;
+    uint32_t P = 0;
+    ok_blob_size(g, n_tokens, &group_bytes, &P);
+    for (uint32_t k = 0; k < n_groups; ++k) {
+        ok_cache view = layer_view(g, src, k);
+        int code = ok_pack(g, &view, page_table, n_tokens, blob + k * group_bytes, checksums + (uint64_t)k * P,
+                           bad_index);
+        if (code != OK_CODE_OK)
+            return code; /* a bad table is bad for every group: group 0 reports it, nothing was written */
+    }
+    return OK_CODE_OK;
+}
+
+void ok_restore_layerwise(const ok_geom *g, uint32_t n_groups, const ok_cache *dst, const ok_job *jobs,
+                          uint32_t n_jobs, uint32_t flags, uint8_t *mask, int32_t *first_bad,
+                          uint8_t *group_mask, ok_group_fn consume, void *user)
+{
+    ok_job *gjobs = (ok_job *)malloc((size_t)(n_jobs ? n_jobs : 1) * sizeof(ok_job));
+    uint8_t *gm = (uint8_t *)malloc(n_jobs ? n_jobs : 1);
+    int32_t *gfb = (int32_t *)malloc((size_t)(n_jobs ? n_jobs : 1) * sizeof(int32_t));
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        mask[j] = OK_CODE_OK;
+        first_bad[j] = -1;
+    }
+    for (uint32_t k = 0; k < n_groups; ++k) {
+        for (uint32_t j = 0; j < n_jobs; ++j) {
+            uint64_t group_bytes = 0;
+            uint32_t P = 0;
+            ok_blob_size(g, jobs[j].n_tokens, &group_bytes, &P);
+            gjobs[j] = jobs[j];
+            if (jobs[j].blob)
+                gjobs[j].blob = jobs[j].blob + k * group_bytes;
+            if (jobs[j].checksums)
+                gjobs[j].checksums = jobs[j].checksums + (uint64_t)k * P;
+        }
+        ok_cache view = layer_view(g, dst, k);
+        ok_restore(g, &view, gjobs, n_jobs, flags, gm, gfb);
+        for (uint32_t j = 0; j < n_jobs; ++j) {
+            if (group_mask)
+                group_mask[(uint64_t)k * n_jobs + j] = gm[j];
+            if (mask[j] == OK_CODE_OK && gm[j] != OK_CODE_OK)
+                first_bad[j] = gfb[j]; /* the lowest failing group decides the reported page */
+            if (gm[j] > mask[j])
+                mask[j] = gm[j];
+        }
+        if (consume)
+            consume(user, k, k * g->layers, g->layers);
+    }
+    free(gfb);
+    free(gm);
+    free(gjobs);
+}

@@ -130,6 +130,27 @@ typedef void (*ok_window_fn)(void *user, uint32_t first_job, uint32_t n_jobs, co
 int ok_restore_stream(const ok_geom *g, const ok_cache *ring, const ok_job *jobs, uint32_t n_jobs,
                       uint32_t flags, uint8_t *mask, int32_t *first_bad, ok_window_fn consume, void *user);
 
+/* Layer-wise save and load.  A block's record is cut by layer groups so that a
+ * consumer that walks the layers in order can start on the first layers while
+ * the later ones are still arriving from storage (the streaming of saved state
+ * in Section 4.3; the paper gives no format).  g describes ONE GROUP (g->layers
+ * = layers per group); the cache holds n_groups * g->layers layers.  The
+ * layer-wise blob of a block is the concatenation, for group k = 0..n_groups-1,
+ * of the ordinary blob (as ok_pack makes it) of the cache restricted to the
+ * layers [k*g->layers, (k+1)*g->layers); the checksums are those blobs'
+ * checksums, group after group (n_groups * P values).
+ * ok_restore_layerwise loads group after group, each as one ok_restore of all
+ * jobs over the restricted cache: fail-closed holds per (job, group).  mask[j]
+ * is the largest code over the groups, first_bad[j] the page of the lowest
+ * failing group (or -1); group_mask (n_groups * n_jobs, may be NULL) receives
+ * every group's codes.  `consume` (may be NULL) is called after each group. */
+typedef void (*ok_group_fn)(void *user, uint32_t group, uint32_t first_layer, uint32_t n_layers);
+int ok_pack_layerwise(const ok_geom *g, uint32_t n_groups, const ok_cache *src, const int32_t *page_table,
+                      uint32_t n_tokens, uint8_t *blob, uint64_t *checksums, int32_t *bad_index);
+void ok_restore_layerwise(const ok_geom *g, uint32_t n_groups, const ok_cache *dst, const ok_job *jobs,
+                          uint32_t n_jobs, uint32_t flags, uint8_t *mask, int32_t *first_bad,
+                          uint8_t *group_mask, ok_group_fn consume, void *user);
+
 #ifdef __cplusplus
 }
 #endif

@@ -116,6 +116,48 @@ static int run_sha(const ok_geom *g, uint32_t n_tokens)
     return 0;
 }
 
+/* layer-wise save and load on exact-size buffers: 3 groups of g->layers layers */
+static int run_layerwise(const ok_geom *g, uint32_t n_tokens)
+{
+    const uint32_t G = 3, N = 6;
+    uint64_t slab = (uint64_t)g->page_tokens * g->kv_heads * g->head_dim * g->elem_bytes;
+    uint32_t L = g->layers * G;
+    ok_cache src = {0}, dst = {0};
+    src.num_pages = dst.num_pages = N;
+    src.page_stride = dst.page_stride = slab;
+    src.kv_stride = dst.kv_stride = N * slab;
+    src.layer_stride = dst.layer_stride = 2 * N * slab;
+    src.data = malloc((size_t)(L * 2 * N * slab));
+    dst.data = calloc((size_t)(L * 2 * N * slab), 1);
+    for (uint64_t i = 0; i < L * 2 * N * slab; ++i) src.data[i] = (uint8_t)(i * 13u + 5u);
+    if (g->scale_kv) {
+        uint64_t h4 = g->kv_heads * 4u;
+        src.s_page_stride = dst.s_page_stride = h4;
+        src.s_kv_stride = dst.s_kv_stride = N * h4;
+        src.s_layer_stride = dst.s_layer_stride = g->scale_kv * N * h4;
+        src.scales = malloc((size_t)(L * g->scale_kv * N * h4));
+        dst.scales = calloc((size_t)(L * g->scale_kv * N * h4), 1);
+        for (uint64_t i = 0; i < L * g->scale_kv * N * h4; ++i) src.scales[i] = (uint8_t)(i * 7u);
+    }
+    uint64_t gbytes = 0;
+    uint32_t P = 0;
+    ok_blob_size(g, n_tokens, &gbytes, &P);
+    int32_t *pt = malloc(P * sizeof(int32_t));
+    for (uint32_t p = 0; p < P; ++p) pt[p] = (int32_t)((p * 5u + 1u) % N);
+    uint8_t *blob = malloc((size_t)(G * gbytes));
+    uint64_t *sums = malloc((size_t)G * P * sizeof(uint64_t));
+    int32_t bad = 0;
+    if (ok_pack_layerwise(g, G, &src, pt, n_tokens, blob, sums, &bad) != OK_CODE_OK) return 30;
+    blob[gbytes + 1] ^= 0x10; /* damage in group 1 */
+    ok_job job = {blob, sums, pt, n_tokens};
+    uint8_t mask[1], gm[3];
+    int32_t fb[1];
+    ok_restore_layerwise(g, G, &dst, &job, 1, 0, mask, fb, gm, NULL, NULL);
+    if (mask[0] != OK_CODE_CHECKSUM || gm[0] != 0 || gm[1] != OK_CODE_CHECKSUM || gm[2] != 0 || fb[0] != 0) return 31;
+    free(sums); free(blob); free(pt); free(src.data); free(dst.data); free(src.scales); free(dst.scales);
+    return 0;
+}
+
 int main(void)
 {
     ok_geom bf16 = {3, 2, 8, 4, 2, 0};
@@ -129,6 +171,7 @@ int main(void)
         if ((rc = run(&fp8_shared, 5, 11, lens[i])) != 0) { printf("fp8/1 len %u: %d\n", lens[i], rc); return 1; }
     }
     ok_geom wide = {6, 4, 32, 8, 1, 2};   /* records of 12,480 bytes: three full digest chunks and a short one */
+    if (run_layerwise(&bf16, 9) != 0 || run_layerwise(&fp8, 13) != 0) { printf("layerwise\n"); return 1; }
     if (run_sha(&bf16, 9) != 0 || run_sha(&wide, 17) != 0) { printf("sha\n"); return 1; }
     printf("clean\n");
     return 0;

@@ -614,3 +614,104 @@ def test_stream_restore_refuses_a_job_larger_than_the_ring():
     with pytest.raises(ValueError):
         oracle.restore_stream(g, ring, [oracle.Job(small, _s, None, 1), oracle.Job(blob, sums, None, 6 * g.page_tokens)])
     assert np.array_equal(ring.data, before.data)   # not even the first job was restored
+
+
+# --------------------------------------------------------------------------
+# layer-wise save and load (the ordinary format once per group of layers)
+# --------------------------------------------------------------------------
+def _full_geom(g, n_groups):
+    return oracle.Geom(g.layers * n_groups, g.kv_heads, g.head_dim, g.page_tokens, g.elem_bytes, g.scale_kv, g.head_major)
+
+
+@pytest.mark.parametrize("g", [oracle.Geom(2, 2, 8, 4, 2, 0), oracle.Geom(1, 4, 16, 8, 1, 2),
+                               oracle.Geom(2, 4, 8, 4, 2, 0, head_major=1)])
+@pytest.mark.parametrize("n_tokens_extra", [0, 1, 3])
+def test_layerwise_blob_is_the_ordinary_blob_cut_by_layer_groups(g, n_tokens_extra):
+    G = 3
+    full = _full_geom(g, G)
+    N, T = 7, g.page_tokens
+    n = 2 * T + n_tokens_extra
+    src = random_cache(full, N, seed=90)
+    pt = np.random.default_rng(91).permutation(N)[:n_pages(full, n)].astype(np.int32)
+    whole, _, code, _ = oracle.pack(full, src, pt, n)
+    assert code == 0
+    lw, sums, code, _ = oracle.pack_layerwise(g, G, src, pt, n)
+    assert code == 0 and lw.size == whole.size
+    P = n_pages(full, n)
+    group_bytes, _ = oracle.blob_size(g, n)
+    S_full = full.layers * full.scale_kv * full.kv_heads * 4
+    S_g = S_full // G
+    for k in range(G):
+        for p in range(P):
+            rec_full = whole[oracle.record_offset(full, p):][:oracle.record_bytes(full, n, p)]
+            data_full = rec_full[S_full:]
+            dg = data_full.size // G
+            want = np.concatenate([rec_full[k * S_g:(k + 1) * S_g], data_full[k * dg:(k + 1) * dg]])
+            got = lw[k * group_bytes + oracle.record_offset(g, p):][:oracle.record_bytes(g, n, p)]
+            assert np.array_equal(got, want), (k, p)
+            assert int(sums[k * P + p]) == oracle.crc64(want)
+    # every byte of the ordinary blob appears exactly once
+    assert np.array_equal(np.sort(lw), np.sort(whole))
+
+
+@pytest.mark.parametrize("g", [oracle.Geom(2, 2, 8, 4, 2, 0), oracle.Geom(1, 4, 16, 8, 1, 2)])
+def test_layerwise_restore_groups_are_independent_and_in_order(g):
+    G = 3
+    full = _full_geom(g, G)
+    T, N = g.page_tokens, 12
+    src = random_cache(full, 8, seed=92)
+    lens = [2 * T + 1, T, 3 * T - 1]
+    rng = np.random.default_rng(93)
+    perm = rng.permutation(N).astype(np.int32)
+    lw_jobs, std_jobs, used = [], [], 0
+    for n in lens:
+        P = n_pages(full, n)
+        spt = rng.integers(0, 8, size=P).astype(np.int32)
+        b, s_, _, _ = oracle.pack_layerwise(g, G, src, spt, n)
+        wb, ws, _, _ = oracle.pack(full, src, spt, n)
+        lw_jobs.append(oracle.Job(b, s_, perm[used:used + P].copy(), n))
+        std_jobs.append(oracle.Job(wb, ws, perm[used:used + P].copy(), n))
+        used += P
+    clean = _sentinel_cache(full, N, seed=94)
+    # all good: same destination as the ordinary restore of the ordinary blobs
+    a, b_ = clone_cache(clean), clone_cache(clean)
+    oracle.restore(full, a, std_jobs)
+    seen = []
+    mask, fb, gm = oracle.restore_layerwise(g, G, b_, lw_jobs, lambda k, l0, nl: seen.append((k, l0, nl)))
+    assert mask.tolist() == [0, 0, 0] and fb.tolist() == [-1, -1, -1] and gm.tolist() == [[0, 0, 0]] * 3
+    assert seen == [(0, 0, g.layers), (1, g.layers, g.layers), (2, 2 * g.layers, g.layers)]
+    assert np.array_equal(a.data, b_.data)
+    if g.scale_kv:
+        assert np.array_equal(a.scales, b_.scales)
+    # job 0 damaged inside group 1 (second page), job 2 inside groups 0 and 2
+    gb0, P0 = oracle.blob_size(g, lens[0])
+    gb2, P2 = oracle.blob_size(g, lens[2])
+    lw_jobs[0].blob[gb0 + oracle.record_offset(g, 1) + 5] ^= 0x01
+    lw_jobs[2].blob[3] ^= 0x80
+    lw_jobs[2].checksums[2 * P2 + 2] ^= np.uint64(4)
+    c = clone_cache(clean)
+    snapshots = []
+    mask, fb, gm = oracle.restore_layerwise(g, G, c, lw_jobs, lambda k, l0, nl: snapshots.append(c.data.copy()))
+    assert mask.tolist() == [1, 0, 1] and fb.tolist() == [1, -1, 0]
+    assert gm.tolist() == [[0, 0, 1], [1, 0, 0], [0, 0, 1]]
+    # layer by layer: a (job, group) that verified holds the ordinary result, one that failed the sentinel
+    L_full = full.layers
+    va = a.data.reshape(L_full, -1)
+    vz = clean.data.reshape(L_full, -1)
+    vc = c.data.reshape(L_full, -1)
+    per_layer = va.shape[1]
+    slab = slab_bytes(full)
+    for k in range(G):
+        for l in range(k * g.layers, (k + 1) * g.layers):
+            expect = vz[l].copy().reshape(2, N, slab)
+            good = va[l].reshape(2, N, slab)
+            for j, jb in enumerate(lw_jobs):
+                if gm[k][j] == 0:
+                    for page in jb.page_table:
+                        expect[:, page] = good[:, page]
+            assert np.array_equal(vc[l].reshape(2, N, slab), expect), (k, l)
+    # in order: after the call-back of group k the layers of the groups up to k are final
+    for k in range(G):
+        snap = snapshots[k].reshape(L_full, per_layer)
+        assert np.array_equal(snap[:(k + 1) * g.layers], vc[:(k + 1) * g.layers])
+        assert np.array_equal(snap[(k + 1) * g.layers:], vz[(k + 1) * g.layers:])
