@@ -50,7 +50,7 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress", "longwindow", "digest"],
+    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress", "longwindow", "digest", "layerwise"],
                     help="gqa7b is the headline workload (full JSON line); the others print a shorter line "
                          "with the save and restore phases of that workload's shape")
     ap.add_argument("--window-blocks", type=int, default=48,
@@ -923,6 +923,93 @@ def run_digest(args):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------
+# layer-wise load from the host tier: when is each group of layers ready?
+# ---------------------------------------------------------------------------
+def run_layerwise(args):
+    import torch
+    import synth
+    import paper_2609_39358_b200 as gk
+
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    w = synth.GQA7B
+    group_layers, n_groups = 4, w.layers // 4
+    g_geom = gk.Geom(group_layers, w.kv_heads, w.head_dim, w.page_tokens, gk.GK_BF16, 0)
+    f_geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, gk.GK_BF16, 0)
+    ctx_g, ctx_f = gk.Context(g_geom, device.index), gk.Context(f_geom, device.index)
+    slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
+    stream = torch.cuda.current_stream(device)
+    out = {}
+    for name, lens in (("prompt_5200_tokens", [5200]), ("batch_4_x_4096_tokens", [4096] * 4)):
+        pages = [-(-n // w.page_tokens) for n in lens]
+        N = sum(pages)
+        data = synth.kv_bytes_bf16(2 * w.layers * N * slab // 2, w.sigma, w.seed(900), device)
+        src = gk.Cache(data, N, 2 * N * slab, N * slab, slab)
+        dst = gk.Cache(torch.zeros_like(data), N, 2 * N * slab, N * slab, slab)
+        tables, off = [], 0
+        perm = torch.from_numpy(synth.page_permutation(N, w.seed(901))).to(device)
+        for P in pages:
+            tables.append(perm[off:off + P].contiguous())
+            off += P
+        lw_jobs, std_jobs, total = [], [], 0
+        for n, P, pt in zip(lens, pages, tables):
+            nb, _ = gk.gk_blob_size(f_geom, n)
+            total += nb
+            lw_jobs.append(gk.Job(torch.empty(nb, dtype=torch.uint8, pin_memory=True),
+                                  torch.empty(n_groups * P, dtype=torch.int64, pin_memory=True), pt, n))
+            std_jobs.append(gk.Job(torch.empty(nb, dtype=torch.uint8, pin_memory=True),
+                                   torch.empty(P, dtype=torch.int64, pin_memory=True), pt, n))
+        ctx_g.gk_pack_layerwise(n_groups, src, lw_jobs, host=True)
+        ctx_f.gk_pack_host(src, std_jobs)
+        torch.cuda.synchronize(device)
+        nj = len(lens)
+        mask = torch.zeros(nj, dtype=torch.uint8, device=device)
+        fb = torch.zeros(nj, dtype=torch.int32, device=device)
+        reps = 5
+        whole_ms, group_ms = [], []
+        for r in range(reps + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            ctx_f.gk_restore_host(std_jobs, dst, mask, fb)
+            e1.record(stream)
+            torch.cuda.synchronize(device)
+            assert int(mask.sum().item()) == 0
+            ready = []
+            g0 = torch.cuda.Event(enable_timing=True)
+            g0.record(stream)
+
+            def on_group(group, first_layer, n_layers, st):
+                ev = torch.cuda.Event(enable_timing=True)
+                ev.record(stream)
+                ready.append(ev)
+
+            ctx_g.gk_restore_layerwise(n_groups, lw_jobs, dst, mask, fb, None, on_group, host=True)
+            torch.cuda.synchronize(device)
+            assert int(mask.sum().item()) == 0
+            if r > 0:
+                whole_ms.append(e0.elapsed_time(e1))
+                group_ms.append([g0.elapsed_time(ev) for ev in ready])
+        gm = np.mean(np.array(group_ms), axis=0)
+        out[name] = {"blob_gib": total / 2**30, "ordinary_restore_host_ms": float(np.mean(whole_ms)),
+                     "layerwise_group_ready_ms": [round(float(x), 3) for x in gm],
+                     "layerwise_total_ms": float(gm[-1]),
+                     "first_group_ready_after_fraction": float(gm[0] / np.mean(whole_ms)),
+                     "host_link_gbs_layerwise": total / (float(gm[-1]) * 1e-3) / 1e9}
+        del data, src, dst, lw_jobs, std_jobs
+        torch.cuda.empty_cache()
+    line = {"metric": "layer-wise restore from pinned host memory: ms until each group of layers is ready",
+            "value": out["prompt_5200_tokens"]["layerwise_group_ready_ms"][0], "unit": "ms", "n_gpus": 1,
+            "steps": 5, "warmup": 1, "ms_per_step": out["prompt_5200_tokens"]["layerwise_total_ms"],
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": f"layerwise: gqa7b geometry, {n_groups} groups of {group_layers} layers; a 5,200-token "
+                                   "prompt block and a batch of 4 x 4,096 tokens, blobs in pinned host memory",
+                       "step": "gk_restore_layerwise_host, an event recorded in the group call-back; beside it "
+                               "gk_restore_host of the same blocks in the ordinary format"},
+            "cases": out}
+    print(json.dumps(line), flush=True)
+
+
 def synth_requests(n_blocks):
     return f"{max(n_blocks // 2, 1)} requests x {min(n_blocks, 2)} blocks"
 
@@ -935,6 +1022,8 @@ def main():
         run_longwindow(args)
     elif args.workload == "digest":
         run_digest(args)
+    elif args.workload == "layerwise":
+        run_layerwise(args)
     elif args.workload != "gqa7b" or args.single_pass:
         run_other_workload(args)
     else:

@@ -269,6 +269,47 @@ int gk_restore_stream(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk
                       uint8_t *mask_dev, int32_t *first_bad_page_dev, gk_window_fn consume, void *user,
                       void *stream);
 
+/* Layer-wise save and load.  A consumer that walks the layers in order (a
+ * forward pass) can start on the first layers of a block while the later ones
+ * are still arriving from the host tier, if the block's record is cut by layer
+ * groups (Section 4.3 streams saved state in from storage; the paper gives no
+ * format).  Here the context's geometry describes ONE GROUP (geom.layers = layers
+ * per group) and the cache holds n_groups * geom.layers layers.  The layer-wise
+ * blob of a block is the concatenation, for group k = 0 .. n_groups-1, of the
+ * ordinary blob (as gk_pack_batch makes it) of the cache restricted to the layers
+ * [k*geom.layers, (k+1)*geom.layers); its checksums are those blobs' checksums,
+ * group after group.  So jobs[j].blob holds n_groups * gk_blob_size() bytes and
+ * jobs[j].checksums n_groups * n_pages entries.
+ *
+ * gk_pack_layerwise / gk_pack_layerwise_host: one gk_pack_batch / gk_pack_host
+ * per group (status_dev as there).
+ *
+ * gk_restore_layerwise / gk_restore_layerwise_host: group after group, each as
+ * one gk_restore / gk_restore_host of all jobs over the restricted cache, so
+ * fail-closed holds per (job, group): of a block that fails in one group, the
+ * groups that verified HAVE been written to the block's own pages and the failing
+ * ones have not; the block as a whole is usable only if mask_dev[j] == GK_JOB_OK.
+ * mask_dev[j] (device, n_jobs bytes) is the largest code over the groups,
+ * first_bad_page_dev[j] the page reported by the lowest failing group (or -1);
+ * group_mask_dev (device, n_groups * n_jobs bytes, group-major; may be NULL)
+ * receives every group's codes.  After the work of group k has been enqueued,
+ * on_group (may be NULL) is called ON THE HOST; it must only enqueue work on
+ * `stream` (e.g. layer k's attention); group_mask points at group k's codes (NULL
+ * if group_mask_dev is NULL).  In the host tier the copies of group k+1 run while
+ * group k is verified, committed and consumed. */
+typedef void (*gk_group_fn)(void *user, uint32_t group, uint32_t first_layer, uint32_t n_layers,
+                            const uint8_t *group_mask, void *stream);
+int gk_pack_layerwise(gk_ctx *ctx, uint32_t n_groups, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,
+                      uint8_t *status_dev, void *stream);
+int gk_pack_layerwise_host(gk_ctx *ctx, uint32_t n_groups, const gk_cache *src, const gk_job *jobs,
+                           uint32_t n_jobs, uint8_t *status_dev, void *stream);
+int gk_restore_layerwise(gk_ctx *ctx, uint32_t n_groups, const gk_job *jobs, uint32_t n_jobs,
+                         const gk_cache *dst, uint8_t *mask_dev, int32_t *first_bad_page_dev,
+                         uint8_t *group_mask_dev, gk_group_fn on_group, void *user, void *stream);
+int gk_restore_layerwise_host(gk_ctx *ctx, uint32_t n_groups, const gk_job *jobs, uint32_t n_jobs,
+                              const gk_cache *dst, uint8_t *mask_dev, int32_t *first_bad_page_dev,
+                              uint8_t *group_mask_dev, gk_group_fn on_group, void *user, void *stream);
+
 /* Block fingerprints (Section 2.2: the lookup key of a block's state is derived
  * from the block's input, byte for byte, and from the identities of model and
  * tenant; Section 2.1: records of one model or tenant stay out of another's reach;

@@ -28,7 +28,8 @@ JOB_OK, JOB_CHECKSUM, JOB_PAGE_TABLE, JOB_MISSING, JOB_TIMEOUT = 0, 1, 2, 3, 4
 EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "gk_pack_batch", "gk_pack",
            "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times",
            "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit", "gk_restore_stream",
-           "gk_fingerprints", "gk_blob_digests"]
+           "gk_fingerprints", "gk_blob_digests", "gk_pack_layerwise", "gk_pack_layerwise_host",
+           "gk_restore_layerwise", "gk_restore_layerwise_host"]
 
 
 class GkError(RuntimeError):
@@ -67,6 +68,8 @@ class CWindowBlock(ctypes.Structure):
     _fields_ = [("job", ctypes.c_uint32), ("n_tokens", ctypes.c_uint32), ("page_table", ctypes.c_void_p)]
 
 
+GROUP_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_uint32, ctypes.c_void_p,
+                            ctypes.c_void_p)
 WINDOW_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.POINTER(CWindowBlock), ctypes.c_uint32, ctypes.c_void_p,
                              ctypes.c_void_p)
 
@@ -145,6 +148,13 @@ def load_library() -> ctypes.CDLL:
     L.gk_restore_host.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp]
     L.gk_restore_stream.restype = ctypes.c_int
     L.gk_restore_stream.argtypes = [vp, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, WINDOW_FN, vp, vp]
+    for name in ("gk_pack_layerwise", "gk_pack_layerwise_host"):
+        getattr(L, name).restype = ctypes.c_int
+        getattr(L, name).argtypes = [vp, u32, ctypes.POINTER(CCache), ctypes.POINTER(CJob), u32, vp, vp]
+    for name in ("gk_restore_layerwise", "gk_restore_layerwise_host"):
+        getattr(L, name).restype = ctypes.c_int
+        getattr(L, name).argtypes = [vp, u32, ctypes.POINTER(CJob), u32, ctypes.POINTER(CCache), vp, vp, vp, GROUP_FN,
+                                     vp, vp]
     L.gk_fingerprints.restype = ctypes.c_int
     L.gk_fingerprints.argtypes = [vp, vp, vp, ctypes.POINTER(ctypes.c_int32), u32, ctypes.c_char_p, ctypes.c_char_p, vp, vp]
     L.gk_blob_digests.restype = ctypes.c_int
@@ -353,6 +363,38 @@ class Context:
         if raised:
             raise raised[0]
         self._check(rc, "gk_restore_stream")
+
+    def gk_pack_layerwise(self, n_groups: int, src: Cache, jobs, status: Optional[torch.Tensor] = None, stream=None,
+                          host: bool = False):
+        """The context's geometry describes one layer group; ``src`` holds n_groups of them."""
+        cc = src.c()
+        fn = self._lib.gk_pack_layerwise_host if host else self._lib.gk_pack_layerwise
+        self._check(fn(self._h, n_groups, ctypes.byref(cc), self._jobs(jobs), len(jobs), _ptr(status),
+                       _stream_handle(stream)), "gk_pack_layerwise")
+
+    def gk_restore_layerwise(self, n_groups: int, jobs, dst: Cache, mask: torch.Tensor, first_bad_page: torch.Tensor,
+                             group_mask: Optional[torch.Tensor] = None, on_group: Optional[Callable] = None,
+                             stream=None, host: bool = False):
+        """``on_group(group, first_layer, n_layers, stream_handle)`` runs on the host after the work of
+        each group has been enqueued; it may only enqueue work on that stream."""
+        cc = dst.c()
+        raised = []
+
+        def _cb(_user, group, first_layer, n_layers, _gm, st):
+            if on_group is None:
+                return
+            try:
+                on_group(int(group), int(first_layer), int(n_layers), st or 0)
+            except BaseException as e:  # must not unwind through the C frames
+                raised.append(e)
+
+        cb = GROUP_FN(_cb)
+        fn = self._lib.gk_restore_layerwise_host if host else self._lib.gk_restore_layerwise
+        rc = fn(self._h, n_groups, self._jobs(jobs), len(jobs), ctypes.byref(cc), _ptr(mask), _ptr(first_bad_page),
+                _ptr(group_mask), cb, None, _stream_handle(stream))
+        if raised:
+            raise raised[0]
+        self._check(rc, "gk_restore_layerwise")
 
     def gk_fingerprints(self, data: torch.Tensor, offsets: torch.Tensor, parent: Optional[Sequence[int]],
                         model: bytes, tenant: bytes, keys: torch.Tensor, stream=None):

@@ -131,6 +131,10 @@ struct gk_ctx {
     uint32_t slot_next = 0;  // the slot the next batch goes to (carried across calls)
     bool pdl_next = false;   // the kernel just enqueued lets the next one start early (small calls)
 
+    // layer-wise restore: the codes and pages of the group in flight
+    uint8_t *d_group_tmp = nullptr;
+    size_t group_tmp_cap = 0;
+
     // streaming restore: the ids 0..iota_cap-1, from which window page tables are cut
     int32_t *d_iota = nullptr;
     uint64_t iota_cap = 0;
@@ -851,6 +855,7 @@ int gk_ctx_destroy(gk_ctx *c)
     if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->d_ws) cudaFree(c->d_ws);
     if (c->d_iota) cudaFree(c->d_iota);
+    if (c->d_group_tmp) cudaFree(c->d_group_tmp);
     if (c->d_init_term) cudaFree(c->d_init_term);
     if (c->d_thread_const) cudaFree(c->d_thread_const);
     if (c->d_error) cudaFree(c->d_error);
@@ -1332,6 +1337,120 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
     c->stats.pages += pages;
     c->stats.bytes_blob += bytes;
     return GK_OK;
+}
+
+// ---------------------------------------------------------------------------
+// layer-wise save and load: the ordinary calls, once per group of layers, over
+// the cache restricted to the group and the group's part of every blob
+// ---------------------------------------------------------------------------
+static gk_cache group_view(const gk_ctx *c, const gk_cache *k, uint32_t group)
+{
+    gk_cache v = *k;
+    v.data = (uint8_t *)k->data + (uint64_t)group * c->gd.layers * k->layer_stride;
+    if (k->scales) v.scales = (uint8_t *)k->scales + (uint64_t)group * c->gd.layers * k->s_layer_stride;
+    return v;
+}
+
+static void group_jobs(const gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, uint32_t group, std::vector<gk_job> &out)
+{
+    out.assign(jobs, jobs + n_jobs);
+    for (uint32_t j = 0; j < n_jobs; ++j) {
+        const uint32_t np = pages_of(jobs[j].n_tokens, c->gd.page_tokens);
+        const uint64_t bytes = (uint64_t)np * c->gd.S + (uint64_t)jobs[j].n_tokens * c->gd.tokB;
+        if (out[j].blob) out[j].blob = (uint8_t *)jobs[j].blob + (uint64_t)group * bytes;
+        if (out[j].checksums) out[j].checksums = jobs[j].checksums + (uint64_t)group * np;
+    }
+}
+
+static int pack_layerwise_impl(gk_ctx *c, uint32_t n_groups, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,
+                               uint8_t *status_dev, void *stream, bool host)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0 || n_groups == 0) return GK_OK;
+    if (!jobs || !src) return fail(c, GK_ERR_ARG, "null jobs or cache");
+    for (uint32_t j = 0; j < n_jobs; ++j)
+        if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
+    std::vector<gk_job> gj;
+    for (uint32_t k = 0; k < n_groups; ++k) {
+        const gk_cache view = group_view(c, src, k);
+        group_jobs(c, jobs, n_jobs, k, gj);
+        const int rc = host ? gk_pack_host(c, &view, gj.data(), n_jobs, status_dev, stream)
+                            : gk_pack_batch(c, &view, gj.data(), n_jobs, status_dev, stream);
+        if (rc != GK_OK) return rc;
+    }
+    return GK_OK;
+}
+
+static int restore_layerwise_impl(gk_ctx *c, uint32_t n_groups, const gk_job *jobs, uint32_t n_jobs,
+                                  const gk_cache *dst, uint8_t *mask_dev, int32_t *first_bad_page_dev,
+                                  uint8_t *group_mask_dev, gk_group_fn on_group, void *user, void *stream, bool host)
+{
+    if (!c) return GK_ERR_ARG;
+    if (n_jobs == 0 || n_groups == 0) return GK_OK;
+    if (!jobs || !dst || !mask_dev || !first_bad_page_dev)
+        return fail(c, GK_ERR_ARG, "null jobs, cache, mask or first_bad_page");
+    for (uint32_t j = 0; j < n_jobs; ++j)
+        if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    // per-group result arrays: pages always, codes unless the caller keeps them
+    const size_t need = align_up((size_t)n_jobs * 4, 256) + (size_t)n_jobs;
+    if (need > c->group_tmp_cap) {
+        GK_CUDA(c, cudaDeviceSynchronize());
+        if (c->d_group_tmp) cudaFree(c->d_group_tmp);
+        c->d_group_tmp = nullptr;
+        c->group_tmp_cap = 0;
+        if (cudaMalloc(&c->d_group_tmp, need * 2) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(c, GK_ERR_NOMEM, "layer-wise result arrays of %zu bytes", need * 2);
+        }
+        c->group_tmp_cap = need * 2;
+    }
+    int32_t *gfb = (int32_t *)c->d_group_tmp;
+    uint8_t *gm_own = c->d_group_tmp + align_up((size_t)n_jobs * 4, 256);
+    std::vector<gk_job> gj;
+    for (uint32_t k = 0; k < n_groups; ++k) {
+        const gk_cache view = group_view(c, dst, k);
+        group_jobs(c, jobs, n_jobs, k, gj);
+        uint8_t *gm = group_mask_dev ? group_mask_dev + (size_t)k * n_jobs : gm_own;
+        const int rc = host ? restore_host_impl(c, gj.data(), n_jobs, &view, gm, gfb, stream, k == 0)
+                            : gk_restore(c, gj.data(), n_jobs, &view, gm, gfb, stream);
+        if (rc != GK_OK) return rc;
+        merge_group_kernel<<<(n_jobs + 127) / 128, 128, 0, st>>>(mask_dev, first_bad_page_dev, gm, gfb, n_jobs, k == 0);
+        GK_CUDA(c, cudaGetLastError());
+        c->stats.kernels_launched++;
+        if (on_group)
+            on_group(user, k, k * c->gd.layers, c->gd.layers, group_mask_dev ? gm : nullptr, stream);
+    }
+    return GK_OK;
+}
+
+int gk_pack_layerwise(gk_ctx *c, uint32_t n_groups, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,
+                      uint8_t *status_dev, void *stream)
+{
+    return pack_layerwise_impl(c, n_groups, src, jobs, n_jobs, status_dev, stream, false);
+}
+
+int gk_pack_layerwise_host(gk_ctx *c, uint32_t n_groups, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,
+                           uint8_t *status_dev, void *stream)
+{
+    return pack_layerwise_impl(c, n_groups, src, jobs, n_jobs, status_dev, stream, true);
+}
+
+int gk_restore_layerwise(gk_ctx *c, uint32_t n_groups, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
+                         uint8_t *mask_dev, int32_t *first_bad_page_dev, uint8_t *group_mask_dev, gk_group_fn on_group,
+                         void *user, void *stream)
+{
+    return restore_layerwise_impl(c, n_groups, jobs, n_jobs, dst, mask_dev, first_bad_page_dev, group_mask_dev,
+                                  on_group, user, stream, false);
+}
+
+int gk_restore_layerwise_host(gk_ctx *c, uint32_t n_groups, const gk_job *jobs, uint32_t n_jobs, const gk_cache *dst,
+                              uint8_t *mask_dev, int32_t *first_bad_page_dev, uint8_t *group_mask_dev,
+                              gk_group_fn on_group, void *user, void *stream)
+{
+    return restore_layerwise_impl(c, n_groups, jobs, n_jobs, dst, mask_dev, first_bad_page_dev, group_mask_dev,
+                                  on_group, user, stream, true);
 }
 
 int gk_fingerprints(gk_ctx *c, const void *data_dev, const uint64_t *offsets_dev, const int32_t *parent, uint32_t n,

@@ -46,6 +46,20 @@ __global__ void iota_kernel(int32_t *ids, uint32_t n)
     if (i < n) ids[i] = (int32_t)i;
 }
 
+// Layer-wise restore: folds the codes of one layer group into the block-level result.
+// mask = largest code so far; first_bad = the page reported by the lowest failing group.
+__global__ void merge_group_kernel(uint8_t *mask, int32_t *first_bad, const uint8_t *group_mask,
+                                   const int32_t *group_first_bad, uint32_t n_jobs, int first_group)
+{
+    const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= n_jobs) return;
+    const uint8_t gm = group_mask[j];
+    const uint8_t m = first_group ? (uint8_t)0 : mask[j];
+    if (first_group) first_bad[j] = -1;
+    if (m == 0 && gm != 0) first_bad[j] = group_first_bad[j];
+    mask[j] = gm > m ? gm : m;
+}
+
 // One CTA per job.  Initialises the job's result words, records the lowest
 // out-of-range page id and fills page_job.  All CTAs together clear the claim
 // words of the destination cache.

@@ -20,7 +20,8 @@ int main(void)
                     (any_fn)gk_page_checksums_noalloc, (any_fn)gk_restore, (any_fn)gk_restore_host,
                     (any_fn)gk_verify, (any_fn)gk_commit, (any_fn)gk_get_stats, (any_fn)gk_ctx_set_tuning,
                     (any_fn)gk_get_kernel_times, (any_fn)gk_restore_stream, (any_fn)gk_fingerprints,
-                    (any_fn)gk_blob_digests};
+                    (any_fn)gk_blob_digests, (any_fn)gk_pack_layerwise, (any_fn)gk_pack_layerwise_host,
+                    (any_fn)gk_restore_layerwise, (any_fn)gk_restore_layerwise_host};
     for (unsigned i = 0; i < sizeof(fns) / sizeof(fns[0]); ++i)
         if (!fns[i]) return 4;
     printf("abi ok: %u entry points\n", (unsigned)(sizeof(fns) / sizeof(fns[0])) + 1u);

@@ -527,3 +527,87 @@ def test_gqa7b_full_digests_and_keys(gk):
                               + b"GKB0").digest()
         assert hd[j].tobytes() == root
     ctx.close()
+
+
+def test_layerwise_full_size_host_tier(gk):
+    """GQA-7B geometry cut into 8 groups of 4 layers, 3 blocks of 4,096 / 4,096 / 5,200 tokens,
+    saved to and loaded from pinned host memory group by group; one (block, group) damaged."""
+    w = synth.GQA7B
+    T = w.page_tokens
+    gl, G = 4, w.layers // 4
+    g_geom = gk.Geom(gl, w.kv_heads, w.head_dim, w.page_tokens)
+    og_group = oracle.Geom(gl, w.kv_heads, w.head_dim, w.page_tokens, 2, 0)
+    ctx = gk.Context(g_geom, 0)
+    s = _slab(w)
+    lens = [4096, 4096, 5200]
+    pages = [-(-n // T) for n in lens]
+    N = sum(pages)
+    src = _dev_cache(gk, w, N, synth.kv_bytes_bf16(w.layers * N * s, w.sigma, w.seed(70), "cuda"))
+    Nd = N + 50
+    sentinel = synth.sentinel_bytes(2 * w.layers * Nd * s, w.seed(71), "cuda")
+    dst = _dev_cache(gk, w, Nd, sentinel.clone())
+    sperm, dperm = synth.page_permutation(N, w.seed(72)), synth.page_permutation(Nd, w.seed(73))
+    jobs_s, jobs_d, spts, dpts, host, off = [], [], [], [], [], 0
+    for n, P in zip(lens, pages):
+        gb, _ = gk.gk_blob_size(g_geom, n)
+        hb = torch.empty(G * gb, dtype=torch.uint8, pin_memory=True)
+        hs = torch.empty(G * P, dtype=torch.int64, pin_memory=True)
+        spts.append(sperm[off:off + P])
+        dpts.append(dperm[off:off + P])
+        host.append((hb, hs, gb))
+        jobs_s.append(gk.Job(hb, hs, torch.from_numpy(spts[-1].copy()).cuda(), n))
+        jobs_d.append(gk.Job(hb, hs, torch.from_numpy(dpts[-1].copy()).cuda(), n))
+        off += P
+    status = torch.full((3,), 255, dtype=torch.uint8, device="cuda")
+    ctx.gk_pack_layerwise(G, src, jobs_s, status, host=True)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0, 0, 0]
+    # sampled (block, group, page) records against the oracle
+    rng = np.random.default_rng(w.seed(74))
+    sv = _view(w, src)
+    for _ in range(12):
+        j, k = int(rng.integers(0, 3)), int(rng.integers(0, G))
+        P = pages[j]
+        p = int(rng.integers(0, P)) if rng.random() < 0.6 else P - 1
+        t = min(T, lens[j] - p * T)
+        page = sv[k * gl:(k + 1) * gl, :, int(spts[j][p])].contiguous().cpu().numpy().reshape(-1)
+        blob, sums, code, _ = oracle.pack(og_group, oracle.Cache(page, 1, 2 * s, s, s), np.zeros(1, dtype=np.int32), t)
+        assert code == 0
+        hb, hs, gb = host[j]
+        lo = k * gb + oracle.record_offset(og_group, p)
+        assert np.array_equal(hb[lo:lo + blob.size].numpy(), blob), (j, k, p)
+        assert int(hs[k * P + p].item()) & 0xFFFFFFFFFFFFFFFF == int(sums[0])
+    # damage block 1 inside group 5, then load
+    host[1][0][5 * host[1][2] + 1_000_003] ^= 0x20
+    mask = torch.full((3,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.full((3,), -7, dtype=torch.int32, device="cuda")
+    gm = torch.full((G, 3), 255, dtype=torch.uint8, device="cuda")
+    seen = []
+    ctx.gk_restore_layerwise(G, jobs_d, dst, mask, fb, gm, lambda k, l0, nl, st: seen.append((k, l0, nl)), host=True)
+    torch.cuda.synchronize()
+    assert seen == [(k, k * gl, gl) for k in range(G)]
+    want_gm = [[0, 0, 0] for _ in range(G)]
+    want_gm[5][1] = 1
+    assert gm.cpu().tolist() == want_gm and mask.cpu().tolist() == [0, 1, 0]
+    assert fb.cpu().tolist()[1] == 1_000_003 // oracle.record_bytes(og_group, 4096, 0)
+    dv, zv = _view(w, dst), sentinel.view(w.layers, 2, Nd, T, -1)
+    untouched = torch.ones(Nd, dtype=torch.bool, device="cuda")
+    for j, (n, P) in enumerate(zip(lens, pages)):
+        full = n // T
+        s_idx = torch.from_numpy(spts[j][:full].astype(np.int64)).cuda()
+        d_idx = torch.from_numpy(dpts[j][:full].astype(np.int64)).cuda()
+        untouched[torch.from_numpy(dpts[j].astype(np.int64)).cuda()] = False
+        for k in range(G):
+            ls = slice(k * gl, (k + 1) * gl)
+            if want_gm[k][j]:
+                assert torch.equal(dv[ls][:, :, d_idx], zv[ls][:, :, d_idx])        # the failing group wrote nothing
+            else:
+                assert torch.equal(dv[ls][:, :, d_idx], sv[ls][:, :, s_idx])
+        if full < P:
+            t, sp, dp = n - full * T, int(spts[j][full]), int(dpts[j][full])
+            assert torch.equal(dv[:, :, dp, :t], sv[:, :, sp, :t])
+            assert torch.equal(dv[:, :, dp, t:], zv[:, :, dp, t:])
+    rest = torch.nonzero(untouched).flatten()
+    assert torch.equal(dv[:, :, rest], zv[:, :, rest])
+    assert ctx.gk_get_stats()["device_wait_expired"] == 0
+    ctx.close()
