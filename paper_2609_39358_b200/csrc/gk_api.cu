@@ -507,6 +507,24 @@ uint32_t stream_grid(const gk_ctx *c, int occ, uint32_t n_items)
     return g ? g : 1u;
 }
 
+// Per-kernel timing (tuning key "profile"): takes a pair of events from the pool, records the
+// first one, and hands the pair back; the caller records the second one behind its launch.
+int prof_begin(gk_ctx *c, int cls, cudaStream_t st, gk_ctx::ProfSlot **slot)
+{
+    *slot = nullptr;
+    if (!c->profile) return GK_OK;
+    if (c->prof_used == c->prof_pool.size()) {
+        gk_ctx::ProfSlot ns{};
+        GK_CUDA(c, cudaEventCreate(&ns.a));
+        GK_CUDA(c, cudaEventCreate(&ns.b));
+        c->prof_pool.push_back(ns);
+    }
+    *slot = &c->prof_pool[c->prof_used++];
+    (*slot)->cls = cls;
+    GK_CUDA(c, cudaEventRecord((*slot)->a, st));
+    return GK_OK;
+}
+
 // Launches a streaming kernel; right behind the small-call preparation kernel it is
 // launched as a programmatic dependent, so that its CTAs are resident and their
 // rings set up by the time the preparation kernel ends.
@@ -538,17 +556,8 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
     }
     const uint32_t grid = stream_grid(c, occ, items);
     gk_ctx::ProfSlot *slot = nullptr;
-    if (c->profile) {
-        if (c->prof_used == c->prof_pool.size()) {
-            gk_ctx::ProfSlot ns{};
-            GK_CUDA(c, cudaEventCreate(&ns.a));
-            GK_CUDA(c, cudaEventCreate(&ns.b));
-            c->prof_pool.push_back(ns);
-        }
-        slot = &c->prof_pool[c->prof_used++];
-        slot->cls = MODE;  // kSingle == 3: booked with the fused restore kernel
-        GK_CUDA(c, cudaEventRecord(slot->a, st));
-    }
+    int rc_prof = prof_begin(c, MODE, st, &slot);  // kSingle == 3: booked with the fused restore kernel
+    if (rc_prof != GK_OK) return rc_prof;
     // every work item is drawn once, and every CTA draws once more to learn that none is left
     StreamParams Q = P;
     const int ci = MODE == kCommit ? 1 : 0;
@@ -589,17 +598,8 @@ int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
     }
     const uint32_t grid = stream_grid(c, c->occ_fused, items);
     gk_ctx::ProfSlot *slot = nullptr;
-    if (c->profile) {
-        if (c->prof_used == c->prof_pool.size()) {
-            gk_ctx::ProfSlot ns{};
-            GK_CUDA(c, cudaEventCreate(&ns.a));
-            GK_CUDA(c, cudaEventCreate(&ns.b));
-            c->prof_pool.push_back(ns);
-        }
-        slot = &c->prof_pool[c->prof_used++];
-        slot->cls = 3;
-        GK_CUDA(c, cudaEventRecord(slot->a, st));
-    }
+    int rc_prof = prof_begin(c, 3, st, &slot);
+    if (rc_prof != GK_OK) return rc_prof;
     StreamParams Q = P;
     Q.ctr_base_v = c->ctr_next[0];
     Q.ctr_base_c = c->ctr_next[1];
