@@ -1048,3 +1048,20 @@ def test_argument_errors(gk):
     with pytest.raises(gk.GkError):
         gk.Context(gk.Geom(2, 1, 4, 16), 0)               # row of 8 bytes: not a multiple of 16
     ctx.close()
+
+
+def test_round_trip_from_plain_c(gk, tmp_path):
+    """The C ABI used from a C program that knows nothing of Python or torch."""
+    import os
+    import subprocess
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    libdir = os.path.join(root, "paper_2609_39358_b200")
+    cuda = os.environ.get("CUDA_HOME", "/usr/local/cuda")
+    exe = tmp_path / "roundtrip_gpu"
+    build = subprocess.run(["gcc", "-std=c11", "-O1", "-Wall", "-Wextra", "-Werror", os.path.join(root, "tests", "c", "roundtrip_gpu.c"),
+                            "-o", str(exe), "-I" + os.path.join(cuda, "include"), "-L" + libdir, "-l:libgk.so",
+                            "-L" + os.path.join(cuda, "lib64"), "-lcudart", "-Wl,-rpath," + libdir,
+                            "-Wl,-rpath," + os.path.join(cuda, "lib64")], capture_output=True, text=True)
+    assert build.returncode == 0, build.stderr
+    run = subprocess.run([str(exe)], capture_output=True, text=True, timeout=120)
+    assert run.returncode == 0 and "roundtrip ok" in run.stdout, (run.returncode, run.stdout, run.stderr)
