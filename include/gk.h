@@ -76,15 +76,19 @@ extern "C" {
 #define GK_BF16 0u
 #define GK_FP8_E4M3 1u
 
-/* Per-job result codes (mask entries).  Any non-zero code means that not one
- * byte of that job was written to the destination. */
+/* Per-job result codes (mask entries).  Codes 1 to 3 mean that not one byte of
+ * that job was written to the destination; the commit decision of a job is taken
+ * once, for the whole job, so a job is never reported OK and written in part. */
 #define GK_JOB_OK 0u          /* every page verified; block committed */
 #define GK_JOB_CHECKSUM 1u    /* a page record failed its checksum */
 #define GK_JOB_PAGE_TABLE 2u  /* page id out of [0,num_pages), or a destination page
                                  claimed more than once within the call */
 #define GK_JOB_MISSING 3u     /* blob or checksums pointer is null */
-#define GK_JOB_TIMEOUT 4u     /* a bounded wait inside a kernel ran out; nothing of
-                                 the call was committed */
+#define GK_JOB_TIMEOUT 4u     /* a bounded wait inside a kernel ran out before this job was known
+                                 to have verified (or the context still carries an earlier such
+                                 failure, see gk_ctx_clear_error): the job is NOT restored.  Its
+                                 destination pages are untouched, except in the one case described
+                                 at gk_stats.device_wait_expired */
 
 /* Test hook for sabotage tests (Section 3, sabotage-testing paragraph): switches the
  * checksum defence off so that a test can show the attack succeeds without it.
@@ -96,7 +100,9 @@ extern "C" {
  * library (the paper leaves the cache layout to the runtime it wraps). */
 #define GK_FLAG_HEAD_MAJOR 2u
 
-/* Single-pass restore.  Section 2.2 has the runtime recompute every block whose
+/* Single-pass restore.  NOT fail-closed: unverified bytes are written (into the
+ * failing block's own pages); a departure from the block-level rule, off by default.
+ * Section 2.2 has the runtime recompute every block whose
  * record fails a check, which rewrites that block's pages; a caller that does so
  * may set this flag: gk_restore* then checks and scatters each record in ONE pass
  * over the blob (2 bytes of memory traffic per blob byte instead of 3).  A block
@@ -145,10 +151,19 @@ typedef struct {
     uint64_t calls_pack, calls_restore, calls_restore_host;
     uint64_t jobs, pages, bytes_blob; /* submitted so far */
     uint64_t kernels_launched;        /* kernels enqueued by this context so far */
-    uint32_t device_wait_expired;     /* non-zero once a bounded wait inside a kernel has run out:
-                                         from then on no call of this context commits anything and
-                                         the destination of the call that hit it is undefined */
-    uint32_t reserved;
+    uint32_t device_wait_expired;     /* non-zero once a bounded wait inside a kernel has run out.
+                                         In the call that hit it, every job is either committed whole
+                                         and reported GK_JOB_OK (it had verified before) or reported
+                                         GK_JOB_TIMEOUT with nothing of it written.  The one exception:
+                                         a wait on the kernel's own copy pipeline (a bulk copy that
+                                         never completes, i.e. a hardware fault) leaves the jobs that
+                                         had tiles in flight in that CTA partly written; they are
+                                         reported GK_JOB_TIMEOUT, never GK_JOB_OK.  Every later call of
+                                         the context reports GK_JOB_TIMEOUT for all jobs and writes
+                                         nothing until gk_ctx_clear_error */
+    uint32_t allocations;             /* device or pinned-host (re)allocations made so far by calls on this
+                                         context (each one synchronises the device): stays constant once
+                                         gk_ctx_reserve has sized everything */
     uint64_t calls_restore_stream;    /* its windows are counted in calls_restore_host as well */
 } gk_stats;
 
@@ -162,6 +177,30 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device);
 int gk_ctx_destroy(gk_ctx *ctx);
 /* Text of the last error of this context (never NULL; empty if none). */
 const char *gk_last_error(const gk_ctx *ctx);
+
+/* Sizes everything a context allocates lazily, so that no later call within the
+ * stated bounds allocates, frees or synchronises the device (a serving engine
+ * calls this once at start-up; Section 2.2 has a request complete normally
+ * whatever happens to stored state, which a mid-request device synchronisation
+ * would not honour).  Bounds, per call: max_jobs jobs, max_pages page records in
+ * total, a destination (or source) cache of num_pages pages and, for the host
+ * tier, max_host_batch_bytes of blob bytes per staging slot (two slots are kept;
+ * 0 = the host tier is not used; a host-tier call stages min(the call's blobs,
+ * 256 MiB) per slot, or its largest single blob if that is larger).  Covers
+ * gk_pack*, gk_restore*, gk_verify, gk_commit, gk_page_checksums and the
+ * layer-wise and streaming calls; gk_fingerprints and gk_blob_digests size their
+ * own scratch on first use.  Synchronises the device.  gk_get_stats().allocations
+ * tells whether a later call had to grow something after all. */
+int gk_ctx_reserve(gk_ctx *ctx, uint32_t max_jobs, uint64_t max_pages, uint64_t num_pages,
+                   uint64_t max_host_batch_bytes);
+
+/* Clears the context's record of a device wait that ran out (Section 5, second
+ * item, and Section 2.2: a failed load is a miss, the block is recomputed and the
+ * request completes; the store stays usable).  A wait can run out without any
+ * fault, e.g. on a GPU that is time-sliced with another process.  Enqueued on
+ * `stream`: calls issued after it on that stream commit again.  The caller should
+ * first have treated every job reported GK_JOB_TIMEOUT as not restored. */
+int gk_ctx_clear_error(gk_ctx *ctx, void *stream);
 
 /* Save (Section 2.2: the block's state is written out once it has been computed;
  * here: gathered into one contiguous record with checksums).  jobs is a HOST array of n_jobs entries;
@@ -229,7 +268,8 @@ int gk_commit(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk_cache *
  * in PINNED host memory.  Blobs are copied in batches into an internal device
  * staging ring on an internal copy stream while the previous batch is verified
  * and committed on `stream`; the checksum is taken over the bytes as they arrived
- * in device memory.  All page tables are validated before the first copy.  The
+ * in device memory.  All page tables are validated on `stream` before anything is
+ * verified or committed (the copies, on their own stream, may start earlier).  The
  * call returns after the last stage has been enqueued; results are valid after
  * `stream` has been synchronised.  The host buffers must stay valid until then.
  * The first copy starts only when the work already enqueued on `stream` has
@@ -269,7 +309,9 @@ int gk_restore_stream(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk
                       uint8_t *mask_dev, int32_t *first_bad_page_dev, gk_window_fn consume, void *user,
                       void *stream);
 
-/* Layer-wise save and load.  A consumer that walks the layers in order (a
+/* Layer-wise save and load.  Fail-closed per (block, group of layers), not per
+ * block: a departure from the block-level rule that the caller opts into by using
+ * these calls; never the default format.  A consumer that walks the layers in order (a
  * forward pass) can start on the first layers of a block while the later ones
  * are still arriving from the host tier, if the block's record is cut by layer
  * groups (Section 4.3 streams saved state in from storage; the paper gives no
@@ -356,10 +398,14 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * the GPU), "profile" (1 = time every streaming kernel, see gk_get_kernel_times),
  * "fused" (1, the default: gk_restore verifies and commits in one launch; 0: a
  * verify launch, a checksum-compare launch and a commit launch), "wait_limit_ms"
- * (time limit of every wait inside a kernel, default 2000), "test_drop_verify"
- * (tests only: the fused restore kernel verifies nothing, so that every commit
- * wait runs into its limit and the time-out handling can be checked without
- * hanging or faulting the GPU). */
+ * (time limit of every wait inside a kernel, default 2000), "commit_reverse" (1,
+ * the default: the commit side reads a job's records from the last to the first,
+ * so that what was verified last is still in L2), "l2_hints" (bit 0: verify loads
+ * ask L2 to keep the lines, bit 1: commit loads ask it to drop them; default 0),
+ * "test_drop_verify" (tests only: with value k > 0 the fused restore kernel
+ * verifies nothing of the jobs k-1, k, ..., so that the commit waits of exactly
+ * those jobs run into their limit and the time-out handling can be checked
+ * without hanging or faulting the GPU). */
 int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
 
 /* Page checksums of a device blob for callers that must not allocate.  (The
@@ -392,7 +438,11 @@ int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
  * overlap on the GPU -- different streams, or the same blob checked from two
  * threads -- race on it and may both return wrong checksums, so serialise them.
  * Work is enqueued on `stream`; checksums_dev is valid once it has been
- * synchronised. */
+ * synchronised.  Should a bounded wait inside the kernel run out (it cannot be
+ * reported here: the call has returned), NO entry of checksums_dev is written:
+ * a caller that must tell fills checksums_dev with a value of its own first
+ * (a CRC-64 can take any value, so compare with the stored checksums: an
+ * unwritten array fails that comparison like damage does). */
 #define GK_NOALLOC_MAX_PAGES 8192u
 #define GK_NOALLOC_MAX_PAGE_TOKENS 256u
 int gk_page_checksums_noalloc(const gk_geom *geom, const void *blob_dev, uint32_t n_tokens,

@@ -29,7 +29,7 @@ EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "
            "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times",
            "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit", "gk_restore_stream",
            "gk_fingerprints", "gk_blob_digests", "gk_pack_layerwise", "gk_pack_layerwise_host",
-           "gk_restore_layerwise", "gk_restore_layerwise_host"]
+           "gk_restore_layerwise", "gk_restore_layerwise_host", "gk_ctx_reserve", "gk_ctx_clear_error"]
 
 
 class GkError(RuntimeError):
@@ -60,7 +60,7 @@ class CStats(ctypes.Structure):
     _fields_ = [("calls_pack", ctypes.c_uint64), ("calls_restore", ctypes.c_uint64),
                 ("calls_restore_host", ctypes.c_uint64), ("jobs", ctypes.c_uint64), ("pages", ctypes.c_uint64),
                 ("bytes_blob", ctypes.c_uint64), ("kernels_launched", ctypes.c_uint64),
-                ("device_wait_expired", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+                ("device_wait_expired", ctypes.c_uint32), ("allocations", ctypes.c_uint32),
                 ("calls_restore_stream", ctypes.c_uint64)]
 
 
@@ -167,6 +167,10 @@ def load_library() -> ctypes.CDLL:
     L.gk_page_checksums_noalloc.argtypes = [ctypes.POINTER(CGeom), vp, u32, vp, ctypes.c_int, vp]
     L.gk_ctx_set_tuning.restype = ctypes.c_int
     L.gk_ctx_set_tuning.argtypes = [vp, ctypes.c_char_p, u32]
+    L.gk_ctx_reserve.restype = ctypes.c_int
+    L.gk_ctx_reserve.argtypes = [vp, u32, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64]
+    L.gk_ctx_clear_error.restype = ctypes.c_int
+    L.gk_ctx_clear_error.argtypes = [vp, vp]
     _lib = L
     return L
 
@@ -297,6 +301,13 @@ class Context:
     def set_tuning(self, key: str, value: int):
         self._check(self._lib.gk_ctx_set_tuning(self._h, key.encode(), value), "gk_ctx_set_tuning")
 
+    def gk_ctx_reserve(self, max_jobs: int, max_pages: int, num_pages: int, max_host_batch_bytes: int = 0):
+        self._check(self._lib.gk_ctx_reserve(self._h, max_jobs, max_pages, num_pages, max_host_batch_bytes),
+                    "gk_ctx_reserve")
+
+    def gk_ctx_clear_error(self, stream=None):
+        self._check(self._lib.gk_ctx_clear_error(self._h, _stream_handle(stream)), "gk_ctx_clear_error")
+
     def gk_pack_batch(self, src: Cache, jobs: Sequence[Job], status: Optional[torch.Tensor] = None, stream=None):
         cc = src.c()
         self._check(self._lib.gk_pack_batch(self._h, ctypes.byref(cc), self._jobs(jobs), len(jobs), _ptr(status),
@@ -423,4 +434,4 @@ class Context:
     def gk_get_stats(self) -> dict:
         st = CStats()
         self._check(self._lib.gk_get_stats(self._h, ctypes.byref(st)), "gk_get_stats")
-        return {name: int(getattr(st, name)) for name, _ in CStats._fields_ if name != "reserved"}
+        return {name: int(getattr(st, name)) for name, _ in CStats._fields_ }

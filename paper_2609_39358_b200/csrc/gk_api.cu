@@ -5,6 +5,7 @@
 // runs in the kernels of gk_kernels.cuh; there is no CPU fallback.
 #include "../../include/gk.h"
 
+#include <algorithm>
 #include <cmath>
 #include <cstdarg>
 #include <cstdio>
@@ -103,7 +104,9 @@ struct gk_ctx {
     unsigned long long wait_limit_ns = kWaitLimitNs;
     uint32_t ctr_next[2] = {0, 0};  // what the device work counters will read when the next launch of
                                     // the current call starts (the first kernel of a call zeroes them)
-    bool test_drop_verify = false;  // test hook: see gk_ctx_set_tuning
+    uint32_t test_drop_verify = 0;  // test hook: see gk_ctx_set_tuning
+    bool commit_reverse = true;     // commit side walks a job's pages from the last to the first
+    uint32_t l2_hints = 0;          // bit 0: verify loads evict_last, bit 1: commit loads evict_first
     uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
     uint32_t commit_seg_tiles = 0;
     uint32_t grid_cap = 0;       // 0: SMs * occupancy
@@ -116,9 +119,12 @@ struct gk_ctx {
     // growing device workspace and pinned staging for job tables
     uint8_t *d_ws = nullptr;
     size_t ws_cap = 0;
-    uint8_t *h_stage = nullptr;
-    size_t h_stage_cap = 0;
-    cudaEvent_t ev_stage = nullptr;  // upload of the job table has been consumed
+    // pinned staging for job tables, two halves used in turn: the host fills one while the
+    // upload of the previous call may still be reading the other
+    uint8_t *h_stage = nullptr;      // 2 * h_stage_cap bytes
+    size_t h_stage_cap = 0;          // bytes of one half
+    cudaEvent_t ev_stage[2] = {nullptr, nullptr};  // upload from that half has been consumed
+    uint32_t stage_next = 0;
     cudaEvent_t ev_entry = nullptr;  // host tier: where the caller's stream stood when the call came in
 
     // host tier
@@ -152,6 +158,9 @@ struct gk_ctx {
     struct SegPowers { uint64_t seg_bytes = 0; uint64_t x_seg = 0; std::vector<uint64_t> pw; uint64_t used = 0; };
     SegPowers seg_cache[4];
     uint64_t seg_cache_clock = 0;
+
+    // host tier: buffers already seen to be pinned host memory (exact start addresses)
+    std::vector<const void *> pinned_seen;
 
     gk_stats stats{};
     char err[512] = {0};
@@ -317,7 +326,7 @@ Tiling commit_tiling(const gk_ctx *c, uint64_t total_pages, int occ)
 
 // Views into the workspace for one call.
 struct WsLayout {
-    size_t jobs, page_job, seg_res, bad_range, bad_dup, bad_crc, page_cnt, job_done, claims, total;
+    size_t jobs, page_job, page_acc, bad_range, bad_dup, bad_crc, page_cnt, job_done, job_latch, claims, total;
 };
 
 WsLayout ws_layout(uint32_t n_jobs, uint64_t total_pages, uint32_t nseg_max, uint64_t num_pages)
@@ -326,12 +335,13 @@ WsLayout ws_layout(uint32_t n_jobs, uint64_t total_pages, uint32_t nseg_max, uin
     size_t o = 0;
     l.jobs = o;      o = align_up(o + (size_t)n_jobs * sizeof(JobDev) + (size_t)nseg_max * 8, 256);  // + seg_pow
     l.page_job = o;  o = align_up(o + (size_t)total_pages * 4, 256);
-    l.seg_res = o;   o = align_up(o + (size_t)total_pages * nseg_max * 8, 256);
+    l.page_acc = o;  o = align_up(o + (size_t)total_pages * 8, 256);
     l.bad_range = o; o = align_up(o + (size_t)n_jobs * 4, 256);
     l.bad_dup = o;   o = align_up(o + (size_t)n_jobs * 4, 256);
     l.bad_crc = o;   o = align_up(o + (size_t)n_jobs * 4, 256);
     l.page_cnt = o;  o = align_up(o + (size_t)total_pages * 4, 256);
     l.job_done = o;  o = align_up(o + (size_t)n_jobs * 4, 256);
+    l.job_latch = o; o = align_up(o + (size_t)n_jobs * 4, 256);
     l.claims = o;    o = align_up(o + (size_t)num_pages * 8, 256);
     l.total = o;
     return l;
@@ -350,22 +360,38 @@ int ensure_workspace(gk_ctx *c, size_t need)
         return fail(c, GK_ERR_NOMEM, "workspace of %zu bytes", cap);
     }
     c->ws_cap = cap;
+    c->stats.allocations++;
     return GK_OK;
 }
 
 int ensure_host_stage(gk_ctx *c, size_t need)
 {
     if (need <= c->h_stage_cap) return GK_OK;
-    GK_CUDA(c, cudaEventSynchronize(c->ev_stage));
+    for (int i = 0; i < 2; ++i) GK_CUDA(c, cudaEventSynchronize(c->ev_stage[i]));
     if (c->h_stage) cudaFreeHost(c->h_stage);
     c->h_stage = nullptr;
     c->h_stage_cap = 0;
     const size_t cap = align_up(need * 2, 1 << 16);
-    if (cudaMallocHost(&c->h_stage, cap) != cudaSuccess) {
+    if (cudaMallocHost(&c->h_stage, 2 * cap) != cudaSuccess) {
         cudaGetLastError();
-        return fail(c, GK_ERR_NOMEM, "pinned staging of %zu bytes", cap);
+        return fail(c, GK_ERR_NOMEM, "pinned staging of %zu bytes", 2 * cap);
     }
     c->h_stage_cap = cap;
+    c->stats.allocations++;
+    return GK_OK;
+}
+
+// The half of the pinned staging area that the next upload may fill: waits only for the
+// upload that used this half two calls ago.
+int next_host_stage(gk_ctx *c, size_t need, uint8_t **out, cudaEvent_t *ev)
+{
+    int rc = ensure_host_stage(c, need);
+    if (rc != GK_OK) return rc;
+    const uint32_t h = c->stage_next;
+    c->stage_next ^= 1u;
+    GK_CUDA(c, cudaEventSynchronize(c->ev_stage[h]));
+    *out = c->h_stage + (size_t)h * c->h_stage_cap;
+    *ev = c->ev_stage[h];
     return GK_OK;
 }
 
@@ -396,12 +422,13 @@ WorkDev make_work(gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t total_
     w.page_begin = 0;
     w.total_pages = total_pages;
     w.page_job = (int32_t *)(c->d_ws + l.page_job);
-    w.seg_res = (uint64_t *)(c->d_ws + l.seg_res);
+    w.page_acc = (uint64_t *)(c->d_ws + l.page_acc);
     w.bad_range = (int32_t *)(c->d_ws + l.bad_range);
     w.bad_dup = (int32_t *)(c->d_ws + l.bad_dup);
     w.bad_crc = (int32_t *)(c->d_ws + l.bad_crc);
     w.page_cnt = (uint32_t *)(c->d_ws + l.page_cnt);
     w.job_done = (uint32_t *)(c->d_ws + l.job_done);
+    w.job_latch = (uint32_t *)(c->d_ws + l.job_latch);
     w.claims = (unsigned long long *)(c->d_ws + l.claims);
     w.error = c->d_error;
     w.work_ctr = c->d_error + 16;
@@ -459,16 +486,17 @@ int upload_jobs(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const WsLayout &
                 uint64_t *total_pages_out, uint64_t *total_bytes_out)
 {
     const size_t table_bytes = (size_t)n_jobs * sizeof(JobDev) + (size_t)crc.nseg_max * 8;
-    int rc = ensure_host_stage(c, table_bytes);
+    uint8_t *stage = nullptr;
+    cudaEvent_t ev = nullptr;
+    int rc = next_host_stage(c, table_bytes, &stage, &ev);
     if (rc != GK_OK) return rc;
-    GK_CUDA(c, cudaEventSynchronize(c->ev_stage));
-    JobDev *h = (JobDev *)c->h_stage;
+    JobDev *h = (JobDev *)stage;
     if ((rc = fill_job_table(c, jobs, n_jobs, h, blob_override, sums_override, need_tables, total_pages_out,
                              total_bytes_out)) != GK_OK)
         return rc;
-    fill_seg_pow(c, crc, reinterpret_cast<uint64_t *>(c->h_stage + (size_t)n_jobs * sizeof(JobDev)));
+    fill_seg_pow(c, crc, reinterpret_cast<uint64_t *>(stage + (size_t)n_jobs * sizeof(JobDev)));
     GK_CUDA(c, cudaMemcpyAsync(c->d_ws + l.jobs, h, table_bytes, cudaMemcpyHostToDevice, st));
-    GK_CUDA(c, cudaEventRecord(c->ev_stage, st));
+    GK_CUDA(c, cudaEventRecord(ev, st));
     return GK_OK;
 }
 
@@ -558,12 +586,13 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
     gk_ctx::ProfSlot *slot = nullptr;
     int rc_prof = prof_begin(c, MODE, st, &slot);  // kSingle == 3: booked with the fused restore kernel
     if (rc_prof != GK_OK) return rc_prof;
-    // every work item is drawn once, and every CTA draws once more to learn that none is left
+    // A CTA takes the item with its own number first and draws the others from the counter; every
+    // CTA that has an item draws once more to learn that none is left: `items` draws per launch.
     StreamParams Q = P;
     const int ci = MODE == kCommit ? 1 : 0;
     if (ci) Q.ctr_base_c = c->ctr_next[1];
     else Q.ctr_base_v = c->ctr_next[0];
-    c->ctr_next[ci] += items + grid;
+    c->ctr_next[ci] += items;
     GK_CUDA(c, launch_streaming(c, stream_kernel<MODE, NT, SB, ST, MINB>, grid, Cfg::kThreads, Cfg::kSmemBytes, st, Q));
     if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
@@ -603,8 +632,9 @@ int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
     StreamParams Q = P;
     Q.ctr_base_v = c->ctr_next[0];
     Q.ctr_base_c = c->ctr_next[1];
+    // the verify side draws every item (and once more per CTA); the commit side as in launch_stream
     c->ctr_next[0] += P.n_items + grid;
-    c->ctr_next[1] += P.n_items_c + grid;
+    c->ctr_next[1] += P.n_items_c;
     GK_CUDA(c, launch_streaming(c, restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE,
                                                   GK_FUSED_CSTAGES, GK_FUSED_MINB>,
                                 grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st, Q));
@@ -656,6 +686,89 @@ struct HostPlan {
     uint64_t pages = 0;
 };
 
+// The two device staging slots of the host tier, each of at least `want` bytes.
+int ensure_slots(gk_ctx *c, uint64_t want)
+{
+    if (want < 256) want = 256;
+    if (want <= c->slot_cap) return GK_OK;
+    GK_CUDA(c, cudaDeviceSynchronize());
+    for (int i = 0; i < kSlots; ++i) {
+        if (c->d_slot[i]) cudaFree(c->d_slot[i]);
+        c->d_slot[i] = nullptr;
+        c->slot_used[i] = false;
+    }
+    c->slot_cap = 0;
+    c->slot_next = 0;
+    for (int i = 0; i < kSlots; ++i) {
+        if (cudaMalloc(&c->d_slot[i], want) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(c, GK_ERR_NOMEM, "host-tier staging slot of %llu bytes", (unsigned long long)want);
+        }
+    }
+    c->slot_cap = want;
+    c->stats.allocations++;
+    return GK_OK;
+}
+
+// The page ids 0..num_pages-1 on the device; the windows of a streaming restore take their
+// page tables as slices of them.
+int ensure_iota(gk_ctx *c, uint64_t num_pages, cudaStream_t st)
+{
+    if (c->iota_cap >= num_pages) return GK_OK;
+    GK_CUDA(c, cudaDeviceSynchronize());  // an earlier call's consumer may still read the old array
+    if (c->d_iota) cudaFree(c->d_iota);
+    c->d_iota = nullptr;
+    c->iota_cap = 0;
+    if (cudaMalloc(&c->d_iota, num_pages * sizeof(int32_t)) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, GK_ERR_NOMEM, "page id array of %llu entries", (unsigned long long)num_pages);
+    }
+    c->iota_cap = num_pages;
+    c->stats.allocations++;
+    iota_kernel<<<(unsigned)((num_pages + 255) / 256), 256, 0, st>>>(c->d_iota, (uint32_t)num_pages);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched++;
+    return GK_OK;
+}
+
+// Layer-wise restore: per-group result arrays (pages always, codes unless the caller keeps them).
+int ensure_group_tmp(gk_ctx *c, uint32_t n_jobs)
+{
+    const size_t need = align_up((size_t)n_jobs * 4, 256) + (size_t)n_jobs;
+    if (need <= c->group_tmp_cap) return GK_OK;
+    GK_CUDA(c, cudaDeviceSynchronize());
+    if (c->d_group_tmp) cudaFree(c->d_group_tmp);
+    c->d_group_tmp = nullptr;
+    c->group_tmp_cap = 0;
+    if (cudaMalloc(&c->d_group_tmp, need * 2) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(c, GK_ERR_NOMEM, "layer-wise result arrays of %zu bytes", need * 2);
+    }
+    c->group_tmp_cap = need * 2;
+    c->stats.allocations++;
+    return GK_OK;
+}
+
+// Pinned-memory check of the host tier.  The driver is asked once per buffer: start addresses
+// that passed are remembered (sorted, at most 65,536 of them; the list starts afresh when full),
+// so a call over thousands of blocks that were seen before costs no driver call at all.
+bool is_pinned(gk_ctx *c, const void *ptr)
+{
+    auto it = std::lower_bound(c->pinned_seen.begin(), c->pinned_seen.end(), ptr);
+    if (it != c->pinned_seen.end() && *it == ptr) return true;
+    cudaPointerAttributes a{};
+    if (cudaPointerGetAttributes(&a, ptr) != cudaSuccess || a.type != cudaMemoryTypeHost) {
+        cudaGetLastError();
+        return false;
+    }
+    if (c->pinned_seen.size() >= 65536) {
+        c->pinned_seen.clear();
+        it = c->pinned_seen.end();
+    }
+    c->pinned_seen.insert(it, ptr);
+    return true;
+}
+
 int make_host_plan(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, bool allow_missing, HostPlan &hp)
 {
     std::vector<HostPlan::Plan> &plan = hp.plan;
@@ -670,12 +783,9 @@ int make_host_plan(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, bool allow_mi
         plan[j].need = 0;
         pages += np;
         if (jobs[j].blob && jobs[j].checksums) {
-            cudaPointerAttributes a{};
             for (const void *ptr : {(const void *)jobs[j].blob, (const void *)jobs[j].checksums}) {
-                if (cudaPointerGetAttributes(&a, ptr) != cudaSuccess || a.type != cudaMemoryTypeHost) {
-                    cudaGetLastError();
+                if (!is_pinned(c, ptr))
                     return fail(c, GK_ERR_NOT_PINNED, "job %u: blob and checksums must be pinned host memory", j);
-                }
             }
             plan[j].need = align_up(plan[j].blob_bytes, 256) + align_up(plan[j].sums_bytes, 256);
         } else if (!allow_missing) {
@@ -689,24 +799,8 @@ int make_host_plan(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, bool allow_mi
     uint64_t want = max_need;
     const uint64_t batch_target = 256ull << 20;
     if (want < batch_target) want = total_need < batch_target ? total_need : batch_target;
-    if (want < 256) want = 256;
-    if (want > c->slot_cap) {
-        GK_CUDA(c, cudaDeviceSynchronize());
-        for (int i = 0; i < kSlots; ++i) {
-            if (c->d_slot[i]) cudaFree(c->d_slot[i]);
-            c->d_slot[i] = nullptr;
-            c->slot_used[i] = false;
-        }
-        c->slot_cap = 0;
-        c->slot_next = 0;
-        for (int i = 0; i < kSlots; ++i) {
-            if (cudaMalloc(&c->d_slot[i], want) != cudaSuccess) {
-                cudaGetLastError();
-                return fail(c, GK_ERR_NOMEM, "host-tier staging slot of %llu bytes", (unsigned long long)want);
-            }
-        }
-        c->slot_cap = want;
-    }
+    int rc_slots = ensure_slots(c, want);
+    if (rc_slots != GK_OK) return rc_slots;
     // assign every job a place in a slot
     hp.blob_dev.assign(n_jobs, nullptr);
     hp.sums_dev.assign(n_jobs, nullptr);
@@ -823,7 +917,8 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
         cudaMemcpy(c->d_thread_const, tc.data(), tc.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemset(c->d_error, 0, 256) != cudaSuccess)
         return bail(GK_ERR_CUDA);
-    if (cudaEventCreateWithFlags(&c->ev_stage, cudaEventDisableTiming) != cudaSuccess) return bail(GK_ERR_CUDA);
+    for (int i = 0; i < 2; ++i)
+        if (cudaEventCreateWithFlags(&c->ev_stage[i], cudaEventDisableTiming) != cudaSuccess) return bail(GK_ERR_CUDA);
     if (cudaEventCreateWithFlags(&c->ev_entry, cudaEventDisableTiming) != cudaSuccess) return bail(GK_ERR_CUDA);
     for (int i = 0; i < kSlots; ++i) {
         if (cudaEventCreateWithFlags(&c->ev_slot_free[i], cudaEventDisableTiming) != cudaSuccess ||
@@ -850,7 +945,8 @@ int gk_ctx_destroy(gk_ctx *c)
         if (c->ev_slot_free[i]) cudaEventDestroy(c->ev_slot_free[i]);
         if (c->ev_copied[i]) cudaEventDestroy(c->ev_copied[i]);
     }
-    if (c->ev_stage) cudaEventDestroy(c->ev_stage);
+    for (int i = 0; i < 2; ++i)
+        if (c->ev_stage[i]) cudaEventDestroy(c->ev_stage[i]);
     if (c->ev_entry) cudaEventDestroy(c->ev_entry);
     if (c->h_stage) cudaFreeHost(c->h_stage);
     if (c->d_ws) cudaFree(c->d_ws);
@@ -875,8 +971,40 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     else if (!strcmp(key, "profile")) c->profile = value != 0;
     else if (!strcmp(key, "fused")) c->fused = value != 0;
     else if (!strcmp(key, "wait_limit_ms")) c->wait_limit_ns = (unsigned long long)(value ? value : 1u) * 1000000ull;
-    else if (!strcmp(key, "test_drop_verify")) c->test_drop_verify = value != 0;
+    else if (!strcmp(key, "test_drop_verify")) c->test_drop_verify = value;
+    else if (!strcmp(key, "commit_reverse")) c->commit_reverse = value != 0;
+    else if (!strcmp(key, "l2_hints")) c->l2_hints = value;
     else return fail(c, GK_ERR_ARG, "unknown tuning key %s", key);
+    return GK_OK;
+}
+
+int gk_ctx_reserve(gk_ctx *c, uint32_t max_jobs, uint64_t max_pages, uint64_t num_pages, uint64_t max_host_batch_bytes)
+{
+    if (!c) return GK_ERR_ARG;
+    if (max_pages > 0x7fffffffull || num_pages > 0x7fffffffull) return fail(c, GK_ERR_ARG, "too many pages");
+    DeviceGuard guard(c->device);
+    // the largest tables any call within these bounds builds: a page cut into as many segments as it has granules
+    const uint32_t seg_max = (uint32_t)((c->gd.R + VerifyCfg::kGran - 1) / VerifyCfg::kGran);
+    const WsLayout l = ws_layout(max_jobs, max_pages, seg_max, num_pages);
+    int rc;
+    if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
+    if ((rc = ensure_host_stage(c, (size_t)max_jobs * sizeof(JobDev) + (size_t)seg_max * 8)) != GK_OK) return rc;
+    if (max_jobs && (rc = ensure_group_tmp(c, max_jobs)) != GK_OK) return rc;
+    if (max_host_batch_bytes) {
+        // room for the checksums beside the blobs, and for the alignment of every job's two parts
+        const uint64_t want = max_host_batch_bytes + max_pages * 8 + (uint64_t)max_jobs * 512;
+        if ((rc = ensure_slots(c, want)) != GK_OK) return rc;
+        if (num_pages && (rc = ensure_iota(c, num_pages, 0)) != GK_OK) return rc;
+    }
+    GK_CUDA(c, cudaDeviceSynchronize());
+    return GK_OK;
+}
+
+int gk_ctx_clear_error(gk_ctx *c, void *stream)
+{
+    if (!c) return GK_ERR_ARG;
+    DeviceGuard guard(c->device);
+    GK_CUDA(c, cudaMemsetAsync(c->d_error, 0, 4, (cudaStream_t)stream));
     return GK_OK;
 }
 
@@ -983,6 +1111,8 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
     P.tlc = tlc;
     P.n_items = n_pages * tlv.nseg_max;
     P.n_items_c = n_pages * tlc.nseg_max;
+    P.commit_reverse = c->commit_reverse ? 1u : 0u;
+    P.l2_hints = c->l2_hints;
     if (c->gd.flags & GK_FLAG_SKIP_VERIFY) return launch_commit(c, P, st);
     if (c->gd.flags & GK_FLAG_SINGLE_PASS) {
         // one pass: every tile is checksummed and scattered from the same shared-memory stage;
@@ -1001,7 +1131,7 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
     if (c->fused && (!lone_big_job || c->test_drop_verify)) {
         P.fused = 1u;
         P.inline_final = 1u;
-        if (c->test_drop_verify) P.n_items = 0;  // nothing gets verified: every commit wait must run out
+        P.test_drop_from = c->test_drop_verify;  // tests: the jobs from this one on are never verified
         return launch_fused(c, P, st);
     }
     if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
@@ -1231,21 +1361,7 @@ int gk_restore_stream(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_c
             return fail(c, GK_ERR_TOO_LARGE, "job %u: %u pages do not fit a ring of %llu", j, np[j],
                         (unsigned long long)cd.num_pages);
     }
-    // the page ids 0..num_pages-1 on the device; a window's tables are slices of them
-    if (c->iota_cap < cd.num_pages) {
-        GK_CUDA(c, cudaDeviceSynchronize());  // an earlier call's consumer may still read the old array
-        if (c->d_iota) cudaFree(c->d_iota);
-        c->d_iota = nullptr;
-        c->iota_cap = 0;
-        if (cudaMalloc(&c->d_iota, cd.num_pages * sizeof(int32_t)) != cudaSuccess) {
-            cudaGetLastError();
-            return fail(c, GK_ERR_NOMEM, "page id array of %llu entries", (unsigned long long)cd.num_pages);
-        }
-        c->iota_cap = cd.num_pages;
-        iota_kernel<<<(unsigned)((cd.num_pages + 255) / 256), 256, 0, st>>>(c->d_iota, (uint32_t)cd.num_pages);
-        GK_CUDA(c, cudaGetLastError());
-        c->stats.kernels_launched++;
-    }
+    if ((rc = ensure_iota(c, cd.num_pages, st)) != GK_OK) return rc;
     std::vector<gk_job> wjobs;
     std::vector<gk_window_block> blocks;
     uint32_t j0 = 0;
@@ -1393,19 +1509,8 @@ static int restore_layerwise_impl(gk_ctx *c, uint32_t n_groups, const gk_job *jo
         if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
     DeviceGuard guard(c->device);
     cudaStream_t st = (cudaStream_t)stream;
-    // per-group result arrays: pages always, codes unless the caller keeps them
-    const size_t need = align_up((size_t)n_jobs * 4, 256) + (size_t)n_jobs;
-    if (need > c->group_tmp_cap) {
-        GK_CUDA(c, cudaDeviceSynchronize());
-        if (c->d_group_tmp) cudaFree(c->d_group_tmp);
-        c->d_group_tmp = nullptr;
-        c->group_tmp_cap = 0;
-        if (cudaMalloc(&c->d_group_tmp, need * 2) != cudaSuccess) {
-            cudaGetLastError();
-            return fail(c, GK_ERR_NOMEM, "layer-wise result arrays of %zu bytes", need * 2);
-        }
-        c->group_tmp_cap = need * 2;
-    }
+    int rc_tmp = ensure_group_tmp(c, n_jobs);
+    if (rc_tmp != GK_OK) return rc_tmp;
     int32_t *gfb = (int32_t *)c->d_group_tmp;
     uint8_t *gm_own = c->d_group_tmp + align_up((size_t)n_jobs * 4, 256);
     std::vector<gk_job> gj;
@@ -1475,10 +1580,11 @@ int gk_fingerprints(gk_ctx *c, const void *data_dev, const uint64_t *offsets_dev
     P.inner = c->d_ws + meta;
     P.keys = keys_dev;
     if (parent) {
-        if ((rc = ensure_host_stage(c, (size_t)n * 8)) != GK_OK) return rc;
-        GK_CUDA(c, cudaEventSynchronize(c->ev_stage));
-        int32_t *hp = (int32_t *)c->h_stage;
-        uint32_t *hd = (uint32_t *)(c->h_stage + (size_t)n * 4);
+        uint8_t *stage = nullptr;
+        cudaEvent_t ev = nullptr;
+        if ((rc = next_host_stage(c, (size_t)n * 8, &stage, &ev)) != GK_OK) return rc;
+        int32_t *hp = (int32_t *)stage;
+        uint32_t *hd = (uint32_t *)(stage + (size_t)n * 4);
         uint32_t max_depth = 0;
         for (uint32_t i = 0; i < n; ++i) {
             if (parent[i] < -1 || (parent[i] >= 0 && (uint32_t)parent[i] >= i))
@@ -1487,8 +1593,8 @@ int gk_fingerprints(gk_ctx *c, const void *data_dev, const uint64_t *offsets_dev
             hd[i] = parent[i] < 0 ? 0u : hd[parent[i]] + 1u;
             if (hd[i] > max_depth) max_depth = hd[i];
         }
-        GK_CUDA(c, cudaMemcpyAsync(c->d_ws, c->h_stage, (size_t)n * 8, cudaMemcpyHostToDevice, st));
-        GK_CUDA(c, cudaEventRecord(c->ev_stage, st));
+        GK_CUDA(c, cudaMemcpyAsync(c->d_ws, stage, (size_t)n * 8, cudaMemcpyHostToDevice, st));
+        GK_CUDA(c, cudaEventRecord(ev, st));
         P.parent = (const int32_t *)c->d_ws;
         P.depth = (const uint32_t *)(c->d_ws + (size_t)n * 4);
         P.max_depth = max_depth;
@@ -1607,11 +1713,11 @@ struct NoallocLayout {
     static constexpr size_t init_term = thread_const + 8 * 256;             // [max page tokens + 1] u64
     static constexpr size_t page_job = init_term + 8 * (kNoallocMaxPageTokens + 1) + 248;  // [max pages] i32
     static constexpr size_t page_cnt = page_job + 4 * (size_t)kNoallocMaxPages;            // [max pages] u32
-    static constexpr size_t seg_res = page_cnt + 4 * (size_t)kNoallocMaxPages;             // [max pages] u64
-    static constexpr size_t total = seg_res + 8 * (size_t)kNoallocMaxPages;
+    static constexpr size_t page_acc = page_cnt + 4 * (size_t)kNoallocMaxPages;            // [max pages] u64
+    static constexpr size_t total = page_acc + 8 * (size_t)kNoallocMaxPages;
 };
 static_assert(GK_CRC_NT <= 256, "thread constant table");
-static_assert(NoallocLayout::page_job % 256 == 0 && NoallocLayout::seg_res % 8 == 0, "scratch alignment");
+static_assert(NoallocLayout::page_job % 256 == 0 && NoallocLayout::page_acc % 8 == 0, "scratch alignment");
 
 // The scratch itself: about 133 KiB per GPU that loads the library, held until exit.
 // In host code this name is only a stand-in for the symbol; the device address
@@ -1640,6 +1746,7 @@ __global__ void noalloc_setup_kernel(unsigned char *scratch, JobDev job, GeomDev
     uint64_t *it = reinterpret_cast<uint64_t *>(scratch + NoallocLayout::init_term);
     int32_t *page_job = reinterpret_cast<int32_t *>(scratch + NoallocLayout::page_job);
     uint32_t *page_cnt = reinterpret_cast<uint32_t *>(scratch + NoallocLayout::page_cnt);
+    uint64_t *page_acc = reinterpret_cast<uint64_t *>(scratch + NoallocLayout::page_acc);
     if (threadIdx.x == 0) {
         *jd = job;
         words[0] = kNoPage;  // bad_range
@@ -1649,6 +1756,7 @@ __global__ void noalloc_setup_kernel(unsigned char *scratch, JobDev job, GeomDev
         words[4] = 0;        // error word
         words[5] = 0;        // work counters
         words[6] = 0;
+        words[7] = 0;        // the error word as this call found it
     }
     for (uint32_t t = threadIdx.x; t < (uint32_t)GK_CRC_NT; t += blockDim.x)
         tc[t] = dev_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);
@@ -1657,6 +1765,7 @@ __global__ void noalloc_setup_kernel(unsigned char *scratch, JobDev job, GeomDev
     for (uint32_t p = threadIdx.x; p < job.n_pages; p += blockDim.x) {
         page_job[p] = 0;
         page_cnt[p] = 0u;
+        page_acc[p] = 0ull;
     }
 }
 
@@ -1748,7 +1857,7 @@ int gk_page_checksums_noalloc(const gk_geom *geom, const void *blob_dev, uint32_
     w.page_begin = 0;
     w.total_pages = (uint32_t)pages;
     w.page_job = reinterpret_cast<int32_t *>(sc + NoallocLayout::page_job);
-    w.seg_res = reinterpret_cast<uint64_t *>(sc + NoallocLayout::seg_res);
+    w.page_acc = reinterpret_cast<uint64_t *>(sc + NoallocLayout::page_acc);
     w.bad_range = words + 0;
     w.bad_dup = words + 1;
     w.bad_crc = words + 2;

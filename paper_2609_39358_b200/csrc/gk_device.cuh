@@ -10,6 +10,7 @@ namespace gk {
 // CRC-64/XZ generator polynomial without its x^64 term (bit k = coefficient of x^k).
 constexpr uint64_t kPoly = 0x42F0E1EBA9EA3693ull;
 constexpr int32_t kNoPage = 0x7fffffff;
+constexpr uint32_t kUndecided = 0xffffffffu;  // job_latch: the job's commit decision has not been taken yet
 
 // bounded device waits: by default give up after this many nanoseconds of %globaltimer
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -52,15 +53,17 @@ struct WorkDev {
     uint32_t page_begin;          // first page (of the call) this launch covers
     uint32_t total_pages;         // pages this launch covers
     int32_t *page_job;            // [total_pages] owning job of each page of the call
-    uint64_t *seg_res;            // [total_pages * nseg_max] segment remainders
+    uint64_t *page_acc;           // [total_pages] XOR of the placed segment remainders of each page
     int32_t *bad_range;           // [n_jobs] lowest out-of-range table index, or kNoPage
     int32_t *bad_dup;             // [n_jobs] lowest index of a page claimed twice, or kNoPage
     int32_t *bad_crc;             // [n_jobs] lowest page whose checksum differs, or kNoPage
     uint32_t *page_cnt;           // [total_pages] segments delivered per page (fused restore)
     uint32_t *job_done;           // [n_jobs] pages finalized per job (fused restore)
+    uint32_t *job_latch;          // [n_jobs] commit decision of the job, taken once: kUndecided or a result code
     unsigned long long *claims;   // [num_pages] first claimant of each destination page
     const uint8_t *ext_mask;      // [n_jobs] or null: codes decided outside this call (gk_commit)
-    uint32_t *work_ctr;           // [2] running work-item counters: CRC modes, commit mode
+    uint32_t *work_ctr;           // [2] running work-item counters: CRC modes, commit mode; [2] = the
+                                  // error word as the call's first kernel found it
     uint32_t *error;              // sticky: non-zero once a bounded wait has run out
     const uint64_t *init_term;    // [page_tokens+1] ones * x^(8*len(t)) mod P
     const uint64_t *thread_const; // [NT] x^(32*(NT-1-t)+64) mod P
@@ -74,8 +77,8 @@ struct WorkDev {
 // change a remainder), cut into tiles of stage_bytes and grouped into segments
 // of seg_tiles tiles; the short segment, if any, is the first one.
 struct Tiling {
-    uint32_t stage_bytes;
-    uint32_t gran_bytes;
+    uint32_t stage_bytes;  // a power of two
+    uint32_t gran_bytes;   // a power of two, a multiple of stage_bytes
     uint32_t seg_tiles;
     uint32_t nseg_max;   // segments of a full page
 };
@@ -95,9 +98,10 @@ __device__ __forceinline__ PageShape page_shape(const GeomDev &g, const JobDev &
     PageShape s;
     s.t = (p + 1u < jb.n_pages) ? g.page_tokens : jb.n_tokens - (jb.n_pages - 1u) * g.page_tokens;
     s.len = (uint64_t)g.S + (uint64_t)s.t * g.tokB;
-    uint64_t v = (s.len + tl.gran_bytes - 1) / tl.gran_bytes * tl.gran_bytes;
+    // gran_bytes and stage_bytes are powers of two: masks and shifts, no 64-bit division
+    const uint64_t v = (s.len + tl.gran_bytes - 1) & ~(uint64_t)(tl.gran_bytes - 1u);
     s.pad = (uint32_t)(v - s.len);
-    s.ntiles = (uint32_t)(v / tl.stage_bytes);
+    s.ntiles = (uint32_t)(v >> (31 - __clz((int)tl.stage_bytes)));
     s.nseg = (s.ntiles + tl.seg_tiles - 1u) / tl.seg_tiles;
     s.ntiles0 = s.ntiles - (s.nseg - 1u) * tl.seg_tiles;
     return s;
@@ -165,17 +169,30 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
 // when another thread of the CTA has already given up) it records the failure in
 // *abort_flag (shared) and *error (global) and returns false.  Callers carry on
 // without blocking and without issuing further async copies; the host and the
-// commit kernel treat a set error word as "commit nothing".
+// commit kernel treat a set error word as "commit nothing".  `beat` (may be
+// null) is a shared counter that the role this wait depends on bumps while it is
+// itself inside a bounded wait of its own: as long as it moves, the clock here
+// starts afresh, so that only a partner that has gone silent counts as a failure.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t *abort_flag,
-                                          uint32_t *error, uint32_t where, unsigned long long limit_ns)
+                                          uint32_t *error, uint32_t where, unsigned long long limit_ns,
+                                          const volatile uint32_t *beat = nullptr)
 {
     if (mbar_try_wait(bar, parity)) return true;
     if (*abort_flag) return false;
-    const unsigned long long t0 = global_timer_ns();
+    unsigned long long t0 = global_timer_ns();
+    uint32_t last_beat = beat ? *beat : 0u;
     uint32_t spins = 0;
     while (!mbar_try_wait(bar, parity)) {
         if ((++spins & 0x3ffu) == 0u) {
-            if (*abort_flag || global_timer_ns() - t0 > limit_ns) {
+            const unsigned long long now = global_timer_ns();
+            if (beat) {
+                const uint32_t b = *beat;
+                if (b != last_beat) {
+                    last_beat = b;
+                    t0 = now;
+                }
+            }
+            if (*abort_flag || now - t0 > limit_ns) {
                 *abort_flag = 1u;
                 atomicCAS(error, 0u, where);
                 return false;

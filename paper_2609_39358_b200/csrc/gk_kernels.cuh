@@ -12,7 +12,7 @@
 //                                 its own pages have received the unverified bytes)
 //   restore_kernel<>  verify and commit pipelines side by side in one CTA; a job is
 //                     committed only after all of its pages have verified
-//   finalize_kernel   segment remainders -> page CRC-64/XZ; compare or write
+//   finalize_kernel   page accumulators -> page CRC-64/XZ; compare or write
 //   report_kernel     result codes of a verify-only call
 //
 // Every role of a streaming CTA is one of: loader warp (draws work items from a
@@ -70,6 +70,7 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims,
         // every call draws its work items from zero (the host counts the draws of its launches)
         w.work_ctr[0] = 0u;
         w.work_ctr[1] = 0u;
+        w.work_ctr[2] = *w.error;  // what earlier calls left: a set word refuses every commit of this call
     }
     if (clear_claims) {
         for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < num_pages;
@@ -85,6 +86,7 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims,
     for (uint32_t p = threadIdx.x; p < jb.n_pages; p += blockDim.x) {
         w.page_job[jb.page_base + p] = (int32_t)j;
         w.page_cnt[jb.page_base + p] = 0u;
+        w.page_acc[jb.page_base + p] = 0ull;
         if (jb.page_table) {
             const int32_t id = jb.page_table[p];
             if ((id < 0 || (uint64_t)id >= num_pages) && (int32_t)p < bad) bad = (int32_t)p;
@@ -98,6 +100,7 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims,
         w.bad_dup[j] = kNoPage;
         w.bad_crc[j] = kNoPage;
         w.job_done[j] = 0u;
+        w.job_latch[j] = kUndecided;
     }
 }
 
@@ -149,11 +152,13 @@ __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant_
         w.bad_dup[j] = kNoPage;
         w.bad_crc[j] = kNoPage;
         w.job_done[j] = 0u;
+        w.job_latch[j] = kUndecided;
     }
     for (uint32_t k = threadIdx.x; k < pp.n_seg_pow; k += blockDim.x) pow_out[k] = pp.seg_pow[k];
     if (threadIdx.x == 0) {
         w.work_ctr[0] = 0u;  // every call draws its work items from zero
         w.work_ctr[1] = 0u;
+        w.work_ctr[2] = *w.error;  // what earlier calls left: a set word refuses every commit of this call
     }
     __syncthreads();
     // Both passes run over the pages of the whole call at once (a thread finds the job of its
@@ -174,6 +179,7 @@ __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant_
         const uint32_t p = gp - jb.page_base;
         w.page_job[gp] = (int32_t)j;
         w.page_cnt[gp] = 0u;
+        w.page_acc[gp] = 0ull;
         if (jb.page_table) {
             const int32_t id = jb.page_table[p];
             if (id < 0 || (uint64_t)id >= pp.num_pages)
@@ -205,8 +211,15 @@ __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant_
     }
 }
 
-// Result code of a job from the words the earlier kernels left.
-__device__ __forceinline__ uint32_t job_code(const WorkDev &w, uint32_t j, int32_t *first_bad)
+// Result code of a job from the words the earlier kernels left.  Precedence:
+// missing (3) > page table (2) > checksum (1) > a wait ran out (4) > ok (0).
+// `verified` says that every page of the job is known to have been checked: in
+// the fused kernel the caller has seen the job's page count in job_done (so a
+// wait that ran out elsewhere in the same launch does not taint this job, only
+// an error word that was already set when the call began does); in the kernels
+// that run after a separate verify launch the live error word speaks for it.
+__device__ __forceinline__ uint32_t job_code(const WorkDev &w, uint32_t j, int32_t *first_bad, bool fused,
+                                             bool verified)
 {
     *first_bad = -1;
     if (w.jobs[j].missing) return 3u;
@@ -222,7 +235,8 @@ __device__ __forceinline__ uint32_t job_code(const WorkDev &w, uint32_t j, int32
         *first_bad = r;
         return 1u;
     }
-    if (__ldcg(w.error) != 0u) return 4u;
+    if (!verified) return 4u;
+    if (__ldcg(fused ? &w.work_ctr[2] : w.error) != 0u) return 4u;
     if (w.ext_mask) return (uint32_t)w.ext_mask[j];  // verified elsewhere (another call, another rank)
     return 0u;
 }
@@ -233,16 +247,16 @@ __global__ void report_kernel(WorkDev w, uint8_t *mask_out, int32_t *first_bad_o
     const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= w.n_jobs) return;
     int32_t fb;
-    const uint32_t code = job_code(w, j, &fb);
+    const uint32_t code = job_code(w, j, &fb, false, true);
     mask_out[j] = (uint8_t)code;
     first_bad_out[j] = fb;
 }
 
-// One thread per page.  Merges the page's segment remainders (each was already
-// multiplied by x^(8 * bytes that follow the segment) by the CTA that produced
-// it, so the merge is an XOR), adds the term of the all-ones initial register
-// and the final xor, reflects, and either writes the checksum (write_mode) or
-// compares it with the stored one.
+// One thread per page.  The page's segment remainders have been XORed into
+// page_acc by the CTAs that produced them (each already multiplied by
+// x^(8 * bytes that follow the segment)); this adds the term of the all-ones
+// initial register and the final xor, reflects, and either writes the checksum
+// (write_mode) or compares it with the stored one.
 __global__ void finalize_kernel(GeomDev g, WorkDev w, Tiling tl, int write_mode, uint8_t *status_out)
 {
     const uint32_t idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -255,11 +269,10 @@ __global__ void finalize_kernel(GeomDev g, WorkDev w, Tiling tl, int write_mode,
     if (write_mode && p == 0u && status_out) status_out[j] = bad_table ? 2u : 0u;
     if (jb.missing || bad_table) return;
     if (!write_mode && w.bad_dup[j] != kNoPage) return;
+    // after a wait that ran out some segments never arrived: write nothing that looks like a checksum
+    if (*w.error != 0u) return;
     const PageShape sh = page_shape(g, jb, p, tl);
-    const uint64_t *res = w.seg_res + (uint64_t)gp * tl.nseg_max;
-    uint64_t r = res[0];
-    for (uint32_t q = 1; q < sh.nseg; ++q) r ^= res[q];  // already placed by their producers
-    const uint64_t crc = __brevll(r ^ w.init_term[sh.t] ^ ~0ull);
+    const uint64_t crc = __brevll(w.page_acc[gp] ^ w.init_term[sh.t] ^ ~0ull);
     if (write_mode) {
         jb.checksums[p] = crc;
     } else if (crc != jb.checksums[p]) {
@@ -270,6 +283,20 @@ __global__ void finalize_kernel(GeomDev g, WorkDev w, Tiling tl, int write_mode,
 // ---------------------------------------------------------------------------
 // the streaming kernels
 // ---------------------------------------------------------------------------
+// What the roles of a CTA need to know about a work item.  The loader works it
+// out once and leaves it in shared memory; the other roles read it from there.
+struct Item {
+    uint8_t *rec;    // first byte of the page record in the job's blob
+    uint64_t *sum;   // the record's checksum word
+    uint32_t j, p, q;
+    uint32_t gp;     // page index within the call
+    uint32_t pad;
+    uint32_t tile_begin, tile_count;
+    uint32_t t;
+    uint32_t nseg;
+    int32_t phys;
+};
+
 template <int MODE, int NT, int STAGE_BYTES, int STAGES>
 struct StreamCfg {
     static constexpr bool kCrc = (MODE != kCommit);
@@ -281,7 +308,9 @@ struct StreamCfg {
     static constexpr int kGran = kCrc ? NT * 256 : STAGE_BYTES;  // 8 shift-register steps of 8 words per thread
     static constexpr int kSps = kCrc ? STAGE_BYTES / (NT * 32) : 1;  // 8-word steps per stage
     static constexpr int kTilesPerGran = kGran / STAGE_BYTES;
-    static constexpr size_t kSmemBytes = (size_t)STAGES * STAGE_BYTES + 3 * STAGES * 8 + 2 * 8 * 8 + 16 + 128;
+    // stages | full and empty barriers | tags | item slots | reduction slots [2][8] | abort flag | alignment slack
+    static constexpr size_t kSmemBytes =
+        (size_t)STAGES * STAGE_BYTES + 3 * STAGES * 8 + (STAGES + 1) * sizeof(Item) + 2 * 8 * 8 + 16 + 128;
     static_assert(!kCrc || (NT == 32 || NT == 64 || NT == 128 || NT == 256), "NT must be a power of two");
     static_assert(!kCrc || (STAGE_BYTES % (NT * 32) == 0 && (NT * 256) % STAGE_BYTES == 0), "stage/step mismatch");
     static_assert(STAGE_BYTES % 128 == 0, "stage alignment");
@@ -298,27 +327,22 @@ struct StreamParams {
     uint32_t fused;      // 1: verify and commit run in one launch; commit waits per job
     uint32_t inline_final;  // 1: the CTA that delivers a page's last segment finalizes the page itself
     uint32_t ctr_base_v, ctr_base_c;  // values of the work counters at the start of this launch
+    uint32_t commit_reverse;  // 1: the commit side walks the pages of a job from the last to the first
+    uint32_t l2_hints;        // bit 0: verify loads evict_last; bit 1: commit loads evict_first
+    uint32_t test_drop_from;  // tests only: k > 0 makes the fused kernel verify nothing of jobs k-1, k, ...
     uint8_t *mask_out;        // commit
     int32_t *first_bad_out;   // commit
 };
 
-struct Item {
-    const JobDev *jb;
-    uint32_t j, p, q;
-    uint32_t gp;   // page index within the call
-    uint32_t pad;
-    uint32_t tile_begin, tile_count;
-    int32_t phys;
-    uint32_t t;
-    uint32_t nseg;
-};
-
 // A shared-memory ring of STAGES tiles with a full and an empty barrier each.
+// An item's description lives in one of STAGES + 1 slots: the loader is never
+// more than STAGES items ahead of a role that still reads the slot of its item.
 struct Ring {
     uint8_t *base;    // generic address of stage 0
     uint32_t stage0;  // shared-window address of stage 0
     uint32_t full0, empty0;
-    uint2 *tag;  // per stage: (work item, tile index within the item), or the end mark
+    uint2 *tag;   // per stage: (item slot, tile index within the item), or the end mark
+    Item *items;  // [STAGES + 1]
 };
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
@@ -326,6 +350,33 @@ __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
     return v;
+}
+
+__device__ __forceinline__ uint64_t ld_acquire_u64(const uint64_t *p)
+{
+    uint64_t v;
+    asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+    return v;
+}
+
+__device__ __forceinline__ void red_xor_u64(uint64_t *p, uint64_t v)
+{
+    asm volatile("red.relaxed.gpu.global.xor.b64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
+// Counts one arrival; everything this thread wrote before (the red.xor above it)
+// is visible to whoever sees the count, and the returned count lets the last
+// arriver see what the others wrote.
+__device__ __forceinline__ uint32_t atom_add_acq_rel_u32(uint32_t *p, uint32_t v)
+{
+    uint32_t old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+    return old;
+}
+
+__device__ __forceinline__ void fence_sc_gpu()
+{
+    asm volatile("fence.sc.gpu;" ::: "memory");
 }
 
 // Fused restore: a job may be committed only after all of its pages have been
@@ -341,11 +392,12 @@ __device__ __forceinline__ bool wait_job_verified(const StreamParams &P, uint32_
     if (*abort_flag) return false;
     const unsigned long long t0 = global_timer_ns();
     uint32_t spins = 0;
+    volatile uint32_t *beat = abort_flag + 1;  // tells the storer behind this loader that it is alive
     while (ld_acquire_u32(cnt) < n_pages) {
-        __nanosleep(200);
+        __nanosleep(100);
         if ((++spins & 0x3fu) == 0u) {
+            *beat = *beat + 1u;
             if (*abort_flag || global_timer_ns() - t0 > P.w.wait_limit_ns) {
-                *abort_flag = 1u;
                 atomicCAS(P.w.error, 0u, 0x500u);
                 return false;
             }
@@ -354,40 +406,106 @@ __device__ __forceinline__ bool wait_job_verified(const StreamParams &P, uint32_
     return true;
 }
 
+// The commit decision of a job is taken ONCE, by whichever commit loader meets
+// the job first: it waits (fused kernel) until the job has been verified, works
+// out the result code, and publishes it in job_latch[j] with a compare-and-swap;
+// the winner also writes the job's report.  Every other commit item of the job,
+// in any CTA, reads the latched code, so a job is committed whole or not at all
+// even if a wait runs out somewhere else in the meantime.  Lane 0 decides, the
+// warp gets the code.
+__device__ __forceinline__ uint32_t commit_decision(const StreamParams &P, uint32_t j, const JobDev &jb,
+                                                    volatile uint32_t *abort_flag, int lane)
+{
+    uint32_t code = 0u;
+    if (lane == 0) {
+        code = ld_acquire_u32(P.w.job_latch + j);
+        if (code == kUndecided) {
+            bool verified = true;
+            if (P.fused && !jb.missing && P.w.bad_range[j] == kNoPage && P.w.bad_dup[j] == kNoPage)
+                verified = wait_job_verified(P, j, jb.n_pages, abort_flag);
+            int32_t fb;
+            code = job_code(P.w, j, &fb, P.fused != 0u, verified);
+            const uint32_t old = atomicCAS(P.w.job_latch + j, kUndecided, code);
+            if (old != kUndecided) {
+                code = old;
+            } else if (P.mask_out) {
+                P.mask_out[j] = (uint8_t)code;
+                P.first_bad_out[j] = fb;
+                // a CTA that had to give up on one of this job's items may have changed the verdict meanwhile
+                fence_sc_gpu();
+                if (ld_acquire_u32(P.w.job_latch + j) != code) P.mask_out[j] = 4u;
+            }
+        }
+    }
+    return __shfl_sync(0xffffffffu, code, 0);
+}
+
+// A CTA that has given up (one of its own bounded waits ran out) can no longer
+// write the items it draws.  If such an item belongs to a job that was accepted,
+// the job ends up partly written: its verdict becomes "a wait ran out" (4), for
+// the report and for every commit item of the job that has not started yet.
+__device__ __forceinline__ void revoke_job(const StreamParams &P, uint32_t j)
+{
+    atomicExch(P.w.job_latch + j, 4u);
+    fence_sc_gpu();
+    if (P.mask_out) P.mask_out[j] = 4u;
+}
+
+// Geometry of work item `item` of a launch (no decision is taken here).
+// Returns false if the item does not exist (a short last page has fewer segments).
 template <int MODE>
-__device__ __forceinline__ bool get_item(const StreamParams &P, const Tiling &tl, uint32_t item, Item &it, bool report,
-                                         volatile uint32_t *abort_flag)
+__device__ __forceinline__ bool item_geometry(const StreamParams &P, const Tiling &tl, uint32_t item,
+                                              const JobDev *&jbp, Item &it)
 {
     const uint32_t local = item / tl.nseg_max;
-    it.q = item - local * tl.nseg_max;
-    const uint32_t gp = P.w.page_begin + local;
-    it.gp = gp;
+    uint32_t q = item - local * tl.nseg_max;
+    uint32_t gp = P.w.page_begin + local;
     it.j = (uint32_t)P.w.page_job[gp];
-    it.jb = &P.w.jobs[it.j];
-    const JobDev jb = *it.jb;
+    jbp = &P.w.jobs[it.j];
+    const JobDev jb = *jbp;
     it.p = gp - jb.page_base;
-    if (MODE == kCommit) {
-        if (P.fused && !jb.missing && P.w.bad_range[it.j] == kNoPage && P.w.bad_dup[it.j] == kNoPage)
-            wait_job_verified(P, it.j, jb.n_pages, abort_flag);
-        int32_t fb;
-        const uint32_t code = job_code(P.w, it.j, &fb);
-        if (report && it.p == 0u && it.q == 0u && P.mask_out) {
-            P.mask_out[it.j] = (uint8_t)code;
-            P.first_bad_out[it.j] = fb;
-        }
-        if (code != 0u) return false;
-    } else {
-        if (jb.missing || P.w.bad_range[it.j] != kNoPage) return false;
-        if ((MODE == kVerify || MODE == kSingle) && P.w.bad_dup[it.j] != kNoPage) return false;
+    if (MODE == kCommit && P.commit_reverse) {
+        // same items, walked from the end of the job: what was verified last is read back first
+        it.p = jb.n_pages - 1u - it.p;
+        gp = jb.page_base + it.p;
     }
+    it.gp = gp;
     const PageShape sh = page_shape(P.g, jb, it.p, tl);
     it.nseg = sh.nseg;
-    if (it.q >= sh.nseg) return false;
+    if (q >= sh.nseg) return false;
+    if (MODE == kCommit && P.commit_reverse) q = sh.nseg - 1u - q;
+    it.q = q;
     it.pad = sh.pad;
     it.t = sh.t;
-    it.tile_begin = it.q == 0u ? 0u : sh.ntiles0 + (it.q - 1u) * tl.seg_tiles;
-    it.tile_count = it.q == 0u ? sh.ntiles0 : tl.seg_tiles;
-    it.phys = (MODE != kVerify) ? jb.page_table[it.p] : 0;
+    it.tile_begin = q == 0u ? 0u : sh.ntiles0 + (q - 1u) * tl.seg_tiles;
+    it.tile_count = q == 0u ? sh.ntiles0 : tl.seg_tiles;
+    it.rec = jb.blob + (uint64_t)it.p * P.g.R;
+    it.sum = jb.checksums + it.p;
+    it.phys = 0;
+    return true;
+}
+
+// Loader only: geometry plus the decision whether the item is to be processed.
+template <int MODE>
+__device__ __forceinline__ bool admit_item(const StreamParams &P, const Tiling &tl, uint32_t item, Item &it,
+                                           volatile uint32_t *abort_flag, int lane)
+{
+    const JobDev *jbp;
+    const bool exists = item_geometry<MODE>(P, tl, item, jbp, it);
+    if (MODE == kCommit) {
+        // every item asks, existing or not, so that a job whose pages all fail to exist cannot occur
+        const uint32_t code = commit_decision(P, it.j, *jbp, abort_flag, lane);
+        if (code != 0u || !exists) return false;
+        if (*abort_flag) {
+            if (lane == 0) revoke_job(P, it.j);
+            return false;
+        }
+    } else {
+        if (!exists || jbp->missing || P.w.bad_range[it.j] != kNoPage) return false;
+        if ((MODE == kVerify || MODE == kSingle) && P.w.bad_dup[it.j] != kNoPage) return false;
+        if (MODE == kVerify && P.test_drop_from != 0u && it.j + 1u >= P.test_drop_from) return false;
+    }
+    if (MODE != kVerify) it.phys = jbp->page_table[it.p];
     return true;
 }
 
@@ -615,42 +733,62 @@ struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES> {
 
 // Work is handed out dynamically: the loader warp of a CTA draws item numbers
 // from a global counter (so the CTAs that are resident take all the work, in
-// order, whatever their number) and tags every stage it fills with the item and
-// the tile index; the other roles of the CTA follow the tags.  A stage tagged
-// kEndOfWork tells them to leave.
+// order, whatever their number), and tags every stage it fills with the item's
+// slot and the tile index; the other roles of the CTA follow the tags.  A stage
+// tagged kEndOfWork tells them to leave.  Where no CTA ever waits for another
+// one's item (everything but the verify side of the fused kernel) a CTA takes
+// the item with its own number first, without asking the counter.
 constexpr uint32_t kEndOfWork = 0xffffffffu;
+constexpr uint32_t kNoJob = 0xffffffffu;
 
+template <bool STATIC_FIRST>
 __device__ __forceinline__ uint32_t next_item(uint32_t *ctr, uint32_t base, int lane)
 {
     uint32_t v = 0;
-    if (lane == 0) v = atomicAdd(ctr, 1u) - base;
+    if (lane == 0) v = atomicAdd(ctr, 1u) - base + (STATIC_FIRST ? gridDim.x : 0u);
     return __shfl_sync(0xffffffffu, v, 0);
 }
 
+// Commit modes, after this CTA has given up: every job that may still have a tile
+// of this CTA in flight loses its "accepted" verdict (see revoke_job).
+template <int STAGES>
+__device__ __forceinline__ void revoke_in_flight(const StreamParams &P, const Ring &ring)
+{
+    for (int k = 0; k <= STAGES; ++k) {
+        const uint32_t j = ring.items[k].j;
+        if (j != kNoJob) revoke_job(P, j);
+    }
+}
+
 // ------------------------------ loader role ------------------------------
-// One warp.  Draws work items, walks each tile by tile, waits for a free stage
-// and fills it: front padding zeroed by the lanes (CRC modes), scale values
-// gathered by the lanes (pack), everything else by bulk async copies issued by
-// lane 0 that complete on the stage's full barrier.  In commit mode it also
-// writes the job's result code when it meets the job's first item.
-template <int MODE, int STAGE_BYTES, int STAGES, bool ZERO_PAD>
+// One warp.  Draws work items, decides whether each is to be processed, walks it
+// tile by tile, waits for a free stage and fills it: front padding zeroed by the
+// lanes (CRC modes), scale values gathered by the lanes (pack), everything else
+// by bulk async copies issued by lane 0 that complete on the stage's full barrier.
+template <int MODE, int STAGE_BYTES, int STAGES, bool ZERO_PAD, bool STATIC_FIRST>
 __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling &tl, uint32_t n_items, uint32_t *ctr,
                                             uint32_t ctr_base, const Ring &ring, volatile uint32_t *abort_flag,
                                             int lane)
 {
-    uint32_t n = 0;
-    for (;;) {
-        const uint32_t item = next_item(ctr, ctr_base, lane);
-        if (item >= n_items) break;
+    uint32_t n = 0;       // tiles issued
+    uint32_t n_adm = 0;   // items admitted
+    bool revoked = false;
+    uint64_t policy = 0;
+    const bool hint = (MODE == kVerify && (P.l2_hints & 1u)) || (MODE == kCommit && (P.l2_hints & 2u));
+    if (hint) policy = (MODE == kVerify) ? policy_evict_last() : policy_evict_first();
+    for (uint32_t item = STATIC_FIRST ? blockIdx.x : next_item<false>(ctr, ctr_base, lane); item < n_items;
+         item = next_item<STATIC_FIRST>(ctr, ctr_base, lane)) {
         Item it;
-        if (!get_item<MODE>(P, tl, item, it, lane == 0, abort_flag)) continue;
-        const uint8_t *rec = (MODE == kPack) ? nullptr : it.jb->blob + (uint64_t)it.p * P.g.R;
+        if (!admit_item<MODE>(P, tl, item, it, abort_flag, lane)) continue;
+        const uint32_t slot = n_adm % (uint32_t)(STAGES + 1);
+        ++n_adm;
         const Chunks ch = chunks_of(P.g, it.t);
         for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
             const uint32_t s = n % STAGES;
             const uint32_t use = n / STAGES;
             if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE,
                                     P.w.wait_limit_ns);
+            if (k == 0u && lane == 0) ring.items[slot] = it;  // the stage's barrier publishes it with the tile
             uint32_t lead, nreal;
             uint64_t r0;
             tile_range<STAGE_BYTES>(it.tile_begin + k, it.pad, lead, r0, nreal);
@@ -684,8 +822,13 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
             }
             __syncwarp();
             if (lane == 0) {
-                ring.tag[s] = make_uint2(item, k);
-                if (!*abort_flag) {
+                ring.tag[s] = make_uint2(slot, k);
+                if (*abort_flag) {
+                    if (MODE == kCommit && !revoked) {
+                        revoke_in_flight<STAGES>(P, ring);
+                        revoked = true;
+                    }
+                } else {
                     const uint32_t bar = ring.full0 + 8u * s;
                     if (MODE == kPack) {
                         const uint32_t data_bytes = nreal - scale_bytes;
@@ -701,6 +844,7 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                             while (d0 < d1) {
                                 uint32_t nb = ch.len - off;
                                 if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
+                                if (nb == 0u) break;  // cannot happen with a valid geometry; never spin
                                 bulk_g2s(so, chunk_addr(P.cache, ch, chunk, it.phys, off), nb, bar);
                                 d0 += nb;
                                 so += nb;
@@ -713,7 +857,8 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                             mbar_arrive(bar);
                         } else {
                             mbar_arrive_expect_tx(bar, nreal);
-                            bulk_g2s(sbase + lead, rec + r0, nreal, bar);
+                            if (hint) bulk_g2s_hint(sbase + lead, it.rec + r0, nreal, bar, policy);
+                            else bulk_g2s(sbase + lead, it.rec + r0, nreal, bar);
                         }
                     }
                 }
@@ -743,55 +888,60 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
 }
 
 // ------------------------------ storer role ------------------------------
-// One warp.  Waits for each tile to land, reads its tag, and writes it out with
-// bulk async copies: one contiguous piece into the blob (pack), or one piece per
-// slab into the destination cache plus the scale values by the lanes (commit).
-// A stage goes back to the loader once the copy of the following tile has been
-// issued and the stage's own copy has finished reading shared memory.
+// One warp.  Waits for each tile to land, reads its tag and its item's slot, and
+// writes it out with bulk async copies: one contiguous piece into the blob
+// (pack), or one piece per slab into the destination cache plus the scale values
+// by the lanes (commit).  A stage goes back to the loader once the copy of the
+// following tile has been issued and the stage's own copy has finished reading
+// shared memory.  The storer takes no decision of its own: a tile that the
+// loader put into the ring is a tile to be written.
 template <int MODE, int STAGE_BYTES, int STAGES>
-__device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling &tl, const Ring &ring,
-                                            volatile uint32_t *abort_flag, int lane)
+__device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &ring, volatile uint32_t *abort_flag,
+                                            int lane)
 {
     uint32_t n = 0;
-    uint32_t cur_item = kEndOfWork;
-    Item it{};
-    uint8_t *rec = nullptr;
-    Chunks ch{};
+    bool revoked = false;
     for (;; ++n) {
         const uint32_t s = n % STAGES;
+        // the loader ahead of a commit storer may itself be waiting, job after job, for verification
         bool ok = mbar_wait(ring.full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | MODE,
-                            P.w.wait_limit_ns);
+                            P.w.wait_limit_ns, MODE == kCommit ? abort_flag + 1 : nullptr);
         ok = __all_sync(0xffffffffu, ok);
-        if (!ok) break;  // the CTA has given up: nothing more is stored (decided by the whole warp)
+        if (!ok) {  // the CTA has given up: nothing more is stored (decided by the whole warp)
+            if (MODE == kCommit && lane == 0 && !revoked) revoke_in_flight<STAGES>(P, ring);
+            break;
+        }
         const uint2 tag = ring.tag[s];
         if (tag.x == kEndOfWork) break;
-        if (tag.x != cur_item) {
-            cur_item = tag.x;
-            get_item<MODE>(P, tl, cur_item, it, false, abort_flag);
-            rec = it.jb->blob + (uint64_t)it.p * P.g.R;
-            ch = chunks_of(P.g, it.t);
-        }
+        const Item &it = ring.items[tag.x];
+        const int32_t phys = it.phys;
+        const Chunks ch = chunks_of(P.g, it.t);
         uint32_t lead, nreal;
         uint64_t r0;
         tile_range<STAGE_BYTES>(it.tile_begin + tag.y, it.pad, lead, r0, nreal);
         const uint32_t sbase = ring.stage0 + s * STAGE_BYTES;
         const uint8_t *sgen = ring.base + (size_t)s * STAGE_BYTES;
+        const bool aborted = *abort_flag != 0u;
+        if (aborted && MODE == kCommit && lane == 0 && !revoked) {
+            revoke_in_flight<STAGES>(P, ring);
+            revoked = true;
+        }
         uint32_t scale_bytes = 0u;
         if ((MODE == kCommit || MODE == kSingle) && r0 < P.g.S && nreal > 0u) {
             const uint64_t e1 = (r0 + nreal < P.g.S) ? r0 + nreal : P.g.S;
             scale_bytes = (uint32_t)(e1 - r0);
-            if (!*abort_flag) {
+            if (!aborted) {
                 for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
                     const uint32_t v = *reinterpret_cast<const uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0));
-                    *reinterpret_cast<uint32_t *>(scale_addr(P.g, P.cache, i, it.phys)) = v;
+                    *reinterpret_cast<uint32_t *>(scale_addr(P.g, P.cache, i, phys)) = v;
                 }
             }
         }
         __syncwarp();
         if (lane == 0) {
-            if (!*abort_flag && nreal > 0u) {
+            if (!aborted && nreal > 0u) {
                 if (MODE == kPack) {
-                    bulk_s2g(rec + r0, sbase + lead, nreal);
+                    bulk_s2g(it.rec + r0, sbase + lead, nreal);
                 } else {
                     const uint32_t data_bytes = nreal - scale_bytes;
                     uint64_t d0 = r0 + scale_bytes - P.g.S;
@@ -802,7 +952,8 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling 
                     while (d0 < d1) {
                         uint32_t nb = ch.len - off;
                         if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
-                        bulk_s2g(chunk_addr(P.cache, ch, chunk, it.phys, off), so, nb);
+                        if (nb == 0u) break;  // cannot happen with a valid geometry; never spin
+                        bulk_s2g(chunk_addr(P.cache, ch, chunk, phys, off), so, nb);
                         d0 += nb;
                         so += nb;
                         ++chunk;
@@ -825,10 +976,12 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Tiling 
 }
 
 // ----------------------------- consumer role -----------------------------
-// NT threads.  Reduce each segment to its remainder (see the top of this file)
-// and leave it in seg_res.  In the fused restore kernel the CTA that delivers
-// the last segment of a page also finalizes the page -- merge, compare with the
-// stored checksum -- and counts it in job_done, which the commit side waits on.
+// NT threads.  Reduce each segment to its remainder (see the top of this file),
+// place it inside its page and XOR it into the page's accumulator.  Where pages
+// are finalized inline, the CTA that delivers the last segment of a page also
+// finishes it -- final xor, reflection, then write the checksum (pack) or compare
+// it with the stored one and count the page in job_done, which the commit side
+// of the fused kernel waits on.
 template <int MODE, int NT, int STAGE_BYTES, int STAGES>
 __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring &ring, uint64_t *red,
                                               volatile uint32_t *abort_flag, int tid, int warp, int lane)
@@ -852,14 +1005,12 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
             : "r"(ok ? 0u : 1u), "n"(NT)
             : "memory");
         if (any_failed) break;
-        const uint32_t item = ring.tag[pos.stage].x;
-        if (item == kEndOfWork) break;
-        Item it;
-        get_item<MODE>(P, P.tl, item, it, false, abort_flag);
+        const uint32_t slot = ring.tag[pos.stage].x;
+        if (slot == kEndOfWork) break;
+        const uint32_t ngran = ring.items[slot].tile_count / kTilesPerGran;
         uint32_t R[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) R[i] = 0u;
-        const uint32_t ngran = it.tile_count / kTilesPerGran;
         for (uint32_t gi = 0; gi < ngran; ++gi)
             GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, ring.base, ring.full0, ring.empty0, pos, abort_flag,
                                                                 P.w.error, P.w.wait_limit_ns, tid, lane);
@@ -867,41 +1018,38 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
         uint64_t v = thread_remainder<NT>(R, kt);
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) v ^= __shfl_xor_sync(0xffffffffu, v, d);
-        uint64_t *slot = red + 8 * parity_red;
-        if (lane == 0) slot[warp] = v;
+        uint64_t *rslot = red + 8 * parity_red;
+        if (lane == 0) rslot[warp] = v;
         asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
         if (tid == 0) {
+            const Item &it = ring.items[slot];  // still this item's: see Ring
             uint64_t tot = 0;
 #pragma unroll
-            for (int i = 0; i < NT / 32; ++i) tot ^= slot[i];
+            for (int i = 0; i < NT / 32; ++i) tot ^= rslot[i];
             // place the segment: the short segment comes first and all others are full, so
             // (nseg - 1 - q) full segments follow this one
-            if (it.nseg > 1u) tot = gf_mul(tot, P.w.seg_pow[it.nseg - 1u - it.q]);
-            uint64_t *res = P.w.seg_res + (uint64_t)it.gp * P.tl.nseg_max;
+            const uint32_t nseg = it.nseg;
+            if (nseg > 1u) tot = gf_mul(tot, P.w.seg_pow[nseg - 1u - it.q]);
+            uint64_t *acc = P.w.page_acc + it.gp;
             if (!P.inline_final) {
-                res[it.q] = tot;
+                red_xor_u64(acc, tot);
             } else {
+                uint64_t stored = 0;
+                if (MODE != kPack) stored = *it.sum;  // in flight together with the two atomics below
                 uint64_t r = tot;
                 bool last = true;
-                if (it.nseg > 1u) {
-                    __stcg(&res[it.q], tot);
-                    __threadfence();
-                    last = atomicAdd(&P.w.page_cnt[it.gp], 1u) + 1u == it.nseg;
-                    if (last) {
-                        __threadfence();
-                        r = __ldcg(&res[0]);
-                        for (uint32_t q = 1; q < it.nseg; ++q) r ^= __ldcg(&res[q]);
-                    }
+                if (nseg > 1u) {
+                    red_xor_u64(acc, tot);
+                    last = atom_add_acq_rel_u32(&P.w.page_cnt[it.gp], 1u) + 1u == nseg;
+                    if (last) r = ld_acquire_u64(acc);
                 }
                 if (last) {
                     const uint64_t crc = __brevll(r ^ P.w.init_term[it.t] ^ ~0ull);
                     if (MODE == kPack) {
-                        it.jb->checksums[it.p] = crc;
+                        *it.sum = crc;
                     } else {
-                        if (crc != it.jb->checksums[it.p] || *abort_flag)
-                            atomicMin(&P.w.bad_crc[it.j], (int32_t)it.p);
-                        __threadfence();
-                        atomicAdd(&P.w.job_done[it.j], 1u);
+                        if (crc != stored || *abort_flag) atomicMin(&P.w.bad_crc[it.j], (int32_t)it.p);
+                        atom_add_acq_rel_u32(&P.w.job_done[it.j], 1u);
                     }
                 }
             }
@@ -910,11 +1058,12 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
     }
 }
 
-__device__ __forceinline__ void ring_init(Ring &ring, uint8_t *base, uint64_t *bars, uint2 *tags, int stages,
-                                          uint32_t empty_count)
+__device__ __forceinline__ void ring_init(Ring &ring, uint8_t *base, uint64_t *bars, uint2 *tags, Item *items,
+                                          int stages, uint32_t empty_count)
 {
     ring.base = base;
     ring.tag = tags;
+    ring.items = items;
     ring.stage0 = smem_u32(base);
     ring.full0 = smem_u32(bars);
     ring.empty0 = smem_u32(bars + stages);
@@ -923,6 +1072,7 @@ __device__ __forceinline__ void ring_init(Ring &ring, uint8_t *base, uint64_t *b
             mbar_init(ring.full0 + 8u * s, 1u);
             mbar_init(ring.empty0 + 8u * s, empty_count);
         }
+        for (int s = 0; s <= stages; ++s) items[s].j = kNoJob;
     }
 }
 
@@ -938,13 +1088,15 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
     uint64_t *red = bars + 2 * STAGES;  // [2][8]
     volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
     uint2 *tags = (uint2 *)(red + 18);
+    Item *items = (Item *)(tags + STAGES);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     Ring ring;
-    ring_init(ring, smem, bars, tags, STAGES, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)));
+    ring_init(ring, smem, bars, tags, items, STAGES, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)));
     if (threadIdx.x == 0) {
-        *abort_flag = 0u;
+        abort_flag[0] = 0u;
+        abort_flag[1] = 0u;  // the commit loader's sign of life while it waits for a job
         fence_mbar_init();
     }
     grid_dependency_wait();  // everything above is CTA-local; the tables of the call are read below
@@ -952,13 +1104,13 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
 
     if (warp == Cfg::kLoaderWarp) {
         if (MODE == kCommit)
-            loader_role<MODE, STAGE_BYTES, STAGES, false>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, ring,
+            loader_role<MODE, STAGE_BYTES, STAGES, false, true>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, ring,
                                                           abort_flag, lane);
         else
-            loader_role<MODE, STAGE_BYTES, STAGES, true>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, ring,
-                                                         abort_flag, lane);
+            loader_role<MODE, STAGE_BYTES, STAGES, true, true>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, ring,
+                                                               abort_flag, lane);
     } else if (Cfg::kStore && warp == Cfg::kStorerWarp) {
-        storer_role<MODE, STAGE_BYTES, STAGES>(P, MODE == kCommit ? P.tlc : P.tl, ring, abort_flag, lane);
+        storer_role<MODE, STAGE_BYTES, STAGES>(P, ring, abort_flag, lane);
     } else if constexpr (Cfg::kCrc) {
         consumer_role<MODE, NT, STAGE_BYTES, STAGES>(P, ring, red, abort_flag, threadIdx.x, warp, lane);
     }
@@ -968,13 +1120,13 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
 // Fused restore: the verify pipeline (loader warp + NT consumer threads) and the
 // commit pipeline (loader warp + storer warp) of one CTA run side by side on
 // two rings.  Verify is bound by the integer pipes, commit by DRAM, so the two
-// overlap; fail-closed order is kept per job by wait_job_verified().
+// overlap; fail-closed order is kept per job by commit_decision().
 template <int NT, int VSB, int VST, int CSB, int CST>
 struct RestoreCfg {
     static constexpr int kConsWarps = NT / 32;
     static constexpr int kThreads = NT + 96;
-    static constexpr size_t kSmemBytes =
-        (size_t)VST * VSB + (size_t)CST * CSB + 3 * (VST + CST) * 8 + 2 * 8 * 8 + 16 + 128;
+    static constexpr size_t kSmemBytes = (size_t)VST * VSB + (size_t)CST * CSB + 3 * (VST + CST) * 8 +
+                                         (VST + CST + 2) * sizeof(Item) + 2 * 8 * 8 + 16 + 128;
 };
 
 template <int NT, int VSB, int VST, int CSB, int CST, int MINB>
@@ -990,14 +1142,17 @@ __global__ void __launch_bounds__(NT + 96, MINB) restore_kernel(const __grid_con
     volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
     uint2 *vtags = (uint2 *)(red + 18);
     uint2 *ctags = vtags + VST;
+    Item *vitems = (Item *)(ctags + CST);
+    Item *citems = vitems + (VST + 1);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     Ring vring, cring;
-    ring_init(vring, vbase, vbars, vtags, VST, (uint32_t)(NT / 32));
-    ring_init(cring, cbase, cbars, ctags, CST, 1u);
+    ring_init(vring, vbase, vbars, vtags, vitems, VST, (uint32_t)(NT / 32));
+    ring_init(cring, cbase, cbars, ctags, citems, CST, 1u);
     if (threadIdx.x == 0) {
-        *abort_flag = 0u;
+        abort_flag[0] = 0u;
+        abort_flag[1] = 0u;  // the commit loader's sign of life while it waits for a job
         fence_mbar_init();
     }
     grid_dependency_wait();  // everything above is CTA-local; the tables of the call are read below
@@ -1007,12 +1162,13 @@ __global__ void __launch_bounds__(NT + 96, MINB) restore_kernel(const __grid_con
     if (warp < kCons) {
         consumer_role<kVerify, NT, VSB, VST>(P, vring, red, abort_flag, threadIdx.x, warp, lane);
     } else if (warp == kCons) {
-        loader_role<kVerify, VSB, VST, true>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, vring, abort_flag, lane);
+        loader_role<kVerify, VSB, VST, true, false>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, vring, abort_flag,
+                                                    lane);
     } else if (warp == kCons + 1) {
-        loader_role<kCommit, CSB, CST, false>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, cring, abort_flag,
-                                              lane);
+        loader_role<kCommit, CSB, CST, false, true>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, cring,
+                                                    abort_flag, lane);
     } else {
-        storer_role<kCommit, CSB, CST>(P, P.tlc, cring, abort_flag, lane);
+        storer_role<kCommit, CSB, CST>(P, cring, abort_flag, lane);
     }
     __syncthreads();
 }

@@ -87,6 +87,41 @@ def _check_sampled_records(w, src, jobs_meta, rng, n_samples):
         assert int(sums[p].item()) & 0xFFFFFFFFFFFFFFFF == crc, f"checksum {p} of job {j} differs"
 
 
+def _check_all_checksums(w, blobs, sums, lens):
+    """EVERY checksum of every block against the oracle's CRC-64 of the record bytes as the
+    GPU packed them (blobs copied to the host block by block; the oracle runs on a few
+    host threads, ctypes releases the interpreter lock)."""
+    from concurrent.futures import ThreadPoolExecutor
+    import os
+    og = oracle_geom(w)
+    with ThreadPoolExecutor(max_workers=max(1, min(16, os.cpu_count() or 1))) as pool:
+        for blob, sm, n in zip(blobs, sums, lens):
+            host = blob.cpu().numpy()
+            got = sm.cpu().numpy().view(np.uint64)
+            P = -(-n // w.page_tokens)
+            offs = [oracle.record_offset(og, p) for p in range(P)] + [host.size]
+            want = list(pool.map(lambda p: oracle.crc64(host[offs[p]:offs[p + 1]]), range(P)))
+            assert [int(x) for x in got] == want, "a checksum differs from the oracle's"
+
+
+def _check_whole_block(w, src, blob, sums, spt, n):
+    """All bytes and all checksums of one block against oracle.pack over the block's source pages."""
+    og = oracle_geom(w)
+    idx = torch.from_numpy(np.ascontiguousarray(spt).astype(np.int64)).cuda()
+    P = idx.numel()
+    pages = _view(w, src)[:, :, idx].contiguous().cpu().numpy().reshape(-1)   # [L][2][P][T][row]
+    s = _slab(w)
+    oc = oracle.Cache(pages, P, 2 * P * s, P * s, s)
+    if w.scale_kv:
+        oc.scales = _scale_view(w, src)[:, :, idx].contiguous().cpu().numpy().reshape(-1)
+        h4 = w.kv_heads * 4
+        oc.s_layer_stride, oc.s_kv_stride, oc.s_page_stride = w.scale_kv * P * h4, P * h4, h4
+    want_blob, want_sums, code, _ = oracle.pack(og, oc, np.arange(P, dtype=np.int32), n)
+    assert code == 0
+    assert np.array_equal(blob.cpu().numpy(), want_blob), "blob bytes differ from the oracle's"
+    assert np.array_equal(sums.cpu().numpy().view(np.uint64), want_sums), "checksums differ from the oracle's"
+
+
 def _check_destination(w, src, dst, sentinel, jobs, masks):
     """jobs: list of (src table np, dst table np, n_tokens).  Every committed page
     equals its source on the valid range; everything else equals the sentinel."""
@@ -145,6 +180,10 @@ def test_gqa7b_full(gk):
     assert status.cpu().tolist() == [0] * NB
     rng = np.random.default_rng(w.seed(4))
     _check_sampled_records(w, src, [(blobs[i], sums[i], spts[i], n_tok) for i in range(NB)], rng, 24)
+    # all 4,096 checksums of the batch, and every byte of two whole blocks, against the oracle
+    _check_all_checksums(w, blobs, sums, [n_tok] * NB)
+    for i in (0, NB - 1):
+        _check_whole_block(w, src, blobs[i], sums[i], spts[i], n_tok)
     mask = torch.full((NB,), 255, dtype=torch.uint8, device="cuda")
     fb = torch.zeros(NB, dtype=torch.int32, device="cuda")
     ctx.gk_restore([gk.Job(blobs[i], sums[i], d_dpts[i], n_tok, i // 2) for i in range(NB)], dst, mask, fb)
@@ -190,6 +229,10 @@ def test_corpus_full_device_and_host_tier(gk):
     meta = [(blobs[i], sums[i], spts[i], lens[i]) for i in range(NB)]
     _check_sampled_records(w, src, meta, rng, 16)
     _check_sampled_records(w, src, meta[-1:], rng, 6)          # the tail block, its partial page included
+    # the 280-token tail block whole (its 8-token last page included) and one full block, byte for byte
+    _check_whole_block(w, src, blobs[-1], sums[-1], spts[-1], lens[-1])
+    _check_whole_block(w, src, blobs[40], sums[40], spts[40], lens[40])
+    _check_all_checksums(w, blobs[-3:], sums[-3:], lens[-3:])
     jobs_meta = [(spts[i], dpts[i], lens[i]) for i in range(NB)]
     mask = torch.full((NB,), 255, dtype=torch.uint8, device="cuda")
     fb = torch.zeros(NB, dtype=torch.int32, device="cuda")

@@ -821,7 +821,9 @@ def test_device_wait_time_out_is_fail_closed(gk):
     """Failure detection without a GPU fault: the commit side's bounded wait for
     "all pages of the job verified" is made to run out (test hook: nothing gets
     verified, limit 50 ms).  The kernel must return by itself, report code 4 for
-    every job, write nothing, and leave the context refusing to commit."""
+    every job, write nothing, and leave the context refusing to commit until the
+    error is cleared; after gk_ctx_clear_error the SAME context restores the same
+    jobs correctly."""
     from gpu_harness import assert_cache_equal, dev_cache, dev_i32, sums_to_dev
     og = G_MID
     src = random_cache(og, 8, seed=360)
@@ -845,16 +847,251 @@ def test_device_wait_time_out_is_fail_closed(gk):
     torch.cuda.synchronize()
     assert mask.cpu().tolist() == [4, 4]
     assert_cache_equal(d, clean)
-    ctx.close()
-    # a fresh context on the same device works: nothing was left broken
-    ctx = _ctx(gk, og)
-    want = clone_cache(clean)
-    wmask, _ = oracle.restore(og, want, jobs)
+    # the unfused path (separate verify and commit launches) refuses as well
+    ctx.set_tuning("fused", 0)
     mask.fill_(255)
     ctx.gk_restore(gjobs, d, mask, fb)
     torch.cuda.synchronize()
+    assert mask.cpu().tolist() == [4, 4]
+    assert_cache_equal(d, clean)
+    ctx.set_tuning("fused", 1)
+    # cleared: the same context commits the same jobs, bit-exact
+    want = clone_cache(clean)
+    wmask, _ = oracle.restore(og, want, jobs)
+    ctx.gk_ctx_clear_error()
+    mask.fill_(255)
+    ctx.gk_restore(gjobs, d, mask, fb)
+    torch.cuda.synchronize()
+    assert ctx.gk_get_stats()["device_wait_expired"] == 0
     assert mask.cpu().tolist() == wmask.tolist() == [0, 0]
     assert_cache_equal(d, want)
+    ctx.close()
+
+
+def test_partial_time_out_commits_whole_jobs_or_nothing(gk):
+    """A wait that runs out for SOME jobs of a fused restore: the hook leaves the jobs
+    from index 3 on unverified (limit 50 ms, no fault, no hang).  The jobs before them
+    have verified and must be committed whole with code 0 -- the decision of a job is
+    taken once and does not change when another job's wait runs out later -- and the
+    others must report code 4 with not one byte written.  Several segments and commit
+    items per page, so that every job's items are spread over many CTAs."""
+    from gpu_harness import assert_cache_equal, dev_cache, dev_i32, sums_to_dev
+    og = G_BIG
+    T = og.page_tokens
+    lens = [5 * T, 2 * T + 3, 7 * T, 4 * T, 3 * T + 1, 6 * T]
+    n_pages = sum(-(-n // T) for n in lens)
+    src = random_cache(og, n_pages, seed=370)
+    jobs = _oracle_jobs(og, src, lens, 371, n_pages + 6)
+    jobs[1].blob[12345] ^= 0x40                     # a job that verified as damaged keeps its code 1
+    clean = random_cache(og, n_pages + 6, seed=372)
+    # expectation: the oracle's result for the jobs that were verified, nothing for the rest
+    want = clone_cache(clean)
+    wmask, wfb = oracle.restore(og, want, jobs[:3])
+    assert wmask.tolist() == [0, 1, 0]
+    for seg, cst in ((0, 0), (1, 2)):
+        ctx = _ctx(gk, og, wait_limit_ms=50, test_drop_verify=4, seg_granules=seg, commit_seg_tiles=cst)
+        d = dev_cache(clean)
+        keep = [(torch.from_numpy(j.blob).cuda(), sums_to_dev(j.checksums), dev_i32(j.page_table)) for j in jobs]
+        gjobs = [gk.Job(b, s, t, j.n_tokens) for (b, s, t), j in zip(keep, jobs)]
+        mask = torch.full((6,), 255, dtype=torch.uint8, device="cuda")
+        fb = torch.full((6,), -9, dtype=torch.int32, device="cuda")
+        ctx.gk_restore(gjobs, d, mask, fb)
+        torch.cuda.synchronize()
+        assert mask.cpu().tolist() == [0, 1, 0, 4, 4, 4]
+        assert fb.cpu().tolist() == wfb.tolist() + [-1, -1, -1]
+        assert_cache_equal(d, want)
+        assert ctx.gk_get_stats()["device_wait_expired"] != 0
+        ctx.close()
+
+
+def test_one_segment_per_page_on_1_mib_records(gk):
+    """The tiling every full-size call takes -- a whole page record as ONE checksum segment
+    (many tiles per work item, no segment merge) -- forced on a small case of 1 MiB records
+    and compared in full: pack, checksums alone, verify + commit as separate calls, and the
+    fused restore, with damage in a full page and in the short last page."""
+    from gpu_harness import assert_cache_equal, dev_cache, dev_i32, gpu_pack, gpu_restore, sums_to_dev
+    og = oracle.Geom(16, 8, 128, 16)               # 64 KiB per token, 1 MiB per full page record
+    T = og.page_tokens
+    assert oracle.record_bytes(og, 4 * T, 0) == 1 << 20
+    lens = [3 * T + 5, 2 * T, T + 15]
+    total = sum(n_pages(og, n) for n in lens)
+    src = random_cache(og, total + 2, seed=380)
+    rng = np.random.default_rng(381)
+    tables = [rng.integers(0, total + 2, size=n_pages(og, n)).astype(np.int32) for n in lens]
+    granules = (1 << 20) // 32768
+    for seg in (granules, 2 * granules):           # exactly one record, and "longer than any record"
+        ctx = _ctx(gk, og, seg_granules=seg)
+        got, status = gpu_pack(ctx, og, dev_cache(src), tables, lens)
+        assert status.tolist() == [0, 0, 0]
+        ojobs, perm, used = [], rng.permutation(total + 3).astype(np.int32), 0
+        for (blob, sums), pt, n in zip(got, tables, lens):
+            wb, ws, code, _ = oracle.pack(og, src, pt, n)
+            assert code == 0 and np.array_equal(blob, wb) and np.array_equal(sums, ws)
+            # the checksums alone, from the blob
+            sums2 = torch.zeros(ws.size, dtype=torch.int64, device="cuda")
+            ctx.gk_page_checksums(torch.from_numpy(wb).cuda(), n, sums2)
+            torch.cuda.synchronize()
+            assert np.array_equal(sums2.cpu().numpy().view(np.uint64), ws)
+            P = n_pages(og, n)
+            ojobs.append(oracle.Job(wb.copy(), ws.copy(), perm[used:used + P].copy(), n))
+            used += P
+        ojobs[0].blob[oracle.record_offset(og, 3) + 77] ^= 0x01      # in the 5-token last page of job 0
+        ojobs[2].blob[(1 << 20) - 1] ^= 0x80                          # last byte of a full page of job 2
+        clean = random_cache(og, total + 3, seed=382)
+        want = clone_cache(clean)
+        wmask, wfb = oracle.restore(og, want, ojobs)
+        assert wmask.tolist() == [1, 0, 1] and wfb.tolist() == [3, -1, 0]
+        for host_tier in (False, True):
+            d = dev_cache(clean)
+            mask, fb = gpu_restore(ctx, d, ojobs, host_tier=host_tier)
+            assert mask.tolist() == wmask.tolist() and fb.tolist() == wfb.tolist()
+            assert_cache_equal(d, want)
+        # the two halves as separate calls (verify-only kernel, then commit-only kernel)
+        d = dev_cache(clean)
+        keep = [(torch.from_numpy(j.blob).cuda(), sums_to_dev(j.checksums), dev_i32(j.page_table)) for j in ojobs]
+        gjobs = [gk.Job(b, s_, t, j.n_tokens) for (b, s_, t), j in zip(keep, ojobs)]
+        mask = torch.full((3,), 255, dtype=torch.uint8, device="cuda")
+        fb = torch.full((3,), -9, dtype=torch.int32, device="cuda")
+        ctx.gk_verify(gjobs, d, mask, fb)
+        torch.cuda.synchronize()
+        assert mask.cpu().tolist() == wmask.tolist() and fb.cpu().tolist() == wfb.tolist()
+        assert_cache_equal(d, clean)
+        ctx.gk_commit(gjobs, d, mask)
+        torch.cuda.synchronize()
+        assert_cache_equal(d, want)
+        assert ctx.gk_get_stats()["device_wait_expired"] == 0
+        ctx.close()
+
+
+@pytest.mark.parametrize("n_jobs", [65, 96])
+def test_device_tier_call_of_many_tiny_jobs(gk, n_jobs):
+    """More than 64 jobs in ONE device-tier call: gk_pack_batch and gk_restore then take the
+    staged job-table upload followed by the validation and claim kernels (smaller calls pass
+    the table as kernel arguments).  Every kind of damage the random suite knows, several of
+    each, full destination image against the oracle."""
+    from gpu_harness import assert_cache_equal, dev_cache, gpu_pack, gpu_restore
+    og = G_MID
+    T = og.page_tokens
+    rng = np.random.default_rng(8800 + n_jobs)
+    lens = [int(rng.integers(1, 3 * T + 1)) for _ in range(n_jobs)]
+    Ns = 40
+    src = random_cache(og, Ns, seed=8801)
+    tables = [rng.integers(0, Ns, size=n_pages(og, n)).astype(np.int32) for n in lens]
+    tables[7][0] = Ns + 1                           # save: an id out of range -> status 2, nothing written
+    for fused in (1, 0):
+        ctx = _ctx(gk, og, fused=fused)
+        got, status = gpu_pack(ctx, og, dev_cache(src), tables, lens)
+        wstatus = [0] * n_jobs
+        wstatus[7] = 2
+        assert status.tolist() == wstatus
+        total = sum(n_pages(og, n) for n in lens)
+        Nd = total + 5
+        perm = rng.permutation(Nd).astype(np.int32)
+        ojobs, used = [], 0
+        for j, ((blob, sums), pt, n) in enumerate(zip(got, tables, lens)):
+            P = n_pages(og, n)
+            if j == 7:
+                assert not blob.any() and not sums.any()        # left as the harness zeroed them
+                pt = tables[7].copy()
+                pt[0] = 0
+                wb, ws, code, _ = oracle.pack(og, src, pt, n)
+            else:
+                wb, ws, code, _ = oracle.pack(og, src, pt, n)
+                assert code == 0 and np.array_equal(blob, wb) and np.array_equal(sums, ws)
+            ojobs.append(oracle.Job(wb.copy(), ws.copy(), perm[used:used + P].copy(), n))
+            used += P
+        for j, jb in enumerate(ojobs):
+            kind = j % 8
+            if kind == 1:
+                for _ in range(1 + j % 4):
+                    jb.blob[int(rng.integers(0, jb.blob.size))] ^= np.uint8(1 << int(rng.integers(0, 8)))
+            elif kind == 2:
+                jb.checksums[int(rng.integers(0, jb.checksums.size))] ^= np.uint64(1) << np.uint64(int(rng.integers(0, 64)))
+            elif kind == 3:
+                ojobs[j] = oracle.Job(None, None, jb.page_table, jb.n_tokens)
+            elif kind == 4:
+                jb.page_table[int(rng.integers(0, jb.page_table.size))] = Nd + 2 if j % 16 == 4 else -1
+            elif kind == 5:
+                jb.page_table[0] = ojobs[(j + 1) % n_jobs].page_table[0]
+        clean = random_cache(og, Nd, seed=8802)
+        want = clone_cache(clean)
+        wmask, wfb = oracle.restore(og, want, ojobs)
+        assert set(wmask.tolist()) == {0, 1, 2, 3}
+        d = dev_cache(clean)
+        mask, fb = gpu_restore(ctx, d, ojobs, host_tier=False)
+        assert mask.tolist() == wmask.tolist()
+        assert fb.tolist() == wfb.tolist()
+        assert_cache_equal(d, want)
+        ctx.close()
+
+
+def test_reserve_sizes_everything_once(gk):
+    """After gk_ctx_reserve no call within the stated bounds allocates (and so none frees or
+    synchronises the device): the context's allocation counter stays where reserve left it
+    across small and large calls of every kind, on both tiers, and the results stay bit-exact."""
+    from gpu_harness import assert_cache_equal, dev_cache, dev_i32, gpu_pack, gpu_restore, sums_to_dev
+    og = G_MID
+    T = og.page_tokens
+    rng = np.random.default_rng(8900)
+    ctx = _ctx(gk, og)
+    max_jobs, max_pages, num_pages = 100, 320, 400
+    blob_max = oracle.blob_size(og, 3 * T)[0]
+    ctx.gk_ctx_reserve(max_jobs, max_pages, num_pages, max_jobs * blob_max)
+    base = ctx.gk_get_stats()["allocations"]
+    assert base > 0
+    src = random_cache(og, 60, seed=8901)
+    for n_jobs in (1, 4, 64, 65, 100):
+        lens = [int(rng.integers(1, 3 * T + 1)) for _ in range(n_jobs)]
+        tables = [rng.integers(0, 60, size=n_pages(og, n)).astype(np.int32) for n in lens]
+        got, status = gpu_pack(ctx, og, dev_cache(src), tables, lens)
+        assert not status.any()
+        total = sum(n_pages(og, n) for n in lens)
+        perm = rng.permutation(num_pages).astype(np.int32)
+        ojobs, used = [], 0
+        for (blob, sums), pt, n in zip(got, tables, lens):
+            wb, ws, code, _ = oracle.pack(og, src, pt, n)
+            assert np.array_equal(blob, wb) and np.array_equal(sums, ws)
+            P = n_pages(og, n)
+            ojobs.append(oracle.Job(wb, ws, perm[used:used + P].copy(), n))
+            used += P
+        ojobs[0].blob[5] ^= 1
+        clean = random_cache(og, num_pages, seed=8902 + n_jobs)
+        want = clone_cache(clean)
+        wmask, wfb = oracle.restore(og, want, ojobs)
+        for host_tier in (False, True):
+            d = dev_cache(clean)
+            mask, fb = gpu_restore(ctx, d, ojobs, host_tier=host_tier)
+            assert mask.tolist() == wmask.tolist() and fb.tolist() == wfb.tolist()
+            assert_cache_equal(d, want)
+        # the two halves and the checksum-only call
+        d = dev_cache(clean)
+        keep = [(torch.from_numpy(j.blob).cuda(), sums_to_dev(j.checksums), dev_i32(j.page_table)) for j in ojobs]
+        gjobs = [gk.Job(b, s_, t, j.n_tokens) for (b, s_, t), j in zip(keep, ojobs)]
+        mask = torch.full((n_jobs,), 255, dtype=torch.uint8, device="cuda")
+        fb = torch.zeros(n_jobs, dtype=torch.int32, device="cuda")
+        ctx.gk_verify(gjobs, d, mask, fb)
+        ctx.gk_commit(gjobs, d, mask)
+        sums2 = torch.zeros(ojobs[1 % n_jobs].checksums.size, dtype=torch.int64, device="cuda")
+        ctx.gk_page_checksums(keep[1 % n_jobs][0], ojobs[1 % n_jobs].n_tokens, sums2)
+        torch.cuda.synchronize()
+        assert_cache_equal(d, want)
+        # save to the host tier
+        hjobs, hkeep = [], []
+        for (blob, sums), pt, n in zip(got, tables, lens):
+            hb = torch.empty(blob.size, dtype=torch.uint8, pin_memory=True)
+            hs = torch.empty(sums.size, dtype=torch.int64, pin_memory=True)
+            hkeep.append((hb, hs))
+            hjobs.append(gk.Job(hb, hs, dev_i32(pt), n))
+        ctx.gk_pack_host(dev_cache(src), hjobs)
+        torch.cuda.synchronize()
+        for (hb, hs), (blob, sums) in zip(hkeep, got):
+            assert np.array_equal(hb.numpy(), blob) and np.array_equal(hs.numpy().view(np.uint64), sums)
+        assert ctx.gk_get_stats()["allocations"] == base, f"a call of {n_jobs} jobs allocated after reserve"
+    ctx.close()
+    # without reserve the same calls do allocate: the counter means something
+    ctx = _ctx(gk, og)
+    got, _ = gpu_pack(ctx, og, dev_cache(src), [np.zeros(1, dtype=np.int32)] * 70, [T] * 70)
+    assert ctx.gk_get_stats()["allocations"] > 0
     ctx.close()
 
 
