@@ -46,7 +46,7 @@
  *   shared by its calls: calls on one context must be issued in stream order on
  *   one stream at a time (use one context per concurrent stream).  gk_pack,
  *   gk_pack_batch, gk_restore, gk_verify and gk_commit calls of at most 64 jobs
- *   and 16,384 pages make no host-device copy and no synchronisation once the
+ *   and 2,048 pages make no host-device copy and no synchronisation once the
  *   workspace has its size, and may be captured in a CUDA graph and replayed;
  *   the other entry points and larger calls may not.
  *   Requirements: row % 16 == 0, scale section bytes % 16 == 0, all base

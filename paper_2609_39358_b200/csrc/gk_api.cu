@@ -100,6 +100,7 @@ struct gk_ctx {
     int device = 0;
     int sm_count = 0;
     int occ_verify = 0, occ_pack = 0, occ_commit = 0, occ_fused = 0, occ_single = 0;
+    uint64_t *d_thread_const = nullptr;
     bool fused = true;           // restore runs verify and commit in one launch
     unsigned long long wait_limit_ns = kWaitLimitNs;
     uint32_t ctr_next[2] = {0, 0};  // what the device work counters will read when the next launch of
@@ -107,13 +108,13 @@ struct gk_ctx {
     uint32_t test_drop_verify = 0;  // test hook: see gk_ctx_set_tuning
     bool commit_reverse = true;     // commit side walks a job's pages from the last to the first
     uint32_t l2_hints = 0;          // bit 0: verify loads evict_last, bit 1: commit loads evict_first
+    unsigned long long *trace = nullptr;  // builds with GK_TRACE: device buffer for time stamps (tuning keys)
     uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
     uint32_t commit_seg_tiles = 0;
     uint32_t grid_cap = 0;       // 0: SMs * occupancy
 
     // constant tables + sticky error word
     uint64_t *d_init_term = nullptr;
-    uint64_t *d_thread_const = nullptr;
     uint32_t *d_error = nullptr;
 
     // growing device workspace and pinned staging for job tables
@@ -274,7 +275,8 @@ Tiling crc_tiling(const gk_ctx *c, uint32_t stage_bytes, uint64_t total_pages, i
         const double item_us = 20.0;
         double best = 1e30;
         uint32_t best_k = 1;
-        const uint32_t kmax = gran_full > 1 ? gran_full / 2 : 1;  // at least two granules per segment
+        uint32_t kmax = gran_full > 1 ? gran_full / 2 : 1;  // at least two granules per segment
+        if (kmax > kPrepMaxSeg) kmax = kPrepMaxSeg;               // and the table must fit the preparation launch
         for (uint32_t k = 1; k <= kmax; ++k) {
             const uint32_t g = (gran_full + k - 1) / k;            // granules per segment
             const uint32_t nseg = (gran_full + g - 1) / g;
@@ -301,13 +303,13 @@ Tiling crc_tiling(const gk_ctx *c, uint32_t stage_bytes, uint64_t total_pages, i
     return t;
 }
 
-Tiling commit_tiling(const gk_ctx *c, uint64_t total_pages, int occ)
+Tiling commit_tiling(const gk_ctx *c, uint32_t stage_bytes, uint64_t total_pages, int occ)
 {
     Tiling t;
-    t.stage_bytes = GK_COPY_STAGE;
-    t.gran_bytes = GK_COPY_STAGE;
+    t.stage_bytes = stage_bytes;
+    t.gran_bytes = stage_bytes;
     const uint32_t tiles_full = (uint32_t)((c->gd.R + t.stage_bytes - 1) / t.stage_bytes);
-    uint32_t st = 16u;
+    uint32_t st = (256u << 10) / stage_bytes;  // 256 KiB per commit item
     if (c->commit_seg_tiles) {
         st = c->commit_seg_tiles;
     } else if (total_pages > 0) {
@@ -333,7 +335,7 @@ WsLayout ws_layout(uint32_t n_jobs, uint64_t total_pages, uint32_t nseg_max, uin
 {
     WsLayout l;
     size_t o = 0;
-    l.jobs = o;      o = align_up(o + (size_t)n_jobs * sizeof(JobDev) + (size_t)nseg_max * 8, 256);  // + seg_pow
+    l.jobs = o;      o = align_up(o + (size_t)n_jobs * sizeof(JobDev) + (size_t)nseg_max * 16, 256);  // + seg_pow
     l.page_job = o;  o = align_up(o + (size_t)total_pages * 4, 256);
     l.page_acc = o;  o = align_up(o + (size_t)total_pages * 8, 256);
     l.bad_range = o; o = align_up(o + (size_t)n_jobs * 4, 256);
@@ -407,9 +409,13 @@ const gk_ctx::SegPowers &seg_powers(gk_ctx *c, uint64_t seg_bytes, uint32_t n)
         e = oldest;
         e->seg_bytes = seg_bytes;
         e->x_seg = gf_xpow(8ull * seg_bytes);
-        e->pw.assign(1, 1ull);
+        e->pw.assign({1ull, 1ull << 32});
     }
-    while (e->pw.size() < n) e->pw.push_back(gf_mul(e->pw.back(), e->x_seg));
+    while (e->pw.size() < 2 * (size_t)n) {
+        const uint64_t next = gf_mul(e->pw[e->pw.size() - 2], e->x_seg);
+        e->pw.push_back(next);
+        e->pw.push_back(gf_mul(next, 1ull << 32));
+    }
     e->used = ++c->seg_cache_clock;
     return *e;
 }
@@ -434,7 +440,6 @@ WorkDev make_work(gk_ctx *c, const WsLayout &l, uint32_t n_jobs, uint32_t total_
     w.work_ctr = c->d_error + 16;
     w.init_term = c->d_init_term;
     w.thread_const = c->d_thread_const;
-    w.x_seg = seg_powers(c, (uint64_t)crc.seg_tiles * crc.stage_bytes, 1).x_seg;
     w.seg_pow = (const uint64_t *)(c->d_ws + l.jobs + (size_t)n_jobs * sizeof(JobDev));
     w.wait_limit_ns = c->wait_limit_ns;
     return w;
@@ -472,12 +477,13 @@ int fill_job_table(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, JobDev *h, ui
     return GK_OK;
 }
 
-// powers of x^(8 * segment bytes), which place segment remainders inside their page
+// powers of x^(8 * segment bytes), which place segment remainders inside their page: for every
+// power k the pair (power, power * x^32), one factor for each 32-bit half of a remainder
 void fill_seg_pow(gk_ctx *c, const Tiling &crc, uint64_t *pw)
 {
     if (crc.nseg_max == 0) return;
     const gk_ctx::SegPowers &sp = seg_powers(c, (uint64_t)crc.seg_tiles * crc.stage_bytes, crc.nseg_max);
-    std::memcpy(pw, sp.pw.data(), (size_t)crc.nseg_max * 8);
+    std::memcpy(pw, sp.pw.data(), (size_t)crc.nseg_max * 16);
 }
 
 // Fills the pinned job table (and the segment powers behind it) and enqueues the upload.
@@ -485,7 +491,7 @@ int upload_jobs(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const WsLayout &
                 uint8_t *const *blob_override, uint64_t *const *sums_override, bool need_tables, cudaStream_t st,
                 uint64_t *total_pages_out, uint64_t *total_bytes_out)
 {
-    const size_t table_bytes = (size_t)n_jobs * sizeof(JobDev) + (size_t)crc.nseg_max * 8;
+    const size_t table_bytes = (size_t)n_jobs * sizeof(JobDev) + (size_t)crc.nseg_max * 16;
     uint8_t *stage = nullptr;
     cudaEvent_t ev = nullptr;
     int rc = next_host_stage(c, table_bytes, &stage, &ev);
@@ -504,7 +510,9 @@ int upload_jobs(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const WsLayout &
 // preparation launch (no staging copy, no separate validate / claim launches).
 bool is_small_call(uint32_t n_jobs, uint64_t pages, const Tiling &crc)
 {
-    return n_jobs <= kPrepMaxJobs && crc.nseg_max <= kPrepMaxSeg && pages <= 16384;
+    // one CTA walks all pages of the call three times: beyond two pages per thread the parallel
+    // validation and claim kernels are faster, staging copy included
+    return n_jobs <= kPrepMaxJobs && crc.nseg_max <= kPrepMaxSeg && pages <= 2048;
 }
 
 int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tiling &crc, const WorkDev &w,
@@ -515,7 +523,7 @@ int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tili
     int rc = fill_job_table(c, jobs, n_jobs, pp.jobs, nullptr, nullptr, need_tables, pages_out, bytes_out);
     if (rc != GK_OK) return rc;
     fill_seg_pow(c, crc, pp.seg_pow);
-    pp.n_seg_pow = crc.nseg_max;
+    pp.n_seg_pow = 2 * crc.nseg_max;
     pp.do_claims = do_claims ? 1u : 0u;
     pp.num_pages = num_pages;
     pp.status_out = status_out;
@@ -525,6 +533,15 @@ int launch_prep_small(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tili
     c->stats.kernels_launched++;
     c->pdl_next = !c->profile;  // timing events between the two launches would break the pairing
     return GK_OK;
+}
+
+// Draws from a work counter in one launch.  A loader draws once per item it meets and stops at
+// the first number that is past the end; taking the first item without drawing (the CTA's own
+// number) saves one draw per CTA.  The host adds these up so that it can tell every later
+// launch of the call what its counter starts from.
+uint32_t draws_of(uint32_t n_items, uint32_t grid, bool static_first)
+{
+    return n_items + (static_first ? 0u : grid);
 }
 
 uint32_t stream_grid(const gk_ctx *c, int occ, uint32_t n_items)
@@ -586,13 +603,12 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
     gk_ctx::ProfSlot *slot = nullptr;
     int rc_prof = prof_begin(c, MODE, st, &slot);  // kSingle == 3: booked with the fused restore kernel
     if (rc_prof != GK_OK) return rc_prof;
-    // A CTA takes the item with its own number first and draws the others from the counter; every
-    // CTA that has an item draws once more to learn that none is left: `items` draws per launch.
     StreamParams Q = P;
     const int ci = MODE == kCommit ? 1 : 0;
     if (ci) Q.ctr_base_c = c->ctr_next[1];
     else Q.ctr_base_v = c->ctr_next[0];
-    c->ctr_next[ci] += items;
+    Q.trace = c->trace;
+    c->ctr_next[ci] += draws_of(items, grid, true);
     GK_CUDA(c, launch_streaming(c, stream_kernel<MODE, NT, SB, ST, MINB>, grid, Cfg::kThreads, Cfg::kSmemBytes, st, Q));
     if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
@@ -632,9 +648,10 @@ int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
     StreamParams Q = P;
     Q.ctr_base_v = c->ctr_next[0];
     Q.ctr_base_c = c->ctr_next[1];
-    // the verify side draws every item (and once more per CTA); the commit side as in launch_stream
-    c->ctr_next[0] += P.n_items + grid;
-    c->ctr_next[1] += P.n_items_c;
+    Q.trace = c->trace;
+    // the verify side draws every item, the commit side takes the first one of each CTA without drawing
+    c->ctr_next[0] += draws_of(P.n_items, grid, false);
+    c->ctr_next[1] += draws_of(P.n_items_c, grid, true);
     GK_CUDA(c, launch_streaming(c, restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE,
                                                   GK_FUSED_CSTAGES, GK_FUSED_MINB>,
                                 grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st, Q));
@@ -648,12 +665,12 @@ int launch_validate(gk_ctx *c, const WorkDev &w, uint64_t num_pages, int clear_c
 {
     uint32_t grid = w.n_jobs;
     if (clear_claims) {
-        uint32_t g2 = (uint32_t)((num_pages + 255) / 256);
+        uint32_t g2 = (uint32_t)((num_pages + 1023) / 1024);
         if (g2 > 2048) g2 = 2048;
         if (g2 > grid) grid = g2;
     }
     c->ctr_next[0] = c->ctr_next[1] = 0;  // the kernel zeroes the device counters
-    validate_kernel<<<grid, 256, 0, st>>>(w, num_pages, clear_claims, status_out);
+    validate_kernel<<<grid, 1024, 0, st>>>(w, num_pages, clear_claims, status_out);
     GK_CUDA(c, cudaGetLastError());
     c->stats.kernels_launched++;
     return GK_OK;
@@ -881,41 +898,40 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
     if (prop.major != 10) return bail(GK_ERR_UNSUPPORTED);  // built for sm_100a only
     c->sm_count = prop.multiProcessorCount;
 
-    auto *kv = stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB>;
-    auto *kp = stream_kernel<kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>;
-    auto *kc = stream_kernel<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES, GK_COPY_MINB>;
-    if (cudaFuncSetAttribute(kv, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)VerifyCfg::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(kp, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)PackCfg::kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(kc, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CommitCfg::kSmemBytes) != cudaSuccess)
+    // every streaming kernel: shared-memory size, then how many CTAs of it an SM holds
+    auto prepare = [&](auto *kernel, int threads, size_t smem, int *occ) {
+        return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess &&
+               cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, kernel, threads, smem) == cudaSuccess && *occ >= 1;
+    };
+    if (!prepare(stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB>, VerifyCfg::kThreads,
+                 VerifyCfg::kSmemBytes, &c->occ_verify) ||
+        !prepare(stream_kernel<kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>, PackCfg::kThreads,
+                 PackCfg::kSmemBytes, &c->occ_pack) ||
+        !prepare(restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES, GK_FUSED_MINB>,
+                 FusedCfg::kThreads, FusedCfg::kSmemBytes, &c->occ_fused) ||
+        !prepare(stream_kernel<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES, GK_COPY_MINB>, CommitCfg::kThreads,
+                 CommitCfg::kSmemBytes, &c->occ_commit) ||
+        !prepare(stream_kernel<kSingle, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>, SingleCfg::kThreads,
+                 SingleCfg::kSmemBytes, &c->occ_single)) {
+        cudaGetLastError();
         return bail(GK_ERR_CUDA);
-    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_verify, kv, VerifyCfg::kThreads, VerifyCfg::kSmemBytes) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_pack, kp, PackCfg::kThreads, PackCfg::kSmemBytes) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_commit, kc, CommitCfg::kThreads, CommitCfg::kSmemBytes) != cudaSuccess)
-        return bail(GK_ERR_CUDA);
-    auto *kf = restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES, GK_FUSED_MINB>;
-    if (cudaFuncSetAttribute(kf, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FusedCfg::kSmemBytes) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_fused, kf, FusedCfg::kThreads, FusedCfg::kSmemBytes) != cudaSuccess)
-        return bail(GK_ERR_CUDA);
-    auto *ks = stream_kernel<kSingle, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>;
-    if (cudaFuncSetAttribute(ks, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SingleCfg::kSmemBytes) != cudaSuccess ||
-        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&c->occ_single, ks, SingleCfg::kThreads, SingleCfg::kSmemBytes) != cudaSuccess)
-        return bail(GK_ERR_CUDA);
-    if (c->occ_verify < 1 || c->occ_pack < 1 || c->occ_commit < 1 || c->occ_fused < 1 || c->occ_single < 1)
-        return bail(GK_ERR_UNSUPPORTED);
+    }
 
     // tables: ones * x^(8*len(t)) for every page fill t, and the per-thread placement constants
     std::vector<uint64_t> init(gd.page_tokens + 1, 0);
     for (uint32_t t = 1; t <= gd.page_tokens; ++t)
         init[t] = gf_mul(~0ull, gf_xpow(8ull * (gd.S + (uint64_t)t * gd.tokB)));
-    std::vector<uint64_t> tc(GK_CRC_NT);
-    for (int t = 0; t < GK_CRC_NT; ++t) tc[t] = gf_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);
-    if (cudaMalloc(&c->d_init_term, init.size() * 8) != cudaSuccess ||
-        cudaMalloc(&c->d_thread_const, tc.size() * 8) != cudaSuccess ||
-        cudaMalloc(&c->d_error, 256) != cudaSuccess)
+    if (cudaMalloc(&c->d_init_term, init.size() * 8) != cudaSuccess || cudaMalloc(&c->d_error, 256) != cudaSuccess)
         return bail(GK_ERR_NOMEM);
     if (cudaMemcpy(c->d_init_term, init.data(), init.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
-        cudaMemcpy(c->d_thread_const, tc.data(), tc.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemset(c->d_error, 0, 256) != cudaSuccess)
+        return bail(GK_ERR_CUDA);
+    std::vector<uint64_t> tc(GK_CRC_NT + 2 * (GK_CRC_NT / 32));
+    for (int t = 0; t < GK_CRC_NT; ++t) tc[t] = gf_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);
+    for (int w = 0; w < GK_CRC_NT / 32; ++w)  // the two words that stick out above warp w
+        for (int i = 0; i < 2; ++i) tc[GK_CRC_NT + 2 * w + i] = gf_xpow(1024ull * (GK_CRC_NT / 32 - w) + 64ull + 32ull * i);
+    if (cudaMalloc(&c->d_thread_const, tc.size() * 8) != cudaSuccess) return bail(GK_ERR_NOMEM);
+    if (cudaMemcpy(c->d_thread_const, tc.data(), tc.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess)
         return bail(GK_ERR_CUDA);
     for (int i = 0; i < 2; ++i)
         if (cudaEventCreateWithFlags(&c->ev_stage[i], cudaEventDisableTiming) != cudaSuccess) return bail(GK_ERR_CUDA);
@@ -974,6 +990,10 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     else if (!strcmp(key, "test_drop_verify")) c->test_drop_verify = value;
     else if (!strcmp(key, "commit_reverse")) c->commit_reverse = value != 0;
     else if (!strcmp(key, "l2_hints")) c->l2_hints = value;
+#ifdef GK_TRACE
+    else if (!strcmp(key, "trace_lo")) c->trace = (unsigned long long *)(((uintptr_t)c->trace & ~(uintptr_t)0xffffffffull) | value);
+    else if (!strcmp(key, "trace_hi")) c->trace = (unsigned long long *)(((uintptr_t)c->trace & 0xffffffffull) | ((uintptr_t)value << 32));
+#endif
     else return fail(c, GK_ERR_ARG, "unknown tuning key %s", key);
     return GK_OK;
 }
@@ -988,7 +1008,7 @@ int gk_ctx_reserve(gk_ctx *c, uint32_t max_jobs, uint64_t max_pages, uint64_t nu
     const WsLayout l = ws_layout(max_jobs, max_pages, seg_max, num_pages);
     int rc;
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
-    if ((rc = ensure_host_stage(c, (size_t)max_jobs * sizeof(JobDev) + (size_t)seg_max * 8)) != GK_OK) return rc;
+    if ((rc = ensure_host_stage(c, (size_t)max_jobs * sizeof(JobDev) + (size_t)seg_max * 16)) != GK_OK) return rc;
     if (max_jobs && (rc = ensure_group_tmp(c, max_jobs)) != GK_OK) return rc;
     if (max_host_batch_bytes) {
         // room for the checksums beside the blobs, and for the alignment of every job's two parts
@@ -1024,7 +1044,7 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
 
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
-    const Tiling tl = crc_tiling(c, GK_PACK_STAGE, pages, c->occ_pack);
+    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_pack);
     const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tl);
@@ -1154,10 +1174,11 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
     const bool single = (c->gd.flags & GK_FLAG_SINGLE_PASS) && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
-    const bool fused = !single && c->fused && !(n_jobs == 1 && pages * c->gd.R >= (256ull << 20));
-    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages, single ? c->occ_single : fused ? c->occ_fused : c->occ_verify,
-                                  fused && n_jobs > 1);
-    const Tiling tlc = commit_tiling(c, pages, fused ? c->occ_fused : c->occ_commit);
+    const bool fused = !single && c->fused && !(c->gd.flags & GK_FLAG_SKIP_VERIFY) &&
+                       !(n_jobs == 1 && pages * c->gd.R >= (256ull << 20));
+    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages,
+                                  single ? c->occ_single : fused ? c->occ_fused : c->occ_verify, fused && n_jobs > 1);
+    const Tiling tlc = commit_tiling(c, GK_COPY_STAGE, pages, fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tlv);
@@ -1187,7 +1208,7 @@ static int prepare_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
     *tlv = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify);
-    *tlc = commit_tiling(c, pages, c->occ_commit);
+    *tlc = commit_tiling(c, GK_COPY_STAGE, pages, c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv->nseg_max, cd->num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     *w = make_work(c, l, n_jobs, (uint32_t)pages, *tlv);
@@ -1293,9 +1314,11 @@ static int restore_host_impl(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, con
 
     // batches are what is launched, so size the work items for a batch, not for the call
     const uint64_t pages_per_launch = (pages + batch_end.size() - 1) / batch_end.size();
-    const int occ = c->fused ? c->occ_fused : c->occ_verify;
-    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages_per_launch, occ, c->fused && n_jobs > batch_end.size());
-    const Tiling tlc = commit_tiling(c, pages_per_launch, c->fused ? c->occ_fused : c->occ_commit);
+    const bool single = (c->gd.flags & GK_FLAG_SINGLE_PASS) && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
+    const bool fused = c->fused && !single && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
+    const int occ = single ? c->occ_single : fused ? c->occ_fused : c->occ_verify;
+    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages_per_launch, occ, fused && n_jobs > batch_end.size());
+    const Tiling tlc = commit_tiling(c, GK_COPY_STAGE, pages_per_launch, fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     uint64_t bytes = 0;
@@ -1402,7 +1425,7 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
     if ((rc = make_host_plan(c, jobs, n_jobs, false, hp)) != GK_OK) return rc;
 
     uint64_t pages = hp.pages, bytes = 0;
-    const Tiling tl = crc_tiling(c, GK_PACK_STAGE, (pages + hp.batch_end.size() - 1) / hp.batch_end.size(), c->occ_pack);
+    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, (pages + hp.batch_end.size() - 1) / hp.batch_end.size(), c->occ_pack);
     const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     if ((rc = upload_jobs(c, jobs, n_jobs, l, tl, hp.blob_dev.data(), hp.sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
@@ -1716,7 +1739,7 @@ struct NoallocLayout {
     static constexpr size_t page_acc = page_cnt + 4 * (size_t)kNoallocMaxPages;            // [max pages] u64
     static constexpr size_t total = page_acc + 8 * (size_t)kNoallocMaxPages;
 };
-static_assert(GK_CRC_NT <= 256, "thread constant table");
+static_assert(GK_CRC_NT + 2 * (GK_CRC_NT / 32) <= 256, "thread constant table");
 static_assert(NoallocLayout::page_job % 256 == 0 && NoallocLayout::page_acc % 8 == 0, "scratch alignment");
 
 // The scratch itself: about 133 KiB per GPU that loads the library, held until exit.
@@ -1760,6 +1783,8 @@ __global__ void noalloc_setup_kernel(unsigned char *scratch, JobDev job, GeomDev
     }
     for (uint32_t t = threadIdx.x; t < (uint32_t)GK_CRC_NT; t += blockDim.x)
         tc[t] = dev_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);
+    for (uint32_t k = threadIdx.x; k < 2u * (GK_CRC_NT / 32); k += blockDim.x)  // the words above each warp
+        tc[GK_CRC_NT + k] = dev_xpow(1024ull * (GK_CRC_NT / 32 - k / 2u) + 64ull + 32ull * (k & 1u));
     for (uint32_t t = threadIdx.x; t <= g.page_tokens; t += blockDim.x)
         it[t] = t ? gf_mul(~0ull, dev_xpow(8ull * (g.S + (uint64_t)t * g.tokB))) : 0ull;
     for (uint32_t p = threadIdx.x; p < job.n_pages; p += blockDim.x) {
@@ -1868,7 +1893,6 @@ int gk_page_checksums_noalloc(const gk_geom *geom, const void *blob_dev, uint32_
     w.work_ctr = reinterpret_cast<uint32_t *>(words + 5);
     w.init_term = reinterpret_cast<const uint64_t *>(sc + NoallocLayout::init_term);
     w.thread_const = reinterpret_cast<const uint64_t *>(sc + NoallocLayout::thread_const);
-    w.x_seg = gf_xpow(8ull * tl.seg_tiles * tl.stage_bytes);
     w.wait_limit_ns = kWaitLimitNs;
 
     noalloc_setup_kernel<<<1, 256, 0, st>>>(sc, job, gd);

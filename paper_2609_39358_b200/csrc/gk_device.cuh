@@ -66,9 +66,10 @@ struct WorkDev {
                                   // error word as the call's first kernel found it
     uint32_t *error;              // sticky: non-zero once a bounded wait has run out
     const uint64_t *init_term;    // [page_tokens+1] ones * x^(8*len(t)) mod P
-    const uint64_t *thread_const; // [NT] x^(32*(NT-1-t)+64) mod P
-    const uint64_t *seg_pow;      // [nseg_max] (x^(8*segment bytes))^k mod P: places segment remainders
-    uint64_t x_seg;               // x^(8*segment bytes) mod P
+    const uint64_t *thread_const; // [NT] x^(32*(NT-1-t)+64) mod P, then for each warp w of NT/32 the constants
+                                  // of the two words above it: x^(1024*(NT/32-w)+64) and that times x^32
+    const uint64_t *seg_pow;      // [nseg_max][2] (x^(8*segment bytes))^k mod P and that times x^32: place
+                                  // the two halves of a segment remainder
     unsigned long long wait_limit_ns;  // time limit of every device-side wait
 };
 
@@ -92,11 +93,16 @@ struct PageShape {
     uint32_t ntiles0;  // tiles in segment 0
 };
 
-__device__ __forceinline__ PageShape page_shape(const GeomDev &g, const JobDev &jb, uint32_t p,
-                                                const Tiling &tl)
+__device__ __forceinline__ uint32_t page_fill(const GeomDev &g, const JobDev &jb, uint32_t p)
+{
+    return (p + 1u < jb.n_pages) ? g.page_tokens : jb.n_tokens - (jb.n_pages - 1u) * g.page_tokens;
+}
+
+// Shape of the record of a page that holds t tokens.
+__device__ __forceinline__ PageShape page_shape_t(const GeomDev &g, uint32_t t, const Tiling &tl)
 {
     PageShape s;
-    s.t = (p + 1u < jb.n_pages) ? g.page_tokens : jb.n_tokens - (jb.n_pages - 1u) * g.page_tokens;
+    s.t = t;
     s.len = (uint64_t)g.S + (uint64_t)s.t * g.tokB;
     // gran_bytes and stage_bytes are powers of two: masks and shifts, no 64-bit division
     const uint64_t v = (s.len + tl.gran_bytes - 1) & ~(uint64_t)(tl.gran_bytes - 1u);
@@ -105,6 +111,12 @@ __device__ __forceinline__ PageShape page_shape(const GeomDev &g, const JobDev &
     s.nseg = (s.ntiles + tl.seg_tiles - 1u) / tl.seg_tiles;
     s.ntiles0 = s.ntiles - (s.nseg - 1u) * tl.seg_tiles;
     return s;
+}
+
+__device__ __forceinline__ PageShape page_shape(const GeomDev &g, const JobDev &jb, uint32_t p,
+                                                const Tiling &tl)
+{
+    return page_shape_t(g, page_fill(g, jb, p), tl);
 }
 
 // ---- GF(2)[x] mod P on 64-bit values (bit k = coefficient of x^k) ----
@@ -151,6 +163,21 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+
+// Non-blocking form: try_wait may suspend the thread for a while before it answers "not yet",
+// which a loop that watches two barriers cannot afford.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(ok)
         : "r"(bar), "r"(parity)

@@ -83,6 +83,7 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims,
     if (threadIdx.x == 0) s_bad = kNoPage;
     __syncthreads();
     int32_t bad = kNoPage;
+#pragma unroll 4
     for (uint32_t p = threadIdx.x; p < jb.n_pages; p += blockDim.x) {
         w.page_job[jb.page_base + p] = (int32_t)j;
         w.page_cnt[jb.page_base + p] = 0u;
@@ -131,10 +132,10 @@ __global__ void claim_kernel(WorkDev w)
 // claim_kernel do, separated by a CTA barrier.  Only the claim words that this
 // call can touch are cleared.
 constexpr uint32_t kPrepMaxJobs = 64;
-constexpr uint32_t kPrepMaxSeg = 96;
+constexpr uint32_t kPrepMaxSeg = 64;
 struct PrepSmallParams {
     JobDev jobs[kPrepMaxJobs];
-    uint64_t seg_pow[kPrepMaxSeg];
+    uint64_t seg_pow[2 * kPrepMaxSeg];
     uint32_t n_seg_pow;
     uint32_t do_claims;
     uint64_t num_pages;
@@ -304,13 +305,15 @@ struct StreamCfg {
     static constexpr int kConsWarps = kCrc ? NT / 32 : 0;
     static constexpr int kLoaderWarp = kConsWarps;
     static constexpr int kStorerWarp = kConsWarps + 1;
-    static constexpr int kThreads = 32 * (kConsWarps + 1 + (kStore ? 1 : 0));
+    static constexpr bool kOwnFinisher = kCrc && !kStore;   // else the storer warp finishes the segments
+    static constexpr int kFinisherWarp = kConsWarps + 1;    // where it is a warp of its own
+    static constexpr int kThreads = 32 * (kConsWarps + 1 + (kStore ? 1 : 0) + (kOwnFinisher ? 1 : 0));
     static constexpr int kGran = kCrc ? NT * 256 : STAGE_BYTES;  // 8 shift-register steps of 8 words per thread
     static constexpr int kSps = kCrc ? STAGE_BYTES / (NT * 32) : 1;  // 8-word steps per stage
     static constexpr int kTilesPerGran = kGran / STAGE_BYTES;
     // stages | full and empty barriers | tags | item slots | reduction slots [2][8] | abort flag | alignment slack
     static constexpr size_t kSmemBytes =
-        (size_t)STAGES * STAGE_BYTES + 3 * STAGES * 8 + (STAGES + 1) * sizeof(Item) + 2 * 8 * 8 + 16 + 128;
+        (size_t)STAGES * STAGE_BYTES + 3 * STAGES * 8 + (STAGES + 1) * sizeof(Item) + 2 * 12 * 8 + 4 * 8 + 16 + 16;
     static_assert(!kCrc || (NT == 32 || NT == 64 || NT == 128 || NT == 256), "NT must be a power of two");
     static_assert(!kCrc || (STAGE_BYTES % (NT * 32) == 0 && (NT * 256) % STAGE_BYTES == 0), "stage/step mismatch");
     static_assert(STAGE_BYTES % 128 == 0, "stage alignment");
@@ -330,6 +333,7 @@ struct StreamParams {
     uint32_t commit_reverse;  // 1: the commit side walks the pages of a job from the last to the first
     uint32_t l2_hints;        // bit 0: verify loads evict_last; bit 1: commit loads evict_first
     uint32_t test_drop_from;  // tests only: k > 0 makes the fused kernel verify nothing of jobs k-1, k, ...
+    unsigned long long *trace;  // builds with GK_TRACE: time stamps of the first item of every role, else null
     uint8_t *mask_out;        // commit
     int32_t *first_bad_out;   // commit
 };
@@ -343,6 +347,10 @@ struct Ring {
     uint32_t full0, empty0;
     uint2 *tag;   // per stage: (item slot, tile index within the item), or the end mark
     Item *items;  // [STAGES + 1]
+    // CRC rings: hand-over of a reduced segment from the consumer warps to the finisher warp
+    // (see finisher_role).  Two hand-over slots, used in turn.
+    uint64_t *red;   // [2][kHandOverWords]
+    uint32_t tail0;  // four barriers: slot 0 posted, slot 1 posted, slot 0 taken, slot 1 taken
 };
 
 __device__ __forceinline__ uint32_t ld_acquire_u32(const uint32_t *p)
@@ -372,6 +380,12 @@ __device__ __forceinline__ uint32_t atom_add_acq_rel_u32(uint32_t *p, uint32_t v
     uint32_t old;
     asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
     return old;
+}
+
+// As above without the returned value: the thread does not wait for the memory system.
+__device__ __forceinline__ void red_add_release_u32(uint32_t *p, uint32_t v)
+{
+    asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
 __device__ __forceinline__ void fence_sc_gpu()
@@ -409,12 +423,31 @@ __device__ __forceinline__ bool wait_job_verified(const StreamParams &P, uint32_
 // The commit decision of a job is taken ONCE, by whichever commit loader meets
 // the job first: it waits (fused kernel) until the job has been verified, works
 // out the result code, and publishes it in job_latch[j] with a compare-and-swap;
-// the winner also writes the job's report.  Every other commit item of the job,
-// in any CTA, reads the latched code, so a job is committed whole or not at all
-// even if a wait runs out somewhere else in the meantime.  Lane 0 decides, the
-// warp gets the code.
+// the winner also writes the job's report (write_report, which it may put off
+// until it has issued the copies of its own item).  Every other commit item of
+// the job, in any CTA, reads the latched code, so a job is committed whole or
+// not at all even if a wait runs out somewhere else in the meantime.  Lane 0
+// decides, the warp gets the code.
+struct Report {
+    uint32_t pending = 0u;  // lane 0: this loader took the decision and still owes the report
+    uint32_t j = 0u, code = 0u;
+    int32_t first_bad = -1;
+};
+
+__device__ __forceinline__ void write_report(const StreamParams &P, Report &rep)
+{
+    if (!rep.pending) return;
+    rep.pending = 0u;
+    if (!P.mask_out) return;
+    P.mask_out[rep.j] = (uint8_t)rep.code;
+    P.first_bad_out[rep.j] = rep.first_bad;
+    // a CTA that had to give up on one of this job's items may have changed the verdict meanwhile
+    fence_sc_gpu();
+    if (ld_acquire_u32(P.w.job_latch + rep.j) != rep.code) P.mask_out[rep.j] = 4u;
+}
+
 __device__ __forceinline__ uint32_t commit_decision(const StreamParams &P, uint32_t j, const JobDev &jb,
-                                                    volatile uint32_t *abort_flag, int lane)
+                                                    volatile uint32_t *abort_flag, int lane, Report &rep)
 {
     uint32_t code = 0u;
     if (lane == 0) {
@@ -428,12 +461,12 @@ __device__ __forceinline__ uint32_t commit_decision(const StreamParams &P, uint3
             const uint32_t old = atomicCAS(P.w.job_latch + j, kUndecided, code);
             if (old != kUndecided) {
                 code = old;
-            } else if (P.mask_out) {
-                P.mask_out[j] = (uint8_t)code;
-                P.first_bad_out[j] = fb;
-                // a CTA that had to give up on one of this job's items may have changed the verdict meanwhile
-                fence_sc_gpu();
-                if (ld_acquire_u32(P.w.job_latch + j) != code) P.mask_out[j] = 4u;
+            } else {
+                write_report(P, rep);  // at most one report is owed at a time
+                rep.pending = 1u;
+                rep.j = j;
+                rep.code = code;
+                rep.first_bad = fb;
             }
         }
     }
@@ -451,11 +484,24 @@ __device__ __forceinline__ void revoke_job(const StreamParams &P, uint32_t j)
     if (P.mask_out) P.mask_out[j] = 4u;
 }
 
-// Geometry of work item `item` of a launch (no decision is taken here).
-// Returns false if the item does not exist (a short last page has fewer segments).
+// Tiles of segment q of a page record with shape sh.  Returns false if the page
+// has no such segment (a short last page has fewer).
+__device__ __forceinline__ bool segment_tiles(const PageShape &sh, const Tiling &tl, uint32_t q, Item &it)
+{
+    it.nseg = sh.nseg;
+    if (q >= sh.nseg) return false;
+    it.q = q;
+    it.pad = sh.pad;
+    it.t = sh.t;
+    it.tile_begin = q == 0u ? 0u : sh.ntiles0 + (q - 1u) * tl.seg_tiles;
+    it.tile_count = q == 0u ? sh.ntiles0 : tl.seg_tiles;
+    return true;
+}
+
+// Geometry of work item `item` of a launch from the tables of the call.  No decision is taken here.
 template <int MODE>
-__device__ __forceinline__ bool item_geometry(const StreamParams &P, const Tiling &tl, uint32_t item,
-                                              const JobDev *&jbp, Item &it)
+__device__ __forceinline__ bool item_from_tables(const StreamParams &P, const Tiling &tl, uint32_t item,
+                                                 const JobDev *&jbp, Item &it)
 {
     const uint32_t local = item / tl.nseg_max;
     uint32_t q = item - local * tl.nseg_max;
@@ -471,41 +517,53 @@ __device__ __forceinline__ bool item_geometry(const StreamParams &P, const Tilin
     }
     it.gp = gp;
     const PageShape sh = page_shape(P.g, jb, it.p, tl);
-    it.nseg = sh.nseg;
-    if (q >= sh.nseg) return false;
-    if (MODE == kCommit && P.commit_reverse) q = sh.nseg - 1u - q;
-    it.q = q;
-    it.pad = sh.pad;
-    it.t = sh.t;
-    it.tile_begin = q == 0u ? 0u : sh.ntiles0 + (q - 1u) * tl.seg_tiles;
-    it.tile_count = q == 0u ? sh.ntiles0 : tl.seg_tiles;
+    if (MODE == kCommit && P.commit_reverse && q < sh.nseg) q = sh.nseg - 1u - q;
     it.rec = jb.blob + (uint64_t)it.p * P.g.R;
     it.sum = jb.checksums + it.p;
     it.phys = 0;
-    return true;
+    return segment_tiles(sh, tl, q, it);
 }
+
+// The last job this commit loader asked about: consecutive items mostly belong to
+// one job, whose latched decision need not be fetched again.
+struct JobCache {
+    uint32_t j = kUndecided, code = kUndecided;
+};
 
 // Loader only: geometry plus the decision whether the item is to be processed.
 template <int MODE>
 __device__ __forceinline__ bool admit_item(const StreamParams &P, const Tiling &tl, uint32_t item, Item &it,
-                                           volatile uint32_t *abort_flag, int lane)
+                                           volatile uint32_t *abort_flag, int lane, Report &rep, JobCache &jc)
 {
-    const JobDev *jbp;
-    const bool exists = item_geometry<MODE>(P, tl, item, jbp, it);
+    const JobDev *jbp = nullptr;
+    const bool exists = item_from_tables<MODE>(P, tl, item, jbp, it);
+    const bool skip = jbp->missing || P.w.bad_range[it.j] != kNoPage ||
+                      ((MODE == kVerify || MODE == kSingle) && P.w.bad_dup[it.j] != kNoPage);
+    // the table entry does not depend on the decision: have it on its way while the decision is awaited
+    if (MODE != kVerify && exists && !skip) it.phys = jbp->page_table[it.p];
     if (MODE == kCommit) {
-        // every item asks, existing or not, so that a job whose pages all fail to exist cannot occur
-        const uint32_t code = commit_decision(P, it.j, *jbp, abort_flag, lane);
-        if (code != 0u || !exists) return false;
-        if (*abort_flag) {
+        // every item asks, existing or not, so that every job of the launch gets its report
+        uint32_t code;
+        if (jc.j == it.j && jc.code != kUndecided) {
+            code = jc.code;
+        } else {
+            code = commit_decision(P, it.j, *jbp, abort_flag, lane, rep);
+            jc.j = it.j;
+            jc.code = code;
+        }
+        bool take = code == 0u && exists;
+        if (take && *abort_flag) {
             if (lane == 0) revoke_job(P, it.j);
+            take = false;
+        }
+        if (!take) {
+            if (lane == 0) write_report(P, rep);
             return false;
         }
     } else {
-        if (!exists || jbp->missing || P.w.bad_range[it.j] != kNoPage) return false;
-        if ((MODE == kVerify || MODE == kSingle) && P.w.bad_dup[it.j] != kNoPage) return false;
+        if (!exists || skip) return false;
         if (MODE == kVerify && P.test_drop_from != 0u && it.j + 1u >= P.test_drop_from) return false;
     }
-    if (MODE != kVerify) it.phys = jbp->page_table[it.p];
     return true;
 }
 
@@ -648,16 +706,18 @@ template <> struct FrobExp<64> { static constexpr int e = 11; };
 template <> struct FrobExp<128> { static constexpr int e = 12; };
 template <> struct FrobExp<256> { static constexpr int e = 13; };
 
-// Remainder of one thread's 32 streams, already placed at the thread's distance
-// from the end of the segment and multiplied by x^64:
-//   x^(32*(NT-1-t)+64) * sum_s x^(31-s) * (R_s)^(32*NT)   mod P
+// The 32 streams of one thread as ONE unreduced polynomial,
+//   sum_s x^(31-s) * (R_s)^(32*NT)   (degree < 95),
+// in three 32-bit words: a0 = degrees 0..31, a1 = 32..63, a2 = 64..94.
 template <int NT>
-__device__ __forceinline__ uint64_t thread_remainder(const uint32_t (&R)[64], uint64_t kt)
+__device__ __forceinline__ void thread_poly(const uint32_t (&R)[64], uint32_t &a0, uint32_t &a1, uint32_t &a2)
 {
     uint32_t Q[64];
     gk_frob<FrobExp<NT>::e>(R, Q);
-    // sum_s x^(31-s) * Q_s: bit s of Q[k] is the coefficient of x^(k+31-s)
-    uint32_t a0 = 0u, a1 = 0u, a2 = 0u;
+    // bit s of Q[k] is the coefficient of x^(k+31-s)
+    a0 = 0u;
+    a1 = 0u;
+    a2 = 0u;
 #pragma unroll
     for (int k = 0; k < 64; ++k) {
         const uint32_t v = __brev(Q[k]);
@@ -672,17 +732,47 @@ __device__ __forceinline__ uint64_t thread_remainder(const uint32_t (&R)[64], ui
             a2 ^= hi;
         }
     }
-    // fold degrees 64..94 back
-    uint64_t lo64 = ((uint64_t)a1 << 32) | a0;
-    uint32_t hi = a2;
+}
+
+// w(x) * c(x) mod P for a 32-bit w: Horner over the bits of w, 32 steps of
+// "times x, fold, add c if the bit is set" on a 64-bit value in two registers.
+__device__ __forceinline__ uint64_t gf_mul32(uint32_t w, uint64_t c)
+{
+    const uint32_t cl = (uint32_t)c, ch = (uint32_t)(c >> 32);
+    constexpr uint32_t pl = (uint32_t)kPoly, ph = (uint32_t)(kPoly >> 32);
+    uint32_t rl = 0u, rh = 0u;
 #pragma unroll
-    for (int b = 30; b >= 0; --b) {
-        if ((hi >> b) & 1u) {
-            lo64 ^= kPoly << b;
-            if (b) hi ^= (uint32_t)(kPoly >> (64 - b));
-        }
+    for (int i = 31; i >= 0; --i) {
+        const uint32_t m = (uint32_t)((int32_t)rh >> 31);
+        rh = __funnelshift_l(rl, rh, 1);
+        rl <<= 1;
+        const uint32_t b = (uint32_t)((int32_t)(w << (31 - i)) >> 31);
+        rl ^= (m & pl) ^ (b & cl);
+        rh ^= (m & ph) ^ (b & ch);
     }
-    return gf_mul(kt, lo64);
+    return ((uint64_t)rh << 32) | rl;
+}
+
+// Threads -> CTA.  Thread t's polynomial sits 32 bits above thread t+1's, so the
+// words of neighbouring threads overlap: inside a warp the three words that fall
+// on one 32-bit slot are XORed across lanes, which leaves every lane ONE word to
+// multiply by its constant kt = x^(32*(NT-1-t)+64) (32 steps instead of the 95 a
+// whole polynomial would take), and two words that stick out above the warp's
+// first lane (returned to lane 0 in over0, over1: slots 32 and 33 of the warp).
+// Returns the XOR over the warp of the lanes' products (valid in every lane).
+__device__ __forceinline__ uint64_t warp_remainder(uint32_t a0, uint32_t a1, uint32_t a2, uint64_t kt, int lane,
+                                                   uint32_t &over0, uint32_t &over1)
+{
+    const uint32_t a1n = __shfl_down_sync(0xffffffffu, a1, 1);   // a1 of lane + 1
+    const uint32_t a2n = __shfl_down_sync(0xffffffffu, a2, 1);   // a2 of lane + 1
+    const uint32_t a2nn = __shfl_down_sync(0xffffffffu, a2, 2);  // a2 of lane + 2
+    const uint32_t word = a0 ^ (lane < 31 ? a1n : 0u) ^ (lane < 30 ? a2nn : 0u);
+    over0 = a1 ^ a2n;  // meaningful in lane 0 only
+    over1 = a2;
+    uint64_t v = gf_mul32(word, kt);
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v ^= __shfl_xor_sync(0xffffffffu, v, d);
+    return v;
 }
 
 // Ring position of a pipeline role: stage index and the parity of its use count.
@@ -741,6 +831,23 @@ struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES> {
 constexpr uint32_t kEndOfWork = 0xffffffffu;
 constexpr uint32_t kNoJob = 0xffffffffu;
 
+// Developer aid, compiled in with -DGK_TRACE only: every role of every CTA leaves the
+// %globaltimer value of its first pass through a few marked places in P.trace
+// ([CTA][role 0..3][event 0..15]; roles: verify/pack loader, commit loader, consumer, storer).
+#ifdef GK_TRACE
+#define GK_TRACE_EVT(P, role, ev)                                                                     \
+    do {                                                                                              \
+        if ((P).trace && (threadIdx.x & 31) == 0) {                                                   \
+            unsigned long long *slot_ = (P).trace + ((size_t)blockIdx.x * 4 + (role)) * 16 + (ev);     \
+            if (*slot_ == 0ull) *slot_ = global_timer_ns();                                           \
+        }                                                                                             \
+    } while (0)
+#else
+#define GK_TRACE_EVT(P, role, ev) \
+    do {                          \
+    } while (0)
+#endif
+
 template <bool STATIC_FIRST>
 __device__ __forceinline__ uint32_t next_item(uint32_t *ctr, uint32_t base, int lane)
 {
@@ -760,12 +867,176 @@ __device__ __forceinline__ void revoke_in_flight(const StreamParams &P, const Ri
     }
 }
 
+// ----------------------------- finisher role -----------------------------
+// The kernels that verify have a warp for it; in the kernels that pack, whose
+// consumers need the registers a further warp would take, consumer warp 0 does
+// it after its own part of the segment.  Takes what the consumer warps
+// hand over at the end of a segment and finishes it: adds the words that stick
+// out above each warp (times their constants) to the warps' partial remainders,
+// places the segment inside its page and XORs it into the page's accumulator.
+// Where pages are finalized inline, the CTA that delivers the last segment of a
+// page also finishes the page -- final xor, reflection, then write the checksum
+// (pack) or compare it with the stored one and count the page in job_done, which
+// the commit side of the fused kernel waits on.  Neither the consumers nor the
+// loader are held up by any of this (the round trips to memory in particular).
+//
+// Hand-over slot (two of them, used in turn), 12 x 8 bytes: [0..3] the consumer
+// warps' partial remainders, [4..7] as 32-bit words the two words above each
+// warp, [8..11] a copy of what the finisher needs to know about the item.
+struct HandOver {
+    uint64_t *sum;
+    uint32_t gp, j, p, q, nseg, t;
+};
+constexpr int kHandOverWords = 12;
+
+struct Finisher {
+    uint32_t done = 0;   // segments finished so far
+    uint64_t kover = 0;  // lanes 0 .. 2*NT/32-1: constants of the words above the warps
+};
+
+template <int NT>
+__device__ __forceinline__ void finisher_init(const StreamParams &P, Finisher &fin, int lane)
+{
+    if (NT > 0 && lane < 2 * (NT / 32)) fin.kover = P.w.thread_const[NT + lane];
+}
+
+// Has the next segment been handed over?  (Every lane may ask; use finisher_ready for a warp-wide answer.)
+__device__ __forceinline__ bool finisher_posted(const Ring &ring, const Finisher &fin)
+{
+    return mbar_test_wait(ring.tail0 + 8u * (fin.done & 1u), (fin.done >> 1) & 1u);
+}
+
+__device__ __forceinline__ bool finisher_ready(const Ring &ring, const Finisher &fin)
+{
+    return __shfl_sync(0xffffffffu, finisher_posted(ring, fin) ? 1 : 0, 0) != 0;
+}
+
+// Finishes the segment in hand-over slot fin.done & 1 (the whole warp takes part).  `taken` is
+// the barrier to arrive on once the slot has been read, or 0.
+template <int MODE, int NT>
+__device__ __forceinline__ void finish_segment(const StreamParams &P, const Ring &ring, Finisher &fin,
+                                               const HandOver &it, uint32_t taken, volatile uint32_t *abort_flag,
+                                               int lane)
+{
+    constexpr int kW = NT / 32;
+    const uint32_t par = fin.done & 1u;
+    const uint64_t *slot = ring.red + kHandOverWords * par;
+    const uint32_t *oslot = reinterpret_cast<const uint32_t *>(slot + 4);
+    const uint32_t nseg = it.nseg;
+    // the factors that place the two halves of the remainder inside the page: loads first, arithmetic below
+    uint64_t kplace = 0ull;
+    if (nseg > 1u && lane < 2) kplace = P.w.seg_pow[2u * (nseg - 1u - it.q) + lane];
+    uint64_t tot = 0;
+    if (lane < 2 * kW) tot = gf_mul32(oslot[lane], fin.kover);
+    if (lane < kW) tot ^= slot[lane];
+    __syncwarp();
+    if (taken != 0u && lane == 0) mbar_arrive(taken);  // the slot has been read: it may be used again
+#pragma unroll
+    for (int d = 4; d > 0; d >>= 1) tot ^= __shfl_xor_sync(0xffffffffu, tot, d);
+    // place the segment: the short segment comes first and all others are full, so (nseg - 1 - q)
+    // full segments follow this one
+    if (nseg > 1u) {
+        tot = __shfl_sync(0xffffffffu, tot, 0);
+        uint64_t part = 0;
+        if (lane < 2) part = gf_mul32(lane == 0 ? (uint32_t)tot : (uint32_t)(tot >> 32), kplace);
+        tot = part ^ __shfl_xor_sync(0xffffffffu, part, 1);
+    }
+    if (lane == 0) {
+        uint64_t *acc = P.w.page_acc + it.gp;
+        if (!P.inline_final) {
+            red_xor_u64(acc, tot);
+        } else {
+            uint64_t stored = 0;
+            if (MODE != kPack) stored = *it.sum;  // in flight together with the two atomics below
+            uint64_t r = tot;
+            bool last = true;
+            if (nseg > 1u) {
+                red_xor_u64(acc, tot);
+                last = atom_add_acq_rel_u32(&P.w.page_cnt[it.gp], 1u) + 1u == nseg;
+                if (last) r = ld_acquire_u64(acc);
+            }
+            if (last) {
+                const uint64_t crc = __brevll(r ^ P.w.init_term[it.t] ^ ~0ull);
+                if (MODE == kPack) {
+                    *it.sum = crc;
+                } else {
+                    if (crc != stored || *abort_flag) atomicMin(&P.w.bad_crc[it.j], (int32_t)it.p);
+                    red_add_release_u32(&P.w.job_done[it.j], 1u);  // nobody here waits for the count
+                }
+            }
+        }
+    }
+    __syncwarp();
+    ++fin.done;
+    GK_TRACE_EVT(P, 2, 3);
+}
+
+__device__ __forceinline__ HandOver hand_over_of(const Item &it)
+{
+    HandOver h;
+    h.sum = it.sum;
+    h.gp = it.gp;
+    h.j = it.j;
+    h.p = it.p;
+    h.q = it.q;
+    h.nseg = it.nseg;
+    h.t = it.t;
+    return h;
+}
+
+// Finishes segments until the loader's count of admitted items has been reached (the count is
+// known once the loader has put the end mark into the ring).
+template <int MODE, int NT>
+__device__ __forceinline__ void finisher_drain(const StreamParams &P, const Ring &ring, Finisher &fin,
+                                               volatile uint32_t *abort_flag, int lane)
+{
+    volatile uint32_t *n_final = abort_flag + 2;
+    for (;;) {
+        bool posted = finisher_posted(ring, fin);
+        if (!posted) {
+            const unsigned long long t0 = global_timer_ns();
+            uint32_t spins = 0;
+            for (;;) {
+                if (finisher_posted(ring, fin)) {
+                    posted = true;
+                    break;
+                }
+                if (*n_final == fin.done) break;
+                __nanosleep(64);
+                if ((++spins & 0xffu) == 0u) {
+                    // the consumers' own waits are bounded; this one only has to outlast them
+                    if (global_timer_ns() - t0 > 4ull * P.w.wait_limit_ns) {
+                        *abort_flag = 1u;
+                        atomicCAS(P.w.error, 0u, 0x700u | MODE);
+                        break;
+                    }
+                }
+            }
+        }
+        posted = __shfl_sync(0xffffffffu, posted ? 1 : 0, 0) != 0;  // one decision for the warp
+        if (!posted) break;
+        const uint32_t par = fin.done & 1u;
+        const HandOver it = *reinterpret_cast<const HandOver *>(ring.red + kHandOverWords * par + 8);
+        finish_segment<MODE, NT>(P, ring, fin, it, ring.tail0 + 8u * (2u + par), abort_flag, lane);
+    }
+}
+
+// The role as a warp of its own (kernels whose storer warp, if any, has no time for it).
+template <int MODE, int NT>
+__device__ __forceinline__ void finisher_role(const StreamParams &P, const Ring &ring, volatile uint32_t *abort_flag,
+                                              int lane)
+{
+    Finisher fin;
+    finisher_init<NT>(P, fin, lane);
+    finisher_drain<MODE, NT>(P, ring, fin, abort_flag, lane);
+}
+
 // ------------------------------ loader role ------------------------------
 // One warp.  Draws work items, decides whether each is to be processed, walks it
 // tile by tile, waits for a free stage and fills it: front padding zeroed by the
 // lanes (CRC modes), scale values gathered by the lanes (pack), everything else
 // by bulk async copies issued by lane 0 that complete on the stage's full barrier.
-template <int MODE, int STAGE_BYTES, int STAGES, bool ZERO_PAD, bool STATIC_FIRST>
+template <int MODE, int NT, int STAGE_BYTES, int STAGES, bool ZERO_PAD, bool STATIC_FIRST>
 __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling &tl, uint32_t n_items, uint32_t *ctr,
                                             uint32_t ctr_base, const Ring &ring, volatile uint32_t *abort_flag,
                                             int lane)
@@ -773,15 +1044,23 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
     uint32_t n = 0;       // tiles issued
     uint32_t n_adm = 0;   // items admitted
     bool revoked = false;
+    Report rep;
+    JobCache jc;
     uint64_t policy = 0;
     const bool hint = (MODE == kVerify && (P.l2_hints & 1u)) || (MODE == kCommit && (P.l2_hints & 2u));
     if (hint) policy = (MODE == kVerify) ? policy_evict_last() : policy_evict_first();
+    GK_TRACE_EVT(P, MODE == kCommit ? 1 : 0, 1);
     for (uint32_t item = STATIC_FIRST ? blockIdx.x : next_item<false>(ctr, ctr_base, lane); item < n_items;
          item = next_item<STATIC_FIRST>(ctr, ctr_base, lane)) {
         Item it;
-        if (!admit_item<MODE>(P, tl, item, it, abort_flag, lane)) continue;
+        if (!admit_item<MODE>(P, tl, item, it, abort_flag, lane, rep, jc)) continue;
+        GK_TRACE_EVT(P, MODE == kCommit ? 1 : 0, 2);
         const uint32_t slot = n_adm % (uint32_t)(STAGES + 1);
         ++n_adm;
+#ifdef GK_TRACE
+        if (n_adm == 16u) GK_TRACE_EVT(P, MODE == kCommit ? 1 : 0, 6);
+        if (n_adm == 48u) GK_TRACE_EVT(P, MODE == kCommit ? 1 : 0, 7);
+#endif
         const Chunks ch = chunks_of(P.g, it.t);
         for (uint32_t k = 0; k < it.tile_count; ++k, ++n) {
             const uint32_t s = n % STAGES;
@@ -865,6 +1144,8 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
             }
             __syncwarp();
         }
+        if (MODE == kCommit && lane == 0) write_report(P, rep);  // the item's copies are on their way
+        GK_TRACE_EVT(P, MODE == kCommit ? 1 : 0, 3);
     }
     // tell the other roles of this CTA that there is no more work
     {
@@ -875,9 +1156,11 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
         if (lane == 0) {
             ring.tag[s] = make_uint2(kEndOfWork, 0u);
             mbar_arrive(ring.full0 + 8u * s);
+            if (NT > 0) abort_flag[2] = n_adm;  // tells the finisher warp how many segments there are
         }
         ++n;
     }
+    GK_TRACE_EVT(P, MODE == kCommit ? 1 : 0, 4);
     // before leaving: every load this CTA issued must have landed
     if (lane == 0) {
         for (uint32_t back = 0; back < (uint32_t)STAGES && back < n; ++back) {
@@ -913,6 +1196,7 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
         }
         const uint2 tag = ring.tag[s];
         if (tag.x == kEndOfWork) break;
+        GK_TRACE_EVT(P, 3, 0);
         const Item &it = ring.items[tag.x];
         const int32_t phys = it.phys;
         const Chunks ch = chunks_of(P.g, it.t);
@@ -962,6 +1246,7 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
                 }
             }
             bulk_commit();
+            GK_TRACE_EVT(P, 3, 1);
             if (n > 0u) {
                 bulk_wait_read<1>();
                 mbar_arrive(ring.empty0 + 8u * ((n - 1u) % STAGES));
@@ -973,24 +1258,32 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
         bulk_wait_all();
         if (n > 0u) mbar_arrive(ring.empty0 + 8u * ((n - 1u) % STAGES));
     }
+    GK_TRACE_EVT(P, 3, 2);
 }
 
 // ----------------------------- consumer role -----------------------------
-// NT threads.  Reduce each segment to its remainder (see the top of this file),
-// place it inside its page and XOR it into the page's accumulator.  Where pages
-// are finalized inline, the CTA that delivers the last segment of a page also
-// finishes it -- final xor, reflection, then write the checksum (pack) or compare
-// it with the stored one and count the page in job_done, which the commit side
-// of the fused kernel waits on.
-template <int MODE, int NT, int STAGE_BYTES, int STAGES>
-__device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring &ring, uint64_t *red,
+// NT threads.  Reduce each segment to one partial remainder per warp (see the
+// top of this file) and hand these over to the loader warp of the ring, which
+// finishes the segment (finish_segment) while the consumers start on the next.
+template <int MODE, int NT, int STAGE_BYTES, int STAGES, bool OWN_FINISHER>
+__device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring &ring,
                                               volatile uint32_t *abort_flag, int tid, int warp, int lane)
 {
     const uint64_t kt = P.w.thread_const[tid];
+    Finisher fin;  // kernels without a finisher warp: consumer warp 0 finishes the segments itself
+    if (!OWN_FINISHER && warp == 0) finisher_init<NT>(P, fin, lane);
     RingPos pos;
     uint32_t parity_red = 0;
+    uint32_t n_done = 0;  // segments handed over so far
+#ifdef GK_TRACE
+    uint32_t trace_items = 0;
+    unsigned long long tr_sum[4] = {0, 0, 0, 0}, tr_t0 = 0, tr_t1 = 0, tr_t2 = 0, tr_t3 = 0;
+#endif
     constexpr int kTilesPerGran = (NT * 256) / STAGE_BYTES;
     for (;;) {
+#ifdef GK_TRACE
+        tr_t0 = global_timer_ns();
+#endif
         // the first tile of the next item (or the end mark) says what comes next
         const bool ok = mbar_wait(ring.full0 + 8u * pos.stage, pos.phase, abort_flag, P.w.error, 0x400u | MODE,
                                   P.w.wait_limit_ns);
@@ -1007,6 +1300,10 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
         if (any_failed) break;
         const uint32_t slot = ring.tag[pos.stage].x;
         if (slot == kEndOfWork) break;
+        GK_TRACE_EVT(P, 2, 0);
+#ifdef GK_TRACE
+        tr_t1 = global_timer_ns();
+#endif
         const uint32_t ngran = ring.items[slot].tile_count / kTilesPerGran;
         uint32_t R[64];
 #pragma unroll
@@ -1014,56 +1311,84 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
         for (uint32_t gi = 0; gi < ngran; ++gi)
             GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, ring.base, ring.full0, ring.empty0, pos, abort_flag,
                                                                 P.w.error, P.w.wait_limit_ns, tid, lane);
+        GK_TRACE_EVT(P, 2, 1);
+#ifdef GK_TRACE
+        tr_t2 = global_timer_ns();
+#endif
         // merge streams -> thread -> warp -> CTA
-        uint64_t v = thread_remainder<NT>(R, kt);
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) v ^= __shfl_xor_sync(0xffffffffu, v, d);
-        uint64_t *rslot = red + 8 * parity_red;
-        if (lane == 0) rslot[warp] = v;
-        asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
-        if (tid == 0) {
-            const Item &it = ring.items[slot];  // still this item's: see Ring
-            uint64_t tot = 0;
-#pragma unroll
-            for (int i = 0; i < NT / 32; ++i) tot ^= rslot[i];
-            // place the segment: the short segment comes first and all others are full, so
-            // (nseg - 1 - q) full segments follow this one
-            const uint32_t nseg = it.nseg;
-            if (nseg > 1u) tot = gf_mul(tot, P.w.seg_pow[nseg - 1u - it.q]);
-            uint64_t *acc = P.w.page_acc + it.gp;
-            if (!P.inline_final) {
-                red_xor_u64(acc, tot);
-            } else {
-                uint64_t stored = 0;
-                if (MODE != kPack) stored = *it.sum;  // in flight together with the two atomics below
-                uint64_t r = tot;
-                bool last = true;
-                if (nseg > 1u) {
-                    red_xor_u64(acc, tot);
-                    last = atom_add_acq_rel_u32(&P.w.page_cnt[it.gp], 1u) + 1u == nseg;
-                    if (last) r = ld_acquire_u64(acc);
-                }
-                if (last) {
-                    const uint64_t crc = __brevll(r ^ P.w.init_term[it.t] ^ ~0ull);
-                    if (MODE == kPack) {
-                        *it.sum = crc;
-                    } else {
-                        if (crc != stored || *abort_flag) atomicMin(&P.w.bad_crc[it.j], (int32_t)it.p);
-                        atom_add_acq_rel_u32(&P.w.job_done[it.j], 1u);
-                    }
-                }
+        uint32_t a0, a1, a2, over0, over1;
+        thread_poly<NT>(R, a0, a1, a2);
+        const uint64_t v = warp_remainder(a0, a1, a2, kt, lane, over0, over1);
+        uint64_t *rslot = ring.red + kHandOverWords * parity_red;
+        uint32_t *oslot = reinterpret_cast<uint32_t *>(rslot + 4);  // [2 * NT / 32] words sticking out above the warps
+        if (OWN_FINISHER) {
+            // hand the segment over to the finisher warp and go on with the next one
+            if (n_done >= 2u)  // the slot's previous segment must have been taken
+                mbar_wait(ring.tail0 + 8u * (2u + parity_red), ((n_done >> 1) - 1u) & 1u, abort_flag, P.w.error,
+                          0x600u | MODE, P.w.wait_limit_ns);
+            if (lane == 0) {
+                rslot[warp] = v;
+                oslot[2 * warp] = over0;
+                oslot[2 * warp + 1] = over1;
+                // what the finisher needs to know about the item (its slot in the ring may be gone by then)
+                if (warp == 0) *reinterpret_cast<HandOver *>(rslot + 8) = hand_over_of(ring.items[slot]);
+                mbar_arrive(ring.tail0 + 8u * parity_red);
+            }
+            GK_TRACE_EVT(P, 2, 2);
+        } else {
+            // no finisher warp in this kernel: warp 0 finishes the segment once all warps have left their
+            // parts; the others go on (the two slots alternate, and the barrier of the next segment keeps
+            // them from getting two segments ahead of warp 0)
+            if (lane == 0) {
+                rslot[warp] = v;
+                oslot[2 * warp] = over0;
+                oslot[2 * warp + 1] = over1;
+            }
+            asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
+            GK_TRACE_EVT(P, 2, 2);
+            if (warp == 0) finish_segment<MODE, NT>(P, ring, fin, hand_over_of(ring.items[slot]), 0u, abort_flag, lane);
+        }
+#ifdef GK_TRACE
+        tr_t3 = global_timer_ns();
+#endif
+#ifdef GK_TRACE
+        {
+            // steady state: when this CTA's 16th and 48th item were finished, and where the time between went
+            if (++trace_items == 16u) GK_TRACE_EVT(P, 2, 5);
+            if (trace_items > 16u && trace_items <= 48u) {
+                const unsigned long long now = global_timer_ns();
+                tr_sum[0] += tr_t1 - tr_t0;  // waiting for the item's first tile
+                tr_sum[1] += tr_t2 - tr_t1;  // main loop
+                tr_sum[2] += tr_t3 - tr_t2;  // epilogue up to the hand-over
+                tr_sum[3] += now - tr_t3;
+            }
+            if (trace_items == 48u) {
+                GK_TRACE_EVT(P, 2, 6);
+                if (P.trace && threadIdx.x == 0)
+                    for (int k = 0; k < 4; ++k) P.trace[((size_t)blockIdx.x * 4 + 2) * 16 + 8 + k] = tr_sum[k] + 1ull;
             }
         }
+#endif
+        ++n_done;
         parity_red ^= 1u;
     }
 }
 
 __device__ __forceinline__ void ring_init(Ring &ring, uint8_t *base, uint64_t *bars, uint2 *tags, Item *items,
-                                          int stages, uint32_t empty_count)
+                                          int stages, uint32_t empty_count, uint64_t *red = nullptr,
+                                          uint64_t *tail_bars = nullptr, uint32_t consumer_warps = 0)
 {
     ring.base = base;
     ring.tag = tags;
     ring.items = items;
+    ring.red = red;
+    ring.tail0 = tail_bars ? smem_u32(tail_bars) : 0u;
+    if (threadIdx.x == 0 && tail_bars) {
+        for (int k = 0; k < 2; ++k) {
+            mbar_init(ring.tail0 + 8u * k, consumer_warps);  // posted: one arrival per consumer warp
+            mbar_init(ring.tail0 + 8u * (2 + k), 1u);        // taken: the loader warp
+        }
+    }
     ring.stage0 = smem_u32(base);
     ring.full0 = smem_u32(bars);
     ring.empty0 = smem_u32(bars + stages);
@@ -1083,36 +1408,44 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
 {
     using Cfg = StreamCfg<MODE, NT, STAGE_BYTES, STAGES>;
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 15) & ~(uintptr_t)15);  // bulk copies need 16 bytes
     uint64_t *bars = (uint64_t *)(smem + (size_t)STAGES * STAGE_BYTES);
-    uint64_t *red = bars + 2 * STAGES;  // [2][8]
-    volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
-    uint2 *tags = (uint2 *)(red + 18);
+    uint64_t *red = bars + 2 * STAGES;                 // [2][kHandOverWords]
+    uint64_t *tail_bars = red + 2 * kHandOverWords;    // [4]
+    volatile uint32_t *abort_flag = (volatile uint32_t *)(tail_bars + 4);
+    uint2 *tags = (uint2 *)(tail_bars + 6);
     Item *items = (Item *)(tags + STAGES);
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
 
     Ring ring;
-    ring_init(ring, smem, bars, tags, items, STAGES, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)));
+    ring_init(ring, smem, bars, tags, items, STAGES, (uint32_t)(Cfg::kConsWarps + (Cfg::kStore ? 1 : 0)), red,
+              Cfg::kOwnFinisher ? tail_bars : nullptr, (uint32_t)Cfg::kConsWarps);
     if (threadIdx.x == 0) {
         abort_flag[0] = 0u;
-        abort_flag[1] = 0u;  // the commit loader's sign of life while it waits for a job
+        abort_flag[1] = 0u;           // the commit loader's sign of life while it waits for a job
+        abort_flag[2] = 0xffffffffu;  // segments of this CTA: not known yet (finisher warp)
         fence_mbar_init();
     }
+    GK_TRACE_EVT(P, 0, 0);
     grid_dependency_wait();  // everything above is CTA-local; the tables of the call are read below
+    GK_TRACE_EVT(P, 0, 5);
     __syncthreads();
 
     if (warp == Cfg::kLoaderWarp) {
         if (MODE == kCommit)
-            loader_role<MODE, STAGE_BYTES, STAGES, false, true>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, ring,
-                                                          abort_flag, lane);
+            loader_role<MODE, 0, STAGE_BYTES, STAGES, false, true>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c,
+                                                                   ring, abort_flag, lane);
         else
-            loader_role<MODE, STAGE_BYTES, STAGES, true, true>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, ring,
-                                                               abort_flag, lane);
+            loader_role<MODE, NT, STAGE_BYTES, STAGES, true, true>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, ring,
+                                                                   abort_flag, lane);
     } else if (Cfg::kStore && warp == Cfg::kStorerWarp) {
         storer_role<MODE, STAGE_BYTES, STAGES>(P, ring, abort_flag, lane);
     } else if constexpr (Cfg::kCrc) {
-        consumer_role<MODE, NT, STAGE_BYTES, STAGES>(P, ring, red, abort_flag, threadIdx.x, warp, lane);
+        if (Cfg::kOwnFinisher && warp == Cfg::kFinisherWarp)
+            finisher_role<MODE, NT>(P, ring, abort_flag, lane);
+        else
+            consumer_role<MODE, NT, STAGE_BYTES, STAGES, Cfg::kOwnFinisher>(P, ring, abort_flag, threadIdx.x, warp, lane);
     }
     __syncthreads();
 }
@@ -1124,23 +1457,24 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
 template <int NT, int VSB, int VST, int CSB, int CST>
 struct RestoreCfg {
     static constexpr int kConsWarps = NT / 32;
-    static constexpr int kThreads = NT + 96;
+    static constexpr int kThreads = NT + 128;
     static constexpr size_t kSmemBytes = (size_t)VST * VSB + (size_t)CST * CSB + 3 * (VST + CST) * 8 +
-                                         (VST + CST + 2) * sizeof(Item) + 2 * 8 * 8 + 16 + 128;
+                                         (VST + CST + 2) * sizeof(Item) + 2 * 12 * 8 + 4 * 8 + 16 + 16;
 };
 
 template <int NT, int VSB, int VST, int CSB, int CST, int MINB>
-__global__ void __launch_bounds__(NT + 96, MINB) restore_kernel(const __grid_constant__ StreamParams P)
+__global__ void __launch_bounds__(NT + 128, MINB) restore_kernel(const __grid_constant__ StreamParams P)
 {
     extern __shared__ uint8_t smem_raw[];
-    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 15) & ~(uintptr_t)15);  // bulk copies need 16 bytes
     uint8_t *vbase = smem;
     uint8_t *cbase = smem + (size_t)VST * VSB;
     uint64_t *vbars = (uint64_t *)(cbase + (size_t)CST * CSB);
     uint64_t *cbars = vbars + 2 * VST;
-    uint64_t *red = cbars + 2 * CST;  // [2][8]
-    volatile uint32_t *abort_flag = (volatile uint32_t *)(red + 16);
-    uint2 *vtags = (uint2 *)(red + 18);
+    uint64_t *red = cbars + 2 * CST;                   // [2][kHandOverWords]
+    uint64_t *tail_bars = red + 2 * kHandOverWords;    // [4]
+    volatile uint32_t *abort_flag = (volatile uint32_t *)(tail_bars + 4);
+    uint2 *vtags = (uint2 *)(tail_bars + 6);
     uint2 *ctags = vtags + VST;
     Item *vitems = (Item *)(ctags + CST);
     Item *citems = vitems + (VST + 1);
@@ -1148,27 +1482,39 @@ __global__ void __launch_bounds__(NT + 96, MINB) restore_kernel(const __grid_con
     const int lane = threadIdx.x & 31;
 
     Ring vring, cring;
-    ring_init(vring, vbase, vbars, vtags, vitems, VST, (uint32_t)(NT / 32));
+    ring_init(vring, vbase, vbars, vtags, vitems, VST, (uint32_t)(NT / 32), red, tail_bars, (uint32_t)(NT / 32));
     ring_init(cring, cbase, cbars, ctags, citems, CST, 1u);
     if (threadIdx.x == 0) {
         abort_flag[0] = 0u;
-        abort_flag[1] = 0u;  // the commit loader's sign of life while it waits for a job
+        abort_flag[1] = 0u;           // the commit loader's sign of life while it waits for a job
+        abort_flag[2] = 0xffffffffu;  // segments of this CTA: not known yet (finisher warp)
         fence_mbar_init();
     }
+    GK_TRACE_EVT(P, 0, 0);
+#ifdef GK_TRACE
+    if (P.trace && threadIdx.x == 0) {
+        uint32_t smid;
+        asm volatile("mov.u32 %0, %%smid;" : "=r"(smid));
+        P.trace[((size_t)blockIdx.x * 4 + 0) * 16 + 15] = smid + 1u;
+    }
+#endif
     grid_dependency_wait();  // everything above is CTA-local; the tables of the call are read below
+    GK_TRACE_EVT(P, 0, 5);
     __syncthreads();
 
     constexpr int kCons = NT / 32;
     if (warp < kCons) {
-        consumer_role<kVerify, NT, VSB, VST>(P, vring, red, abort_flag, threadIdx.x, warp, lane);
+        consumer_role<kVerify, NT, VSB, VST, true>(P, vring, abort_flag, threadIdx.x, warp, lane);
     } else if (warp == kCons) {
-        loader_role<kVerify, VSB, VST, true, false>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, vring, abort_flag,
-                                                    lane);
+        loader_role<kVerify, NT, VSB, VST, true, false>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, vring,
+                                                        abort_flag, lane);
     } else if (warp == kCons + 1) {
-        loader_role<kCommit, CSB, CST, false, true>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, cring,
-                                                    abort_flag, lane);
-    } else {
+        loader_role<kCommit, 0, CSB, CST, false, true>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, cring,
+                                                       abort_flag, lane);
+    } else if (warp == kCons + 2) {
         storer_role<kCommit, CSB, CST>(P, cring, abort_flag, lane);
+    } else {
+        finisher_role<kVerify, NT>(P, vring, abort_flag, lane);
     }
     __syncthreads();
 }

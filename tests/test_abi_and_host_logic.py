@@ -176,6 +176,41 @@ def test_bit_sliced_scheme_reproduces_crc():
     assert crc == oracle.crc64(data)
 
 
+def test_word_slot_merge_of_the_thread_polynomials():
+    """How the kernels merge the threads of a CTA, restated with Python integers.  Every
+    thread holds an UNREDUCED polynomial of up to 95 bits (three 32-bit words a0, a1, a2)
+    that sits 32 bits above its right-hand neighbour's.  Inside a warp the words that fall on
+    the same 32-bit slot are XORed across lanes, so that each lane is left with ONE word to
+    multiply by its constant x^(32*(NT-1-t)+64); the two words that stick out above a warp's
+    first lane are multiplied by two constants of their own.  The sum must equal the plain
+    definition: sum over threads of poly_t * x^(32*(NT-1-t)+64) mod P."""
+    rng = np.random.default_rng(7)
+    for NT, WS in ((8, 4), (16, 4), (12, 2), (128, 32)):
+        NW = NT // WS
+        polys = [int(rng.integers(0, 1 << 62)) | (int(rng.integers(0, 1 << 33)) << 62) for _ in range(NT)]
+        assert max(p.bit_length() for p in polys) <= 95
+        want = 0
+        for t, p in enumerate(polys):
+            want ^= _mod(_clmul(p, 1 << (32 * (NT - 1 - t) + 64)))
+        M = 0xFFFFFFFF
+        a0 = [p & M for p in polys]
+        a1 = [(p >> 32) & M for p in polys]
+        a2 = [p >> 64 for p in polys]
+        got = 0
+        for w in range(NW):
+            def word(arr, lane):
+                return arr[w * WS + lane] if lane < WS else 0
+            for lane in range(WS):
+                t = w * WS + lane
+                slot_word = a0[t] ^ word(a1, lane + 1) ^ word(a2, lane + 2)
+                got ^= _mod(_clmul(slot_word, _mod(1 << (32 * (NT - 1 - t) + 64))))
+            over0 = word(a1, 0) ^ word(a2, 1)
+            over1 = word(a2, 0)
+            got ^= _mod(_clmul(over0, _mod(1 << (32 * WS * (NW - w) + 64))))
+            got ^= _mod(_clmul(over1, _mod(1 << (32 * WS * (NW - w) + 96))))
+        assert got == want, (NT, WS)
+
+
 def test_sha256_round_constants_in_the_kernel_source_match_the_derived_ones():
     """The kernels carry the SHA-256 round constants and initial state as typed literals;
     the oracle derives them from the primes.  Neither reads the other: compare them here."""
