@@ -11,10 +11,13 @@ cache through seeded random-permutation page tables.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
 
-Prints ONE JSON line on rank 0.  `value` counts the KV bytes the step reads plus
-writes (2 x blob bytes for the save, 2 x blob bytes for the restore) per second,
-summed over all GPUs; the restore phase alone, tokens/s and the per-kernel
-roofline are reported beside it.  With N > 1 (launched by torch.distributed.run)
+Prints ONE JSON line on rank 0.  `value` is the metric itself: restored KV GB/s,
+counting the bytes the restore phase of a step must read plus the bytes it must
+write (2 x blob bytes), over the device time of that phase, summed over all
+GPUs; the save phase, the whole step, tokens/s, the per-kernel roofline (against
+the measured copy peak and against the nominal 8,000 GB/s), the other workload
+shapes, lone-block latencies, the host-tier end-to-end leg and the CPU oracle's
+timings are reported beside it.  With N > 1 (launched by torch.distributed.run)
 every rank runs its own batch on its own GPU: the path has no exchange step, so
 this is weak scaling over independent request batches.
 """
@@ -42,6 +45,7 @@ UNIT = "GB/s"
 # (17.18 GB read + 8.56 GB written for 8.59 GB of blobs); the full --set full
 # capture of a 2-block launch gives 2.96.
 RESTORE_DRAM_BYTES_PER_BLOB_BYTE = 25.74 / 8.59
+NOMINAL_HBM_GBS = 8000.0   # the HBM peak the target is stated against
 
 
 def parse_args():
@@ -64,6 +68,7 @@ def parse_args():
     ap.add_argument("--e2e-pipelined-steps", type=int, default=10,
                     help="steps of the pipelined end-to-end leg (save of step k+1 overlaps restore of step k)")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the other workload shapes and the latency cases")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-baseline-blocks", type=int, default=4)
     ap.add_argument("--reference-seconds", type=float, default=100.0,
@@ -266,38 +271,56 @@ def build_workload(args, device, rank):
                 src_pages=src_pages)
 
 
-def oracle_sample(wl, n_blocks, steps, warmup):
-    """Times the CPU oracle (as it stands, single-threaded) on the first n_blocks
-    blocks of the batch: pack from a host copy of the source cache, then restore
-    into a host destination cache.  Returns (seconds per step, bytes per step,
-    tokens per step, checksums of the packed blocks)."""
+def oracle_sample(wl, n_blocks):
+    """Times the CPU oracle, as it stands, on blocks of the batch: pack from a host copy of
+    the source cache, then restore into a host destination cache.  Two legs: one thread over
+    the first n_blocks blocks, and one thread per block over as many blocks as the box has
+    cores (at most the batch), every thread calling the unchanged oracle through ctypes on its
+    own block and its own destination pages.  Returns the times (whole and restore phase
+    alone) of both legs and the oracle's checksums of the sampled blocks."""
     import oracle
+    from concurrent.futures import ThreadPoolExecutor
     w = wl["w"]
     og = oracle.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, w.elem_bytes, 0)
     P, n_tok, slab = wl["P"], wl["n_tok"], wl["slab"]
     src_pages = wl["src_pages"]
     src_host = wl["src"].data.cpu().numpy()
     src = oracle.Cache(src_host, src_pages, 2 * src_pages * slab, src_pages * slab, slab)
-    dpages = n_blocks * P
-    dst = oracle.Cache(np.zeros(2 * w.layers * dpages * slab, dtype=np.uint8), dpages, 2 * dpages * slab,
-                       dpages * slab, slab)
     src_perm = wl["src_perm"].cpu().numpy()
-    dperm = np.random.default_rng(7).permutation(dpages).astype(np.int32)
-    times, sums_out = [], None
-    for it in range(warmup + steps):
-        t0 = time.perf_counter()
-        jobs = []
-        for i in range(n_blocks):
-            blob, sums, code, _ = oracle.pack(og, src, src_perm[i * P:(i + 1) * P], n_tok)
-            assert code == 0
-            jobs.append(oracle.Job(blob, sums, dperm[i * P:(i + 1) * P], n_tok))
-        mask, _ = oracle.restore(og, dst, jobs)
-        dt = time.perf_counter() - t0
+
+    def one_block(i, dst, dperm, slot):
+        t_begin = time.perf_counter()
+        blob, sums, code, _ = oracle.pack(og, src, src_perm[i * P:(i + 1) * P], n_tok)
+        assert code == 0
+        t = time.perf_counter()
+        mask, _ = oracle.restore(og, dst, [oracle.Job(blob, sums, dperm[slot * P:(slot + 1) * P], n_tok)])
         assert not mask.any()
-        if it >= warmup:
-            times.append(dt)
-        sums_out = [j.checksums for j in jobs]
-    return float(np.mean(times)), 4 * n_blocks * wl["blob_bytes"], n_blocks * n_tok, sums_out
+        t_end = time.perf_counter()
+        return sums, t_end - t, t_end - t_begin
+
+    def dst_for(blocks):
+        dpages = blocks * P
+        return (oracle.Cache(np.zeros(2 * w.layers * dpages * slab, dtype=np.uint8), dpages, 2 * dpages * slab,
+                             dpages * slab, slab),
+                np.random.default_rng(7).permutation(dpages).astype(np.int32))
+
+    dst, dperm = dst_for(n_blocks)
+    t0 = time.perf_counter()
+    res = [one_block(i, dst, dperm, i) for i in range(n_blocks)]
+    t_single = time.perf_counter() - t0
+    sums_out = [r[0] for r in res]
+    t_single_restore = sum(r[1] for r in res)
+    del dst
+    threads = max(1, min(os.cpu_count() or 1, wl["n_blocks"]))
+    dst, dperm = dst_for(threads)
+    with ThreadPoolExecutor(max_workers=threads) as pool:
+        t0 = time.perf_counter()
+        res = list(pool.map(lambda i: one_block(i, dst, dperm, i), range(threads)))
+        t_multi = time.perf_counter() - t0
+    # the threads' restore phases overlap one another's save phases: the restore's share of the wall time
+    t_multi_restore = t_multi * sum(r[1] for r in res) / max(sum(r[2] for r in res), 1e-9)
+    return dict(t_single=t_single, t_single_restore=t_single_restore, t_multi=t_multi, t_multi_restore=t_multi_restore,
+                threads=threads, blob_bytes=wl["blob_bytes"], n_tok=n_tok, sums=sums_out)
 
 
 # ---------------------------------------------------------------------------
@@ -332,26 +355,33 @@ def run_reference(args):
             oracle.restore(og, dst, [oracle.Job(blob, sums, dpt, n_tok)])
             per_page = (time.perf_counter() - t0) / N
             pages = int(min(1024, max(8, args.reference_seconds / (per_page * n_iter))))
-    times = []
+    times, rtimes = [], []
     blob_bytes = oracle.blob_size(og, n_tok)[0]
     for it in range(args.warmup + args.steps):
         t0 = time.perf_counter()
         blob, sums, code, _ = oracle.pack(og, src, spt, n_tok)
+        t1 = time.perf_counter()
         mask, _ = oracle.restore(og, dst, [oracle.Job(blob, sums, dpt, n_tok)])
-        dt = time.perf_counter() - t0
+        t2 = time.perf_counter()
         assert code == 0 and not mask.any()
         if it >= args.warmup:
-            times.append(dt)
-    t = float(np.mean(times))
-    value = 4 * blob_bytes / t / 1e9
-    sample = f"one block of {n_tok} tokens ({pages} pages, {blob_bytes / 2**20:.0f} MiB blob) saved and restored per step"
+            times.append(t2 - t0)
+            rtimes.append(t2 - t1)
+    t, tr = float(np.mean(times)), float(np.median(rtimes))
+    value = 2 * blob_bytes / tr / 1e9       # the metric: restored bytes read + written over the restore phase
+    hi = host_info()
+    sample = (f"one block of {n_tok} tokens ({pages} pages, {blob_bytes / 2**20:.0f} MiB blob) saved and restored per "
+              f"step by the CPU oracle, one thread ({hi['cpu_model']}, {hi['nproc']} cores in the box)")
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
             "config": {"workload": "gqa7b (32 layers, 8 KV heads, head_dim 128, bf16, 16-token pages), bounded sample",
-                       "sample": sample},
-            "tokens_per_s": n_tok / t,
-            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+                       "sample": sample,
+                       "value_definition": "restored KV bytes read + written (2 x blob bytes) / time of the restore "
+                                           "phase of a step (median over the timed steps)"},
+            "tokens_per_s": n_tok / tr,
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample,
+                             "nproc": hi["nproc"], "cpu_model": hi["cpu_model"]},
             "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
             "gpu_launches": 0}
     print(json.dumps(line), flush=True)
@@ -419,10 +449,13 @@ def run_ours(args):
     launches = stats["kernels_launched"] - launches0
     assert int(mask.sum().item()) == 0 and int(status.sum().item()) == 0, "a clean block was rejected"
     assert stats["device_wait_expired"] == 0
-    pack_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in phase_events]))
-    restore_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in phase_events]))
+    pack_all = [e[0].elapsed_time(e[1]) for e in phase_events]
+    restore_all = [e[1].elapsed_time(e[2]) for e in phase_events]
+    pack_ms, restore_ms = float(np.median(pack_all)), float(np.median(restore_all))
+    # the slowest rank's restore phase decides the job's rate (weak scaling over independent batches)
+    restore_ms_job = max_over_ranks(restore_ms)
 
-    value = world * 4 * batch_bytes / (step_ms * 1e-3) / 1e9
+    value = world * 2 * batch_bytes / (restore_ms_job * 1e-3) / 1e9
     peak, peak_kind = measured_peak()
 
     def kernel_entry(name, alg_bytes_per_launch):
@@ -432,7 +465,7 @@ def run_ours(args):
         per = ms / n
         ach = alg_bytes_per_launch / (per * 1e-3) / 1e9
         return {"launches": n, "ms_per_launch": per, "algorithmic_bytes_per_launch": alg_bytes_per_launch,
-                "achieved": ach, "unit": "GB/s", "frac": ach / peak}
+                "achieved": ach, "unit": "GB/s", "frac": ach / peak, "frac_of_nominal_8000": ach / NOMINAL_HBM_GBS}
 
     # algorithmic bytes: the fused restore kernel reads every blob byte twice (verify, then
     # commit -- a block may be written only after all of it has verified, and blocks are larger
@@ -446,7 +479,8 @@ def run_ours(args):
         dom = kernels["restore"]
         roofline = {"bound": "hbm", "kernel": "restore_kernel (fused verify + commit: blob -> CRC check -> paged cache)",
                     "achieved": dom["achieved"], "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                    "frac": dom["frac"], "traffic": RESTORE_DRAM_BYTES_PER_BLOB_BYTE * batch_bytes,
+                    "frac": dom["frac"], "frac_of_nominal_8000": dom["achieved"] / NOMINAL_HBM_GBS,
+                    "traffic": RESTORE_DRAM_BYTES_PER_BLOB_BYTE * batch_bytes,
                     "traffic_note": "ncu dram read+write per blob byte of a launch of this workload (one-pass capture), "
                                     "times the blob bytes of the launch",
                     "algorithmic_bytes_per_launch": 3 * batch_bytes, "ms_per_launch": dom["ms_per_launch"],
@@ -457,7 +491,7 @@ def run_ours(args):
         dom = kernels["commit"]
         roofline = {"bound": "hbm", "kernel": "stream_kernel<kCommit> (blob -> paged cache), after stream_kernel<kVerify>",
                     "achieved": dom["achieved"], "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                    "frac": dom["frac"], "traffic": None,
+                    "frac": dom["frac"], "frac_of_nominal_8000": dom["achieved"] / NOMINAL_HBM_GBS, "traffic": None,
                     "algorithmic_bytes_per_launch": 2 * batch_bytes, "ms_per_launch": dom["ms_per_launch"]}
 
     # ---- end to end: the same step with HOST buffers -- gk_pack_host saves the batch into pinned
@@ -598,6 +632,10 @@ def run_ours(args):
         e2e = {"value": world * 4 * batch_bytes / (pipe_ms * 1e-3) / 1e9, "unit": UNIT,
                "h2d_bytes_per_step": link + 2 * n_blocks * 40, "d2h_bytes_per_step": link + n_blocks * 6,
                "ms_per_step": pipe_ms, "steps": pipe_steps,
+               "link_gbs": {"each_direction": link / (pipe_ms * 1e-3) / 1e9,
+                            "note": "bytes that cross the host link per step in one direction / step time; value "
+                                    "counts 2 x blob bytes for the save and 2 x for the restore (read + write), "
+                                    "the link itself carries 1 x out and 1 x in"},
                "tokens_per_s": world * n_blocks * n_tok / (pipe_ms * 1e-3),
                "pipelining": pipe_note,
                "one_step_at_a_time": {"value": world * 4 * batch_bytes / (e2e_ms * 1e-3) / 1e9,
@@ -615,14 +653,39 @@ def run_ours(args):
     cpu_baseline = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         nb = min(args.cpu_baseline_blocks, n_blocks)
-        t, nbytes, ntoks, osums = oracle_sample(wl, nb, steps=1, warmup=0)
+        o = oracle_sample(wl, nb)
         for i in range(nb):   # the pool blobs the GPU packed carry the same checksums
             got = wl["pack_jobs"][i].checksums.cpu().numpy().view(np.uint64)
-            assert np.array_equal(got, osums[i]), "GPU checksums differ from the oracle's"
-        cpu_baseline = {"value": nbytes / t / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-                        "sample": f"save + restore of the first {nb} blocks of the batch ({ntoks} tokens, "
-                                  f"{nb * blob_bytes / 2**30:.1f} GiB of blobs), {t:.1f} s",
-                        "tokens_per_s": ntoks / t}
+            assert np.array_equal(got, o["sums"][i]), "GPU checksums differ from the oracle's"
+        hi = host_info()
+        bb, nt, th = o["blob_bytes"], o["n_tok"], o["threads"]
+        cpu_baseline = {"value": 2 * nb * bb / o["t_single_restore"] / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+                        "sample": f"restore phase of save + restore of the first {nb} blocks of the batch ({nb * nt} "
+                                  f"tokens, {nb * bb / 2**30:.1f} GiB of blobs) by one thread: {o['t_single_restore']:.1f} s "
+                                  f"of {o['t_single']:.1f} s; value = 2 x blob bytes / restore time, as the headline",
+                        "tokens_per_s": nb * nt / o["t_single_restore"],
+                        "save_plus_restore_gbs": 4 * nb * bb / o["t_single"] / 1e9,
+                        "threaded": {"value": 2 * th * bb / o["t_multi_restore"] / 1e9, "unit": UNIT, "cores": th,
+                                     "sample": f"one thread per block over {th} blocks at once, {o['t_multi']:.1f} s for "
+                                               f"save + restore; restore share {o['t_multi_restore']:.1f} s",
+                                     "save_plus_restore_gbs": 4 * th * bb / o["t_multi"] / 1e9,
+                                     "tokens_per_s": th * nt / o["t_multi_restore"]},
+                        "nproc": hi["nproc"], "cpu_model": hi["cpu_model"]}
+
+    # ---- the other workload shapes and the lone-block latencies (one GPU, after the headline's memory is free)
+    workloads, latency = None, None
+    if world == 1 and not args.no_workloads and not args.blocks:
+        wl_keep = {k: wl[k] for k in ("n_blocks", "n_tok", "pool_blocks", "dst_pages")}
+        ctx.close()
+        wl.clear()
+        import gc
+        gc.collect()
+        torch.cuda.empty_cache()
+        wl.update(wl_keep)
+        workloads = {}
+        for name in ("tiny", "corpus", "corpus_host", "fp8", "stress_wave", "stress_wave_one_third_damaged"):
+            workloads[name] = workload_case(name, device, steps=5, warmup=2)
+        latency = latency_cases(device)
 
     if rank == 0:
         line = {
@@ -631,22 +694,29 @@ def run_ours(args):
             "vs_baseline": None, "dtype": "u64", "data": "synthetic",
             "config": {
                 "workload": ("gqa7b: 32 layers, 8 KV heads, head_dim 128, bf16 N(0,0.5), 16-token pages; "
-                             f"{n_blocks} blocks of {n_tok} tokens per step per GPU "
+                             f"{n_blocks} blocks of {wl['n_tok']} tokens per step per GPU "
                              f"({synth_requests(n_blocks)}), pool of {wl['pool_blocks']} blocks, "
                              f"{wl['dst_pages']}-page destination cache, seeded random-permutation page tables"),
                 "step": "gk_pack_batch (save) + gk_restore (validate, verify, commit) of the batch",
-                "value_definition": "(2 x blob bytes saved + 2 x blob bytes restored) / step time, all GPUs",
+                "value_definition": "restored KV bytes read + written (2 x blob bytes of the batch) / device time of "
+                                    "the restore phase of a step (median over the timed steps, slowest GPU), all GPUs",
                 "batch_blob_bytes": batch_bytes, "l2": "inputs larger than L2 (8 GiB per phase vs 126 MB)",
                 "parallelism": f"replicas x{world}, no collective"},
-            "tokens_per_s": world * n_blocks * n_tok / (step_ms * 1e-3),
-            "frac_of_hbm_peak": value / world / peak,
+            "tokens_per_s": world * n_blocks * n_tok / (restore_ms_job * 1e-3),
+            "north_star": {
+                "what": "device-resident restore against the HBM peak, bytes read plus bytes written",
+                "restore_useful_2_bytes_per_byte": fractions(2 * batch_bytes / (restore_ms * 1e-3) / 1e9, peak),
+                "restore_dram_model_3_bytes_per_byte": fractions(3 * batch_bytes / (restore_ms * 1e-3) / 1e9, peak),
+                "note": "a block is written only after all of it has verified and blocks exceed L2, so every blob "
+                        "byte crosses DRAM three times (read to verify, read to commit, written): the DRAM-model "
+                        "rate is the memory system's, the useful rate is two thirds of it"},
             "phases": {
-                "pack": {"ms": pack_ms, "gbs": 2 * batch_bytes / (pack_ms * 1e-3) / 1e9},
-                "restore": {"ms": restore_ms, "gbs_useful": 2 * batch_bytes / (restore_ms * 1e-3) / 1e9,
-                            "gbs_dram_model": 3 * batch_bytes / (restore_ms * 1e-3) / 1e9,
-                            "tokens_per_s": n_blocks * n_tok / (restore_ms * 1e-3),
-                            "frac_of_hbm_peak_dram_model": 3 * batch_bytes / (restore_ms * 1e-3) / 1e9 / peak}},
-            "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline, "e2e": e2e,
+                "save": dict(stats_ms(pack_all), **fractions(2 * batch_bytes / (pack_ms * 1e-3) / 1e9, peak)),
+                "restore": dict(stats_ms(restore_all), tokens_per_s=n_blocks * wl["n_tok"] / (restore_ms * 1e-3)),
+                "whole_step": {"ms_per_step": step_ms,
+                               "gbs_save_plus_restore": world * 4 * batch_bytes / (step_ms * 1e-3) / 1e9}},
+            "roofline": roofline, "kernels": kernels, "workloads": workloads, "latency": latency,
+            "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": launches, "clocks": clocks,
         }
         print(json.dumps(line), flush=True)
@@ -654,39 +724,74 @@ def run_ours(args):
 
 
 # ---------------------------------------------------------------------------
-# the other workload shapes: save + restore phases only
+# the other workload shapes: save and restore phases, with the damage the
+# configuration prescribes, and the mask census
 # ---------------------------------------------------------------------------
-def run_other_workload(args):
-    import torch
-    import synth
-    import paper_2609_39358_b200 as gk
+def host_info():
+    """Cores and CPU model of the box (for the CPU baseline record)."""
+    model = "unknown"
+    try:
+        with open("/proc/cpuinfo") as f:
+            for line in f:
+                if line.lower().startswith("model name"):
+                    model = line.split(":", 1)[1].strip()
+                    break
+    except OSError:
+        pass
+    return {"nproc": os.cpu_count() or 1, "cpu_model": model}
 
-    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
-    torch.cuda.set_device(device)
-    w = synth.WORKLOADS[args.workload]
-    if args.workload == "gqa7b":
-        lens = [synth.GQA7B_BLOCK_TOKENS] * (args.blocks or synth.GQA7B_REQUESTS * synth.GQA7B_BLOCKS_PER_REQUEST)
-        dst_pages = synth.GQA7B_DST_PAGES
-    elif args.workload == "tiny":
-        lens, dst_pages = synth.TINY_BLOCKS, synth.TINY_DST_PAGES
-    elif args.workload == "corpus":
-        lens, dst_pages = synth.CORPUS_BLOCKS, synth.CORPUS_DST_PAGES
-    elif args.workload == "fp8":
-        lens, dst_pages = synth.FP8_BLOCKS, sum(-(-n // w.page_tokens) for n in synth.FP8_BLOCKS) + 100
-    else:   # one wave of the stress mix: the blocks of the first requests that fit a 65,536-page cache
+
+def fractions(gbs, peak):
+    return {"gbs": gbs, "frac_of_measured_peak": gbs / peak, "frac_of_nominal_8000": gbs / NOMINAL_HBM_GBS}
+
+
+def stats_ms(xs):
+    xs = [float(x) for x in xs]
+    return {"median": float(np.median(xs)), "best": float(np.min(xs)), "mean": float(np.mean(xs)), "n": len(xs)}
+
+
+def shape_of(synth, name, blocks=0):
+    """(workload, block lengths, destination pages, block ids or None) of a named case."""
+    if name in ("stress_wave", "stress_wave_one_third_damaged", "stress"):
+        w = synth.STRESS
+        # one wave of the stress mix: the blocks of the first requests that fit a 65,536-page cache
         all_len = synth.stress_block_lengths(w.seed(0))
-        lens, dst_pages, used = [], 65536, 0
+        lens, ids, dst_pages, used = [], [], 65536, 0
         for req in synth.stress_requests(w.seed(1)):
             need = sum(-(-int(all_len[b]) // w.page_tokens) for b in req)
             if used + need > dst_pages:
                 break
             lens += [int(all_len[b]) for b in req]
+            ids += [int(b) for b in req]
             used += need
+        return w, lens, dst_pages, ids
+    w = synth.WORKLOADS[name.replace("_host", "")]
+    if name == "gqa7b":
+        return w, [synth.GQA7B_BLOCK_TOKENS] * (blocks or synth.GQA7B_REQUESTS * synth.GQA7B_BLOCKS_PER_REQUEST), synth.GQA7B_DST_PAGES, None
+    if name == "tiny":
+        return w, synth.TINY_BLOCKS, synth.TINY_DST_PAGES, None
+    if name in ("corpus", "corpus_host"):
+        return w, synth.CORPUS_BLOCKS, synth.CORPUS_DST_PAGES, None
+    if name == "fp8":
+        return w, synth.FP8_BLOCKS, sum(-(-n // w.page_tokens) for n in synth.FP8_BLOCKS) + 100, None
+    raise ValueError(name)
+
+
+def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0):
+    """Save and restore phases of one workload shape, each timed on its own over `steps`
+    calls (the damage the configuration prescribes is applied between the two, so the
+    restore is timed with it in place).  Returns a record for the bench line."""
+    import torch
+    import synth
+    import paper_2609_39358_b200 as gk
+
+    w, lens, dst_pages, ids = shape_of(synth, name, blocks)
+    host_tier = name.endswith("_host")
     dtype = gk.GK_BF16 if w.dtype == "bf16" else gk.GK_FP8_E4M3
-    flags = gk.GK_FLAG_SINGLE_PASS if args.single_pass else 0
+    flags = gk.GK_FLAG_SINGLE_PASS if single_pass else 0
     geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, dtype, w.scale_kv, flags)
     ctx = gk.Context(geom, device.index)
-    restore_traffic = 2 if args.single_pass else 3     # DRAM bytes per blob byte of the restore
+    restore_traffic = 2 if single_pass else 3     # DRAM bytes per blob byte of the restore
     slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
     pages = [-(-n // w.page_tokens) for n in lens]
     src_pages = sum(pages)
@@ -704,12 +809,17 @@ def run_other_workload(args):
     src, dst = cache(src_pages, w.seed(10)), cache(dst_pages, w.seed(11))
     sperm = torch.from_numpy(synth.page_permutation(src_pages, w.seed(12))).to(device)
     dperm = torch.from_numpy(synth.page_permutation(dst_pages, w.seed(13))).to(device)
-    pack_jobs, restore_jobs, off, total = [], [], 0, 0
+    pack_jobs, restore_jobs, blobs, off, total = [], [], [], 0, 0
     for n, P in zip(lens, pages):
         nb, _ = gk.gk_blob_size(geom, n)
         total += nb
-        blob = torch.empty(nb, dtype=torch.uint8, device=device)
-        sums = torch.zeros(P, dtype=torch.int64, device=device)
+        if host_tier:
+            blob = torch.empty(nb, dtype=torch.uint8, pin_memory=True)
+            sums = torch.zeros(P, dtype=torch.int64, pin_memory=True)
+        else:
+            blob = torch.empty(nb, dtype=torch.uint8, device=device)
+            sums = torch.zeros(P, dtype=torch.int64, device=device)
+        blobs.append(blob)
         pack_jobs.append(gk.Job(blob, sums, sperm[off:off + P].contiguous(), n))
         restore_jobs.append(gk.Job(blob, sums, dperm[off:off + P].contiguous(), n))
         off += P
@@ -719,46 +829,169 @@ def run_other_workload(args):
     fb = torch.zeros(nj, dtype=torch.int32, device=device)
     status = torch.zeros(nj, dtype=torch.uint8, device=device)
     stream = torch.cuda.current_stream(device)
+    do_pack = (lambda: ctx.gk_pack_host(src, pack_jobs, status)) if host_tier else (lambda: ctx.gk_pack_batch(src, pack_jobs, status))
+    do_restore = ((lambda: ctx.gk_restore_host(restore_jobs, dst, mask, fb)) if host_tier
+                  else (lambda: ctx.gk_restore(restore_jobs, dst, mask, fb)))
+    if host_tier:
+        steps, warmup = min(steps, 2), 1
 
-    def step(ev=None):
-        if ev:
-            ev[0].record(stream)
-        ctx.gk_pack_batch(src, pack_jobs, status)
-        if ev:
-            ev[1].record(stream)
-        ctx.gk_restore(restore_jobs, dst, mask, fb)
-        if ev:
-            ev[2].record(stream)
+    def timed(fn, reps):
+        for _ in range(warmup):
+            fn()
+        torch.cuda.synchronize(device)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(2)] for _ in range(reps)]
+        for k in range(reps):
+            ev[k][0].record(stream)
+            fn()
+            ev[k][1].record(stream)
+        torch.cuda.synchronize(device)
+        return [e[0].elapsed_time(e[1]) for e in ev]
 
-    for _ in range(max(args.warmup, 3)):
-        step()
+    pack_ms = timed(do_pack, steps)
+    assert int(status.sum().item()) == 0
+
+    # damage, as the configuration prescribes it (seeded); expected number of rejected blocks
+    expect_rejected, damage = 0, "none"
+    rng = np.random.default_rng(w.seed(14))
+    R = w.layers * w.scale_kv * w.kv_heads * 4 + w.page_tokens * 2 * w.layers * (slab // w.page_tokens)
+    S = w.layers * w.scale_kv * w.kv_heads * 4
+    if name == "tiny":
+        j = int(rng.integers(0, nj))
+        pos = int(synth.bit_flip_positions(blobs[j].numel() * 8, 1, w.seed(15))[0])
+        blobs[j][pos >> 3] ^= 1 << (pos & 7)
+        expect_rejected, damage = 1, "one flipped bit in one of the 4 blobs"
+    elif name == "fp8":
+        ja, jb_ = (int(x) for x in rng.choice(nj, size=2, replace=False))
+        pa, pb = int(rng.integers(0, pages[ja])), int(rng.integers(0, pages[jb_]))
+        start, xors = synth.byte_run_corruption(pa * R, pa * R + S, 8, w.seed(6))
+        blobs[ja][start:start + 8] ^= torch.from_numpy(xors).to(device)
+        start, xors = synth.byte_run_corruption(pb * R + S, pb * R + S + slab, 8, w.seed(7))
+        blobs[jb_][start:start + 8] ^= torch.from_numpy(xors).to(device)
+        expect_rejected, damage = 2, "8 consecutive bytes in a scale section of one blob and in the K data of another"
+    elif name.startswith("stress"):
+        frac = 1.0 / 3.0 if name.endswith("one_third_damaged") else 0.01
+        bad_ids, bad_flips = synth.stress_corrupted_blocks(w.seed(2), frac=frac)
+        bad = dict(zip(bad_ids.tolist(), bad_flips.tolist()))
+        for j, b in enumerate(ids):
+            if b in bad:
+                for pos in synth.bit_flip_positions(blobs[j].numel() * 8, bad[b], w.seed(50_000 + b)):
+                    blobs[j][int(pos) >> 3] ^= 1 << (int(pos) & 7)
+                expect_rejected += 1
+        damage = f"1 to 8 flipped bits in the blobs of a seeded {frac:.2%} of the pool's blocks"
     torch.cuda.synchronize(device)
-    events = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
-    for k in range(args.steps):
-        step(events[k])
-    torch.cuda.synchronize(device)
-    assert int(mask.sum().item()) == 0 and int(status.sum().item()) == 0
-    pack_ms = float(np.mean([e[0].elapsed_time(e[1]) for e in events]))
-    restore_ms = float(np.mean([e[1].elapsed_time(e[2]) for e in events]))
-    step_ms = pack_ms + restore_ms
+
+    restore_ms = timed(do_restore, steps)
+    mask_host = mask.cpu().numpy()
+    committed = int(sum(b.numel() for b, m in zip(blobs, mask_host) if m == 0))
+    codes = np.bincount(mask_host, minlength=5)
+    census = {"ok": int(codes[0]), "checksum": int(codes[1]), "page_table": int(codes[2]), "missing": int(codes[3]),
+              "wait_ran_out": int(codes[4]), "expected_rejected": expect_rejected}
+    assert census["checksum"] == expect_rejected and census["ok"] == nj - expect_rejected, census
+    assert ctx.gk_get_stats()["device_wait_expired"] == 0
     peak, peak_kind = measured_peak()
-    line = {"metric": METRIC, "value": 4 * total / (step_ms * 1e-3) / 1e9, "unit": UNIT, "n_gpus": 1,
-            "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": step_ms, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
-            "config": {"workload": f"{args.workload}: {w.layers} layers, {w.kv_heads} KV heads, head_dim {w.head_dim}, "
-                                   f"{w.dtype}, {w.page_tokens}-token pages; {nj} blocks, {sum(lens)} tokens, "
-                                   f"{total / 2**30:.2f} GiB of blobs, {dst_pages}-page destination",
-                       "step": "gk_pack_batch + gk_restore of all blocks in one call each"
+    pm, rm = float(np.median(pack_ms)), float(np.median(restore_ms))
+    rec = {"workload": f"{name}: {w.layers} layers, {w.kv_heads} KV heads, head_dim {w.head_dim}, {w.dtype}, "
+                       f"{w.page_tokens}-token pages; {nj} blocks, {sum(lens)} tokens, {total / 2**30:.2f} GiB of blobs, "
+                       f"{dst_pages}-page destination" + (", blobs in pinned host memory" if host_tier else ""),
+           "jobs": nj, "tokens": int(sum(lens)), "blob_bytes": int(total), "damage": damage, "mask_census": census,
+           "save_ms": stats_ms(pack_ms), "restore_ms": stats_ms(restore_ms),
+           "restored_tokens_per_s": sum(lens) / (rm * 1e-3)}
+    if host_tier:
+        rec["save_host_link_gbs"] = total / (pm * 1e-3) / 1e9
+        rec["restore_host_link_gbs"] = total / (rm * 1e-3) / 1e9
+    else:
+        rec["save"] = fractions(2 * total / (pm * 1e-3) / 1e9, peak)
+        # every blob is read once to be verified; only the accepted ones are read again and written
+        rec["committed_blob_bytes"] = committed
+        rec["restore_useful"] = fractions((total + committed) / (rm * 1e-3) / 1e9, peak)
+        rec["restore_dram_model"] = dict(fractions((total + (restore_traffic - 1) * committed) / (rm * 1e-3) / 1e9, peak),
+                                         dram_bytes="blob bytes read to verify + %d x the bytes of the accepted blobs"
+                                                    % (restore_traffic - 1))
+    ctx.close()
+    del src, dst, blobs, pack_jobs, restore_jobs
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return rec
+
+
+def latency_cases(device, token_counts=(256, 1024, 5200, 24018), reps=15):
+    """Restore of ONE block of the GQA-7B geometry, the serving case of a single recurring
+    prompt: device time per call, L2 flushed before every call (the blob is cold in HBM, as
+    it is after sitting in the pool), median and best; beside it the time the bytes alone
+    would take at the measured copy peak (blob read twice and written once, and read once)."""
+    import torch
+    import synth
+    import paper_2609_39358_b200 as gk
+    w = synth.GQA7B
+    geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, gk.GK_BF16, 0)
+    slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
+    peak, _ = measured_peak()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device=device)
+    stream = torch.cuda.current_stream(device)
+    out = {}
+    for n in token_counts:
+        ctx = gk.Context(geom, device.index)
+        nb, P = gk.gk_blob_size(geom, n)
+        data = synth.kv_bytes_bf16(w.layers * P * slab, w.sigma, w.seed(600 + n), device)
+        src = gk.Cache(data, P, 2 * P * slab, P * slab, slab)
+        dst = gk.Cache(torch.zeros_like(data), P, 2 * P * slab, P * slab, slab)
+        blob = torch.empty(nb, dtype=torch.uint8, device=device)
+        sums = torch.zeros(P, dtype=torch.int64, device=device)
+        spt = torch.from_numpy(synth.page_permutation(P, w.seed(601))).to(device)
+        dpt = torch.from_numpy(synth.page_permutation(P, w.seed(602))).to(device)
+        ctx.gk_pack(src, spt, n, blob, sums)
+        jobs = gk.JobArray([gk.Job(blob, sums, dpt, n)])
+        mask = torch.zeros(1, dtype=torch.uint8, device=device)
+        fb = torch.zeros(1, dtype=torch.int32, device=device)
+        for _ in range(3):
+            ctx.gk_restore(jobs, dst, mask, fb)
+        torch.cuda.synchronize(device)
+        ts = []
+        for _ in range(reps):
+            flush.fill_(1)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            ctx.gk_restore(jobs, dst, mask, fb)
+            e1.record(stream)
+            torch.cuda.synchronize(device)
+            ts.append(e0.elapsed_time(e1) * 1e3)
+        assert int(mask.item()) == 0
+        # back to back, without the flush: what a caller sees who restores the same block again at once
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            ctx.gk_restore(jobs, dst, mask, fb)
+        e1.record(stream)
+        torch.cuda.synchronize(device)
+        warm = e0.elapsed_time(e1) * 1e3 / reps
+        med = float(np.median(ts))
+        bound3 = 3 * nb / (peak * 1e9) * 1e6
+        out[f"{n}_tokens"] = {"blob_mib": nb / 2**20, "restore_us_median": med, "restore_us_best": float(np.min(ts)),
+                              "restore_us_back_to_back": warm, "bound_us_3_bytes_per_byte": bound3,
+                              "frac_of_bound": bound3 / med, "bound_us_2_bytes_per_byte": 2 * nb / (peak * 1e9) * 1e6,
+                              "restored_tokens_per_s": n / (med * 1e-6)}
+        ctx.close()
+        del data, src, dst, blob
+        torch.cuda.empty_cache()
+    return out
+
+
+def run_other_workload(args):
+    import torch
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    name = {"stress": "stress_wave"}.get(args.workload, args.workload)
+    rec = workload_case(name, device, steps=max(args.steps, 1) if args.steps < 50 else 10, warmup=max(args.warmup, 3),
+                        single_pass=args.single_pass, blocks=args.blocks)
+    pm, rm = rec["save_ms"]["median"], rec["restore_ms"]["median"]
+    line = {"metric": METRIC, "value": rec["restore_useful"]["gbs"], "unit": UNIT, "n_gpus": 1,
+            "steps": rec["restore_ms"]["n"], "warmup": max(args.warmup, 3), "ms_per_step": pm + rm,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": rec["workload"],
+                       "step": "gk_pack_batch, then gk_restore, of all blocks in one call each, timed separately"
                                + (" (restore in a single pass: GK_FLAG_SINGLE_PASS)" if args.single_pass else "")},
-            "tokens_per_s": sum(lens) / (step_ms * 1e-3),
-            "phases": {"pack": {"ms": pack_ms, "gbs": 2 * total / (pack_ms * 1e-3) / 1e9,
-                                "frac_of_hbm_peak": 2 * total / (pack_ms * 1e-3) / 1e9 / peak},
-                       "restore": {"ms": restore_ms, "gbs_useful": 2 * total / (restore_ms * 1e-3) / 1e9,
-                                   "dram_bytes_per_blob_byte": restore_traffic,
-                                   "gbs_dram_model": restore_traffic * total / (restore_ms * 1e-3) / 1e9,
-                                   "frac_of_hbm_peak_dram_model": restore_traffic * total / (restore_ms * 1e-3) / 1e9 / peak,
-                                   "tokens_per_s": sum(lens) / (restore_ms * 1e-3)}},
-            "peak": {"hbm_gbs": peak, "kind": f"of {peak_kind}"}}
+            "case": rec}
     print(json.dumps(line), flush=True)
 
 

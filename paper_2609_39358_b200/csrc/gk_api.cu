@@ -108,6 +108,7 @@ struct gk_ctx {
     uint32_t test_drop_verify = 0;  // test hook: see gk_ctx_set_tuning
     bool commit_reverse = true;     // commit side walks a job's pages from the last to the first
     uint32_t l2_hints = 0;          // bit 0: verify loads evict_last, bit 1: commit loads evict_first
+    uint32_t commit_items_per_cta = 3;       // small calls: commit work items wanted per resident CTA
     unsigned long long *trace = nullptr;  // builds with GK_TRACE: device buffer for time stamps (tuning keys)
     uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
     uint32_t commit_seg_tiles = 0;
@@ -314,8 +315,9 @@ Tiling commit_tiling(const gk_ctx *c, uint32_t stage_bytes, uint64_t total_pages
         st = c->commit_seg_tiles;
     } else if (total_pages > 0) {
         const uint64_t items = total_pages * ((tiles_full + st - 1) / st);
-        if (items < items_wanted(c, occ)) {
-            const uint64_t per_page = (items_wanted(c, occ) + total_pages - 1) / total_pages;
+        const uint64_t want = (uint64_t)c->commit_items_per_cta * c->sm_count * occ;
+        if (items < want) {
+            const uint64_t per_page = (want + total_pages - 1) / total_pages;
             st = (uint32_t)((tiles_full + per_page - 1) / per_page);
         }
     }
@@ -990,6 +992,7 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     else if (!strcmp(key, "test_drop_verify")) c->test_drop_verify = value;
     else if (!strcmp(key, "commit_reverse")) c->commit_reverse = value != 0;
     else if (!strcmp(key, "l2_hints")) c->l2_hints = value;
+    else if (!strcmp(key, "commit_items_per_cta")) c->commit_items_per_cta = value ? value : 1u;
 #ifdef GK_TRACE
     else if (!strcmp(key, "trace_lo")) c->trace = (unsigned long long *)(((uintptr_t)c->trace & ~(uintptr_t)0xffffffffull) | value);
     else if (!strcmp(key, "trace_hi")) c->trace = (unsigned long long *)(((uintptr_t)c->trace & 0xffffffffull) | ((uintptr_t)value << 32));
@@ -1115,7 +1118,7 @@ int gk_page_checksums(gk_ctx *c, const void *blob_dev, uint32_t n_tokens, uint64
 
 // verify + commit for the pages [page_begin, page_begin + n_pages) of the call
 static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const Tiling &tlv, const Tiling &tlc,
-                                 uint32_t page_begin, uint32_t n_pages, uint32_t jobs_in_launch, uint8_t *mask_dev,
+                                 uint32_t page_begin, uint32_t n_pages, uint8_t *mask_dev,
                                  int32_t *first_bad_dev, cudaStream_t st)
 {
     int rc;
@@ -1144,11 +1147,7 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
         c->stats.kernels_launched++;
         return GK_OK;
     }
-    // one job cannot overlap its own verify and commit (it is committed only after all of it has
-    // verified); from about 256 MiB on the two dedicated kernels then beat the fused one by more
-    // than their two extra launches cost (5,200 tokens of the GQA-7B shape: 386 us against 403 us)
-    const bool lone_big_job = jobs_in_launch == 1 && (uint64_t)n_pages * c->gd.R >= (256ull << 20);
-    if (c->fused && (!lone_big_job || c->test_drop_verify)) {
+    if (c->fused) {
         P.fused = 1u;
         P.inline_final = 1u;
         P.test_drop_from = c->test_drop_verify;  // tests: the jobs from this one on are never verified
@@ -1174,8 +1173,7 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
     const bool single = (c->gd.flags & GK_FLAG_SINGLE_PASS) && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
-    const bool fused = !single && c->fused && !(c->gd.flags & GK_FLAG_SKIP_VERIFY) &&
-                       !(n_jobs == 1 && pages * c->gd.R >= (256ull << 20));
+    const bool fused = !single && c->fused && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
     const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages,
                                   single ? c->occ_single : fused ? c->occ_fused : c->occ_verify, fused && n_jobs > 1);
     const Tiling tlc = commit_tiling(c, GK_COPY_STAGE, pages, fused ? c->occ_fused : c->occ_commit);
@@ -1190,7 +1188,7 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
         if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
         if ((rc = launch_claim(c, w, st)) != GK_OK) return rc;
     }
-    if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, 0, (uint32_t)pages, n_jobs, mask_dev, first_bad_page_dev, st)) != GK_OK)
+    if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, 0, (uint32_t)pages, mask_dev, first_bad_page_dev, st)) != GK_OK)
         return rc;
     c->stats.calls_restore++;
     c->stats.jobs += n_jobs;
@@ -1344,7 +1342,7 @@ static int restore_host_impl(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, con
         }
         GK_CUDA(c, cudaEventRecord(c->ev_copied[slot], c->copy_stream));
         GK_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied[slot], 0));
-        if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, page0, npages, j1 - j0, mask_dev, first_bad_page_dev, st)) != GK_OK)
+        if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, page0, npages, mask_dev, first_bad_page_dev, st)) != GK_OK)
             return rc;
         GK_CUDA(c, cudaEventRecord(c->ev_slot_free[slot], st));
         c->slot_used[slot] = true;
