@@ -388,6 +388,25 @@ int gk_fingerprints(gk_ctx *ctx, const void *data_dev, const uint64_t *offsets_d
 int gk_blob_digests(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const uint8_t *keys_dev,
                     uint8_t *digests_dev, uint8_t *page_digests_dev, void *stream);
 
+/* Bounds-checked build.  Section 3's sabotage paragraph reports that an address
+ * sanitizer found the one out-of-bounds read of the paper's own code; a GPU
+ * library cannot lean on such a tool everywhere, so this one can be compiled
+ * with -DGK_DEBUG (libgk_debug.so): every access of a streaming kernel to caller
+ * memory -- bulk copies from and to caches and blobs, scale values, checksum
+ * words -- is then compared with the extent of the object it belongs to (cache
+ * extents from the strides and num_pages, blob and checksum extents from
+ * n_tokens).  An access that falls outside is skipped, never made, and the first
+ * one is recorded; nothing traps and the context stays usable.
+ * gk_debug_status copies the record out (blocking): out[0] = 0 if every access so
+ * far was inside, else role << 8 | kind (kind 1 cache, 2 blob, 3 scales, 4
+ * checksums, 5 staging tile; role 0 loader, 1 commit loader, 2 finisher, 3
+ * storer), out[1..2] = offset of the refused access from its object's base,
+ * out[3] = its size.  In the ordinary build it returns GK_ERR_UNSUPPORTED.
+ * gk_debug_range_ok is the predicate itself, for host tests: 1 if
+ * [addr, addr+bytes) lies inside [base, base+extent), else 0. */
+int gk_debug_status(gk_ctx *ctx, uint32_t out[4]);
+int gk_debug_range_ok(uint64_t addr, uint64_t bytes, uint64_t base, uint64_t extent);
+
 /* Counters of this context.  Reads the device error word with a blocking copy. */
 int gk_get_stats(gk_ctx *ctx, gk_stats *out);
 
@@ -405,7 +424,10 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * "test_drop_verify" (tests only: with value k > 0 the fused restore kernel
  * verifies nothing of the jobs k-1, k, ..., so that the commit waits of exactly
  * those jobs run into their limit and the time-out handling can be checked
- * without hanging or faulting the GPU). */
+ * without hanging or faulting the GPU), and in the bounds-checked build only
+ * "debug_extent_cut" (tests: cache extents are taken to be this many bytes smaller
+ * than they are, so that a perfectly valid access to the last page is refused and
+ * the reporting can be checked without any access outside an object). */
 int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
 
 /* Page checksums of a device blob for callers that must not allocate.  (The

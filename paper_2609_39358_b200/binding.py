@@ -29,7 +29,8 @@ EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "
            "gk_page_checksums", "gk_restore", "gk_restore_host", "gk_get_stats", "gk_ctx_set_tuning", "gk_get_kernel_times",
            "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit", "gk_restore_stream",
            "gk_fingerprints", "gk_blob_digests", "gk_pack_layerwise", "gk_pack_layerwise_host",
-           "gk_restore_layerwise", "gk_restore_layerwise_host", "gk_ctx_reserve", "gk_ctx_clear_error"]
+           "gk_restore_layerwise", "gk_restore_layerwise_host", "gk_ctx_reserve", "gk_ctx_clear_error",
+           "gk_debug_status", "gk_debug_range_ok"]
 
 
 class GkError(RuntimeError):
@@ -171,6 +172,10 @@ def load_library() -> ctypes.CDLL:
     L.gk_ctx_reserve.argtypes = [vp, u32, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64]
     L.gk_ctx_clear_error.restype = ctypes.c_int
     L.gk_ctx_clear_error.argtypes = [vp, vp]
+    L.gk_debug_status.restype = ctypes.c_int
+    L.gk_debug_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
+    L.gk_debug_range_ok.restype = ctypes.c_int
+    L.gk_debug_range_ok.argtypes = [ctypes.c_uint64] * 4
     _lib = L
     return L
 
@@ -246,6 +251,10 @@ GK_NOALLOC_MAX_PAGES = 8192
 GK_NOALLOC_MAX_PAGE_TOKENS = 256
 
 
+def gk_debug_range_ok(addr: int, nbytes: int, base: int, extent: int) -> bool:
+    return bool(load_library().gk_debug_range_ok(addr, nbytes, base, extent))
+
+
 def gk_page_checksums_noalloc(geom: Geom, blob: torch.Tensor, n_tokens: int, checksums: torch.Tensor,
                               device: int = 0, stream=None) -> None:
     """Page checksums of a device blob through the entry point that allocates
@@ -282,8 +291,20 @@ class Context:
 
     def close(self):
         if getattr(self, "_h", None):
+            status = self.gk_debug_status()
             self._lib.gk_ctx_destroy(self._h)
             self._h = None
+            if status is not None and status[0] != 0:
+                raise GkError(-8, "bounds-checked build",
+                              f"an access outside its object was refused: kind/role {status[0]:#x}, offset "
+                              f"{status[1] | (status[2] << 32)}, {status[3]} bytes")
+
+    def gk_debug_status(self):
+        """(kind/role, offset low, offset high, bytes) of the first refused access with the bounds-checked
+        library (all zero if there was none); None with the ordinary library."""
+        out = (ctypes.c_uint32 * 4)()
+        rc = self._lib.gk_debug_status(self._h, out)
+        return None if rc != GK_OK else tuple(int(x) for x in out)
 
     def __del__(self):
         try:

@@ -8,6 +8,7 @@ import sys
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libgk.so")
+DEBUG_LIB_PATH = os.path.join(_HERE, "libgk_debug.so")   # the bounds-checked build (-DGK_DEBUG)
 
 _SOURCES = ["gk_api.cu"]
 _DEPS = ["gk_api.cu", "gk_kernels.cuh", "gk_device.cuh", "gk_sha256.cuh", "gk_gf2_generated.inc", "gen_tables.py",
@@ -21,7 +22,13 @@ def _nvcc() -> str:
     return "nvcc"
 
 
-def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | None = None) -> str:
+def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | None = None, debug: bool = False) -> str:
+    """Builds libgk.so, or with debug=True libgk_debug.so: the same sources with -DGK_DEBUG, in which the
+    streaming kernels compare every access to caller memory with the extent of its object (use it through
+    GK_LIB_PATH)."""
+    lib_path = DEBUG_LIB_PATH if debug else LIB_PATH
+    if debug:
+        extra_flags = list(extra_flags or []) + ["-DGK_DEBUG"]
     sys.path.insert(0, _CSRC)
     try:
         import gen_tables
@@ -30,9 +37,9 @@ def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | N
         sys.path.pop(0)
     deps = [os.path.join(_CSRC, d) for d in _DEPS]
     newest = max(os.path.getmtime(d) for d in deps if os.path.exists(d))
-    if not force and os.path.exists(LIB_PATH) and os.path.getmtime(LIB_PATH) >= newest:
-        return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
+    if not force and os.path.exists(lib_path) and os.path.getmtime(lib_path) >= newest:
+        return lib_path
+    tmp = lib_path + f".tmp{os.getpid()}"
     cmd = [_nvcc(), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-shared", "-Xcompiler", "-fPIC", "-Xcompiler", "-Wall", "--use_fast_math",
            "-I", os.path.join(_HERE, "..", "include")]
@@ -44,9 +51,9 @@ def build(force: bool = False, verbose: bool = False, extra_flags: list[str] | N
         cmd += os.environ["GK_NVCC_FLAGS"].split()
     cmd += [os.path.join(_CSRC, s) for s in _SOURCES] + ["-o", tmp, "-lcudart"]
     subprocess.check_call(cmd)
-    os.replace(tmp, LIB_PATH)
-    return LIB_PATH
+    os.replace(tmp, lib_path)
+    return lib_path
 
 
 if __name__ == "__main__":
-    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv, debug="--debug" in sys.argv))

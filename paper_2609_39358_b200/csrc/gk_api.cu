@@ -109,6 +109,7 @@ struct gk_ctx {
     bool commit_reverse = true;     // commit side walks a job's pages from the last to the first
     uint32_t l2_hints = 0;          // bit 0: verify loads evict_last, bit 1: commit loads evict_first
     uint32_t commit_items_per_cta = 3;       // small calls: commit work items wanted per resident CTA
+    uint64_t debug_extent_cut = 0;  // bounds-checked build, tests: cache extents are reported this much smaller
     unsigned long long *trace = nullptr;  // builds with GK_TRACE: device buffer for time stamps (tuning keys)
     uint32_t seg_granules = 0;   // segment length in granules for the CRC modes
     uint32_t commit_seg_tiles = 0;
@@ -247,6 +248,15 @@ int check_cache(gk_ctx *c, const gk_cache *k, CacheDev *out)
     out->s_layer_stride = k->s_layer_stride;
     out->s_kv_stride = k->s_kv_stride;
     out->s_page_stride = k->s_page_stride;
+    // where the last byte that a page table of this geometry can address lies (the bounds-checked build
+    // compares every access with these)
+    const uint64_t slab = (uint64_t)c->gd.page_tokens * c->gd.row;
+    out->data_extent = (uint64_t)(c->gd.layers - 1u) * k->layer_stride + k->kv_stride + (k->num_pages - 1u) * k->page_stride + slab;
+    out->scales_extent = c->gd.scale_kv ? (uint64_t)(c->gd.layers - 1u) * k->s_layer_stride +
+                                              (uint64_t)(c->gd.scale_kv - 1u) * k->s_kv_stride +
+                                              (k->num_pages - 1u) * k->s_page_stride + 4ull * c->gd.kv_heads
+                                        : 0u;
+    out->data_extent -= c->debug_extent_cut < out->data_extent ? c->debug_extent_cut : out->data_extent;
     return GK_OK;
 }
 
@@ -993,6 +1003,9 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     else if (!strcmp(key, "commit_reverse")) c->commit_reverse = value != 0;
     else if (!strcmp(key, "l2_hints")) c->l2_hints = value;
     else if (!strcmp(key, "commit_items_per_cta")) c->commit_items_per_cta = value ? value : 1u;
+#ifdef GK_DEBUG
+    else if (!strcmp(key, "debug_extent_cut")) c->debug_extent_cut = value;
+#endif
 #ifdef GK_TRACE
     else if (!strcmp(key, "trace_lo")) c->trace = (unsigned long long *)(((uintptr_t)c->trace & ~(uintptr_t)0xffffffffull) | value);
     else if (!strcmp(key, "trace_hi")) c->trace = (unsigned long long *)(((uintptr_t)c->trace & 0xffffffffull) | ((uintptr_t)value << 32));
@@ -1700,6 +1713,24 @@ int gk_get_kernel_times(gk_ctx *c, double ms[4], uint64_t launches[4])
     return GK_OK;
 }
 
+int gk_debug_range_ok(uint64_t addr, uint64_t bytes, uint64_t base, uint64_t extent)
+{
+    return range_inside(addr, bytes, base, extent) ? 1 : 0;
+}
+
+int gk_debug_status(gk_ctx *c, uint32_t out[4])
+{
+    if (!c || !out) return GK_ERR_ARG;
+#ifdef GK_DEBUG
+    DeviceGuard guard(c->device);
+    GK_CUDA(c, cudaMemcpy(out, c->d_error + 8, 16, cudaMemcpyDeviceToHost));
+    return GK_OK;
+#else
+    out[0] = out[1] = out[2] = out[3] = 0u;
+    return fail(c, GK_ERR_UNSUPPORTED, "this library was built without GK_DEBUG");
+#endif
+}
+
 int gk_get_stats(gk_ctx *c, gk_stats *out)
 {
     if (!c || !out) return GK_ERR_ARG;
@@ -1778,6 +1809,7 @@ __global__ void noalloc_setup_kernel(unsigned char *scratch, JobDev job, GeomDev
         words[5] = 0;        // work counters
         words[6] = 0;
         words[7] = 0;        // the error word as this call found it
+        words[12] = 0;       // the bounds-checked build's record of a refused access
     }
     for (uint32_t t = threadIdx.x; t < (uint32_t)GK_CRC_NT; t += blockDim.x)
         tc[t] = dev_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);

@@ -34,7 +34,17 @@ struct CacheDev {
     uint64_t num_pages, layer_stride, kv_stride, page_stride;
     uint8_t *scales;
     uint64_t s_layer_stride, s_kv_stride, s_page_stride;
+    uint64_t data_extent, scales_extent;  // bytes from the base pointers to the end of the last slab / scale row
 };
+
+// Is [addr, addr + bytes) inside [base, base + extent)?  (The bounds-checked build asks this before
+// every access to caller memory; a host test asks it, too.)
+__host__ __device__ inline bool range_inside(uint64_t addr, uint64_t bytes, uint64_t base, uint64_t extent)
+{
+    if (addr < base) return false;
+    const uint64_t off = addr - base;
+    return off <= extent && bytes <= extent - off;
+}
 
 struct JobDev {
     uint8_t *blob;
@@ -283,6 +293,13 @@ __device__ __forceinline__ void bulk_wait_read()
 __device__ __forceinline__ void bulk_wait_all()
 {
     asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+// Counts `bytes` as arrived on a barrier without a copy (the bounds-checked build: a refused
+// copy must still let the waiters go on).
+__device__ __forceinline__ void mbar_complete_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.complete_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
 
 __device__ __forceinline__ void fence_proxy_async_smem()

@@ -848,6 +848,42 @@ constexpr uint32_t kNoJob = 0xffffffffu;
     } while (0)
 #endif
 
+// Bounds-checked build (-DGK_DEBUG): before every access of a streaming kernel to caller
+// memory -- the bulk copies from and to cache and blobs, the scale values, the checksum words --
+// the address range is compared with the extent of the object it belongs to.  An access that
+// falls outside is NOT made (a refused load still counts as arrived, so that nothing waits for
+// it); the first one leaves what it was in the debug words behind the context's error word:
+// [8] = role << 8 | kind, [9..10] = offset from the object's base, [11] = bytes.  Nothing traps.
+enum DebugKind : uint32_t { kDbgCache = 1, kDbgBlob = 2, kDbgScales = 3, kDbgSums = 4, kDbgStage = 5 };
+#ifdef GK_DEBUG
+__device__ __noinline__ void debug_report(const StreamParams &P, uint32_t kind, uint32_t role, uint64_t addr,
+                                          uint64_t bytes, uint64_t base)
+{
+    if (atomicCAS(P.w.error + 8, 0u, (role << 8) | kind) == 0u) {
+        const uint64_t off = addr - base;
+        P.w.error[9] = (uint32_t)off;
+        P.w.error[10] = (uint32_t)(off >> 32);
+        P.w.error[11] = (uint32_t)bytes;
+    }
+}
+__device__ __forceinline__ bool debug_ok(const StreamParams &P, uint32_t kind, uint32_t role, const void *addr,
+                                         uint64_t bytes, const void *base, uint64_t extent)
+{
+    if (range_inside((uint64_t)addr, bytes, (uint64_t)base, extent)) return true;
+    debug_report(P, kind, role, (uint64_t)addr, bytes, (uint64_t)base);
+    return false;
+}
+// extent of the blob of the job an item belongs to
+__device__ __forceinline__ uint64_t debug_blob_bytes(const StreamParams &P, uint32_t j)
+{
+    const JobDev &jb = P.w.jobs[j];
+    return (uint64_t)jb.n_pages * P.g.S + (uint64_t)jb.n_tokens * P.g.tokB;
+}
+#define GK_DEBUG_OK(P, kind, role, addr, bytes, base, extent) debug_ok(P, kind, role, addr, bytes, base, extent)
+#else
+#define GK_DEBUG_OK(P, kind, role, addr, bytes, base, extent) true
+#endif
+
 template <bool STATIC_FIRST>
 __device__ __forceinline__ uint32_t next_item(uint32_t *ctr, uint32_t base, int lane)
 {
@@ -947,7 +983,13 @@ __device__ __forceinline__ void finish_segment(const StreamParams &P, const Ring
             red_xor_u64(acc, tot);
         } else {
             uint64_t stored = 0;
-            if (MODE != kPack) stored = *it.sum;  // in flight together with the two atomics below
+#ifdef GK_DEBUG
+            const bool sum_ok = debug_ok(P, kDbgSums, 2u, it.sum, 8u, P.w.jobs[it.j].checksums,
+                                         8ull * P.w.jobs[it.j].n_pages);
+#else
+            constexpr bool sum_ok = true;
+#endif
+            if (MODE != kPack && sum_ok) stored = *it.sum;  // in flight together with the two atomics below
             uint64_t r = tot;
             bool last = true;
             if (nseg > 1u) {
@@ -958,7 +1000,7 @@ __device__ __forceinline__ void finish_segment(const StreamParams &P, const Ring
             if (last) {
                 const uint64_t crc = __brevll(r ^ P.w.init_term[it.t] ^ ~0ull);
                 if (MODE == kPack) {
-                    *it.sum = crc;
+                    if (sum_ok) *it.sum = crc;
                 } else {
                     if (crc != stored || *abort_flag) atomicMin(&P.w.bad_crc[it.j], (int32_t)it.p);
                     red_add_release_u32(&P.w.job_done[it.j], 1u);  // nobody here waits for the count
@@ -1089,7 +1131,9 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
                         const uint32_t i = i0 + 32u * u;
-                        v[u] = (i < i_end) ? *reinterpret_cast<const uint32_t *>(scale_addr(P.g, P.cache, i, it.phys)) : 0u;
+                        const uint8_t *sa = scale_addr(P.g, P.cache, i < i_end ? i : (uint32_t)(r0 >> 2), it.phys);
+                        v[u] = (i < i_end && GK_DEBUG_OK(P, kDbgScales, 0u, sa, 4u, P.cache.scales, P.cache.scales_extent))
+                                   ? *reinterpret_cast<const uint32_t *>(sa) : 0u;
                     }
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
@@ -1124,7 +1168,13 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                                 uint32_t nb = ch.len - off;
                                 if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
                                 if (nb == 0u) break;  // cannot happen with a valid geometry; never spin
-                                bulk_g2s(so, chunk_addr(P.cache, ch, chunk, it.phys, off), nb, bar);
+                                const uint8_t *ca = chunk_addr(P.cache, ch, chunk, it.phys, off);
+                                if (GK_DEBUG_OK(P, kDbgCache, 0u, ca, nb, P.cache.data, P.cache.data_extent) &&
+                                    GK_DEBUG_OK(P, kDbgStage, 0u, (const void *)(uintptr_t)so, nb,
+                                                (const void *)(uintptr_t)sbase, STAGE_BYTES))
+                                    bulk_g2s(so, ca, nb, bar);
+                                else
+                                    mbar_complete_tx(bar, nb);
                                 d0 += nb;
                                 so += nb;
                                 ++chunk;
@@ -1136,7 +1186,16 @@ __device__ __forceinline__ void loader_role(const StreamParams &P, const Tiling 
                             mbar_arrive(bar);
                         } else {
                             mbar_arrive_expect_tx(bar, nreal);
-                            if (hint) bulk_g2s_hint(sbase + lead, it.rec + r0, nreal, bar, policy);
+#ifdef GK_DEBUG
+                            const bool in_blob = debug_ok(P, kDbgBlob, MODE == kCommit ? 1u : 0u, it.rec + r0, nreal,
+                                                          P.w.jobs[it.j].blob, debug_blob_bytes(P, it.j)) &&
+                                                 debug_ok(P, kDbgStage, 0u, (const void *)(uintptr_t)(lead + nreal), 0u,
+                                                          nullptr, STAGE_BYTES);
+#else
+                            constexpr bool in_blob = true;
+#endif
+                            if (!in_blob) mbar_complete_tx(bar, nreal);
+                            else if (hint) bulk_g2s_hint(sbase + lead, it.rec + r0, nreal, bar, policy);
                             else bulk_g2s(sbase + lead, it.rec + r0, nreal, bar);
                         }
                     }
@@ -1217,7 +1276,9 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
             if (!aborted) {
                 for (uint32_t i = (uint32_t)(r0 >> 2) + lane; i < (uint32_t)(e1 >> 2); i += 32u) {
                     const uint32_t v = *reinterpret_cast<const uint32_t *>(sgen + lead + (4u * i - (uint32_t)r0));
-                    *reinterpret_cast<uint32_t *>(scale_addr(P.g, P.cache, i, phys)) = v;
+                    uint8_t *sa = scale_addr(P.g, P.cache, i, phys);
+                    if (GK_DEBUG_OK(P, kDbgScales, 3u, sa, 4u, P.cache.scales, P.cache.scales_extent))
+                        *reinterpret_cast<uint32_t *>(sa) = v;
                 }
             }
         }
@@ -1225,7 +1286,10 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
         if (lane == 0) {
             if (!aborted && nreal > 0u) {
                 if (MODE == kPack) {
-                    bulk_s2g(it.rec + r0, sbase + lead, nreal);
+#ifdef GK_DEBUG
+                    if (debug_ok(P, kDbgBlob, 3u, it.rec + r0, nreal, P.w.jobs[it.j].blob, debug_blob_bytes(P, it.j)))
+#endif
+                        bulk_s2g(it.rec + r0, sbase + lead, nreal);
                 } else {
                     const uint32_t data_bytes = nreal - scale_bytes;
                     uint64_t d0 = r0 + scale_bytes - P.g.S;
@@ -1237,7 +1301,8 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
                         uint32_t nb = ch.len - off;
                         if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
                         if (nb == 0u) break;  // cannot happen with a valid geometry; never spin
-                        bulk_s2g(chunk_addr(P.cache, ch, chunk, phys, off), so, nb);
+                        uint8_t *ca = chunk_addr(P.cache, ch, chunk, phys, off);
+                        if (GK_DEBUG_OK(P, kDbgCache, 3u, ca, nb, P.cache.data, P.cache.data_extent)) bulk_s2g(ca, so, nb);
                         d0 += nb;
                         so += nb;
                         ++chunk;
