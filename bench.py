@@ -64,6 +64,10 @@ def parse_args():
                          "its checksum receive the unverified bytes); prints the short line, never the headline")
     ap.add_argument("--blocks", type=int, default=0,
                     help="restore this many blocks instead of the workload's 16 (small cases for profiling)")
+    ap.add_argument("--unfused", action="store_true",
+                    help="restore with a verify launch, a compare launch and a commit launch instead of the fused "
+                         "kernel (the kernels gk_verify and gk_commit run; for profiling)")
+    ap.add_argument("--tune", default="", help="tuning keys for the headline context, key=value[,key=value...]")
     ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the one-step-at-a-time end-to-end leg")
     ap.add_argument("--e2e-pipelined-steps", type=int, default=10,
                     help="steps of the pipelined end-to-end leg (save of step k+1 overlaps restore of step k)")
@@ -421,6 +425,11 @@ def run_ours(args):
         if events:
             events[2].record(stream)
 
+    if args.unfused:
+        ctx.set_tuning("fused", 0)
+    for kv in filter(None, args.tune.split(",")):
+        key, val = kv.split("=")
+        ctx.set_tuning(key, int(val))
     # warm-up: the per-kernel timing events are created here, not in the timed region
     ctx.set_tuning("profile", 1)
     for _ in range(max(args.warmup, 3)):
@@ -672,6 +681,19 @@ def run_ours(args):
                                      "tokens_per_s": th * nt / o["t_multi_restore"]},
                         "nproc": hi["nproc"], "cpu_model": hi["cpu_model"]}
 
+    # ---- the integer side: measured rate of three-input logic operations, and what it allows the checksum
+    alu = None
+    if rank == 0:
+        rate = ctx.gk_measure_logic_rate()
+        mhz = (clocks or {}).get("sm_max_mhz") or 1965.0
+        sms = torch.cuda.get_device_properties(device).multi_processor_count
+        instr_per_byte = 3.05    # integer-pipe instructions per blob byte of the verify kernel (ncu, profiles/)
+        alu = {"logic_lane_ops_per_s": rate, "lanes_per_clock_per_sm": rate / (sms * mhz * 1e6),
+               "how": "one kernel of independent lop3 chains, 8 CTAs x 256 threads per SM, CUDA events, best of 3",
+               "verify_alone_bound_gbs": rate / instr_per_byte / 1e9,
+               "note": f"the checksum costs {instr_per_byte} integer-pipe instructions per byte, so verification "
+                       "alone cannot stream faster than this; in the fused restore kernel it hides under the DRAM time"}
+
     # ---- the other workload shapes and the lone-block latencies (one GPU, after the headline's memory is free)
     workloads, latency = None, None
     if world == 1 and not args.no_workloads and not args.blocks:
@@ -715,7 +737,7 @@ def run_ours(args):
                 "restore": dict(stats_ms(restore_all), tokens_per_s=n_blocks * wl["n_tok"] / (restore_ms * 1e-3)),
                 "whole_step": {"ms_per_step": step_ms,
                                "gbs_save_plus_restore": world * 4 * batch_bytes / (step_ms * 1e-3) / 1e9}},
-            "roofline": roofline, "kernels": kernels, "workloads": workloads, "latency": latency,
+            "roofline": roofline, "kernels": kernels, "alu": alu, "workloads": workloads, "latency": latency,
             "cpu_baseline": cpu_baseline, "e2e": e2e,
             "gpu_launches": launches, "clocks": clocks,
         }

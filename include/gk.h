@@ -470,6 +470,14 @@ int gk_ctx_set_tuning(gk_ctx *ctx, const char *key, uint32_t value);
 int gk_page_checksums_noalloc(const gk_geom *geom, const void *blob_dev, uint32_t n_tokens,
                               uint64_t *checksums_dev, int device, void *stream);
 
+/* Measurement aid (the paper has no counterpart): the rate at which this GPU
+ * executes three-input logic operations, the instruction the checksum kernels
+ * are made of -- lane operations per second over all SMs, from one kernel of
+ * independent lop3 chains timed with CUDA events (best of three launches).  The
+ * roofline of the checksum-bound kernels is this rate divided by their
+ * instructions per byte.  Blocks until the measurement is done. */
+int gk_measure_logic_rate(gk_ctx *ctx, double *lane_ops_per_second, void *stream);
+
 /* Per-kernel device time of the streaming kernels, for measurements.  With the
  * tuning key "profile" set to 1 every launch of a streaming kernel is bracketed
  * by CUDA events on its stream.  This call waits for the recorded events, and

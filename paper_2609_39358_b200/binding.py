@@ -30,7 +30,7 @@ EXPORTS = ["gk_blob_size", "gk_ctx_create", "gk_ctx_destroy", "gk_last_error", "
            "gk_page_checksums_noalloc", "gk_pack_host", "gk_verify", "gk_commit", "gk_restore_stream",
            "gk_fingerprints", "gk_blob_digests", "gk_pack_layerwise", "gk_pack_layerwise_host",
            "gk_restore_layerwise", "gk_restore_layerwise_host", "gk_ctx_reserve", "gk_ctx_clear_error",
-           "gk_debug_status", "gk_debug_range_ok"]
+           "gk_debug_status", "gk_debug_range_ok", "gk_measure_logic_rate"]
 
 
 class GkError(RuntimeError):
@@ -172,6 +172,8 @@ def load_library() -> ctypes.CDLL:
     L.gk_ctx_reserve.argtypes = [vp, u32, ctypes.c_uint64, ctypes.c_uint64, ctypes.c_uint64]
     L.gk_ctx_clear_error.restype = ctypes.c_int
     L.gk_ctx_clear_error.argtypes = [vp, vp]
+    L.gk_measure_logic_rate.restype = ctypes.c_int
+    L.gk_measure_logic_rate.argtypes = [vp, ctypes.POINTER(ctypes.c_double), vp]
     L.gk_debug_status.restype = ctypes.c_int
     L.gk_debug_status.argtypes = [vp, ctypes.POINTER(ctypes.c_uint32)]
     L.gk_debug_range_ok.restype = ctypes.c_int
@@ -444,6 +446,13 @@ class Context:
                         page_digests: Optional[torch.Tensor] = None, stream=None):
         self._check(self._lib.gk_blob_digests(self._h, self._jobs(jobs), len(jobs), _ptr(keys), _ptr(digests),
                                               _ptr(page_digests), _stream_handle(stream)), "gk_blob_digests")
+
+    def gk_measure_logic_rate(self, stream=None) -> float:
+        """Three-input logic operations per second (lanes x instructions) of this GPU, measured."""
+        out = ctypes.c_double(0.0)
+        self._check(self._lib.gk_measure_logic_rate(self._h, ctypes.byref(out), _stream_handle(stream)),
+                    "gk_measure_logic_rate")
+        return float(out.value)
 
     def gk_get_kernel_times(self) -> dict:
         """{'verify'|'pack'|'commit'|'restore': (ms, launches)} since the previous call (needs tuning key profile=1)."""

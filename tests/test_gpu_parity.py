@@ -1129,6 +1129,17 @@ def test_restore_beside_another_kernel_that_occupies_the_gpu(gk):
     ctx.close()
 
 
+def test_logic_rate_measurement_is_plausible(gk):
+    """The measured rate of three-input logic operations (the denominator of the checksum kernels'
+    roofline): between 32 and 128 lanes per clock per SM at the device's maximum clock."""
+    ctx = _ctx(gk, G_MID)
+    rate = ctx.gk_measure_logic_rate()
+    props = torch.cuda.get_device_properties(0)
+    per_sm_clk = rate / (props.multi_processor_count * getattr(props, "clock_rate", 1965000) * 1e3)
+    assert 32.0 <= per_sm_clk <= 128.0, per_sm_clk
+    ctx.close()
+
+
 def test_padded_strides_leave_the_padding_alone(gk):
     """Caches whose pages, K/V planes and layers are separated by padding: pack reads
     only slab bytes, restore writes only slab bytes."""
