@@ -54,7 +54,8 @@ def parse_args():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress", "longwindow", "digest", "layerwise"],
+    ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress", "longwindow", "digest", "layerwise",
+                                                            "latency", "records"],
                     help="gqa7b is the headline workload (full JSON line); the others print a shorter line "
                          "with the save and restore phases of that workload's shape")
     ap.add_argument("--window-blocks", type=int, default=48,
@@ -67,6 +68,10 @@ def parse_args():
     ap.add_argument("--unfused", action="store_true",
                     help="restore with a verify launch, a compare launch and a commit launch instead of the fused "
                          "kernel (the kernels gk_verify and gk_commit run; for profiling)")
+    ap.add_argument("--tokens", type=int, default=0,
+                    help="latency: restore one block of this many tokens (default: 256, 1,024, 5,200 and 24,018)")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="records: layers per page record of the gqa7b geometry (64 KiB per layer), 4 GiB of blobs")
     ap.add_argument("--tune", default="", help="tuning keys for the headline context, key=value[,key=value...]")
     ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the one-step-at-a-time end-to-end leg")
     ap.add_argument("--e2e-pipelined-steps", type=int, default=10,
@@ -799,7 +804,7 @@ def shape_of(synth, name, blocks=0):
     raise ValueError(name)
 
 
-def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0):
+def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0, layers=0):
     """Save and restore phases of one workload shape, each timed on its own over `steps`
     calls (the damage the configuration prescribes is applied between the two, so the
     restore is timed with it in place).  Returns a record for the bench line."""
@@ -808,6 +813,12 @@ def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0):
     import paper_2609_39358_b200 as gk
 
     w, lens, dst_pages, ids = shape_of(synth, name, blocks)
+    if layers:
+        # small page records: the gqa7b geometry with fewer layers per record, about 4 GiB of blobs
+        import dataclasses
+        w = dataclasses.replace(w, layers=layers)
+        lens = [4096 * (32 // layers) // 2] * 16 if layers < 32 else [4096] * 8
+        dst_pages = sum(-(-n // w.page_tokens) for n in lens)
     host_tier = name.endswith("_host")
     dtype = gk.GK_BF16 if w.dtype == "bf16" else gk.GK_FP8_E4M3
     flags = gk.GK_FLAG_SINGLE_PASS if single_pass else 0
@@ -999,13 +1010,29 @@ def latency_cases(device, token_counts=(256, 1024, 5200, 24018), reps=15):
     return out
 
 
+def run_latency(args):
+    import torch
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    cases = latency_cases(device, (args.tokens,) if args.tokens else (256, 1024, 5200, 24018),
+                          reps=max(3, min(args.steps, 15)))
+    first = next(iter(cases.values()))
+    line = {"metric": "restore of one block, device time per call", "value": first["restore_us_median"], "unit": "us",
+            "n_gpus": 1, "steps": max(3, min(args.steps, 15)), "warmup": 3, "ms_per_step": first["restore_us_median"] / 1e3,
+            "higher_is_better": False, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": "latency: gqa7b geometry, one block per call, L2 flushed before every call"},
+            "latency": cases}
+    print(json.dumps(line), flush=True)
+
+
 def run_other_workload(args):
     import torch
     device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
     torch.cuda.set_device(device)
-    name = {"stress": "stress_wave"}.get(args.workload, args.workload)
+    name = {"stress": "stress_wave", "records": "gqa7b"}.get(args.workload, args.workload)
     rec = workload_case(name, device, steps=max(args.steps, 1) if args.steps < 50 else 10, warmup=max(args.warmup, 3),
-                        single_pass=args.single_pass, blocks=args.blocks)
+                        single_pass=args.single_pass, blocks=args.blocks,
+                        layers=args.layers if args.workload == "records" else 0)
     pm, rm = rec["save_ms"]["median"], rec["restore_ms"]["median"]
     line = {"metric": METRIC, "value": rec["restore_useful"]["gbs"], "unit": UNIT, "n_gpus": 1,
             "steps": rec["restore_ms"]["n"], "warmup": max(args.warmup, 3), "ms_per_step": pm + rm,
@@ -1279,6 +1306,8 @@ def main():
         run_digest(args)
     elif args.workload == "layerwise":
         run_layerwise(args)
+    elif args.workload == "latency":
+        run_latency(args)
     elif args.workload != "gqa7b" or args.single_pass:
         run_other_workload(args)
     else:

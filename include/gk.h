@@ -165,6 +165,9 @@ typedef struct {
                                          context (each one synchronises the device): stays constant once
                                          gk_ctx_reserve has sized everything */
     uint64_t calls_restore_stream;    /* its windows are counted in calls_restore_host as well */
+    uint64_t quartet_launches;        /* packing and fused-restore launches that reduced one page record per
+                                         warp, four pages to a work item (small records in large calls; tuning
+                                         key "quad") */
 } gk_stats;
 
 /* Sizes of a block of n_tokens (Section 2.2: one record per block).  Either output may be NULL. */
@@ -424,7 +427,11 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * "test_drop_verify" (tests only: with value k > 0 the fused restore kernel
  * verifies nothing of the jobs k-1, k, ..., so that the commit waits of exactly
  * those jobs run into their limit and the time-out handling can be checked
- * without hanging or faulting the GPU), and in the bounds-checked build only
+ * without hanging or faulting the GPU), "quad" (page quartets: 0, the default:
+ * packing and fused-restore launches of at least 8 pages per resident CTA whose
+ * page records are at most 256 KiB reduce one record per warp instead of one per
+ * CTA -- a quarter of the per-thread checksum epilogues per byte; 1 = never;
+ * 2 = in every such launch, whatever its size), and in the bounds-checked build only
  * "debug_extent_cut" (tests: cache extents are taken to be this many bytes smaller
  * than they are, so that a perfectly valid access to the last page is refused and
  * the reporting can be checked without any access outside an object). */

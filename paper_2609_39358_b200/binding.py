@@ -62,7 +62,7 @@ class CStats(ctypes.Structure):
                 ("calls_restore_host", ctypes.c_uint64), ("jobs", ctypes.c_uint64), ("pages", ctypes.c_uint64),
                 ("bytes_blob", ctypes.c_uint64), ("kernels_launched", ctypes.c_uint64),
                 ("device_wait_expired", ctypes.c_uint32), ("allocations", ctypes.c_uint32),
-                ("calls_restore_stream", ctypes.c_uint64)]
+                ("calls_restore_stream", ctypes.c_uint64), ("quartet_launches", ctypes.c_uint64)]
 
 
 class CWindowBlock(ctypes.Structure):
@@ -283,6 +283,13 @@ class Context:
         if rc != GK_OK:
             raise GkError(rc, "gk_ctx_create")
         self._h = h
+        # GK_TUNING="key=value,key=value": tuning keys applied to every new context of the process
+        # (gk_ctx_set_tuning; e.g. quad=2 makes every pack and fused restore use page quartets)
+        for kv in filter(None, os.environ.get("GK_TUNING", "").split(",")):
+            key, _, value = kv.partition("=")
+            rc = self._lib.gk_ctx_set_tuning(self._h, key.strip().encode(), int(value))
+            if rc != GK_OK:
+                raise GkError(rc, f"GK_TUNING: {kv}")
 
     def __enter__(self):
         return self

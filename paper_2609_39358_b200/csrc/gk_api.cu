@@ -21,8 +21,10 @@
 #ifndef GK_CRC_NT
 #define GK_CRC_NT 128
 #endif
-// Ring shapes below are measured optima on B200 (8 GiB GQA-7B-like batch): with 16 KiB x 3
-// stages pack runs at 6.4 TB/s (8 KiB x 6: 6.0, 16 KiB x 2: 4.9, x 4: 6.0, x 5: 5.9 TB/s).
+// Ring shapes below are measured on B200.  Packing with 16 KiB x 5 stages (8 GiB of 2 MiB records:
+// 2.62 ms against 2.65 ms with 3 stages; 4 GiB of 64 KiB records as page quartets: 1.30 against
+// 1.43 ms -- the loader's look-ups at the start of every item need the deeper ring); the verifying
+// kernels are bound by the integer pipe and do with 3.
 #ifndef GK_CRC_STAGE
 #define GK_CRC_STAGE 16384
 #endif
@@ -33,7 +35,7 @@
 #define GK_PACK_STAGE GK_CRC_STAGE
 #endif
 #ifndef GK_PACK_STAGES
-#define GK_PACK_STAGES GK_CRC_STAGES
+#define GK_PACK_STAGES 5
 #endif
 #ifndef GK_VERIFY_MINB
 #define GK_VERIFY_MINB 2
@@ -100,6 +102,7 @@ struct gk_ctx {
     int device = 0;
     int sm_count = 0;
     int occ_verify = 0, occ_pack = 0, occ_commit = 0, occ_fused = 0, occ_single = 0;
+    uint32_t quad_mode = 0;      // page quartets: 0 = where they pay, 1 = never, 2 = wherever they are possible
     uint64_t *d_thread_const = nullptr;
     bool fused = true;           // restore runs verify and commit in one launch
     unsigned long long wait_limit_ns = kWaitLimitNs;
@@ -267,9 +270,37 @@ uint64_t items_wanted(const gk_ctx *c, int occ) { return 2ull * (uint64_t)c->sm_
 // Tiling of the CRC modes for a call of total_pages pages.  Large calls use one
 // segment per page (the per-thread epilogue is paid once per page); small calls
 // cut pages into segments of at least two granules so that every SM gets work.
-Tiling crc_tiling(const gk_ctx *c, uint32_t stage_bytes, uint64_t total_pages, int occ, bool overlap_jobs = false)
+//
+// Page quartets (`quad_for`: the call is a pack or a fused restore): records of at most
+// 256 KiB in a call with at least two quartets for every resident CTA are reduced one per
+// WARP instead of one per CTA, four pages to a work item (see Tiling).
+enum QuadUse { kNoQuad = 0, kQuadPack = 1, kQuadRestore = 2 };
+
+bool quad_wanted(const gk_ctx *c, QuadUse quad_for, uint64_t total_pages, int occ)
+{
+    if (quad_for == kNoQuad || c->quad_mode == 1u || c->seg_granules) return false;
+    if (quad_for == kQuadPack && c->gd.S != 0u) return false;  // scale values are gathered by a whole warp per record
+    if (c->quad_mode == 2u) return true;
+    return c->gd.R <= (256u << 10) && total_pages >= 8ull * (uint64_t)c->sm_count * (uint64_t)occ;
+}
+
+uint32_t crc_items(const Tiling &tl, uint64_t pages)
+{
+    return tl.quad ? (uint32_t)((pages + 3) / 4) : (uint32_t)pages * tl.nseg_max;
+}
+
+Tiling crc_tiling(const gk_ctx *c, uint32_t stage_bytes, uint64_t total_pages, int occ, bool overlap_jobs = false,
+                  QuadUse quad_for = kNoQuad)
 {
     Tiling t;
+    if (quad_wanted(c, quad_for, total_pages, occ)) {
+        t.quad = 1u;
+        t.stage_bytes = stage_bytes / 4;   // one record's part of a stage
+        t.gran_bytes = 32u * 256u;         // 8 shift-register steps of 8 words for each of 32 threads
+        t.seg_tiles = (uint32_t)((c->gd.R + t.gran_bytes - 1) / t.gran_bytes) * (t.gran_bytes / t.stage_bytes);
+        t.nseg_max = 1;
+        return t;
+    }
     t.stage_bytes = stage_bytes;
     t.gran_bytes = VerifyCfg::kGran;
     const uint32_t gran_full = (uint32_t)((c->gd.R + t.gran_bytes - 1) / t.gran_bytes);
@@ -603,7 +634,7 @@ cudaError_t launch_streaming(gk_ctx *c, Kernel kernel, uint32_t grid, int thread
     return cudaLaunchKernelEx(&cfg, kernel, Q);
 }
 
-template <class Cfg, int MODE, int NT, int SB, int ST, int MINB>
+template <class Cfg, int MODE, int NT, int SB, int ST, int MINB, bool QUAD = false>
 int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
 {
     const uint32_t items = MODE == kCommit ? P.n_items_c : P.n_items;
@@ -621,9 +652,10 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
     else Q.ctr_base_v = c->ctr_next[0];
     Q.trace = c->trace;
     c->ctr_next[ci] += draws_of(items, grid, true);
-    GK_CUDA(c, launch_streaming(c, stream_kernel<MODE, NT, SB, ST, MINB>, grid, Cfg::kThreads, Cfg::kSmemBytes, st, Q));
+    GK_CUDA(c, launch_streaming(c, stream_kernel<MODE, NT, SB, ST, MINB, QUAD>, grid, Cfg::kThreads, Cfg::kSmemBytes, st, Q));
     if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
+    if (QUAD) c->stats.quartet_launches++;
     return GK_OK;
 }
 
@@ -633,6 +665,9 @@ int launch_verify(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 }
 int launch_pack(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
+    if (P.tl.quad)
+        return launch_stream<PackCfg, kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB, true>(c, c->occ_pack, P,
+                                                                                                            st);
     return launch_stream<PackCfg, kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>(c, c->occ_pack, P, st);
 }
 // single-pass restore; per-kernel timing books it under "restore" (index 3)
@@ -671,11 +706,17 @@ int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
     // the verify side draws every item, the commit side takes the first one of each CTA without drawing
     c->ctr_next[0] += draws_of(P.n_items, grid, false);
     c->ctr_next[1] += draws_of(P.n_items_c, grid, true);
-    GK_CUDA(c, launch_streaming(c, restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE,
-                                                  GK_FUSED_CSTAGES, GK_FUSED_MINB>,
-                                grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st, Q));
+    if (P.tl.quad)
+        GK_CUDA(c, launch_streaming(c, restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE,
+                                                      GK_FUSED_CSTAGES, GK_FUSED_MINB, true>,
+                                    grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st, Q));
+    else
+        GK_CUDA(c, launch_streaming(c, restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE,
+                                                      GK_FUSED_CSTAGES, GK_FUSED_MINB>,
+                                    grid, FusedCfg::kThreads, FusedCfg::kSmemBytes, st, Q));
     if (slot) GK_CUDA(c, cudaEventRecord(slot->b, st));
     c->stats.kernels_launched++;
+    if (P.tl.quad) c->stats.quartet_launches++;
     return GK_OK;
 }
 
@@ -918,6 +959,7 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
     c->sm_count = prop.multiProcessorCount;
 
     // every streaming kernel: shared-memory size, then how many CTAs of it an SM holds
+    int occ_quad[2] = {0, 0};
     auto prepare = [&](auto *kernel, int threads, size_t smem, int *occ) {
         return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess &&
                cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, kernel, threads, smem) == cudaSuccess && *occ >= 1;
@@ -931,7 +973,14 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
         !prepare(stream_kernel<kCommit, 0, GK_COPY_STAGE, GK_COPY_STAGES, GK_COPY_MINB>, CommitCfg::kThreads,
                  CommitCfg::kSmemBytes, &c->occ_commit) ||
         !prepare(stream_kernel<kSingle, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB>, SingleCfg::kThreads,
-                 SingleCfg::kSmemBytes, &c->occ_single)) {
+                 SingleCfg::kSmemBytes, &c->occ_single) ||
+        // the page-quartet forms of the packing and of the fused kernel: same block shape, same occupancy
+        !prepare(stream_kernel<kPack, GK_CRC_NT, GK_PACK_STAGE, GK_PACK_STAGES, GK_PACK_MINB, true>, PackCfg::kThreads,
+                 PackCfg::kSmemBytes, &occ_quad[0]) ||
+        !prepare(restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES, GK_FUSED_MINB,
+                                true>,
+                 FusedCfg::kThreads, FusedCfg::kSmemBytes, &occ_quad[1]) ||
+        occ_quad[0] < c->occ_pack || occ_quad[1] < c->occ_fused) {
         cudaGetLastError();
         return bail(GK_ERR_CUDA);
     }
@@ -945,10 +994,13 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
     if (cudaMemcpy(c->d_init_term, init.data(), init.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess ||
         cudaMemset(c->d_error, 0, 256) != cudaSuccess)
         return bail(GK_ERR_CUDA);
-    std::vector<uint64_t> tc(GK_CRC_NT + 2 * (GK_CRC_NT / 32));
+    std::vector<uint64_t> tc(QuadConst<GK_CRC_NT>::kOver0 + 2);
     for (int t = 0; t < GK_CRC_NT; ++t) tc[t] = gf_xpow(32ull * (GK_CRC_NT - 1 - t) + 64ull);
     for (int w = 0; w < GK_CRC_NT / 32; ++w)  // the two words that stick out above warp w
         for (int i = 0; i < 2; ++i) tc[GK_CRC_NT + 2 * w + i] = gf_xpow(1024ull * (GK_CRC_NT / 32 - w) + 64ull + 32ull * i);
+    // page quartets: a record reduced by one warp alone
+    for (int t = 0; t < 32; ++t) tc[QuadConst<GK_CRC_NT>::kLane0 + t] = gf_xpow(32ull * (31 - t) + 64ull);
+    for (int i = 0; i < 2; ++i) tc[QuadConst<GK_CRC_NT>::kOver0 + i] = gf_xpow(1024ull + 64ull + 32ull * i);
     if (cudaMalloc(&c->d_thread_const, tc.size() * 8) != cudaSuccess) return bail(GK_ERR_NOMEM);
     if (cudaMemcpy(c->d_thread_const, tc.data(), tc.size() * 8, cudaMemcpyHostToDevice) != cudaSuccess)
         return bail(GK_ERR_CUDA);
@@ -1010,6 +1062,7 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     else if (!strcmp(key, "commit_reverse")) c->commit_reverse = value != 0;
     else if (!strcmp(key, "l2_hints")) c->l2_hints = value;
     else if (!strcmp(key, "commit_items_per_cta")) c->commit_items_per_cta = value ? value : 1u;
+    else if (!strcmp(key, "quad")) c->quad_mode = value <= 2u ? value : 0u;
 #ifdef GK_DEBUG
     else if (!strcmp(key, "debug_extent_cut")) c->debug_extent_cut = value;
 #endif
@@ -1067,7 +1120,7 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
 
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
-    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_pack);
+    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_pack, false, kQuadPack);
     const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     WorkDev w = make_work(c, l, n_jobs, (uint32_t)pages, tl);
@@ -1084,7 +1137,7 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
     P.cache = cd;
     P.w = w;
     P.tl = tl;
-    P.n_items = (uint32_t)pages * tl.nseg_max;
+    P.n_items = crc_items(tl, pages);
     P.inline_final = 1u;  // checksums are written by the CTA that delivers a page's last segment
     if ((rc = launch_pack(c, P, st)) != GK_OK) return rc;
     c->stats.calls_pack++;
@@ -1128,7 +1181,7 @@ int gk_page_checksums(gk_ctx *c, const void *blob_dev, uint32_t n_tokens, uint64
     P.g = c->gd;
     P.w = w;
     P.tl = tl;
-    P.n_items = (uint32_t)pages * tl.nseg_max;
+    P.n_items = crc_items(tl, pages);
     if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
     if ((rc = launch_finalize(c, w, tl, 1, nullptr, st)) != GK_OK) return rc;
     c->stats.pages += pages;
@@ -1152,7 +1205,7 @@ static int enqueue_verify_commit(gk_ctx *c, WorkDev w, const CacheDev &cd, const
     P.first_bad_out = first_bad_dev;
     P.tl = tlv;
     P.tlc = tlc;
-    P.n_items = n_pages * tlv.nseg_max;
+    P.n_items = crc_items(tlv, n_pages);
     P.n_items_c = n_pages * tlc.nseg_max;
     P.commit_reverse = c->commit_reverse ? 1u : 0u;
     P.l2_hints = c->l2_hints;
@@ -1195,7 +1248,8 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
     const bool single = (c->gd.flags & GK_FLAG_SINGLE_PASS) && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
     const bool fused = !single && c->fused && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
     const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages,
-                                  single ? c->occ_single : fused ? c->occ_fused : c->occ_verify, fused && n_jobs > 1);
+                                  single ? c->occ_single : fused ? c->occ_fused : c->occ_verify, fused && n_jobs > 1,
+                                  fused ? kQuadRestore : kNoQuad);
     const Tiling tlc = commit_tiling(c, GK_COPY_STAGE, pages, fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
@@ -1262,7 +1316,7 @@ int gk_verify(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *ds
         P.g = c->gd;
         P.w = w;
         P.tl = tlv;
-        P.n_items = (uint32_t)pages * tlv.nseg_max;
+        P.n_items = crc_items(tlv, pages);
         if ((rc = launch_verify(c, P, st)) != GK_OK) return rc;
         if ((rc = launch_finalize(c, w, tlv, 0, nullptr, st)) != GK_OK) return rc;
     }
@@ -1335,7 +1389,8 @@ static int restore_host_impl(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, con
     const bool single = (c->gd.flags & GK_FLAG_SINGLE_PASS) && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
     const bool fused = c->fused && !single && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
     const int occ = single ? c->occ_single : fused ? c->occ_fused : c->occ_verify;
-    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages_per_launch, occ, fused && n_jobs > batch_end.size());
+    const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages_per_launch, occ, fused && n_jobs > batch_end.size(),
+                                  fused ? kQuadRestore : kNoQuad);
     const Tiling tlc = commit_tiling(c, GK_COPY_STAGE, pages_per_launch, fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
@@ -1443,7 +1498,8 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
     if ((rc = make_host_plan(c, jobs, n_jobs, false, hp)) != GK_OK) return rc;
 
     uint64_t pages = hp.pages, bytes = 0;
-    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, (pages + hp.batch_end.size() - 1) / hp.batch_end.size(), c->occ_pack);
+    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, (pages + hp.batch_end.size() - 1) / hp.batch_end.size(), c->occ_pack,
+                                 false, kQuadPack);
     const WsLayout l = ws_layout(n_jobs, pages, tl.nseg_max, 0);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     if ((rc = upload_jobs(c, jobs, n_jobs, l, tl, hp.blob_dev.data(), hp.sums_dev.data(), true, st, &pages, &bytes)) != GK_OK)
@@ -1468,7 +1524,7 @@ int gk_pack_host(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n_
         P.cache = cd;
         P.w = wb;
         P.tl = tl;
-        P.n_items = npages * tl.nseg_max;
+        P.n_items = crc_items(tl, npages);
         P.inline_final = 1u;
         if ((rc = launch_pack(c, P, st)) != GK_OK) return rc;
         GK_CUDA(c, cudaEventRecord(c->ev_copied[slot], st));

@@ -77,7 +77,9 @@ struct WorkDev {
     uint32_t *error;              // sticky: non-zero once a bounded wait has run out
     const uint64_t *init_term;    // [page_tokens+1] ones * x^(8*len(t)) mod P
     const uint64_t *thread_const; // [NT] x^(32*(NT-1-t)+64) mod P, then for each warp w of NT/32 the constants
-                                  // of the two words above it: x^(1024*(NT/32-w)+64) and that times x^32
+                                  // of the two words above it: x^(1024*(NT/32-w)+64) and that times x^32;
+                                  // then the same for a record that ONE warp reduces (page quartets): 32
+                                  // lane constants x^(32*(31-lane)+64) and x^(1024+64), x^(1024+96)
     const uint64_t *seg_pow;      // [nseg_max][2] (x^(8*segment bytes))^k mod P and that times x^32: place
                                   // the two halves of a segment remainder
     unsigned long long wait_limit_ns;  // time limit of every device-side wait
@@ -87,11 +89,17 @@ struct WorkDev {
 // zero-padded AT THE FRONT to a multiple of gran_bytes (leading zeros do not
 // change a remainder), cut into tiles of stage_bytes and grouped into segments
 // of seg_tiles tiles; the short segment, if any, is the first one.
+//
+// Page quartets (quad = 1; small records in large calls): a work item is FOUR
+// consecutive pages of the launch, one per consumer warp, every record whole
+// (one segment); stage_bytes is then the quarter of a shared-memory stage that
+// one record's tile takes, and a launch of n pages has (n + 3) / 4 items.
 struct Tiling {
     uint32_t stage_bytes;  // a power of two
     uint32_t gran_bytes;   // a power of two, a multiple of stage_bytes
     uint32_t seg_tiles;
     uint32_t nseg_max;   // segments of a full page
+    uint32_t quad = 0;
 };
 
 struct PageShape {

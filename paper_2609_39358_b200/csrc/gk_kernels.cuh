@@ -298,6 +298,21 @@ struct Item {
     int32_t phys;
 };
 
+// Page quartets: what the roles of a CTA need to know about an item of four
+// pages, one per consumer warp, in the place of an Item.  Everything else about
+// a page follows from (job, page) and the tables of the call.
+struct QuadPages {
+    uint32_t j[4];  // owning job of each page, or kNoJob: this warp's result is dropped
+    uint32_t p[4];  // page index within the job
+};
+struct QuadItem {
+    uint32_t tile_count;  // tiles of the quartet (those of its longest record)
+    uint32_t reserved;
+    QuadPages pages;
+};
+static_assert(sizeof(QuadItem) <= sizeof(Item), "a quartet must fit an item slot");
+static_assert(sizeof(QuadPages) == 32, "the quartet's pages take the item copy's place in a hand-over slot");
+
 template <int MODE, int NT, int STAGE_BYTES, int STAGES>
 struct StreamCfg {
     static constexpr bool kCrc = (MODE != kCommit);
@@ -325,7 +340,7 @@ struct StreamParams {
     WorkDev w;
     Tiling tl;        // tiling of the CRC modes (verify, pack)
     Tiling tlc;       // tiling of the commit mode
-    uint32_t n_items;    // CRC work items: pages of the launch * tl.nseg_max
+    uint32_t n_items;    // CRC work items: pages of the launch * tl.nseg_max (page quartets: a quarter of the pages)
     uint32_t n_items_c;  // commit work items: pages of the launch * tlc.nseg_max
     uint32_t fused;      // 1: verify and commit run in one launch; commit waits per job
     uint32_t inline_final;  // 1: the CTA that delivers a page's last segment finalizes the page itself
@@ -736,17 +751,20 @@ __device__ __forceinline__ void thread_poly(const uint32_t (&R)[64], uint32_t &a
 
 // w(x) * c(x) mod P for a 32-bit w: Horner over the bits of w, 32 steps of
 // "times x, fold, add c if the bit is set" on a 64-bit value in two registers.
+// The loop stays a loop (four steps per trip): the steps depend on one another
+// anyway, and the instruction cache has better uses than 32 copies of them.
 __device__ __forceinline__ uint64_t gf_mul32(uint32_t w, uint64_t c)
 {
     const uint32_t cl = (uint32_t)c, ch = (uint32_t)(c >> 32);
     constexpr uint32_t pl = (uint32_t)kPoly, ph = (uint32_t)(kPoly >> 32);
     uint32_t rl = 0u, rh = 0u;
-#pragma unroll
-    for (int i = 31; i >= 0; --i) {
+#pragma unroll 4
+    for (int i = 0; i < 32; ++i) {
         const uint32_t m = (uint32_t)((int32_t)rh >> 31);
         rh = __funnelshift_l(rl, rh, 1);
         rl <<= 1;
-        const uint32_t b = (uint32_t)((int32_t)(w << (31 - i)) >> 31);
+        const uint32_t b = (uint32_t)((int32_t)w >> 31);
+        w <<= 1;
         rl ^= (m & pl) ^ (b & cl);
         rh ^= (m & ph) ^ (b & ch);
     }
@@ -790,10 +808,12 @@ struct RingPos {
 
 // The eight 8-word steps of one granule (after which the registers are back in
 // natural order).  Every kSps steps a new stage is awaited and the finished one
-// is handed back to the loader.
-template <int U, int MODE, int NT, int STAGE_BYTES, int STAGES>
+// is handed back to the loader.  NT threads share TILE_BYTES of every stage (the
+// whole stage, or with page quartets the warp's quarter of it: `smem` then points
+// at that quarter of stage 0 and `tid` is the lane).
+template <int U, int MODE, int NT, int STAGE_BYTES, int STAGES, int TILE_BYTES>
 struct GranuleSteps {
-    static constexpr int kSps = STAGE_BYTES / (NT * 32);  // 8-word steps per stage
+    static constexpr int kSps = TILE_BYTES / (NT * 32);  // 8-word steps per stage
     static __device__ __forceinline__ void run(uint32_t (&R)[64], const uint8_t *smem, uint32_t full0, uint32_t empty0,
                                                RingPos &pos, volatile uint32_t *abort_flag, uint32_t *error,
                                                unsigned long long limit_ns, int tid, int lane)
@@ -809,12 +829,12 @@ struct GranuleSteps {
             if (lane == 0) mbar_arrive(empty0 + 8u * pos.stage);
             pos.template advance<STAGES>();
         }
-        GranuleSteps<U + 1, MODE, NT, STAGE_BYTES, STAGES>::run(R, smem, full0, empty0, pos, abort_flag, error, limit_ns,
-                                                                tid, lane);
+        GranuleSteps<U + 1, MODE, NT, STAGE_BYTES, STAGES, TILE_BYTES>::run(R, smem, full0, empty0, pos, abort_flag, error,
+                                                                            limit_ns, tid, lane);
     }
 };
-template <int MODE, int NT, int STAGE_BYTES, int STAGES>
-struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES> {
+template <int MODE, int NT, int STAGE_BYTES, int STAGES, int TILE_BYTES>
+struct GranuleSteps<8, MODE, NT, STAGE_BYTES, STAGES, TILE_BYTES> {
     static __device__ __forceinline__ void run(uint32_t (&)[64], const uint8_t *, uint32_t, uint32_t, RingPos &,
                                                volatile uint32_t *, uint32_t *, unsigned long long, int, int)
     {
@@ -930,10 +950,21 @@ struct Finisher {
     uint64_t kover = 0;  // lanes 0 .. 2*NT/32-1: constants of the words above the warps
 };
 
+// Where the constants of a record reduced by one warp (page quartets) start in thread_const.
 template <int NT>
+struct QuadConst {
+    static constexpr int kLane0 = NT + 2 * (NT / 32);  // 32 lane constants
+    static constexpr int kOver0 = kLane0 + 32;         // constants of the two words above the warp
+};
+
+template <int NT, bool QUAD = false>
 __device__ __forceinline__ void finisher_init(const StreamParams &P, Finisher &fin, int lane)
 {
-    if (NT > 0 && lane < 2 * (NT / 32)) fin.kover = P.w.thread_const[NT + lane];
+    if (QUAD) {
+        if (lane < 8) fin.kover = P.w.thread_const[QuadConst<NT>::kOver0 + (lane & 1)];
+    } else if (NT > 0 && lane < 2 * (NT / 32)) {
+        fin.kover = P.w.thread_const[NT + lane];
+    }
 }
 
 // Has the next segment been handed over?  (Every lane may ask; use finisher_ready for a warp-wide answer.)
@@ -1026,9 +1057,89 @@ __device__ __forceinline__ HandOver hand_over_of(const Item &it)
     return h;
 }
 
+// Page quartets: the four consumer warps hand over one whole record each (hand-over slot as
+// above, with the quartet's pages in the place of the item copy).  Lanes 0..7 multiply the
+// words above the warps by their constants, lanes 0..3 then finish one page each: final xor,
+// reflection, and either the checksum is written (pack) or compared with the stored one and
+// the page counted in job_done.
+//
+// `ahead` (pack, where a consumer warp does this between two records): what lanes 0..3 need
+// from the tables of the call, fetched by them when the quartet began, so that no load from
+// global memory stands between the end of the records and the next quartet.
+struct QuadAhead {
+    uint64_t *sum = nullptr;  // the page's checksum word, or null: no page in this lane
+    uint64_t init = 0;        // the term of the all-ones initial register for the page's length
+};
+
+__device__ __forceinline__ QuadAhead quad_ahead(const StreamParams &P, const QuadPages &pg, int lane)
+{
+    QuadAhead a;
+    if (lane < 4 && pg.j[lane] != kNoJob) {
+        const JobDev jb = P.w.jobs[pg.j[lane]];
+        a.sum = jb.checksums + pg.p[lane];
+        a.init = P.w.init_term[page_fill(P.g, jb, pg.p[lane])];
+    }
+    return a;
+}
+
+template <int MODE>
+__device__ __forceinline__ void finish_quad(const StreamParams &P, const Ring &ring, Finisher &fin,
+                                            const QuadPages &pg, uint32_t taken, volatile uint32_t *abort_flag,
+                                            int lane, const QuadAhead *ahead = nullptr)
+{
+    static_assert(MODE == kVerify || MODE == kPack, "page quartets: pack and verify only");
+    const uint32_t par = fin.done & 1u;
+    const uint64_t *slot = ring.red + kHandOverWords * par;
+    const uint32_t *oslot = reinterpret_cast<const uint32_t *>(slot + 4);
+    uint64_t tot = 0;
+    if (lane < 8) tot = gf_mul32(oslot[lane], fin.kover);
+    tot ^= __shfl_xor_sync(0xffffffffu, tot, 1);                                 // both words of a warp
+    const uint64_t above = __shfl_sync(0xffffffffu, tot, (2 * lane) & 31);       // lane w: those of warp w
+    uint32_t j = kNoJob, p = 0u;
+    uint64_t r = 0;
+    if (lane < 4) {
+        j = pg.j[lane];
+        p = pg.p[lane];
+        r = slot[lane] ^ above;
+    }
+    __syncwarp();
+    if (taken != 0u && lane == 0) mbar_arrive(taken);  // the slot has been read: it may be used again
+#ifndef GK_DEBUG
+    if (MODE == kPack && ahead != nullptr && P.inline_final) {
+        if (ahead->sum) *ahead->sum = __brevll(r ^ ahead->init ^ ~0ull);
+        __syncwarp();
+        ++fin.done;
+        return;
+    }
+#endif
+    if (j != kNoJob) {
+        const JobDev jb = P.w.jobs[j];
+        if (!P.inline_final) {
+            red_xor_u64(P.w.page_acc + jb.page_base + p, r);
+        } else {
+            uint64_t *sum = jb.checksums + p;
+#ifdef GK_DEBUG
+            const bool sum_ok = debug_ok(P, kDbgSums, 2u, sum, 8u, jb.checksums, 8ull * jb.n_pages);
+#else
+            constexpr bool sum_ok = true;
+#endif
+            const uint64_t crc = __brevll(r ^ P.w.init_term[page_fill(P.g, jb, p)] ^ ~0ull);
+            if (MODE == kPack) {
+                if (sum_ok) *sum = crc;
+            } else {
+                const uint64_t stored = sum_ok ? *sum : 0ull;
+                if (crc != stored || *abort_flag) atomicMin(&P.w.bad_crc[j], (int32_t)p);
+                red_add_release_u32(&P.w.job_done[j], 1u);  // nobody here waits for the count
+            }
+        }
+    }
+    __syncwarp();
+    ++fin.done;
+}
+
 // Finishes segments until the loader's count of admitted items has been reached (the count is
 // known once the loader has put the end mark into the ring).
-template <int MODE, int NT>
+template <int MODE, int NT, bool QUAD = false>
 __device__ __forceinline__ void finisher_drain(const StreamParams &P, const Ring &ring, Finisher &fin,
                                                volatile uint32_t *abort_flag, int lane)
 {
@@ -1058,19 +1169,24 @@ __device__ __forceinline__ void finisher_drain(const StreamParams &P, const Ring
         posted = __shfl_sync(0xffffffffu, posted ? 1 : 0, 0) != 0;  // one decision for the warp
         if (!posted) break;
         const uint32_t par = fin.done & 1u;
-        const HandOver it = *reinterpret_cast<const HandOver *>(ring.red + kHandOverWords * par + 8);
-        finish_segment<MODE, NT>(P, ring, fin, it, ring.tail0 + 8u * (2u + par), abort_flag, lane);
+        if constexpr (QUAD) {
+            const QuadPages pg = *reinterpret_cast<const QuadPages *>(ring.red + kHandOverWords * par + 8);
+            finish_quad<MODE>(P, ring, fin, pg, ring.tail0 + 8u * (2u + par), abort_flag, lane);
+        } else {
+            const HandOver it = *reinterpret_cast<const HandOver *>(ring.red + kHandOverWords * par + 8);
+            finish_segment<MODE, NT>(P, ring, fin, it, ring.tail0 + 8u * (2u + par), abort_flag, lane);
+        }
     }
 }
 
 // The role as a warp of its own (kernels whose storer warp, if any, has no time for it).
-template <int MODE, int NT>
+template <int MODE, int NT, bool QUAD = false>
 __device__ __forceinline__ void finisher_role(const StreamParams &P, const Ring &ring, volatile uint32_t *abort_flag,
                                               int lane)
 {
     Finisher fin;
-    finisher_init<NT>(P, fin, lane);
-    finisher_drain<MODE, NT>(P, ring, fin, abort_flag, lane);
+    finisher_init<NT, QUAD>(P, fin, lane);
+    finisher_drain<MODE, NT, QUAD>(P, ring, fin, abort_flag, lane);
 }
 
 // ------------------------------ loader role ------------------------------
@@ -1326,17 +1442,251 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
     GK_TRACE_EVT(P, 3, 2);
 }
 
+// ------------------------- page quartets: loader, storer -------------------------
+// Small records (tens of KiB) pay the per-thread epilogue of the checksum once per record
+// and NT threads, which costs as much as the record's main loop when the record is short.
+// With page quartets a work item is four consecutive pages of the launch and every
+// consumer warp reduces one WHOLE record on its own (32 threads per record: a quarter of
+// the epilogues per byte): a shared-memory stage holds one tile of STAGE_BYTES / 4 bytes
+// of each of the four records.  Lanes 0..3 of the loader (and of the storer) serve one page
+// each and issue its copies themselves.  Records of a quartet that are shorter than its
+// longest one (the last page of a job) get whole tiles of zeros in front; a page that is
+// not to be processed (missing job, bad table, past the end of the launch) has job kNoJob:
+// nothing is copied for it, its warp reduces whatever the stage holds and the result is
+// dropped.
+template <int MODE, int STAGE_BYTES, int STAGES, bool STATIC_FIRST>
+__device__ __forceinline__ void loader_role_quad(const StreamParams &P, uint32_t *ctr, uint32_t ctr_base,
+                                                 const Ring &ring, volatile uint32_t *abort_flag, int lane)
+{
+    static_assert(MODE == kVerify || MODE == kPack, "page quartets: pack and verify only");
+    constexpr uint32_t QB = STAGE_BYTES / 4;
+    uint32_t n = 0;      // tiles (stages) issued
+    uint32_t n_adm = 0;  // items admitted
+    uint64_t policy = 0;
+    const bool hint = MODE == kVerify && (P.l2_hints & 1u);
+    if (hint) policy = policy_evict_last();
+    GK_TRACE_EVT(P, 0, 1);
+    for (uint32_t item = STATIC_FIRST ? blockIdx.x : next_item<false>(ctr, ctr_base, lane); item < P.n_items;
+         item = next_item<STATIC_FIRST>(ctr, ctr_base, lane)) {
+        // lanes 0..3: one page each
+        uint32_t j = kNoJob, p = 0u, t = 0u, ntiles = 0u, pad = 0u;
+        int32_t phys = 0;
+        uint8_t *rec = nullptr;
+        const uint32_t local = item * 4u + (uint32_t)lane;
+        if (lane < 4 && local < P.w.total_pages) {
+            const uint32_t gp = P.w.page_begin + local;
+            const uint32_t jj = (uint32_t)P.w.page_job[gp];
+            const JobDev jb = P.w.jobs[jj];
+            bool skip = jb.missing || P.w.bad_range[jj] != kNoPage;
+            if (MODE == kVerify)
+                skip = skip || P.w.bad_dup[jj] != kNoPage || (P.test_drop_from != 0u && jj + 1u >= P.test_drop_from);
+            if (!skip) {
+                j = jj;
+                p = gp - jb.page_base;
+                const PageShape sh = page_shape(P.g, jb, p, P.tl);
+                t = sh.t;
+                ntiles = sh.ntiles;
+                pad = sh.pad;
+                rec = jb.blob + (uint64_t)p * P.g.R;
+                if (MODE == kPack) phys = jb.page_table[p];
+            }
+        }
+        uint32_t nmax = ntiles;  // 0 in the lanes without a page
+        nmax = max(nmax, __shfl_xor_sync(0xffffffffu, nmax, 1));
+        nmax = max(nmax, __shfl_xor_sync(0xffffffffu, nmax, 2));
+        nmax = __shfl_sync(0xffffffffu, nmax, 0);
+        if (nmax == 0u) continue;
+        pad += (nmax - ntiles) * QB;  // a shorter record starts later: whole tiles of zeros in front
+        GK_TRACE_EVT(P, 0, 2);
+        const uint32_t slot = n_adm % (uint32_t)(STAGES + 1);
+        ++n_adm;
+        const Chunks ch = chunks_of(P.g, t);
+        for (uint32_t k = 0; k < nmax; ++k, ++n) {
+            const uint32_t s = n % STAGES;
+            const uint32_t use = n / STAGES;
+            if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE,
+                                    P.w.wait_limit_ns);
+            if (k == 0u && lane < 4) {  // the stage's barrier publishes it with the tile
+                QuadItem *q = reinterpret_cast<QuadItem *>(ring.items + slot);
+                q->pages.j[lane] = j;
+                q->pages.p[lane] = p;
+                if (lane == 0) q->tile_count = nmax;
+            }
+            uint32_t lead = 0u, nreal = 0u;
+            uint64_t r0 = 0;
+            if (j != kNoJob) tile_range<(int)QB>(k, pad, lead, r0, nreal);
+            const uint32_t sbase = ring.stage0 + s * STAGE_BYTES;
+            uint8_t *sgen = ring.base + (size_t)s * STAGE_BYTES;
+#pragma unroll
+            for (int wq = 0; wq < 4; ++wq) {  // front padding, zeroed by all lanes
+                const uint32_t lw = __shfl_sync(0xffffffffu, lead, wq);
+                for (uint32_t o = lane * 16u; o < lw; o += 512u)
+                    *reinterpret_cast<uint4 *>(sgen + wq * QB + o) = make_uint4(0u, 0u, 0u, 0u);
+            }
+            uint32_t total = nreal;  // bytes the copies of this stage will deliver
+            total += __shfl_xor_sync(0xffffffffu, total, 1);
+            total += __shfl_xor_sync(0xffffffffu, total, 2);
+            __syncwarp();
+            uint32_t aborted = 0u;
+            const uint32_t bar = ring.full0 + 8u * s;
+            if (lane == 0) {
+                ring.tag[s] = make_uint2(slot, k);
+                aborted = *abort_flag;
+                if (!aborted) {
+                    if (total == 0u) mbar_arrive(bar);
+                    else mbar_arrive_expect_tx(bar, total);
+                }
+            }
+            aborted = __shfl_sync(0xffffffffu, aborted, 0);
+            if (!aborted && nreal > 0u) {  // lanes 0..3 that have a page
+                const uint32_t so0 = sbase + (uint32_t)lane * QB + lead;
+                if (MODE == kPack) {
+                    // no scale sections in this mode: the record is its data part
+                    uint64_t d0 = r0;
+                    const uint64_t d1 = d0 + nreal;
+                    uint32_t so = so0;
+                    uint32_t chunk = (uint32_t)(d0 / ch.len);
+                    uint32_t off = (uint32_t)(d0 - (uint64_t)chunk * ch.len);
+                    while (d0 < d1) {
+                        uint32_t nb = ch.len - off;
+                        if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
+                        if (nb == 0u) break;  // cannot happen with a valid geometry; never spin
+                        const uint8_t *ca = chunk_addr(P.cache, ch, chunk, phys, off);
+                        if (GK_DEBUG_OK(P, kDbgCache, 0u, ca, nb, P.cache.data, P.cache.data_extent) &&
+                            GK_DEBUG_OK(P, kDbgStage, 0u, (const void *)(uintptr_t)so, nb,
+                                        (const void *)(uintptr_t)sbase, STAGE_BYTES))
+                            bulk_g2s(so, ca, nb, bar);
+                        else
+                            mbar_complete_tx(bar, nb);
+                        d0 += nb;
+                        so += nb;
+                        ++chunk;
+                        off = 0u;
+                    }
+                } else {
+#ifdef GK_DEBUG
+                    const bool in_blob = debug_ok(P, kDbgBlob, 0u, rec + r0, nreal, P.w.jobs[j].blob,
+                                                  debug_blob_bytes(P, j)) &&
+                                         debug_ok(P, kDbgStage, 0u, (const void *)(uintptr_t)(lead + nreal), 0u, nullptr,
+                                                  QB);
+#else
+                    constexpr bool in_blob = true;
+#endif
+                    if (!in_blob) mbar_complete_tx(bar, nreal);
+                    else if (hint) bulk_g2s_hint(so0, rec + r0, nreal, bar, policy);
+                    else bulk_g2s(so0, rec + r0, nreal, bar);
+                }
+            }
+            __syncwarp();
+        }
+        GK_TRACE_EVT(P, 0, 3);
+    }
+    // tell the other roles of this CTA that there is no more work
+    {
+        const uint32_t s = n % STAGES;
+        const uint32_t use = n / STAGES;
+        if (use > 0u) mbar_wait(ring.empty0 + 8u * s, (use - 1u) & 1u, abort_flag, P.w.error, 0x100u | MODE,
+                                P.w.wait_limit_ns);
+        if (lane == 0) {
+            ring.tag[s] = make_uint2(kEndOfWork, 0u);
+            mbar_arrive(ring.full0 + 8u * s);
+            abort_flag[2] = n_adm;  // tells the finisher warp how many items there are
+        }
+        ++n;
+    }
+    GK_TRACE_EVT(P, 0, 4);
+    // before leaving: every load this CTA issued must have landed
+    if (lane == 0) {
+        for (uint32_t back = 0; back < (uint32_t)STAGES && back < n; ++back) {
+            const uint32_t m = n - 1u - back;
+            mbar_drain(ring.full0 + 8u * (m % STAGES), (m / STAGES) & 1u, P.w.wait_limit_ns);
+        }
+    }
+}
+
+// Pack with page quartets: lanes 0..3 write the tile of one record each into its blob.  Bulk
+// copy groups belong to the thread that issued them, so each of the four lanes commits and
+// awaits its own; lane 0 hands the stage back once all four have read it.
+template <int STAGE_BYTES, int STAGES>
+__device__ __forceinline__ void storer_role_quad(const StreamParams &P, const Ring &ring, volatile uint32_t *abort_flag,
+                                                 int lane)
+{
+    constexpr uint32_t QB = STAGE_BYTES / 4;
+    uint32_t n = 0;
+    bool live = false;  // this lane has a page of the current item
+    uint8_t *rec = nullptr;
+    uint32_t pad = 0u;
+#ifdef GK_DEBUG
+    uint32_t cur_j = 0u;
+#endif
+    for (;; ++n) {
+        const uint32_t s = n % STAGES;
+        bool ok = mbar_wait(ring.full0 + 8u * s, (n / STAGES) & 1u, abort_flag, P.w.error, 0x300u | kPack,
+                            P.w.wait_limit_ns);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;  // the CTA has given up: nothing more is stored (decided by the whole warp)
+        const uint2 tag = ring.tag[s];
+        if (tag.x == kEndOfWork) break;
+        GK_TRACE_EVT(P, 3, 0);
+        if (tag.y == 0u) {  // first tile of an item: where this lane's record lies
+            const QuadItem &q = *reinterpret_cast<const QuadItem *>(ring.items + tag.x);
+            live = false;
+            if (lane < 4 && q.pages.j[lane] != kNoJob) {
+                const JobDev jb = P.w.jobs[q.pages.j[lane]];
+                const uint32_t p = q.pages.p[lane];
+                const PageShape sh = page_shape(P.g, jb, p, P.tl);
+                pad = sh.pad + (q.tile_count - sh.ntiles) * QB;
+                rec = jb.blob + (uint64_t)p * P.g.R;
+                live = true;
+#ifdef GK_DEBUG
+                cur_j = q.pages.j[lane];
+#endif
+            }
+        }
+        if (live && *abort_flag == 0u) {
+            uint32_t lead, nreal;
+            uint64_t r0;
+            tile_range<(int)QB>(tag.y, pad, lead, r0, nreal);
+            if (nreal > 0u) {
+#ifdef GK_DEBUG
+                if (debug_ok(P, kDbgBlob, 3u, rec + r0, nreal, P.w.jobs[cur_j].blob, debug_blob_bytes(P, cur_j)))
+#endif
+                    bulk_s2g(rec + r0, ring.stage0 + s * STAGE_BYTES + (uint32_t)lane * QB + lead, nreal);
+            }
+        }
+        if (lane < 4) {
+            bulk_commit();
+            if (n > 0u) bulk_wait_read<1>();
+        }
+        __syncwarp();
+        if (lane == 0 && n > 0u) mbar_arrive(ring.empty0 + 8u * ((n - 1u) % STAGES));
+    }
+    if (lane < 4) bulk_wait_all();
+    __syncwarp();
+    if (lane == 0 && n > 0u) mbar_arrive(ring.empty0 + 8u * ((n - 1u) % STAGES));
+    GK_TRACE_EVT(P, 3, 2);
+}
+
 // ----------------------------- consumer role -----------------------------
 // NT threads.  Reduce each segment to one partial remainder per warp (see the
 // top of this file) and hand these over to the loader warp of the ring, which
 // finishes the segment (finish_segment) while the consumers start on the next.
-template <int MODE, int NT, int STAGE_BYTES, int STAGES, bool OWN_FINISHER>
+//
+// QUAD (page quartets): every warp reduces a record of its own -- 32 threads per
+// record, the warp's quarter of every stage -- and hands over that record's
+// remainder; nothing is merged across warps.
+template <int MODE, int NT, int STAGE_BYTES, int STAGES, bool OWN_FINISHER, bool QUAD = false>
 __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring &ring,
                                               volatile uint32_t *abort_flag, int tid, int warp, int lane)
 {
-    const uint64_t kt = P.w.thread_const[tid];
+    static_assert(!QUAD || NT == 128, "page quartets: four consumer warps");
+    constexpr int kRecThreads = QUAD ? 32 : NT;                         // threads that share a record
+    constexpr int kTileBytes = QUAD ? STAGE_BYTES / 4 : STAGE_BYTES;    // bytes of a stage they share
+    const uint64_t kt = P.w.thread_const[QUAD ? QuadConst<NT>::kLane0 + lane : tid];
+    const uint8_t *my_base = QUAD ? ring.base + (size_t)warp * kTileBytes : ring.base;
+    const int my_tid = QUAD ? lane : tid;
     Finisher fin;  // kernels without a finisher warp: consumer warp 0 finishes the segments itself
-    if (!OWN_FINISHER && warp == 0) finisher_init<NT>(P, fin, lane);
+    if (!OWN_FINISHER && warp == 0) finisher_init<NT, QUAD>(P, fin, lane);
     RingPos pos;
     uint32_t parity_red = 0;
     uint32_t n_done = 0;  // segments handed over so far
@@ -1344,7 +1694,7 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
     uint32_t trace_items = 0;
     unsigned long long tr_sum[4] = {0, 0, 0, 0}, tr_t0 = 0, tr_t1 = 0, tr_t2 = 0, tr_t3 = 0;
 #endif
-    constexpr int kTilesPerGran = (NT * 256) / STAGE_BYTES;
+    constexpr int kTilesPerGran = (kRecThreads * 256) / kTileBytes;
     for (;;) {
 #ifdef GK_TRACE
         tr_t0 = global_timer_ns();
@@ -1369,20 +1719,24 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
 #ifdef GK_TRACE
         tr_t1 = global_timer_ns();
 #endif
-        const uint32_t ngran = ring.items[slot].tile_count / kTilesPerGran;
+        const uint32_t ngran = (QUAD ? reinterpret_cast<const QuadItem *>(ring.items + slot)->tile_count
+                                     : ring.items[slot].tile_count) / kTilesPerGran;
+        QuadAhead ahead;
+        if (QUAD && !OWN_FINISHER && warp == 0)
+            ahead = quad_ahead(P, reinterpret_cast<const QuadItem *>(ring.items + slot)->pages, lane);
         uint32_t R[64];
 #pragma unroll
         for (int i = 0; i < 64; ++i) R[i] = 0u;
         for (uint32_t gi = 0; gi < ngran; ++gi)
-            GranuleSteps<0, MODE, NT, STAGE_BYTES, STAGES>::run(R, ring.base, ring.full0, ring.empty0, pos, abort_flag,
-                                                                P.w.error, P.w.wait_limit_ns, tid, lane);
+            GranuleSteps<0, MODE, kRecThreads, STAGE_BYTES, STAGES, kTileBytes>::run(
+                R, my_base, ring.full0, ring.empty0, pos, abort_flag, P.w.error, P.w.wait_limit_ns, my_tid, lane);
         GK_TRACE_EVT(P, 2, 1);
 #ifdef GK_TRACE
         tr_t2 = global_timer_ns();
 #endif
         // merge streams -> thread -> warp -> CTA
         uint32_t a0, a1, a2, over0, over1;
-        thread_poly<NT>(R, a0, a1, a2);
+        thread_poly<kRecThreads>(R, a0, a1, a2);
         const uint64_t v = warp_remainder(a0, a1, a2, kt, lane, over0, over1);
         uint64_t *rslot = ring.red + kHandOverWords * parity_red;
         uint32_t *oslot = reinterpret_cast<uint32_t *>(rslot + 4);  // [2 * NT / 32] words sticking out above the warps
@@ -1396,7 +1750,13 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
                 oslot[2 * warp] = over0;
                 oslot[2 * warp + 1] = over1;
                 // what the finisher needs to know about the item (its slot in the ring may be gone by then)
-                if (warp == 0) *reinterpret_cast<HandOver *>(rslot + 8) = hand_over_of(ring.items[slot]);
+                if (warp == 0) {
+                    if (QUAD)
+                        *reinterpret_cast<QuadPages *>(rslot + 8) =
+                            reinterpret_cast<const QuadItem *>(ring.items + slot)->pages;
+                    else
+                        *reinterpret_cast<HandOver *>(rslot + 8) = hand_over_of(ring.items[slot]);
+                }
                 mbar_arrive(ring.tail0 + 8u * parity_red);
             }
             GK_TRACE_EVT(P, 2, 2);
@@ -1411,7 +1771,13 @@ __device__ __forceinline__ void consumer_role(const StreamParams &P, const Ring 
             }
             asm volatile("bar.sync 1, %0;" ::"n"(NT) : "memory");
             GK_TRACE_EVT(P, 2, 2);
-            if (warp == 0) finish_segment<MODE, NT>(P, ring, fin, hand_over_of(ring.items[slot]), 0u, abort_flag, lane);
+            if (warp == 0) {
+                if constexpr (QUAD)
+                    finish_quad<MODE>(P, ring, fin, reinterpret_cast<const QuadItem *>(ring.items + slot)->pages, 0u,
+                                      abort_flag, lane, &ahead);
+                else
+                    finish_segment<MODE, NT>(P, ring, fin, hand_over_of(ring.items[slot]), 0u, abort_flag, lane);
+            }
         }
 #ifdef GK_TRACE
         tr_t3 = global_timer_ns();
@@ -1467,10 +1833,11 @@ __device__ __forceinline__ void ring_init(Ring &ring, uint8_t *base, uint64_t *b
 }
 
 // pack, verify-only and commit-only launches
-template <int MODE, int NT, int STAGE_BYTES, int STAGES, int MINB>
+template <int MODE, int NT, int STAGE_BYTES, int STAGES, int MINB, bool QUAD = false>
 __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThreads, MINB)
     stream_kernel(const __grid_constant__ StreamParams P)
 {
+    static_assert(!QUAD || MODE == kPack, "page quartets: the packing kernel and the fused restore");
     using Cfg = StreamCfg<MODE, NT, STAGE_BYTES, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 15) & ~(uintptr_t)15);  // bulk copies need 16 bytes
@@ -1501,16 +1868,22 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
         if (MODE == kCommit)
             loader_role<MODE, 0, STAGE_BYTES, STAGES, false, true>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c,
                                                                    ring, abort_flag, lane);
+        else if constexpr (QUAD)
+            loader_role_quad<MODE, STAGE_BYTES, STAGES, true>(P, P.w.work_ctr, P.ctr_base_v, ring, abort_flag, lane);
         else
             loader_role<MODE, NT, STAGE_BYTES, STAGES, true, true>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, ring,
                                                                    abort_flag, lane);
     } else if (Cfg::kStore && warp == Cfg::kStorerWarp) {
-        storer_role<MODE, STAGE_BYTES, STAGES>(P, ring, abort_flag, lane);
+        if constexpr (QUAD)
+            storer_role_quad<STAGE_BYTES, STAGES>(P, ring, abort_flag, lane);
+        else
+            storer_role<MODE, STAGE_BYTES, STAGES>(P, ring, abort_flag, lane);
     } else if constexpr (Cfg::kCrc) {
         if (Cfg::kOwnFinisher && warp == Cfg::kFinisherWarp)
             finisher_role<MODE, NT>(P, ring, abort_flag, lane);
         else
-            consumer_role<MODE, NT, STAGE_BYTES, STAGES, Cfg::kOwnFinisher>(P, ring, abort_flag, threadIdx.x, warp, lane);
+            consumer_role<MODE, NT, STAGE_BYTES, STAGES, Cfg::kOwnFinisher, QUAD>(P, ring, abort_flag, threadIdx.x, warp,
+                                                                                  lane);
     }
     __syncthreads();
 }
@@ -1527,7 +1900,7 @@ struct RestoreCfg {
                                          (VST + CST + 2) * sizeof(Item) + 2 * 12 * 8 + 4 * 8 + 16 + 16;
 };
 
-template <int NT, int VSB, int VST, int CSB, int CST, int MINB>
+template <int NT, int VSB, int VST, int CSB, int CST, int MINB, bool QUAD = false>
 __global__ void __launch_bounds__(NT + 128, MINB) restore_kernel(const __grid_constant__ StreamParams P)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -1569,17 +1942,20 @@ __global__ void __launch_bounds__(NT + 128, MINB) restore_kernel(const __grid_co
 
     constexpr int kCons = NT / 32;
     if (warp < kCons) {
-        consumer_role<kVerify, NT, VSB, VST, true>(P, vring, abort_flag, threadIdx.x, warp, lane);
+        consumer_role<kVerify, NT, VSB, VST, true, QUAD>(P, vring, abort_flag, threadIdx.x, warp, lane);
     } else if (warp == kCons) {
-        loader_role<kVerify, NT, VSB, VST, true, false>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, vring,
-                                                        abort_flag, lane);
+        if constexpr (QUAD)
+            loader_role_quad<kVerify, VSB, VST, false>(P, P.w.work_ctr, P.ctr_base_v, vring, abort_flag, lane);
+        else
+            loader_role<kVerify, NT, VSB, VST, true, false>(P, P.tl, P.n_items, P.w.work_ctr, P.ctr_base_v, vring,
+                                                            abort_flag, lane);
     } else if (warp == kCons + 1) {
         loader_role<kCommit, 0, CSB, CST, false, true>(P, P.tlc, P.n_items_c, P.w.work_ctr + 1, P.ctr_base_c, cring,
                                                        abort_flag, lane);
     } else if (warp == kCons + 2) {
         storer_role<kCommit, CSB, CST>(P, cring, abort_flag, lane);
     } else {
-        finisher_role<kVerify, NT>(P, vring, abort_flag, lane);
+        finisher_role<kVerify, NT, QUAD>(P, vring, abort_flag, lane);
     }
     __syncthreads();
 }
