@@ -55,7 +55,7 @@ def parse_args():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="gqa7b", choices=["gqa7b", "tiny", "corpus", "fp8", "stress", "longwindow", "digest", "layerwise",
-                                                            "latency", "records"],
+                                                            "latency", "records", "layerwise-device"],
                     help="gqa7b is the headline workload (full JSON line); the others print a shorter line "
                          "with the save and restore phases of that workload's shape")
     ap.add_argument("--window-blocks", type=int, default=48,
@@ -71,7 +71,8 @@ def parse_args():
     ap.add_argument("--tokens", type=int, default=0,
                     help="latency: restore one block of this many tokens (default: 256, 1,024, 5,200 and 24,018)")
     ap.add_argument("--layers", type=int, default=1,
-                    help="records: layers per page record of the gqa7b geometry (64 KiB per layer), 4 GiB of blobs")
+                    help="records: layers per page record of the gqa7b geometry (64 KiB per layer), 4 GiB of blobs; "
+                         "layerwise-device: layers per group (not given: groups of 32, 8, 4, 2 and 1 layers in turn)")
     ap.add_argument("--tune", default="", help="tuning keys for the headline context, key=value[,key=value...]")
     ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the one-step-at-a-time end-to-end leg")
     ap.add_argument("--e2e-pipelined-steps", type=int, default=10,
@@ -1292,6 +1293,83 @@ def run_layerwise(args):
     print(json.dumps(line), flush=True)
 
 
+# ---------------------------------------------------------------------------
+# layer-wise save and load on the device tier: what the smaller records cost
+# ---------------------------------------------------------------------------
+def run_layerwise_device(args):
+    """The headline batch (16 blocks x 4,096 tokens of the gqa7b geometry, 8 GiB) saved and restored
+    group of layers by group of layers with gk_pack_layerwise / gk_restore_layerwise, blobs on the device:
+    one ordinary call per group, records `group_layers` layers tall."""
+    import torch
+    import synth
+    import paper_2609_39358_b200 as gk
+
+    device = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(device)
+    w = synth.GQA7B
+    peak, _ = measured_peak()
+    slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
+    n_blocks, n_tok = 16, 4096
+    P = n_tok // w.page_tokens
+    N = n_blocks * P
+    data = synth.kv_bytes_bf16(2 * w.layers * N * slab // 2, w.sigma, w.seed(950), device)
+    src = gk.Cache(data, N, 2 * N * slab, N * slab, slab)
+    dst = gk.Cache(torch.zeros_like(data), N, 2 * N * slab, N * slab, slab)
+    perm_s = torch.from_numpy(synth.page_permutation(N, w.seed(951))).to(device)
+    perm_d = torch.from_numpy(synth.page_permutation(N, w.seed(952))).to(device)
+    stream = torch.cuda.current_stream(device)
+    reps = max(3, min(args.steps, 10))
+    out = {}
+    for g in ((args.layers,) if any(a.startswith("--layers") for a in sys.argv) else (32, 8, 4, 2, 1)):
+        n_groups = w.layers // g
+        geom = gk.Geom(g, w.kv_heads, w.head_dim, w.page_tokens, gk.GK_BF16, 0)
+        full = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, gk.GK_BF16, 0)
+        ctx = gk.Context(geom, device.index)
+        nb, _ = gk.gk_blob_size(full, n_tok)
+        sj, rj, keep = [], [], []
+        for b in range(n_blocks):
+            blob = torch.empty(nb, dtype=torch.uint8, device=device)
+            sums = torch.zeros(n_groups * P, dtype=torch.int64, device=device)
+            keep.append((blob, sums))
+            sj.append(gk.Job(blob, sums, perm_s[b * P:(b + 1) * P].contiguous(), n_tok))
+            rj.append(gk.Job(blob, sums, perm_d[b * P:(b + 1) * P].contiguous(), n_tok))
+        sj, rj = gk.JobArray(sj), gk.JobArray(rj)
+        mask = torch.zeros(n_blocks, dtype=torch.uint8, device=device)
+        fb = torch.zeros(n_blocks, dtype=torch.int32, device=device)
+        ts = {"save": [], "restore": []}
+        for r in range(reps + 3):
+            for name, fn in (("save", lambda: ctx.gk_pack_layerwise(n_groups, src, sj)),
+                             ("restore", lambda: ctx.gk_restore_layerwise(n_groups, rj, dst, mask, fb))):
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(stream)
+                fn()
+                e1.record(stream)
+                torch.cuda.synchronize(device)
+                if r >= 3:
+                    ts[name].append(e0.elapsed_time(e1))
+        assert int(mask.sum().item()) == 0
+        total = n_blocks * nb
+        sm, rm = float(np.median(ts["save"])), float(np.median(ts["restore"]))
+        out[f"{g}_layers_per_group"] = {
+            "groups": n_groups, "record_kib": 2 * g * slab // 1024, "save_ms": stats_ms(ts["save"]),
+            "restore_ms": stats_ms(ts["restore"]),
+            "save_frac_of_measured_peak": 2 * total / (sm * 1e-3) / 1e9 / peak,
+            "restore_frac_of_measured_peak_3_bytes": 3 * total / (rm * 1e-3) / 1e9 / peak,
+            "quartet_launches": ctx.gk_get_stats()["quartet_launches"]}
+        ctx.close()
+        del sj, rj, keep
+        torch.cuda.empty_cache()
+    first = next(iter(out.values()))
+    line = {"metric": METRIC, "value": 2 * n_blocks * nb / (first["restore_ms"]["median"] * 1e-3) / 1e9, "unit": UNIT,
+            "n_gpus": 1, "steps": reps, "warmup": 3, "ms_per_step": first["save_ms"]["median"] + first["restore_ms"]["median"],
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u64", "data": "synthetic",
+            "config": {"workload": "layerwise-device: gqa7b geometry, 16 blocks x 4,096 tokens (8 GiB of blobs on the "
+                                   "device), saved and restored one group of layers at a time",
+                       "step": "gk_pack_layerwise, then gk_restore_layerwise, timed separately"},
+            "cases": out}
+    print(json.dumps(line), flush=True)
+
+
 def synth_requests(n_blocks):
     return f"{max(n_blocks // 2, 1)} requests x {min(n_blocks, 2)} blocks"
 
@@ -1306,6 +1384,8 @@ def main():
         run_digest(args)
     elif args.workload == "layerwise":
         run_layerwise(args)
+    elif args.workload == "layerwise-device":
+        run_layerwise_device(args)
     elif args.workload == "latency":
         run_latency(args)
     elif args.workload != "gqa7b" or args.single_pass:

@@ -146,6 +146,14 @@ struct gk_ctx {
     // layer-wise restore: the codes and pages of the group in flight
     uint8_t *d_group_tmp = nullptr;
     size_t group_tmp_cap = 0;
+    // layer-wise calls on the device tier: the groups go in turn to this context and to a twin of it, each on a
+    // stream of its own, so that the first launches of a group overlap the last ones of the group before
+    gk_ctx *twin = nullptr;
+    bool is_twin = false;
+    cudaStream_t lw_stream[2] = {nullptr, nullptr};
+    cudaEvent_t lw_entry = nullptr;
+    cudaEvent_t lw_done[2] = {nullptr, nullptr};    // the group's work on its stream has been enqueued
+    cudaEvent_t lw_merged[2] = {nullptr, nullptr};  // the group's result arrays have been read (caller's stream)
 
     // streaming restore: the ids 0..iota_cap-1, from which window page tables are cut
     int32_t *d_iota = nullptr;
@@ -272,7 +280,7 @@ uint64_t items_wanted(const gk_ctx *c, int occ) { return 2ull * (uint64_t)c->sm_
 // cut pages into segments of at least two granules so that every SM gets work.
 //
 // Page quartets (`quad_for`: the call is a pack or a fused restore): records of at most
-// 256 KiB in a call with at least two quartets for every resident CTA are reduced one per
+// 256 KiB in a call with enough quartets for every resident CTA are reduced one per
 // WARP instead of one per CTA, four pages to a work item (see Tiling).
 enum QuadUse { kNoQuad = 0, kQuadPack = 1, kQuadRestore = 2 };
 
@@ -281,7 +289,12 @@ bool quad_wanted(const gk_ctx *c, QuadUse quad_for, uint64_t total_pages, int oc
     if (quad_for == kNoQuad || c->quad_mode == 1u || c->seg_granules) return false;
     if (quad_for == kQuadPack && c->gd.S != 0u) return false;  // scale values are gathered by a whole warp per record
     if (c->quad_mode == 2u) return true;
-    return c->gd.R <= (256u << 10) && total_pages >= 8ull * (uint64_t)c->sm_count * (uint64_t)occ;
+    // a quartet is four records long, and the last round of items is as long as the longest item: records of
+    // up to 128 KiB from two quartets per resident CTA on, records of up to 256 KiB from eight on (a 1 GiB
+    // call of 256 KiB records restores in 0.50 ms as single pages and in 0.52 ms as 1,024 quartets)
+    const uint64_t resident = (uint64_t)c->sm_count * (uint64_t)occ;
+    if (c->gd.R <= (128u << 10)) return total_pages >= 8ull * resident;
+    return c->gd.R <= (256u << 10) && total_pages >= 32ull * resident;
 }
 
 uint32_t crc_items(const Tiling &tl, uint64_t pages)
@@ -1022,6 +1035,13 @@ int gk_ctx_destroy(gk_ctx *c)
     if (!c) return GK_OK;
     DeviceGuard guard(c->device);
     cudaDeviceSynchronize();
+    if (c->twin) gk_ctx_destroy(c->twin);
+    for (int i = 0; i < 2; ++i) {
+        if (c->lw_stream[i]) cudaStreamDestroy(c->lw_stream[i]);
+        if (c->lw_done[i]) cudaEventDestroy(c->lw_done[i]);
+        if (c->lw_merged[i]) cudaEventDestroy(c->lw_merged[i]);
+    }
+    if (c->lw_entry) cudaEventDestroy(c->lw_entry);
     if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
     for (auto &ps : c->prof_pool) {
         cudaEventDestroy(ps.a);
@@ -1071,6 +1091,45 @@ int gk_ctx_set_tuning(gk_ctx *c, const char *key, uint32_t value)
     else if (!strcmp(key, "trace_hi")) c->trace = (unsigned long long *)(((uintptr_t)c->trace & 0xffffffffull) | ((uintptr_t)value << 32));
 #endif
     else return fail(c, GK_ERR_ARG, "unknown tuning key %s", key);
+    if (c->twin) return gk_ctx_set_tuning(c->twin, key, value);
+    return GK_OK;
+}
+
+// The twin of a context (layer-wise calls on the device tier): same geometry, same tuning, its own workspace,
+// error word and counters; gk_get_stats, gk_ctx_clear_error and gk_debug_status of the context cover both.
+static int ensure_twin(gk_ctx *c)
+{
+    if (c->twin) return GK_OK;
+    gk_ctx *t = nullptr;
+    int rc = gk_ctx_create(&t, &c->geom, c->device);
+    if (rc != GK_OK) return fail(c, rc, "layer-wise: no second context");
+    t->seg_granules = c->seg_granules;
+    t->commit_seg_tiles = c->commit_seg_tiles;
+    t->grid_cap = c->grid_cap;
+    t->fused = c->fused;
+    t->wait_limit_ns = c->wait_limit_ns;
+    t->test_drop_verify = c->test_drop_verify;
+    t->commit_reverse = c->commit_reverse;
+    t->l2_hints = c->l2_hints;
+    t->commit_items_per_cta = c->commit_items_per_cta;
+    t->quad_mode = c->quad_mode;
+    t->debug_extent_cut = c->debug_extent_cut;
+    t->trace = c->trace;
+    for (int i = 0; i < 2; ++i) {
+        if (cudaStreamCreateWithFlags(&c->lw_stream[i], cudaStreamNonBlocking) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->lw_done[i], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&c->lw_merged[i], cudaEventDisableTiming) != cudaSuccess) {
+            gk_ctx_destroy(t);
+            return fail(c, GK_ERR_CUDA, "layer-wise: streams and events");
+        }
+    }
+    if (cudaEventCreateWithFlags(&c->lw_entry, cudaEventDisableTiming) != cudaSuccess) {
+        gk_ctx_destroy(t);
+        return fail(c, GK_ERR_CUDA, "layer-wise: streams and events");
+    }
+    t->is_twin = true;
+    c->twin = t;
+    c->stats.allocations++;
     return GK_OK;
 }
 
@@ -1086,6 +1145,10 @@ int gk_ctx_reserve(gk_ctx *c, uint32_t max_jobs, uint64_t max_pages, uint64_t nu
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
     if ((rc = ensure_host_stage(c, (size_t)max_jobs * sizeof(JobDev) + (size_t)seg_max * 16)) != GK_OK) return rc;
     if (max_jobs && (rc = ensure_group_tmp(c, max_jobs)) != GK_OK) return rc;
+    if (max_jobs && !c->profile && !c->is_twin) {  // layer-wise calls on the device tier use a second context
+        if ((rc = ensure_twin(c)) != GK_OK) return rc;
+        if ((rc = gk_ctx_reserve(c->twin, max_jobs, max_pages, num_pages, 0)) != GK_OK) return rc;
+    }
     if (max_host_batch_bytes) {
         // room for the checksums beside the blobs, and for the alignment of every job's two parts
         const uint64_t want = max_host_batch_bytes + max_pages * 8 + (uint64_t)max_jobs * 512;
@@ -1101,6 +1164,7 @@ int gk_ctx_clear_error(gk_ctx *c, void *stream)
     if (!c) return GK_ERR_ARG;
     DeviceGuard guard(c->device);
     GK_CUDA(c, cudaMemsetAsync(c->d_error, 0, 4, (cudaStream_t)stream));
+    if (c->twin) GK_CUDA(c, cudaMemsetAsync(c->twin->d_error, 0, 4, (cudaStream_t)stream));
     return GK_OK;
 }
 
@@ -1575,6 +1639,13 @@ static void group_jobs(const gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, uin
     }
 }
 
+// Layer-wise calls on the device tier alternate between the context and its twin (see gk_ctx::twin); per-kernel
+// timing keeps everything in one context, where its event pool is.
+static bool lw_two_streams(const gk_ctx *c, uint32_t n_groups, bool host)
+{
+    return !host && n_groups > 1 && !c->profile;
+}
+
 static int pack_layerwise_impl(gk_ctx *c, uint32_t n_groups, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,
                                uint8_t *status_dev, void *stream, bool host)
 {
@@ -1584,14 +1655,40 @@ static int pack_layerwise_impl(gk_ctx *c, uint32_t n_groups, const gk_cache *src
     for (uint32_t j = 0; j < n_jobs; ++j)
         if (jobs[j].n_tokens == 0) return fail(c, GK_ERR_ARG, "job %u: n_tokens == 0", j);
     std::vector<gk_job> gj;
+    if (!lw_two_streams(c, n_groups, host)) {
+        for (uint32_t k = 0; k < n_groups; ++k) {
+            const gk_cache view = group_view(c, src, k);
+            group_jobs(c, jobs, n_jobs, k, gj);
+            const int rc = host ? gk_pack_host(c, &view, gj.data(), n_jobs, status_dev, stream)
+                                : gk_pack_batch(c, &view, gj.data(), n_jobs, status_dev, stream);
+            if (rc != GK_OK) return rc;
+        }
+        return GK_OK;
+    }
+    // device tier: the groups are independent of one another (their own layers of the cache, their own part of
+    // every blob), so they go in turn to two contexts on two streams; every group writes the same status bytes
+    DeviceGuard guard(c->device);
+    cudaStream_t st = (cudaStream_t)stream;
+    int rc = ensure_twin(c);
+    if (rc != GK_OK) return rc;
+    GK_CUDA(c, cudaEventRecord(c->lw_entry, st));
+    for (int i = 0; i < 2; ++i) GK_CUDA(c, cudaStreamWaitEvent(c->lw_stream[i], c->lw_entry, 0));
     for (uint32_t k = 0; k < n_groups; ++k) {
+        gk_ctx *ck = (k & 1u) ? c->twin : c;
         const gk_cache view = group_view(c, src, k);
         group_jobs(c, jobs, n_jobs, k, gj);
-        const int rc = host ? gk_pack_host(c, &view, gj.data(), n_jobs, status_dev, stream)
-                            : gk_pack_batch(c, &view, gj.data(), n_jobs, status_dev, stream);
-        if (rc != GK_OK) return rc;
+        rc = gk_pack_batch(ck, &view, gj.data(), n_jobs, status_dev, c->lw_stream[k & 1u]);
+        if (rc != GK_OK) {
+            if (ck != c) fail(c, rc, "%s", ck->err);
+            break;
+        }
     }
-    return GK_OK;
+    // the caller's stream goes on when both streams are through (also after a failure: what was enqueued runs)
+    for (int i = 0; i < 2; ++i) {
+        GK_CUDA(c, cudaEventRecord(c->lw_done[i], c->lw_stream[i]));
+        GK_CUDA(c, cudaStreamWaitEvent(st, c->lw_done[i], 0));
+    }
+    return rc;
 }
 
 static int restore_layerwise_impl(gk_ctx *c, uint32_t n_groups, const gk_job *jobs, uint32_t n_jobs,
@@ -1611,20 +1708,63 @@ static int restore_layerwise_impl(gk_ctx *c, uint32_t n_groups, const gk_job *jo
     int32_t *gfb = (int32_t *)c->d_group_tmp;
     uint8_t *gm_own = c->d_group_tmp + align_up((size_t)n_jobs * 4, 256);
     std::vector<gk_job> gj;
+    if (!lw_two_streams(c, n_groups, host)) {
+        for (uint32_t k = 0; k < n_groups; ++k) {
+            const gk_cache view = group_view(c, dst, k);
+            group_jobs(c, jobs, n_jobs, k, gj);
+            uint8_t *gm = group_mask_dev ? group_mask_dev + (size_t)k * n_jobs : gm_own;
+            const int rc = host ? restore_host_impl(c, gj.data(), n_jobs, &view, gm, gfb, stream, k == 0)
+                                : gk_restore(c, gj.data(), n_jobs, &view, gm, gfb, stream);
+            if (rc != GK_OK) return rc;
+            merge_group_kernel<<<(n_jobs + 127) / 128, 128, 0, st>>>(mask_dev, first_bad_page_dev, gm, gfb, n_jobs,
+                                                                     k == 0);
+            GK_CUDA(c, cudaGetLastError());
+            c->stats.kernels_launched++;
+            if (on_group)
+                on_group(user, k, k * c->gd.layers, c->gd.layers, group_mask_dev ? gm : nullptr, stream);
+        }
+        return GK_OK;
+    }
+    // Device tier: group k runs in context k & 1 on stream k & 1 (the groups touch different layers of the cache
+    // and different parts of the blobs).  The caller's stream waits for group k, merges its codes into the
+    // block-level result and is handed to on_group, in the order of the groups; a context's result arrays are
+    // reused by group k + 2 only after the merge of group k has read them.
+    int rc = ensure_twin(c);
+    if (rc != GK_OK) return rc;
+    if ((rc = ensure_group_tmp(c->twin, n_jobs)) != GK_OK) return fail(c, rc, "%s", c->twin->err);
+    GK_CUDA(c, cudaEventRecord(c->lw_entry, st));
+    for (int i = 0; i < 2; ++i) GK_CUDA(c, cudaStreamWaitEvent(c->lw_stream[i], c->lw_entry, 0));
     for (uint32_t k = 0; k < n_groups; ++k) {
+        const uint32_t i = k & 1u;
+        gk_ctx *ck = i ? c->twin : c;
+        int32_t *gfb_k = (int32_t *)ck->d_group_tmp;
+        uint8_t *gm_k = group_mask_dev ? group_mask_dev + (size_t)k * n_jobs
+                                       : ck->d_group_tmp + align_up((size_t)n_jobs * 4, 256);
         const gk_cache view = group_view(c, dst, k);
         group_jobs(c, jobs, n_jobs, k, gj);
-        uint8_t *gm = group_mask_dev ? group_mask_dev + (size_t)k * n_jobs : gm_own;
-        const int rc = host ? restore_host_impl(c, gj.data(), n_jobs, &view, gm, gfb, stream, k == 0)
-                            : gk_restore(c, gj.data(), n_jobs, &view, gm, gfb, stream);
-        if (rc != GK_OK) return rc;
-        merge_group_kernel<<<(n_jobs + 127) / 128, 128, 0, st>>>(mask_dev, first_bad_page_dev, gm, gfb, n_jobs, k == 0);
+        if (k >= 2u) GK_CUDA(c, cudaStreamWaitEvent(c->lw_stream[i], c->lw_merged[i], 0));
+        rc = gk_restore(ck, gj.data(), n_jobs, &view, gm_k, gfb_k, c->lw_stream[i]);
+        if (rc != GK_OK) {
+            if (ck != c) fail(c, rc, "%s", ck->err);
+            break;
+        }
+        GK_CUDA(c, cudaEventRecord(c->lw_done[i], c->lw_stream[i]));
+        GK_CUDA(c, cudaStreamWaitEvent(st, c->lw_done[i], 0));
+        merge_group_kernel<<<(n_jobs + 127) / 128, 128, 0, st>>>(mask_dev, first_bad_page_dev, gm_k, gfb_k, n_jobs,
+                                                                 k == 0);
         GK_CUDA(c, cudaGetLastError());
         c->stats.kernels_launched++;
+        GK_CUDA(c, cudaEventRecord(c->lw_merged[i], st));
         if (on_group)
-            on_group(user, k, k * c->gd.layers, c->gd.layers, group_mask_dev ? gm : nullptr, stream);
+            on_group(user, k, k * c->gd.layers, c->gd.layers, group_mask_dev ? gm_k : nullptr, stream);
     }
-    return GK_OK;
+    if (rc != GK_OK) {  // whatever was enqueued on the two streams still runs: the caller's stream waits for it
+        for (int i = 0; i < 2; ++i) {
+            cudaEventRecord(c->lw_done[i], c->lw_stream[i]);
+            cudaStreamWaitEvent(st, c->lw_done[i], 0);
+        }
+    }
+    return rc;
 }
 
 int gk_pack_layerwise(gk_ctx *c, uint32_t n_groups, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,
@@ -1842,6 +1982,7 @@ int gk_debug_status(gk_ctx *c, uint32_t out[4])
 #ifdef GK_DEBUG
     DeviceGuard guard(c->device);
     GK_CUDA(c, cudaMemcpy(out, c->d_error + 8, 16, cudaMemcpyDeviceToHost));
+    if (out[0] == 0u && c->twin) GK_CUDA(c, cudaMemcpy(out, c->twin->d_error + 8, 16, cudaMemcpyDeviceToHost));
     return GK_OK;
 #else
     out[0] = out[1] = out[2] = out[3] = 0u;
@@ -1857,6 +1998,20 @@ int gk_get_stats(gk_ctx *c, gk_stats *out)
     GK_CUDA(c, cudaMemcpy(&e, c->d_error, 4, cudaMemcpyDeviceToHost));
     c->stats.device_wait_expired = e;
     *out = c->stats;
+    if (c->twin) {  // what the twin did counts as this context's own (its calls are counted here, not there)
+        gk_stats t{};
+        const int rc = gk_get_stats(c->twin, &t);
+        if (rc != GK_OK) return rc;
+        out->calls_pack += t.calls_pack;
+        out->calls_restore += t.calls_restore;
+        out->jobs += t.jobs;
+        out->pages += t.pages;
+        out->bytes_blob += t.bytes_blob;
+        out->kernels_launched += t.kernels_launched;
+        out->quartet_launches += t.quartet_launches;
+        out->allocations += t.allocations;
+        if (out->device_wait_expired == 0) out->device_wait_expired = t.device_wait_expired;
+    }
     return GK_OK;
 }
 
