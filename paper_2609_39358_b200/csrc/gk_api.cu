@@ -706,8 +706,11 @@ int launch_fused(gk_ctx *c, const StreamParams &P, cudaStream_t st)
     // only half the integer lanes, and one CTA per SM is a little faster than two (8 GiB of 2 MiB records:
     // 3.80 against 3.83 ms; 3 MiB records 8.41 against 8.50 ms; 768 KiB records and fp8 records, whose scale
     // values the loader's and storer's lanes move one by one, are slower that way).
+    // Not for a call of one or two blocks: a block is committed only after all of it has verified, so its two
+    // phases follow one another, and the verifying phase alone wants both CTAs of an SM (one block of 24,018
+    // tokens: 1.62 ms with two CTAs per SM, 1.77 ms with one).
     if (!c->grid_cap && c->gd.S == 0 && c->gd.R >= (1u << 20) && P.n_items >= 8u * (uint32_t)c->sm_count &&
-        grid > (uint32_t)c->sm_count)
+        P.w.n_jobs >= 4u && grid > (uint32_t)c->sm_count)
         grid = (uint32_t)c->sm_count;
     gk_ctx::ProfSlot *slot = nullptr;
     int rc_prof = prof_begin(c, 3, st, &slot);

@@ -521,7 +521,7 @@ __device__ __forceinline__ bool item_from_tables(const StreamParams &P, const Ti
     const uint32_t local = item / tl.nseg_max;
     uint32_t q = item - local * tl.nseg_max;
     uint32_t gp = P.w.page_begin + local;
-    it.j = (uint32_t)P.w.page_job[gp];
+    it.j = P.w.n_jobs == 1u ? 0u : (uint32_t)P.w.page_job[gp];  // one dependent load less at the start of a lone block
     jbp = &P.w.jobs[it.j];
     const JobDev jb = *jbp;
     it.p = gp - jb.page_base;
