@@ -71,7 +71,7 @@ def parse_args():
     ap.add_argument("--tokens", type=int, default=0,
                     help="latency: restore one block of this many tokens (default: 256, 1,024, 5,200 and 24,018)")
     ap.add_argument("--layers", type=int, default=1,
-                    help="records: layers per page record of the gqa7b geometry (64 KiB per layer), 4 GiB of blobs; "
+                    help="records: layers per page record of the gqa7b geometry (64 KiB per layer), 8 GiB of blobs; "
                          "layerwise-device: layers per group (not given: groups of 32, 8, 4, 2 and 1 layers in turn)")
     ap.add_argument("--tune", default="", help="tuning keys for the headline context, key=value[,key=value...]")
     ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the one-step-at-a-time end-to-end leg")
@@ -713,6 +713,9 @@ def run_ours(args):
         workloads = {}
         for name in ("tiny", "corpus", "corpus_host", "fp8", "stress_wave", "stress_wave_one_third_damaged"):
             workloads[name] = workload_case(name, device, steps=5, warmup=2)
+        # small page records (the gqa7b geometry with one and two layers per record, 8 GiB of blobs)
+        for layers in (1, 2):
+            workloads[f"records_{64 * layers}_kib"] = workload_case("gqa7b", device, steps=5, warmup=2, layers=layers)
         latency = latency_cases(device)
 
     if rank == 0:
@@ -815,10 +818,10 @@ def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0, 
 
     w, lens, dst_pages, ids = shape_of(synth, name, blocks)
     if layers:
-        # small page records: the gqa7b geometry with fewer layers per record, about 4 GiB of blobs
+        # small page records: the gqa7b geometry with fewer layers per record, 8 GiB of blobs as in the headline
         import dataclasses
         w = dataclasses.replace(w, layers=layers)
-        lens = [4096 * (32 // layers) // 2] * 16 if layers < 32 else [4096] * 8
+        lens = [4096 * max(32 // layers, 1)] * 16
         dst_pages = sum(-(-n // w.page_tokens) for n in lens)
     host_tier = name.endswith("_host")
     dtype = gk.GK_BF16 if w.dtype == "bf16" else gk.GK_FP8_E4M3
