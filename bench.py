@@ -821,7 +821,7 @@ def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0, 
         # small page records: the gqa7b geometry with fewer layers per record, 8 GiB of blobs as in the headline
         import dataclasses
         w = dataclasses.replace(w, layers=layers)
-        lens = [4096 * max(32 // layers, 1)] * 16
+        lens = [4096 * max(32 // layers, 1)] * (blocks or 16)
         dst_pages = sum(-(-n // w.page_tokens) for n in lens)
     host_tier = name.endswith("_host")
     dtype = gk.GK_BF16 if w.dtype == "bf16" else gk.GK_FP8_E4M3

@@ -341,7 +341,15 @@ int gk_restore_stream(gk_ctx *ctx, const gk_job *jobs, uint32_t n_jobs, const gk
  * on_group (may be NULL) is called ON THE HOST; it must only enqueue work on
  * `stream` (e.g. layer k's attention); group_mask points at group k's codes (NULL
  * if group_mask_dev is NULL).  In the host tier the copies of group k+1 run while
- * group k is verified, committed and consumed. */
+ * group k is verified, committed and consumed.  On the device tier the groups
+ * (which touch different layers of the cache and different parts of the blobs)
+ * go in turn to this context and to a second, internal one on two internal
+ * streams, so that the first launches of a group overlap the last ones of the
+ * group before; `stream` waits for each group in order before on_group sees it,
+ * and for all of them before the call's work on `stream` is complete.  The
+ * internal context is created at the first such call (or by gk_ctx_reserve);
+ * its counters and its error word are part of this context's (gk_get_stats,
+ * gk_ctx_clear_error). */
 typedef void (*gk_group_fn)(void *user, uint32_t group, uint32_t first_layer, uint32_t n_layers,
                             const uint8_t *group_mask, void *stream);
 int gk_pack_layerwise(gk_ctx *ctx, uint32_t n_groups, const gk_cache *src, const gk_job *jobs, uint32_t n_jobs,

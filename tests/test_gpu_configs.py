@@ -194,6 +194,55 @@ def test_gqa7b_full(gk):
     ctx.close()
 
 
+def test_small_records_full(gk):
+    """The gqa7b geometry with ONE layer per record (64 KiB records, the layer-wise format's smallest group):
+    8 blocks of 32,768 tokens = 16,384 pages, 1 GiB of blobs.  Calls of this size take the page-quartet form
+    of the packing and of the fused restore kernel (one record per warp).  All 16,384 checksums and every
+    byte of two blocks against the oracle; one blob damaged; full destination check."""
+    import dataclasses
+    w = dataclasses.replace(synth.GQA7B, layers=1)
+    geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens)
+    ctx = gk.Context(geom, 0)
+    n_tok, NB = 32768, 8
+    nbytes, P = gk.gk_blob_size(geom, n_tok)
+    s = _slab(w)
+    src_pages, dst_pages = NB * P, NB * P + 100
+    src = _dev_cache(gk, w, src_pages, synth.kv_bytes_bf16(w.layers * src_pages * s, w.sigma, w.seed(40), "cuda"))
+    sentinel = synth.sentinel_bytes(2 * w.layers * dst_pages * s, w.seed(41), "cuda")
+    dst = _dev_cache(gk, w, dst_pages, sentinel.clone())
+    sperm = synth.page_permutation(src_pages, w.seed(42))
+    dperm = synth.page_permutation(dst_pages, w.seed(43))
+    blobs = [torch.empty(nbytes, dtype=torch.uint8, device="cuda") for _ in range(NB)]
+    sums = [torch.zeros(P, dtype=torch.int64, device="cuda") for _ in range(NB)]
+    spts = [sperm[i * P:(i + 1) * P] for i in range(NB)]
+    dpts = [dperm[i * P:(i + 1) * P] for i in range(NB)]
+    d_spts = [torch.from_numpy(x.copy()).cuda() for x in spts]
+    d_dpts = [torch.from_numpy(x.copy()).cuda() for x in dpts]
+    status = torch.full((NB,), 255, dtype=torch.uint8, device="cuda")
+    ctx.gk_pack_batch(src, [gk.Job(blobs[i], sums[i], d_spts[i], n_tok) for i in range(NB)], status)
+    torch.cuda.synchronize()
+    assert status.cpu().tolist() == [0] * NB
+    assert ctx.gk_get_stats()["quartet_launches"] == 1
+    _check_all_checksums(w, blobs, sums, [n_tok] * NB)
+    for i in (0, NB - 1):
+        _check_whole_block(w, src, blobs[i], sums[i], spts[i], n_tok)
+    # one byte of block 5 flipped, in the third page of a quartet
+    bad_page = 4 * 277 + 2
+    blobs[5][bad_page * (nbytes // P) + 12345] ^= 0x10
+    mask = torch.full((NB,), 255, dtype=torch.uint8, device="cuda")
+    fb = torch.zeros(NB, dtype=torch.int32, device="cuda")
+    ctx.gk_restore([gk.Job(blobs[i], sums[i], d_dpts[i], n_tok) for i in range(NB)], dst, mask, fb)
+    torch.cuda.synchronize()
+    want = [0] * NB
+    want[5] = 1
+    assert mask.cpu().tolist() == want
+    assert fb.cpu().tolist() == [-1 if m == 0 else bad_page for m in want]
+    assert ctx.gk_get_stats()["quartet_launches"] == 2
+    _check_destination(w, src, dst, sentinel, [(spts[i], dpts[i], n_tok) for i in range(NB)], want)
+    assert ctx.gk_get_stats()["device_wait_expired"] == 0
+    ctx.close()
+
+
 def test_corpus_full_device_and_host_tier(gk):
     """95 blocks of 1,024 tokens + a 280-token tail block (partial last page) into a
     6,200-page cache: once from device blobs, once from pinned host memory."""
