@@ -752,6 +752,35 @@ int launch_validate(gk_ctx *c, const WorkDev &w, uint64_t num_pages, int clear_c
     return GK_OK;
 }
 
+// Large calls of at most kPrepMaxJobs jobs: the job table rides in the validation kernel's arguments instead of
+// a staging copy in front of it (one stream operation less per call: layer-wise calls make one call per group).
+bool table_fits_args(uint32_t n_jobs, const Tiling &crc)
+{
+    return n_jobs <= kPrepMaxJobs && crc.nseg_max <= kPrepMaxSeg;
+}
+
+int launch_validate_args(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const Tiling &crc, const WorkDev &w,
+                         uint64_t num_pages, int clear_claims, bool need_tables, cudaStream_t st, uint64_t *pages_out,
+                         uint64_t *bytes_out, uint8_t *status_out = nullptr)
+{
+    PrepSmallParams pp{};
+    int rc = fill_job_table(c, jobs, n_jobs, pp.jobs, nullptr, nullptr, need_tables, pages_out, bytes_out);
+    if (rc != GK_OK) return rc;
+    fill_seg_pow(c, crc, pp.seg_pow);
+    pp.n_seg_pow = 2 * crc.nseg_max;
+    uint32_t grid = n_jobs;
+    if (clear_claims) {
+        uint32_t g2 = (uint32_t)((num_pages + 1023) / 1024);
+        if (g2 > 2048) g2 = 2048;
+        if (g2 > grid) grid = g2;
+    }
+    c->ctr_next[0] = c->ctr_next[1] = 0;  // the kernel zeroes the device counters
+    validate_args_kernel<<<grid, 1024, 0, st>>>(pp, w, num_pages, clear_claims, status_out);
+    GK_CUDA(c, cudaGetLastError());
+    c->stats.kernels_launched++;
+    return GK_OK;
+}
+
 int launch_claim(gk_ctx *c, const WorkDev &w, cudaStream_t st)
 {
     claim_kernel<<<(w.total_pages + 255) / 256, 256, 0, st>>>(w);
@@ -1196,8 +1225,16 @@ int gk_pack_batch(gk_ctx *c, const gk_cache *src, const gk_job *jobs, uint32_t n
                                     status_dev)) != GK_OK)
             return rc;
     } else {
-        if ((rc = upload_jobs(c, jobs, n_jobs, l, tl, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
-        if ((rc = launch_validate(c, w, cd.num_pages, 0, st, status_dev)) != GK_OK) return rc;
+        if (table_fits_args(n_jobs, tl)) {
+            if ((rc = launch_validate_args(c, jobs, n_jobs, tl, w, cd.num_pages, 0, true, st, &pages, &bytes,
+                                           status_dev)) != GK_OK)
+                return rc;
+        } else {
+            if ((rc = upload_jobs(c, jobs, n_jobs, l, tl, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK)
+                return rc;
+            if ((rc = launch_validate(c, w, cd.num_pages, 0, st, status_dev)) != GK_OK) return rc;
+        }
+        c->pdl_next = !c->profile;  // the packing kernel sets its rings up while the validation runs
     }
     StreamParams P{};
     P.g = c->gd;
@@ -1325,9 +1362,16 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
         if ((rc = launch_prep_small(c, jobs, n_jobs, tlv, w, cd.num_pages, true, true, st, &pages, &bytes)) != GK_OK)
             return rc;
     } else {
-        if ((rc = upload_jobs(c, jobs, n_jobs, l, tlv, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK) return rc;
-        if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
+        if (table_fits_args(n_jobs, tlv)) {
+            if ((rc = launch_validate_args(c, jobs, n_jobs, tlv, w, cd.num_pages, 1, true, st, &pages, &bytes)) != GK_OK)
+                return rc;
+        } else {
+            if ((rc = upload_jobs(c, jobs, n_jobs, l, tlv, nullptr, nullptr, true, st, &pages, &bytes)) != GK_OK)
+                return rc;
+            if ((rc = launch_validate(c, w, cd.num_pages, 1, st)) != GK_OK) return rc;
+        }
         if ((rc = launch_claim(c, w, st)) != GK_OK) return rc;
+        c->pdl_next = !c->profile;  // the first streaming kernel sets its rings up while the claims are made
     }
     if ((rc = enqueue_verify_commit(c, w, cd, tlv, tlc, 0, (uint32_t)pages, mask_dev, first_bad_page_dev, st)) != GK_OK)
         return rc;

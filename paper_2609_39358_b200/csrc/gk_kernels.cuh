@@ -60,12 +60,35 @@ __global__ void merge_group_kernel(uint8_t *mask, int32_t *first_bad, const uint
     mask[j] = gm > m ? gm : m;
 }
 
+// Job table and segment powers of a call of at most kPrepMaxJobs jobs, as kernel arguments.
+constexpr uint32_t kPrepMaxJobs = 64;
+constexpr uint32_t kPrepMaxSeg = 64;
+struct PrepSmallParams {
+    JobDev jobs[kPrepMaxJobs];
+    uint64_t seg_pow[2 * kPrepMaxSeg];
+    uint32_t n_seg_pow;
+    uint32_t do_claims;
+    uint64_t num_pages;
+    uint8_t *status_out;  // save calls: 0 or 2 per job; else null
+};
+
 // One CTA per job.  Initialises the job's result words, records the lowest
 // out-of-range page id and fills page_job.  All CTAs together clear the claim
 // words of the destination cache.
-__global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims, uint8_t *status_out)
+// ARGS: the job table (at most kPrepMaxJobs jobs) and the segment powers travel as kernel arguments -- no
+// staging copy in front of the call; block 0 leaves them in the workspace for the kernels that follow.
+template <bool ARGS>
+__device__ __forceinline__ void validate_body(const PrepSmallParams *pp, const WorkDev &w, uint64_t num_pages,
+                                              int clear_claims, uint8_t *status_out)
 {
+    allow_dependent_launch();  // the kernel directly behind this one may set itself up meanwhile
     const uint32_t j = blockIdx.x;
+    if (ARGS && blockIdx.x == 0) {
+        JobDev *jobs_out = const_cast<JobDev *>(w.jobs);
+        uint64_t *pow_out = const_cast<uint64_t *>(w.seg_pow);
+        for (uint32_t k = threadIdx.x; k < w.n_jobs; k += blockDim.x) jobs_out[k] = pp->jobs[k];
+        for (uint32_t k = threadIdx.x; k < pp->n_seg_pow; k += blockDim.x) pow_out[k] = pp->seg_pow[k];
+    }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         // every call draws its work items from zero (the host counts the draws of its launches)
         w.work_ctr[0] = 0u;
@@ -78,7 +101,7 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims,
             w.claims[i] = 0ull;
     }
     if (j >= w.n_jobs) return;
-    const JobDev jb = w.jobs[j];
+    const JobDev jb = ARGS ? pp->jobs[j] : w.jobs[j];
     __shared__ int32_t s_bad;
     if (threadIdx.x == 0) s_bad = kNoPage;
     __syncthreads();
@@ -105,12 +128,24 @@ __global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims,
     }
 }
 
+__global__ void validate_kernel(WorkDev w, uint64_t num_pages, int clear_claims, uint8_t *status_out)
+{
+    validate_body<false>(nullptr, w, num_pages, clear_claims, status_out);
+}
+
+__global__ void validate_args_kernel(const __grid_constant__ PrepSmallParams pp, WorkDev w, uint64_t num_pages,
+                                     int clear_claims, uint8_t *status_out)
+{
+    validate_body<true>(&pp, w, num_pages, clear_claims, status_out);
+}
+
 // One thread per page of the call.  The first job to claim a destination page
 // leaves (job+1, index) in its claim word; every later claimant marks itself
 // and that first claimant.  Jobs that are missing or already failed the range
 // check claim nothing.
 __global__ void claim_kernel(WorkDev w)
 {
+    allow_dependent_launch();  // the streaming kernel behind this one may set up its rings meanwhile
     const uint32_t g = blockIdx.x * blockDim.x + threadIdx.x;
     if (g >= w.total_pages) return;
     const uint32_t j = (uint32_t)w.page_job[g];
@@ -131,17 +166,6 @@ __global__ void claim_kernel(WorkDev w)
 // copy.  Writes the tables to the workspace, then does what validate_kernel and
 // claim_kernel do, separated by a CTA barrier.  Only the claim words that this
 // call can touch are cleared.
-constexpr uint32_t kPrepMaxJobs = 64;
-constexpr uint32_t kPrepMaxSeg = 64;
-struct PrepSmallParams {
-    JobDev jobs[kPrepMaxJobs];
-    uint64_t seg_pow[2 * kPrepMaxSeg];
-    uint32_t n_seg_pow;
-    uint32_t do_claims;
-    uint64_t num_pages;
-    uint8_t *status_out;  // save calls: 0 or 2 per job; else null
-};
-
 __global__ void __launch_bounds__(1024) prep_small_kernel(const __grid_constant__ PrepSmallParams pp, WorkDev w)
 {
     allow_dependent_launch();  // the streaming kernel behind this one may set up its rings meanwhile
