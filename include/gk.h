@@ -431,7 +431,8 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * (time limit of every wait inside a kernel, default 2000), "commit_reverse" (1,
  * the default: the commit side reads a job's records from the last to the first,
  * so that what was verified last is still in L2), "l2_hints" (bit 0: verify loads
- * ask L2 to keep the lines, bit 1: commit loads ask it to drop them; default 0),
+ * ask L2 to keep the lines, bit 1: commit loads ask it to drop them, bit 2: commit
+ * stores ask it to drop the written lines first; default 0),
  * "test_drop_verify" (tests only: with value k > 0 the fused restore kernel
  * verifies nothing of the jobs k-1, k, ..., so that the commit waits of exactly
  * those jobs run into their limit and the time-out handling can be checked

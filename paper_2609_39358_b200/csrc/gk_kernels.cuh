@@ -370,7 +370,7 @@ struct StreamParams {
     uint32_t inline_final;  // 1: the CTA that delivers a page's last segment finalizes the page itself
     uint32_t ctr_base_v, ctr_base_c;  // values of the work counters at the start of this launch
     uint32_t commit_reverse;  // 1: the commit side walks the pages of a job from the last to the first
-    uint32_t l2_hints;        // bit 0: verify loads evict_last; bit 1: commit loads evict_first
+    uint32_t l2_hints;        // bit 0: verify loads evict_last; bit 1: commit loads evict_first; bit 2: commit stores evict_first
     uint32_t test_drop_from;  // tests only: k > 0 makes the fused kernel verify nothing of jobs k-1, k, ...
     unsigned long long *trace;  // builds with GK_TRACE: time stamps of the first item of every role, else null
     uint8_t *mask_out;        // commit
@@ -1383,6 +1383,10 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
 {
     uint32_t n = 0;
     bool revoked = false;
+    // commit: the written pages are not read again by this call -- let them leave L2 before the blob does
+    const bool store_hint = MODE == kCommit && (P.l2_hints & 4u);
+    uint64_t store_policy = 0;
+    if (store_hint) store_policy = policy_evict_first();
     for (;; ++n) {
         const uint32_t s = n % STAGES;
         // the loader ahead of a commit storer may itself be waiting, job after job, for verification
@@ -1442,7 +1446,10 @@ __device__ __forceinline__ void storer_role(const StreamParams &P, const Ring &r
                         if ((uint64_t)nb > d1 - d0) nb = (uint32_t)(d1 - d0);
                         if (nb == 0u) break;  // cannot happen with a valid geometry; never spin
                         uint8_t *ca = chunk_addr(P.cache, ch, chunk, phys, off);
-                        if (GK_DEBUG_OK(P, kDbgCache, 3u, ca, nb, P.cache.data, P.cache.data_extent)) bulk_s2g(ca, so, nb);
+                        if (GK_DEBUG_OK(P, kDbgCache, 3u, ca, nb, P.cache.data, P.cache.data_extent)) {
+                            if (store_hint) bulk_s2g_hint(ca, so, nb, store_policy);
+                            else bulk_s2g(ca, so, nb);
+                        }
                         d0 += nb;
                         so += nb;
                         ++chunk;
