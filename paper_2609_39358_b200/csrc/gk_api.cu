@@ -279,7 +279,7 @@ uint64_t items_wanted(const gk_ctx *c, int occ) { return 2ull * (uint64_t)c->sm_
 // segment per page (the per-thread epilogue is paid once per page); small calls
 // cut pages into segments of at least two granules so that every SM gets work.
 //
-// Page quartets (`quad_for`: the call is a pack or a fused restore): records of at most
+// Page quartets (`quad_for`: the call packs, or verifies -- alone or in a fused restore): records of at most
 // 256 KiB in a call with enough quartets for every resident CTA are reduced one per
 // WARP instead of one per CTA, four pages to a work item (see Tiling).
 enum QuadUse { kNoQuad = 0, kQuadPack = 1, kQuadRestore = 2 };
@@ -674,6 +674,9 @@ int launch_stream(gk_ctx *c, int occ, const StreamParams &P, cudaStream_t st)
 
 int launch_verify(gk_ctx *c, const StreamParams &P, cudaStream_t st)
 {
+    if (P.tl.quad)
+        return launch_stream<VerifyCfg, kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB, true>(
+            c, c->occ_verify, P, st);
     return launch_stream<VerifyCfg, kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB>(c, c->occ_verify, P, st);
 }
 int launch_pack(gk_ctx *c, const StreamParams &P, cudaStream_t st)
@@ -1004,7 +1007,7 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
     c->sm_count = prop.multiProcessorCount;
 
     // every streaming kernel: shared-memory size, then how many CTAs of it an SM holds
-    int occ_quad[2] = {0, 0};
+    int occ_quad[3] = {0, 0, 0};
     auto prepare = [&](auto *kernel, int threads, size_t smem, int *occ) {
         return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) == cudaSuccess &&
                cudaOccupancyMaxActiveBlocksPerMultiprocessor(occ, kernel, threads, smem) == cudaSuccess && *occ >= 1;
@@ -1025,7 +1028,9 @@ int gk_ctx_create(gk_ctx **out, const gk_geom *geom, int device)
         !prepare(restore_kernel<GK_CRC_NT, GK_CRC_STAGE, GK_FUSED_VSTAGES, GK_COPY_STAGE, GK_FUSED_CSTAGES, GK_FUSED_MINB,
                                 true>,
                  FusedCfg::kThreads, FusedCfg::kSmemBytes, &occ_quad[1]) ||
-        occ_quad[0] < c->occ_pack || occ_quad[1] < c->occ_fused) {
+        !prepare(stream_kernel<kVerify, GK_CRC_NT, GK_CRC_STAGE, GK_CRC_STAGES, GK_VERIFY_MINB, true>, VerifyCfg::kThreads,
+                 VerifyCfg::kSmemBytes, &occ_quad[2]) ||
+        occ_quad[0] < c->occ_pack || occ_quad[1] < c->occ_fused || occ_quad[2] < c->occ_verify) {
         cudaGetLastError();
         return bail(GK_ERR_CUDA);
     }
@@ -1274,7 +1279,7 @@ int gk_page_checksums(gk_ctx *c, const void *blob_dev, uint32_t n_tokens, uint64
     jb.page_table = nullptr;
     jb.n_tokens = n_tokens;
     uint64_t pages = pages_of(n_tokens, c->gd.page_tokens), bytes = 0;
-    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify);
+    const Tiling tl = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify, false, kQuadRestore);
     const WsLayout l = ws_layout(1, pages, tl.nseg_max, 0);
     int rc;
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
@@ -1353,7 +1358,7 @@ int gk_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const gk_cache *d
     const bool fused = !single && c->fused && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
     const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages,
                                   single ? c->occ_single : fused ? c->occ_fused : c->occ_verify, fused && n_jobs > 1,
-                                  fused ? kQuadRestore : kNoQuad);
+                                  single ? kNoQuad : kQuadRestore);
     const Tiling tlc = commit_tiling(c, GK_COPY_STAGE, pages, fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
@@ -1390,7 +1395,7 @@ static int prepare_restore(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, const
     if (rc != GK_OK) return rc;
     uint64_t pages = 0, bytes = 0;
     for (uint32_t j = 0; j < n_jobs; ++j) pages += pages_of(jobs[j].n_tokens, c->gd.page_tokens);
-    *tlv = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify);
+    *tlv = crc_tiling(c, GK_CRC_STAGE, pages, c->occ_verify, false, kQuadRestore);
     *tlc = commit_tiling(c, GK_COPY_STAGE, pages, c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv->nseg_max, cd->num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;
@@ -1501,7 +1506,7 @@ static int restore_host_impl(gk_ctx *c, const gk_job *jobs, uint32_t n_jobs, con
     const bool fused = c->fused && !single && !(c->gd.flags & GK_FLAG_SKIP_VERIFY);
     const int occ = single ? c->occ_single : fused ? c->occ_fused : c->occ_verify;
     const Tiling tlv = crc_tiling(c, GK_CRC_STAGE, pages_per_launch, occ, fused && n_jobs > batch_end.size(),
-                                  fused ? kQuadRestore : kNoQuad);
+                                  single ? kNoQuad : kQuadRestore);
     const Tiling tlc = commit_tiling(c, GK_COPY_STAGE, pages_per_launch, fused ? c->occ_fused : c->occ_commit);
     const WsLayout l = ws_layout(n_jobs, pages, tlv.nseg_max, cd.num_pages);
     if ((rc = ensure_workspace(c, l.total)) != GK_OK) return rc;

@@ -1868,7 +1868,7 @@ template <int MODE, int NT, int STAGE_BYTES, int STAGES, int MINB, bool QUAD = f
 __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThreads, MINB)
     stream_kernel(const __grid_constant__ StreamParams P)
 {
-    static_assert(!QUAD || MODE == kPack, "page quartets: the packing kernel and the fused restore");
+    static_assert(!QUAD || MODE == kPack || MODE == kVerify, "page quartets: packing, verifying, and the fused restore");
     using Cfg = StreamCfg<MODE, NT, STAGE_BYTES, STAGES>;
     extern __shared__ uint8_t smem_raw[];
     uint8_t *smem = (uint8_t *)(((uintptr_t)smem_raw + 15) & ~(uintptr_t)15);  // bulk copies need 16 bytes
@@ -1911,7 +1911,7 @@ __global__ void __launch_bounds__(StreamCfg<MODE, NT, STAGE_BYTES, STAGES>::kThr
             storer_role<MODE, STAGE_BYTES, STAGES>(P, ring, abort_flag, lane);
     } else if constexpr (Cfg::kCrc) {
         if (Cfg::kOwnFinisher && warp == Cfg::kFinisherWarp)
-            finisher_role<MODE, NT>(P, ring, abort_flag, lane);
+            finisher_role<MODE, NT, QUAD>(P, ring, abort_flag, lane);
         else
             consumer_role<MODE, NT, STAGE_BYTES, STAGES, Cfg::kOwnFinisher, QUAD>(P, ring, abort_flag, threadIdx.x, warp,
                                                                                   lane);

@@ -40,7 +40,7 @@ def _ctx(gk, og, **tuning):
     return ctx
 
 
-def _round_trip(gk, og, lens, seed, quad, expect_quartets, damage=True, host_tier=False):
+def _round_trip(gk, og, lens, seed, quad, expect_quartets, damage=True, host_tier=False, **tuning):
     """Packs blocks of the given lengths, checks blobs and checksums against the oracle, damages
     some, restores, and compares codes, first bad pages and the whole destination image."""
     from gpu_harness import assert_cache_equal, dev_cache, gpu_pack, gpu_restore
@@ -49,7 +49,7 @@ def _round_trip(gk, og, lens, seed, quad, expect_quartets, damage=True, host_tie
     Ns = 48
     src = random_cache(og, Ns, seed=seed + 1)
     tables = [rng.integers(0, Ns, size=n_pages(og, n)).astype(np.int32) for n in lens]
-    ctx = _ctx(gk, og, quad=quad)
+    ctx = _ctx(gk, og, quad=quad, **tuning)
     got, status = gpu_pack(ctx, og, dev_cache(src), tables, lens)
     assert status.tolist() == [0] * n_jobs
     total = sum(n_pages(og, n) for n in lens)
@@ -131,6 +131,30 @@ def test_chosen_for_large_calls_of_small_records(gk, og):
         lens.append(int(rng.integers(1, 400 * T)))
     _round_trip(gk, og, lens, 4800, quad=0, expect_quartets=2)
     _round_trip(gk, og, lens, 4800, quad=1, expect_quartets=0)
+
+
+def test_verify_alone_and_page_checksums(gk):
+    """The verifying kernel on its own (restore with the tuning key fused = 0: a verify launch, a compare
+    launch, a commit launch; and gk_page_checksums) takes the same form."""
+    from gpu_harness import gk_geom
+    og = G_20K
+    T = og.page_tokens
+    rng = np.random.default_rng(5100)
+    lens = [int(rng.integers(1, 5 * T + 1)) for _ in range(40)]
+    _round_trip(gk, og, lens, 5200, quad=2, expect_quartets=2, fused=0)
+    # checksums of an existing blob
+    n = 37 * T + 5
+    src = random_cache(og, n_pages(og, n), seed=5300)
+    blob, sums, code, _ = oracle.pack(og, src, np.arange(n_pages(og, n), dtype=np.int32), n)
+    assert code == 0
+    ctx = gk.Context(gk_geom(og), 0)
+    ctx.set_tuning("quad", 2)
+    out = torch.zeros(n_pages(og, n), dtype=torch.int64, device="cuda")
+    ctx.gk_page_checksums(torch.from_numpy(blob).cuda(), n, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().view(np.uint64), sums)
+    assert ctx.gk_get_stats()["quartet_launches"] == 1
+    ctx.close()
 
 
 def test_host_tier_in_batches(gk):
