@@ -73,7 +73,7 @@ def parse_args():
     ap.add_argument("--layers", type=int, default=1,
                     help="records: layers per page record of the gqa7b geometry (64 KiB per layer), 8 GiB of blobs; "
                          "layerwise-device: layers per group (not given: groups of 32, 8, 4, 2 and 1 layers in turn)")
-    ap.add_argument("--tune", default="", help="tuning keys for the headline context, key=value[,key=value...]")
+    ap.add_argument("--tune", default="", help="tuning keys for the context of the run, key=value[,key=value...]")
     ap.add_argument("--e2e-steps", type=int, default=3, help="steps of the one-step-at-a-time end-to-end leg")
     ap.add_argument("--e2e-pipelined-steps", type=int, default=10,
                     help="steps of the pipelined end-to-end leg (save of step k+1 overlaps restore of step k)")
@@ -795,6 +795,8 @@ def shape_of(synth, name, blocks=0):
             lens += [int(all_len[b]) for b in req]
             ids += [int(b) for b in req]
             used += need
+            if blocks and len(lens) >= blocks:   # a shorter wave (small cases for profiling)
+                break
         return w, lens, dst_pages, ids
     w = synth.WORKLOADS[name.replace("_host", "")]
     if name == "gqa7b":
@@ -808,7 +810,7 @@ def shape_of(synth, name, blocks=0):
     raise ValueError(name)
 
 
-def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0, layers=0):
+def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0, layers=0, tune=""):
     """Save and restore phases of one workload shape, each timed on its own over `steps`
     calls (the damage the configuration prescribes is applied between the two, so the
     restore is timed with it in place).  Returns a record for the bench line."""
@@ -828,6 +830,9 @@ def workload_case(name, device, steps=5, warmup=2, single_pass=False, blocks=0, 
     flags = gk.GK_FLAG_SINGLE_PASS if single_pass else 0
     geom = gk.Geom(w.layers, w.kv_heads, w.head_dim, w.page_tokens, dtype, w.scale_kv, flags)
     ctx = gk.Context(geom, device.index)
+    for kv in filter(None, tune.split(",")):
+        key, val = kv.split("=")
+        ctx.set_tuning(key, int(val))
     restore_traffic = 2 if single_pass else 3     # DRAM bytes per blob byte of the restore
     slab = w.page_tokens * w.kv_heads * w.head_dim * w.elem_bytes
     pages = [-(-n // w.page_tokens) for n in lens]
@@ -1036,7 +1041,7 @@ def run_other_workload(args):
     torch.cuda.set_device(device)
     name = {"stress": "stress_wave", "records": "gqa7b"}.get(args.workload, args.workload)
     rec = workload_case(name, device, steps=max(args.steps, 1) if args.steps < 50 else 10, warmup=max(args.warmup, 3),
-                        single_pass=args.single_pass, blocks=args.blocks,
+                        single_pass=args.single_pass, blocks=args.blocks, tune=args.tune,
                         layers=args.layers if args.workload == "records" else 0)
     pm, rm = rec["save_ms"]["median"], rec["restore_ms"]["median"]
     line = {"metric": METRIC, "value": rec["restore_useful"]["gbs"], "unit": UNIT, "n_gpus": 1,
