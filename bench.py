@@ -553,6 +553,26 @@ def run_ours(args):
             c1.record(stream)
             torch.cuda.synchronize(device)
             link_rate[name] = 3 * blob_bytes / (c0.elapsed_time(c1) * 1e-3) / 1e9
+        # both directions at once (two streams): the ceiling of the pipelined save + restore below
+        if len(keep) >= 2:
+            tmp2 = torch.empty(blob_bytes, dtype=torch.uint8, device=device)
+            s_a, s_b = torch.cuda.Stream(device), torch.cuda.Stream(device)
+            c0, c1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize(device)
+            c0.record(stream)
+            s_a.wait_event(c0)
+            s_b.wait_event(c0)
+            for _ in range(3):
+                with torch.cuda.stream(s_a):
+                    tmp.copy_(keep[0][0], non_blocking=True)       # host -> device
+                with torch.cuda.stream(s_b):
+                    keep[1][0].copy_(tmp2, non_blocking=True)      # device -> host (the step below packs it afresh)
+            stream.wait_stream(s_a)
+            stream.wait_stream(s_b)
+            c1.record(stream)
+            torch.cuda.synchronize(device)
+            link_rate["each_direction_when_both_run"] = 3 * blob_bytes / (c0.elapsed_time(c1) * 1e-3) / 1e9
+            del tmp2
         del tmp
         e2e_step()
         torch.cuda.synchronize(device)
