@@ -621,9 +621,11 @@ def test_gqa7b_full_digests_and_keys(gk):
     ctx.close()
 
 
-def test_layerwise_full_size_host_tier(gk):
+@pytest.mark.parametrize("host_tier", [True, False])
+def test_layerwise_full_size(gk, host_tier):
     """GQA-7B geometry cut into 8 groups of 4 layers, 3 blocks of 4,096 / 4,096 / 5,200 tokens,
-    saved to and loaded from pinned host memory group by group; one (block, group) damaged."""
+    saved and loaded group by group -- to and from pinned host memory, and on the device tier, where
+    the groups alternate between the context and its twin on two streams; one (block, group) damaged."""
     w = synth.GQA7B
     T = w.page_tokens
     gl, G = 4, w.layers // 4
@@ -642,8 +644,12 @@ def test_layerwise_full_size_host_tier(gk):
     jobs_s, jobs_d, spts, dpts, host, off = [], [], [], [], [], 0
     for n, P in zip(lens, pages):
         gb, _ = gk.gk_blob_size(g_geom, n)
-        hb = torch.empty(G * gb, dtype=torch.uint8, pin_memory=True)
-        hs = torch.empty(G * P, dtype=torch.int64, pin_memory=True)
+        if host_tier:
+            hb = torch.empty(G * gb, dtype=torch.uint8, pin_memory=True)
+            hs = torch.empty(G * P, dtype=torch.int64, pin_memory=True)
+        else:
+            hb = torch.empty(G * gb, dtype=torch.uint8, device="cuda")
+            hs = torch.empty(G * P, dtype=torch.int64, device="cuda")
         spts.append(sperm[off:off + P])
         dpts.append(dperm[off:off + P])
         host.append((hb, hs, gb))
@@ -651,7 +657,7 @@ def test_layerwise_full_size_host_tier(gk):
         jobs_d.append(gk.Job(hb, hs, torch.from_numpy(dpts[-1].copy()).cuda(), n))
         off += P
     status = torch.full((3,), 255, dtype=torch.uint8, device="cuda")
-    ctx.gk_pack_layerwise(G, src, jobs_s, status, host=True)
+    ctx.gk_pack_layerwise(G, src, jobs_s, status, host=host_tier)
     torch.cuda.synchronize()
     assert status.cpu().tolist() == [0, 0, 0]
     # sampled (block, group, page) records against the oracle
@@ -667,7 +673,7 @@ def test_layerwise_full_size_host_tier(gk):
         assert code == 0
         hb, hs, gb = host[j]
         lo = k * gb + oracle.record_offset(og_group, p)
-        assert np.array_equal(hb[lo:lo + blob.size].numpy(), blob), (j, k, p)
+        assert np.array_equal(hb[lo:lo + blob.size].cpu().numpy(), blob), (j, k, p)
         assert int(hs[k * P + p].item()) & 0xFFFFFFFFFFFFFFFF == int(sums[0])
     # damage block 1 inside group 5, then load
     host[1][0][5 * host[1][2] + 1_000_003] ^= 0x20
@@ -675,7 +681,8 @@ def test_layerwise_full_size_host_tier(gk):
     fb = torch.full((3,), -7, dtype=torch.int32, device="cuda")
     gm = torch.full((G, 3), 255, dtype=torch.uint8, device="cuda")
     seen = []
-    ctx.gk_restore_layerwise(G, jobs_d, dst, mask, fb, gm, lambda k, l0, nl, st: seen.append((k, l0, nl)), host=True)
+    ctx.gk_restore_layerwise(G, jobs_d, dst, mask, fb, gm, lambda k, l0, nl, st: seen.append((k, l0, nl)),
+                             host=host_tier)
     torch.cuda.synchronize()
     assert seen == [(k, k * gl, gl) for k in range(G)]
     want_gm = [[0, 0, 0] for _ in range(G)]
