@@ -437,10 +437,11 @@ int gk_get_stats(gk_ctx *ctx, gk_stats *out);
  * verifies nothing of the jobs k-1, k, ..., so that the commit waits of exactly
  * those jobs run into their limit and the time-out handling can be checked
  * without hanging or faulting the GPU), "quad" (page quartets: 0, the default:
- * packing and fused-restore launches whose page records are at most 128 KiB and
- * that have at least 8 pages per resident CTA (records of up to 256 KiB: 32 pages)
- * reduce one record per warp instead of one per CTA -- a quarter of the
- * per-thread checksum epilogues per byte; 1 = never;
+ * packing and verifying launches whose page records are at most 96 KiB and that
+ * have at least 3.5 pages per resident CTA (verifying launches also with records
+ * of up to 128 KiB from 12 pages per resident CTA on) reduce one record per warp
+ * instead of one per CTA -- a quarter of the per-thread checksum epilogues per
+ * byte; 1 = never;
  * 2 = in every such launch, whatever its size), and in the bounds-checked build only
  * "debug_extent_cut" (tests: cache extents are taken to be this many bytes smaller
  * than they are, so that a perfectly valid access to the last page is refused and

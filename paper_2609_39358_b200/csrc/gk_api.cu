@@ -279,9 +279,12 @@ uint64_t items_wanted(const gk_ctx *c, int occ) { return 2ull * (uint64_t)c->sm_
 // segment per page (the per-thread epilogue is paid once per page); small calls
 // cut pages into segments of at least two granules so that every SM gets work.
 //
-// Page quartets (`quad_for`: the call packs, or verifies -- alone or in a fused restore): records of at most
-// 256 KiB in a call with enough quartets for every resident CTA are reduced one per
-// WARP instead of one per CTA, four pages to a work item (see Tiling).
+// Page quartets (`quad_for`: the call packs, or verifies -- alone or in a fused restore): small records in a
+// call with enough quartets for every resident CTA are reduced one per WARP instead of one per CTA, four pages
+// to a work item (see Tiling).  Where they pay (B200, gqa7b geometry with 1, 2, 4 layers per record): 64 KiB
+// records from about 1,000 pages on (8 GiB: save 0.82 -> 1.03 of the copy peak, restore 0.88 -> 1.03; 512
+// pages: 35 us as single pages, 39 us as quartets); 128 KiB records only where the kernel verifies, and from
+// about 4,000 pages on (8 GiB: restore 1.01 -> 1.03, save 1.02 either way); 256 KiB records nowhere.
 enum QuadUse { kNoQuad = 0, kQuadPack = 1, kQuadRestore = 2 };
 
 bool quad_wanted(const gk_ctx *c, QuadUse quad_for, uint64_t total_pages, int occ)
@@ -289,12 +292,9 @@ bool quad_wanted(const gk_ctx *c, QuadUse quad_for, uint64_t total_pages, int oc
     if (quad_for == kNoQuad || c->quad_mode == 1u || c->seg_granules) return false;
     if (quad_for == kQuadPack && c->gd.S != 0u) return false;  // scale values are gathered by a whole warp per record
     if (c->quad_mode == 2u) return true;
-    // a quartet is four records long, and the last round of items is as long as the longest item: records of
-    // up to 128 KiB from two quartets per resident CTA on, records of up to 256 KiB from eight on (a 1 GiB
-    // call of 256 KiB records restores in 0.50 ms as single pages and in 0.52 ms as 1,024 quartets)
     const uint64_t resident = (uint64_t)c->sm_count * (uint64_t)occ;
-    if (c->gd.R <= (128u << 10)) return total_pages >= 8ull * resident;
-    return c->gd.R <= (256u << 10) && total_pages >= 32ull * resident;
+    if (c->gd.R <= (96u << 10)) return 2ull * total_pages >= 7ull * resident;
+    return quad_for == kQuadRestore && c->gd.R <= (128u << 10) && total_pages >= 12ull * resident;
 }
 
 uint32_t crc_items(const Tiling &tl, uint64_t pages)
